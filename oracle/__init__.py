@@ -1,0 +1,121 @@
+"""fp64 CPU oracle (TEST INFRASTRUCTURE ONLY).
+
+Slow, plain reference for the chunkwise delta-rule triangular inversion
+``A = (I + N)^{-1}`` with ``N = tril(diag(beta) K K^T * exp(g_i - g_j), -1)``
+(Eq. 3 with the GDN row of Table 1) and the WY factors
+``W = A diag(beta) K``, ``U = A diag(beta) V``.
+
+Only ``tests/``, ``__graft_entry__.smoke()`` and ``bench.py``'s CPU-baseline
+and ``--impl reference`` legs may import this package.  It shares no code with
+the CUDA library and the CUDA library never calls it.
+
+* ``build_A`` / ``wy``      -- the C implementation (``tri_inv_oracle.c``), plain
+  triple loops in double, OpenMP over independent chunks.
+* ``oracle.algorithms``     -- numpy fp64 restatements of the paper's inversion
+  algorithms (Algs. 2, 4, 5 and the 2x2 block formula), step by step.
+
+Parity pins (tests/test_oracle_pins.py): hand-worked 2x2/3x3/4x4 closed forms,
+the first-difference matrix, the 2^{i-j-1} growth example and binomial powers
+(Sec. 3.2), residuals to 1e-12, exact rational brute force, LAPACK, the
+|A_ij| <= 1 invariant (Sec. 2.2), and the sequential delta-rule recurrence.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "tri_inv_oracle.c")
+_LIB = os.path.join(_HERE, "libtri_inv_oracle.so")
+
+F32, BF16 = 0, 1
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (-O2, OpenMP) next to its source."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-std=c11", "-o", _LIB, _SRC, "-lm"]
+        )
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        vp, i32 = ctypes.c_void_p, ctypes.c_int
+        lib.tri_inv_oracle_build.restype = i32
+        lib.tri_inv_oracle_build.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, i32]
+        lib.tri_inv_oracle_wy.restype = i32
+        lib.tri_inv_oracle_wy.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, i32, i32]
+        lib.tri_inv_oracle_threads.restype = i32
+        lib.tri_inv_oracle_threads.argtypes = [i32]
+        _lib = lib
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _kv(a: np.ndarray):
+    """Storage array -> (contiguous array, dtype code).  uint16 means bf16 bit patterns."""
+    if a.dtype == np.float32:
+        return np.ascontiguousarray(a), F32
+    if a.dtype == np.uint16:
+        return np.ascontiguousarray(a), BF16
+    raise TypeError("K/V must be float32 or uint16 (bf16 bits), got %s" % a.dtype)
+
+
+def threads(n_threads: int = 0) -> int:
+    return int(_load().tri_inv_oracle_threads(int(n_threads)))
+
+
+def build_A(K, beta, g, C, cu_seqlens=None, n_threads=0, return_N=False):
+    """A = (I+N)^{-1} per chunk in fp64.
+
+    K [B,T,H,d_k] float32 or uint16 (bf16 bits); beta, g [B,T,H] float32.
+    Returns A [B,T,H,C] float64 (and N, same shape, when ``return_N``).
+    """
+    K, dt = _kv(K)
+    B, T, H, d_k = K.shape
+    beta = np.ascontiguousarray(beta, dtype=np.float32)
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    assert beta.shape == (B, T, H) and g.shape == (B, T, H)
+    A = np.zeros((B, T, H, C), dtype=np.float64)
+    N = np.zeros((B, T, H, C), dtype=np.float64) if return_N else None
+    cu = None if cu_seqlens is None else np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    n_seqs = 0 if cu is None else len(cu) - 1
+    rc = _load().tri_inv_oracle_build(_ptr(K), dt, _ptr(beta), _ptr(g), _ptr(A), _ptr(N),
+                                      B, T, H, d_k, C, _ptr(cu), n_seqs, int(n_threads))
+    if rc != 0:
+        raise ValueError("tri_inv_oracle_build: invalid arguments")
+    return (A, N) if return_N else A
+
+
+def wy(A, K, V, beta, C, cu_seqlens=None, n_threads=0):
+    """W = A diag(beta) K, U = A diag(beta) V in fp64 from a given A [B,T,H,C]."""
+    K, dt = _kv(K)
+    B, T, H, d_k = K.shape
+    d_v = 0
+    if V is not None:
+        V, dtv = _kv(V)
+        assert dtv == dt and V.shape[:3] == (B, T, H)
+        d_v = V.shape[3]
+    A = np.ascontiguousarray(A, dtype=np.float64)
+    assert A.shape == (B, T, H, C)
+    beta = np.ascontiguousarray(beta, dtype=np.float32)
+    W = np.zeros((B, T, H, d_k), dtype=np.float64)
+    U = np.zeros((B, T, H, d_v), dtype=np.float64) if V is not None else None
+    cu = None if cu_seqlens is None else np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    n_seqs = 0 if cu is None else len(cu) - 1
+    rc = _load().tri_inv_oracle_wy(_ptr(A), _ptr(K), _ptr(V), dt, _ptr(beta), _ptr(W), _ptr(U),
+                                   B, T, H, d_k, d_v, C, _ptr(cu), n_seqs, int(n_threads))
+    if rc != 0:
+        raise ValueError("tri_inv_oracle_wy: invalid arguments")
+    return W, U

@@ -1,0 +1,129 @@
+"""numpy fp64 restatements of the paper's inversion algorithms (TEST INFRASTRUCTURE ONLY).
+
+Each function inverts ``I + L`` for one strictly lower triangular ``L`` (n a
+power of two), taking the steps in the paper's order and notation.  They exist
+so the tests can check that the two schemes the CUDA library implements reach,
+in exact arithmetic, the same matrix as forward substitution; they are never
+used by the product.
+
+Sign convention: every routine here inverts ``I + L``; Eq. 3's ``I - phi .* L^-``
+is the same thing with ``L := -phi .* L^-``.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def forward_substitution(L: np.ndarray) -> np.ndarray:
+    """Column sweep in scalar form (Sec. 3.1): solve (I+L) X = I column by column."""
+    n = L.shape[0]
+    X = np.zeros((n, n))
+    for j in range(n):
+        X[j, j] = 1.0
+        for i in range(j + 1, n):
+            s = 0.0
+            for k in range(j, i):
+                s += L[i, k] * X[k, j]
+            X[i, j] = -s
+    return X
+
+
+def neumann_series(L: np.ndarray) -> np.ndarray:
+    """(I+L)^{-1} = I - L + L^2 - ... ; L^n = 0 so the sum is finite (Sec. 3.2)."""
+    n = L.shape[0]
+    X = np.eye(n)
+    P = np.eye(n)
+    for _ in range(1, n):
+        P = -(P @ L)
+        X = X + P
+    return X
+
+
+def mch(L: np.ndarray) -> np.ndarray:
+    """Alg. 5 (repeated squaring).  X <- I - L, Y <- L, then log2(n) - 1 rounds of
+    Y <- Y.Y ; X <- X + X.Y, which sums the series up to power n - 1."""
+    n = L.shape[0]
+    X = np.eye(n) - L
+    Y = L.copy()
+    rounds = max(int(np.log2(n)) - 1, 0)
+    for _ in range(rounds):
+        Y = Y @ Y
+        X = X + X @ Y
+    return X
+
+
+def product_form(L: np.ndarray) -> np.ndarray:
+    """prod_{k=0}^{log2(n)-1} (I + (-L)^{2^k}) -- the same series factorised."""
+    n = L.shape[0]
+    X = np.eye(n)
+    P = -L
+    for _ in range(max(int(np.log2(n)), 1)):
+        X = X @ (np.eye(n) + P)
+        P = P @ P
+    return X
+
+
+def _diag_blocks(X: np.ndarray, b: int, parity: int) -> np.ndarray:
+    n = X.shape[0]
+    D = np.zeros_like(X)
+    for t in range(n // b):
+        if t % 2 == parity:
+            s = slice(t * b, (t + 1) * b)
+            D[s, s] = X[s, s]
+    return D
+
+
+def mbh(L: np.ndarray, X0: np.ndarray | None = None, b0: int = 1) -> np.ndarray:
+    """Alg. 4 (unrolled Bunch-Hopcroft): for b = b0, 2 b0, ... < n:
+    X <- D_e + D_o - D_o . L . D_e with D_e / D_o the 1st,3rd,.. / 2nd,4th,.. b x b
+    diagonal blocks of X (Lemma C.1 stops at b = n/2; the b = n step is a no-op)."""
+    n = L.shape[0]
+    X = np.eye(n) if X0 is None else X0.copy()
+    b = b0
+    while b < n:
+        De = _diag_blocks(X, b, 0)
+        Do = _diag_blocks(X, b, 1)
+        X = De + Do - Do @ L @ De
+        b *= 2
+    return X
+
+
+def mxr(L: np.ndarray, b0: int = 16) -> np.ndarray:
+    """Alg. 2 with r = 0: Alg. 5 on the b0 x b0 diagonal blocks, then Alg. 4 from b0."""
+    n = L.shape[0]
+    b0 = min(b0, n)
+    Y = np.zeros_like(L)
+    for t in range(n // b0):
+        s = slice(t * b0, (t + 1) * b0)
+        Y[s, s] = mch(L[s, s])
+    return mbh(L, Y, b0)
+
+
+def block_recursive(L: np.ndarray, leaf: int = 16) -> np.ndarray:
+    """The 2x2 block identity of Sec. 3.3 written for a lower triangular matrix:
+    inv([[M11, 0], [N21, M22]]) = [[X11, 0], [-X22 N21 X11, X22]], recursing down
+    to ``leaf`` x ``leaf`` blocks that are inverted by forward substitution."""
+    n = L.shape[0]
+    if n <= leaf:
+        return forward_substitution(L)
+    h = n // 2
+    X11 = block_recursive(L[:h, :h], leaf)
+    X22 = block_recursive(L[h:, h:], leaf)
+    X = np.zeros((n, n))
+    X[:h, :h] = X11
+    X[h:, h:] = X22
+    X[h:, :h] = -(X22 @ L[h:, :h] @ X11)
+    return X
+
+
+def chunk_N(K: np.ndarray, beta: np.ndarray, g: np.ndarray) -> np.ndarray:
+    """One chunk's N from its keys [C,d], betas [C] and cumulative log-decays [C]."""
+    K = K.astype(np.float64)
+    beta = beta.astype(np.float64)
+    g = g.astype(np.float64)
+    C = K.shape[0]
+    N = np.zeros((C, C))
+    for i in range(C):
+        for j in range(i):
+            N[i, j] = beta[i] * float(K[i] @ K[j]) * np.exp(g[i] - g[j])
+    return N

@@ -1,0 +1,202 @@
+/*
+ * fp64 CPU oracle for the chunkwise delta-rule triangular inversion.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain reference that the
+ * tests, the smoke check and the bench's cpu_baseline leg compare the CUDA
+ * library against.  It shares no code with the CUDA path and the product
+ * never calls it.
+ *
+ * What it computes, per (sequence, head, chunk) with r <= C real rows:
+ *
+ *   S_ij = k_i . k_j                                   (Gram entries, j < i)
+ *   N_ij = beta_i * S_ij * exp(g_i - g_j)   for j < i  (Eq. 3 with the GDN row
+ *          0 otherwise                                   of Table 1; the decay
+ *                                                        matrix is exp(g_i-g_j))
+ *   A    = (I + N)^{-1}   by forward substitution      (Sec. 3.1, column sweep
+ *                                                        in its scalar form)
+ *   W    = A diag(beta) K,   U = A diag(beta) V        (WY factors)
+ *
+ * Inputs arrive in their storage type (fp32 or bf16 bit patterns) and are
+ * widened exactly to double; every sum runs in double in index order.  There
+ * is no blocking, tiling or reordering: each loop is the formula.
+ *
+ * Layouts (all contiguous, row-major):
+ *   K [B,T,H,d_k], V [B,T,H,d_v], beta and g [B,T,H] (g is the within-chunk
+ *   cumulative log-decay), A and N [B,T,H,C] (row = token, C columns of its
+ *   chunk), W [B,T,H,d_k], U [B,T,H,d_v].
+ * Dense mode: cu_seqlens == NULL, B sequences of T tokens.  Ragged mode:
+ * B == 1, T == total tokens, sequence s covers [cu_seqlens[s], cu_seqlens[s+1]).
+ * Chunks restart at every sequence start; a short last chunk is the leading
+ * r x r block of an identity-padded C x C problem, and only its r rows are
+ * written (columns >= r of those rows are 0).
+ *
+ * OpenMP runs independent chunks on separate threads; that is the only
+ * parallelism.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+
+static double widen(const void* base, int dtype, size_t idx) {
+  if (dtype == ORACLE_F32) return (double)((const float*)base)[idx];
+  uint32_t bits = ((uint32_t)((const uint16_t*)base)[idx]) << 16; /* bf16 = top half of fp32 */
+  float f;
+  memcpy(&f, &bits, sizeof f);
+  return (double)f;
+}
+
+typedef struct { int64_t tok0; int rows; } chunk_t;
+
+/* List every chunk as (first token, real rows).  Returns count, or -1 on a bad cu_seqlens. */
+static int64_t list_chunks(int B, int T, int C, const int32_t* cu, int n_seqs, chunk_t** out) {
+  int64_t n = 0, cap = 0;
+  int nseq = cu ? n_seqs : B;
+  for (int pass = 0; pass < 2; ++pass) {
+    n = 0;
+    for (int s = 0; s < nseq; ++s) {
+      int64_t beg = cu ? cu[s] : (int64_t)s * T;
+      int64_t end = cu ? cu[s + 1] : (int64_t)(s + 1) * T;
+      if (end < beg) return -1;
+      for (int64_t t = beg; t < end; t += C) {
+        if (pass) { (*out)[n].tok0 = t; (*out)[n].rows = (int)((end - t) < C ? (end - t) : C); }
+        ++n;
+      }
+    }
+    if (!pass) { cap = n; *out = (chunk_t*)malloc(sizeof(chunk_t) * (size_t)(cap ? cap : 1)); if (!*out) return -1; }
+  }
+  return n;
+}
+
+/*
+ * A = (I+N)^{-1} for every chunk; N_out (nullable) receives N itself.
+ * All pointers are HOST pointers.  Returns 0, or 1 on invalid arguments.
+ */
+int tri_inv_oracle_build(const void* K, int kv_dtype, const float* beta, const float* g,
+                         double* A, double* N_out,
+                         int B, int T, int H, int d_k, int C,
+                         const int32_t* cu_seqlens, int n_seqs, int n_threads) {
+  if (!K || !beta || !g || !A || B < 1 || T < 0 || H < 1 || d_k < 1 || C < 1) return 1;
+  if (cu_seqlens && (B != 1 || n_seqs < 0 || cu_seqlens[0] != 0 || cu_seqlens[n_seqs] != T)) return 1;
+  chunk_t* ch = NULL;
+  int64_t n_chunks = list_chunks(B, T, C, cu_seqlens, n_seqs, &ch);
+  if (n_chunks < 0) { free(ch); return 1; }
+#ifdef _OPENMP
+  if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+  int64_t total = n_chunks * H;
+#pragma omp parallel
+  {
+    double* N = (double*)malloc(sizeof(double) * (size_t)C * C);
+    double* X = (double*)malloc(sizeof(double) * (size_t)C * C);
+#pragma omp for schedule(static)
+    for (int64_t w = 0; w < total; ++w) {
+      int64_t c = w / H;
+      int h = (int)(w % H);
+      int64_t t0 = ch[c].tok0;
+      int r = ch[c].rows;
+      /* N: strictly lower, row-scaled by beta, decayed by exp(g_i - g_j) */
+      for (int i = 0; i < C; ++i)
+        for (int j = 0; j < C; ++j) N[i * C + j] = 0.0;
+      for (int i = 0; i < r; ++i) {
+        size_t bi = (size_t)(t0 + i) * H + h;
+        for (int j = 0; j < i; ++j) {
+          size_t bj = (size_t)(t0 + j) * H + h;
+          double s = 0.0;
+          for (int k = 0; k < d_k; ++k)
+            s += widen(K, kv_dtype, bi * d_k + k) * widen(K, kv_dtype, bj * d_k + k);
+          N[i * C + j] = (double)beta[bi] * s * exp((double)g[bi] - (double)g[bj]);
+        }
+      }
+      /* forward substitution on (I+N) X = I, one column at a time */
+      for (int i = 0; i < C; ++i)
+        for (int j = 0; j < C; ++j) X[i * C + j] = 0.0;
+      for (int j = 0; j < r; ++j) {
+        X[j * C + j] = 1.0;
+        for (int i = j + 1; i < r; ++i) {
+          double s = 0.0;
+          for (int k = j; k < i; ++k) s += N[i * C + k] * X[k * C + j];
+          X[i * C + j] = -s;
+        }
+      }
+      for (int i = 0; i < r; ++i) {
+        size_t row = ((size_t)(t0 + i) * H + h) * C;
+        for (int j = 0; j < C; ++j) {
+          A[row + j] = X[i * C + j];
+          if (N_out) N_out[row + j] = N[i * C + j];
+        }
+      }
+    }
+    free(N);
+    free(X);
+  }
+  free(ch);
+  return 0;
+}
+
+/*
+ * W = A diag(beta) K and U = A diag(beta) V from a given A (double, layout
+ * [B,T,H,C]).  V, U may both be NULL to skip U.  HOST pointers.
+ */
+int tri_inv_oracle_wy(const double* A, const void* K, const void* V, int kv_dtype, const float* beta,
+                      double* W, double* U,
+                      int B, int T, int H, int d_k, int d_v, int C,
+                      const int32_t* cu_seqlens, int n_seqs, int n_threads) {
+  if (!A || !K || !beta || !W || B < 1 || T < 0 || H < 1 || d_k < 1 || C < 1) return 1;
+  if ((V == NULL) != (U == NULL)) return 1;
+  if (V && d_v < 1) return 1;
+  if (cu_seqlens && (B != 1 || n_seqs < 0 || cu_seqlens[0] != 0 || cu_seqlens[n_seqs] != T)) return 1;
+  chunk_t* ch = NULL;
+  int64_t n_chunks = list_chunks(B, T, C, cu_seqlens, n_seqs, &ch);
+  if (n_chunks < 0) { free(ch); return 1; }
+#ifdef _OPENMP
+  if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+  int64_t total = n_chunks * H;
+#pragma omp parallel for schedule(static)
+  for (int64_t w = 0; w < total; ++w) {
+    int64_t c = w / H;
+    int h = (int)(w % H);
+    int64_t t0 = ch[c].tok0;
+    int r = ch[c].rows;
+    for (int i = 0; i < r; ++i) {
+      size_t ri = (size_t)(t0 + i) * H + h;
+      for (int k = 0; k < d_k; ++k) {
+        double s = 0.0;
+        for (int j = 0; j <= i; ++j) {
+          size_t rj = (size_t)(t0 + j) * H + h;
+          s += A[ri * C + j] * (double)beta[rj] * widen(K, kv_dtype, rj * d_k + k);
+        }
+        W[ri * d_k + k] = s;
+      }
+      if (V) {
+        for (int k = 0; k < d_v; ++k) {
+          double s = 0.0;
+          for (int j = 0; j <= i; ++j) {
+            size_t rj = (size_t)(t0 + j) * H + h;
+            s += A[ri * C + j] * (double)beta[rj] * widen(V, kv_dtype, rj * d_v + k);
+          }
+          U[ri * d_v + k] = s;
+        }
+      }
+    }
+  }
+  free(ch);
+  return 0;
+}
+
+/* Threads an OpenMP region would use for a given request (0 = runtime default). */
+int tri_inv_oracle_threads(int n_threads) {
+#ifdef _OPENMP
+  if (n_threads > 0) return n_threads;
+  return omp_get_max_threads();
+#else
+  (void)n_threads;
+  return 1;
+#endif
+}

@@ -1,0 +1,308 @@
+"""Pins for the fp64 oracle: it is checked against things other than itself.
+
+Closed forms worked by hand, the paper's own examples (Sec. 3.2), exact
+rational arithmetic, LAPACK, the defining identities, the |A_ij| <= 1
+invariant of DeltaNet matrices (Sec. 2.2) and the sequential delta-rule
+recurrence the chunk form was derived from.
+"""
+import os
+from fractions import Fraction
+from math import comb
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import algorithms as alg
+from paper_2605_21325_b200 import workloads as wl
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def load(name):
+    return np.loadtxt(os.path.join(GOLD, name), comments="#")
+
+
+def keys_for_integer_N(N):
+    """Integer keys k_i (d = n) with k_i . k_j = N_ij for j < i: row i solves a unit
+    lower-triangular integer system against the earlier rows, so it stays integral."""
+    n = N.shape[0]
+    K = np.zeros((n, n))
+    for i in range(n):
+        K[i, i] = 1.0
+        for j in range(i):
+            K[i, j] = N[i, j] - sum(K[i, m] * K[j, m] for m in range(j))
+    return K
+
+
+def run_single(K, beta=None, g=None, C=None, dtype=np.float32):
+    """Oracle on one sequence, one head; returns (A, N) as [T, C] arrays."""
+    T, d = K.shape
+    C = T if C is None else C
+    beta = np.ones(T) if beta is None else beta
+    g = np.zeros(T) if g is None else g
+    A, N = oracle.build_A(K.reshape(1, T, 1, d).astype(dtype), np.asarray(beta, np.float32).reshape(1, T, 1),
+                          np.asarray(g, np.float32).reshape(1, T, 1), C, return_N=True)
+    return A[0, :, 0, :], N[0, :, 0, :]
+
+
+# ---------------------------------------------------------------- closed forms (hand-worked)
+
+def test_closed_form_2x2_and_3x3():
+    # k0=(1,0), k1=(1,1): k1.k0 = 1; beta1 = 0.5; g1-g0 = -ln 2  =>  n21 = 0.25, A21 = -0.25
+    K = np.array([[1.0, 0.0], [1.0, 1.0]])
+    A, N = run_single(K, beta=[1.0, 0.5], g=[0.0, -np.log(2.0)])
+    assert abs(N[1, 0] - 0.25) < 1e-7          # g is stored in fp32
+    assert A[0, 0] == 1.0 and A[1, 1] == 1.0 and A[0, 1] == 0.0
+    assert abs(A[1, 0] + 0.25) < 1e-7
+    # 3x3 with integer N: n21=2, n31=-1, n32=3  =>  A21=-2, A32=-3, A31 = n32 n21 - n31 = 7
+    N3 = np.array([[0, 0, 0], [2, 0, 0], [-1, 3, 0]], float)
+    A, N = run_single(keys_for_integer_N(N3))
+    assert np.array_equal(N, N3)
+    assert np.array_equal(A, np.array([[1, 0, 0], [-2, 1, 0], [7, -3, 1]], float))
+
+
+def test_closed_form_4x4_golden():
+    G = load("closed_form_4x4.txt")
+    N4, A4 = G[:4], G[4:]
+    A, N = run_single(keys_for_integer_N(N4))
+    assert np.array_equal(N, N4)
+    assert np.array_equal(A, A4)
+
+
+def test_first_difference_matrix():
+    # all keys equal one unit vector, beta = 1, g = 0: N = ones strictly lower
+    K = np.zeros((5, 3)); K[:, 1] = 1.0
+    A, N = run_single(K)
+    assert np.array_equal(N, np.tril(np.ones((5, 5)), -1))
+    assert np.array_equal(A, load("first_difference_n5.txt"))
+    inp = wl.first_difference_case(2, 128, 2, 16, 64, wl.BF16)
+    A = oracle.build_A(inp.K, inp.beta, inp.g, 64)
+    exp = np.eye(64) - np.eye(64, k=-1)
+    for b in range(2):
+        for c in range(2):
+            assert np.array_equal(A[b, c * 64:(c + 1) * 64, 1, :], exp)
+
+
+def test_growth_example_powers_of_two():
+    # Sec. 3.2: N = -(ones strictly lower)  =>  A_ij = sum_k binom(i-j-1, k-1) = 2^(i-j-1)
+    K = np.zeros((6, 2)); K[:, 0] = 1.0
+    A, N = run_single(K, beta=-np.ones(6))
+    assert np.array_equal(A, load("growth_example_n6.txt"))
+    n = 128
+    K = np.zeros((n, 2)); K[:, 0] = 1.0
+    A, _ = run_single(K, beta=-np.ones(n))
+    i, j = np.tril_indices(n, -1)
+    assert np.array_equal(A[i, j], 2.0 ** (i - j - 1))      # exact in fp64 up to 2^126
+
+
+def test_series_terms_are_binomials():
+    # pins the series/product code used below, against the paper's closed form
+    n = 6
+    Lm = np.tril(np.ones((n, n)), -1)
+    assert np.array_equal(np.linalg.matrix_power(Lm, 3), load("ones_power3_n6.txt"))
+    n = 16
+    Lm = np.tril(np.ones((n, n)), -1)
+    for k in (1, 2, 5, 8):
+        P = np.linalg.matrix_power(Lm, k)
+        for i in range(n):
+            for j in range(n):
+                expect = comb(i - j - 1, k - 1) if i > j else 0
+                assert P[i, j] == expect
+    # repeated squaring on the same matrix (negated) gives the growth example
+    X = alg.mch(-Lm)
+    i, j = np.tril_indices(n, -1)
+    assert np.array_equal(X[i, j], 2.0 ** (i - j - 1))
+
+
+# ---------------------------------------------------------------- exact rational brute force
+
+def exact_inverse(N):
+    n = len(N)
+    M = [[Fraction(int(i == j)) + Fraction(N[i][j]) for j in range(n)] for i in range(n)]
+    X = [[Fraction(int(i == j)) for j in range(n)] for i in range(n)]
+    for i in range(n):                      # Gauss-Jordan, no pivoting needed (unit diagonal)
+        for r in range(n):
+            if r != i and M[r][i] != 0:
+                f = M[r][i]
+                M[r] = [a - f * b for a, b in zip(M[r], M[i])]
+                X[r] = [a - f * b for a, b in zip(X[r], X[i])]
+    return X
+
+
+@pytest.mark.parametrize("n,seed", [(2, 0), (3, 1), (5, 2), (8, 3)])
+def test_exact_rational_brute_force(n, seed):
+    rng = np.random.default_rng(seed)
+    K = rng.integers(-2, 3, size=(n, 4)).astype(np.float64)
+    beta = rng.choice([0.5, 1.0, -1.0, 2.0], size=n)
+    A, N = run_single(K, beta=beta)
+    S = K @ K.T
+    Nx = [[Fraction(beta[i]) * Fraction(int(S[i, j])) if j < i else Fraction(0) for j in range(n)] for i in range(n)]
+    X = exact_inverse(Nx)
+    for i in range(n):
+        for j in range(n):
+            assert float(Nx[i][j]) == N[i, j]
+            ref = float(X[i][j])
+            assert abs(A[i, j] - ref) <= 1e-12 * max(1.0, abs(ref))
+
+
+# ---------------------------------------------------------------- identities on model-like inputs
+
+@pytest.fixture(scope="module")
+def small_gdn():
+    inp = wl.make("t", 2, 192, 3, 32, 48, 64, wl.BF16, seed=7)
+    A, N = oracle.build_A(inp.K, inp.beta, inp.g, inp.C, return_N=True)
+    W, U = oracle.wy(A, inp.K, inp.V, inp.beta, inp.C)
+    return inp, A, N, W, U
+
+
+def chunks_of(inp):
+    for t0, r in inp.chunk_list():
+        b, t = divmod(t0, inp.T)
+        for h in range(inp.H):
+            yield b, t, h, r
+
+
+def test_residual_unit_diagonal_zero_upper(small_gdn):
+    inp, A, N, _, _ = small_gdn
+    C = inp.C
+    for b, t, h, r in chunks_of(inp):
+        a, n = A[b, t:t + r, h, :r], N[b, t:t + r, h, :r]
+        I = np.eye(r)
+        assert np.abs((I + n) @ a - I).max() <= 1e-12
+        assert np.abs(a @ (I + n) - I).max() <= 1e-12
+        assert np.array_equal(np.diag(a), np.ones(r))
+        iu = np.triu_indices(r, 1)
+        assert not a[iu].any() and not np.signbit(a[iu]).any()
+        assert not n[np.triu_indices(r, 0)].any()
+
+
+def test_N_matches_definition_and_lapack(small_gdn):
+    inp, A, N, _, _ = small_gdn
+    Kf = inp.kv_as_f32("K").astype(np.float64)
+    for b, t, h, r in chunks_of(inp):
+        n = alg.chunk_N(Kf[b, t:t + r, h], inp.beta[b, t:t + r, h], inp.g[b, t:t + r, h])
+        assert np.abs(n - N[b, t:t + r, h, :r]).max() <= 1e-15
+        ref = np.linalg.inv(np.eye(r) + n)
+        assert np.abs(ref - A[b, t:t + r, h, :r]).max() <= 1e-12
+
+
+def test_entries_bounded_by_one_and_condition_number(small_gdn):
+    # Sec. 2.2: inverse of a DeltaNet matrix has entries in [-1,1]; kappa_2 <= n^2 (Cor. 2.1).
+    # bf16 storage rounding moves |k| off 1 by <= 2^-9, so allow that slack.
+    inp, A, N, _, _ = small_gdn
+    assert np.abs(A).max() <= 1.0 + 1e-2
+    for b, t, h, r in chunks_of(inp):
+        assert np.linalg.cond(np.eye(r) + N[b, t:t + r, h, :r], 2) <= r * r
+    for seed in range(3):
+        x = wl.make("u", 1, 128, 2, 128, 128, 128, wl.F32, seed=100 + seed)
+        x.g[:] = 0                                      # ungated DeltaNet, unit keys, beta in (0,1)
+        a = oracle.build_A(x.K, x.beta, x.g, 128)
+        assert np.abs(a).max() <= 1.0 + 1e-5
+
+
+def test_wy_solve_identities(small_gdn):
+    inp, A, N, W, U = small_gdn
+    Kf = inp.kv_as_f32("K").astype(np.float64)
+    Vf = inp.kv_as_f32("V").astype(np.float64)
+    for b, t, h, r in chunks_of(inp):
+        n = N[b, t:t + r, h, :r]
+        bt = inp.beta[b, t:t + r, h].astype(np.float64)[:, None]
+        assert np.abs((np.eye(r) + n) @ W[b, t:t + r, h] - bt * Kf[b, t:t + r, h]).max() <= 1e-12
+        assert np.abs((np.eye(r) + n) @ U[b, t:t + r, h] - bt * Vf[b, t:t + r, h]).max() <= 1e-12
+        # row recurrence w_i = beta_i k_i - sum_{j<i} N_ij w_j
+        w = np.zeros((r, inp.d_k))
+        for i in range(r):
+            w[i] = bt[i] * Kf[b, t + i, h] - n[i, :i] @ w[:i]
+        assert np.abs(w - W[b, t:t + r, h]).max() <= 1e-12
+
+
+def test_delta_rule_recurrence(small_gdn):
+    """Sequential gated delta rule, token by token (O(C d^2), no matrix inverse):
+         S_t = a_t S_{t-1} (I - beta_t k_t k_t^T) + beta_t v_t k_t^T,   a_t = exp(g_t - g_{t-1}), S_0 = 0
+       equals sum_t exp(g_last - g_t) u_t k_t^T with U from the oracle; and, without decay,
+       prod_t (I - beta_t k_t k_t^T) = I - W^T K.  This ties N's conventions (beta on rows,
+       exp(g_i - g_j), + sign) to the model the chunk form came from."""
+    inp, A, N, W, U = small_gdn
+    Kf = inp.kv_as_f32("K").astype(np.float64)
+    Vf = inp.kv_as_f32("V").astype(np.float64)
+    for b, t, h, r in list(chunks_of(inp))[:6]:
+        k, v = Kf[b, t:t + r, h], Vf[b, t:t + r, h]
+        bt = inp.beta[b, t:t + r, h].astype(np.float64)
+        g = inp.g[b, t:t + r, h].astype(np.float64)
+        S = np.zeros((inp.d_v, inp.d_k))
+        P = np.eye(inp.d_k)
+        for i in range(r):
+            a = np.exp(g[i] - (g[i - 1] if i else g[0]))     # first token's own decay cancels from S_0 = 0
+            S = a * (S - bt[i] * np.outer(S @ k[i], k[i])) + bt[i] * np.outer(v[i], k[i])
+            P = a * (P - bt[i] * np.outer(P @ k[i], k[i]))
+        u = U[b, t:t + r, h]
+        S_chunk = sum(np.exp(g[r - 1] - g[i]) * np.outer(u[i], k[i]) for i in range(r))
+        assert np.abs(S - S_chunk).max() <= 1e-12
+        # decayed transition: P = e^{g_last - g_0}... written with omega = A diag(beta e^{g}) K
+        a_mat = A[b, t:t + r, h, :r]
+        omega = a_mat @ ((bt * np.exp(g - g[0]))[:, None] * k)
+        P_chunk = np.exp(g[r - 1] - g[0]) * np.eye(inp.d_k) - sum(np.exp(g[r - 1] - g[i]) * np.outer(omega[i], k[i]) for i in range(r))
+        assert np.abs(P - P_chunk).max() <= 1e-12
+    # ungated: ordered product of Householder-like factors equals I - W^T K
+    x = wl.make("v", 1, 64, 1, 16, 16, 64, wl.F32, seed=11)
+    x.g[:] = 0
+    a = oracle.build_A(x.K, x.beta, x.g, 64)
+    w, _ = oracle.wy(a, x.K, x.V, x.beta, 64)
+    k = x.K[0, :, 0].astype(np.float64)
+    P = np.eye(16)
+    for i in range(64):
+        P = P - float(x.beta[0, i, 0]) * np.outer(P @ k[i], k[i])
+    assert np.abs(P - (np.eye(16) - w[0, :, 0].T @ k)).max() <= 1e-12
+
+
+# ---------------------------------------------------------------- the paper's algorithms reach the same matrix
+
+@pytest.mark.parametrize("n", [2, 4, 8, 16, 64, 128])
+def test_algorithms_agree_with_substitution(n):
+    x = wl.make("w", 1, n, 1, 128, 8, n, wl.F32, seed=20 + n)
+    A, N = oracle.build_A(x.K, x.beta, x.g, n, return_N=True)
+    a, L = A[0, :, 0], N[0, :, 0]
+    assert np.abs(alg.forward_substitution(L) - a).max() <= 1e-14
+    if n <= 16:
+        assert np.abs(alg.neumann_series(L) - a).max() <= 1e-13
+    assert np.abs(alg.mch(L) - a).max() <= 1e-13           # Alg. 5
+    assert np.abs(alg.product_form(L) - a).max() <= 1e-13  # factorised series
+    assert np.abs(alg.mbh(L) - a).max() <= 1e-13           # Alg. 4 from b0 = 1
+    assert np.abs(alg.mxr(L, 16) - a).max() <= 1e-13       # Alg. 2
+    assert np.abs(alg.block_recursive(L, 16) - a).max() <= 1e-13
+    if n >= 4:
+        h = n // 2                                         # 2x2 block formula from two half-size oracle inverses
+        X11 = oracle.build_A(x.K[:, :h], x.beta[:, :h], x.g[:, :h], h)[0, :, 0]
+        X22 = oracle.build_A(x.K[:, h:], x.beta[:, h:], x.g[:, h:], h)[0, :, 0]
+        assert np.abs(a[:h, :h] - X11).max() <= 1e-14 and np.abs(a[h:, h:] - X22).max() <= 1e-14
+        assert np.abs(a[h:, :h] + X22 @ L[h:, :h] @ X11).max() <= 1e-13
+
+
+# ---------------------------------------------------------------- layout: ragged packing, partial chunks, heads
+
+def test_ragged_and_partial_chunks_match_per_sequence_runs():
+    rng = np.random.default_rng(5)
+    cu = np.array([0, 1, 70, 134, 200], np.int32)          # lengths 1, 69, 64, 66
+    x = wl.make("r", 1, int(cu[-1]), 2, 16, 8, 64, wl.BF16, seed=31, kind="stress", cu_seqlens=cu, rng=rng)
+    x.g[:] = (rng.standard_normal(x.g.shape) * 0.1).astype(np.float32)
+    A = oracle.build_A(x.K, x.beta, x.g, 64, cu_seqlens=cu)
+    W, U = oracle.wy(A, x.K, x.V, x.beta, 64, cu_seqlens=cu)
+    for s in range(4):
+        b, e = int(cu[s]), int(cu[s + 1])
+        As = oracle.build_A(x.K[:, b:e], x.beta[:, b:e], x.g[:, b:e], 64)
+        Ws, Us = oracle.wy(As, x.K[:, b:e], x.V[:, b:e], x.beta[:, b:e], 64)
+        assert np.array_equal(As, A[:, b:e]) and np.array_equal(Ws, W[:, b:e]) and np.array_equal(Us, U[:, b:e])
+    # the 69-token sequence: second chunk has 5 real rows; columns >= 5 of those rows are zero
+    assert not A[0, 65:70, :, 5:].any()
+    assert np.array_equal(A[0, 65, 0, :1], [1.0])
+    # heads are independent: permuting heads permutes outputs
+    A2 = oracle.build_A(x.K[:, :, ::-1], x.beta[:, :, ::-1], x.g[:, :, ::-1], 64, cu_seqlens=cu)
+    assert np.array_equal(A2[:, :, ::-1], A)
+
+
+def test_threads_do_not_change_results():
+    x = wl.config(2, shrink=32)
+    a1 = oracle.build_A(x.K, x.beta, x.g, x.C, n_threads=1)
+    a4 = oracle.build_A(x.K, x.beta, x.g, x.C, n_threads=4)
+    assert np.array_equal(a1, a4)
