@@ -1,0 +1,153 @@
+/*
+ * tri_inv.h -- C ABI of the B200 (sm_100a) chunkwise delta-rule triangular inversion.
+ *
+ * For every chunk of C tokens of every (sequence, head) the library forms the
+ * strictly lower triangular matrix
+ *
+ *     N_ij = beta_i * (k_i . k_j) * exp(g_i - g_j)   (i > j),   0 otherwise
+ *
+ * (Eq. 3 of the paper with the DeltaNet/GDN rows of Table 1: phi = diag(beta) K K^T
+ * masked by the strictly-lower ones matrix and scaled by the decay matrix
+ * exp(g_i - g_j); the matrix inverted is I + N), computes
+ *
+ *     A = (I + N)^{-1}
+ *
+ * by one of the direct schemes of Sec. 3 and optionally applies it:
+ *
+ *     W = A diag(beta) K,      U = A diag(beta) V          (WY factors).
+ *
+ * Everything here is plain C: pointers and sizes, no C++ or torch types.
+ * All tensor pointers are DEVICE pointers unless stated otherwise; the caller
+ * allocates and owns every buffer.  Calls are asynchronous on the given CUDA
+ * stream (a cudaStream_t passed as void*; NULL = the legacy default stream)
+ * and never synchronise the device.  No function throws, aborts or traps;
+ * every function returns a TRI_INV_* status.  There is no CPU fallback: on a
+ * machine without a usable GPU the compute calls return TRI_INV_ERR_CUDA.
+ *
+ * Tensor layouts (contiguous, row-major, flat token index t in [0, B*T)):
+ *   K     [B, T, H, d_k]   kv_dtype (fp32, or bf16 as 16-bit patterns)
+ *   V     [B, T, H, d_v]   kv_dtype
+ *   beta  [B, T, H]        fp32
+ *   g     [B, T, H]        fp32, cumulative log-decay within each chunk (only
+ *                          differences inside a chunk are used)
+ *   A     [B, T, H, C]     fp32; row = token, column j = j-th token of its chunk.
+ *                          Upper triangle is +0.0 and the diagonal 1.0f, bit-exact.
+ *   W     [B, T, H, d_k]   kv_dtype (round-to-nearest-even from fp32 accumulators)
+ *   U     [B, T, H, d_v]   kv_dtype
+ * Base pointers must be 16-byte aligned.
+ *
+ * Chunking: dense mode (cu_seqlens == NULL) has B sequences of T tokens; ragged
+ * mode has B == 1, T == total tokens and sequence s = [cu_seqlens[s], cu_seqlens[s+1]).
+ * Chunks restart at each sequence start.  A short last chunk with r < C tokens
+ * is the leading r x r block of an identity-padded problem: only its r rows
+ * are written, with columns >= r of A equal to +0.0.  Rows that belong to no
+ * token are never read as data nor written.
+ */
+#ifndef TRI_INV_H_
+#define TRI_INV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------- */
+enum {
+  TRI_INV_OK = 0,
+  TRI_INV_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, bad size, bad cu_seqlens */
+  TRI_INV_ERR_UNSUPPORTED = 2,   /* a valid request this build has no kernel for */
+  TRI_INV_ERR_CUDA = 3,          /* a CUDA runtime call or the launch failed */
+  TRI_INV_ERR_DEVICE_TIMEOUT = 4 /* a bounded device-side wait expired (see tri_inv_last_device_status) */
+};
+
+/* ---- storage type of K, V, W, U ------------------------------------------ */
+enum { TRI_INV_F32 = 0, TRI_INV_BF16 = 1 };
+
+/* ---- inversion scheme ("method" argument) -------------------------------- */
+enum {
+  /* 2x2 block recursion A = [[A11, 0], [-A22 N21 A11, A22]] from 16x16 leaves
+   * (Sec. 3.3, Eq. for the block inverse written for a lower-triangular matrix;
+   * the unrolled form is Alg. 4).  Leaves by forward substitution (Sec. 3.1). */
+  TRI_INV_BLOCK_RECURSIVE = 0,
+  /* Repeated squaring of the nilpotent series (Alg. 5 / Sec. 3.2):
+   * X <- I - N, Y <- N, then log2(C) - 1 rounds of Y <- Y.Y, X <- X + X.Y,
+   * i.e. prod_k (I + (-N)^(2^k)).  Exact in exact arithmetic, not stable. */
+  TRI_INV_PRODUCT_SERIES = 1,
+  TRI_INV_METHOD_MASK = 0xff,
+  /* flag, block-recursive only: invert the 16x16 leaves with the product series
+   * instead of substitution -- the mixed recursion of Alg. 2 (r = 0). */
+  TRI_INV_LEAF_SERIES = 0x100,
+  /* flag: run the plain fp32 CUDA-core kernel even where a tensor-core kernel
+   * exists (same results up to rounding; for cross-checks and odd shapes). */
+  TRI_INV_FORCE_SIMT = 0x10000
+};
+
+/* ---- problem descriptor --------------------------------------------------- */
+typedef struct tri_inv_desc {
+  int32_t B;        /* sequences in dense mode; must be 1 in ragged mode */
+  int32_t T;        /* tokens per sequence (dense) or total tokens (ragged) */
+  int32_t H;        /* heads */
+  int32_t d_k;      /* key dimension   (multiple of 8) */
+  int32_t d_v;      /* value dimension (multiple of 8); ignored by tri_inv_build */
+  int32_t C;        /* chunk size: 16, 32, 64 or 128 */
+  int32_t kv_dtype; /* TRI_INV_F32 or TRI_INV_BF16 */
+  int32_t n_seqs;   /* ragged mode: number of sequences; else 0 */
+  const int32_t* cu_seqlens; /* HOST pointer to n_seqs+1 non-decreasing offsets with
+                                cu_seqlens[0] == 0 and cu_seqlens[n_seqs] == T, or NULL.
+                                Read during the call only. */
+} tri_inv_desc;
+
+/*
+ * A = (I + N)^{-1} for every chunk (spec call `tri_inv_build(K, beta, g, C, method) -> A`;
+ * N as in Eq. 3 / Table 1, inversion per Sec. 3).
+ *   K, beta, g : inputs (device).   A : output (device), rows of real tokens only.
+ * Errors: INVALID_ARG for null/misaligned pointers or an inconsistent descriptor,
+ * UNSUPPORTED for an unknown method, CUDA if the launch fails.
+ */
+int tri_inv_build(const void* K, const float* beta, const float* g, float* A,
+                  const tri_inv_desc* desc, int method, void* cuda_stream);
+
+/*
+ * W = A diag(beta) K and U = A diag(beta) V from a given A
+ * (spec call `tri_inv_wy(A, K, V, beta) -> W, U`; the WY/UT transform
+ * the inverse exists for, Sec. 1).  A is read as stored by tri_inv_build
+ * (its lower triangle including the diagonal is used).  V and U may both be
+ * NULL to compute W only.
+ */
+int tri_inv_wy(const float* A, const void* K, const void* V, const float* beta,
+               void* W, void* U, const tri_inv_desc* desc, void* cuda_stream);
+
+/*
+ * Fused build + invert + WY in one kernel: K and V tiles are read once.
+ * A may be NULL when only W and U are wanted.
+ */
+int tri_inv_fused(const void* K, const void* V, const float* beta, const float* g,
+                  float* A, void* W, void* U,
+                  const tri_inv_desc* desc, int method, void* cuda_stream);
+
+/*
+ * Number of chunk matrices (chunks x heads) the descriptor describes.
+ * Host-only arithmetic; no device work.
+ */
+int tri_inv_count_matrices(const tri_inv_desc* desc, int64_t* out);
+
+/*
+ * After the caller has synchronised the stream: reads and clears the device
+ * status word of the current device.  *out is TRI_INV_OK, or
+ * TRI_INV_ERR_DEVICE_TIMEOUT if a kernel gave up on a bounded wait (the
+ * kernel then returned early and its outputs are incomplete).  This call
+ * copies 4 bytes from the device and so synchronises with it.
+ */
+int tri_inv_last_device_status(int* out);
+
+/* Kernel launches issued by this library in this process so far (host counter). */
+int64_t tri_inv_launch_count(void);
+
+/* Static string for a status code. */
+const char* tri_inv_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRI_INV_H_ */

@@ -1,0 +1,188 @@
+"""Thin ctypes binding over ``libtri_inv.so`` (the C ABI declared in ``include/tri_inv.h``).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels.
+torch is used for device memory and streams.  There is no CPU path: if the
+library is missing or a call fails, these functions raise.
+
+Tensors follow the header's layouts: K/V ``[B,T,H,d]`` (bf16 or fp32), beta/g
+``[B,T,H]`` fp32, A ``[B,T,H,C]`` fp32, W/U like K/V.  All must be contiguous
+CUDA tensors on the current device.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libtri_inv.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT = 0, 1, 2, 3, 4
+F32, BF16 = 0, 1
+BLOCK_RECURSIVE, PRODUCT_SERIES = 0, 1
+LEAF_SERIES = 0x100
+FORCE_SIMT = 0x10000
+
+EXPORTS = ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_count_matrices",
+           "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
+                ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("C", ctypes.c_int32),
+                ("kv_dtype", ctypes.c_int32), ("n_seqs", ctypes.c_int32),
+                ("cu_seqlens", ctypes.c_void_p)]
+
+
+class TriInvError(RuntimeError):
+    def __init__(self, fn, status):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (fn, status_string(status), status))
+
+
+_lib = None
+
+
+def load():
+    """Load the library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("%s not found: build it with `python -m paper_2605_21325_b200.build` "
+                              "(there is no CPU fallback)" % LIB_PATH)
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32, dp = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(Desc)
+        lib.tri_inv_build.argtypes = [vp, vp, vp, vp, dp, i32, vp]
+        lib.tri_inv_wy.argtypes = [vp, vp, vp, vp, vp, vp, dp, vp]
+        lib.tri_inv_fused.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
+        lib.tri_inv_count_matrices.argtypes = [dp, ctypes.POINTER(ctypes.c_int64)]
+        lib.tri_inv_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
+        for f in ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_count_matrices", "tri_inv_last_device_status"):
+            getattr(lib, f).restype = i32
+        lib.tri_inv_launch_count.restype = ctypes.c_int64
+        lib.tri_inv_launch_count.argtypes = []
+        lib.tri_inv_status_string.restype = ctypes.c_char_p
+        lib.tri_inv_status_string.argtypes = [i32]
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load().tri_inv_status_string(int(status)).decode()
+
+
+def launch_count() -> int:
+    return int(load().tri_inv_launch_count())
+
+
+def last_device_status() -> int:
+    out = ctypes.c_int(0)
+    rc = load().tri_inv_last_device_status(ctypes.byref(out))
+    if rc != OK:
+        raise TriInvError("tri_inv_last_device_status", rc)
+    return out.value
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("K/V must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def make_desc(B, T, H, d_k, d_v, C, kv_dtype, cu_seqlens=None):
+    """Returns (Desc, keepalive).  ``cu_seqlens`` is a host int array of n_seqs+1 offsets or None."""
+    keep = None
+    ptr, n_seqs = None, 0
+    if cu_seqlens is not None:
+        keep = np.ascontiguousarray(np.asarray(cu_seqlens), dtype=np.int32)
+        ptr, n_seqs = keep.ctypes.data, len(keep) - 1
+    return Desc(B, T, H, d_k, d_v, C, kv_dtype, n_seqs, ptr), keep
+
+
+def count_matrices(desc: Desc) -> int:
+    out = ctypes.c_int64(0)
+    rc = load().tri_inv_count_matrices(ctypes.byref(desc), ctypes.byref(out))
+    if rc != OK:
+        raise TriInvError("tri_inv_count_matrices", rc)
+    return out.value
+
+
+def _p(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "tensors must be contiguous CUDA tensors"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def build(K, beta, g, C, method=BLOCK_RECURSIVE, cu_seqlens=None, out=None, stream=None):
+    """A = (I+N)^{-1} per chunk -> A [B,T,H,C] fp32 (rows of real tokens written)."""
+    B, T, H, d_k = K.shape
+    desc, keep = make_desc(B, T, H, d_k, d_k, C, _dtype_code(K), cu_seqlens)
+    A = torch.zeros((B, T, H, C), dtype=torch.float32, device=K.device) if out is None else out
+    rc = load().tri_inv_build(_p(K), _p(beta), _p(g), _p(A), ctypes.byref(desc), int(method), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_build", rc)
+    return A
+
+
+def wy(A, K, V, beta, cu_seqlens=None, out=None, stream=None):
+    """W = A diag(beta) K, U = A diag(beta) V from a stored A."""
+    B, T, H, d_k = K.shape
+    C = A.shape[-1]
+    d_v = V.shape[-1] if V is not None else d_k
+    desc, keep = make_desc(B, T, H, d_k, d_v, C, _dtype_code(K), cu_seqlens)
+    if out is None:
+        W = torch.zeros_like(K)
+        U = torch.zeros_like(V) if V is not None else None
+    else:
+        W, U = out
+    rc = load().tri_inv_wy(_p(A), _p(K), _p(V), _p(beta), _p(W), _p(U), ctypes.byref(desc), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_wy", rc)
+    return W, U
+
+
+def fused(K, V, beta, g, C, method=BLOCK_RECURSIVE, cu_seqlens=None, want_A=True, out=None, stream=None):
+    """Fused build + invert + WY -> (A or None, W, U)."""
+    B, T, H, d_k = K.shape
+    d_v = V.shape[-1]
+    desc, keep = make_desc(B, T, H, d_k, d_v, C, _dtype_code(K), cu_seqlens)
+    if out is None:
+        A = torch.zeros((B, T, H, C), dtype=torch.float32, device=K.device) if want_A else None
+        W, U = torch.zeros_like(K), torch.zeros_like(V)
+    else:
+        A, W, U = out
+    rc = load().tri_inv_fused(_p(K), _p(V), _p(beta), _p(g), _p(A), _p(W), _p(U), ctypes.byref(desc), int(method), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_fused", rc)
+    return A, W, U
+
+
+# ---- moving workloads.Inputs (numpy, host) to the device and results back -------------------
+
+def kv_to_torch(a: np.ndarray, device="cuda", pin=False) -> torch.Tensor:
+    """float32 array or uint16 bf16 bit patterns -> torch tensor of the matching dtype."""
+    t = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
+    if device == "cpu":
+        return t.pin_memory() if pin else t
+    return t.to(device)
+
+
+def to_device(inp, device="cuda"):
+    """workloads.Inputs -> dict of CUDA tensors."""
+    return {"K": kv_to_torch(inp.K, device), "V": kv_to_torch(inp.V, device),
+            "beta": torch.from_numpy(inp.beta).to(device), "g": torch.from_numpy(inp.g).to(device)}
+
+
+def to_numpy_f64(t: torch.Tensor) -> np.ndarray:
+    """Device result -> float64 numpy (bf16 widened exactly)."""
+    return t.detach().to("cpu").to(torch.float64).numpy()

@@ -1,0 +1,209 @@
+// extern "C" boundary: argument validation, chunk table for packed sequences, dispatch.
+#include <atomic>
+#include <mutex>
+#include <vector>
+
+#include "common.cuh"
+
+namespace tri_inv {
+namespace {
+
+__device__ int g_device_status = 0;  // raised by kernels that give up on a bounded wait
+
+std::atomic<long long> g_launches{0};
+
+int* status_word_for_current_device(cudaError_t* err) {
+  // One address per device; looked up once per device under a lock.
+  static std::mutex mu;
+  static int* cache[64] = {nullptr};
+  int dev = 0;
+  *err = cudaGetDevice(&dev);
+  if (*err != cudaSuccess) return nullptr;
+  if (dev < 0 || dev >= 64) { *err = cudaErrorInvalidDevice; return nullptr; }
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cache[dev]) {
+    void* ptr = nullptr;
+    *err = cudaGetSymbolAddress(&ptr, g_device_status);
+    if (*err != cudaSuccess) return nullptr;
+    cache[dev] = (int*)ptr;
+  }
+  return cache[dev];
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_desc(const tri_inv_desc* d, bool need_dv) {
+  if (!d) return TRI_INV_ERR_INVALID_ARG;
+  if (d->B < 1 || d->T < 0 || d->H < 1) return TRI_INV_ERR_INVALID_ARG;
+  if (d->d_k < 8 || (d->d_k & 7)) return TRI_INV_ERR_INVALID_ARG;
+  if (need_dv && (d->d_v < 8 || (d->d_v & 7))) return TRI_INV_ERR_INVALID_ARG;
+  if (d->C != 16 && d->C != 32 && d->C != 64 && d->C != 128) return TRI_INV_ERR_INVALID_ARG;
+  if (d->kv_dtype != TRI_INV_F32 && d->kv_dtype != TRI_INV_BF16) return TRI_INV_ERR_INVALID_ARG;
+  if ((long long)d->B * d->T > 0x7fffffffLL) return TRI_INV_ERR_INVALID_ARG;
+  if (d->cu_seqlens) {
+    if (d->B != 1 || d->n_seqs < 0) return TRI_INV_ERR_INVALID_ARG;
+    if (d->cu_seqlens[0] != 0 || d->cu_seqlens[d->n_seqs] != d->T) return TRI_INV_ERR_INVALID_ARG;
+    for (int s = 0; s < d->n_seqs; ++s)
+      if (d->cu_seqlens[s + 1] < d->cu_seqlens[s]) return TRI_INV_ERR_INVALID_ARG;
+  } else if (d->n_seqs != 0) {
+    return TRI_INV_ERR_INVALID_ARG;
+  }
+  return TRI_INV_OK;
+}
+
+void ragged_table(const tri_inv_desc* d, std::vector<ChunkEntry>* tab) {
+  for (int s = 0; s < d->n_seqs; ++s) {
+    int beg = d->cu_seqlens[s], end = d->cu_seqlens[s + 1];
+    for (int t = beg; t < end; t += d->C) tab->push_back(ChunkEntry{t, (end - t) < d->C ? (end - t) : d->C});
+  }
+}
+
+int check_method(int method) {
+  int m = method & TRI_INV_METHOD_MASK;
+  if (m != TRI_INV_BLOCK_RECURSIVE && m != TRI_INV_PRODUCT_SERIES) return TRI_INV_ERR_UNSUPPORTED;
+  if (method & ~(TRI_INV_METHOD_MASK | TRI_INV_LEAF_SERIES | TRI_INV_FORCE_SIMT)) return TRI_INV_ERR_UNSUPPORTED;
+  if ((method & TRI_INV_LEAF_SERIES) && m != TRI_INV_BLOCK_RECURSIVE) return TRI_INV_ERR_UNSUPPORTED;
+  return TRI_INV_OK;
+}
+
+// Fills the parameter block, builds the ragged chunk table when needed, picks a kernel.
+int run(KParams p, const tri_inv_desc* d, void* stream_v) {
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  p.H = d->H; p.d_k = d->d_k; p.d_v = d->d_v; p.T = d->T;
+  p.kv_dtype = d->kv_dtype;
+  p.chunk_tab = nullptr;
+  cudaError_t err;
+  p.status = status_word_for_current_device(&err);
+  if (!p.status) return TRI_INV_ERR_CUDA;
+
+  ChunkEntry* dev_tab = nullptr;
+  if (d->cu_seqlens) {
+    std::vector<ChunkEntry> tab;
+    ragged_table(d, &tab);
+    p.n_chunks = (int)tab.size();
+    p.chunks_per_seq = 0;
+    if (p.n_chunks == 0) return TRI_INV_OK;
+    // The table is scratch owned by this call: allocated and freed in stream order.
+    if (cudaMallocAsync((void**)&dev_tab, tab.size() * sizeof(ChunkEntry), stream) != cudaSuccess) return TRI_INV_ERR_CUDA;
+    if (cudaMemcpyAsync(dev_tab, tab.data(), tab.size() * sizeof(ChunkEntry), cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+      cudaFreeAsync(dev_tab, stream);
+      return TRI_INV_ERR_CUDA;
+    }
+    // The host vector is pageable: the copy above has been staged before it returns.
+    p.chunk_tab = dev_tab;
+  } else {
+    p.chunks_per_seq = (d->T + d->C - 1) / d->C;
+    long long n = (long long)p.chunks_per_seq * d->B;
+    if (n > 0x7fffffffLL) return TRI_INV_ERR_INVALID_ARG;
+    p.n_chunks = (int)n;
+    if (p.n_chunks == 0) return TRI_INV_OK;
+  }
+
+  bool handled = false;
+  err = cudaSuccess;
+  if (!(p.method & TRI_INV_FORCE_SIMT)) err = launch_tc(p, d->C, stream, &handled);
+  if (err == cudaSuccess && !handled) err = launch_simt(p, d->C, stream);
+  if (err == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (dev_tab) cudaFreeAsync(dev_tab, stream);
+  return err == cudaSuccess ? TRI_INV_OK : TRI_INV_ERR_CUDA;
+}
+
+}  // namespace
+}  // namespace tri_inv
+
+using namespace tri_inv;
+
+extern "C" {
+
+int tri_inv_build(const void* K, const float* beta, const float* g, float* A,
+                  const tri_inv_desc* desc, int method, void* cuda_stream) {
+  int rc = check_desc(desc, false);
+  if (rc) return rc;
+  if (!K || !beta || !g || !A) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(beta) || !aligned16(g) || !aligned16(A)) return TRI_INV_ERR_INVALID_ARG;
+  if ((rc = check_method(method))) return rc;
+  KParams p{};
+  p.K = K; p.beta = beta; p.g = g; p.A = A;
+  p.method = method;
+  p.ops = kStoreA;
+  return run(p, desc, cuda_stream);
+}
+
+int tri_inv_wy(const float* A, const void* K, const void* V, const float* beta,
+               void* W, void* U, const tri_inv_desc* desc, void* cuda_stream) {
+  bool with_v = V || U;
+  int rc = check_desc(desc, with_v);
+  if (rc) return rc;
+  if (!A || !K || !beta || !W) return TRI_INV_ERR_INVALID_ARG;
+  if ((V == nullptr) != (U == nullptr)) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(A) || !aligned16(K) || !aligned16(V) || !aligned16(beta) || !aligned16(W) || !aligned16(U))
+    return TRI_INV_ERR_INVALID_ARG;
+  KParams p{};
+  p.A_in = A; p.K = K; p.V = V; p.beta = beta; p.W = W; p.U = U;
+  p.method = TRI_INV_BLOCK_RECURSIVE;
+  p.ops = kLoadA | kDoWY;
+  return run(p, desc, cuda_stream);
+}
+
+int tri_inv_fused(const void* K, const void* V, const float* beta, const float* g,
+                  float* A, void* W, void* U,
+                  const tri_inv_desc* desc, int method, void* cuda_stream) {
+  int rc = check_desc(desc, true);
+  if (rc) return rc;
+  if (!K || !V || !beta || !g || !W || !U) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(beta) || !aligned16(g) || !aligned16(A) || !aligned16(W) || !aligned16(U))
+    return TRI_INV_ERR_INVALID_ARG;
+  if ((rc = check_method(method))) return rc;
+  KParams p{};
+  p.K = K; p.V = V; p.beta = beta; p.g = g; p.A = A; p.W = W; p.U = U;
+  p.method = method;
+  p.ops = kDoWY | (A ? kStoreA : 0);
+  return run(p, desc, cuda_stream);
+}
+
+int tri_inv_count_matrices(const tri_inv_desc* desc, int64_t* out) {
+  int rc = check_desc(desc, false);
+  if (rc) return rc;
+  if (!out) return TRI_INV_ERR_INVALID_ARG;
+  long long n = 0;
+  if (desc->cu_seqlens) {
+    for (int s = 0; s < desc->n_seqs; ++s) {
+      long long len = desc->cu_seqlens[s + 1] - desc->cu_seqlens[s];
+      n += (len + desc->C - 1) / desc->C;
+    }
+  } else {
+    n = (long long)desc->B * ((desc->T + desc->C - 1) / desc->C);
+  }
+  *out = n * desc->H;
+  return TRI_INV_OK;
+}
+
+int tri_inv_last_device_status(int* out) {
+  if (!out) return TRI_INV_ERR_INVALID_ARG;
+  cudaError_t err;
+  int* word = status_word_for_current_device(&err);
+  if (!word) return TRI_INV_ERR_CUDA;
+  int v = 0;
+  if (cudaMemcpy(&v, word, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return TRI_INV_ERR_CUDA;
+  if (v != 0) {
+    int zero = 0;
+    if (cudaMemcpy(word, &zero, sizeof zero, cudaMemcpyHostToDevice) != cudaSuccess) return TRI_INV_ERR_CUDA;
+  }
+  *out = v;
+  return TRI_INV_OK;
+}
+
+int64_t tri_inv_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+const char* tri_inv_status_string(int status) {
+  switch (status) {
+    case TRI_INV_OK: return "ok";
+    case TRI_INV_ERR_INVALID_ARG: return "invalid argument";
+    case TRI_INV_ERR_UNSUPPORTED: return "unsupported request";
+    case TRI_INV_ERR_CUDA: return "CUDA runtime error";
+    case TRI_INV_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,71 @@
+// Shared declarations of the CUDA side: kernel parameter block, chunk lookup, launchers.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tri_inv.h"
+
+namespace tri_inv {
+
+// What a launch does besides inverting.
+enum : int {
+  kStoreA = 1,  // write A to global memory
+  kDoWY = 2,    // compute W (and U when V != nullptr)
+  kLoadA = 4,   // skip build + inversion, read A from A_in (tri_inv_wy)
+};
+
+// One entry per chunk of tokens in ragged mode.
+struct ChunkEntry {
+  int32_t tok0;  // first flat token of the chunk
+  int32_t rows;  // real tokens in it (1..C)
+};
+
+struct KParams {
+  const void* K;
+  const void* V;
+  const float* beta;
+  const float* g;
+  const float* A_in;
+  float* A;
+  void* W;
+  void* U;
+  const ChunkEntry* chunk_tab;  // ragged mode, else nullptr
+  int* status;                  // device status word (0 = ok); kernels only ever raise it
+  int32_t H, d_k, d_v, T;
+  int32_t chunks_per_seq;       // dense mode: ceil(T / C)
+  int32_t n_chunks;             // token chunks (all sequences); matrices = n_chunks * H
+  int32_t kv_dtype;
+  int32_t method;               // TRI_INV_* method with flags
+  int32_t ops;                  // kStoreA | kDoWY | kLoadA
+};
+
+// Flat work item -> (first token, real rows, head).  Consecutive items walk the heads of
+// one chunk of tokens, so neighbouring CTAs touch neighbouring memory.
+__device__ __forceinline__ void locate(const KParams& p, int C, long long item, long long& tok0, int& rows, int& h) {
+  int c = (int)(item / p.H);
+  h = (int)(item - (long long)c * p.H);
+  if (p.chunk_tab) {
+    ChunkEntry e = p.chunk_tab[c];
+    tok0 = e.tok0;
+    rows = e.rows;
+  } else {
+    int b = c / p.chunks_per_seq;
+    int ci = c - b * p.chunks_per_seq;
+    tok0 = (long long)b * p.T + (long long)ci * C;
+    int left = p.T - ci * C;
+    rows = left < C ? left : C;
+  }
+}
+
+__device__ __forceinline__ float load_kv(const void* base, int dtype, size_t idx) {
+  if (dtype == TRI_INV_F32) return ((const float*)base)[idx];
+  return __bfloat162float(((const __nv_bfloat16*)base)[idx]);
+}
+
+// Launchers (defined next to their kernels).  Return a cudaError_t from the launch.
+cudaError_t launch_simt(const KParams& p, int C, cudaStream_t stream);
+// Tensor-core path: returns cudaErrorNotSupported when it has no kernel for the request.
+cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
+
+}  // namespace tri_inv
