@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Throughput of the fused build + invert + WY path on synthetic GDN-shaped data.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--method block_recursive]
+    python bench.py --impl reference ...        # the fp64 CPU oracle, timed on the host cores
+
+A step is one pass of the whole hot path (stage K/V, Gram, gate, inversion, store A, WY,
+store W/U: one fused kernel launch) over one batch of the chosen configuration; the default is
+configuration 2 (B=4, T=4096, H=16, d=128, C=64, bf16: 4096 chunk matrices), the one the metric
+is quoted on.  Inputs are seeded synthetic tensors resident in HBM before the timed region; L2 is
+flushed (a 256 MiB write) before every timed step; each step is timed with CUDA events on the
+launching stream.  With N > 1 (torchrun, one rank per GPU) every rank runs its own copy of the
+batch -- chunks are independent, so there is no collective on the data path -- and the value is
+the total over ranks divided by the slowest rank's time (weak scaling).
+
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "chunk matrices inverted/sec (C=64, d=128, bf16) + % of roofline; max err vs fp64 oracle"
+UNIT = "chunk-matrices/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per chunk matrix moved by the fused kernel (dram__bytes_read.sum + dram__bytes_write.sum
+# of one ncu capture divided by the matrices of that launch); see profiles/.  None = not captured yet.
+NCU_TRAFFIC_BYTES_PER_MATRIX = {}
+
+
+def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True):
+    """Compulsory traffic of the fused path per chunk matrix: K, V, beta, g read once; A, W, U written once."""
+    b = C * d_k * elt + C * d_v * elt + 2 * C * 4 + C * d_k * elt + C * d_v * elt
+    if want_A:
+        b += C * C * 4
+    return b
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def time_oracle(inp, target_seconds=15.0, n_threads=0):
+    """The fp64 oracle, as it stands, on a bounded sample of the workload: leading tokens of each sequence."""
+    import numpy as np
+    import oracle
+    from paper_2605_21325_b200 import workloads as wl
+    cores = oracle.threads(n_threads)
+    # calibrate on a small slice, then size the sample for ~target_seconds
+    def run(T):
+        sub = wl.Inputs(inp.name, inp.B, T, inp.H, inp.d_k, inp.d_v, inp.C, inp.kv_dtype,
+                        np.ascontiguousarray(inp.K[:, :T]), np.ascontiguousarray(inp.V[:, :T]),
+                        np.ascontiguousarray(inp.beta[:, :T]), np.ascontiguousarray(inp.g[:, :T]))
+        t0 = time.perf_counter()
+        A = oracle.build_A(sub.K, sub.beta, sub.g, sub.C, n_threads=n_threads)
+        oracle.wy(A, sub.K, sub.V, sub.beta, sub.C, n_threads=n_threads)
+        return sub.n_matrices, time.perf_counter() - t0
+    n0, t0 = run(min(inp.T, 2 * inp.C))
+    per = t0 / max(n0, 1)
+    chunks = int(max(1, min(inp.T // inp.C, target_seconds / max(per * inp.B * inp.H, 1e-9))))
+    # repeat the sample until about target_seconds of CPU work has been done
+    n, t, passes = 0, 0.0, 0
+    while t < target_seconds and passes < 1000:
+        dn, dt = run(chunks * inp.C)
+        n, t, passes = n + dn, t + dt, passes + 1
+    return {"value": n / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "first %d tokens of each of the %d sequences of %s, %d passes (%d chunk matrices, %.1f s; build + WY in fp64)"
+                      % (chunks * inp.C, inp.B, inp.name, passes, n, t)}, n, t
+
+
+def run_reference(args):
+    """--impl reference: the oracle is the reference arm (there is no reference implementation to install)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2605_21325_b200 import workloads as wl
+    inp = wl.config(args.config)
+    per_step_target = max(2.0, min(15.0, 120.0 / max(args.steps + args.warmup, 1)))
+    vals = []
+    base = None
+    for s in range(args.warmup + args.steps):
+        base, n, t = time_oracle(inp, target_seconds=per_step_target)
+        if s >= args.warmup:
+            vals.append((n, t))
+    n_tot = sum(n for n, _ in vals)
+    t_tot = sum(t for _, t in vals)
+    value = n_tot / t_tot
+    base["value"] = value
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / max(len(vals), 1), "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": inp.name, "B": inp.B, "T": inp.T, "H": inp.H, "d_k": inp.d_k, "d_v": inp.d_v,
+                      "C": inp.C, "note": "each step is a bounded sample of the workload"},
+           "cpu_baseline": base,
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--method", default="block_recursive", choices=["block_recursive", "mixed_recursion", "product_series"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-flush", action="store_true", help="skip the L2 flush between steps (profiling runs)")
+    ap.add_argument("--simt", action="store_true", help="force the CUDA-core kernel")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import __graft_entry__ as entry
+    from paper_2605_21325_b200 import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        entry.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2605_21325_b200 import binding
+
+    method = {"block_recursive": binding.BLOCK_RECURSIVE, "mixed_recursion": binding.BLOCK_RECURSIVE | binding.LEAF_SERIES,
+              "product_series": binding.PRODUCT_SERIES}[args.method]
+    if args.simt:
+        method |= binding.FORCE_SIMT
+
+    inp = wl.config(args.config)                    # same seeded batch on every rank (weak scaling)
+    n_mat = inp.n_matrices
+    dev = binding.to_device(inp)
+    K, V, beta, g = dev["K"], dev["V"], dev["beta"], dev["g"]
+    A = torch.empty((inp.B, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda")
+    W, U = torch.empty_like(K), torch.empty_like(V)
+    flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        binding.fused(K, V, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U), stream=stream)
+
+    for _ in range(max(args.warmup, 3)):
+        if flush is not None:
+            flush.fill_(1)
+        step()
+    torch.cuda.synchronize()
+    if binding.last_device_status() != 0:
+        raise SystemExit("device status word raised during warm-up")
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        # the timed region lasts milliseconds: keep the GPU busy with the same step until the sampler has
+        # produced readings under load, then go straight into the timed steps
+        sampler.start()
+        t_end = time.time() + 5.0
+        while sampler.proc and len(sampler.lines) < 4 and time.time() < t_end:
+            for _ in range(20):
+                step()
+            torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = binding.launch_count()
+    evs = []
+    for _ in range(args.steps):
+        if flush is not None:
+            flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        step()
+        e1.record(stream)
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    launches = binding.launch_count() - launches0
+    times_ms = [a.elapsed_time(b) for a, b in evs]
+    total_ms = sum(times_ms)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    clocks = sampler.stop() if rank == 0 else None
+    ms_per_step = total_ms / args.steps
+    value = world * n_mat / (ms_per_step * 1e-3)
+
+    # ---- end to end through the public API with host buffers: H2D of the inputs, kernel, D2H of A, W, U
+    hK, hV = binding.kv_to_torch(inp.K, "cpu", pin=True), binding.kv_to_torch(inp.V, "cpu", pin=True)
+    hb, hg = torch.from_numpy(inp.beta).pin_memory(), torch.from_numpy(inp.g).pin_memory()
+    hA = torch.empty(A.shape, dtype=A.dtype).pin_memory()
+    hW, hU = torch.empty(W.shape, dtype=W.dtype).pin_memory(), torch.empty(U.shape, dtype=U.dtype).pin_memory()
+    h2d = sum(x.numel() * x.element_size() for x in (hK, hV, hb, hg))
+    d2h = sum(x.numel() * x.element_size() for x in (hA, hW, hU))
+
+    def e2e_step():
+        K.copy_(hK, non_blocking=True); V.copy_(hV, non_blocking=True)
+        beta.copy_(hb, non_blocking=True); g.copy_(hg, non_blocking=True)
+        step()
+        hA.copy_(A, non_blocking=True); hW.copy_(W, non_blocking=True); hU.copy_(U, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    e2e_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * n_mat * e2e_steps / (e2e_ms * 1e-3)
+
+    # ---- accuracy of what was just timed, on a sample the oracle computes directly
+    err = None
+    if rank == 0:
+        import oracle
+        Ts = min(inp.T, 4 * inp.C) if inp.cu_seqlens is None else None
+        if Ts is not None:
+            A_ref = oracle.build_A(inp.K[:, :Ts], inp.beta[:, :Ts], inp.g[:, :Ts], inp.C)
+            W_ref, U_ref = oracle.wy(A_ref, inp.K[:, :Ts], inp.V[:, :Ts], inp.beta[:, :Ts], inp.C)
+            a = binding.to_numpy_f64(A[:, :Ts]); w = binding.to_numpy_f64(W[:, :Ts]); u = binding.to_numpy_f64(U[:, :Ts])
+        else:
+            A_ref = oracle.build_A(inp.K, inp.beta, inp.g, inp.C, cu_seqlens=inp.cu_seqlens)
+            W_ref, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, inp.C, cu_seqlens=inp.cu_seqlens)
+            a, w, u = binding.to_numpy_f64(A), binding.to_numpy_f64(W), binding.to_numpy_f64(U)
+        err = {"A_max_ratio": float(np.abs(a - A_ref).max() / np.abs(A_ref).max()),
+               "W_max_ratio": float(np.abs(w - W_ref).max() / np.abs(W_ref).max()),
+               "U_max_ratio": float(np.abs(u - U_ref).max() / np.abs(U_ref).max()),
+               "sample": "first %d tokens of every sequence" % Ts if Ts else "all tokens"}
+
+    if rank == 0:
+        elt = 2 if inp.kv_dtype == wl.BF16 else 4
+        alg_bytes = algorithmic_bytes_per_matrix(inp.C, inp.d_k, inp.d_v, elt)
+        kernel_ms = statistics.mean(times_ms)               # one launch per step, timed alone by its event pair
+        achieved = alg_bytes * n_mat / (kernel_ms * 1e-3) / 1e9
+        peak, peak_kind = measured_peak_gbs()
+        traffic = NCU_TRAFFIC_BYTES_PER_MATRIX.get((args.config, args.method))
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": None if traffic is None else traffic * n_mat, "peak_source": "of " + peak_kind,
+                    "kernel": "fused build+invert+WY", "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
+                    "algorithmic_bytes_per_launch": alg_bytes * n_mat}
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            cpu, _, _ = time_oracle(inp, target_seconds=15.0)
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+               "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+               "dtype": "bf16" if inp.kv_dtype == wl.BF16 else "f32", "data": "synthetic",
+               "config": {"workload": inp.name, "B": inp.B, "T": inp.T, "H": inp.H, "d_k": inp.d_k, "d_v": inp.d_v, "C": inp.C,
+                          "chunk_matrices_per_gpu": n_mat, "method": args.method, "outputs": "A fp32 + W,U",
+                          "l2": "flushed before every timed step (256 MiB write)" if flush is not None else "not flushed",
+                          "parallelism": "independent replicas, no collective" if world > 1 else "single GPU"},
+               "gb_per_s": achieved, "roofline": roofline, "cpu_baseline": cpu,
+               "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+               "gpu_launches": launches, "clocks": clocks, "error_vs_oracle": err}
+        print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
