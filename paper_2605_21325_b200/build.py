@@ -34,6 +34,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC",
            "-I", os.path.join(ROOT, "include"), "-I", os.path.join(PKG, "csrc"),
            "-o", LIB] + sources()
+    cmd += os.environ.get("TRI_INV_NVCC_FLAGS", "").split()
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -8,7 +8,7 @@
 namespace tri_inv {
 namespace {
 
-__device__ int g_device_status = 0;  // raised by kernels that give up on a bounded wait
+__device__ int g_device_status[128] = {0};  // word 0: raised by kernels that give up on a bounded wait
 
 std::atomic<long long> g_launches{0};
 
@@ -192,6 +192,18 @@ int tri_inv_last_device_status(int* out) {
   *out = v;
   return TRI_INV_OK;
 }
+
+#ifdef TRI_INV_PHASE_CLOCKS
+// Development builds only: copies the 128 status/counter words to the host and clears them.
+int tri_inv_debug_counters(int* out) {
+  cudaError_t err;
+  int* word = status_word_for_current_device(&err);
+  if (!word) return TRI_INV_ERR_CUDA;
+  if (cudaMemcpy(out, word, 128 * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return TRI_INV_ERR_CUDA;
+  if (cudaMemset(word, 0, 128 * sizeof(int)) != cudaSuccess) return TRI_INV_ERR_CUDA;
+  return TRI_INV_OK;
+}
+#endif
 
 int64_t tri_inv_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 

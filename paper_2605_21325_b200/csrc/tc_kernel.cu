@@ -92,6 +92,20 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Optional per-phase cycle counters (development builds only: -DTRI_INV_PHASE_CLOCKS).
+#ifdef TRI_INV_PHASE_CLOCKS
+#define PHASE_BEGIN() long long ph_t = clock64()
+#define PHASE(k)                                                                  \
+  do {                                                                            \
+    long long now = clock64();                                                    \
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(p.status + 8 + 8 * (threadIdx.x >> 5) + (k), (int)(now - ph_t)); \
+    ph_t = now;                                                                   \
+  } while (0)
+#else
+#define PHASE_BEGIN() do {} while (0)
+#define PHASE(k) do {} while (0)
+#endif
+
 // ------------------------------------------------------------------------------------------ layout
 template <int C, int D>
 struct Cfg {
@@ -230,7 +244,7 @@ __device__ __forceinline__ void wy_apply(const uint32_t (&af)[C / 16][4], uint32
 }
 
 template <int C, int D>
-__global__ void __launch_bounds__(Cfg<C, D>::NT) tc_kernel(const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                          const __grid_constant__ CUtensorMap tmV, KParams p) {
   using cfg = Cfg<C, D>;
   constexpr int LD = cfg::LD;
@@ -263,6 +277,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT) tc_kernel(const __grid_constant
     long long tok0;
     int rows, h;
     locate(p, C, item, tok0, rows, h);
+    PHASE_BEGIN();
 
     // ---- 1. stage K, V (TMA) and beta, g
     if (tid == 0) {
@@ -308,6 +323,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT) tc_kernel(const __grid_constant
       }
     }
     __syncthreads();
+    PHASE(0);
 
     if (!load_a) {
       // ---- 2. Gram tiles of this warp's rows, 3. gate + mask, N -> shared memory
@@ -350,6 +366,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT) tc_kernel(const __grid_constant
         }
       }
       __syncwarp();
+      PHASE(1);
 
       // ---- 4. leaf: invert this warp's 16x16 diagonal block, lane j owns column j
       {
@@ -376,11 +393,14 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT) tc_kernel(const __grid_constant
         }
       }
       __syncthreads();
+      PHASE(2);
 
       // ---- 5. merges
       merge_level<C, 16>(sX, warp, lane);
+      PHASE(3);
       merge_level<C, 32>(sX, warp, lane);
       if constexpr (C == 128) merge_level<C, 64>(sX, warp, lane);
+      PHASE(4);
     }
 
     // ---- 6. store A
@@ -399,6 +419,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT) tc_kernel(const __grid_constant
       }
     }
 
+    PHASE(5);
     // ---- 7. WY apply
     if (do_wy) {
       uint32_t af[C / 16][4];
@@ -424,7 +445,9 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT) tc_kernel(const __grid_constant
       wy_apply<C, D>(af, sK, warp, lane, reinterpret_cast<__nv_bfloat16*>(p.W), tok0, rows, h, p.H);
       if (need_v) wy_apply<C, D>(af, sV, warp, lane, reinterpret_cast<__nv_bfloat16*>(p.U), tok0, rows, h, p.H);
     }
+    PHASE(6);
     __syncthreads();  // all warps are done with the tiles and sX before the next item's copies land
+    PHASE(7);
   }
 }
 
@@ -466,6 +489,8 @@ cudaError_t launch_one(const KParams& p, cudaStream_t stream) {
   static int ctas_per_sm = 0, n_sm = 0;
   if (!ctas_per_sm) {
     cudaError_t e = cudaFuncSetAttribute(tc_kernel<C, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(tc_kernel<C, D>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     int dev = 0, occ = 0;
     cudaGetDevice(&dev);
