@@ -4,14 +4,18 @@
 // one warp per 16 rows.  Per item:
 //   1. TMA (cp.async.bulk.tensor, 128-byte swizzle) stages the C x d tiles of K and V in
 //      shared memory; beta and g come in with plain loads.
-//   2. Gram tiles S = K K^T on or below the diagonal: bf16 MMA (m16n8k16), fp32 accumulate.
-//   3. Gate + strict-lower mask in registers, N written to shared memory in fp32.
+//   2. Gram S = K K^T: tcgen05.mma (kind::f16, bf16 operands straight from the TMA-written tiles,
+//      fp32 accumulator in tensor memory), issued by one thread, completion through an mbarrier.
+//   3. Each warp reads its 16 rows of S from tensor memory (tcgen05.ld 16x256b: the m16n8 accumulator
+//      fragment layout), applies gate + strict-lower mask, writes N to shared memory in fp32.
 //   4. 16x16 leaves inverted by forward substitution, one lane per column (Sec. 3.1).
 //   5. Block-recursive merges X21 = -(X22 N21) X11 for b = 16, 32, (64) as TF32 MMAs
 //      (m16n8k8, fp32 accumulate) on fp32 data kept in shared memory (Sec. 3.3).
 //   6. A stored with 16-byte coalesced stores; upper triangle and diagonal are constants.
-//   7. W = (A diag(beta)) K and U = (A diag(beta)) V: bf16 MMA with the K / V tiles still in
-//      shared memory as the B operand; results leave as 16-byte stores straight from registers.
+//   7. A' = A diag(beta) is written as a bf16 K-major swizzled operand over the fp32 matrix's space;
+//      W = A' K and U = A' V are tcgen05.mma with the K / V tiles still in shared memory as the
+//      MN-major B operand; accumulators come back from tensor memory and leave as 16-byte stores.
+//   The next item's tiles are requested as soon as the last MMA of this item has completed.
 // Inputs of the inversion stay fp32 in shared memory; only the Gram product and the WY
 // apply see bf16 operands (the Gram operands are the bf16 inputs themselves, so exact).
 #include <cuda.h>
@@ -121,8 +125,8 @@ struct Cfg {
   static constexpr int OFF_BETA = OFF_X + C * LD * 4;
   static constexpr int OFF_G = OFF_BETA + C * 4;
   static constexpr int OFF_BAR = OFF_G + C * 4;
-  static constexpr int BYTES = OFF_BAR + 16;
-  static constexpr int SMEM = BYTES + 1024;     // slack to align the base to 1024 B (swizzle atom)
+  static constexpr int BYTES = OFF_BAR + 32;     // two mbarriers and the TMEM base-address slot
+  static constexpr int SMEM = BYTES;
 };
 
 // Byte offset of the 16-byte chunk holding features [f, f+8) of row r inside a swizzled tile.
@@ -188,77 +192,131 @@ __device__ __forceinline__ void merge_level(float* sX, int warp, int lane) {
   __syncthreads();
 }
 
-// W (or U) = A' . tile for this warp's 16 rows; A' fragments are already scaled by beta and in bf16.
-template <int C, int D>
-__device__ __forceinline__ void wy_apply(const uint32_t (&af)[C / 16][4], uint32_t tile, int warp, int lane,
-                                         __nv_bfloat16* out, long long tok0, int rows, int h, int H) {
-  constexpr int NTN = D / 8;
-  float acc[NTN][4];
+// ------------------------------------------------------------------------------------------ tcgen05 helpers
+// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets
+// (all >> 4), descriptor version 1 at bit 46, 128-byte swizzle (code 2) at bits 61..63.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3fffu);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor for kind::f16: fp32 accumulate, bf16 x bf16, A K-major,
+// B K-major (b_mn = 0) or MN-major (b_mn = 1), shape M x N.
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// 16 lanes x 16 columns: the accumulator fragment of two adjacent m16n8 tiles
+// (regs 0..3: columns 0..7, regs 4..7: columns 8..15; thread t: rows t/4 and t/4+8, columns 2(t%4), +1).
+__device__ __forceinline__ void tmem_ld_16x16(float (&r)[2][4], uint32_t taddr) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=f"(r[0][0]), "=f"(r[0][1]), "=f"(r[0][2]), "=f"(r[0][3]), "=f"(r[1][0]), "=f"(r[1][1]), "=f"(r[1][2]), "=f"(r[1][3])
+               : "r"(taddr));
+}
+// 16 lanes x 64 columns -> 8 n-tiles of accumulator fragments.
+__device__ __forceinline__ void tmem_ld_16x64(float (&r)[8][4], uint32_t taddr) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=f"(r[0][0]), "=f"(r[0][1]), "=f"(r[0][2]), "=f"(r[0][3]), "=f"(r[1][0]), "=f"(r[1][1]), "=f"(r[1][2]), "=f"(r[1][3]),
+        "=f"(r[2][0]), "=f"(r[2][1]), "=f"(r[2][2]), "=f"(r[2][3]), "=f"(r[3][0]), "=f"(r[3][1]), "=f"(r[3][2]), "=f"(r[3][3]),
+        "=f"(r[4][0]), "=f"(r[4][1]), "=f"(r[4][2]), "=f"(r[4][3]), "=f"(r[5][0]), "=f"(r[5][1]), "=f"(r[5][2]), "=f"(r[5][3]),
+        "=f"(r[6][0]), "=f"(r[6][1]), "=f"(r[6][2]), "=f"(r[6][3]), "=f"(r[7][0]), "=f"(r[7][1]), "=f"(r[7][2]), "=f"(r[7][3])
+      : "r"(taddr));
+}
+// 16 lanes x 128 columns -> 16 n-tiles of accumulator fragments.
+__device__ __forceinline__ void tmem_ld_16x128(float (&r)[16][4], uint32_t taddr) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,"
+      "%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%64];"
+      : "=f"(r[0][0]), "=f"(r[0][1]), "=f"(r[0][2]), "=f"(r[0][3]), "=f"(r[1][0]), "=f"(r[1][1]), "=f"(r[1][2]), "=f"(r[1][3]),
+        "=f"(r[2][0]), "=f"(r[2][1]), "=f"(r[2][2]), "=f"(r[2][3]), "=f"(r[3][0]), "=f"(r[3][1]), "=f"(r[3][2]), "=f"(r[3][3]),
+        "=f"(r[4][0]), "=f"(r[4][1]), "=f"(r[4][2]), "=f"(r[4][3]), "=f"(r[5][0]), "=f"(r[5][1]), "=f"(r[5][2]), "=f"(r[5][3]),
+        "=f"(r[6][0]), "=f"(r[6][1]), "=f"(r[6][2]), "=f"(r[6][3]), "=f"(r[7][0]), "=f"(r[7][1]), "=f"(r[7][2]), "=f"(r[7][3]),
+        "=f"(r[8][0]), "=f"(r[8][1]), "=f"(r[8][2]), "=f"(r[8][3]), "=f"(r[9][0]), "=f"(r[9][1]), "=f"(r[9][2]), "=f"(r[9][3]),
+        "=f"(r[10][0]), "=f"(r[10][1]), "=f"(r[10][2]), "=f"(r[10][3]), "=f"(r[11][0]), "=f"(r[11][1]), "=f"(r[11][2]), "=f"(r[11][3]),
+        "=f"(r[12][0]), "=f"(r[12][1]), "=f"(r[12][2]), "=f"(r[12][3]), "=f"(r[13][0]), "=f"(r[13][1]), "=f"(r[13][2]), "=f"(r[13][3]),
+        "=f"(r[14][0]), "=f"(r[14][1]), "=f"(r[14][2]), "=f"(r[14][3]), "=f"(r[15][0]), "=f"(r[15][1]), "=f"(r[15][2]), "=f"(r[15][3])
+      : "r"(taddr));
+}
+
+// Epilogue of one 16-row x 64-column piece of W or U: accumulator fragments from tensor memory ->
+// bf16 -> stmatrix into a per-warp, swizzled 2 KiB staging tile -> 16-byte loads -> coalesced
+// 16-byte global stores (8 lanes cover one 128-byte row segment).
+__device__ __forceinline__ void store_frag_piece_bf16(const float (&f)[8][4], uint32_t stage, int lane, __nv_bfloat16* out_row0,
+                                                      size_t row_stride, int rows_left) {
+  const int mi = lane >> 3, r = (lane & 7) + 8 * (mi & 1);
 #pragma unroll
-  for (int i = 0; i < NTN; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
-  const int krow_l = (lane & 7) + 8 * ((lane >> 3) & 1);
-  const int ncol_l = 8 * (lane >> 4);
-#pragma unroll
-  for (int ks = 0; ks < C / 16; ++ks) {
-    if (ks <= warp) {
-#pragma unroll
-      for (int np = 0; np < NTN / 2; ++np) {
-        uint32_t b[4];
-        ldsm_x4_t(b, tile + tile_off<C>(16 * ks + krow_l, 16 * np + ncol_l));
-        mma_bf16(acc[2 * np], af[ks], b[0], b[1]);
-        mma_bf16(acc[2 * np + 1], af[ks], b[2], b[3]);
-      }
-    }
+  for (int nt = 0; nt < 8; nt += 2) {
+    const uint32_t m0 = pack_bf16(f[nt][0], f[nt][1]), m1 = pack_bf16(f[nt][2], f[nt][3]);
+    const uint32_t m2 = pack_bf16(f[nt + 1][0], f[nt + 1][1]), m3 = pack_bf16(f[nt + 1][2], f[nt + 1][3]);
+    const int chunk = nt + (mi >> 1);
+    const uint32_t addr = stage + r * 128 + ((chunk ^ (r & 7)) << 4);
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
   }
-  // Quad transpose so each lane owns 8 consecutive columns of one row, then 16-byte stores.
-  const int g = lane >> 2, t = lane & 3;
+  __syncwarp();
 #pragma unroll
-  for (int q = 0; q < NTN / 4; ++q) {
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      uint32_t v[4], o[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) v[j] = pack_bf16(acc[4 * q + j][2 * half], acc[4 * q + j][2 * half + 1]);
-      // lane t keeps tile t's pair in slot t and fetches, from lane s, that lane's pair of tile t
-#pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        int s = t ^ r;                       // partner lane within the quad
-        uint32_t send = v[0];
-        send = (s == 1) ? v[1] : send;
-        send = (s == 2) ? v[2] : send;
-        send = (s == 3) ? v[3] : send;       // my pair of the tile the partner owns
-        uint32_t got = __shfl_xor_sync(0xffffffffu, send, r);
-        // partner s holds columns 2s, 2s+1 of my tile: slot s of my output
-        o[0] = (s == 0) ? got : o[0];
-        o[1] = (s == 1) ? got : o[1];
-        o[2] = (s == 2) ? got : o[2];
-        o[3] = (s == 3) ? got : o[3];
-      }
-      int row = 16 * warp + g + 8 * half;
-      if (row < rows) {
-        __nv_bfloat16* dst = out + ((size_t)(tok0 + row) * H + h) * D + 8 * (4 * q + t);
-        *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
-      }
-    }
+  for (int m = 0; m < 4; ++m) {
+    const int rr = 4 * m + (lane >> 3), c = lane & 7;
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stage + rr * 128 + ((c ^ (rr & 7)) << 4)));
+    if (rr < rows_left) *reinterpret_cast<uint4*>(out_row0 + rr * row_stride + 8 * c) = v;
   }
+  __syncwarp();
+}
+__device__ __forceinline__ void store_piece_bf16(uint32_t taddr, uint32_t stage, int lane, __nv_bfloat16* out_row0,
+                                                 size_t row_stride, int rows_left) {
+  float f[8][4];
+  tmem_ld_16x64(f, taddr);
+  tmem_wait_ld();
+  store_frag_piece_bf16(f, stage, lane, out_row0, row_stride, rows_left);
 }
 
 template <int C, int D>
 __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(const __grid_constant__ CUtensorMap tmK,
-                                                         const __grid_constant__ CUtensorMap tmV, KParams p) {
+                                                                             const __grid_constant__ CUtensorMap tmV, KParams p) {
   using cfg = Cfg<C, D>;
+  static_assert(D == 128, "tiles are two 64-feature boxes wide");
   constexpr int LD = cfg::LD;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr int TMEM_COLS = (C == 64) ? 128 : 256;
+  constexpr int kStageOff = C * C * 2;  // per-warp 2 KiB output staging tiles sit behind A' in the N/X matrix's space
+  static_assert(kStageOff + Cfg<C, D>::NW * 2048 <= C * Cfg<C, D>::LD * 4, "staging must fit behind A'");
+  extern __shared__ __align__(1024) uint8_t smem[];  // swizzled tiles need a 1024-byte aligned base
   float* sX = reinterpret_cast<float*>(smem + cfg::OFF_X);
   float* sBeta = reinterpret_cast<float*>(smem + cfg::OFF_BETA);
   float* sG = reinterpret_cast<float*>(smem + cfg::OFF_G);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 24);
   const uint32_t sK = smem_u32(smem + cfg::OFF_K);
   const uint32_t sV = smem_u32(smem + cfg::OFF_V);
-  const uint32_t bar = smem_u32(smem + cfg::OFF_BAR);
+  const uint32_t sAp = smem_u32(smem + cfg::OFF_X);  // A' = A diag(beta) in bf16 reuses the N/X matrix's space
+  const uint32_t bar_k = smem_u32(smem + cfg::OFF_BAR);  // K tile landed
+  const uint32_t bar_mma = bar_k + 8;                    // a batch of MMAs completed
+  const uint32_t bar_v = bar_k + 16;                     // V tile landed
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
+  // Row block of this warp.  TMEM lanes are reachable only from the warp whose id % 4 matches
+  // the 32-lane quadrant: M = 64 puts rows 16q..16q+15 in lanes 32q..32q+15, M = 128 puts row i in lane i.
+  const int rb = (C == 64) ? warp : 2 * (warp & 3) + (warp >> 2);
+  const uint32_t lane_base = (C == 64) ? 32u * warp : 16u * rb;
   const bool do_wy = (p.ops & kDoWY) != 0;
   const bool need_v = do_wy && p.V != nullptr;
   const bool load_a = (p.ops & kLoadA) != 0;
@@ -267,33 +325,66 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
   if (tid == 0) {
     prefetch_tmap(&tmK);
     if (need_v) prefetch_tmap(&tmV);
-    mbar_init(bar, 1);
+    mbar_init(bar_k, 1);
+    mbar_init(bar_v, 1);
+    mbar_init(bar_mma, 1);
     fence_mbar_init();
   }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
   __syncthreads();
-  uint32_t phase = 0;
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const bool misaligned = (sK & 1023u) != 0;  // never expected; the swizzle pattern would not match the copies
+  const uint32_t tmem_rows = tmem + (lane_base << 16);
+  uint32_t ph_load = 0, ph_mma = 0;
+  bool failed = misaligned;
 
-  for (long long item = blockIdx.x; item < total; item += gridDim.x) {
+  // Thread 0 requests the tiles of an item; K and V complete on separate barriers so that the Gram
+  // product can start on K alone and each buffer is refilled as soon as its last reader is done.
+  auto issue_k = [&](long long item) {
+    long long tok0; int rows, h;
+    locate(p, C, item, tok0, rows, h);
+    fence_proxy_async();
+    mbar_expect_tx(bar_k, (uint32_t)cfg::TILE_BYTES);
+#pragma unroll
+    for (int bx = 0; bx < cfg::NBOX; ++bx) tma_load_2d(sK + bx * cfg::BOX_BYTES, &tmK, bar_k, h * D + 64 * bx, (int)tok0);
+  };
+  auto issue_v = [&](long long item) {
+    long long tok0; int rows, h;
+    locate(p, C, item, tok0, rows, h);
+    fence_proxy_async();
+    mbar_expect_tx(bar_v, (uint32_t)cfg::TILE_BYTES);
+#pragma unroll
+    for (int bx = 0; bx < cfg::NBOX; ++bx) tma_load_2d(sV + bx * cfg::BOX_BYTES, &tmV, bar_v, h * D + 64 * bx, (int)tok0);
+  };
+  // beta (threads 0..C-1) and g (threads C..2C-1) of an item, fetched one item ahead into a register
+  auto fetch_bg = [&](long long item) -> float {
+    long long tok0; int rows, h;
+    locate(p, C, item, tok0, rows, h);
+    const int i = tid < C ? tid : tid - C;
+    const float* src = tid < C ? p.beta : p.g;
+    return (i < rows && src) ? src[(size_t)(tok0 + i) * p.H + h] : 0.f;
+  };
+  float bg_next = 0.f;
+  if ((long long)blockIdx.x < total && !misaligned) {
+    if (tid == 0) { issue_k(blockIdx.x); if (need_v) issue_v(blockIdx.x); }
+    bg_next = fetch_bg(blockIdx.x);
+  }
+
+  for (long long item = blockIdx.x; item < total && !misaligned; item += gridDim.x) {
     long long tok0;
     int rows, h;
     locate(p, C, item, tok0, rows, h);
     PHASE_BEGIN();
 
-    // ---- 1. stage K, V (TMA) and beta, g
-    if (tid == 0) {
-      fence_proxy_async();  // earlier generic-proxy accesses to the tiles are ordered before the async writes
-      mbar_expect_tx(bar, (uint32_t)(cfg::TILE_BYTES * (need_v ? 2 : 1)));
-#pragma unroll
-      for (int bx = 0; bx < cfg::NBOX; ++bx) {
-        tma_load_2d(sK + bx * cfg::BOX_BYTES, &tmK, bar, h * D + 64 * bx, (int)tok0);
-        if (need_v) tma_load_2d(sV + bx * cfg::BOX_BYTES, &tmV, bar, h * D + 64 * bx, (int)tok0);
-      }
-    }
-    for (int i = tid; i < C; i += cfg::NT) {
-      size_t bi = (size_t)(tok0 + i) * p.H + h;
-      sBeta[i] = (i < rows) ? p.beta[bi] : 0.f;
-      sG[i] = (i < rows && p.g) ? p.g[bi] : 0.f;
-    }
+    // ---- 1. beta, g were fetched during the previous item (sBeta and sG are adjacent: one store each)
+    sBeta[tid] = bg_next;
+    const bool has_next = item + gridDim.x < total;
+    bool k_requested = false;   // thread 0: next item's K tile already requested
     if (load_a) {
       for (int e = tid; e < C * C; e += cfg::NT) {
         int i = e / C, j = e - i * C;
@@ -302,16 +393,9 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         sX[i * LD + j] = v;
       }
     }
-    bool arrived = mbar_wait_bounded(bar, phase);
-    phase ^= 1;
-    if (!arrived) {
-      // Give the copy one more bounded chance to land before leaving, then report and stop.
-      atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
-      mbar_wait_bounded(bar, phase ^ 1);
-      return;
-    }
     if (rows < C) {
-      // rows past the sequence end hold a neighbour's tokens (or zero fill): clear them
+      // rows past the sequence end hold a neighbour's tokens (or zero fill): clear them before any MMA
+      if (!mbar_wait_bounded(bar_k, ph_load) || (need_v && !mbar_wait_bounded(bar_v, ph_load))) { failed = true; break; }
       for (int e = tid; e < (C - rows) * 8 * cfg::NBOX * 2; e += cfg::NT) {
         int which = e / ((C - rows) * 8 * cfg::NBOX);
         int rem = e - which * (C - rows) * 8 * cfg::NBOX;
@@ -321,56 +405,72 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         uint8_t* base = smem + (which ? cfg::OFF_V : cfg::OFF_K) + bx * cfg::BOX_BYTES + r * 128 + c * 16;
         *reinterpret_cast<uint4*>(base) = make_uint4(0, 0, 0, 0);
       }
+      fence_proxy_async();
     }
     __syncthreads();
     PHASE(0);
 
     if (!load_a) {
-      // ---- 2. Gram tiles of this warp's rows, 3. gate + mask, N -> shared memory
-      uint32_t af[D / 16][4];
-      {
-        const int r = 16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1);
-        const int fo = 8 * (lane >> 4);
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) ldsm_x4(af[ks], sK + tile_off<C>(r, 16 * ks + fo));
-      }
-      const int ra = 16 * warp + g, rb = ra + 8;
-      const float beta_a = sBeta[ra], beta_b = sBeta[rb], g_a = sG[ra], g_b = sG[rb];
-#pragma unroll
-      for (int jb = 0; jb < cfg::NW; ++jb) {
-        if (jb <= warp) {
-          float acc[2][4];
-#pragma unroll
-          for (int i = 0; i < 2; ++i) { acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f; }
-          const int n = 16 * jb + (lane & 7) + 8 * (lane >> 4);
-          const int fo = 8 * ((lane >> 3) & 1);
+      // ---- 2. Gram S = K K^T on the tensor core: one thread issues D/16 MMAs of C x C x 16 into TMEM
+      if (tid == 0) {
+        if (!mbar_wait_bounded(bar_k, ph_load)) {
+          atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);  // the other threads time out on bar_mma
+        } else {
+          tc_fence_after();
+          constexpr uint32_t idesc = umma_idesc(C, C, 0);
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
-            uint32_t b[4];
-            ldsm_x4(b, sK + tile_off<C>(n, 16 * ks + fo));
-            mma_bf16(acc[0], af[ks], b[0], b[1]);
-            mma_bf16(acc[1], af[ks], b[2], b[3]);
+            const uint64_t dk = umma_desc(sK + (ks >> 2) * cfg::BOX_BYTES + (ks & 3) * 32, 16, 1024);
+            umma_bf16(tmem, dk, dk, idesc, ks > 0);
           }
+          umma_commit(bar_mma);
+        }
+      }
+      if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+      ph_mma ^= 1;
+      tc_fence_after();
+      if (tid == 0 && !do_wy && has_next) { issue_k(item + gridDim.x); k_requested = true; }  // K's last reader was the Gram product
+      PHASE(1);
+
+      // ---- 3. gate + mask on this warp's rows, N -> shared memory
+      const int ra = 16 * rb + g, rbw = ra + 8;
+      const float beta_a = sBeta[ra], beta_b = sBeta[rbw], g_a = sG[ra], g_b = sG[rbw];
+      {
+        float sacc[C / 8][4];   // this warp's 16 rows of S, all C columns, in one tensor-memory load
+        if constexpr (C == 64) tmem_ld_16x64(sacc, tmem_rows); else tmem_ld_16x128(sacc, tmem_rows);
+        tmem_wait_ld();
 #pragma unroll
-          for (int nt = 0; nt < 2; ++nt) {
-            const int c = 16 * jb + 8 * nt + 2 * t;
-            const float gc0 = sG[c], gc1 = sG[c + 1];
-            float2 va, vb;
-            va.x = (c < ra) ? beta_a * acc[nt][0] * __expf(g_a - gc0) : 0.f;
-            va.y = (c + 1 < ra) ? beta_a * acc[nt][1] * __expf(g_a - gc1) : 0.f;
-            vb.x = (c < rb) ? beta_b * acc[nt][2] * __expf(g_b - gc0) : 0.f;
-            vb.y = (c + 1 < rb) ? beta_b * acc[nt][3] * __expf(g_b - gc1) : 0.f;
-            *reinterpret_cast<float2*>(sX + ra * LD + c) = va;
-            *reinterpret_cast<float2*>(sX + rb * LD + c) = vb;
+        for (int jb = 0; jb < cfg::NW; ++jb) {
+          if (jb > rb) {
+            // tiles above the diagonal: exact +0.0, so the stored A and the A' operand need no masking later
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+              const int c = 16 * jb + 8 * nt + 2 * t;
+              *reinterpret_cast<float2*>(sX + ra * LD + c) = make_float2(0.f, 0.f);
+              *reinterpret_cast<float2*>(sX + rbw * LD + c) = make_float2(0.f, 0.f);
+            }
+          } else {
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+              const int c = 16 * jb + 8 * nt + 2 * t;
+              const float gc0 = sG[c], gc1 = sG[c + 1];
+              const float (&a4)[4] = sacc[2 * jb + nt];
+              float2 va, vb;
+              va.x = (c < ra) ? beta_a * a4[0] * __expf(g_a - gc0) : 0.f;
+              va.y = (c + 1 < ra) ? beta_a * a4[1] * __expf(g_a - gc1) : 0.f;
+              vb.x = (c < rbw) ? beta_b * a4[2] * __expf(g_b - gc0) : 0.f;
+              vb.y = (c + 1 < rbw) ? beta_b * a4[3] * __expf(g_b - gc1) : 0.f;
+              *reinterpret_cast<float2*>(sX + ra * LD + c) = va;
+              *reinterpret_cast<float2*>(sX + rbw * LD + c) = vb;
+            }
           }
         }
       }
       __syncwarp();
-      PHASE(1);
 
       // ---- 4. leaf: invert this warp's 16x16 diagonal block, lane j owns column j
       {
-        const int base = 16 * warp, j = lane & 15;
+        const int base = 16 * rb, j = lane & 15;
         const float* nb = sX + base * LD + base;
         float x[16];
 #pragma unroll
@@ -403,52 +503,123 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       PHASE(4);
     }
 
-    // ---- 6. store A
-    if ((p.ops & kStoreA) && p.A) {
-      for (int e = tid; e < C * (C / 4); e += cfg::NT) {
-        const int i = e / (C / 4), c4 = e - i * (C / 4);
-        if (i < rows) {
-          float4 v = *reinterpret_cast<const float4*>(sX + i * LD + 4 * c4);
-          const int j = 4 * c4;
-          v.x = (j + 0 < i) ? v.x : (j + 0 == i ? 1.f : 0.f);
-          v.y = (j + 1 < i) ? v.y : (j + 1 == i ? 1.f : 0.f);
-          v.z = (j + 2 < i) ? v.z : (j + 2 == i ? 1.f : 0.f);
-          v.w = (j + 3 < i) ? v.w : (j + 3 == i ? 1.f : 0.f);
-          *reinterpret_cast<float4*>(p.A + ((size_t)(tok0 + i) * p.H + h) * C + j) = v;
-        }
-      }
-    }
-
-    PHASE(5);
-    // ---- 7. WY apply
-    if (do_wy) {
-      uint32_t af[C / 16][4];
-      const int ra = 16 * warp + g;
+    // ---- 6. A leaves shared memory once: stored to global, and scaled by beta into the bf16 operand A'
+    constexpr int NV = C / 8;  // float4 per thread
+    float4 xv[NV];
 #pragma unroll
-      for (int ks = 0; ks < C / 16; ++ks) {
-        if (ks <= warp) {
-          const int c = 16 * ks + 2 * t;
-          const float2 b0 = *reinterpret_cast<const float2*>(sBeta + c);
-          const float2 b1 = *reinterpret_cast<const float2*>(sBeta + c + 8);
-          const float2 x00 = *reinterpret_cast<const float2*>(sX + ra * LD + c);
-          const float2 x10 = *reinterpret_cast<const float2*>(sX + (ra + 8) * LD + c);
-          const float2 x01 = *reinterpret_cast<const float2*>(sX + ra * LD + c + 8);
-          const float2 x11 = *reinterpret_cast<const float2*>(sX + (ra + 8) * LD + c + 8);
-          af[ks][0] = pack_bf16(x00.x * b0.x, x00.y * b0.y);
-          af[ks][1] = pack_bf16(x10.x * b0.x, x10.y * b0.y);
-          af[ks][2] = pack_bf16(x01.x * b1.x, x01.y * b1.y);
-          af[ks][3] = pack_bf16(x11.x * b1.x, x11.y * b1.y);
-        } else {
-          af[ks][0] = af[ks][1] = af[ks][2] = af[ks][3] = 0u;
+    for (int m = 0; m < NV; ++m) {
+      const int e = tid + m * cfg::NT;
+      const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
+      // the matrix in shared memory is complete: +0.0 above the diagonal, 1.0f on it
+      const float4 v = *reinterpret_cast<const float4*>(sX + i * LD + j);
+      xv[m] = v;
+      if ((p.ops & kStoreA) && p.A && i < rows)
+        *reinterpret_cast<float4*>(p.A + ((size_t)(tok0 + i) * p.H + h) * C + j) = v;
+    }
+    PHASE(5);
+
+    if (do_wy) {
+      tc_fence_before();
+      __syncthreads();  // every read of the fp32 matrix (and of S in TMEM) is done: its space becomes A'
+#pragma unroll
+      for (int m = 0; m < NV; ++m) {
+        const int e = tid + m * cfg::NT;
+        const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
+        const float4 b = *reinterpret_cast<const float4*>(sBeta + j);
+        const uint32_t lo = pack_bf16(xv[m].x * b.x, xv[m].y * b.y), hi = pack_bf16(xv[m].z * b.z, xv[m].w * b.w);
+        // K-major, 128-byte swizzle: row i, 64 tokens (128 B) per row and per 64-token block
+        const uint32_t off = (uint32_t)((j >> 6) * (C * 128) + i * 128 + (((((j & 63) >> 3) ^ (i & 7)) << 4) | ((j & 7) * 2)));
+        asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sAp + off), "r"(lo), "r"(hi) : "memory");
+      }
+      fence_proxy_async();  // generic-proxy writes of A' become visible to the tensor core's reads
+      __syncthreads();
+
+      // ---- 7. WY: [W | U] = A' . [K | V] with the staged tiles as the MN-major B operand
+      constexpr int NWU = (C == 64) ? 128 : 256;   // columns per MMA: C = 64 runs W then U through the same 128 columns
+      constexpr uint32_t idesc_wy = umma_idesc(C, NWU, 1);
+      auto issue_wy = [&](uint32_t b_tile) {
+#pragma unroll
+        for (int ks = 0; ks < C / 16; ++ks) {
+          const uint64_t da = umma_desc(sAp + (ks >> 2) * (C * 128) + (ks & 3) * 32, 16, 1024);
+          const uint64_t db = umma_desc(b_tile + ks * 2048, cfg::BOX_BYTES, 1024);
+          umma_bf16(tmem, da, db, idesc_wy, ks > 0);
+        }
+        umma_commit(bar_mma);
+      };
+      if (tid == 0) {
+        bool ok = mbar_wait_bounded(bar_k, ph_load);
+        if (C == 128 && need_v) ok = ok && mbar_wait_bounded(bar_v, ph_load);
+        if (!ok) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+        else { tc_fence_after(); issue_wy(sK); }
+      }
+      if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+      ph_mma ^= 1;
+      tc_fence_after();
+      // this warp's 16 rows of W leave in two 64-column pieces
+      const int row0 = 16 * rb;
+      const size_t row_stride = (size_t)p.H * D;
+      __nv_bfloat16* w_row0 = reinterpret_cast<__nv_bfloat16*>(p.W) + ((size_t)(tok0 + row0) * p.H + h) * D;
+      __nv_bfloat16* u_row0 = reinterpret_cast<__nv_bfloat16*>(p.U) + ((size_t)(tok0 + row0) * p.H + h) * D;
+      const uint32_t stage = sAp + kStageOff + warp * 2048;
+      if (C == 64 && need_v) {
+        store_piece_bf16(tmem_rows, stage, lane, w_row0, row_stride, rows - row0);
+        float f[8][4];
+        tmem_ld_16x64(f, tmem_rows + 64);
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncthreads();  // every warp holds the rest of W in registers: U may overwrite the columns
+        if (tid == 0) {
+          if (!mbar_wait_bounded(bar_v, ph_load)) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+          else { tc_fence_after(); issue_wy(sV); }
+          if (has_next) { issue_k(item + gridDim.x); k_requested = true; }  // K's last reader (the W product) is done
+        }
+        store_frag_piece_bf16(f, stage, lane, w_row0 + 64, row_stride, rows - row0);
+        if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+        ph_mma ^= 1;
+        tc_fence_after();
+        store_piece_bf16(tmem_rows, stage, lane, u_row0, row_stride, rows - row0);
+        tmem_ld_16x64(f, tmem_rows + 64);
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncthreads();  // all MMAs done and all accumulators read: tiles, A' and tensor memory are free
+        ph_load ^= 1;
+        if (has_next) {
+          if (tid == 0) { if (!k_requested) issue_k(item + gridDim.x); issue_v(item + gridDim.x); }
+          bg_next = fetch_bg(item + gridDim.x);
+        }
+        store_frag_piece_bf16(f, stage, lane, u_row0 + 64, row_stride, rows - row0);
+      } else {
+        // C = 128 (W and U side by side in 256 columns) or W only
+        store_piece_bf16(tmem_rows, stage, lane, w_row0, row_stride, rows - row0);
+        store_piece_bf16(tmem_rows + 64, stage, lane, w_row0 + 64, row_stride, rows - row0);
+        if (need_v) {
+          store_piece_bf16(tmem_rows + 128, stage, lane, u_row0, row_stride, rows - row0);
+          store_piece_bf16(tmem_rows + 192, stage, lane, u_row0 + 64, row_stride, rows - row0);
+        }
+        tc_fence_before();
+        __syncthreads();
+        ph_load ^= 1;
+        if (has_next) {
+          if (tid == 0) { issue_k(item + gridDim.x); if (need_v) issue_v(item + gridDim.x); }
+          bg_next = fetch_bg(item + gridDim.x);
         }
       }
-      wy_apply<C, D>(af, sK, warp, lane, reinterpret_cast<__nv_bfloat16*>(p.W), tok0, rows, h, p.H);
-      if (need_v) wy_apply<C, D>(af, sV, warp, lane, reinterpret_cast<__nv_bfloat16*>(p.U), tok0, rows, h, p.H);
+    } else {
+      // build only: the fp32 matrix has been read by everyone after this barrier
+      tc_fence_before();
+      __syncthreads();
+      ph_load ^= 1;
+      if (has_next) {
+        if (tid == 0 && !k_requested) issue_k(item + gridDim.x);
+        bg_next = fetch_bg(item + gridDim.x);
+      }
     }
     PHASE(6);
-    __syncthreads();  // all warps are done with the tiles and sX before the next item's copies land
-    PHASE(7);
   }
+  if (failed) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------ host side
@@ -492,11 +663,19 @@ cudaError_t launch_one(const KParams& p, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(tc_kernel<C, D>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    int dev = 0, occ = 0;
+    int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, tc_kernel<C, D>, cfg::NT, cfg::SMEM);
-    if (e != cudaSuccess) return e;
+    // Resident CTAs per SM: bounded by tensor memory (512 columns per SM, TMEM_COLS per CTA), by
+    // shared memory and by registers (128 per thread at C = 64).  The runtime's occupancy query
+    // does not model tensor-memory allocation, so the bound is taken from the layout itself.
+    int smem_per_sm = 0;
+    cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
+    int by_smem = smem_per_sm / (cfg::SMEM + 1024);  // 1 KiB per CTA is reserved by the system
+    int by_tmem = 512 / ((C == 64) ? 128 : 256);
+    int by_regs = (C == 64) ? 4 : 1;
+    int occ = by_smem < by_tmem ? by_smem : by_tmem;
+    occ = occ < by_regs ? occ : by_regs;
     ctas_per_sm = occ > 0 ? occ : 1;
   }
   long long tokens = p.chunk_tab ? (long long)p.T : (long long)p.T * (p.n_chunks / p.chunks_per_seq);
