@@ -99,6 +99,7 @@ int run(KParams p, const tri_inv_desc* d, void* stream_v) {
     if (p.n_chunks == 0) return TRI_INV_OK;
   }
 
+  if ((long long)p.n_chunks * d->H > 0x7fffffffLL) return TRI_INV_ERR_INVALID_ARG;  // kernels index work items in 32 bits
   bool handled = false;
   err = cudaSuccess;
   if (!(p.method & TRI_INV_FORCE_SIMT)) err = launch_tc(p, d->C, stream, &handled);

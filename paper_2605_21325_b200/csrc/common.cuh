@@ -41,19 +41,20 @@ struct KParams {
 };
 
 // Flat work item -> (first token, real rows, head).  Consecutive items walk the heads of
-// one chunk of tokens, so neighbouring CTAs touch neighbouring memory.
-__device__ __forceinline__ void locate(const KParams& p, int C, long long item, long long& tok0, int& rows, int& h) {
-  int c = (int)(item / p.H);
-  h = (int)(item - (long long)c * p.H);
+// one chunk of tokens, so neighbouring CTAs touch neighbouring memory.  Items and tokens are
+// below 2^31 (checked on the host), so 32-bit unsigned division is enough.
+__device__ __forceinline__ void locate(const KParams& p, int C, int item, int& tok0, int& rows, int& h) {
+  const unsigned c = (unsigned)item / (unsigned)p.H;
+  h = (int)((unsigned)item - c * (unsigned)p.H);
   if (p.chunk_tab) {
     ChunkEntry e = p.chunk_tab[c];
     tok0 = e.tok0;
     rows = e.rows;
   } else {
-    int b = c / p.chunks_per_seq;
-    int ci = c - b * p.chunks_per_seq;
-    tok0 = (long long)b * p.T + (long long)ci * C;
-    int left = p.T - ci * C;
+    const unsigned b = c / (unsigned)p.chunks_per_seq;
+    const int ci = (int)(c - b * (unsigned)p.chunks_per_seq);
+    tok0 = (int)b * p.T + ci * C;
+    const int left = p.T - ci * C;
     rows = left < C ? left : C;
   }
 }

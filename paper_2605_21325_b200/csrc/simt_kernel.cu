@@ -91,13 +91,12 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
   float* sb = Ks + C * kSliceLd;
   float* sg = sb + C;
   const int tid = threadIdx.x;
-  const long long total = (long long)p.n_chunks * p.H;
+  const int total = p.n_chunks * p.H;
   constexpr int kAcc = (C * C + kThreads - 1) / kThreads;
   const int method = p.method & TRI_INV_METHOD_MASK;
 
-  for (long long item = blockIdx.x; item < total; item += gridDim.x) {
-    long long tok0;
-    int rows, h;
+  for (int item = blockIdx.x; item < total; item += gridDim.x) {
+    int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
     __syncthreads();  // previous item's readers are done with shared memory
     for (int i = tid; i < C; i += kThreads) {

@@ -320,7 +320,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
   const bool do_wy = (p.ops & kDoWY) != 0;
   const bool need_v = do_wy && p.V != nullptr;
   const bool load_a = (p.ops & kLoadA) != 0;
-  const long long total = (long long)p.n_chunks * p.H;
+  const int total = p.n_chunks * p.H;
 
   if (tid == 0) {
     prefetch_tmap(&tmK);
@@ -345,39 +345,38 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
 
   // Thread 0 requests the tiles of an item; K and V complete on separate barriers so that the Gram
   // product can start on K alone and each buffer is refilled as soon as its last reader is done.
-  auto issue_k = [&](long long item) {
-    long long tok0; int rows, h;
+  auto issue_k = [&](int item) {
+    int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
     fence_proxy_async();
     mbar_expect_tx(bar_k, (uint32_t)cfg::TILE_BYTES);
 #pragma unroll
-    for (int bx = 0; bx < cfg::NBOX; ++bx) tma_load_2d(sK + bx * cfg::BOX_BYTES, &tmK, bar_k, h * D + 64 * bx, (int)tok0);
+    for (int bx = 0; bx < cfg::NBOX; ++bx) tma_load_2d(sK + bx * cfg::BOX_BYTES, &tmK, bar_k, h * D + 64 * bx, tok0);
   };
-  auto issue_v = [&](long long item) {
-    long long tok0; int rows, h;
+  auto issue_v = [&](int item) {
+    int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
     fence_proxy_async();
     mbar_expect_tx(bar_v, (uint32_t)cfg::TILE_BYTES);
 #pragma unroll
-    for (int bx = 0; bx < cfg::NBOX; ++bx) tma_load_2d(sV + bx * cfg::BOX_BYTES, &tmV, bar_v, h * D + 64 * bx, (int)tok0);
+    for (int bx = 0; bx < cfg::NBOX; ++bx) tma_load_2d(sV + bx * cfg::BOX_BYTES, &tmV, bar_v, h * D + 64 * bx, tok0);
   };
   // beta (threads 0..C-1) and g (threads C..2C-1) of an item, fetched one item ahead into a register
-  auto fetch_bg = [&](long long item) -> float {
-    long long tok0; int rows, h;
+  auto fetch_bg = [&](int item) -> float {
+    int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
     const int i = tid < C ? tid : tid - C;
     const float* src = tid < C ? p.beta : p.g;
     return (i < rows && src) ? src[(size_t)(tok0 + i) * p.H + h] : 0.f;
   };
   float bg_next = 0.f;
-  if ((long long)blockIdx.x < total && !misaligned) {
+  if ((int)blockIdx.x < total && !misaligned) {
     if (tid == 0) { issue_k(blockIdx.x); if (need_v) issue_v(blockIdx.x); }
     bg_next = fetch_bg(blockIdx.x);
   }
 
-  for (long long item = blockIdx.x; item < total && !misaligned; item += gridDim.x) {
-    long long tok0;
-    int rows, h;
+  for (int item = blockIdx.x; item < total && !misaligned; item += gridDim.x) {
+    int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
     PHASE_BEGIN();
 
@@ -506,6 +505,10 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
     // ---- 6. A leaves shared memory once: stored to global, and scaled by beta into the bf16 operand A'
     constexpr int NV = C / 8;  // float4 per thread
     float4 xv[NV];
+    // thread's first float4 of A: row tid / (C/4), columns 4 (tid % (C/4)); later ones are NT / (C/4) rows further down
+    const size_t a_step = (size_t)(cfg::NT / (C / 4)) * p.H * C;
+    float* a_dst = ((p.ops & kStoreA) && p.A)
+                       ? p.A + ((size_t)(tok0 + tid / (C / 4)) * p.H + h) * C + 4 * (tid % (C / 4)) : nullptr;
 #pragma unroll
     for (int m = 0; m < NV; ++m) {
       const int e = tid + m * cfg::NT;
@@ -513,8 +516,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       // the matrix in shared memory is complete: +0.0 above the diagonal, 1.0f on it
       const float4 v = *reinterpret_cast<const float4*>(sX + i * LD + j);
       xv[m] = v;
-      if ((p.ops & kStoreA) && p.A && i < rows)
-        *reinterpret_cast<float4*>(p.A + ((size_t)(tok0 + i) * p.H + h) * C + j) = v;
+      if (a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
     }
     PHASE(5);
 
