@@ -64,6 +64,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
       ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y)
       : "memory");
 }
+// Pulls a tile into L2 only (no shared memory needed): issued an item ahead so that the real
+// copy, which has to wait for its buffer, finds the data on chip.
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* tm, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(x), "r"(y) : "memory");
+}
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tm) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
@@ -77,12 +82,12 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t addr) {
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void mma_tf32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -90,6 +95,11 @@ __device__ __forceinline__ uint32_t to_tf32(float x) {
   uint32_t r;
   asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
   return r;
+}
+__device__ __forceinline__ float ex2_approx(float x) {  // 2^x, relative error about 2^-22
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -102,7 +112,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 #define PHASE(k)                                                                  \
   do {                                                                            \
     long long now = clock64();                                                    \
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(p.status + 8 + 8 * (threadIdx.x >> 5) + (k), (int)(now - ph_t)); \
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(p.status + 8 + 12 * (threadIdx.x >> 5) + (k), (int)(now - ph_t)); \
     ph_t = now;                                                                   \
   } while (0)
 #else
@@ -345,34 +355,36 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
 
   // Thread 0 requests the tiles of an item; K and V complete on separate barriers so that the Gram
   // product can start on K alone and each buffer is refilled as soon as its last reader is done.
-  auto issue_k = [&](int item) {
-    int tok0, rows, h;
-    locate(p, C, item, tok0, rows, h);
+  // The tiles of an item are requested by single threads of different warps, so that no warp carries
+  // all of the control work: K by warp 2, V by warp 3, the L2 prefetch by warp 1, the MMAs by warp 0.
+  // K and V complete on separate barriers: the Gram product starts on K alone, and each buffer is
+  // refilled as soon as its last reader is done.
+  constexpr int kTidL2 = 32, kTidK = 64, kTidV = 96;
+  auto issue_k = [&](int tok0, int h) {
     fence_proxy_async();
     mbar_expect_tx(bar_k, (uint32_t)cfg::TILE_BYTES);
 #pragma unroll
     for (int bx = 0; bx < cfg::NBOX; ++bx) tma_load_2d(sK + bx * cfg::BOX_BYTES, &tmK, bar_k, h * D + 64 * bx, tok0);
   };
-  auto issue_v = [&](int item) {
-    int tok0, rows, h;
-    locate(p, C, item, tok0, rows, h);
+  auto issue_v = [&](int tok0, int h) {
     fence_proxy_async();
     mbar_expect_tx(bar_v, (uint32_t)cfg::TILE_BYTES);
 #pragma unroll
     for (int bx = 0; bx < cfg::NBOX; ++bx) tma_load_2d(sV + bx * cfg::BOX_BYTES, &tmV, bar_v, h * D + 64 * bx, tok0);
   };
   // beta (threads 0..C-1) and g (threads C..2C-1) of an item, fetched one item ahead into a register
-  auto fetch_bg = [&](int item) -> float {
-    int tok0, rows, h;
-    locate(p, C, item, tok0, rows, h);
+  auto fetch_bg = [&](int tok0, int rows, int h) -> float {
     const int i = tid < C ? tid : tid - C;
     const float* src = tid < C ? p.beta : p.g;
     return (i < rows && src) ? src[(size_t)(tok0 + i) * p.H + h] : 0.f;
   };
   float bg_next = 0.f;
   if ((int)blockIdx.x < total && !misaligned) {
-    if (tid == 0) { issue_k(blockIdx.x); if (need_v) issue_v(blockIdx.x); }
-    bg_next = fetch_bg(blockIdx.x);
+    int tok0, rows, h;
+    locate(p, C, blockIdx.x, tok0, rows, h);
+    if (tid == kTidK) issue_k(tok0, h);
+    if (tid == kTidV && need_v) issue_v(tok0, h);
+    bg_next = fetch_bg(tok0, rows, h);
   }
 
   for (int item = blockIdx.x; item < total && !misaligned; item += gridDim.x) {
@@ -381,9 +393,19 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
     PHASE_BEGIN();
 
     // ---- 1. beta, g were fetched during the previous item (sBeta and sG are adjacent: one store each)
-    sBeta[tid] = bg_next;
+    // g is kept multiplied by log2(e) so that the gate can use ex2 directly
+    sBeta[tid] = bg_next * (tid < C ? 1.f : 1.4426950408889634f);
     const bool has_next = item + gridDim.x < total;
-    bool k_requested = false;   // thread 0: next item's K tile already requested
+    int nx_tok0 = 0, nx_rows = 0, nx_h = 0;   // the next item of this CTA
+    if (has_next) locate(p, C, item + gridDim.x, nx_tok0, nx_rows, nx_h);
+    if (tid == kTidL2 && has_next) {
+      // pull the next tiles into L2 now; the copies into shared memory follow when the buffers are free
+#pragma unroll
+      for (int bx = 0; bx < cfg::NBOX; ++bx) {
+        tma_prefetch_l2_2d(&tmK, nx_h * D + 64 * bx, nx_tok0);
+        if (need_v) tma_prefetch_l2_2d(&tmV, nx_h * D + 64 * bx, nx_tok0);
+      }
+    }
     if (load_a) {
       for (int e = tid; e < C * C; e += cfg::NT) {
         int i = e / C, j = e - i * C;
@@ -428,7 +450,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
       ph_mma ^= 1;
       tc_fence_after();
-      if (tid == 0 && !do_wy && has_next) { issue_k(item + gridDim.x); k_requested = true; }  // K's last reader was the Gram product
+      if (tid == kTidK && !do_wy && has_next) issue_k(nx_tok0, nx_h);  // K's last reader was the Gram product
       PHASE(1);
 
       // ---- 3. gate + mask on this warp's rows, N -> shared memory
@@ -452,13 +474,19 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt) {
               const int c = 16 * jb + 8 * nt + 2 * t;
-              const float gc0 = sG[c], gc1 = sG[c + 1];
+              const float2 gc = *reinterpret_cast<const float2*>(sG + c);
               const float (&a4)[4] = sacc[2 * jb + nt];
               float2 va, vb;
-              va.x = (c < ra) ? beta_a * a4[0] * __expf(g_a - gc0) : 0.f;
-              va.y = (c + 1 < ra) ? beta_a * a4[1] * __expf(g_a - gc1) : 0.f;
-              vb.x = (c < rbw) ? beta_b * a4[2] * __expf(g_b - gc0) : 0.f;
-              vb.y = (c + 1 < rbw) ? beta_b * a4[3] * __expf(g_b - gc1) : 0.f;
+              va.x = beta_a * a4[0] * ex2_approx(g_a - gc.x);
+              va.y = beta_a * a4[1] * ex2_approx(g_a - gc.y);
+              vb.x = beta_b * a4[2] * ex2_approx(g_b - gc.x);
+              vb.y = beta_b * a4[3] * ex2_approx(g_b - gc.y);
+              if (jb == rb) {  // the diagonal tile: strict-lower mask by selection
+                va.x = (c < ra) ? va.x : 0.f;
+                va.y = (c + 1 < ra) ? va.y : 0.f;
+                vb.x = (c < rbw) ? vb.x : 0.f;
+                vb.y = (c + 1 < rbw) ? vb.y : 0.f;
+              }
               *reinterpret_cast<float2*>(sX + ra * LD + c) = va;
               *reinterpret_cast<float2*>(sX + rbw * LD + c) = vb;
             }
@@ -466,6 +494,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         }
       }
       __syncwarp();
+      PHASE(2);
 
       // ---- 4. leaf: invert this warp's 16x16 diagonal block, lane j owns column j
       {
@@ -492,14 +521,14 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         }
       }
       __syncthreads();
-      PHASE(2);
+      PHASE(3);
 
       // ---- 5. merges
       merge_level<C, 16>(sX, warp, lane);
-      PHASE(3);
+      PHASE(4);
       merge_level<C, 32>(sX, warp, lane);
       if constexpr (C == 128) merge_level<C, 64>(sX, warp, lane);
-      PHASE(4);
+      PHASE(5);
     }
 
     // ---- 6. A leaves shared memory once: stored to global, and scaled by beta into the bf16 operand A'
@@ -518,7 +547,8 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       xv[m] = v;
       if (a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
     }
-    PHASE(5);
+    if (has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);  // consumed at the top of the next item
+    PHASE(6);
 
     if (do_wy) {
       tc_fence_before();
@@ -535,6 +565,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       }
       fence_proxy_async();  // generic-proxy writes of A' become visible to the tensor core's reads
       __syncthreads();
+      PHASE(7);
 
       // ---- 7. WY: [W | U] = A' . [K | V] with the staged tiles as the MN-major B operand
       constexpr int NWU = (C == 64) ? 128 : 256;   // columns per MMA: C = 64 runs W then U through the same 128 columns
@@ -557,6 +588,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
       ph_mma ^= 1;
       tc_fence_after();
+      PHASE(8);
       // this warp's 16 rows of W leave in two 64-column pieces
       const int row0 = 16 * rb;
       const size_t row_stride = (size_t)p.H * D;
@@ -573,22 +605,21 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         if (tid == 0) {
           if (!mbar_wait_bounded(bar_v, ph_load)) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
           else { tc_fence_after(); issue_wy(sV); }
-          if (has_next) { issue_k(item + gridDim.x); k_requested = true; }  // K's last reader (the W product) is done
         }
+        if (tid == kTidK && has_next) issue_k(nx_tok0, nx_h);  // K's last reader (the W product) is done
         store_frag_piece_bf16(f, stage, lane, w_row0 + 64, row_stride, rows - row0);
+        PHASE(9);
         if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
         ph_mma ^= 1;
         tc_fence_after();
+        PHASE(10);
         store_piece_bf16(tmem_rows, stage, lane, u_row0, row_stride, rows - row0);
         tmem_ld_16x64(f, tmem_rows + 64);
         tmem_wait_ld();
         tc_fence_before();
         __syncthreads();  // all MMAs done and all accumulators read: tiles, A' and tensor memory are free
         ph_load ^= 1;
-        if (has_next) {
-          if (tid == 0) { if (!k_requested) issue_k(item + gridDim.x); issue_v(item + gridDim.x); }
-          bg_next = fetch_bg(item + gridDim.x);
-        }
+        if (tid == kTidV && has_next) issue_v(nx_tok0, nx_h);
         store_frag_piece_bf16(f, stage, lane, u_row0 + 64, row_stride, rows - row0);
       } else {
         // C = 128 (W and U side by side in 256 columns) or W only
@@ -601,22 +632,17 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         tc_fence_before();
         __syncthreads();
         ph_load ^= 1;
-        if (has_next) {
-          if (tid == 0) { issue_k(item + gridDim.x); if (need_v) issue_v(item + gridDim.x); }
-          bg_next = fetch_bg(item + gridDim.x);
-        }
+        if (tid == kTidK && has_next) issue_k(nx_tok0, nx_h);
+        if (tid == kTidV && has_next && need_v) issue_v(nx_tok0, nx_h);
       }
     } else {
       // build only: the fp32 matrix has been read by everyone after this barrier
       tc_fence_before();
       __syncthreads();
       ph_load ^= 1;
-      if (has_next) {
-        if (tid == 0 && !k_requested) issue_k(item + gridDim.x);
-        bg_next = fetch_bg(item + gridDim.x);
-      }
+      if (tid == kTidK && has_next && (p.ops & kLoadA)) issue_k(nx_tok0, nx_h);  // otherwise requested after the Gram product
     }
-    PHASE(6);
+    PHASE(11);
   }
   if (failed) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
   tc_fence_before();
