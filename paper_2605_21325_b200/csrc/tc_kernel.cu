@@ -378,6 +378,17 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
     const float* src = tid < C ? p.beta : p.g;
     return (i < rows && src) ? src[(size_t)(tok0 + i) * p.H + h] : 0.f;
   };
+  // Gram S = K K^T: D/16 MMAs of C x C x 16 into the first C columns of tensor memory (thread 0)
+  auto issue_gram = [&]() {
+    constexpr uint32_t idesc = umma_idesc(C, C, 0);
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+      const uint64_t dk = umma_desc(sK + (ks >> 2) * cfg::BOX_BYTES + (ks & 3) * 32, 16, 1024);
+      umma_bf16(tmem, dk, dk, idesc, ks > 0);
+    }
+    umma_commit(bar_mma);
+  };
+  bool gram_early = false;  // thread 0: the Gram product of the coming item was already issued at the end of the last one
   float bg_next = 0.f;
   if ((int)blockIdx.x < total && !misaligned) {
     int tok0, rows, h;
@@ -398,6 +409,12 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
     const bool has_next = item + gridDim.x < total;
     int nx_tok0 = 0, nx_rows = 0, nx_h = 0;   // the next item of this CTA
     if (has_next) locate(p, C, item + gridDim.x, nx_tok0, nx_rows, nx_h);
+    if (has_next) {
+      // next item's beta / g element of this thread: into L2 now, into a register later
+      const int i = tid < C ? tid : tid - C;
+      const float* src = tid < C ? p.beta : p.g;
+      if (i < nx_rows && src) asm volatile("prefetch.global.L2 [%0];" ::"l"(src + (size_t)(nx_tok0 + i) * p.H + nx_h));
+    }
     if (tid == kTidL2 && has_next) {
       // pull the next tiles into L2 now; the copies into shared memory follow when the buffers are free
 #pragma unroll
@@ -433,20 +450,15 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
 
     if (!load_a) {
       // ---- 2. Gram S = K K^T on the tensor core: one thread issues D/16 MMAs of C x C x 16 into TMEM
-      if (tid == 0) {
+      if (tid == 0 && !gram_early) {
         if (!mbar_wait_bounded(bar_k, ph_load)) {
           atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);  // the other threads time out on bar_mma
         } else {
           tc_fence_after();
-          constexpr uint32_t idesc = umma_idesc(C, C, 0);
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            const uint64_t dk = umma_desc(sK + (ks >> 2) * cfg::BOX_BYTES + (ks & 3) * 32, 16, 1024);
-            umma_bf16(tmem, dk, dk, idesc, ks > 0);
-          }
-          umma_commit(bar_mma);
+          issue_gram();
         }
       }
+      gram_early = false;
       if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
       ph_mma ^= 1;
       tc_fence_after();
@@ -547,7 +559,6 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       xv[m] = v;
       if (a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
     }
-    if (has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);  // consumed at the top of the next item
     PHASE(6);
 
     if (do_wy) {
@@ -566,6 +577,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       fence_proxy_async();  // generic-proxy writes of A' become visible to the tensor core's reads
       __syncthreads();
       PHASE(7);
+      if (has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);  // consumed at the top of the next item
 
       // ---- 7. WY: [W | U] = A' . [K | V] with the staged tiles as the MN-major B operand
       constexpr int NWU = (C == 64) ? 128 : 256;   // columns per MMA: C = 64 runs W then U through the same 128 columns
@@ -596,31 +608,39 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       __nv_bfloat16* u_row0 = reinterpret_cast<__nv_bfloat16*>(p.U) + ((size_t)(tok0 + row0) * p.H + h) * D;
       const uint32_t stage = sAp + kStageOff + warp * 2048;
       if (C == 64 && need_v) {
-        store_piece_bf16(tmem_rows, stage, lane, w_row0, row_stride, rows - row0);
-        float f[8][4];
-        tmem_ld_16x64(f, tmem_rows + 64);
+        float f0[8][4], f1[8][4];
+        tmem_ld_16x64(f0, tmem_rows);
+        tmem_ld_16x64(f1, tmem_rows + 64);
         tmem_wait_ld();
         tc_fence_before();
-        __syncthreads();  // every warp holds the rest of W in registers: U may overwrite the columns
+        __syncthreads();  // every warp holds its rows of W in registers: U may overwrite the columns
         if (tid == 0) {
           if (!mbar_wait_bounded(bar_v, ph_load)) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
           else { tc_fence_after(); issue_wy(sV); }
         }
         if (tid == kTidK && has_next) issue_k(nx_tok0, nx_h);  // K's last reader (the W product) is done
-        store_frag_piece_bf16(f, stage, lane, w_row0 + 64, row_stride, rows - row0);
+        store_frag_piece_bf16(f0, stage, lane, w_row0, row_stride, rows - row0);
+        store_frag_piece_bf16(f1, stage, lane, w_row0 + 64, row_stride, rows - row0);
         PHASE(9);
         if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
         ph_mma ^= 1;
         tc_fence_after();
         PHASE(10);
-        store_piece_bf16(tmem_rows, stage, lane, u_row0, row_stride, rows - row0);
-        tmem_ld_16x64(f, tmem_rows + 64);
+        tmem_ld_16x64(f0, tmem_rows);
+        tmem_ld_16x64(f1, tmem_rows + 64);
         tmem_wait_ld();
         tc_fence_before();
         __syncthreads();  // all MMAs done and all accumulators read: tiles, A' and tensor memory are free
         ph_load ^= 1;
         if (tid == kTidV && has_next) issue_v(nx_tok0, nx_h);
-        store_frag_piece_bf16(f, stage, lane, u_row0 + 64, row_stride, rows - row0);
+        if (tid == 0 && has_next && nx_rows == C && !load_a && mbar_try_wait(bar_k, ph_load)) {
+          // the next K tile has landed and tensor memory is free: start the next Gram product now
+          tc_fence_after();
+          issue_gram();
+          gram_early = true;
+        }
+        store_frag_piece_bf16(f0, stage, lane, u_row0, row_stride, rows - row0);
+        store_frag_piece_bf16(f1, stage, lane, u_row0 + 64, row_stride, rows - row0);
       } else {
         // C = 128 (W and U side by side in 256 columns) or W only
         store_piece_bf16(tmem_rows, stage, lane, w_row0, row_stride, rows - row0);
@@ -637,10 +657,17 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       }
     } else {
       // build only: the fp32 matrix has been read by everyone after this barrier
+      if (has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);
       tc_fence_before();
       __syncthreads();
       ph_load ^= 1;
       if (tid == kTidK && has_next && (p.ops & kLoadA)) issue_k(nx_tok0, nx_h);  // otherwise requested after the Gram product
+      if (tid == 0 && has_next && nx_rows == C && !load_a && mbar_try_wait(bar_k, ph_load)) {
+        // the next K tile has landed and tensor memory is free: start the next Gram product now
+        tc_fence_after();
+        issue_gram();
+        gram_early = true;
+      }
     }
     PHASE(11);
   }
