@@ -36,7 +36,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per chunk matrix moved by the fused kernel (dram__bytes_read.sum + dram__bytes_write.sum
 # of one ncu capture divided by the matrices of that launch); see profiles/.  None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_MATRIX = {}
+NCU_TRAFFIC_BYTES_PER_MATRIX = {(2, "block_recursive"): 68960}  # profiles/tc_kernel_c64_cfg2.md
 
 
 def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True):
@@ -129,6 +129,24 @@ def time_oracle(inp, target_seconds=15.0, n_threads=0):
     return {"value": n / t, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": "first %d tokens of each of the %d sequences of %s, %d passes (%d chunk matrices, %.1f s; build + WY in fp64)"
                       % (chunks * inp.C, inp.B, inp.name, passes, n, t)}, n, t
+
+
+def reduce_max(value: float, device="cpu") -> float:
+    """Max over ranks of a host scalar (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(local_ms_per_step: float, matrices_per_rank: int, world: int, device="cpu"):
+    """Whole-job value under weak scaling: every rank processed `matrices_per_rank` per step and the job
+    runs at the pace of its slowest rank."""
+    ms = reduce_max(local_ms_per_step, device)
+    return world * matrices_per_rank / (ms * 1e-3), ms
 
 
 def run_reference(args):
@@ -254,13 +272,8 @@ def main():
     launches = binding.launch_count() - launches0
     times_ms = [a.elapsed_time(b) for a, b in evs]
     total_ms = sum(times_ms)
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
     clocks = sampler.stop() if rank == 0 else None
-    ms_per_step = total_ms / args.steps
-    value = world * n_mat / (ms_per_step * 1e-3)
+    value, ms_per_step = aggregate_throughput(total_ms / args.steps, n_mat, world, "cuda")
 
     # ---- end to end through the public API with host buffers: H2D of the inputs, kernel, D2H of A, W, U
     hK, hV = binding.kv_to_torch(inp.K, "cpu", pin=True), binding.kv_to_torch(inp.V, "cpu", pin=True)
@@ -287,12 +300,7 @@ def main():
         e2e_step()
     e1.record(stream)
     torch.cuda.synchronize()
-    e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * n_mat * e2e_steps / (e2e_ms * 1e-3)
+    e2e_value, _ = aggregate_throughput(e0.elapsed_time(e1) / e2e_steps, n_mat, world, "cuda")
 
     # ---- accuracy of what was just timed, on a sample the oracle computes directly
     err = None
