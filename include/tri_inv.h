@@ -58,7 +58,8 @@ enum {
   TRI_INV_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, bad size, bad cu_seqlens */
   TRI_INV_ERR_UNSUPPORTED = 2,   /* a valid request this build has no kernel for */
   TRI_INV_ERR_CUDA = 3,          /* a CUDA runtime call or the launch failed */
-  TRI_INV_ERR_DEVICE_TIMEOUT = 4 /* a bounded device-side wait expired (see tri_inv_last_device_status) */
+  TRI_INV_ERR_DEVICE_TIMEOUT = 4,/* a bounded device-side wait expired (see tri_inv_last_device_status) */
+  TRI_INV_ERR_TOO_LARGE = 5      /* more chunks than the fixed scratch of tri_inv_fused_packed_static holds */
 };
 
 /* ---- storage type of K, V, W, U ------------------------------------------ */
@@ -125,6 +126,32 @@ int tri_inv_wy(const float* A, const void* K, const void* V, const float* beta,
 int tri_inv_fused(const void* K, const void* V, const float* beta, const float* g,
                   float* A, void* W, void* U,
                   const tri_inv_desc* desc, int method, void* cuda_stream);
+
+/*
+ * Packed-sequence fused call that allocates nothing.  (The paper has no counterpart: this is a
+ * deployment variant of tri_inv_fused, not a step of the method.)
+ *
+ * tri_inv_fused in packed mode (cu_seqlens != NULL) keeps a small table of chunk positions in device
+ * memory that it allocates and frees on the stream.  Callers that may not allocate -- code that runs
+ * where cudaMalloc is forbidden or would stall, a process with a memory budget fixed at start-up, a
+ * host whose allocator belongs to another component -- can use this entry point instead: the table
+ * lives in a fixed device array inside the library (128 KiB, held by every GPU that loads the library
+ * until the process exits).  No cudaMalloc, cudaFree or other allocating call is made; inputs and
+ * outputs are the caller's, exactly as for tri_inv_fused, and results are identical.
+ *
+ *   - Packed mode only: desc->cu_seqlens must be non-NULL (dense calls never allocate; use tri_inv_fused).
+ *   - At most TRI_INV_STATIC_MAX_CHUNKS chunks of tokens (sum over sequences of ceil(len / C));
+ *     more returns TRI_INV_ERR_TOO_LARGE and does nothing.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside of any stream capture.
+ *   - All calls share the one array.  Two calls whose kernels can overlap on the GPU (different
+ *     streams, or the same stream from different host threads without ordering) race on it: order
+ *     them.  Calls on one stream are safe.  Host threads are serialised while the table is filled.
+ */
+#define TRI_INV_STATIC_MAX_CHUNKS 16384
+int tri_inv_fused_packed_static(const void* K, const void* V, const float* beta, const float* g,
+                                float* A, void* W, void* U,
+                                const tri_inv_desc* desc, int method, void* cuda_stream);
 
 /*
  * Number of chunk matrices (chunks x heads) the descriptor describes.

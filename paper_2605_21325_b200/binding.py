@@ -19,13 +19,14 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libtri_inv.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT = 0, 1, 2, 3, 4
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_TOO_LARGE = 0, 1, 2, 3, 4, 5
+STATIC_MAX_CHUNKS = 16384
 F32, BF16 = 0, 1
 BLOCK_RECURSIVE, PRODUCT_SERIES = 0, 1
 LEAF_SERIES = 0x100
 FORCE_SIMT = 0x10000
 
-EXPORTS = ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_count_matrices",
+EXPORTS = ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
            "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
 
 
@@ -57,6 +58,8 @@ def load():
         lib.tri_inv_build.argtypes = [vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_wy.argtypes = [vp, vp, vp, vp, vp, vp, dp, vp]
         lib.tri_inv_fused.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
+        lib.tri_inv_fused_packed_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
+        lib.tri_inv_fused_packed_static.restype = i32
         lib.tri_inv_count_matrices.argtypes = [dp, ctypes.POINTER(ctypes.c_int64)]
         lib.tri_inv_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
         for f in ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_count_matrices", "tri_inv_last_device_status"):
@@ -164,6 +167,23 @@ def fused(K, V, beta, g, C, method=BLOCK_RECURSIVE, cu_seqlens=None, want_A=True
     rc = load().tri_inv_fused(_p(K), _p(V), _p(beta), _p(g), _p(A), _p(W), _p(U), ctypes.byref(desc), int(method), _stream(stream))
     if rc != OK:
         raise TriInvError("tri_inv_fused", rc)
+    return A, W, U
+
+
+def fused_packed_static(K, V, beta, g, C, cu_seqlens, method=BLOCK_RECURSIVE, out=None, stream=None):
+    """Packed-sequence fused call through the entry point that makes no allocation of its own
+    (the chunk table sits in a fixed array inside the library).  ``out`` = (A or None, W, U) must be
+    given by callers that really cannot allocate; without it the outputs are allocated here with torch."""
+    B, T, H, d_k = K.shape
+    d_v = V.shape[-1]
+    desc, keep = make_desc(B, T, H, d_k, d_v, C, _dtype_code(K), cu_seqlens)
+    if out is None:
+        out = (torch.zeros((B, T, H, C), dtype=torch.float32, device=K.device), torch.zeros_like(K), torch.zeros_like(V))
+    A, W, U = out
+    rc = load().tri_inv_fused_packed_static(_p(K), _p(V), _p(beta), _p(g), _p(A), _p(W), _p(U), ctypes.byref(desc),
+                                            int(method), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_fused_packed_static", rc)
     return A, W, U
 
 

@@ -12,6 +12,8 @@ __device__ int g_device_status[128] = {0};  // word 0: raised by kernels that gi
 
 std::atomic<long long> g_launches{0};
 
+}  // namespace
+
 int* status_word_for_current_device(cudaError_t* err) {
   // One address per device; looked up once per device under a lock.
   static std::mutex mu;
@@ -29,6 +31,10 @@ int* status_word_for_current_device(cudaError_t* err) {
   }
   return cache[dev];
 }
+
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -215,6 +221,7 @@ const char* tri_inv_status_string(int status) {
     case TRI_INV_ERR_UNSUPPORTED: return "unsupported request";
     case TRI_INV_ERR_CUDA: return "CUDA runtime error";
     case TRI_INV_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case TRI_INV_ERR_TOO_LARGE: return "more chunks than the static scratch table holds";
     default: return "unknown status";
   }
 }

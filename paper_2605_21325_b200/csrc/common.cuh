@@ -69,4 +69,10 @@ cudaError_t launch_simt(const KParams& p, int C, cudaStream_t stream);
 // Tensor-core path: returns cudaErrorNotSupported when it has no kernel for the request.
 cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
 
+// Adds one to the library's launch counter (tri_inv_launch_count).
+void count_launch();
+
+// Address of the device status word (0 = ok) of the current device; nullptr and *err on failure.
+int* status_word_for_current_device(cudaError_t* err);
+
 }  // namespace tri_inv
