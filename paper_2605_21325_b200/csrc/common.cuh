@@ -32,6 +32,7 @@ struct KParams {
   void* U;
   const ChunkEntry* chunk_tab;  // ragged mode, else nullptr
   int* status;                  // device status word (0 = ok); kernels only ever raise it
+  int* work_counter;            // tensor-core kernel: {next dynamic item, finished CTAs}; both zero between launches
   int32_t H, d_k, d_v, T;
   int32_t chunks_per_seq;       // dense mode: ceil(T / C)
   int32_t n_chunks;             // token chunks (all sequences); matrices = n_chunks * H

@@ -108,6 +108,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // Optional per-phase cycle counters (development builds only: -DTRI_INV_PHASE_CLOCKS).
 #ifdef TRI_INV_PHASE_CLOCKS
+__device__ unsigned long long g_cta_times[4096 * 4];
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+__device__ __forceinline__ unsigned smid() { unsigned r; asm volatile("mov.u32 %0, %%smid;" : "=r"(r)); return r; }
+#define CTA_MARK(k) do { if (threadIdx.x == 0 && blockIdx.x < 4096) g_cta_times[blockIdx.x * 4 + (k)] = (k) == 3 ? smid() : gtime(); } while (0)
 #define PHASE_BEGIN() long long ph_t = clock64()
 #define PHASE(k)                                                                  \
   do {                                                                            \
@@ -116,6 +120,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     ph_t = now;                                                                   \
   } while (0)
 #else
+#define CTA_MARK(k) do {} while (0)
 #define PHASE_BEGIN() do {} while (0)
 #define PHASE(k) do {} while (0)
 #endif
@@ -314,6 +319,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
   float* sBeta = reinterpret_cast<float*>(smem + cfg::OFF_BETA);
   float* sG = reinterpret_cast<float*>(smem + cfg::OFF_G);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 24);
+  volatile int* s_next_item = reinterpret_cast<volatile int*>(smem + cfg::OFF_BAR + 28);
   const uint32_t sK = smem_u32(smem + cfg::OFF_K);
   const uint32_t sV = smem_u32(smem + cfg::OFF_V);
   const uint32_t sAp = smem_u32(smem + cfg::OFF_X);  // A' = A diag(beta) in bf16 reuses the N/X matrix's space
@@ -323,6 +329,8 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
+  CTA_MARK(0);
+  CTA_MARK(3);
   // Row block of this warp.  TMEM lanes are reachable only from the warp whose id % 4 matches
   // the 32-lane quadrant: M = 64 puts rows 16q..16q+15 in lanes 32q..32q+15, M = 128 puts row i in lane i.
   const int rb = (C == 64) ? warp : 2 * (warp & 3) + (warp >> 2);
@@ -331,27 +339,6 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
   const bool need_v = do_wy && p.V != nullptr;
   const bool load_a = (p.ops & kLoadA) != 0;
   const int total = p.n_chunks * p.H;
-
-  if (tid == 0) {
-    prefetch_tmap(&tmK);
-    if (need_v) prefetch_tmap(&tmV);
-    mbar_init(bar_k, 1);
-    mbar_init(bar_v, 1);
-    mbar_init(bar_mma, 1);
-    fence_mbar_init();
-  }
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
-  const bool misaligned = (sK & 1023u) != 0;  // never expected; the swizzle pattern would not match the copies
-  const uint32_t tmem_rows = tmem + (lane_base << 16);
-  uint32_t ph_load = 0, ph_mma = 0;
-  bool failed = misaligned;
 
   // Thread 0 requests the tiles of an item; K and V complete on separate barriers so that the Gram
   // product can start on K alone and each buffer is refilled as soon as its last reader is done.
@@ -378,6 +365,44 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
     const float* src = tid < C ? p.beta : p.g;
     return (i < rows && src) ? src[(size_t)(tok0 + i) * p.H + h] : 0.f;
   };
+  // Prologue.  The threads that own the K and V barriers initialise them and request the first
+  // item's tiles at once, so that the copies run while tensor memory is being allocated.
+  const bool misaligned = (sK & 1023u) != 0;  // never expected; the swizzle pattern would not match the copies
+  float bg_next = 0.f;
+  {
+    int tok0 = 0, rows = 0, h = 0;
+    const bool any = (int)blockIdx.x < total && !misaligned;
+    if (any) locate(p, C, blockIdx.x, tok0, rows, h);
+    if (tid == kTidK) {
+      prefetch_tmap(&tmK);
+      mbar_init(bar_k, 1);
+      fence_mbar_init();
+      if (any) issue_k(tok0, h);
+    }
+    if (tid == kTidV) {
+      if (need_v) prefetch_tmap(&tmV);
+      mbar_init(bar_v, 1);
+      fence_mbar_init();
+      if (any && need_v) issue_v(tok0, h);
+    }
+    if (tid == 0) {
+      mbar_init(bar_mma, 1);
+      fence_mbar_init();
+    }
+    if (any) bg_next = fetch_bg(tok0, rows, h);
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem_rows = tmem + (lane_base << 16);
+  uint32_t ph_load = 0, ph_mma = 0;
+  bool failed = misaligned;
+
   // Gram S = K K^T: D/16 MMAs of C x C x 16 into the first C columns of tensor memory (thread 0)
   auto issue_gram = [&]() {
     constexpr uint32_t idesc = umma_idesc(C, C, 0);
@@ -389,16 +414,11 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
     umma_commit(bar_mma);
   };
   bool gram_early = false;  // thread 0: the Gram product of the coming item was already issued at the end of the last one
-  float bg_next = 0.f;
-  if ((int)blockIdx.x < total && !misaligned) {
-    int tok0, rows, h;
-    locate(p, C, blockIdx.x, tok0, rows, h);
-    if (tid == kTidK) issue_k(tok0, h);
-    if (tid == kTidV && need_v) issue_v(tok0, h);
-    bg_next = fetch_bg(tok0, rows, h);
-  }
-
-  for (int item = blockIdx.x; item < total && !misaligned; item += gridDim.x) {
+  // Work distribution: the first two items of a CTA are fixed (blockIdx, blockIdx + grid), every
+  // later one comes from a device counter, fetched one item ahead of its use so that prefetches
+  // know their target.  SMs that run faster simply take more items.
+  int item = blockIdx.x, nx_item = blockIdx.x + gridDim.x;
+  while (item < total && !misaligned) {
     int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
     PHASE_BEGIN();
@@ -406,9 +426,9 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
     // ---- 1. beta, g were fetched during the previous item (sBeta and sG are adjacent: one store each)
     // g is kept multiplied by log2(e) so that the gate can use ex2 directly
     sBeta[tid] = bg_next * (tid < C ? 1.f : 1.4426950408889634f);
-    const bool has_next = item + gridDim.x < total;
+    const bool has_next = nx_item < total;
     int nx_tok0 = 0, nx_rows = 0, nx_h = 0;   // the next item of this CTA
-    if (has_next) locate(p, C, item + gridDim.x, nx_tok0, nx_rows, nx_h);
+    if (has_next) locate(p, C, nx_item, nx_tok0, nx_rows, nx_h);
     if (has_next) {
       // next item's beta / g element of this thread: into L2 now, into a register later
       const int i = tid < C ? tid : tid - C;
@@ -446,6 +466,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       fence_proxy_async();
     }
     __syncthreads();
+    if (tid == kTidL2) *s_next_item = has_next ? 2 * (int)gridDim.x + atomicAdd(p.work_counter, 1) : total;  // the item after next
     PHASE(0);
 
     if (!load_a) {
@@ -557,7 +578,8 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       // the matrix in shared memory is complete: +0.0 above the diagonal, 1.0f on it
       const float4 v = *reinterpret_cast<const float4*>(sX + i * LD + j);
       xv[m] = v;
-      if (a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
+      // without a WY product there is nothing to overlap the stores with: issue them right away
+      if (!do_wy && a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
     }
     PHASE(6);
 
@@ -596,6 +618,14 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         if (C == 128 && need_v) ok = ok && mbar_wait_bounded(bar_v, ph_load);
         if (!ok) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
         else { tc_fence_after(); issue_wy(sK); }
+      }
+      // A goes to global memory while the W product runs (its registers are free again before W returns)
+      if (a_dst) {
+#pragma unroll
+        for (int m = 0; m < NV; ++m) {
+          const int i = (tid + m * cfg::NT) / (C / 4);
+          if (i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = xv[m];
+        }
       }
       if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
       ph_mma ^= 1;
@@ -670,6 +700,15 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       }
     }
     PHASE(11);
+    item = nx_item;
+    nx_item = *s_next_item;  // written early in this item, several barriers ago
+  }
+  CTA_MARK(2);
+  if (tid == 0 && atomicAdd(p.work_counter + 1, 1) == (int)gridDim.x - 1) {
+    // last CTA out: leave both counters at zero for the next launch that uses this slot
+    p.work_counter[0] = 0;
+    p.work_counter[1] = 0;
+    __threadfence();
   }
   if (failed) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
   tc_fence_before();
@@ -709,9 +748,31 @@ bool make_tmap(CUtensorMap* tm, const void* base, long long tokens, int H, int d
   return r == CUDA_SUCCESS;
 }
 
+// Work counters: 64 pairs per device, handed out round-robin so that launches that overlap on
+// different streams do not share one.  Each pair is returned to zero by the kernel that used it.
+__device__ int g_work_counters[64 * 2];
+
+int* next_work_counter() {
+  static std::mutex mu;
+  static int* base[64] = {nullptr};
+  static unsigned turn = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!base[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_work_counters) != cudaSuccess) return nullptr;
+    base[dev] = static_cast<int*>(ptr);
+  }
+  return base[dev] + 2 * (turn++ % 64);
+}
+
 template <int C, int D>
-cudaError_t launch_one(const KParams& p, cudaStream_t stream) {
+cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   using cfg = Cfg<C, D>;
+  KParams p = p_in;
+  p.work_counter = next_work_counter();
+  if (!p.work_counter) return cudaErrorUnknown;
   static int ctas_per_sm = 0, n_sm = 0;
   if (!ctas_per_sm) {
     cudaError_t e = cudaFuncSetAttribute(tc_kernel<C, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
@@ -746,6 +807,12 @@ cudaError_t launch_one(const KParams& p, cudaStream_t stream) {
 }
 
 }  // namespace
+
+#ifdef TRI_INV_PHASE_CLOCKS
+extern "C" int tri_inv_debug_cta_times(unsigned long long* out, int n) {
+  return cudaMemcpyFromSymbol(out, g_cta_times, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : 3;
+}
+#endif
 
 cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled) {
   *handled = false;
