@@ -140,7 +140,9 @@ struct Cfg {
   static constexpr int OFF_BETA = OFF_X + C * LD * 4;
   static constexpr int OFF_G = OFF_BETA + C * 4;
   static constexpr int OFF_BAR = OFF_G + C * 4;
-  static constexpr int BYTES = OFF_BAR + 32;     // two mbarriers and the TMEM base-address slot
+  static constexpr int OFF_LEAF = OFF_BAR + 32;  // three mbarriers, the TMEM base-address slot, the next-item slot
+  static constexpr int LEAF_LD = 20;             // per-warp 16 x 16 fp32 scratch of the series leaf
+  static constexpr int BYTES = OFF_LEAF + NW * 16 * LEAF_LD * 4;
   static constexpr int SMEM = BYTES;
 };
 
@@ -149,6 +151,75 @@ template <int C>
 __device__ __forceinline__ uint32_t tile_off(int r, int f) {
   int box = f >> 6, c = (f & 63) >> 3;
   return (uint32_t)(box * (C * 128) + r * 128 + ((c ^ (r & 7)) << 4));
+}
+
+// 16x16 leaf by the product series (Alg. 5 on the leaf, the first phase of Alg. 2): X <- I - N, Y <- N,
+// three rounds of Y <- Y.Y, X <- X + X.Y as TF32 m16n8k8 MMAs.  X lives in the leaf's place inside the
+// fp32 matrix (row length LDX), Y in a per-warp scratch (row length LDY); both are re-read as operands.
+template <int LDX, int LDY>
+__device__ __forceinline__ void leaf_series(float* xblk, float* ys, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  float x[2][4], y[2][4];
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    const int c = 8 * nt + 2 * t;
+    const float2 na = *reinterpret_cast<const float2*>(xblk + g * LDX + c);
+    const float2 nb = *reinterpret_cast<const float2*>(xblk + (g + 8) * LDX + c);
+    y[nt][0] = na.x; y[nt][1] = na.y; y[nt][2] = nb.x; y[nt][3] = nb.y;
+    x[nt][0] = (c == g ? 1.f : 0.f) - na.x;
+    x[nt][1] = (c + 1 == g ? 1.f : 0.f) - na.y;
+    x[nt][2] = (c == g + 8 ? 1.f : 0.f) - nb.x;
+    x[nt][3] = (c + 1 == g + 8 ? 1.f : 0.f) - nb.y;
+  }
+  __syncwarp();
+  auto put = [&](float* dst, int ld, const float (&v)[2][4]) {
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+      const int c = 8 * nt + 2 * t;
+      *reinterpret_cast<float2*>(dst + g * ld + c) = make_float2(v[nt][0], v[nt][1]);
+      *reinterpret_cast<float2*>(dst + (g + 8) * ld + c) = make_float2(v[nt][2], v[nt][3]);
+    }
+  };
+  // acc += P . Q for 16x16 matrices in shared memory
+  auto mm = [&](float (&acc)[2][4], const float* pm, int ldp, const float* qm, int ldq) {
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const float* ap = pm + g * ldp + 8 * q + t;
+      const uint32_t a0 = to_tf32(ap[0]), a1 = to_tf32(ap[8 * ldp]), a2 = to_tf32(ap[4]), a3 = to_tf32(ap[8 * ldp + 4]);
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        const float* bp = qm + (8 * q + t) * ldq + 8 * nt + g;
+        mma_tf32(acc[nt], a0, a1, a2, a3, to_tf32(bp[0]), to_tf32(bp[4 * ldq]));
+      }
+    }
+  };
+  put(ys, LDY, y);
+  put(xblk, LDX, x);
+  __syncwarp();
+#pragma unroll
+  for (int r = 0; r < 3; ++r) {
+    float y2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    mm(y2, ys, LDY, ys, LDY);   // Y <- Y.Y
+    __syncwarp();               // every lane has read the old Y
+    put(ys, LDY, y2);
+    __syncwarp();
+    mm(x, xblk, LDX, ys, LDY);  // X <- X + X.Y (the accumulator starts as X)
+    __syncwarp();               // every lane has read the old X
+    put(xblk, LDX, x);
+    __syncwarp();
+  }
+  // exact structure of a unit lower triangular block: constants on and above the diagonal
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+    const int c = 8 * nt + 2 * t;
+    float2 va = *reinterpret_cast<float2*>(xblk + g * LDX + c), vb = *reinterpret_cast<float2*>(xblk + (g + 8) * LDX + c);
+    va.x = (c < g) ? va.x : (c == g ? 1.f : 0.f);
+    va.y = (c + 1 < g) ? va.y : (c + 1 == g ? 1.f : 0.f);
+    vb.x = (c < g + 8) ? vb.x : (c == g + 8 ? 1.f : 0.f);
+    vb.y = (c + 1 < g + 8) ? vb.y : (c + 1 == g + 8 ? 1.f : 0.f);
+    *reinterpret_cast<float2*>(xblk + g * LDX + c) = va;
+    *reinterpret_cast<float2*>(xblk + (g + 8) * LDX + c) = vb;
+  }
 }
 
 // One merge level of the block recursion: for every adjacent pair of B x B diagonal blocks,
@@ -529,8 +600,11 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       __syncwarp();
       PHASE(2);
 
-      // ---- 4. leaf: invert this warp's 16x16 diagonal block, lane j owns column j
-      {
+      // ---- 4. leaf: invert this warp's 16x16 diagonal block
+      if (p.method & TRI_INV_LEAF_SERIES) {
+        leaf_series<LD, cfg::LEAF_LD>(sX + 16 * rb * LD + 16 * rb,
+                                      reinterpret_cast<float*>(smem + cfg::OFF_LEAF) + warp * 16 * cfg::LEAF_LD, lane);
+      } else {  // forward substitution, lane j owns column j
         const int base = 16 * rb, j = lane & 15;
         const float* nb = sX + base * LD + base;
         float x[16];
@@ -817,7 +891,7 @@ extern "C" int tri_inv_debug_cta_times(unsigned long long* out, int n) {
 cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled) {
   *handled = false;
   if (p.kv_dtype != TRI_INV_BF16) return cudaSuccess;
-  if ((p.method & TRI_INV_METHOD_MASK) != TRI_INV_BLOCK_RECURSIVE || (p.method & TRI_INV_LEAF_SERIES)) return cudaSuccess;
+  if ((p.method & TRI_INV_METHOD_MASK) != TRI_INV_BLOCK_RECURSIVE) return cudaSuccess;
   if (p.d_k != 128 || ((p.ops & kDoWY) && p.V && p.d_v != 128)) return cudaSuccess;
   // the stride of the 2-D view (H * d * 2 bytes) is a multiple of 16 because d is a multiple of 8
   *handled = true;
