@@ -126,7 +126,7 @@ __device__ __forceinline__ unsigned smid() { unsigned r; asm volatile("mov.u32 %
 #endif
 
 // ------------------------------------------------------------------------------------------ layout
-template <int C, int D>
+template <int C, int D, bool SER>
 struct Cfg {
   static constexpr int NW = C / 16;             // warps, one per 16 rows
   static constexpr int NT = NW * 32;
@@ -142,8 +142,11 @@ struct Cfg {
   static constexpr int OFF_BAR = OFF_G + C * 4;
   static constexpr int OFF_LEAF = OFF_BAR + 32;  // three mbarriers, the TMEM base-address slot, the next-item slot
   static constexpr int LEAF_LD = 20;             // per-warp 16 x 16 fp32 scratch of the series leaf
-  static constexpr int BYTES = OFF_LEAF + NW * 16 * LEAF_LD * 4;
+  // product-series variant at C = 128: X needs a buffer of its own (at C = 64 it fits where the V tile was)
+  static constexpr int OFF_XS = (OFF_LEAF + NW * 16 * LEAF_LD * 4 + 1023) / 1024 * 1024;
+  static constexpr int BYTES = (SER && C == 128) ? OFF_XS + C * C * 4 : OFF_LEAF + NW * 16 * LEAF_LD * 4;
   static constexpr int SMEM = BYTES;
+  static constexpr int CTAS_PER_SM = (C == 64) ? 4 : 1;
 };
 
 // Byte offset of the 16-byte chunk holding features [f, f+8) of row r inside a swizzled tile.
@@ -302,6 +305,17 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// kind::tf32: fp32 data in shared memory read as TF32, fp32 accumulate, K = 8 per instruction.
+__host__ __device__ constexpr uint32_t umma_idesc_tf32(int M, int N, int b_mn) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -376,15 +390,15 @@ __device__ __forceinline__ void store_piece_bf16(uint32_t taddr, uint32_t stage,
   store_frag_piece_bf16(f, stage, lane, out_row0, row_stride, rows_left);
 }
 
-template <int C, int D>
-__global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(const __grid_constant__ CUtensorMap tmK,
+template <int C, int D, bool SER>
+__global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                              const __grid_constant__ CUtensorMap tmV, KParams p) {
-  using cfg = Cfg<C, D>;
+  using cfg = Cfg<C, D, SER>;
   static_assert(D == 128, "tiles are two 64-feature boxes wide");
   constexpr int LD = cfg::LD;
   constexpr int TMEM_COLS = (C == 64) ? 128 : 256;
   constexpr int kStageOff = C * C * 2;  // per-warp 2 KiB output staging tiles sit behind A' in the N/X matrix's space
-  static_assert(kStageOff + Cfg<C, D>::NW * 2048 <= C * Cfg<C, D>::LD * 4, "staging must fit behind A'");
+  static_assert(kStageOff + cfg::NW * 2048 <= C * cfg::LD * 4, "staging must fit behind A'");
   extern __shared__ __align__(1024) uint8_t smem[];  // swizzled tiles need a 1024-byte aligned base
   float* sX = reinterpret_cast<float*>(smem + cfg::OFF_X);
   float* sBeta = reinterpret_cast<float*>(smem + cfg::OFF_BETA);
@@ -454,7 +468,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       if (need_v) prefetch_tmap(&tmV);
       mbar_init(bar_v, 1);
       fence_mbar_init();
-      if (any && need_v) issue_v(tok0, h);
+      if (any && need_v && !SER) issue_v(tok0, h);  // the series variant loads V after the inversion
     }
     if (tid == 0) {
       mbar_init(bar_mma, 1);
@@ -471,7 +485,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tmem_rows = tmem + (lane_base << 16);
-  uint32_t ph_load = 0, ph_mma = 0;
+  uint32_t ph_k = 0, ph_v = 0, ph_mma = 0;  // parities of the next completion to wait for on each barrier
   bool failed = misaligned;
 
   // Gram S = K K^T: D/16 MMAs of C x C x 16 into the first C columns of tensor memory (thread 0)
@@ -522,11 +536,11 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         sX[i * LD + j] = v;
       }
     }
-    if (rows < C) {
-      // rows past the sequence end hold a neighbour's tokens (or zero fill): clear them before any MMA
-      if (!mbar_wait_bounded(bar_k, ph_load) || (need_v && !mbar_wait_bounded(bar_v, ph_load))) { failed = true; break; }
+    // rows past the sequence end hold a neighbour's tokens (or zero fill): they are cleared before any MMA
+    auto clear_tail_rows = [&](bool k_tile, bool v_tile) {
       for (int e = tid; e < (C - rows) * 8 * cfg::NBOX * 2; e += cfg::NT) {
         int which = e / ((C - rows) * 8 * cfg::NBOX);
+        if (which ? !v_tile : !k_tile) continue;
         int rem = e - which * (C - rows) * 8 * cfg::NBOX;
         int bx = rem / ((C - rows) * 8);
         int rem2 = rem - bx * (C - rows) * 8;
@@ -535,6 +549,11 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         *reinterpret_cast<uint4*>(base) = make_uint4(0, 0, 0, 0);
       }
       fence_proxy_async();
+    };
+    if (rows < C) {
+      const bool v_now = need_v && !SER;
+      if (!mbar_wait_bounded(bar_k, ph_k) || (v_now && !mbar_wait_bounded(bar_v, ph_v))) { failed = true; break; }
+      clear_tail_rows(true, v_now);
     }
     __syncthreads();
     if (tid == kTidL2) *s_next_item = has_next ? 2 * (int)gridDim.x + atomicAdd(p.work_counter, 1) : total;  // the item after next
@@ -543,7 +562,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
     if (!load_a) {
       // ---- 2. Gram S = K K^T on the tensor core: one thread issues D/16 MMAs of C x C x 16 into TMEM
       if (tid == 0 && !gram_early) {
-        if (!mbar_wait_bounded(bar_k, ph_load)) {
+        if (!mbar_wait_bounded(bar_k, ph_k)) {
           atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);  // the other threads time out on bar_mma
         } else {
           tc_fence_after();
@@ -554,9 +573,148 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
       ph_mma ^= 1;
       tc_fence_after();
-      if (tid == kTidK && !do_wy && has_next) issue_k(nx_tok0, nx_h);  // K's last reader was the Gram product
+      if (tid == kTidK && !do_wy && !SER && has_next) issue_k(nx_tok0, nx_h);  // K's last reader was the Gram product
       PHASE(1);
 
+      if constexpr (SER) {
+        // ---- 3'. product series (Alg. 5) on the tensor core.  Y (= N at first) and X (= I - N at first)
+        // are kept in shared memory as fp32 K-major swizzled operands (32 floats per 128-byte row, blocks of
+        // 32 columns); one stored copy of Y serves as the A operand (K-major) and as the B operand
+        // (MN-major).  Step s issues Y.Y (for s < R) and X.Y (for s >= 1) together: the squaring of round
+        // s + 1 does not depend on the X update of round s (App. D.1), so they share one round trip.
+        constexpr int R = (C == 64) ? 5 : 6;  // log2(C) - 1 rounds
+        // Operand storage during the series: Y in the space of the fp32 result matrix (written last),
+        // Y^T where the K tile was and X where the V tile was (C = 128: Y^T over both tiles, X in a buffer of
+        // its own) -- the Gram product is done with K, and K and V are fetched (again) for the WY step afterwards.  TF32 operands must be K-major here:
+        // Y is the A operand of Y.Y, X the A operand of X.Y, and Y^T (rows = columns of Y) the B operand.
+        uint8_t* yb = smem + cfg::OFF_X;
+        uint8_t* ytb = smem + cfg::OFF_K;
+        uint8_t* xb = smem + (C == 64 ? cfg::OFF_V : cfg::OFF_XS);
+        const uint32_t sYb = smem_u32(yb), sYtb = smem_u32(ytb), sXb = smem_u32(xb);
+        auto canon = [](int r, int c) -> uint32_t {  // byte offset of element (r, c) in the swizzled fp32 operand layout
+          return (uint32_t)((c >> 5) * (C * 128) + r * 128 + (((((c & 31) >> 2) ^ (r & 7)) << 4) | ((c & 3) * 4)));
+        };
+        const int ra = 16 * rb + g, rbw = ra + 8;
+        const float beta_a = sBeta[ra], beta_b = sBeta[rbw], g_a = sG[ra], g_b = sG[rbw];
+        float xr[C / 8][4];  // this warp's 16 rows of X, accumulator-fragment layout, kept across rounds
+        // rows ra, rbw of Y (pairs of columns) and the same values into Y^T (column ra / rbw of rows c, c+1)
+        auto put_y = [&](int c, float2 ya, float2 yw) {
+          *reinterpret_cast<float2*>(yb + canon(ra, c)) = ya;
+          *reinterpret_cast<float2*>(yb + canon(rbw, c)) = yw;
+          *reinterpret_cast<float*>(ytb + canon(c, ra)) = ya.x;
+          *reinterpret_cast<float*>(ytb + canon(c + 1, ra)) = ya.y;
+          *reinterpret_cast<float*>(ytb + canon(c, rbw)) = yw.x;
+          *reinterpret_cast<float*>(ytb + canon(c + 1, rbw)) = yw.y;
+        };
+        {
+          float sacc[C / 8][4];
+          if constexpr (C == 64) tmem_ld_16x64(sacc, tmem_rows); else tmem_ld_16x128(sacc, tmem_rows);
+          tmem_wait_ld();
+#pragma unroll
+          for (int nt = 0; nt < C / 8; ++nt) {
+            const int c = 8 * nt + 2 * t;
+            float2 na = make_float2(0.f, 0.f), nb = na;
+            if (nt / 2 <= rb) {  // tiles on or below the diagonal of this row block
+              const float2 gc = *reinterpret_cast<const float2*>(sG + c);
+              na.x = (c < ra) ? beta_a * sacc[nt][0] * ex2_approx(g_a - gc.x) : 0.f;
+              na.y = (c + 1 < ra) ? beta_a * sacc[nt][1] * ex2_approx(g_a - gc.y) : 0.f;
+              nb.x = (c < rbw) ? beta_b * sacc[nt][2] * ex2_approx(g_b - gc.x) : 0.f;
+              nb.y = (c + 1 < rbw) ? beta_b * sacc[nt][3] * ex2_approx(g_b - gc.y) : 0.f;
+            }
+            xr[nt][0] = (c == ra ? 1.f : 0.f) - na.x;
+            xr[nt][1] = (c + 1 == ra ? 1.f : 0.f) - na.y;
+            xr[nt][2] = (c == rbw ? 1.f : 0.f) - nb.x;
+            xr[nt][3] = (c + 1 == rbw ? 1.f : 0.f) - nb.y;
+            put_y(c, na, nb);
+            *reinterpret_cast<float2*>(xb + canon(ra, c)) = make_float2(xr[nt][0], xr[nt][1]);
+            *reinterpret_cast<float2*>(xb + canon(rbw, c)) = make_float2(xr[nt][2], xr[nt][3]);
+          }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        constexpr uint32_t idesc_s = umma_idesc_tf32(C, C, 0);
+        bool dead = false;
+#pragma unroll 1
+        for (int s = 0; s <= R; ++s) {
+          if (tid == 0) {
+            tc_fence_after();
+            if (s < R) {
+#pragma unroll
+              for (int ks = 0; ks < C / 8; ++ks) {
+                const uint32_t koff = (ks >> 2) * (C * 128) + (ks & 3) * 32;
+                umma_tf32(tmem, umma_desc(sYb + koff, 16, 1024), umma_desc(sYtb + koff, 16, 1024), idesc_s, ks > 0);
+              }
+            }
+            if (s >= 1) {
+#pragma unroll
+              for (int ks = 0; ks < C / 8; ++ks) {
+                const uint32_t koff = (ks >> 2) * (C * 128) + (ks & 3) * 32;
+                umma_tf32(tmem + C, umma_desc(sXb + koff, 16, 1024), umma_desc(sYtb + koff, 16, 1024), idesc_s, ks > 0);
+              }
+            }
+            umma_commit(bar_mma);
+          }
+          if (!mbar_wait_bounded(bar_mma, ph_mma)) { dead = true; break; }
+          ph_mma ^= 1;
+          tc_fence_after();
+          if (s < R) {  // Y <- Y.Y, written over the old Y and Y^T (their readers, the MMAs, have completed)
+            float yn[C / 8][4];
+            if constexpr (C == 64) tmem_ld_16x64(yn, tmem_rows); else tmem_ld_16x128(yn, tmem_rows);
+            tmem_wait_ld();
+#pragma unroll
+            for (int nt = 0; nt < C / 8; ++nt)
+              put_y(8 * nt + 2 * t, make_float2(yn[nt][0], yn[nt][1]), make_float2(yn[nt][2], yn[nt][3]));
+          }
+          if (s >= 1) {  // X <- X + X.Y
+            float xn[C / 8][4];
+            if constexpr (C == 64) tmem_ld_16x64(xn, tmem_rows + C); else tmem_ld_16x128(xn, tmem_rows + C);
+            tmem_wait_ld();
+#pragma unroll
+            for (int nt = 0; nt < C / 8; ++nt) {
+              const int c = 8 * nt + 2 * t;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) xr[nt][e] += xn[nt][e];
+              if (s < R) {
+                *reinterpret_cast<float2*>(xb + canon(ra, c)) = make_float2(xr[nt][0], xr[nt][1]);
+                *reinterpret_cast<float2*>(xb + canon(rbw, c)) = make_float2(xr[nt][2], xr[nt][3]);
+              }
+            }
+          }
+          if (s < R) {
+            fence_proxy_async();
+            tc_fence_before();
+            __syncthreads();
+          }
+        }
+        if (dead) { failed = true; break; }
+        // the result goes to the fp32 matrix used by the store and WY steps; the structure of a unit lower
+        // triangular matrix is written as constants
+#pragma unroll
+        for (int nt = 0; nt < C / 8; ++nt) {
+          const int c = 8 * nt + 2 * t;
+          float2 va, vb;
+          va.x = (c < ra) ? xr[nt][0] : (c == ra ? 1.f : 0.f);
+          va.y = (c + 1 < ra) ? xr[nt][1] : (c + 1 == ra ? 1.f : 0.f);
+          vb.x = (c < rbw) ? xr[nt][2] : (c == rbw ? 1.f : 0.f);
+          vb.y = (c + 1 < rbw) ? xr[nt][3] : (c + 1 == rbw ? 1.f : 0.f);
+          *reinterpret_cast<float2*>(sX + ra * LD + c) = va;
+          *reinterpret_cast<float2*>(sX + rbw * LD + c) = vb;
+        }
+        tc_fence_before();
+        __syncthreads();
+        if (do_wy) {
+          // K and V come (back) into their tiles for the WY step
+          if (tid == kTidK) issue_k(tok0, h);
+          if (tid == kTidV && need_v) issue_v(tok0, h);
+          ph_k ^= 1;
+          if (rows < C) {
+            if (!mbar_wait_bounded(bar_k, ph_k) || (need_v && !mbar_wait_bounded(bar_v, ph_v))) { failed = true; break; }
+            clear_tail_rows(true, need_v);
+            __syncthreads();
+          }
+        }
+      } else {
       // ---- 3. gate + mask on this warp's rows, N -> shared memory
       const int ra = 16 * rb + g, rbw = ra + 8;
       const float beta_a = sBeta[ra], beta_b = sBeta[rbw], g_a = sG[ra], g_b = sG[rbw];
@@ -636,6 +794,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
       merge_level<C, 32>(sX, warp, lane);
       if constexpr (C == 128) merge_level<C, 64>(sX, warp, lane);
       PHASE(5);
+      }
     }
 
     // ---- 6. A leaves shared memory once: stored to global, and scaled by beta into the bf16 operand A'
@@ -688,8 +847,8 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         umma_commit(bar_mma);
       };
       if (tid == 0) {
-        bool ok = mbar_wait_bounded(bar_k, ph_load);
-        if (C == 128 && need_v) ok = ok && mbar_wait_bounded(bar_v, ph_load);
+        bool ok = mbar_wait_bounded(bar_k, ph_k);
+        if (C == 128 && need_v) ok = ok && mbar_wait_bounded(bar_v, ph_v);
         if (!ok) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
         else { tc_fence_after(); issue_wy(sK); }
       }
@@ -719,7 +878,7 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         tc_fence_before();
         __syncthreads();  // every warp holds its rows of W in registers: U may overwrite the columns
         if (tid == 0) {
-          if (!mbar_wait_bounded(bar_v, ph_load)) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+          if (!mbar_wait_bounded(bar_v, ph_v)) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
           else { tc_fence_after(); issue_wy(sV); }
         }
         if (tid == kTidK && has_next) issue_k(nx_tok0, nx_h);  // K's last reader (the W product) is done
@@ -735,9 +894,10 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         tmem_wait_ld();
         tc_fence_before();
         __syncthreads();  // all MMAs done and all accumulators read: tiles, A' and tensor memory are free
-        ph_load ^= 1;
-        if (tid == kTidV && has_next) issue_v(nx_tok0, nx_h);
-        if (tid == 0 && has_next && nx_rows == C && !load_a && mbar_try_wait(bar_k, ph_load)) {
+        ph_k ^= 1;
+        ph_v ^= 1;
+        if (tid == kTidV && has_next && !SER) issue_v(nx_tok0, nx_h);
+        if (tid == 0 && has_next && nx_rows == C && !load_a && mbar_try_wait(bar_k, ph_k)) {
           // the next K tile has landed and tensor memory is free: start the next Gram product now
           tc_fence_after();
           issue_gram();
@@ -755,18 +915,20 @@ __global__ void __launch_bounds__(Cfg<C, D>::NT, (C == 64 ? 4 : 1)) tc_kernel(co
         }
         tc_fence_before();
         __syncthreads();
-        ph_load ^= 1;
+        ph_k ^= 1;
+        ph_v ^= 1;
         if (tid == kTidK && has_next) issue_k(nx_tok0, nx_h);
-        if (tid == kTidV && has_next && need_v) issue_v(nx_tok0, nx_h);
+        if (tid == kTidV && has_next && need_v && !SER) issue_v(nx_tok0, nx_h);
       }
     } else {
       // build only: the fp32 matrix has been read by everyone after this barrier
       if (has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);
       tc_fence_before();
       __syncthreads();
-      ph_load ^= 1;
-      if (tid == kTidK && has_next && (p.ops & kLoadA)) issue_k(nx_tok0, nx_h);  // otherwise requested after the Gram product
-      if (tid == 0 && has_next && nx_rows == C && !load_a && mbar_try_wait(bar_k, ph_load)) {
+      ph_k ^= 1;
+      ph_v ^= 1;
+      if (tid == kTidK && has_next && ((p.ops & kLoadA) || SER)) issue_k(nx_tok0, nx_h);  // otherwise requested after the Gram product
+      if (tid == 0 && has_next && nx_rows == C && !load_a && mbar_try_wait(bar_k, ph_k)) {
         // the next K tile has landed and tensor memory is free: start the next Gram product now
         tc_fence_after();
         issue_gram();
@@ -841,17 +1003,17 @@ int* next_work_counter() {
   return base[dev] + 2 * (turn++ % 64);
 }
 
-template <int C, int D>
+template <int C, int D, bool SER>
 cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
-  using cfg = Cfg<C, D>;
+  using cfg = Cfg<C, D, SER>;
   KParams p = p_in;
   p.work_counter = next_work_counter();
   if (!p.work_counter) return cudaErrorUnknown;
   static int ctas_per_sm = 0, n_sm = 0;
   if (!ctas_per_sm) {
-    cudaError_t e = cudaFuncSetAttribute(tc_kernel<C, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
+    cudaError_t e = cudaFuncSetAttribute(tc_kernel<C, D, SER>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(tc_kernel<C, D>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    e = cudaFuncSetAttribute(tc_kernel<C, D, SER>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -863,7 +1025,7 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
     cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
     int by_smem = smem_per_sm / (cfg::SMEM + 1024);  // 1 KiB per CTA is reserved by the system
     int by_tmem = 512 / ((C == 64) ? 128 : 256);
-    int by_regs = (C == 64) ? 4 : 1;
+    int by_regs = cfg::CTAS_PER_SM;
     int occ = by_smem < by_tmem ? by_smem : by_tmem;
     occ = occ < by_regs ? occ : by_regs;
     ctas_per_sm = occ > 0 ? occ : 1;
@@ -876,7 +1038,7 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   long long total = (long long)p.n_chunks * p.H;
   long long cap = (long long)n_sm * ctas_per_sm;
   int grid = (int)(total < cap ? total : cap);
-  tc_kernel<C, D><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
+  tc_kernel<C, D, SER><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
   return cudaGetLastError();
 }
 
@@ -891,12 +1053,12 @@ extern "C" int tri_inv_debug_cta_times(unsigned long long* out, int n) {
 cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled) {
   *handled = false;
   if (p.kv_dtype != TRI_INV_BF16) return cudaSuccess;
-  if ((p.method & TRI_INV_METHOD_MASK) != TRI_INV_BLOCK_RECURSIVE) return cudaSuccess;
+  const bool series = (p.method & TRI_INV_METHOD_MASK) == TRI_INV_PRODUCT_SERIES;
   if (p.d_k != 128 || ((p.ops & kDoWY) && p.V && p.d_v != 128)) return cudaSuccess;
   // the stride of the 2-D view (H * d * 2 bytes) is a multiple of 16 because d is a multiple of 8
   *handled = true;
-  if (C == 64) return launch_one<64, 128>(p, stream);
-  if (C == 128) return launch_one<128, 128>(p, stream);
+  if (C == 64) return series ? launch_one<64, 128, true>(p, stream) : launch_one<64, 128, false>(p, stream);
+  if (C == 128) return series ? launch_one<128, 128, true>(p, stream) : launch_one<128, 128, false>(p, stream);
   *handled = false;
   return cudaSuccess;
 }
