@@ -1,23 +1,26 @@
-// Tensor-core kernel for bf16 keys/values (sm_100a).
+// Tensor-core kernel for bf16 keys/values, d = 128, C = 64 or 128 (sm_100a).
 //
-// One CTA works on one chunk matrix at a time (grid-stride over all (chunk, head) items),
-// one warp per 16 rows.  Per item:
-//   1. TMA (cp.async.bulk.tensor, 128-byte swizzle) stages the C x d tiles of K and V in
-//      shared memory; beta and g come in with plain loads.
-//   2. Gram S = K K^T: tcgen05.mma (kind::f16, bf16 operands straight from the TMA-written tiles,
+// One CTA works on one chunk matrix at a time (first two items fixed, later ones from a device
+// counter), one warp per 16 rows, 4 CTAs per SM at C = 64.  Per item:
+//   1. TMA (cp.async.bulk.tensor, 128-byte swizzle) stages the C x d tiles of K and V in shared
+//      memory on separate mbarriers; the next item's tiles are prefetched into L2 an item ahead and
+//      copied as soon as a buffer's last reader has finished; beta and g travel one item ahead in a register.
+//   2. Gram S = K K^T: tcgen05.mma (kind::f16, bf16 operands straight from the TMA-written tile,
 //      fp32 accumulator in tensor memory), issued by one thread, completion through an mbarrier.
 //   3. Each warp reads its 16 rows of S from tensor memory (tcgen05.ld 16x256b: the m16n8 accumulator
 //      fragment layout), applies gate + strict-lower mask, writes N to shared memory in fp32.
-//   4. 16x16 leaves inverted by forward substitution, one lane per column (Sec. 3.1).
-//   5. Block-recursive merges X21 = -(X22 N21) X11 for b = 16, 32, (64) as TF32 MMAs
-//      (m16n8k8, fp32 accumulate) on fp32 data kept in shared memory (Sec. 3.3).
-//   6. A stored with 16-byte coalesced stores; upper triangle and diagonal are constants.
-//   7. A' = A diag(beta) is written as a bf16 K-major swizzled operand over the fp32 matrix's space;
-//      W = A' K and U = A' V are tcgen05.mma with the K / V tiles still in shared memory as the
-//      MN-major B operand; accumulators come back from tensor memory and leave as 16-byte stores.
-//   The next item's tiles are requested as soon as the last MMA of this item has completed.
-// Inputs of the inversion stay fp32 in shared memory; only the Gram product and the WY
-// apply see bf16 operands (the Gram operands are the bf16 inputs themselves, so exact).
+//   4. Block recursion (Sec. 3.3): 16x16 leaves by forward substitution, one lane per column (Sec. 3.1),
+//      or by the product series on the leaf (Alg. 2); merges X21 = -(X22 N21) X11 for b = 16, 32, (64)
+//      as TF32 m16n8k8 MMAs on fp32 data in shared memory.
+//      Product-series variant (Alg. 5): Y.Y and X.Y as tcgen05.mma kind::tf32 on fp32 operands kept in
+//      shared memory, accumulators in tensor memory, log2(C) round trips.
+//   5. A' = A diag(beta) is written as a bf16 K-major swizzled operand over the fp32 matrix's space;
+//      W = A' K and U = A' V are tcgen05.mma with the K / V tiles as the MN-major B operand; A goes to
+//      global memory with 16-byte coalesced stores while the W product runs.
+//   6. W and U come back from tensor memory, are packed to bf16, transposed through a per-warp swizzled
+//      staging tile with stmatrix and leave as 16-byte stores covering 128 contiguous bytes per row.
+// Every mbarrier wait is bounded; on expiry the kernel raises the status word, frees its tensor
+// memory and returns.
 #include <cuda.h>
 
 #include <mutex>
@@ -73,19 +76,6 @@ __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tm) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
 
-__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 __device__ __forceinline__ void mma_tf32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
   asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
@@ -323,13 +313,6 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// 16 lanes x 16 columns: the accumulator fragment of two adjacent m16n8 tiles
-// (regs 0..3: columns 0..7, regs 4..7: columns 8..15; thread t: rows t/4 and t/4+8, columns 2(t%4), +1).
-__device__ __forceinline__ void tmem_ld_16x16(float (&r)[2][4], uint32_t taddr) {
-  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=f"(r[0][0]), "=f"(r[0][1]), "=f"(r[0][2]), "=f"(r[0][3]), "=f"(r[1][0]), "=f"(r[1][1]), "=f"(r[1][2]), "=f"(r[1][3])
-               : "r"(taddr));
-}
 // 16 lanes x 64 columns -> 8 n-tiles of accumulator fragments.
 __device__ __forceinline__ void tmem_ld_16x64(float (&r)[8][4], uint32_t taddr) {
   asm volatile(
