@@ -124,19 +124,35 @@ struct Cfg {
   static constexpr int NBOX = D / 64;           // TMA boxes per tile: 64 features (128 B) wide
   static constexpr int BOX_BYTES = C * 128;
   static constexpr int TILE_BYTES = NBOX * BOX_BYTES;
+  // Block recursion at C = 128: the K / V tiles share the space of the fp32 N/X matrix (K is only needed
+  // for the Gram product before N is written, and both tiles are fetched again, from L2, for the WY step),
+  // which brings the CTA under half an SM's shared memory: two CTAs per SM instead of one.
+  static constexpr bool ALIAS = (C == 128) && !SER;
+  static constexpr bool RELOAD = SER || ALIAS;    // K (and V) are requested after the inversion
   static constexpr int OFF_K = 0;
   static constexpr int OFF_V = TILE_BYTES;
-  static constexpr int OFF_X = 2 * TILE_BYTES;
-  static constexpr int OFF_BETA = OFF_X + C * LD * 4;
+  static constexpr int X_BYTES = C * LD * 4;
+  static constexpr int OFF_X = ALIAS ? 0 : 2 * TILE_BYTES;
+  // A' (bf16, C x C) and the per-warp 2 KiB output staging tiles: inside the N/X matrix's space once it has
+  // been read (A' first, staging behind it), or, with ALIAS, in a region of their own where the staging
+  // reuses A' after the WY products have completed.
+  static constexpr int OFF_AP = ALIAS ? (X_BYTES + 1023) / 1024 * 1024 : OFF_X;
+  static constexpr int OFF_STAGE = ALIAS ? OFF_AP : OFF_AP + C * C * 2;
+  static_assert(ALIAS || C * C * 2 + NW * 2048 <= X_BYTES, "A' and staging must fit in the N/X matrix's space");
+  static_assert(NW * 2048 <= C * C * 2, "staging must fit in A'");
+  static constexpr int OFF_BETA = ALIAS ? OFF_AP + C * C * 2 : OFF_X + X_BYTES;
   static constexpr int OFF_G = OFF_BETA + C * 4;
   static constexpr int OFF_BAR = OFF_G + C * 4;
-  static constexpr int OFF_LEAF = OFF_BAR + 32;  // three mbarriers, the TMEM base-address slot, the next-item slot
   static constexpr int LEAF_LD = 20;             // per-warp 16 x 16 fp32 scratch of the series leaf
+  static constexpr int LEAF_BYTES = NW * 16 * LEAF_LD * 4;
+  // three mbarriers, the TMEM base-address slot, the next-item slot, then the leaf scratch (inside A' with ALIAS)
+  static constexpr int OFF_LEAF = ALIAS ? OFF_AP : OFF_BAR + 32;
+  static constexpr int END_PLAIN = ALIAS ? OFF_BAR + 32 : OFF_LEAF + LEAF_BYTES;
   // product-series variant at C = 128: X needs a buffer of its own (at C = 64 it fits where the V tile was)
-  static constexpr int OFF_XS = (OFF_LEAF + NW * 16 * LEAF_LD * 4 + 1023) / 1024 * 1024;
-  static constexpr int BYTES = (SER && C == 128) ? OFF_XS + C * C * 4 : OFF_LEAF + NW * 16 * LEAF_LD * 4;
+  static constexpr int OFF_XS = (END_PLAIN + 1023) / 1024 * 1024;
+  static constexpr int BYTES = (SER && C == 128) ? OFF_XS + C * C * 4 : END_PLAIN;
   static constexpr int SMEM = BYTES;
-  static constexpr int CTAS_PER_SM = (C == 64) ? 4 : 1;
+  static constexpr int CTAS_PER_SM = (C == 64) ? 4 : (ALIAS ? 2 : 1);
 };
 
 // Byte offset of the 16-byte chunk holding features [f, f+8) of row r inside a swizzled tile.
@@ -380,8 +396,6 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
   static_assert(D == 128, "tiles are two 64-feature boxes wide");
   constexpr int LD = cfg::LD;
   constexpr int TMEM_COLS = (C == 64) ? 128 : 256;
-  constexpr int kStageOff = C * C * 2;  // per-warp 2 KiB output staging tiles sit behind A' in the N/X matrix's space
-  static_assert(kStageOff + cfg::NW * 2048 <= C * cfg::LD * 4, "staging must fit behind A'");
   extern __shared__ __align__(1024) uint8_t smem[];  // swizzled tiles need a 1024-byte aligned base
   float* sX = reinterpret_cast<float*>(smem + cfg::OFF_X);
   float* sBeta = reinterpret_cast<float*>(smem + cfg::OFF_BETA);
@@ -390,7 +404,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
   volatile int* s_next_item = reinterpret_cast<volatile int*>(smem + cfg::OFF_BAR + 28);
   const uint32_t sK = smem_u32(smem + cfg::OFF_K);
   const uint32_t sV = smem_u32(smem + cfg::OFF_V);
-  const uint32_t sAp = smem_u32(smem + cfg::OFF_X);  // A' = A diag(beta) in bf16 reuses the N/X matrix's space
+  const uint32_t sAp = smem_u32(smem + cfg::OFF_AP);  // A' = A diag(beta), bf16 K-major swizzled operand
   const uint32_t bar_k = smem_u32(smem + cfg::OFF_BAR);  // K tile landed
   const uint32_t bar_mma = bar_k + 8;                    // a batch of MMAs completed
   const uint32_t bar_v = bar_k + 16;                     // V tile landed
@@ -445,13 +459,13 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
       prefetch_tmap(&tmK);
       mbar_init(bar_k, 1);
       fence_mbar_init();
-      if (any) issue_k(tok0, h);
+      if (any && !(cfg::ALIAS && load_a)) issue_k(tok0, h);  // with ALIAS, tri_inv_wy fills the matrix first and fetches K later
     }
     if (tid == kTidV) {
       if (need_v) prefetch_tmap(&tmV);
       mbar_init(bar_v, 1);
       fence_mbar_init();
-      if (any && need_v && !SER) issue_v(tok0, h);  // the series variant loads V after the inversion
+      if (any && need_v && !cfg::RELOAD) issue_v(tok0, h);  // otherwise V is requested after the inversion
     }
     if (tid == 0) {
       mbar_init(bar_mma, 1);
@@ -534,9 +548,9 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
       fence_proxy_async();
     };
     if (rows < C) {
-      const bool v_now = need_v && !SER;
-      if (!mbar_wait_bounded(bar_k, ph_k) || (v_now && !mbar_wait_bounded(bar_v, ph_v))) { failed = true; break; }
-      clear_tail_rows(true, v_now);
+      const bool v_now = need_v && !cfg::RELOAD, k_now = !(cfg::ALIAS && load_a);
+      if ((k_now && !mbar_wait_bounded(bar_k, ph_k)) || (v_now && !mbar_wait_bounded(bar_v, ph_v))) { failed = true; break; }
+      clear_tail_rows(k_now, v_now);
     }
     __syncthreads();
     if (tid == kTidL2) *s_next_item = has_next ? 2 * (int)gridDim.x + atomicAdd(p.work_counter, 1) : total;  // the item after next
@@ -556,7 +570,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
       if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
       ph_mma ^= 1;
       tc_fence_after();
-      if (tid == kTidK && !do_wy && !SER && has_next) issue_k(nx_tok0, nx_h);  // K's last reader was the Gram product
+      if (tid == kTidK && !do_wy && !cfg::RELOAD && has_next) issue_k(nx_tok0, nx_h);  // K's last reader was the Gram product
       PHASE(1);
 
       if constexpr (SER) {
@@ -782,38 +796,67 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
 
     // ---- 6. A leaves shared memory once: stored to global, and scaled by beta into the bf16 operand A'
     constexpr int NV = C / 8;  // float4 per thread
-    float4 xv[NV];
     // thread's first float4 of A: row tid / (C/4), columns 4 (tid % (C/4)); later ones are NT / (C/4) rows further down
     const size_t a_step = (size_t)(cfg::NT / (C / 4)) * p.H * C;
     float* a_dst = ((p.ops & kStoreA) && p.A)
                        ? p.A + ((size_t)(tok0 + tid / (C / 4)) * p.H + h) * C + 4 * (tid % (C / 4)) : nullptr;
-#pragma unroll
-    for (int m = 0; m < NV; ++m) {
-      const int e = tid + m * cfg::NT;
-      const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
-      // the matrix in shared memory is complete: +0.0 above the diagonal, 1.0f on it
-      const float4 v = *reinterpret_cast<const float4*>(sX + i * LD + j);
-      xv[m] = v;
-      // without a WY product there is nothing to overlap the stores with: issue them right away
-      if (!do_wy && a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
-    }
-    PHASE(6);
-
-    if (do_wy) {
-      tc_fence_before();
-      __syncthreads();  // every read of the fp32 matrix (and of S in TMEM) is done: its space becomes A'
+    // bf16 pair stores of one float4 of A scaled by beta: K-major, 128-byte swizzle, 64 tokens per row block
+    auto put_ap = [&](int i, int j, const float4& v) {
+      const float4 b = *reinterpret_cast<const float4*>(sBeta + j);
+      const uint32_t lo = pack_bf16(v.x * b.x, v.y * b.y), hi = pack_bf16(v.z * b.z, v.w * b.w);
+      const uint32_t off = (uint32_t)((j >> 6) * (C * 128) + i * 128 + (((((j & 63) >> 3) ^ (i & 7)) << 4) | ((j & 7) * 2)));
+      asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sAp + off), "r"(lo), "r"(hi) : "memory");
+    };
+    float4 xv[cfg::ALIAS ? 1 : NV];
+    if constexpr (cfg::ALIAS) {
+      // A' has a region of its own: one pass reads the matrix, stores A and writes A'
 #pragma unroll
       for (int m = 0; m < NV; ++m) {
         const int e = tid + m * cfg::NT;
         const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
-        const float4 b = *reinterpret_cast<const float4*>(sBeta + j);
-        const uint32_t lo = pack_bf16(xv[m].x * b.x, xv[m].y * b.y), hi = pack_bf16(xv[m].z * b.z, xv[m].w * b.w);
-        // K-major, 128-byte swizzle: row i, 64 tokens (128 B) per row and per 64-token block
-        const uint32_t off = (uint32_t)((j >> 6) * (C * 128) + i * 128 + (((((j & 63) >> 3) ^ (i & 7)) << 4) | ((j & 7) * 2)));
-        asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sAp + off), "r"(lo), "r"(hi) : "memory");
+        const float4 v = *reinterpret_cast<const float4*>(sX + i * LD + j);
+        if (a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
+        if (do_wy) put_ap(i, j, v);
       }
-      fence_proxy_async();  // generic-proxy writes of A' become visible to the tensor core's reads
-      __syncthreads();
+    } else {
+#pragma unroll
+      for (int m = 0; m < NV; ++m) {
+        const int e = tid + m * cfg::NT;
+        const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
+        // the matrix in shared memory is complete: +0.0 above the diagonal, 1.0f on it
+        const float4 v = *reinterpret_cast<const float4*>(sX + i * LD + j);
+        xv[m] = v;
+        // without a WY product there is nothing to overlap the stores with: issue them right away
+        if (!do_wy && a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
+      }
+    }
+    PHASE(6);
+
+    if (do_wy) {
+      if constexpr (cfg::ALIAS) {
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();  // the fp32 matrix has been read by everyone: K and V may land in its space
+        if (tid == kTidK) issue_k(tok0, h);
+        if (tid == kTidV && need_v) issue_v(tok0, h);
+        if (!load_a) ph_k ^= 1;  // second K copy of this item
+        if (rows < C) {
+          if (!mbar_wait_bounded(bar_k, ph_k) || (need_v && !mbar_wait_bounded(bar_v, ph_v))) { failed = true; break; }
+          clear_tail_rows(true, need_v);
+          __syncthreads();
+        }
+      } else {
+        tc_fence_before();
+        __syncthreads();  // every read of the fp32 matrix (and of S in TMEM) is done: its space becomes A'
+#pragma unroll
+        for (int m = 0; m < NV; ++m) {
+          const int e = tid + m * cfg::NT;
+          const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
+          put_ap(i, j, xv[m]);
+        }
+        fence_proxy_async();  // generic-proxy writes of A' become visible to the tensor core's reads
+        __syncthreads();
+      }
       PHASE(7);
       if (has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);  // consumed at the top of the next item
 
@@ -836,7 +879,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
         else { tc_fence_after(); issue_wy(sK); }
       }
       // A goes to global memory while the W product runs (its registers are free again before W returns)
-      if (a_dst) {
+      if (!cfg::ALIAS && a_dst) {
 #pragma unroll
         for (int m = 0; m < NV; ++m) {
           const int i = (tid + m * cfg::NT) / (C / 4);
@@ -852,7 +895,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
       const size_t row_stride = (size_t)p.H * D;
       __nv_bfloat16* w_row0 = reinterpret_cast<__nv_bfloat16*>(p.W) + ((size_t)(tok0 + row0) * p.H + h) * D;
       __nv_bfloat16* u_row0 = reinterpret_cast<__nv_bfloat16*>(p.U) + ((size_t)(tok0 + row0) * p.H + h) * D;
-      const uint32_t stage = sAp + kStageOff + warp * 2048;
+      const uint32_t stage = smem_u32(smem + cfg::OFF_STAGE) + warp * 2048;
       if (C == 64 && need_v) {
         float f0[8][4], f1[8][4];
         tmem_ld_16x64(f0, tmem_rows);
@@ -879,7 +922,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
         __syncthreads();  // all MMAs done and all accumulators read: tiles, A' and tensor memory are free
         ph_k ^= 1;
         ph_v ^= 1;
-        if (tid == kTidV && has_next && !SER) issue_v(nx_tok0, nx_h);
+        if (tid == kTidV && has_next && !cfg::RELOAD) issue_v(nx_tok0, nx_h);
         if (tid == 0 && has_next && nx_rows == C && !load_a && mbar_try_wait(bar_k, ph_k)) {
           // the next K tile has landed and tensor memory is free: start the next Gram product now
           tc_fence_after();
@@ -890,6 +933,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
         store_frag_piece_bf16(f1, stage, lane, u_row0 + 64, row_stride, rows - row0);
       } else {
         // C = 128 (W and U side by side in 256 columns) or W only
+        if (cfg::ALIAS && tid == kTidK && has_next && !load_a) issue_k(nx_tok0, nx_h);  // all MMAs on the tiles are done
         store_piece_bf16(tmem_rows, stage, lane, w_row0, row_stride, rows - row0);
         store_piece_bf16(tmem_rows + 64, stage, lane, w_row0 + 64, row_stride, rows - row0);
         if (need_v) {
@@ -900,8 +944,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
         __syncthreads();
         ph_k ^= 1;
         ph_v ^= 1;
-        if (tid == kTidK && has_next) issue_k(nx_tok0, nx_h);
-        if (tid == kTidV && has_next && need_v && !SER) issue_v(nx_tok0, nx_h);
+        if (!cfg::ALIAS && tid == kTidK && has_next) issue_k(nx_tok0, nx_h);
+        if (tid == kTidV && has_next && need_v && !cfg::RELOAD) issue_v(nx_tok0, nx_h);
       }
     } else {
       // build only: the fp32 matrix has been read by everyone after this barrier
@@ -910,7 +954,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
       __syncthreads();
       ph_k ^= 1;
       ph_v ^= 1;
-      if (tid == kTidK && has_next && ((p.ops & kLoadA) || SER)) issue_k(nx_tok0, nx_h);  // otherwise requested after the Gram product
+      if (tid == kTidK && has_next && ((p.ops & kLoadA) || cfg::RELOAD)) issue_k(nx_tok0, nx_h);  // otherwise requested after the Gram product
       if (tid == 0 && has_next && nx_rows == C && !load_a && mbar_try_wait(bar_k, ph_k)) {
         // the next K tile has landed and tensor memory is free: start the next Gram product now
         tc_fence_after();
