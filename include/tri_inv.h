@@ -146,7 +146,7 @@ int tri_inv_fused(const void* K, const void* V, const float* beta, const float* 
  *     make that first call outside of any stream capture.
  *   - All calls share the one array.  Two calls whose kernels can overlap on the GPU (different
  *     streams, or the same stream from different host threads without ordering) race on it: order
- *     them.  Calls on one stream are safe.  Host threads are serialised while the table is filled.
+ *     them.  Calls on one stream are safe.
  */
 #define TRI_INV_STATIC_MAX_CHUNKS 16384
 int tri_inv_fused_packed_static(const void* K, const void* V, const float* beta, const float* g,

@@ -1,7 +1,6 @@
 // extern "C" boundary: argument validation, chunk table for packed sequences, dispatch.
 #include <atomic>
 #include <mutex>
-#include <vector>
 
 #include "common.cuh"
 
@@ -36,6 +35,30 @@ void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 namespace {
 
+// Stream-ordered pool for the packed path's chunk tables.  It keeps what it has allocated (release
+// threshold at the maximum), so steady-state calls reuse the same few kilobytes instead of going back
+// to the driver; being private to the library it leaves the process's default pool untouched.
+cudaMemPool_t table_pool_for_current_device() {
+  static std::mutex mu;
+  static cudaMemPool_t pools[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!pools[dev]) {
+    cudaMemPoolProps props = {};
+    props.allocType = cudaMemAllocationTypePinned;
+    props.handleTypes = cudaMemHandleTypeNone;
+    props.location.type = cudaMemLocationTypeDevice;
+    props.location.id = dev;
+    cudaMemPool_t pool = nullptr;
+    if (cudaMemPoolCreate(&pool, &props) != cudaSuccess) return nullptr;
+    unsigned long long keep = ~0ull;
+    cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+    pools[dev] = pool;
+  }
+  return pools[dev];
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int check_desc(const tri_inv_desc* d, bool need_dv) {
@@ -55,13 +78,6 @@ int check_desc(const tri_inv_desc* d, bool need_dv) {
     return TRI_INV_ERR_INVALID_ARG;
   }
   return TRI_INV_OK;
-}
-
-void ragged_table(const tri_inv_desc* d, std::vector<ChunkEntry>* tab) {
-  for (int s = 0; s < d->n_seqs; ++s) {
-    int beg = d->cu_seqlens[s], end = d->cu_seqlens[s + 1];
-    for (int t = beg; t < end; t += d->C) tab->push_back(ChunkEntry{t, (end - t) < d->C ? (end - t) : d->C});
-  }
 }
 
 int check_method(int method) {
@@ -84,18 +100,19 @@ int run(KParams p, const tri_inv_desc* d, void* stream_v) {
 
   ChunkEntry* dev_tab = nullptr;
   if (d->cu_seqlens) {
-    std::vector<ChunkEntry> tab;
-    ragged_table(d, &tab);
-    p.n_chunks = (int)tab.size();
+    long long n = 0;
+    for (int s = 0; s < d->n_seqs; ++s) n += ((long long)d->cu_seqlens[s + 1] - d->cu_seqlens[s] + d->C - 1) / d->C;
+    if (n > 0x7fffffffLL) return TRI_INV_ERR_INVALID_ARG;
+    p.n_chunks = (int)n;
     p.chunks_per_seq = 0;
     if (p.n_chunks == 0) return TRI_INV_OK;
-    // The table is scratch owned by this call: allocated and freed in stream order.
-    if (cudaMallocAsync((void**)&dev_tab, tab.size() * sizeof(ChunkEntry), stream) != cudaSuccess) return TRI_INV_ERR_CUDA;
-    if (cudaMemcpyAsync(dev_tab, tab.data(), tab.size() * sizeof(ChunkEntry), cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+    // The table is scratch owned by this call: allocated, filled (by a small kernel) and freed in stream order.
+    cudaMemPool_t pool = table_pool_for_current_device();
+    if (!pool || cudaMallocFromPoolAsync((void**)&dev_tab, (size_t)n * sizeof(ChunkEntry), pool, stream) != cudaSuccess) return TRI_INV_ERR_CUDA;
+    if (launch_chunk_table(dev_tab, d, stream) != cudaSuccess) {
       cudaFreeAsync(dev_tab, stream);
       return TRI_INV_ERR_CUDA;
     }
-    // The host vector is pageable: the copy above has been staged before it returns.
     p.chunk_tab = dev_tab;
   } else {
     p.chunks_per_seq = (d->T + d->C - 1) / d->C;

@@ -70,6 +70,10 @@ cudaError_t launch_simt(const KParams& p, int C, cudaStream_t stream);
 // Tensor-core path: returns cudaErrorNotSupported when it has no kernel for the request.
 cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
 
+// Fills dev_tab (one entry per chunk of tokens, in sequence order) from the host offsets in d->cu_seqlens
+// with small kernels on the stream; no copy and no synchronisation.
+cudaError_t launch_chunk_table(ChunkEntry* dev_tab, const tri_inv_desc* d, cudaStream_t stream);
+
 // Adds one to the library's launch counter (tri_inv_launch_count).
 void count_launch();
 

@@ -36,11 +36,6 @@ ChunkEntry* static_table_for_current_device(cudaError_t* err) {
   return cache[dev];
 }
 
-// Host staging for the table (filled, then copied; pageable, so the copy is staged before
-// cudaMemcpyAsync returns).  Guarded by a mutex: concurrent host callers take turns.
-ChunkEntry g_host_table[TRI_INV_STATIC_MAX_CHUNKS];
-std::mutex g_host_table_mu;
-
 }  // namespace
 }  // namespace tri_inv
 
@@ -85,19 +80,9 @@ extern "C" int tri_inv_fused_packed_static(const void* K, const void* V, const f
   p.status = status_word_for_current_device(&err);
   if (!p.status) return TRI_INV_ERR_CUDA;
 
-  {
-    std::lock_guard<std::mutex> lock(g_host_table_mu);
-    int64_t n = 0;
-    for (int s = 0; s < desc->n_seqs; ++s) {
-      const int beg = desc->cu_seqlens[s], end = desc->cu_seqlens[s + 1];
-      for (int t = beg; t < end; t += desc->C) g_host_table[n++] = ChunkEntry{t, (end - t) < desc->C ? (end - t) : desc->C};
-    }
-    // Only the first n_chunks entries are read by the kernel, and all of them are rewritten here,
-    // so nothing left by an earlier call needs clearing.
-    if (cudaMemcpyAsync(dev_tab, g_host_table, static_cast<size_t>(n_chunks) * sizeof(ChunkEntry), cudaMemcpyHostToDevice,
-                        stream) != cudaSuccess)
-      return TRI_INV_ERR_CUDA;
-  }
+  // Only the first n_chunks entries are read by the kernel, and all of them are rewritten here (by a small
+  // kernel on the same stream), so nothing left by an earlier call needs clearing.
+  if (launch_chunk_table(dev_tab, desc, stream) != cudaSuccess) return TRI_INV_ERR_CUDA;
 
   bool handled = false;
   err = cudaSuccess;
