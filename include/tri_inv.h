@@ -112,9 +112,9 @@ int tri_inv_build(const void* K, const float* beta, const float* g, float* A,
 /*
  * W = A diag(beta) K and U = A diag(beta) V from a given A
  * (spec call `tri_inv_wy(A, K, V, beta) -> W, U`; the WY/UT transform
- * the inverse exists for, Sec. 1).  A is read as stored by tri_inv_build
- * (its lower triangle including the diagonal is used).  V and U may both be
- * NULL to compute W only.
+ * the inverse exists for, Sec. 1).  A is read as stored by tri_inv_build;
+ * only its strict lower triangle is used (the diagonal is taken as 1, the upper
+ * triangle as 0).  V and U may both be NULL to compute W only.
  */
 int tri_inv_wy(const float* A, const void* K, const void* V, const float* beta,
                void* W, void* U, const tri_inv_desc* desc, void* cuda_stream);

@@ -526,11 +526,21 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
       }
     }
     if (load_a) {
-      for (int e = tid; e < C * C; e += cfg::NT) {
-        int i = e / C, j = e - i * C;
-        float v = (i == j) ? 1.f : 0.f;
-        if (i < rows && j < i) v = p.A_in[((size_t)(tok0 + i) * p.H + h) * C + j];
-        sX[i * LD + j] = v;
+      // tri_inv_wy: the stored A comes in with 16-byte loads; only its strict lower triangle is used
+      // (unit diagonal and zero upper triangle are written as constants)
+      const size_t a_step = (size_t)(cfg::NT / (C / 4)) * p.H * C;
+      const float* a_src = p.A_in + ((size_t)(tok0 + tid / (C / 4)) * p.H + h) * C + 4 * (tid % (C / 4));
+#pragma unroll
+      for (int m = 0; m < C / 8; ++m) {
+        const int e = tid + m * cfg::NT;
+        const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i < rows && j < i) v = *reinterpret_cast<const float4*>(a_src + (size_t)m * a_step);
+        v.x = (j + 0 < i) ? v.x : (j + 0 == i ? 1.f : 0.f);
+        v.y = (j + 1 < i) ? v.y : (j + 1 == i ? 1.f : 0.f);
+        v.z = (j + 2 < i) ? v.z : (j + 2 == i ? 1.f : 0.f);
+        v.w = (j + 3 < i) ? v.w : (j + 3 == i ? 1.f : 0.f);
+        *reinterpret_cast<float4*>(sX + i * LD + j) = v;
       }
     }
     // rows past the sequence end hold a neighbour's tokens (or zero fill): they are cleared before any MMA
