@@ -8,7 +8,7 @@ A step is one pass of the whole hot path (stage K/V, Gram, gate, inversion, stor
 store W/U: one fused kernel launch) over one batch of the chosen configuration; the default is
 configuration 2 (B=4, T=4096, H=16, d=128, C=64, bf16: 4096 chunk matrices), the one the metric
 is quoted on.  Inputs are seeded synthetic tensors resident in HBM before the timed region; L2 is
-flushed (a 256 MiB write) before every timed step; each step is timed with CUDA events on the
+flushed (a 256 MiB write followed by a 256 MiB read) before every timed step; each step is timed with CUDA events on the
 launching stream.  With N > 1 (torchrun, one rank per GPU) every rank runs its own copy of the
 batch -- chunks are independent, so there is no collective on the data path -- and the value is
 the total over ranks divided by the slowest rank's time (weak scaling).
@@ -39,8 +39,13 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_TRAFFIC_BYTES_PER_MATRIX = {(2, "block_recursive"): 68960}  # profiles/tc_kernel_c64_cfg2.md
 
 
-def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True):
-    """Compulsory traffic of the fused path per chunk matrix: K, V, beta, g read once; A, W, U written once."""
+def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True, call="fused"):
+    """Compulsory traffic per chunk matrix.  fused: K, V, beta, g read once; A, W, U written once.
+    build: K, beta, g read; A written.  wy: the strict lower triangle of A, K, V, beta read; W, U written."""
+    if call == "build":
+        return C * d_k * elt + 2 * C * 4 + C * C * 4
+    if call == "wy":
+        return C * (C - 1) // 2 * 4 + C * d_k * elt + C * d_v * elt + C * 4 + C * d_k * elt + C * d_v * elt
     b = C * d_k * elt + C * d_v * elt + 2 * C * 4 + C * d_k * elt + C * d_v * elt
     if want_A:
         b += C * C * 4
@@ -185,6 +190,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--method", default="block_recursive", choices=["block_recursive", "mixed_recursion", "product_series"])
+    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy"],
+                    help="entry point timed: the fused path (default, the metric), tri_inv_build alone, or tri_inv_wy alone")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-flush", action="store_true", help="skip the L2 flush between steps (profiling runs)")
@@ -230,14 +237,29 @@ def main():
     A = torch.empty((inp.B, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda")
     W, U = torch.empty_like(K), torch.empty_like(V)
     flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+    flush_rd = None if args.no_flush else torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream()
 
-    def step():
-        binding.fused(K, V, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U), stream=stream)
-
-    for _ in range(max(args.warmup, 3)):
+    def flush_l2():
+        """Write 256 MiB (evicts everything), then read another 256 MiB so that the lines left in L2 are
+        clean: the timed kernel starts with a cold L2 and does not pay for writing back the flush's data."""
         if flush is not None:
             flush.fill_(1)
+            flush_rd.sum()
+
+    def step():
+        if args.call == "fused":
+            binding.fused(K, V, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U), stream=stream)
+        elif args.call == "build":
+            binding.build(K, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
+        else:
+            binding.wy(A, K, V, beta, cu_seqlens=inp.cu_seqlens, out=(W, U), stream=stream)
+
+    if args.call == "wy":  # tri_inv_wy reads a stored A: produce it once, outside the timed region
+        binding.build(K, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
+
+    for _ in range(max(args.warmup, 3)):
+        flush_l2()
         step()
     torch.cuda.synchronize()
     if binding.last_device_status() != 0:
@@ -245,12 +267,13 @@ def main():
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
-        # the timed region lasts milliseconds: keep the GPU busy with the same step until the sampler has
-        # produced readings under load, then go straight into the timed steps
+        # the timed region lasts milliseconds: keep the GPU busy with the same flush + step pattern until the
+        # sampler has produced readings under load, then go straight into the timed steps
         sampler.start()
         t_end = time.time() + 5.0
         while sampler.proc and len(sampler.lines) < 4 and time.time() < t_end:
             for _ in range(20):
+                flush_l2()
                 step()
             torch.cuda.synchronize()
     if world > 1:
@@ -259,8 +282,7 @@ def main():
     launches0 = binding.launch_count()
     evs = []
     for _ in range(args.steps):
-        if flush is not None:
-            flush.fill_(1)
+        flush_l2()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         step()
@@ -322,14 +344,14 @@ def main():
 
     if rank == 0:
         elt = 2 if inp.kv_dtype == wl.BF16 else 4
-        alg_bytes = algorithmic_bytes_per_matrix(inp.C, inp.d_k, inp.d_v, elt)
+        alg_bytes = algorithmic_bytes_per_matrix(inp.C, inp.d_k, inp.d_v, elt, call=args.call)
         kernel_ms = statistics.mean(times_ms)               # one launch per step, timed alone by its event pair
         achieved = alg_bytes * n_mat / (kernel_ms * 1e-3) / 1e9
         peak, peak_kind = measured_peak_gbs()
-        traffic = NCU_TRAFFIC_BYTES_PER_MATRIX.get((args.config, args.method))
+        traffic = NCU_TRAFFIC_BYTES_PER_MATRIX.get((args.config, args.method)) if args.call == "fused" else None
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": None if traffic is None else traffic * n_mat, "peak_source": "of " + peak_kind,
-                    "kernel": "fused build+invert+WY", "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
+                    "kernel": {"fused": "fused build+invert+WY", "build": "build+invert", "wy": "WY apply"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
                     "algorithmic_bytes_per_launch": alg_bytes * n_mat}
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
@@ -338,8 +360,9 @@ def main():
                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                "dtype": "bf16" if inp.kv_dtype == wl.BF16 else "f32", "data": "synthetic",
                "config": {"workload": inp.name, "B": inp.B, "T": inp.T, "H": inp.H, "d_k": inp.d_k, "d_v": inp.d_v, "C": inp.C,
-                          "chunk_matrices_per_gpu": n_mat, "method": args.method, "outputs": "A fp32 + W,U",
-                          "l2": "flushed before every timed step (256 MiB write)" if flush is not None else "not flushed",
+                          "chunk_matrices_per_gpu": n_mat, "method": args.method, "call": args.call,
+                          "outputs": {"fused": "A fp32 + W,U", "build": "A fp32", "wy": "W,U"}[args.call],
+                          "l2": "flushed before every timed step (256 MiB write, then a 256 MiB read so no dirty lines remain)" if flush is not None else "not flushed",
                           "parallelism": "independent replicas, no collective" if world > 1 else "single GPU"},
                "gb_per_s": achieved, "roofline": roofline, "cpu_baseline": cpu,
                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
