@@ -160,7 +160,7 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2605_21325_b200 import workloads as wl
-    inp = wl.config(args.config)
+    inp = wl.paper_timing_case(args.paper_T) if args.paper_T else wl.config(args.config)
     per_step_target = max(2.0, min(15.0, 120.0 / max(args.steps + args.warmup, 1)))
     vals = []
     base = None
@@ -190,6 +190,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--method", default="block_recursive", choices=["block_recursive", "mixed_recursion", "product_series"])
+    ap.add_argument("--paper-T", type=int, default=0,
+                    help="instead of --config: the paper's timing shape B=32, H=4, d=128 at this sequence length (1024..16384)")
     ap.add_argument("--call", default="fused", choices=["fused", "build", "wy"],
                     help="entry point timed: the fused path (default, the metric), tri_inv_build alone, or tri_inv_wy alone")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -230,7 +232,8 @@ def main():
     if args.simt:
         method |= binding.FORCE_SIMT
 
-    inp = wl.config(args.config)                    # same seeded batch on every rank (weak scaling)
+    # same seeded batch on every rank (weak scaling)
+    inp = wl.paper_timing_case(args.paper_T) if args.paper_T else wl.config(args.config)
     n_mat = inp.n_matrices
     dev = binding.to_device(inp)
     K, V, beta, g = dev["K"], dev["V"], dev["beta"], dev["g"]

@@ -156,6 +156,12 @@ def config(cfg: int, shrink: int = 1) -> Inputs:
     raise ValueError("unknown config %r" % cfg)
 
 
+def paper_timing_case(T: int, C: int = 64) -> Inputs:
+    """Shape of the paper's kernel timing experiment (Sec. 5.1): batch 32, 4 heads, sequence length T up to 16K.
+    The head dimension is not stated there; 128 is assumed.  Same value distributions as the GDN configs."""
+    return make("paper_timing_B32_H4_T%d_C%d" % (T, C), 32, T, 4, 128, 128, C, BF16, 1100 + T // 1024)
+
+
 def first_difference_case(B, T, H, d, C, kv_dtype, cu_seqlens=None) -> Inputs:
     """Every key equals the same unit vector e_0, beta = 1, g = 0, so N is the all-ones
     strictly lower matrix (the example of Sec. 3.2) and every value involved is exactly
