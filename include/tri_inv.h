@@ -75,10 +75,20 @@ enum {
    * X <- I - N, Y <- N, then log2(C) - 1 rounds of Y <- Y.Y, X <- X + X.Y,
    * i.e. prod_k (I + (-N)^(2^k)).  Exact in exact arithmetic, not stable. */
   TRI_INV_PRODUCT_SERIES = 1,
+  /* Newton-Schulz iteration (Alg. 3 / Sec. 3.5): X_0 = I / C, X <- X (2I - (I + N) X).  Iterative: the
+   * result converges to the inverse; TRI_INV_NS_ITERS(m) sets the count (default 2 log2(C), the count
+   * the paper reports as converged at C = 64).  Runs on the fp32 CUDA-core kernel. */
+  TRI_INV_NEWTON_SCHULZ = 2,
   TRI_INV_METHOD_MASK = 0xff,
   /* flag, block-recursive only: invert the 16x16 leaves with the product series
    * instead of substitution -- the mixed recursion of Alg. 2 (r = 0). */
   TRI_INV_LEAF_SERIES = 0x100,
+  /* flag: one step of iterative refinement after the inversion (Alg. 6 / Sec. 3.6):
+   * R <- I - A (I + N), A <- A + R A.  Block recursion and Newton-Schulz only; runs on the
+   * fp32 CUDA-core kernel (TF32 products could not resolve the residual). */
+  TRI_INV_REFINE = 0x200,
+  /* Newton-Schulz iteration count, 1..15, in bits 12..15 (0 = default) */
+#define TRI_INV_NS_ITERS(m) (((m) & 0xf) << 12)
   /* flag: run the plain fp32 CUDA-core kernel even where a tensor-core kernel
    * exists (same results up to rounding; for cross-checks and odd shapes). */
   TRI_INV_FORCE_SIMT = 0x10000

@@ -99,6 +99,27 @@ def mxr(L: np.ndarray, b0: int = 16) -> np.ndarray:
     return mbh(L, Y, b0)
 
 
+def newton_schulz(L: np.ndarray, m: int | None = None, x0_scale: float | None = None) -> np.ndarray:
+    """Alg. 3: A = I + L, X_0 = I / n (the initial guess I / n^{O(1)} of Prop. 3.2 with exponent 1),
+    then m rounds of Y <- A.X, X <- 2X - X.Y.  Default m = 2 log2(n)."""
+    n = L.shape[0]
+    A = np.eye(n) + L
+    X = np.eye(n) * (1.0 / n if x0_scale is None else x0_scale)
+    if m is None:
+        m = 2 * int(np.log2(n))
+    for _ in range(m):
+        Y = A @ X
+        X = 2 * X - X @ Y
+    return X
+
+
+def iterative_refinement(X: np.ndarray, L: np.ndarray) -> np.ndarray:
+    """One step of Sec. 3.6 for the matrix I + L: R <- I - X (I + L), X <- X + R X."""
+    n = L.shape[0]
+    R = np.eye(n) - X @ (np.eye(n) + L)
+    return X + R @ X
+
+
 def block_recursive(L: np.ndarray, leaf: int = 16) -> np.ndarray:
     """The 2x2 block identity of Sec. 3.3 written for a lower triangular matrix:
     inv([[M11, 0], [N21, M22]]) = [[X11, 0], [-X22 N21 X11, X22]], recursing down

@@ -22,8 +22,16 @@ LIB_PATH = os.path.join(_PKG, "libtri_inv.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_TOO_LARGE = 0, 1, 2, 3, 4, 5
 STATIC_MAX_CHUNKS = 16384
 F32, BF16 = 0, 1
-BLOCK_RECURSIVE, PRODUCT_SERIES = 0, 1
+BLOCK_RECURSIVE, PRODUCT_SERIES, NEWTON_SCHULZ = 0, 1, 2
 LEAF_SERIES = 0x100
+REFINE = 0x200
+
+
+def ns_iters(m: int) -> int:
+    """Method flag carrying a Newton-Schulz iteration count (1..15)."""
+    return (int(m) & 0xF) << 12
+
+
 FORCE_SIMT = 0x10000
 
 EXPORTS = ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_packed_static", "tri_inv_count_matrices",

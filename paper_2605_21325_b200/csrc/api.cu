@@ -82,9 +82,11 @@ int check_desc(const tri_inv_desc* d, bool need_dv) {
 
 int check_method(int method) {
   int m = method & TRI_INV_METHOD_MASK;
-  if (m != TRI_INV_BLOCK_RECURSIVE && m != TRI_INV_PRODUCT_SERIES) return TRI_INV_ERR_UNSUPPORTED;
-  if (method & ~(TRI_INV_METHOD_MASK | TRI_INV_LEAF_SERIES | TRI_INV_FORCE_SIMT)) return TRI_INV_ERR_UNSUPPORTED;
+  if (m != TRI_INV_BLOCK_RECURSIVE && m != TRI_INV_PRODUCT_SERIES && m != TRI_INV_NEWTON_SCHULZ) return TRI_INV_ERR_UNSUPPORTED;
+  if (method & ~(TRI_INV_METHOD_MASK | TRI_INV_LEAF_SERIES | TRI_INV_REFINE | TRI_INV_NS_ITERS(15) | TRI_INV_FORCE_SIMT)) return TRI_INV_ERR_UNSUPPORTED;
   if ((method & TRI_INV_LEAF_SERIES) && m != TRI_INV_BLOCK_RECURSIVE) return TRI_INV_ERR_UNSUPPORTED;
+  if ((method & TRI_INV_REFINE) && m == TRI_INV_PRODUCT_SERIES) return TRI_INV_ERR_UNSUPPORTED;
+  if ((method & TRI_INV_NS_ITERS(15)) && m != TRI_INV_NEWTON_SCHULZ) return TRI_INV_ERR_UNSUPPORTED;
   return TRI_INV_OK;
 }
 
@@ -125,7 +127,9 @@ int run(KParams p, const tri_inv_desc* d, void* stream_v) {
   if ((long long)p.n_chunks * d->H > 0x7fffffffLL) return TRI_INV_ERR_INVALID_ARG;  // kernels index work items in 32 bits
   bool handled = false;
   err = cudaSuccess;
-  if (!(p.method & TRI_INV_FORCE_SIMT)) err = launch_tc(p, d->C, stream, &handled);
+  // Newton-Schulz and the refinement step exist on the fp32 CUDA-core kernel only
+  const bool simt_only = (p.method & (TRI_INV_FORCE_SIMT | TRI_INV_REFINE)) || (p.method & TRI_INV_METHOD_MASK) == TRI_INV_NEWTON_SCHULZ;
+  if (!simt_only) err = launch_tc(p, d->C, stream, &handled);
   if (err == cudaSuccess && !handled) err = launch_simt(p, d->C, stream);
   if (err == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);
   if (dev_tab) cudaFreeAsync(dev_tab, stream);

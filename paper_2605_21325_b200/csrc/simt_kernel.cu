@@ -80,6 +80,22 @@ __device__ float* product_series_blocks(float* y, float* x, float* z, int bs, in
   return x;
 }
 
+// acc[m] = (a . b)_ij for the element e = tid + m * kThreads of a C x C lower-triangular product
+// (a and b lower triangular, sum over k = j..i); elements above the diagonal give 0.
+template <int C, int kAcc>
+__device__ __forceinline__ void tri_matmul_regs(float (&acc)[kAcc], const float* a, const float* b, int tid) {
+  constexpr int LD = C + 1;
+#pragma unroll
+  for (int m = 0; m < kAcc; ++m) {
+    const int e = tid + m * kThreads;
+    const int i = e / C, j = e - i * C;
+    float s = 0.f;
+    if (e < C * C && j <= i)
+      for (int k = j; k <= i; ++k) s = fmaf(a[i * LD + k], b[k * LD + j], s);
+    acc[m] = s;
+  }
+}
+
 template <int C>
 __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
   constexpr int LD = C + 1;
@@ -151,6 +167,32 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
 
       if (method == TRI_INV_PRODUCT_SERIES) {
         Xres = product_series_blocks<C>(Nm, Xm, Zm, C, tid);
+      } else if (method == TRI_INV_NEWTON_SCHULZ) {
+        // Alg. 3: M = I + N, X_0 = I / C, then m rounds of Y <- M.X, X <- 2X - X.Y.
+        // All iterates are lower triangular, so the products run over k = j..i only.
+        int iters = (p.method >> 12) & 0xf;
+        if (iters == 0) { iters = 0; for (int m = C; m > 1; m >>= 1) iters += 2; }  // 2 log2(C)
+        for (int e = tid; e < C * C; e += kThreads) {
+          const int i = e / C, j = e - i * C;
+          if (i == j) { Nm[i * LD + j] = 1.f; Xm[i * LD + j] = 1.f / C; }
+        }
+        __syncthreads();
+        for (int it = 0; it < iters; ++it) {
+          tri_matmul_blocks<C>(Zm, Nm, Xm, C, tid);   // Y <- M.X
+          __syncthreads();
+          float q[kAcc];
+          tri_matmul_regs<C, kAcc>(q, Xm, Zm, tid);   // X.Y, held in registers until every read of X is done
+          __syncthreads();
+#pragma unroll
+          for (int m = 0; m < kAcc; ++m) {
+            const int e = tid + m * kThreads;
+            const int i = e / C, j = e - i * C;
+            if (e < C * C && j <= i) Xm[i * LD + j] = 2.f * Xm[i * LD + j] - q[m];
+          }
+          __syncthreads();
+        }
+        for (int e = tid; e < C; e += kThreads) Nm[e * LD + e] = 0.f;  // back to N for an optional refinement step
+        __syncthreads();
       } else {
         constexpr int kLeaf = C < 16 ? C : 16;
         if (p.method & TRI_INV_LEAF_SERIES) {
@@ -231,6 +273,29 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
           __syncthreads();
         }
       }
+    }
+
+    // ---- optional refinement (Alg. 6): R <- I - X.M with M = I + N, then X <- X + R.X
+    if ((p.method & TRI_INV_REFINE) && !(p.ops & kLoadA)) {
+      float* Rm = (Xres == Zm) ? Xm : Zm;  // a buffer that is neither N nor the current result
+      float q[kAcc];
+      tri_matmul_regs<C, kAcc>(q, Xres, Nm, tid);  // X.N (N strictly lower; X.M = X + X.N)
+#pragma unroll
+      for (int m = 0; m < kAcc; ++m) {
+        const int e = tid + m * kThreads;
+        const int i = e / C, j = e - i * C;
+        if (e < C * C) Rm[i * LD + j] = (j <= i) ? ((i == j ? 1.f : 0.f) - Xres[i * LD + j] - q[m]) : 0.f;
+      }
+      __syncthreads();
+      tri_matmul_regs<C, kAcc>(q, Rm, Xres, tid);  // R.X
+      __syncthreads();
+#pragma unroll
+      for (int m = 0; m < kAcc; ++m) {
+        const int e = tid + m * kThreads;
+        const int i = e / C, j = e - i * C;
+        if (e < C * C && j <= i) Xres[i * LD + j] += q[m];
+      }
+      __syncthreads();
     }
 
     // ---- store A: computed strict-lower part, constant diagonal and upper triangle

@@ -306,3 +306,25 @@ def test_threads_do_not_change_results():
     a1 = oracle.build_A(x.K, x.beta, x.g, x.C, n_threads=1)
     a4 = oracle.build_A(x.K, x.beta, x.g, x.C, n_threads=4)
     assert np.array_equal(a1, a4)
+
+
+# ---------------------------------------------------------------- iterative schemes (Alg. 3, Alg. 6)
+
+def test_newton_schulz_and_refinement_converge_to_substitution():
+    x = wl.make("ns", 1, 64, 1, 128, 8, 64, wl.F32, seed=91)
+    A, N = oracle.build_A(x.K, x.beta, x.g, 64, return_N=True)
+    a, L = A[0, :, 0], N[0, :, 0]
+    err = {m: np.linalg.norm(alg.newton_schulz(L, m) - a) / np.linalg.norm(a) for m in (6, 8, 10, 12, 14)}
+    # Sec. 4.2: six iterations are not enough at C = 64, twelve are, more add nothing
+    assert err[6] > 1e-2 and err[10] < 1e-4 and err[12] < 1e-12 and err[14] < 1e-12
+    assert err[6] > err[8] > err[10] > err[12]
+    # the default count is 2 log2(n)
+    assert np.abs(alg.newton_schulz(L) - a).max() < 1e-12
+    # one refinement step squares the residual: it equals one more Newton-Schulz round
+    x8 = alg.newton_schulz(L, 8)
+    assert np.abs(alg.iterative_refinement(x8, L) - alg.newton_schulz(L, 9)).max() < 1e-12
+    r0 = np.abs(np.eye(64) - x8 @ (np.eye(64) + L)).max()
+    r1 = np.abs(np.eye(64) - alg.iterative_refinement(x8, L) @ (np.eye(64) + L)).max()
+    assert r1 < 64 * r0 * r0
+    # refinement leaves an exact inverse unchanged
+    assert np.abs(alg.iterative_refinement(a, L) - a).max() < 1e-14

@@ -293,3 +293,38 @@ def test_runs_on_a_side_stream(bnd):
         A = bnd.build(dev["K"], dev["beta"], dev["g"], inp.C, stream=s)
     s.synchronize()
     assert max_ratio(A.cpu().numpy(), A_ref) <= 2e-3
+
+
+# ---------------------------------------------------------------- Newton-Schulz (Alg. 3) and refinement (Alg. 6)
+
+@pytest.mark.parametrize("cfg,shrink", [(1, 1), (2, 32)])
+def test_newton_schulz_and_refinement(bnd, cfg, shrink):
+    inp = wl.config(cfg, shrink=shrink)
+    A_ref, N_ref, W_ref, U_ref = oracle_all(inp)
+    # default iteration count (2 log2 C) reaches fp32 accuracy
+    A, W, U = run_fused(bnd, inp, bnd.NEWTON_SCHULZ)
+    r_full, _ = check_A(A, inp, A_ref, N_ref, tol=1e-5, tol_res=5e-5)
+    check_WU(W, U, inp, W_ref, U_ref, bnd)
+    # too few iterations leave a visible error; one refinement step equals one more round
+    errs = {}
+    for name, m in (("ns6", bnd.NEWTON_SCHULZ | bnd.ns_iters(6)), ("ns8", bnd.NEWTON_SCHULZ | bnd.ns_iters(8)),
+                    ("ns8+ir", bnd.NEWTON_SCHULZ | bnd.ns_iters(8) | bnd.REFINE), ("ns9", bnd.NEWTON_SCHULZ | bnd.ns_iters(9))):
+        A, _, _ = run_fused(bnd, inp, m)
+        errs[name] = max_ratio(A.cpu().numpy(), A_ref)
+    assert errs["ns6"] > errs["ns8"] > errs["ns8+ir"] and errs["ns6"] > 1e-3
+    assert abs(errs["ns8+ir"] - errs["ns9"]) <= 1e-5 + 0.05 * errs["ns9"]
+    # refinement after the block recursion keeps the result within the fp32 bound
+    A, W, U = run_fused(bnd, inp, bnd.BLOCK_RECURSIVE | bnd.REFINE)
+    check_A(A, inp, A_ref, N_ref, tol=1e-5, tol_res=5e-5)
+    A, _, _ = run_fused(bnd, inp, bnd.BLOCK_RECURSIVE | bnd.LEAF_SERIES | bnd.REFINE)
+    check_A(A, inp, A_ref, N_ref, tol=1e-5, tol_res=5e-5)
+
+
+def test_method_flag_combinations_rejected(bnd):
+    import ctypes
+    d = torch.zeros(64, device="cuda")
+    desc, _ = bnd.make_desc(1, 64, 1, 128, 128, 64, bnd.BF16)
+    L = bnd.load()
+    for bad in (bnd.PRODUCT_SERIES | bnd.REFINE, bnd.BLOCK_RECURSIVE | bnd.ns_iters(4), bnd.NEWTON_SCHULZ | bnd.LEAF_SERIES, 3):
+        rc = L.tri_inv_build(bnd._p(d), bnd._p(d), bnd._p(d), bnd._p(d), ctypes.byref(desc), bad, None)
+        assert rc == bnd.ERR_UNSUPPORTED, bad
