@@ -192,8 +192,9 @@ def main():
     ap.add_argument("--method", default="block_recursive", choices=["block_recursive", "mixed_recursion", "product_series"])
     ap.add_argument("--paper-T", type=int, default=0,
                     help="instead of --config: the paper's timing shape B=32, H=4, d=128 at this sequence length (1024..16384)")
-    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy"],
-                    help="entry point timed: the fused path (default, the metric), tri_inv_build alone, or tri_inv_wy alone")
+    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw"],
+                    help="entry point timed: the fused path (default, the metric), tri_inv_build alone, tri_inv_wy alone, or "
+                         "tri_inv_fused_raw (front end folded in; same shapes, un-normalised keys and logits as inputs)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-flush", action="store_true", help="skip the L2 flush between steps (profiling runs)")
@@ -234,6 +235,8 @@ def main():
 
     # same seeded batch on every rank (weak scaling)
     inp = wl.paper_timing_case(args.paper_T) if args.paper_T else wl.config(args.config)
+    if args.call == "raw":  # same shape, inputs as the projections hand them over
+        inp = wl.make_raw(inp.name + "_raw", inp.B, inp.T, inp.H, inp.d_k, inp.C, inp.kv_dtype, 2000 + args.config, inp.cu_seqlens)
     n_mat = inp.n_matrices
     dev = binding.to_device(inp)
     K, V, beta, g = dev["K"], dev["V"], dev["beta"], dev["g"]
@@ -253,6 +256,8 @@ def main():
     def step():
         if args.call == "fused":
             binding.fused(K, V, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U), stream=stream)
+        elif args.call == "raw":
+            binding.fused_raw(K, V, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U, None, None), stream=stream)
         elif args.call == "build":
             binding.build(K, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
         else:
@@ -333,12 +338,18 @@ def main():
         import oracle
         Ts = min(inp.T, 4 * inp.C) if inp.cu_seqlens is None else None
         if Ts is not None:
-            A_ref = oracle.build_A(inp.K[:, :Ts], inp.beta[:, :Ts], inp.g[:, :Ts], inp.C)
-            W_ref, U_ref = oracle.wy(A_ref, inp.K[:, :Ts], inp.V[:, :Ts], inp.beta[:, :Ts], inp.C)
+            Ko, bo, go = inp.K[:, :Ts], inp.beta[:, :Ts], inp.g[:, :Ts]
+            if args.call == "raw":
+                Ko, bo, go = oracle.raw_front_end(Ko, bo, go, inp.C)
+            A_ref = oracle.build_A(Ko, bo, go, inp.C)
+            W_ref, U_ref = oracle.wy(A_ref, Ko, inp.V[:, :Ts], bo, inp.C)
             a = binding.to_numpy_f64(A[:, :Ts]); w = binding.to_numpy_f64(W[:, :Ts]); u = binding.to_numpy_f64(U[:, :Ts])
         else:
-            A_ref = oracle.build_A(inp.K, inp.beta, inp.g, inp.C, cu_seqlens=inp.cu_seqlens)
-            W_ref, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, inp.C, cu_seqlens=inp.cu_seqlens)
+            Ko, bo, go = inp.K, inp.beta, inp.g
+            if args.call == "raw":
+                Ko, bo, go = oracle.raw_front_end(Ko, bo, go, inp.C, cu_seqlens=inp.cu_seqlens)
+            A_ref = oracle.build_A(Ko, bo, go, inp.C, cu_seqlens=inp.cu_seqlens)
+            W_ref, U_ref = oracle.wy(A_ref, Ko, inp.V, bo, inp.C, cu_seqlens=inp.cu_seqlens)
             a, w, u = binding.to_numpy_f64(A), binding.to_numpy_f64(W), binding.to_numpy_f64(U)
         err = {"sample": "first %d tokens of every sequence" % Ts if Ts else "all tokens"}
         if args.call != "wy":
@@ -356,7 +367,7 @@ def main():
         traffic = NCU_TRAFFIC_BYTES_PER_MATRIX.get((args.config, args.method)) if args.call == "fused" else None
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": None if traffic is None else traffic * n_mat, "peak_source": "of " + peak_kind,
-                    "kernel": {"fused": "fused build+invert+WY", "build": "build+invert", "wy": "WY apply"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
+                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "wy": "WY apply"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
                     "algorithmic_bytes_per_launch": alg_bytes * n_mat}
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
@@ -366,7 +377,7 @@ def main():
                "dtype": "bf16" if inp.kv_dtype == wl.BF16 else "f32", "data": "synthetic",
                "config": {"workload": inp.name, "B": inp.B, "T": inp.T, "H": inp.H, "d_k": inp.d_k, "d_v": inp.d_v, "C": inp.C,
                           "chunk_matrices_per_gpu": n_mat, "method": args.method, "call": args.call,
-                          "outputs": {"fused": "A fp32 + W,U", "build": "A fp32", "wy": "W,U"}[args.call],
+                          "outputs": {"fused": "A fp32 + W,U", "raw": "A fp32 + W,U", "build": "A fp32", "wy": "W,U"}[args.call],
                           "l2": "flushed before every timed step (256 MiB write, then a 256 MiB read so no dirty lines remain)" if flush is not None else "not flushed",
                           "parallelism": "independent replicas, no collective" if world > 1 else "single GPU"},
                "gb_per_s": achieved, "roofline": roofline, "cpu_baseline": cpu,

@@ -138,6 +138,25 @@ int tri_inv_fused(const void* K, const void* V, const float* beta, const float* 
                   const tri_inv_desc* desc, int method, void* cuda_stream);
 
 /*
+ * Fused call with the layer's front end folded in: the kernel takes what the projections produce and
+ * does the three producers that otherwise run as separate passes over memory before the inversion
+ * (the gating recipe of a Gated-DeltaNet layer; in the paper these are among the kernels its fused
+ * layer kernel absorbs, Sec. 5.2):
+ *     beta_t = sigmoid(beta_logit_t)
+ *     g_t    = sum over s <= t of the same chunk of log sigmoid(gate_logit_s)
+ *     k^_t   = K_raw_t / ||K_raw_t||_2            (a zero key stays zero)
+ * and then N, A, W = A diag(beta) K^ and U = A diag(beta) V exactly as tri_inv_fused does with K^, beta, g.
+ * The norms come from the diagonal of the Gram product, so normalising costs no extra pass.
+ *   K_raw, V            [B,T,H,d] kv_dtype;   beta_logit, gate_logit  [B,T,H] fp32
+ *   beta_out, g_out     optional [B,T,H] fp32 outputs (beta and the cumulative log-decay, for the
+ *                       layer's later steps); NULL to skip
+ * A may be NULL.  All methods and both chunking modes of tri_inv_fused apply.
+ */
+int tri_inv_fused_raw(const void* K_raw, const void* V, const float* beta_logit, const float* gate_logit,
+                      float* A, void* W, void* U, float* beta_out, float* g_out,
+                      const tri_inv_desc* desc, int method, void* cuda_stream);
+
+/*
  * Packed-sequence fused call that allocates nothing.  (The paper has no counterpart: this is a
  * deployment variant of tri_inv_fused, not a step of the method.)
  *

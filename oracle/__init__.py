@@ -31,7 +31,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "tri_inv_oracle.c")
 _LIB = os.path.join(_HERE, "libtri_inv_oracle.so")
 
-F32, BF16 = 0, 1
+F32, BF16, F64 = 0, 1, 2
 _lib = None
 
 
@@ -69,7 +69,45 @@ def _kv(a: np.ndarray):
         return np.ascontiguousarray(a), F32
     if a.dtype == np.uint16:
         return np.ascontiguousarray(a), BF16
-    raise TypeError("K/V must be float32 or uint16 (bf16 bits), got %s" % a.dtype)
+    if a.dtype == np.float64:
+        return np.ascontiguousarray(a), F64
+    raise TypeError("K/V must be float32, float64 or uint16 (bf16 bits), got %s" % a.dtype)
+
+
+def _widen(a: np.ndarray) -> np.ndarray:
+    """Storage array -> float64, exactly."""
+    if a.dtype == np.uint16:
+        return (a.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def raw_front_end(K_raw, beta_logit, gate_logit, C, cu_seqlens=None):
+    """The producers a Gated-DeltaNet layer runs before the inversion, in fp64 (the recipe the
+    configurations state for their inputs): beta = sigmoid(beta_logit); per-token log-decay
+    a = log sigmoid(gate_logit), g = its cumulative sum restarting at every chunk; keys divided by
+    their L2 norm over the feature axis (a zero key stays zero).  Returns (K_hat f64, beta f64, g f64)."""
+    Kd = _widen(np.asarray(K_raw))
+    B, T, H, _ = Kd.shape
+    nrm = np.sqrt((Kd * Kd).sum(axis=-1, keepdims=True))
+    K_hat = np.divide(Kd, nrm, out=np.zeros_like(Kd), where=nrm > 0)
+    x = np.asarray(beta_logit, dtype=np.float64)
+    beta = 1.0 / (1.0 + np.exp(-x))
+    z = np.asarray(gate_logit, dtype=np.float64)
+    a = np.minimum(z, 0.0) - np.log1p(np.exp(-np.abs(z)))
+    a = a.reshape(B * T, H)
+    g = np.zeros_like(a)
+    bounds = [(b * T, (b + 1) * T) for b in range(B)] if cu_seqlens is None else \
+             [(int(cu_seqlens[i]), int(cu_seqlens[i + 1])) for i in range(len(cu_seqlens) - 1)]
+    for beg, end in bounds:
+        t = beg
+        while t < end:
+            e = min(t + C, end)
+            run = np.zeros(H)
+            for r in range(t, e):          # plain running sum, token by token
+                run = run + a[r]
+                g[r] = run
+            t = e
+    return K_hat, beta, g.reshape(B, T, H)
 
 
 def threads(n_threads: int = 0) -> int:
@@ -85,7 +123,7 @@ def build_A(K, beta, g, C, cu_seqlens=None, n_threads=0, return_N=False):
     K, dt = _kv(K)
     B, T, H, d_k = K.shape
     beta = np.ascontiguousarray(beta, dtype=np.float32)
-    g = np.ascontiguousarray(g, dtype=np.float32)
+    g = np.ascontiguousarray(g, dtype=np.float32)   # the C ABI under test takes fp32 beta and g
     assert beta.shape == (B, T, H) and g.shape == (B, T, H)
     A = np.zeros((B, T, H, C), dtype=np.float64)
     N = np.zeros((B, T, H, C), dtype=np.float64) if return_N else None
@@ -105,7 +143,9 @@ def wy(A, K, V, beta, C, cu_seqlens=None, n_threads=0):
     d_v = 0
     if V is not None:
         V, dtv = _kv(V)
-        assert dtv == dt and V.shape[:3] == (B, T, H)
+        if dtv != dt:  # one storage type per call: widen both (exactly) to double
+            K, V, dt = _widen(K), _widen(V), F64
+        assert V.shape[:3] == (B, T, H)
         d_v = V.shape[3]
     A = np.ascontiguousarray(A, dtype=np.float64)
     assert A.shape == (B, T, H, C)

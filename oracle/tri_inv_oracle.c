@@ -16,9 +16,10 @@
  *                                                        in its scalar form)
  *   W    = A diag(beta) K,   U = A diag(beta) V        (WY factors)
  *
- * Inputs arrive in their storage type (fp32 or bf16 bit patterns) and are
- * widened exactly to double; every sum runs in double in index order.  There
- * is no blocking, tiling or reordering: each loop is the formula.
+ * Inputs arrive in their storage type (fp32, bf16 bit patterns, or double for
+ * keys prepared in double by the raw front end) and are widened exactly to
+ * double; every sum runs in double in index order.  There is no blocking,
+ * tiling or reordering: each loop is the formula.
  *
  * Layouts (all contiguous, row-major):
  *   K [B,T,H,d_k], V [B,T,H,d_v], beta and g [B,T,H] (g is the within-chunk
@@ -41,10 +42,11 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1, ORACLE_F64 = 2 };
 
 static double widen(const void* base, int dtype, size_t idx) {
   if (dtype == ORACLE_F32) return (double)((const float*)base)[idx];
+  if (dtype == ORACLE_F64) return ((const double*)base)[idx];
   uint32_t bits = ((uint32_t)((const uint16_t*)base)[idx]) << 16; /* bf16 = top half of fp32 */
   float f;
   memcpy(&f, &bits, sizeof f);

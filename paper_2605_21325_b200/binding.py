@@ -34,7 +34,7 @@ def ns_iters(m: int) -> int:
 
 FORCE_SIMT = 0x10000
 
-EXPORTS = ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
+EXPORTS = ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
            "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
 
 
@@ -66,6 +66,8 @@ def load():
         lib.tri_inv_build.argtypes = [vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_wy.argtypes = [vp, vp, vp, vp, vp, vp, dp, vp]
         lib.tri_inv_fused.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
+        lib.tri_inv_fused_raw.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
+        lib.tri_inv_fused_raw.restype = i32
         lib.tri_inv_fused_packed_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_fused_packed_static.restype = i32
         lib.tri_inv_count_matrices.argtypes = [dp, ctypes.POINTER(ctypes.c_int64)]
@@ -176,6 +178,27 @@ def fused(K, V, beta, g, C, method=BLOCK_RECURSIVE, cu_seqlens=None, want_A=True
     if rc != OK:
         raise TriInvError("tri_inv_fused", rc)
     return A, W, U
+
+
+def fused_raw(K_raw, V, beta_logit, gate_logit, C, method=BLOCK_RECURSIVE, cu_seqlens=None, want_A=True,
+              want_gates=False, out=None, stream=None):
+    """Fused call that also runs the layer's front end (sigmoid, log-sigmoid + chunk cumsum, key
+    normalisation) -> (A or None, W, U, beta or None, g or None)."""
+    B, T, H, d_k = K_raw.shape
+    d_v = V.shape[-1]
+    desc, keep = make_desc(B, T, H, d_k, d_v, C, _dtype_code(K_raw), cu_seqlens)
+    if out is None:
+        A = torch.zeros((B, T, H, C), dtype=torch.float32, device=K_raw.device) if want_A else None
+        W, U = torch.zeros_like(K_raw), torch.zeros_like(V)
+        bo = torch.zeros((B, T, H), dtype=torch.float32, device=K_raw.device) if want_gates else None
+        go = torch.zeros((B, T, H), dtype=torch.float32, device=K_raw.device) if want_gates else None
+    else:
+        A, W, U, bo, go = out
+    rc = load().tri_inv_fused_raw(_p(K_raw), _p(V), _p(beta_logit), _p(gate_logit), _p(A), _p(W), _p(U), _p(bo), _p(go),
+                                  ctypes.byref(desc), int(method), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_fused_raw", rc)
+    return A, W, U, bo, go
 
 
 def fused_packed_static(K, V, beta, g, C, cu_seqlens, method=BLOCK_RECURSIVE, out=None, stream=None):

@@ -189,6 +189,24 @@ int tri_inv_fused(const void* K, const void* V, const float* beta, const float* 
   return run(p, desc, cuda_stream);
 }
 
+int tri_inv_fused_raw(const void* K_raw, const void* V, const float* beta_logit, const float* gate_logit,
+                      float* A, void* W, void* U, float* beta_out, float* g_out,
+                      const tri_inv_desc* desc, int method, void* cuda_stream) {
+  int rc = check_desc(desc, true);
+  if (rc) return rc;
+  if (!K_raw || !V || !beta_logit || !gate_logit || !W || !U) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(K_raw) || !aligned16(V) || !aligned16(beta_logit) || !aligned16(gate_logit) || !aligned16(A) ||
+      !aligned16(W) || !aligned16(U) || !aligned16(beta_out) || !aligned16(g_out))
+    return TRI_INV_ERR_INVALID_ARG;
+  if ((rc = check_method(method))) return rc;
+  KParams p{};
+  p.K = K_raw; p.V = V; p.beta = beta_logit; p.g = gate_logit; p.A = A; p.W = W; p.U = U;
+  p.beta_out = beta_out; p.g_out = g_out;
+  p.method = method;
+  p.ops = kDoWY | kRaw | (A ? kStoreA : 0);
+  return run(p, desc, cuda_stream);
+}
+
 int tri_inv_count_matrices(const tri_inv_desc* desc, int64_t* out) {
   int rc = check_desc(desc, false);
   if (rc) return rc;

@@ -13,6 +13,7 @@ enum : int {
   kStoreA = 1,  // write A to global memory
   kDoWY = 2,    // compute W (and U when V != nullptr)
   kLoadA = 4,   // skip build + inversion, read A from A_in (tri_inv_wy)
+  kRaw = 8,     // K is un-normalised, beta and g are logits: normalise, sigmoid, log-sigmoid + chunk cumsum in the kernel
 };
 
 // One entry per chunk of tokens in ragged mode.
@@ -30,6 +31,8 @@ struct KParams {
   float* A;
   void* W;
   void* U;
+  float* beta_out;              // raw front end: sigmoid(beta logits), optional
+  float* g_out;                 // raw front end: within-chunk cumulative log-decay, optional
   const ChunkEntry* chunk_tab;  // ragged mode, else nullptr
   int* status;                  // device status word (0 = ok); kernels only ever raise it
   int* work_counter;            // tensor-core kernel: {next dynamic item, finished CTAs}; both zero between launches

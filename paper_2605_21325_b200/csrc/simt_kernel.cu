@@ -23,7 +23,7 @@ constexpr int kSliceLd = kSlice + 1;  // padded row length of the staging tile
 template <int C>
 struct SimtSmem {
   static constexpr int LD = C + 1;
-  static constexpr size_t floats = 3 * (size_t)C * LD + (size_t)C * kSliceLd + 2 * C;
+  static constexpr size_t floats = 3 * (size_t)C * LD + (size_t)C * kSliceLd + 3 * C;
   static constexpr size_t bytes = floats * sizeof(float);
 };
 
@@ -106,6 +106,8 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
   float* Ks = Zm + C * LD;  // [C][kSliceLd]
   float* sb = Ks + C * kSliceLd;
   float* sg = sb + C;
+  float* sr = sg + C;  // raw front end: 1 / |k_i|
+  const bool raw = (p.ops & kRaw) != 0;
   const int tid = threadIdx.x;
   const int total = p.n_chunks * p.H;
   constexpr int kAcc = (C * C + kThreads - 1) / kThreads;
@@ -117,8 +119,26 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
     __syncthreads();  // previous item's readers are done with shared memory
     for (int i = tid; i < C; i += kThreads) {
       size_t bi = (size_t)(tok0 + i) * p.H + h;
-      sb[i] = (i < rows) ? p.beta[bi] : 0.f;
-      sg[i] = (i < rows && p.g) ? p.g[bi] : 0.f;
+      float b = (i < rows) ? p.beta[bi] : 0.f;
+      float gg = (i < rows && p.g) ? p.g[bi] : 0.f;
+      if (raw) {  // beta logits -> sigmoid; gate logits -> log sigmoid (summed over the chunk below)
+        b = (i < rows) ? 1.f / (1.f + expf(-b)) : 0.f;
+        gg = (i < rows) ? fminf(gg, 0.f) - log1pf(expf(-fabsf(gg))) : 0.f;
+        if (p.beta_out && i < rows) p.beta_out[bi] = b;
+      }
+      sb[i] = b;
+      sg[i] = gg;
+      sr[i] = 1.f;
+    }
+    if (raw) {
+      __syncthreads();
+      if (tid == 0) {  // within-chunk cumulative log-decay, in token order
+        float run = 0.f;
+        for (int i = 0; i < C; ++i) { run += sg[i]; sg[i] = run; }
+      }
+      __syncthreads();
+      if (p.g_out)
+        for (int i = tid; i < rows; i += kThreads) p.g_out[(size_t)(tok0 + i) * p.H + h] = sg[i];
     }
     for (int e = tid; e < C * LD; e += kThreads) { Xm[e] = 0.f; Zm[e] = 0.f; Nm[e] = 0.f; }
     float* Xres = Xm;
@@ -148,7 +168,7 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
         for (int m = 0; m < kAcc; ++m) {
           int e = tid + m * kThreads;
           int i = e / C, j = e - i * C;
-          if (e < C * C && j < i) {
+          if (e < C * C && (j < i || (raw && j == i))) {
             float s = acc[m];
 #pragma unroll
             for (int kk = 0; kk < kSlice; ++kk) s = fmaf(Ks[i * kSliceLd + kk], Ks[j * kSliceLd + kk], s);
@@ -156,12 +176,21 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
           }
         }
       }
+      if (raw) {  // 1 / |k_i| from the Gram diagonal; the Gram of the normalised keys is S_ij r_i r_j
+#pragma unroll
+        for (int m = 0; m < kAcc; ++m) {
+          int e = tid + m * kThreads;
+          int i = e / C, j = e - i * C;
+          if (e < C * C && j == i) sr[i] = acc[m] > 0.f ? rsqrtf(acc[m]) : 0.f;
+        }
+        __syncthreads();
+      }
       // ---- gate and mask: select, never multiply an overflowed exp by zero
 #pragma unroll
       for (int m = 0; m < kAcc; ++m) {
         int e = tid + m * kThreads;
         int i = e / C, j = e - i * C;
-        if (e < C * C && j < i && i < rows) Nm[i * LD + j] = sb[i] * acc[m] * expf(sg[i] - sg[j]);
+        if (e < C * C && j < i && i < rows) Nm[i * LD + j] = sb[i] * (acc[m] * sr[i] * sr[j]) * expf(sg[i] - sg[j]);
       }
       __syncthreads();
 
@@ -321,7 +350,7 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
           for (int e = tid; e < C * kSlice; e += kThreads) {
             int j = e / kSlice, cc = e - j * kSlice;
             float v = 0.f;
-            if (j < rows && c0 + cc < d) v = sb[j] * load_kv(src, p.kv_dtype, ((size_t)(tok0 + j) * p.H + h) * d + c0 + cc);
+            if (j < rows && c0 + cc < d) v = sb[j] * (which ? 1.f : sr[j]) * load_kv(src, p.kv_dtype, ((size_t)(tok0 + j) * p.H + h) * d + c0 + cc);
             Ks[j * kSliceLd + cc] = v;
           }
           __syncthreads();

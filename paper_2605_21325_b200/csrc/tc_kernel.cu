@@ -147,7 +147,9 @@ struct Cfg {
   static constexpr int LEAF_BYTES = NW * 16 * LEAF_LD * 4;
   // three mbarriers, the TMEM base-address slot, the next-item slot, then the leaf scratch (inside A' with ALIAS)
   static constexpr int OFF_LEAF = ALIAS ? OFF_AP : OFF_BAR + 32;
-  static constexpr int END_PLAIN = ALIAS ? OFF_BAR + 32 : OFF_LEAF + LEAF_BYTES;
+  // raw front end: 1 / |k_i| per row, and the per-warp totals of the log-decay scan
+  static constexpr int OFF_R = ALIAS ? OFF_BAR + 32 : OFF_LEAF + LEAF_BYTES;
+  static constexpr int END_PLAIN = OFF_R + C * 4 + 32;
   // product-series variant at C = 128: X needs a buffer of its own (at C = 64 it fits where the V tile was)
   static constexpr int OFF_XS = (END_PLAIN + 1023) / 1024 * 1024;
   static constexpr int BYTES = (SER && C == 128) ? OFF_XS + C * C * 4 : END_PLAIN;
@@ -400,6 +402,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
   float* sX = reinterpret_cast<float*>(smem + cfg::OFF_X);
   float* sBeta = reinterpret_cast<float*>(smem + cfg::OFF_BETA);
   float* sG = reinterpret_cast<float*>(smem + cfg::OFF_G);
+  float* sR = reinterpret_cast<float*>(smem + cfg::OFF_R);          // raw front end: 1 / |k_i|
+  float* sScan = sR + C;                                            // raw front end: scan totals per warp
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 24);
   volatile int* s_next_item = reinterpret_cast<volatile int*>(smem + cfg::OFF_BAR + 28);
   const uint32_t sK = smem_u32(smem + cfg::OFF_K);
@@ -420,6 +424,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
   const bool do_wy = (p.ops & kDoWY) != 0;
   const bool need_v = do_wy && p.V != nullptr;
   const bool load_a = (p.ops & kLoadA) != 0;
+  const bool raw = (p.ops & kRaw) != 0;
   const int total = p.n_chunks * p.H;
 
   // Thread 0 requests the tiles of an item; K and V complete on separate barriers so that the Gram
@@ -507,7 +512,32 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
 
     // ---- 1. beta, g were fetched during the previous item (sBeta and sG are adjacent: one store each)
     // g is kept multiplied by log2(e) so that the gate can use ex2 directly
-    sBeta[tid] = bg_next * (tid < C ? 1.f : 1.4426950408889634f);
+    if (!raw) {
+      sBeta[tid] = bg_next * (tid < C ? 1.f : 1.4426950408889634f);
+    } else {
+      // raw front end: beta = sigmoid(logit); g = cumulative sum over the chunk of log sigmoid(gate logit)
+      const int i = tid < C ? tid : tid - C;
+      const size_t gi = (size_t)(tok0 + i) * p.H + h;
+      if (tid < C) {
+        const float b = (i < rows) ? 1.f / (1.f + __expf(-bg_next)) : 0.f;
+        sBeta[i] = b;
+        if (p.beta_out && i < rows) p.beta_out[gi] = b;
+      }
+      float a = 0.f;
+      if (tid >= C && i < rows) a = fminf(bg_next, 0.f) - log1pf(__expf(-fabsf(bg_next)));
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const float y = __shfl_up_sync(0xffffffffu, a, off);
+        if (lane >= off) a += y;
+      }
+      if (tid >= C && lane == 31) sScan[warp - cfg::NW / 2] = a;
+      __syncthreads();
+      if (tid >= C) {
+        for (int w = 0; w < warp - cfg::NW / 2; ++w) a += sScan[w];
+        sG[i] = a * 1.4426950408889634f;
+        if (p.g_out && i < rows) p.g_out[gi] = a;
+      }
+    }
     const bool has_next = nx_item < total;
     int nx_tok0 = 0, nx_rows = 0, nx_h = 0;   // the next item of this CTA
     if (has_next) locate(p, C, nx_item, nx_tok0, nx_rows, nx_h);
@@ -557,6 +587,32 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
       }
       fence_proxy_async();
     };
+    // raw front end: the K tile in shared memory becomes the normalised keys (row i times 1 / |k_i|, bf16 in place)
+    auto rescale_k_tile = [&]() {
+      for (int e = tid; e < C * 8 * cfg::NBOX; e += cfg::NT) {
+        const int bx = e / (C * 8), rem = e - bx * (C * 8), r = rem >> 3, c = rem & 7;
+        uint4* ptr = reinterpret_cast<uint4*>(smem + cfg::OFF_K + bx * cfg::BOX_BYTES + r * 128 + c * 16);
+        uint4 v = *ptr;
+        const float sc = sR[r];
+        uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float2 f = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[q]));
+          w[q] = pack_bf16(f.x * sc, f.y * sc);
+        }
+        *ptr = v;
+      }
+    };
+    // after K (and V) were requested again for the WY step: padding rows cleared, keys normalised
+    auto finish_reload = [&]() -> bool {
+      if (rows < C || raw) {
+        if (!mbar_wait_bounded(bar_k, ph_k) || (need_v && rows < C && !mbar_wait_bounded(bar_v, ph_v))) return false;
+        if (rows < C) clear_tail_rows(true, need_v);
+        if (raw) { rescale_k_tile(); fence_proxy_async(); }
+        __syncthreads();
+      }
+      return true;
+    };
     if (rows < C) {
       const bool v_now = need_v && !cfg::RELOAD, k_now = !(cfg::ALIAS && load_a);
       if ((k_now && !mbar_wait_bounded(bar_k, ph_k)) || (v_now && !mbar_wait_bounded(bar_v, ph_v))) { failed = true; break; }
@@ -582,6 +638,20 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
       tc_fence_after();
       if (tid == kTidK && !do_wy && !cfg::RELOAD && has_next) issue_k(nx_tok0, nx_h);  // K's last reader was the Gram product
       PHASE(1);
+      // raw front end: the Gram diagonal is |k_i|^2; 1 / |k_i| of this warp's rows goes to shared memory for
+      // every warp's gate (S_ij r_i r_j is the Gram entry of the normalised keys) and for the K tile's rescaling
+      auto publish_inv_norms = [&](const float (&sacc)[C / 8][4]) {
+#pragma unroll
+        for (int jb = 0; jb < cfg::NW; ++jb) {
+          if (jb == rb && t == (g >> 1)) {
+            const float da = (g & 1) ? sacc[2 * jb][1] : sacc[2 * jb][0];
+            const float db = (g & 1) ? sacc[2 * jb + 1][3] : sacc[2 * jb + 1][2];
+            sR[16 * rb + g] = da > 0.f ? rsqrtf(da) : 0.f;
+            sR[16 * rb + g + 8] = db > 0.f ? rsqrtf(db) : 0.f;
+          }
+        }
+        __syncthreads();
+      };
 
       if constexpr (SER) {
         // ---- 3'. product series (Alg. 5) on the tensor core.  Y (= N at first) and X (= I - N at first)
@@ -617,16 +687,23 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
           float sacc[C / 8][4];
           if constexpr (C == 64) tmem_ld_16x64(sacc, tmem_rows); else tmem_ld_16x128(sacc, tmem_rows);
           tmem_wait_ld();
+          float ba = beta_a, bb = beta_b;
+          if (raw) {
+            publish_inv_norms(sacc);
+            ba *= sR[ra];
+            bb *= sR[rbw];
+          }
 #pragma unroll
           for (int nt = 0; nt < C / 8; ++nt) {
             const int c = 8 * nt + 2 * t;
             float2 na = make_float2(0.f, 0.f), nb = na;
             if (nt / 2 <= rb) {  // tiles on or below the diagonal of this row block
               const float2 gc = *reinterpret_cast<const float2*>(sG + c);
-              na.x = (c < ra) ? beta_a * sacc[nt][0] * ex2_approx(g_a - gc.x) : 0.f;
-              na.y = (c + 1 < ra) ? beta_a * sacc[nt][1] * ex2_approx(g_a - gc.y) : 0.f;
-              nb.x = (c < rbw) ? beta_b * sacc[nt][2] * ex2_approx(g_b - gc.x) : 0.f;
-              nb.y = (c + 1 < rbw) ? beta_b * sacc[nt][3] * ex2_approx(g_b - gc.y) : 0.f;
+              const float2 rc = raw ? *reinterpret_cast<const float2*>(sR + c) : make_float2(1.f, 1.f);
+              na.x = (c < ra) ? ba * rc.x * sacc[nt][0] * ex2_approx(g_a - gc.x) : 0.f;
+              na.y = (c + 1 < ra) ? ba * rc.y * sacc[nt][1] * ex2_approx(g_a - gc.y) : 0.f;
+              nb.x = (c < rbw) ? bb * rc.x * sacc[nt][2] * ex2_approx(g_b - gc.x) : 0.f;
+              nb.y = (c + 1 < rbw) ? bb * rc.y * sacc[nt][3] * ex2_approx(g_b - gc.y) : 0.f;
             }
             xr[nt][0] = (c == ra ? 1.f : 0.f) - na.x;
             xr[nt][1] = (c + 1 == ra ? 1.f : 0.f) - na.y;
@@ -715,11 +792,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
           if (tid == kTidK) issue_k(tok0, h);
           if (tid == kTidV && need_v) issue_v(tok0, h);
           ph_k ^= 1;
-          if (rows < C) {
-            if (!mbar_wait_bounded(bar_k, ph_k) || (need_v && !mbar_wait_bounded(bar_v, ph_v))) { failed = true; break; }
-            clear_tail_rows(true, need_v);
-            __syncthreads();
-          }
+          if (!finish_reload()) { failed = true; break; }
         }
       } else {
       // ---- 3. gate + mask on this warp's rows, N -> shared memory
@@ -729,6 +802,12 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
         float sacc[C / 8][4];   // this warp's 16 rows of S, all C columns, in one tensor-memory load
         if constexpr (C == 64) tmem_ld_16x64(sacc, tmem_rows); else tmem_ld_16x128(sacc, tmem_rows);
         tmem_wait_ld();
+        float ba = beta_a, bb = beta_b;
+        if (raw) {
+          publish_inv_norms(sacc);
+          ba *= sR[ra];
+          bb *= sR[rbw];
+        }
 #pragma unroll
         for (int jb = 0; jb < cfg::NW; ++jb) {
           if (jb > rb) {
@@ -744,12 +823,13 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
             for (int nt = 0; nt < 2; ++nt) {
               const int c = 16 * jb + 8 * nt + 2 * t;
               const float2 gc = *reinterpret_cast<const float2*>(sG + c);
+              const float2 rc = raw ? *reinterpret_cast<const float2*>(sR + c) : make_float2(1.f, 1.f);
               const float (&a4)[4] = sacc[2 * jb + nt];
               float2 va, vb;
-              va.x = beta_a * a4[0] * ex2_approx(g_a - gc.x);
-              va.y = beta_a * a4[1] * ex2_approx(g_a - gc.y);
-              vb.x = beta_b * a4[2] * ex2_approx(g_b - gc.x);
-              vb.y = beta_b * a4[3] * ex2_approx(g_b - gc.y);
+              va.x = ba * rc.x * a4[0] * ex2_approx(g_a - gc.x);
+              va.y = ba * rc.y * a4[1] * ex2_approx(g_a - gc.y);
+              vb.x = bb * rc.x * a4[2] * ex2_approx(g_b - gc.x);
+              vb.y = bb * rc.y * a4[3] * ex2_approx(g_b - gc.y);
               if (jb == rb) {  // the diagonal tile: strict-lower mask by selection
                 va.x = (c < ra) ? va.x : 0.f;
                 va.y = (c + 1 < ra) ? va.y : 0.f;
@@ -850,11 +930,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
         if (tid == kTidK) issue_k(tok0, h);
         if (tid == kTidV && need_v) issue_v(tok0, h);
         if (!load_a) ph_k ^= 1;  // second K copy of this item
-        if (rows < C) {
-          if (!mbar_wait_bounded(bar_k, ph_k) || (need_v && !mbar_wait_bounded(bar_v, ph_v))) { failed = true; break; }
-          clear_tail_rows(true, need_v);
-          __syncthreads();
-        }
+        if (!finish_reload()) { failed = true; break; }
       } else {
         tc_fence_before();
         __syncthreads();  // every read of the fp32 matrix (and of S in TMEM) is done: its space becomes A'
@@ -864,6 +940,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
           const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
           put_ap(i, j, xv[m]);
         }
+        if (raw && !cfg::RELOAD) rescale_k_tile();  // the Gram product, K's only reader so far, has completed
         fence_proxy_async();  // generic-proxy writes of A' become visible to the tensor core's reads
         __syncthreads();
       }

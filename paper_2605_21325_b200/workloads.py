@@ -128,6 +128,21 @@ def make(name, B, T, H, d_k, d_v, C, kv_dtype, seed, kind="gdn", cu_seqlens=None
                   np.ascontiguousarray(beta), np.ascontiguousarray(g), cu, {"kind": kind, "seed": seed})
 
 
+def make_raw(name, B, T, H, d, C, kv_dtype, seed, cu_seqlens=None):
+    """Inputs of the fused front end: un-normalised keys K ~ N(0,1) (row norms around sqrt(d)), values
+    V ~ N(0,1), beta logits ~ N(0,1) and gate logits ~ N(2,1) -- what the projections of a
+    Gated-DeltaNet layer hand over before sigmoid, log-sigmoid + cumsum and key normalisation.
+    Returned as an Inputs whose ``beta`` holds the beta logits and ``g`` the gate logits."""
+    rng = np.random.default_rng(seed)
+    K = rng.standard_normal((B, T, H, d), dtype=np.float32)
+    V = rng.standard_normal((B, T, H, d), dtype=np.float32)
+    zb = rng.standard_normal((B, T, H), dtype=np.float32)
+    zg = rng.standard_normal((B, T, H), dtype=np.float32) + np.float32(2.0)
+    cu = None if cu_seqlens is None else np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    return Inputs(name, B, T, H, d, d, C, kv_dtype, _store(K, kv_dtype), _store(V, kv_dtype), zb, zg, cu,
+                  {"kind": "raw", "seed": seed})
+
+
 def ragged_lengths(n_seqs: int, max_len: int, rng) -> np.ndarray:
     lens = rng.integers(1, max_len + 1, size=n_seqs)
     return np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)

@@ -328,3 +328,35 @@ def test_newton_schulz_and_refinement_converge_to_substitution():
     assert r1 < 64 * r0 * r0
     # refinement leaves an exact inverse unchanged
     assert np.abs(alg.iterative_refinement(a, L) - a).max() < 1e-14
+
+
+# ---------------------------------------------------------------- raw front end (sigmoid, log-sigmoid + chunk cumsum, key norm)
+
+def test_raw_front_end_hand_values_and_generator_recipe():
+    # hand values: sigmoid(0) = 1/2, log sigmoid(0) = -ln 2, (3,4) / 5 = (0.6, 0.8)
+    K = np.array([[3.0, 4.0], [0.0, 2.0], [0.0, 0.0]], np.float32).reshape(1, 3, 1, 2)
+    Kh, b, g = oracle.raw_front_end(K, np.zeros((1, 3, 1)), np.zeros((1, 3, 1)), 2)
+    assert np.allclose(Kh[0, :, 0], [[0.6, 0.8], [0.0, 1.0], [0.0, 0.0]], atol=1e-15)   # a zero key stays zero
+    assert np.array_equal(b[0, :, 0], [0.5, 0.5, 0.5])
+    assert np.allclose(g[0, :, 0], [-np.log(2), -2 * np.log(2), -np.log(2)], atol=1e-15)  # the sum restarts at the chunk (C = 2)
+    # large |logit|: no overflow, log sigmoid(-50) = -50 - log1p(e^-50), log sigmoid(50) = -e^-50
+    _, b, g = oracle.raw_front_end(K, np.array([50.0, -50.0, 0.0]).reshape(1, 3, 1), np.array([-50.0, 50.0, 0.0]).reshape(1, 3, 1), 4)
+    assert abs(b[0, 0, 0] - 1.0) < 1e-15 and 0 < b[0, 1, 0] < 1e-20
+    assert abs(g[0, 0, 0] + 50.0) < 1e-12 and abs(g[0, 1, 0] + 50.0) < 1e-12
+    # the generator of the configurations applies the same recipe (in fp32): same A up to fp32 rounding
+    raw = wl.make_raw("raw", 2, 160, 2, 32, 64, wl.F32, seed=17)
+    Kh, b, g = oracle.raw_front_end(raw.K, raw.beta, raw.g, 64)
+    assert np.abs(np.linalg.norm(Kh, axis=-1) - 1).max() < 1e-12
+    assert (np.diff(g.reshape(2, 160, 2)[:, :64], axis=1) <= 0).all()       # log-decays are negative inside a chunk
+    rng = np.random.default_rng(17)                                          # wl.make draws K, V, beta, g noise in this order
+    ref = wl.make("prep", 2, 160, 2, 32, 32, 64, wl.F32, seed=17, rng=rng)
+    assert np.abs(oracle.build_A(Kh, b, g, 64) - oracle.build_A(ref.K, ref.beta, ref.g, 64)).max() < 5e-6
+    # ragged: the sum restarts at every sequence and chunk
+    cu = np.array([0, 70, 160], np.int32)
+    raw1 = wl.make_raw("raw", 1, 160, 2, 32, 64, wl.F32, seed=18, cu_seqlens=cu)
+    _, _, g = oracle.raw_front_end(raw1.K, raw1.beta, raw1.g, 64, cu_seqlens=cu)
+    z = raw1.g.astype(np.float64)
+    ls = np.minimum(z, 0) - np.log1p(np.exp(-np.abs(z)))
+    for t in (0, 64, 70, 134):
+        assert np.allclose(g[0, t], ls[0, t], atol=1e-15)
+    assert np.allclose(g[0, 69], ls[0, 64:70].sum(axis=0), atol=1e-13)

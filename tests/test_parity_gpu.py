@@ -328,3 +328,52 @@ def test_method_flag_combinations_rejected(bnd):
     for bad in (bnd.PRODUCT_SERIES | bnd.REFINE, bnd.BLOCK_RECURSIVE | bnd.ns_iters(4), bnd.NEWTON_SCHULZ | bnd.LEAF_SERIES, 3):
         rc = L.tri_inv_build(bnd._p(d), bnd._p(d), bnd._p(d), bnd._p(d), ctypes.byref(desc), bad, None)
         assert rc == bnd.ERR_UNSUPPORTED, bad
+
+
+# ---------------------------------------------------------------- fused front end (raw keys and logits)
+
+def oracle_raw(raw):
+    Kh, b, g = oracle.raw_front_end(raw.K, raw.beta, raw.g, raw.C, cu_seqlens=raw.cu_seqlens)
+    A, N = oracle.build_A(Kh, b, g, raw.C, cu_seqlens=raw.cu_seqlens, return_N=True)
+    W, U = oracle.wy(A, Kh, raw.V, b, raw.C, cu_seqlens=raw.cu_seqlens)
+    return A, N, W, U, b, g
+
+
+@pytest.mark.parametrize("C,dtype,d", [(64, wl.BF16, 128), (128, wl.BF16, 128), (64, wl.F32, 64), (32, wl.BF16, 64)])
+def test_fused_raw_front_end(bnd, C, dtype, d):
+    cu = np.array([0, 3 * C + 7, 5 * C + 7, 5 * C + 8], np.int32)          # partial chunks and a one-token sequence
+    for cu_seqlens, B, T in ((None, 2, 4 * C), (cu, 1, int(cu[-1]))):
+        raw = wl.make_raw("raw", B, T, 3, d, C, dtype, seed=60 + C, cu_seqlens=cu_seqlens)
+        A_ref, N_ref, W_ref, U_ref, b_ref, g_ref = oracle_raw(raw)
+        dev = bnd.to_device(raw)
+        for m in methods(bnd):
+            out = (nan_like((B, T, 3, C), torch.float32), nan_like(dev["K"].shape, dev["K"].dtype), nan_like(dev["V"].shape, dev["V"].dtype),
+                   nan_like((B, T, 3), torch.float32), nan_like((B, T, 3), torch.float32))
+            A, W, U, bo, go = bnd.fused_raw(dev["K"], dev["V"], dev["beta"], dev["g"], C, method=m, cu_seqlens=cu_seqlens, out=out)
+            torch.cuda.synchronize()
+            assert bnd.last_device_status() == 0
+            check_A(A, raw, A_ref, N_ref)
+            check_WU(W, U, raw, W_ref, U_ref, bnd)
+            assert np.abs(bo.cpu().numpy() - b_ref).max() <= 1e-6
+            assert np.abs(go.cpu().numpy() - g_ref).max() <= 1e-5 * max(1.0, np.abs(g_ref).max())
+        # gates are optional
+        A2, W2, U2, bo2, go2 = bnd.fused_raw(dev["K"], dev["V"], dev["beta"], dev["g"], C, cu_seqlens=cu_seqlens)
+        torch.cuda.synchronize()
+        assert bo2 is None and go2 is None
+        check_A(A2, raw, A_ref, N_ref)
+
+
+def test_fused_raw_equals_fused_on_prepared_inputs(bnd):
+    # the same layer step done in two passes (front end on the host in fp32, then tri_inv_fused) and in one
+    raw = wl.make_raw("raw", 2, 256, 4, 128, 64, wl.BF16, seed=71)
+    Kh, b, g = oracle.raw_front_end(raw.K, raw.beta, raw.g, 64)
+    prep = wl.Inputs("prep", 2, 256, 4, 128, 128, 64, wl.BF16, wl.f32_to_bf16_bits(Kh.astype(np.float32)), raw.V,
+                     b.astype(np.float32), g.astype(np.float32))
+    d_raw, d_prep = bnd.to_device(raw), bnd.to_device(prep)
+    A1, W1, U1, _, _ = bnd.fused_raw(d_raw["K"], d_raw["V"], d_raw["beta"], d_raw["g"], 64)
+    A2, W2, U2 = bnd.fused(d_prep["K"], d_prep["V"], d_prep["beta"], d_prep["g"], 64)
+    torch.cuda.synchronize()
+    # two-pass keys are rounded to bf16 after normalising, the fused path normalises the Gram in fp32: close, not equal
+    assert (A1 - A2).abs().max().item() <= 2e-3
+    assert (W1.float() - W2.float()).abs().max().item() <= 1e-2 * W2.float().abs().max().item()
+    assert (U1.float() - U2.float()).abs().max().item() <= 1e-2 * U2.float().abs().max().item()
