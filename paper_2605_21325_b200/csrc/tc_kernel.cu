@@ -391,7 +391,7 @@ __device__ __forceinline__ void store_piece_bf16(uint32_t taddr, uint32_t stage,
   store_frag_piece_bf16(f, stage, lane, out_row0, row_stride, rows_left);
 }
 
-template <int C, int D, bool SER>
+template <int C, int D, bool SER, bool RAW>
 __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                              const __grid_constant__ CUtensorMap tmV, KParams p) {
   using cfg = Cfg<C, D, SER>;
@@ -424,7 +424,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
   const bool do_wy = (p.ops & kDoWY) != 0;
   const bool need_v = do_wy && p.V != nullptr;
   const bool load_a = (p.ops & kLoadA) != 0;
-  const bool raw = (p.ops & kRaw) != 0;
+  constexpr bool raw = RAW;  // the front end (sigmoid, log-sigmoid + chunk cumsum, key normalisation) is compiled in or out
   const int total = p.n_chunks * p.H;
 
   // Thread 0 requests the tiles of an item; K and V complete on separate barriers so that the Gram
@@ -1117,7 +1117,7 @@ int* next_work_counter() {
   return base[dev] + 2 * (turn++ % 64);
 }
 
-template <int C, int D, bool SER>
+template <int C, int D, bool SER, bool RAW>
 cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   using cfg = Cfg<C, D, SER>;
   KParams p = p_in;
@@ -1125,9 +1125,9 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   if (!p.work_counter) return cudaErrorUnknown;
   static int ctas_per_sm = 0, n_sm = 0;
   if (!ctas_per_sm) {
-    cudaError_t e = cudaFuncSetAttribute(tc_kernel<C, D, SER>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
+    cudaError_t e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(tc_kernel<C, D, SER>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -1152,7 +1152,7 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   long long total = (long long)p.n_chunks * p.H;
   long long cap = (long long)n_sm * ctas_per_sm;
   int grid = (int)(total < cap ? total : cap);
-  tc_kernel<C, D, SER><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
+  tc_kernel<C, D, SER, RAW><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
   return cudaGetLastError();
 }
 
@@ -1171,8 +1171,15 @@ cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handle
   if (p.d_k != 128 || ((p.ops & kDoWY) && p.V && p.d_v != 128)) return cudaSuccess;
   // the stride of the 2-D view (H * d * 2 bytes) is a multiple of 16 because d is a multiple of 8
   *handled = true;
-  if (C == 64) return series ? launch_one<64, 128, true>(p, stream) : launch_one<64, 128, false>(p, stream);
-  if (C == 128) return series ? launch_one<128, 128, true>(p, stream) : launch_one<128, 128, false>(p, stream);
+  const bool raw = (p.ops & kRaw) != 0;
+  if (C == 64) {
+    if (raw) return series ? launch_one<64, 128, true, true>(p, stream) : launch_one<64, 128, false, true>(p, stream);
+    return series ? launch_one<64, 128, true, false>(p, stream) : launch_one<64, 128, false, false>(p, stream);
+  }
+  if (C == 128) {
+    if (raw) return series ? launch_one<128, 128, true, true>(p, stream) : launch_one<128, 128, false, true>(p, stream);
+    return series ? launch_one<128, 128, true, false>(p, stream) : launch_one<128, 128, false, false>(p, stream);
+  }
   *handled = false;
   return cudaSuccess;
 }
