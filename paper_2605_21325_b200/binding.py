@@ -218,6 +218,63 @@ def fused_packed_static(K, V, beta, g, C, cu_seqlens, method=BLOCK_RECURSIVE, ou
     return A, W, U
 
 
+class HostPipeline:
+    """tri_inv_fused for callers whose tensors live in pinned host memory.
+
+    The batch is cut into slices (whole sequences when B >= n_slices, else whole chunks of one sequence) and
+    each slice goes host -> device, through the fused kernel, and device -> host on its own stream, so the
+    upload of one slice overlaps the kernel of the previous one and the download of the one before.  Device
+    buffers are allocated once here; ``run`` allocates nothing.  Dense mode only (packed batches: one slice)."""
+
+    def __init__(self, B, T, H, d_k, d_v, C, dtype=torch.bfloat16, n_slices=4, n_streams=3, cu_seqlens=None, device="cuda"):
+        self.shape = (B, T, H, d_k, d_v, C)
+        self.cu_seqlens = cu_seqlens
+        self.K = torch.empty((B, T, H, d_k), dtype=dtype, device=device)
+        self.V = torch.empty((B, T, H, d_v), dtype=dtype, device=device)
+        self.beta = torch.empty((B, T, H), dtype=torch.float32, device=device)
+        self.g = torch.empty((B, T, H), dtype=torch.float32, device=device)
+        self.A = torch.empty((B, T, H, C), dtype=torch.float32, device=device)
+        self.W, self.U = torch.empty_like(self.K), torch.empty_like(self.V)
+        if cu_seqlens is not None:
+            self.slices = [(0, slice(None))]                      # axis, range
+        elif B >= n_slices:
+            step = -(-B // n_slices)
+            self.slices = [(0, slice(b, min(b + step, B))) for b in range(0, B, step)]
+        elif B == 1 and T >= n_slices * C:
+            step = -(-(T // C) // n_slices) * C
+            self.slices = [(1, slice(t, min(t + step, T))) for t in range(0, T, step)]
+        else:
+            self.slices = [(0, slice(None))]
+        self.streams = [torch.cuda.Stream(device=device) for _ in range(min(n_streams, len(self.slices)))]
+
+    @staticmethod
+    def _cut(t, axis, rng):
+        return t[rng] if axis == 0 else t[:, rng]
+
+    def run(self, hK, hV, hbeta, hg, hA, hW, hU, method=BLOCK_RECURSIVE):
+        """All arguments are pinned host tensors of the full batch; hA may be None.  Returns after enqueueing;
+        the current stream is made to wait for every slice, so a synchronize (or event) on it covers the call."""
+        C = self.shape[5]
+        cur = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(cur)
+        for n, (axis, rng) in enumerate(self.slices):
+            st = self.streams[n % len(self.streams)]
+            st.wait_event(start)
+            with torch.cuda.stream(st):
+                cut = lambda t: self._cut(t, axis, rng)
+                for dst, src in ((self.K, hK), (self.V, hV), (self.beta, hbeta), (self.g, hg)):
+                    cut(dst).copy_(cut(src), non_blocking=True)
+                fused(cut(self.K), cut(self.V), cut(self.beta), cut(self.g), C, method=method, cu_seqlens=self.cu_seqlens,
+                      out=(cut(self.A) if hA is not None else None, cut(self.W), cut(self.U)), stream=st)
+                if hA is not None:
+                    cut(hA).copy_(cut(self.A), non_blocking=True)
+                cut(hW).copy_(cut(self.W), non_blocking=True)
+                cut(hU).copy_(cut(self.U), non_blocking=True)
+        for st in self.streams:
+            cur.wait_stream(st)
+
+
 # ---- moving workloads.Inputs (numpy, host) to the device and results back -------------------
 
 def kv_to_torch(a: np.ndarray, device="cuda", pin=False) -> torch.Tensor:

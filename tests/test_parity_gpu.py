@@ -377,3 +377,43 @@ def test_fused_raw_equals_fused_on_prepared_inputs(bnd):
     assert (A1 - A2).abs().max().item() <= 2e-3
     assert (W1.float() - W2.float()).abs().max().item() <= 1e-2 * W2.float().abs().max().item()
     assert (U1.float() - U2.float()).abs().max().item() <= 1e-2 * U2.float().abs().max().item()
+
+
+# ---------------------------------------------------------------- host-to-host pipeline
+
+@pytest.mark.parametrize("B,T", [(4, 512), (1, 2048), (2, 192)])
+def test_host_pipeline_matches_single_call(bnd, B, T):
+    inp = wl.make("pipe", B, T, 4, 128, 128, 64, wl.BF16, seed=83)
+    dev = bnd.to_device(inp)
+    A, W, U = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], 64)
+    pipe = bnd.HostPipeline(B, T, 4, 128, 128, 64)
+    hK, hV = bnd.kv_to_torch(inp.K, "cpu", pin=True), bnd.kv_to_torch(inp.V, "cpu", pin=True)
+    hb, hg = torch.from_numpy(inp.beta).pin_memory(), torch.from_numpy(inp.g).pin_memory()
+    hA = torch.full(A.shape, float("nan")).pin_memory()
+    hW, hU = torch.zeros(W.shape, dtype=W.dtype).pin_memory(), torch.zeros(U.shape, dtype=U.dtype).pin_memory()
+    for _ in range(2):
+        pipe.run(hK, hV, hb, hg, hA, hW, hU)
+    torch.cuda.synchronize()
+    assert torch.equal(hA, A.cpu()) and torch.equal(hW, W.cpu()) and torch.equal(hU, U.cpu())
+
+
+def test_concurrent_launches_on_two_streams(bnd):
+    # launches that overlap on the GPU use different work counters and their own tensor memory
+    inp1, inp2 = wl.config(2, shrink=4), wl.config(4, shrink=4)
+    d1, d2 = bnd.to_device(inp1), bnd.to_device(inp2)
+    ref1 = bnd.fused(d1["K"], d1["V"], d1["beta"], d1["g"], inp1.C)
+    ref2 = bnd.fused(d2["K"], d2["V"], d2["beta"], d2["g"], inp2.C, method=bnd.PRODUCT_SERIES)
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    outs1, outs2 = [], []
+    for _ in range(6):
+        with torch.cuda.stream(s1):
+            outs1.append(bnd.fused(d1["K"], d1["V"], d1["beta"], d1["g"], inp1.C, stream=s1))
+        with torch.cuda.stream(s2):
+            outs2.append(bnd.fused(d2["K"], d2["V"], d2["beta"], d2["g"], inp2.C, method=bnd.PRODUCT_SERIES, stream=s2))
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    for o in outs1:
+        assert all(torch.equal(a, b) for a, b in zip(o, ref1))
+    for o in outs2:
+        assert all(torch.equal(a, b) for a, b in zip(o, ref2))
