@@ -116,8 +116,11 @@ __device__ __forceinline__ unsigned smid() { unsigned r; asm volatile("mov.u32 %
 #endif
 
 // ------------------------------------------------------------------------------------------ layout
-template <int C, int D, bool SER>
+template <int C, int D, bool SER, bool BO = false>
 struct Cfg {
+  // BO: build-only specialisation (tri_inv_build at C = 64): no V tile, no WY operand or staging, 64 TMEM
+  // columns, so six CTAs fit on an SM instead of four.
+  static_assert(!BO || (C == 64 && !SER), "the build-only variant exists for the C = 64 block recursion");
   static constexpr int NW = C / 16;             // warps, one per 16 rows
   static constexpr int NT = NW * 32;
   static constexpr int LD = C + 4;              // fp32 row length of the N/X matrix (LD % 16 == 4)
@@ -132,7 +135,7 @@ struct Cfg {
   static constexpr int OFF_K = 0;
   static constexpr int OFF_V = TILE_BYTES;
   static constexpr int X_BYTES = C * LD * 4;
-  static constexpr int OFF_X = ALIAS ? 0 : 2 * TILE_BYTES;
+  static constexpr int OFF_X = ALIAS ? 0 : (BO ? TILE_BYTES : 2 * TILE_BYTES);
   // A' (bf16, C x C) and the per-warp 2 KiB output staging tiles: inside the N/X matrix's space once it has
   // been read (A' first, staging behind it), or, with ALIAS, in a region of their own where the staging
   // reuses A' after the WY products have completed.
@@ -146,15 +149,16 @@ struct Cfg {
   static constexpr int LEAF_LD = 20;             // per-warp 16 x 16 fp32 scratch of the series leaf
   static constexpr int LEAF_BYTES = NW * 16 * LEAF_LD * 4;
   // three mbarriers, the TMEM base-address slot, the next-item slot, then the leaf scratch (inside A' with ALIAS)
-  static constexpr int OFF_LEAF = ALIAS ? OFF_AP : OFF_BAR + 32;
+  static constexpr int OFF_LEAF = ALIAS ? OFF_AP : (BO ? OFF_K : OFF_BAR + 32);  // BO: in the K tile, dead after the Gram product
   // raw front end: 1 / |k_i| per row, and the per-warp totals of the log-decay scan
-  static constexpr int OFF_R = ALIAS ? OFF_BAR + 32 : OFF_LEAF + LEAF_BYTES;
+  static constexpr int OFF_R = (ALIAS || BO) ? OFF_BAR + 32 : OFF_LEAF + LEAF_BYTES;
   static constexpr int END_PLAIN = OFF_R + C * 4 + 32;
   // product-series variant at C = 128: X needs a buffer of its own (at C = 64 it fits where the V tile was)
   static constexpr int OFF_XS = (END_PLAIN + 1023) / 1024 * 1024;
   static constexpr int BYTES = (SER && C == 128) ? OFF_XS + C * C * 4 : END_PLAIN;
   static constexpr int SMEM = BYTES;
-  static constexpr int CTAS_PER_SM = (C == 64) ? 4 : (ALIAS ? 2 : 1);
+  static constexpr int CTAS_PER_SM = (C == 64) ? (BO ? 6 : 4) : (ALIAS ? 2 : 1);
+  static constexpr int TMEM_COLS = (C == 64) ? (BO ? 64 : 128) : 256;
 };
 
 // Byte offset of the 16-byte chunk holding features [f, f+8) of row r inside a swizzled tile.
@@ -391,13 +395,13 @@ __device__ __forceinline__ void store_piece_bf16(uint32_t taddr, uint32_t stage,
   store_frag_piece_bf16(f, stage, lane, out_row0, row_stride, rows_left);
 }
 
-template <int C, int D, bool SER, bool RAW>
-__global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK,
+template <int C, int D, bool SER, bool RAW, bool BO>
+__global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                              const __grid_constant__ CUtensorMap tmV, KParams p) {
-  using cfg = Cfg<C, D, SER>;
+  using cfg = Cfg<C, D, SER, BO>;
   static_assert(D == 128, "tiles are two 64-feature boxes wide");
   constexpr int LD = cfg::LD;
-  constexpr int TMEM_COLS = (C == 64) ? 128 : 256;
+  constexpr int TMEM_COLS = cfg::TMEM_COLS;
   extern __shared__ __align__(1024) uint8_t smem[];  // swizzled tiles need a 1024-byte aligned base
   float* sX = reinterpret_cast<float*>(smem + cfg::OFF_X);
   float* sBeta = reinterpret_cast<float*>(smem + cfg::OFF_BETA);
@@ -421,7 +425,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
   // the 32-lane quadrant: M = 64 puts rows 16q..16q+15 in lanes 32q..32q+15, M = 128 puts row i in lane i.
   const int rb = (C == 64) ? warp : 2 * (warp & 3) + (warp >> 2);
   const uint32_t lane_base = (C == 64) ? 32u * warp : 16u * rb;
-  const bool do_wy = (p.ops & kDoWY) != 0;
+  const bool do_wy = !BO && (p.ops & kDoWY) != 0;
   const bool need_v = do_wy && p.V != nullptr;
   const bool load_a = (p.ops & kLoadA) != 0;
   constexpr bool raw = RAW;  // the front end (sigmoid, log-sigmoid + chunk cumsum, key normalisation) is compiled in or out
@@ -636,7 +640,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
       if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
       ph_mma ^= 1;
       tc_fence_after();
-      if (tid == kTidK && !do_wy && !cfg::RELOAD && has_next) issue_k(nx_tok0, nx_h);  // K's last reader was the Gram product
+      if (!BO && tid == kTidK && !do_wy && !cfg::RELOAD && has_next) issue_k(nx_tok0, nx_h);  // K's last reader was the Gram product
       PHASE(1);
       // raw front end: the Gram diagonal is |k_i|^2; 1 / |k_i| of this warp's rows goes to shared memory for
       // every warp's gate (S_ij r_i r_j is the Gram entry of the normalised keys) and for the K tile's rescaling
@@ -873,6 +877,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER>::NT, Cfg<C, D, SER>::CTAS_PER_S
         }
       }
       __syncthreads();
+      if (BO && tid == kTidK && has_next) issue_k(nx_tok0, nx_h);  // the leaf scratch inside the K tile is no longer needed
       PHASE(3);
 
       // ---- 5. merges
@@ -1117,17 +1122,17 @@ int* next_work_counter() {
   return base[dev] + 2 * (turn++ % 64);
 }
 
-template <int C, int D, bool SER, bool RAW>
+template <int C, int D, bool SER, bool RAW, bool BO = false>
 cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
-  using cfg = Cfg<C, D, SER>;
+  using cfg = Cfg<C, D, SER, BO>;
   KParams p = p_in;
   p.work_counter = next_work_counter();
   if (!p.work_counter) return cudaErrorUnknown;
   static int ctas_per_sm = 0, n_sm = 0;
   if (!ctas_per_sm) {
-    cudaError_t e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
+    cudaError_t e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -1138,7 +1143,7 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
     int smem_per_sm = 0;
     cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
     int by_smem = smem_per_sm / (cfg::SMEM + 1024);  // 1 KiB per CTA is reserved by the system
-    int by_tmem = 512 / ((C == 64) ? 128 : 256);
+    int by_tmem = 512 / cfg::TMEM_COLS;
     int by_regs = cfg::CTAS_PER_SM;
     int occ = by_smem < by_tmem ? by_smem : by_tmem;
     occ = occ < by_regs ? occ : by_regs;
@@ -1152,7 +1157,7 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   long long total = (long long)p.n_chunks * p.H;
   long long cap = (long long)n_sm * ctas_per_sm;
   int grid = (int)(total < cap ? total : cap);
-  tc_kernel<C, D, SER, RAW><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
+  tc_kernel<C, D, SER, RAW, BO><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
   return cudaGetLastError();
 }
 
@@ -1173,6 +1178,7 @@ cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handle
   *handled = true;
   const bool raw = (p.ops & kRaw) != 0;
   if (C == 64) {
+    if (!raw && !series && !(p.ops & (kDoWY | kLoadA))) return launch_one<64, 128, false, false, true>(p, stream);  // tri_inv_build
     if (raw) return series ? launch_one<64, 128, true, true>(p, stream) : launch_one<64, 128, false, true>(p, stream);
     return series ? launch_one<64, 128, true, false>(p, stream) : launch_one<64, 128, false, false>(p, stream);
   }
