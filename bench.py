@@ -36,7 +36,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per chunk matrix moved by the fused kernel (dram__bytes_read.sum + dram__bytes_write.sum
 # of one ncu capture divided by the matrices of that launch); see profiles/.  None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_MATRIX = {(2, "block_recursive"): 68960}  # profiles/tc_kernel_c64_cfg2.md
+NCU_TRAFFIC_BYTES_PER_MATRIX = {(2, "block_recursive"): 68890}  # profiles/tc_kernel_c64_cfg2.md
 
 
 def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True, call="fused"):
@@ -243,7 +243,7 @@ def main():
     A = torch.empty((inp.B, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda")
     W, U = torch.empty_like(K), torch.empty_like(V)
     flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
-    flush_rd = None if args.no_flush else torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device="cuda")
+    flush_rd = None if args.no_flush else torch.zeros(64 * 1024 * 1024, dtype=torch.float32, device="cuda")
     stream = torch.cuda.current_stream()
 
     def flush_l2():
