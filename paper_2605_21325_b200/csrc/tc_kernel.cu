@@ -50,12 +50,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after kSpinLimit polls (each poll itself blocks for a
-// hardware-defined time slice), so a lost copy cannot hang the GPU.
-constexpr uint32_t kSpinLimit = 1u << 22;
+// Bounded wait: gives up after about two seconds of wall time (the global timer is read every 64 polls,
+// each poll itself blocks for a hardware-defined time slice) or after kSpinLimit polls, whichever comes
+// first, so a lost copy or product cannot hang the GPU.
+constexpr uint32_t kSpinLimit = 1u << 24;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
+  if (mbar_try_wait(bar, parity)) return true;
+  unsigned long long t0;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  for (uint32_t i = 1; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 0) {
+      unsigned long long t1;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+      if (t1 - t0 > kWaitLimitNs) return false;
+    }
+  }
   return false;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -1128,26 +1139,36 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   KParams p = p_in;
   p.work_counter = next_work_counter();
   if (!p.work_counter) return cudaErrorUnknown;
-  static int ctas_per_sm = 0, n_sm = 0;
-  if (!ctas_per_sm) {
-    cudaError_t e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    if (e != cudaSuccess) return e;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    // Resident CTAs per SM: bounded by tensor memory (512 columns per SM, TMEM_COLS per CTA), by
-    // shared memory and by registers (128 per thread at C = 64).  The runtime's occupancy query
-    // does not model tensor-memory allocation, so the bound is taken from the layout itself.
-    int smem_per_sm = 0;
-    cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
-    int by_smem = smem_per_sm / (cfg::SMEM + 1024);  // 1 KiB per CTA is reserved by the system
-    int by_tmem = 512 / cfg::TMEM_COLS;
-    int by_regs = cfg::CTAS_PER_SM;
-    int occ = by_smem < by_tmem ? by_smem : by_tmem;
-    occ = occ < by_regs ? occ : by_regs;
-    ctas_per_sm = occ > 0 ? occ : 1;
+  // Per-device set-up (function attributes are per device) and grid size, done once per device under a lock.
+  static std::mutex mu;
+  static int ctas_per_sm_of[64] = {0}, n_sm_of[64] = {0};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  int ctas_per_sm, n_sm;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ctas_per_sm_of[dev]) {
+      e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
+      if (e != cudaSuccess) return e;
+      e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+      if (e != cudaSuccess) return e;
+      int sms = 0, smem_per_sm = 0;
+      if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+      if ((e = cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev)) != cudaSuccess) return e;
+      // Resident CTAs per SM: bounded by tensor memory (512 columns per SM, TMEM_COLS per CTA), by shared
+      // memory and by registers (the launch bound).  The runtime's occupancy query does not model
+      // tensor-memory allocation, so the bound is taken from the layout itself.
+      int by_smem = smem_per_sm / (cfg::SMEM + 1024);  // 1 KiB per CTA is reserved by the system
+      int by_tmem = 512 / cfg::TMEM_COLS;
+      int occ = by_smem < by_tmem ? by_smem : by_tmem;
+      occ = occ < cfg::CTAS_PER_SM ? occ : cfg::CTAS_PER_SM;
+      n_sm_of[dev] = sms > 0 ? sms : 1;
+      ctas_per_sm_of[dev] = occ > 0 ? occ : 1;
+    }
+    ctas_per_sm = ctas_per_sm_of[dev];
+    n_sm = n_sm_of[dev];
   }
   long long tokens = p.chunk_tab ? (long long)p.T : (long long)p.T * (p.n_chunks / p.chunks_per_seq);
   CUtensorMap tmK, tmV;
