@@ -25,89 +25,11 @@
 
 #include <mutex>
 
-#include "common.cuh"
+#include "tc_device.cuh"
 
 namespace tri_inv {
 namespace {
 
-// ------------------------------------------------------------------------------------------ PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after about two seconds of wall time (the global timer is read every 64 polls,
-// each poll itself blocks for a hardware-defined time slice) or after kSpinLimit polls, whichever comes
-// first, so a lost copy or product cannot hang the GPU.
-constexpr uint32_t kSpinLimit = 1u << 24;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  unsigned long long t0;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
-  for (uint32_t i = 1; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63u) == 0) {
-      unsigned long long t1;
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-      if (t1 - t0 > kWaitLimitNs) return false;
-    }
-  }
-  return false;
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y)
-      : "memory");
-}
-// Pulls a tile into L2 only (no shared memory needed): issued an item ahead so that the real
-// copy, which has to wait for its buffer, finds the data on chip.
-__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* tm, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tm) {
-  asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
-}
-
-__device__ __forceinline__ void mma_tf32(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t to_tf32(float x) {
-  uint32_t r;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-  return r;
-}
-__device__ __forceinline__ float ex2_approx(float x) {  // 2^x, relative error about 2^-22
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
-// Optional per-phase cycle counters (development builds only: -DTRI_INV_PHASE_CLOCKS).
 #ifdef TRI_INV_PHASE_CLOCKS
 __device__ unsigned long long g_cta_times[4096 * 4];
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
@@ -173,239 +95,6 @@ struct Cfg {
 };
 
 // Byte offset of the 16-byte chunk holding features [f, f+8) of row r inside a swizzled tile.
-template <int C>
-__device__ __forceinline__ uint32_t tile_off(int r, int f) {
-  int box = f >> 6, c = (f & 63) >> 3;
-  return (uint32_t)(box * (C * 128) + r * 128 + ((c ^ (r & 7)) << 4));
-}
-
-// 16x16 leaf by the product series (Alg. 5 on the leaf, the first phase of Alg. 2): X <- I - N, Y <- N,
-// three rounds of Y <- Y.Y, X <- X + X.Y as TF32 m16n8k8 MMAs.  X lives in the leaf's place inside the
-// fp32 matrix (row length LDX), Y in a per-warp scratch (row length LDY); both are re-read as operands.
-template <int LDX, int LDY>
-__device__ __forceinline__ void leaf_series(float* xblk, float* ys, int lane) {
-  const int g = lane >> 2, t = lane & 3;
-  float x[2][4], y[2][4];
-#pragma unroll
-  for (int nt = 0; nt < 2; ++nt) {
-    const int c = 8 * nt + 2 * t;
-    const float2 na = *reinterpret_cast<const float2*>(xblk + g * LDX + c);
-    const float2 nb = *reinterpret_cast<const float2*>(xblk + (g + 8) * LDX + c);
-    y[nt][0] = na.x; y[nt][1] = na.y; y[nt][2] = nb.x; y[nt][3] = nb.y;
-    x[nt][0] = (c == g ? 1.f : 0.f) - na.x;
-    x[nt][1] = (c + 1 == g ? 1.f : 0.f) - na.y;
-    x[nt][2] = (c == g + 8 ? 1.f : 0.f) - nb.x;
-    x[nt][3] = (c + 1 == g + 8 ? 1.f : 0.f) - nb.y;
-  }
-  __syncwarp();
-  auto put = [&](float* dst, int ld, const float (&v)[2][4]) {
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-      const int c = 8 * nt + 2 * t;
-      *reinterpret_cast<float2*>(dst + g * ld + c) = make_float2(v[nt][0], v[nt][1]);
-      *reinterpret_cast<float2*>(dst + (g + 8) * ld + c) = make_float2(v[nt][2], v[nt][3]);
-    }
-  };
-  // acc += P . Q for 16x16 matrices in shared memory
-  auto mm = [&](float (&acc)[2][4], const float* pm, int ldp, const float* qm, int ldq) {
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      const float* ap = pm + g * ldp + 8 * q + t;
-      const uint32_t a0 = to_tf32(ap[0]), a1 = to_tf32(ap[8 * ldp]), a2 = to_tf32(ap[4]), a3 = to_tf32(ap[8 * ldp + 4]);
-#pragma unroll
-      for (int nt = 0; nt < 2; ++nt) {
-        const float* bp = qm + (8 * q + t) * ldq + 8 * nt + g;
-        mma_tf32(acc[nt], a0, a1, a2, a3, to_tf32(bp[0]), to_tf32(bp[4 * ldq]));
-      }
-    }
-  };
-  put(ys, LDY, y);
-  put(xblk, LDX, x);
-  __syncwarp();
-#pragma unroll
-  for (int r = 0; r < 3; ++r) {
-    float y2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-    mm(y2, ys, LDY, ys, LDY);   // Y <- Y.Y
-    __syncwarp();               // every lane has read the old Y
-    put(ys, LDY, y2);
-    __syncwarp();
-    mm(x, xblk, LDX, ys, LDY);  // X <- X + X.Y (the accumulator starts as X)
-    __syncwarp();               // every lane has read the old X
-    put(xblk, LDX, x);
-    __syncwarp();
-  }
-  // exact structure of a unit lower triangular block: constants on and above the diagonal
-#pragma unroll
-  for (int nt = 0; nt < 2; ++nt) {
-    const int c = 8 * nt + 2 * t;
-    float2 va = *reinterpret_cast<float2*>(xblk + g * LDX + c), vb = *reinterpret_cast<float2*>(xblk + (g + 8) * LDX + c);
-    va.x = (c < g) ? va.x : (c == g ? 1.f : 0.f);
-    va.y = (c + 1 < g) ? va.y : (c + 1 == g ? 1.f : 0.f);
-    vb.x = (c < g + 8) ? vb.x : (c == g + 8 ? 1.f : 0.f);
-    vb.y = (c + 1 < g + 8) ? vb.y : (c + 1 == g + 8 ? 1.f : 0.f);
-    *reinterpret_cast<float2*>(xblk + g * LDX + c) = va;
-    *reinterpret_cast<float2*>(xblk + (g + 8) * LDX + c) = vb;
-  }
-}
-
-// One merge level of the block recursion: for every adjacent pair of B x B diagonal blocks,
-// X21 = -(X22 . N21) . X11.  Two warps share each 16-row slab of X21 and split its columns.
-template <int C, int B>
-__device__ __forceinline__ void merge_level(float* sX, int warp, int lane) {
-  constexpr int LD = C + 4;
-  constexpr int MT = B / 16;   // 16-row slabs per X21 block
-  constexpr int NTT = B / 8;   // n-tiles (and k-steps) across a block
-  constexpr int NTR = B / 16;  // n-tiles of the result this warp owns
-  const int g = lane >> 2, t = lane & 3;
-  const int mt = warp >> 1, nh = warp & 1;
-  const int pair = mt / MT, ml = mt - pair * MT;
-  const int c0 = pair * 2 * B, r0 = c0 + B, R0 = r0 + 16 * ml;
-
-  float T[NTT][4];
-#pragma unroll
-  for (int i = 0; i < NTT; ++i) { T[i][0] = T[i][1] = T[i][2] = T[i][3] = 0.f; }
-  // T = X22[slab] . N21 ; X22 is lower triangular: slab ml needs k < 16 (ml + 1)
-#pragma unroll
-  for (int q = 0; q < NTT; ++q) {
-    if (q < 2 * (ml + 1)) {
-      const float* ap = sX + (R0 + g) * LD + r0 + 8 * q + t;
-      uint32_t a0 = to_tf32(ap[0]), a1 = to_tf32(ap[8 * LD]), a2 = to_tf32(ap[4]), a3 = to_tf32(ap[8 * LD + 4]);
-      const float* bp = sX + (r0 + 8 * q + t) * LD + c0 + g;
-#pragma unroll
-      for (int nt = 0; nt < NTT; ++nt) {
-        uint32_t b0 = to_tf32(bp[8 * nt]), b1 = to_tf32(bp[4 * LD + 8 * nt]);
-        mma_tf32(T[nt], a0, a1, a2, a3, b0, b1);
-      }
-    }
-  }
-  // R = T . X11[:, my columns].  T's accumulator fragment is reused as the A operand with the
-  // k index permuted (slot t <-> k = 2t, slot t+4 <-> k = 2t+1); B rows are read with the same map.
-  float R[NTR][4];
-#pragma unroll
-  for (int j = 0; j < NTR; ++j) {
-    R[j][0] = R[j][1] = R[j][2] = R[j][3] = 0.f;
-    const int nt = nh * NTR + j;
-#pragma unroll
-    for (int q = 0; q < NTT; ++q) {
-      if (q >= nt) {  // X11 lower triangular: rows k >= column
-        const float* bp = sX + (c0 + 8 * q + 2 * t) * LD + c0 + 8 * nt + g;
-        uint32_t b0 = to_tf32(bp[0]), b1 = to_tf32(bp[LD]);
-        mma_tf32(R[j], to_tf32(T[q][0]), to_tf32(T[q][2]), to_tf32(T[q][1]), to_tf32(T[q][3]), b0, b1);
-      }
-    }
-  }
-  __syncthreads();  // every warp has finished reading N21 before anyone overwrites it
-#pragma unroll
-  for (int j = 0; j < NTR; ++j) {
-    const int col = c0 + 8 * (nh * NTR + j) + 2 * t;
-    *reinterpret_cast<float2*>(sX + (R0 + g) * LD + col) = make_float2(-R[j][0], -R[j][1]);
-    *reinterpret_cast<float2*>(sX + (R0 + g + 8) * LD + col) = make_float2(-R[j][2], -R[j][3]);
-  }
-  __syncthreads();
-}
-
-// ------------------------------------------------------------------------------------------ tcgen05 helpers
-// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets
-// (all >> 4), descriptor version 1 at bit 46, 128-byte swizzle (code 2) at bits 61..63.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr >> 4) & 0x3fffu);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;
-  return d;
-}
-// Instruction descriptor for kind::f16: fp32 accumulate, bf16 x bf16, A K-major,
-// B K-major (b_mn = 0) or MN-major (b_mn = 1), shape M x N.
-__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, int b_mn) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// kind::tf32: fp32 data in shared memory read as TF32, fp32 accumulate, K = 8 per instruction.
-__host__ __device__ constexpr uint32_t umma_idesc_tf32(int M, int N, int b_mn) {
-  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// 16 lanes x 64 columns -> 8 n-tiles of accumulator fragments.
-__device__ __forceinline__ void tmem_ld_16x64(float (&r)[8][4], uint32_t taddr) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=f"(r[0][0]), "=f"(r[0][1]), "=f"(r[0][2]), "=f"(r[0][3]), "=f"(r[1][0]), "=f"(r[1][1]), "=f"(r[1][2]), "=f"(r[1][3]),
-        "=f"(r[2][0]), "=f"(r[2][1]), "=f"(r[2][2]), "=f"(r[2][3]), "=f"(r[3][0]), "=f"(r[3][1]), "=f"(r[3][2]), "=f"(r[3][3]),
-        "=f"(r[4][0]), "=f"(r[4][1]), "=f"(r[4][2]), "=f"(r[4][3]), "=f"(r[5][0]), "=f"(r[5][1]), "=f"(r[5][2]), "=f"(r[5][3]),
-        "=f"(r[6][0]), "=f"(r[6][1]), "=f"(r[6][2]), "=f"(r[6][3]), "=f"(r[7][0]), "=f"(r[7][1]), "=f"(r[7][2]), "=f"(r[7][3])
-      : "r"(taddr));
-}
-// 16 lanes x 128 columns -> 16 n-tiles of accumulator fragments.
-__device__ __forceinline__ void tmem_ld_16x128(float (&r)[16][4], uint32_t taddr) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.16x256b.x16.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,"
-      "%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%64];"
-      : "=f"(r[0][0]), "=f"(r[0][1]), "=f"(r[0][2]), "=f"(r[0][3]), "=f"(r[1][0]), "=f"(r[1][1]), "=f"(r[1][2]), "=f"(r[1][3]),
-        "=f"(r[2][0]), "=f"(r[2][1]), "=f"(r[2][2]), "=f"(r[2][3]), "=f"(r[3][0]), "=f"(r[3][1]), "=f"(r[3][2]), "=f"(r[3][3]),
-        "=f"(r[4][0]), "=f"(r[4][1]), "=f"(r[4][2]), "=f"(r[4][3]), "=f"(r[5][0]), "=f"(r[5][1]), "=f"(r[5][2]), "=f"(r[5][3]),
-        "=f"(r[6][0]), "=f"(r[6][1]), "=f"(r[6][2]), "=f"(r[6][3]), "=f"(r[7][0]), "=f"(r[7][1]), "=f"(r[7][2]), "=f"(r[7][3]),
-        "=f"(r[8][0]), "=f"(r[8][1]), "=f"(r[8][2]), "=f"(r[8][3]), "=f"(r[9][0]), "=f"(r[9][1]), "=f"(r[9][2]), "=f"(r[9][3]),
-        "=f"(r[10][0]), "=f"(r[10][1]), "=f"(r[10][2]), "=f"(r[10][3]), "=f"(r[11][0]), "=f"(r[11][1]), "=f"(r[11][2]), "=f"(r[11][3]),
-        "=f"(r[12][0]), "=f"(r[12][1]), "=f"(r[12][2]), "=f"(r[12][3]), "=f"(r[13][0]), "=f"(r[13][1]), "=f"(r[13][2]), "=f"(r[13][3]),
-        "=f"(r[14][0]), "=f"(r[14][1]), "=f"(r[14][2]), "=f"(r[14][3]), "=f"(r[15][0]), "=f"(r[15][1]), "=f"(r[15][2]), "=f"(r[15][3])
-      : "r"(taddr));
-}
-
-// Epilogue of one 16-row x 64-column piece of W or U: accumulator fragments from tensor memory ->
-// bf16 -> stmatrix into a per-warp, swizzled 2 KiB staging tile -> 16-byte loads -> coalesced
-// 16-byte global stores (8 lanes cover one 128-byte row segment).
-__device__ __forceinline__ void store_frag_piece_bf16(const float (&f)[8][4], uint32_t stage, int lane, __nv_bfloat16* out_row0,
-                                                      size_t row_stride, int rows_left) {
-  const int mi = lane >> 3, r = (lane & 7) + 8 * (mi & 1);
-#pragma unroll
-  for (int nt = 0; nt < 8; nt += 2) {
-    const uint32_t m0 = pack_bf16(f[nt][0], f[nt][1]), m1 = pack_bf16(f[nt][2], f[nt][3]);
-    const uint32_t m2 = pack_bf16(f[nt + 1][0], f[nt + 1][1]), m3 = pack_bf16(f[nt + 1][2], f[nt + 1][3]);
-    const int chunk = nt + (mi >> 1);
-    const uint32_t addr = stage + r * 128 + ((chunk ^ (r & 7)) << 4);
-    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
-  }
-  __syncwarp();
-#pragma unroll
-  for (int m = 0; m < 4; ++m) {
-    const int rr = 4 * m + (lane >> 3), c = lane & 7;
-    uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stage + rr * 128 + ((c ^ (rr & 7)) << 4)));
-    if (rr < rows_left) *reinterpret_cast<uint4*>(out_row0 + rr * row_stride + 8 * c) = v;
-  }
-  __syncwarp();
-}
-__device__ __forceinline__ void store_piece_bf16(uint32_t taddr, uint32_t stage, int lane, __nv_bfloat16* out_row0,
-                                                 size_t row_stride, int rows_left) {
-  float f[8][4];
-  tmem_ld_16x64(f, taddr);
-  tmem_wait_ld();
-  store_frag_piece_bf16(f, stage, lane, out_row0, row_stride, rows_left);
-}
-
 template <int C, int D, bool SER, bool RAW, bool BO>
 __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                              const __grid_constant__ CUtensorMap tmV, KParams p) {
@@ -864,28 +553,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
       if (p.method & TRI_INV_LEAF_SERIES) {
         leaf_series<LD, cfg::LEAF_LD>(sX + 16 * rb * LD + 16 * rb,
                                       reinterpret_cast<float*>(smem + cfg::OFF_LEAF) + warp * 16 * cfg::LEAF_LD, lane);
-      } else {  // forward substitution, lane j owns column j
-        const int base = 16 * rb, j = lane & 15;
-        const float* nb = sX + base * LD + base;
-        float x[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float s = 0.f;
-#pragma unroll
-          for (int k4 = 0; k4 < (i + 3) / 4; ++k4) {
-            float4 nv = *reinterpret_cast<const float4*>(nb + i * LD + 4 * k4);
-            if (4 * k4 + 0 < i) s = fmaf(nv.x, x[4 * k4 + 0], s);
-            if (4 * k4 + 1 < i) s = fmaf(nv.y, x[4 * k4 + 1], s);
-            if (4 * k4 + 2 < i) s = fmaf(nv.z, x[4 * k4 + 2], s);
-            if (4 * k4 + 3 < i) s = fmaf(nv.w, x[4 * k4 + 3], s);
-          }
-          x[i] = (i < j) ? 0.f : (i == j ? 1.f : -s);
-        }
-        __syncwarp();
-        if (lane < 16) {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) sX[(base + i) * LD + base + j] = x[i];
-        }
+      } else {
+        leaf_substitution<LD>(sX + 16 * rb * LD + 16 * rb, lane);
       }
       __syncthreads();
       if (BO && tid == kTidK && has_next) issue_k(nx_tok0, nx_h);  // the leaf scratch inside the K tile is no longer needed
