@@ -110,6 +110,38 @@ def raw_front_end(K_raw, beta_logit, gate_logit, C, cu_seqlens=None):
     return K_hat, beta, g.reshape(B, T, H)
 
 
+def build_A_kda(K, G, beta, C, cu_seqlens=None, return_N=False):
+    """Per-channel decay (the KDA row of Table 1): phi = (K * Gamma)(K / Gamma)^T with Gamma = exp(G),
+    G [B,T,H,d] the cumulative per-channel log-decay inside each chunk, and beta scaling rows:
+        N_ij = beta_i * sum_c K_ic K_jc exp(G_ic - G_jc)   (i > j),      A = (I + N)^{-1}.
+    The exponent is taken of the difference, so no factor can overflow when G decreases along a chunk.
+    fp64 numpy; the inverse by LAPACK's triangular solve (forward substitution)."""
+    from scipy.linalg import solve_triangular
+    Kd, Gd = _widen(np.asarray(K)), np.asarray(G, dtype=np.float64)
+    bd = np.asarray(beta, dtype=np.float64)
+    B, T, H, d = Kd.shape
+    Kf, Gf, bf = Kd.reshape(B * T, H, d), Gd.reshape(B * T, H, d), bd.reshape(B * T, H)
+    A = np.zeros((B * T, H, C))
+    N = np.zeros((B * T, H, C)) if return_N else None
+    bounds = [(b * T, (b + 1) * T) for b in range(B)] if cu_seqlens is None else \
+             [(int(cu_seqlens[i]), int(cu_seqlens[i + 1])) for i in range(len(cu_seqlens) - 1)]
+    for beg, end in bounds:
+        for t0 in range(beg, end, C):
+            r = min(C, end - t0)
+            for h in range(H):
+                k, g, b = Kf[t0:t0 + r, h], Gf[t0:t0 + r, h], bf[t0:t0 + r, h]
+                n = np.zeros((r, r))
+                for i in range(r):
+                    for j in range(i):
+                        n[i, j] = b[i] * np.sum(k[i] * k[j] * np.exp(g[i] - g[j]))
+                a = solve_triangular(np.eye(r) + n, np.eye(r), lower=True, unit_diagonal=True)
+                A[t0:t0 + r, h, :r] = np.tril(a)
+                if return_N:
+                    N[t0:t0 + r, h, :r] = n
+    A = A.reshape(B, T, H, C)
+    return (A, N.reshape(B, T, H, C)) if return_N else A
+
+
 def threads(n_threads: int = 0) -> int:
     return int(_load().tri_inv_oracle_threads(int(n_threads)))
 

@@ -360,3 +360,32 @@ def test_raw_front_end_hand_values_and_generator_recipe():
     for t in (0, 64, 70, 134):
         assert np.allclose(g[0, t], ls[0, t], atol=1e-15)
     assert np.allclose(g[0, 69], ls[0, 64:70].sum(axis=0), atol=1e-13)
+
+
+# ---------------------------------------------------------------- per-channel decay (KDA row of Table 1)
+
+def test_per_channel_decay_reduces_to_the_scalar_gate_and_to_deltanet():
+    x = wl.make("kda", 2, 150, 2, 16, 16, 64, wl.BF16, seed=33)
+    # Gamma = 1: plain DeltaNet matrix (g = 0)
+    A0 = oracle.build_A_kda(x.K, np.zeros((2, 150, 2, 16)), x.beta, 64)
+    assert np.abs(A0 - oracle.build_A(x.K, x.beta, np.zeros_like(x.g), 64)).max() < 1e-13
+    # the same log-decay on every channel: the GDN scalar gate exp(g_i - g_j)
+    G = np.repeat(x.g[..., None].astype(np.float64), 16, axis=-1)
+    A1, N1 = oracle.build_A_kda(x.K, G, x.beta, 64, return_N=True)
+    A_ref, N_ref = oracle.build_A(x.K, x.beta, x.g, 64, return_N=True)
+    assert np.abs(N1 - N_ref).max() < 1e-14 and np.abs(A1 - A_ref).max() < 1e-13
+    # a hand value: k_0 = (1, 2), k_1 = (3, 1), G_0 = (0, 0), G_1 = (-ln 2, -ln 4), beta_1 = 2:
+    # N_10 = 2 * (3 * 1 / 2 + 1 * 2 / 4) = 4
+    K = np.array([[1.0, 2.0], [3.0, 1.0]], np.float32).reshape(1, 2, 1, 2)
+    Gh = np.array([[0.0, 0.0], [-np.log(2.0), -np.log(4.0)]]).reshape(1, 2, 1, 2)
+    A, N = oracle.build_A_kda(K, Gh, np.array([1.0, 2.0]).reshape(1, 2, 1), 2, return_N=True)
+    assert abs(N[0, 1, 0, 0] - 4.0) < 1e-14 and abs(A[0, 1, 0, 0] + 4.0) < 1e-14
+    # defining identities with a genuinely per-channel gate, ragged chunks included
+    Gp = wl.per_channel_gate(x, seed=5)
+    A2, N2 = oracle.build_A_kda(x.K, Gp, x.beta, 64, return_N=True)
+    for b in range(2):
+        for t0, r in ((0, 64), (64, 64), (128, 22)):
+            n, a = N2[b, t0:t0 + r, 1, :r], A2[b, t0:t0 + r, 1, :r]
+            assert np.abs((np.eye(r) + n) @ a - np.eye(r)).max() < 1e-12
+            assert np.array_equal(np.diag(a), np.ones(r)) and not a[np.triu_indices(r, 1)].any()
+    assert np.abs(A2 - A_ref).max() > 1e-3      # and it is a different matrix from the scalar-gate one
