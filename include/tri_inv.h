@@ -138,6 +138,18 @@ int tri_inv_fused(const void* K, const void* V, const float* beta, const float* 
                   const tri_inv_desc* desc, int method, void* cuda_stream);
 
 /*
+ * Per-channel decay (the KDA row of Table 1: phi = (K * Gamma)(K / Gamma)^T, Gamma = exp(G)):
+ *     N_ij = beta_i * sum_c K_ic K_jc exp(G_ic - G_jc)   (i > j),      A = (I + N)^{-1}
+ * G [B,T,H,d_k] fp32 is the cumulative per-channel log-decay inside each chunk (only differences inside a
+ * chunk are used).  Same layouts, chunking modes, methods and error codes as tri_inv_build.  On the tensor
+ * cores (bf16 keys, d_k = 128, C = 64, block recursion) the two factors are formed around the chunk's middle
+ * row, so |G_i - G_mid| log2(e) must stay inside the fp32 exponent range (about 88 in natural-log units);
+ * other shapes take the exponent of each difference directly.
+ */
+int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A,
+                      const tri_inv_desc* desc, int method, void* cuda_stream);
+
+/*
  * Fused call with the layer's front end folded in: the kernel takes what the projections produce and
  * does the three producers that otherwise run as separate passes over memory before the inversion
  * (the gating recipe of a Gated-DeltaNet layer; in the paper these are among the kernels its fused

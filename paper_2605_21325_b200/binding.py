@@ -34,7 +34,7 @@ def ns_iters(m: int) -> int:
 
 FORCE_SIMT = 0x10000
 
-EXPORTS = ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
+EXPORTS = ("tri_inv_build", "tri_inv_build_kda", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
            "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
 
 
@@ -66,6 +66,8 @@ def load():
         lib.tri_inv_build.argtypes = [vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_wy.argtypes = [vp, vp, vp, vp, vp, vp, dp, vp]
         lib.tri_inv_fused.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
+        lib.tri_inv_build_kda.argtypes = [vp, vp, vp, vp, dp, i32, vp]
+        lib.tri_inv_build_kda.restype = i32
         lib.tri_inv_fused_raw.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_fused_raw.restype = i32
         lib.tri_inv_fused_packed_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
@@ -144,6 +146,17 @@ def build(K, beta, g, C, method=BLOCK_RECURSIVE, cu_seqlens=None, out=None, stre
     rc = load().tri_inv_build(_p(K), _p(beta), _p(g), _p(A), ctypes.byref(desc), int(method), _stream(stream))
     if rc != OK:
         raise TriInvError("tri_inv_build", rc)
+    return A
+
+
+def build_kda(K, G, beta, C, method=BLOCK_RECURSIVE, cu_seqlens=None, out=None, stream=None):
+    """Per-channel decay: A = (I+N)^{-1} with N_ij = beta_i sum_c K_ic K_jc exp(G_ic - G_jc); G [B,T,H,d] fp32."""
+    B, T, H, d_k = K.shape
+    desc, keep = make_desc(B, T, H, d_k, d_k, C, _dtype_code(K), cu_seqlens)
+    A = torch.zeros((B, T, H, C), dtype=torch.float32, device=K.device) if out is None else out
+    rc = load().tri_inv_build_kda(_p(K), _p(G), _p(beta), _p(A), ctypes.byref(desc), int(method), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_build_kda", rc)
     return A
 
 

@@ -129,7 +129,7 @@ int run(KParams p, const tri_inv_desc* d, void* stream_v) {
   err = cudaSuccess;
   // Newton-Schulz and the refinement step exist on the fp32 CUDA-core kernel only
   const bool simt_only = (p.method & (TRI_INV_FORCE_SIMT | TRI_INV_REFINE)) || (p.method & TRI_INV_METHOD_MASK) == TRI_INV_NEWTON_SCHULZ;
-  if (!simt_only) err = launch_tc(p, d->C, stream, &handled);
+  if (!simt_only) err = (p.ops & kKda) ? launch_kda_tc(p, d->C, stream, &handled) : launch_tc(p, d->C, stream, &handled);
   if (err == cudaSuccess && !handled) err = launch_simt(p, d->C, stream);
   if (err == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);
   if (dev_tab) cudaFreeAsync(dev_tab, stream);
@@ -204,6 +204,20 @@ int tri_inv_fused_raw(const void* K_raw, const void* V, const float* beta_logit,
   p.beta_out = beta_out; p.g_out = g_out;
   p.method = method;
   p.ops = kDoWY | kRaw | (A ? kStoreA : 0);
+  return run(p, desc, cuda_stream);
+}
+
+int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A,
+                       const tri_inv_desc* desc, int method, void* cuda_stream) {
+  int rc = check_desc(desc, false);
+  if (rc) return rc;
+  if (!K || !G || !beta || !A) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(G) || !aligned16(beta) || !aligned16(A)) return TRI_INV_ERR_INVALID_ARG;
+  if ((rc = check_method(method))) return rc;
+  KParams p{};
+  p.K = K; p.V = G; p.beta = beta; p.g = nullptr; p.A = A;
+  p.method = method;
+  p.ops = kStoreA | kKda;
   return run(p, desc, cuda_stream);
 }
 

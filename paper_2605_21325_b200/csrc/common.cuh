@@ -13,6 +13,7 @@ enum : int {
   kStoreA = 1,  // write A to global memory
   kDoWY = 2,    // compute W (and U when V != nullptr)
   kLoadA = 4,   // skip build + inversion, read A from A_in (tri_inv_wy)
+  kKda = 16,    // per-channel decay: KParams::V holds G [B,T,H,d_k] fp32 (build only)
   kRaw = 8,     // K is un-normalised, beta and g are logits: normalise, sigmoid, log-sigmoid + chunk cumsum in the kernel
 };
 
@@ -72,6 +73,8 @@ __device__ __forceinline__ float load_kv(const void* base, int dtype, size_t idx
 cudaError_t launch_simt(const KParams& p, int C, cudaStream_t stream);
 // Tensor-core path: returns cudaErrorNotSupported when it has no kernel for the request.
 cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
+// Per-channel decay variant on the tensor cores (bf16 keys, d_k = 128, C = 64, block recursion).
+cudaError_t launch_kda_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
 
 // Fills dev_tab (one entry per chunk of tokens, in sequence order) from the host offsets in d->cu_seqlens
 // with small kernels on the stream; no copy and no synchronisation.

@@ -108,6 +108,7 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
   float* sg = sb + C;
   float* sr = sg + C;  // raw front end: 1 / |k_i|
   const bool raw = (p.ops & kRaw) != 0;
+  const bool kda = (p.ops & kKda) != 0;  // per-channel decay: G in p.V, each Gram term weighted by exp(G_ic - G_jc)
   const int tid = threadIdx.x;
   const int total = p.n_chunks * p.H;
   constexpr int kAcc = (C * C + kThreads - 1) / kThreads;
@@ -162,6 +163,11 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
           float v = 0.f;
           if (i < rows && ks + kk < p.d_k) v = load_kv(p.K, p.kv_dtype, ((size_t)(tok0 + i) * p.H + h) * p.d_k + ks + kk);
           Ks[i * kSliceLd + kk] = v;
+          if (kda) {  // the scratch matrix is free during the Gram phase: it holds the slice of G
+            float gv = 0.f;
+            if (i < rows && ks + kk < p.d_k) gv = ((const float*)p.V)[((size_t)(tok0 + i) * p.H + h) * p.d_k + ks + kk];
+            Zm[i * kSliceLd + kk] = gv;
+          }
         }
         __syncthreads();
 #pragma unroll
@@ -170,11 +176,20 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
           int i = e / C, j = e - i * C;
           if (e < C * C && (j < i || (raw && j == i))) {
             float s = acc[m];
+            if (kda) {
+              for (int kk = 0; kk < kSlice; ++kk)
+                s = fmaf(Ks[i * kSliceLd + kk] * Ks[j * kSliceLd + kk], expf(Zm[i * kSliceLd + kk] - Zm[j * kSliceLd + kk]), s);
+            } else {
 #pragma unroll
-            for (int kk = 0; kk < kSlice; ++kk) s = fmaf(Ks[i * kSliceLd + kk], Ks[j * kSliceLd + kk], s);
+              for (int kk = 0; kk < kSlice; ++kk) s = fmaf(Ks[i * kSliceLd + kk], Ks[j * kSliceLd + kk], s);
+            }
             acc[m] = s;
           }
         }
+      }
+      if (kda) {
+        __syncthreads();
+        for (int e = tid; e < C * LD; e += kThreads) Zm[e] = 0.f;
       }
       if (raw) {  // 1 / |k_i| from the Gram diagonal; the Gram of the normalised keys is S_ij r_i r_j
 #pragma unroll

@@ -5,6 +5,8 @@
 #pragma once
 #include <cuda.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace tri_inv {
@@ -346,6 +348,40 @@ __device__ __forceinline__ void store_piece_bf16(uint32_t taddr, uint32_t stage,
   tmem_wait_ld();
   store_frag_piece_bf16(f, stage, lane, out_row0, row_stride, rows_left);
 }
+
+// ------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)ptr;
+  });
+  return fn;
+}
+
+// 2-D view of a [tokens, H*d] tensor of bf16 (elt = 2) or fp32 (elt = 4); one box = 128 bytes of features
+// (64 bf16 or 32 fp32, swizzled) x C tokens.
+inline bool make_tmap(CUtensorMap* tm, const void* base, long long tokens, int H, int d, int C, int elt = 2) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)H * d, (cuuint64_t)tokens};
+  cuuint64_t strides[1] = {(cuuint64_t)H * d * elt};
+  cuuint32_t box[2] = {(cuuint32_t)(128 / elt), (cuuint32_t)C};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, elt == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 
 }  // namespace
 }  // namespace tri_inv

@@ -417,3 +417,33 @@ def test_concurrent_launches_on_two_streams(bnd):
         assert all(torch.equal(a, b) for a, b in zip(o, ref1))
     for o in outs2:
         assert all(torch.equal(a, b) for a, b in zip(o, ref2))
+
+
+# ---------------------------------------------------------------- per-channel decay (KDA row of Table 1)
+
+@pytest.mark.parametrize("C,dtype,d", [(64, wl.BF16, 128), (64, wl.F32, 64), (32, wl.BF16, 64), (128, wl.BF16, 128)])
+def test_build_kda(bnd, C, dtype, d):
+    cu = np.array([0, 2 * C + 9, 3 * C + 9, 3 * C + 10], np.int32)
+    for cu_seqlens, B, T in ((None, 2, 3 * C), (cu, 1, int(cu[-1]))):
+        inp = wl.make("kda", B, T, 3, d, d, C, dtype, seed=90 + C, cu_seqlens=cu_seqlens)
+        G = wl.per_channel_gate(inp, seed=91)
+        A_ref, N_ref = oracle.build_A_kda(inp.K, G, inp.beta, C, cu_seqlens=cu_seqlens, return_N=True)
+        dev = bnd.to_device(inp)
+        Gd = torch.from_numpy(G).cuda()
+        for m in (bnd.BLOCK_RECURSIVE, bnd.BLOCK_RECURSIVE | bnd.LEAF_SERIES, bnd.PRODUCT_SERIES):
+            A = nan_like((B, T, 3, C), torch.float32)
+            bnd.build_kda(dev["K"], Gd, dev["beta"], C, method=m, cu_seqlens=cu_seqlens, out=A)
+            torch.cuda.synchronize()
+            assert bnd.last_device_status() == 0
+            # bf16 operands K * exp(+-(G - G_mid)) carry 2^-9 relative rounding each: same bound as the bf16 configs
+            check_A(A, inp, A_ref, N_ref)
+
+
+def test_build_kda_with_a_channel_constant_gate_equals_build(bnd):
+    inp = wl.config(2, shrink=16)
+    dev = bnd.to_device(inp)
+    G = torch.from_numpy(np.repeat(inp.g[..., None], 128, axis=-1).copy()).cuda()
+    A1 = bnd.build_kda(dev["K"], G, dev["beta"], 64)
+    A2 = bnd.build(dev["K"], dev["beta"], dev["g"], 64)
+    torch.cuda.synchronize()
+    assert (A1 - A2).abs().max().item() <= 2e-3
