@@ -44,6 +44,8 @@ def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True, call="fused"):
     build: K, beta, g read; A written.  wy: the strict lower triangle of A, K, V, beta read; W, U written."""
     if call == "build":
         return C * d_k * elt + 2 * C * 4 + C * C * 4
+    if call == "kda":  # K, G (fp32 per channel) and beta read; A written
+        return C * d_k * elt + C * d_k * 4 + C * 4 + C * C * 4
     if call == "wy":
         return C * (C - 1) // 2 * 4 + C * d_k * elt + C * d_v * elt + C * 4 + C * d_k * elt + C * d_v * elt
     b = C * d_k * elt + C * d_v * elt + 2 * C * 4 + C * d_k * elt + C * d_v * elt
@@ -192,7 +194,7 @@ def main():
     ap.add_argument("--method", default="block_recursive", choices=["block_recursive", "mixed_recursion", "product_series"])
     ap.add_argument("--paper-T", type=int, default=0,
                     help="instead of --config: the paper's timing shape B=32, H=4, d=128 at this sequence length (1024..16384)")
-    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw"],
+    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw", "kda"],
                     help="entry point timed: the fused path (default, the metric), tri_inv_build alone, tri_inv_wy alone, or "
                          "tri_inv_fused_raw (front end folded in; same shapes, un-normalised keys and logits as inputs)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -242,6 +244,7 @@ def main():
     K, V, beta, g = dev["K"], dev["V"], dev["beta"], dev["g"]
     A = torch.empty((inp.B, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda")
     W, U = torch.empty_like(K), torch.empty_like(V)
+    G = torch.from_numpy(wl.per_channel_gate(inp, seed=3000 + args.config)).cuda() if args.call == "kda" else None
     flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     flush_rd = None if args.no_flush else torch.zeros(64 * 1024 * 1024, dtype=torch.float32, device="cuda")
     stream = torch.cuda.current_stream()
@@ -260,6 +263,8 @@ def main():
             binding.fused_raw(K, V, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U, None, None), stream=stream)
         elif args.call == "build":
             binding.build(K, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
+        elif args.call == "kda":
+            binding.build_kda(K, G, beta, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
         else:
             binding.wy(A, K, V, beta, cu_seqlens=inp.cu_seqlens, out=(W, U), stream=stream)
 
@@ -361,7 +366,12 @@ def main():
         err = {"sample": "first %d tokens of every sequence" % Ts if Ts else "all tokens"}
         if args.call != "wy":
             err["A_max_ratio"] = float(np.abs(a - A_ref).max() / np.abs(A_ref).max())
-        if args.call != "build":
+        if args.call == "kda":
+            Gs = G.cpu().numpy()
+            A_k = oracle.build_A_kda(inp.K[:, :Ts] if Ts else inp.K, Gs[:, :Ts] if Ts else Gs, inp.beta[:, :Ts] if Ts else inp.beta,
+                                     inp.C, cu_seqlens=None if Ts else inp.cu_seqlens)
+            err["A_max_ratio"] = float(np.abs(a - A_k).max() / np.abs(A_k).max())
+        if args.call not in ("build", "kda"):
             err["W_max_ratio"] = float(np.abs(w - W_ref).max() / np.abs(W_ref).max())
             err["U_max_ratio"] = float(np.abs(u - U_ref).max() / np.abs(U_ref).max())
 
@@ -374,7 +384,7 @@ def main():
         traffic = NCU_TRAFFIC_BYTES_PER_MATRIX.get((args.config, args.method)) if args.call == "fused" else None
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": None if traffic is None else traffic * n_mat, "peak_source": "of " + peak_kind,
-                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "wy": "WY apply"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
+                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "kda": "per-channel-decay build+invert", "wy": "WY apply"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
                     "algorithmic_bytes_per_launch": alg_bytes * n_mat}
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
@@ -384,7 +394,7 @@ def main():
                "dtype": "bf16" if inp.kv_dtype == wl.BF16 else "f32", "data": "synthetic",
                "config": {"workload": inp.name, "B": inp.B, "T": inp.T, "H": inp.H, "d_k": inp.d_k, "d_v": inp.d_v, "C": inp.C,
                           "chunk_matrices_per_gpu": n_mat, "method": args.method, "call": args.call,
-                          "outputs": {"fused": "A fp32 + W,U", "raw": "A fp32 + W,U", "build": "A fp32", "wy": "W,U"}[args.call],
+                          "outputs": {"fused": "A fp32 + W,U", "raw": "A fp32 + W,U", "build": "A fp32", "kda": "A fp32", "wy": "W,U"}[args.call],
                           "l2": "flushed before every timed step (256 MiB write, then a 256 MiB read so no dirty lines remain)" if flush is not None else "not flushed",
                           "parallelism": "independent replicas, no collective" if world > 1 else "single GPU"},
                "gb_per_s": achieved, "roofline": roofline, "cpu_baseline": cpu,
