@@ -389,3 +389,7 @@ def test_per_channel_decay_reduces_to_the_scalar_gate_and_to_deltanet():
             assert np.abs((np.eye(r) + n) @ a - np.eye(r)).max() < 1e-12
             assert np.array_equal(np.diag(a), np.ones(r)) and not a[np.triu_indices(r, 1)].any()
     assert np.abs(A2 - A_ref).max() > 1e-3      # and it is a different matrix from the scalar-gate one
+    # only differences inside a chunk enter: a per-(chunk, head, channel) offset of G changes nothing
+    off = np.random.default_rng(6).standard_normal((2, 3, 2, 16)).repeat(64, axis=1)[:, :150]
+    N3 = oracle.build_A_kda(x.K, Gp + off, x.beta, 64, return_N=True)[1]
+    assert np.abs(N3 - N2).max() < 1e-12
