@@ -11,6 +11,11 @@ the CUDA library and the CUDA library never calls it.
 
 * ``build_A`` / ``wy``      -- the C implementation (``tri_inv_oracle.c``), plain
   triple loops in double, OpenMP over independent chunks.
+* ``gdn_recurrence``        -- the layer as its token-by-token recurrence (C, double); ``chunk_scan`` -- the
+  chunk form that consumes W and U (numpy).  Pins: a hand-worked scalar example, exact read-back of a write,
+  orthonormal keys reducing to causal linear attention (Sec. 1), the no-write closed form, and the two
+  agreeing with each other through ``build_A`` / ``wy``.
+* ``build_A_kda``           -- per-channel decay (KDA row of Table 1), numpy + LAPACK.
 * ``oracle.algorithms``     -- numpy fp64 restatements of the paper's inversion
   algorithms (Algs. 2, 4, 5 and the 2x2 block formula), step by step.
 
@@ -53,6 +58,9 @@ def _load():
         lib.tri_inv_oracle_build.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, i32]
         lib.tri_inv_oracle_wy.restype = i32
         lib.tri_inv_oracle_wy.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, i32, i32]
+        lib.tri_inv_oracle_gdn_recurrence.restype = i32
+        lib.tri_inv_oracle_gdn_recurrence.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, ctypes.c_double,
+                                                      i32, i32, i32, i32, i32, i32, vp, i32, i32]
         lib.tri_inv_oracle_threads.restype = i32
         lib.tri_inv_oracle_threads.argtypes = [i32]
         _lib = lib
@@ -140,6 +148,62 @@ def build_A_kda(K, G, beta, C, cu_seqlens=None, return_N=False):
                     N[t0:t0 + r, h, :r] = n
     A = A.reshape(B, T, H, C)
     return (A, N.reshape(B, T, H, C)) if return_N else A
+
+
+def gdn_recurrence(Q, K, V, beta, g, C, scale=1.0, S0=None, cu_seqlens=None, n_threads=0):
+    """The gated delta-rule layer token by token (decay, delta-rule write, read) in fp64: the definition
+    that the chunkwise path re-formulates.  Returns (O [B,T,H,d_v], S_final [n_sequences,H,d_k,d_v])."""
+    Q, dq = _kv(Q)
+    K, dk = _kv(K)
+    V, dv = _kv(V)
+    if not (dq == dk == dv):
+        Q, K, V, dk = _widen(Q), _widen(K), _widen(V), F64
+    B, T, H, d_k = K.shape
+    d_v = V.shape[3]
+    beta = np.ascontiguousarray(beta, dtype=np.float32)
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    cu = None if cu_seqlens is None else np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    n_seqs = B if cu is None else len(cu) - 1
+    S0 = None if S0 is None else np.ascontiguousarray(S0, dtype=np.float64)
+    assert S0 is None or S0.shape == (n_seqs, H, d_k, d_v)
+    O = np.zeros((B, T, H, d_v))
+    S = np.zeros((n_seqs, H, d_k, d_v))
+    rc = _load().tri_inv_oracle_gdn_recurrence(_ptr(Q), _ptr(K), _ptr(V), dk, _ptr(beta), _ptr(g), _ptr(S0),
+                                               _ptr(O), _ptr(S), float(scale), B, T, H, d_k, d_v, C,
+                                               _ptr(cu), 0 if cu is None else n_seqs, int(n_threads))
+    if rc != 0:
+        raise ValueError("tri_inv_oracle_gdn_recurrence: invalid arguments")
+    return O, S
+
+
+def chunk_scan(Q, K, W, U, g, C, scale=1.0, S0=None, cu_seqlens=None):
+    """What the chunk-scan entry point computes from its inputs, in fp64, chunk by chunk in order.  With
+    gamma_i = exp(g_i), D_ij = gamma_i / gamma_j (j <= i, else 0) and the state S entering the chunk:
+        U~ = U - W S,   O = scale * (diag(gamma) Q S + ((Q K^T) * D) U~),
+        S <- gamma_last S + (diag(gamma_last / gamma) K)^T U~.
+    W is the decay-weighted factor A diag(beta * gamma) K, U = A diag(beta) V; with those two exact this is the
+    token-by-token recurrence re-bracketed (the identity the pins check).  Returns (O, S_final)."""
+    Qd, Kd, Wd, Ud = _widen(np.asarray(Q)), _widen(np.asarray(K)), _widen(np.asarray(W)), _widen(np.asarray(U))
+    gd = np.asarray(g, dtype=np.float64)
+    B, T, H, d_k = Kd.shape
+    d_v = Ud.shape[3]
+    bounds = [(b * T, (b + 1) * T) for b in range(B)] if cu_seqlens is None else \
+             [(int(cu_seqlens[i]), int(cu_seqlens[i + 1])) for i in range(len(cu_seqlens) - 1)]
+    Qf, Kf, Wf, Uf, gf = (x.reshape((B * T,) + x.shape[2:]) for x in (Qd, Kd, Wd, Ud, gd))
+    O = np.zeros((B * T, H, d_v))
+    S_all = np.zeros((len(bounds), H, d_k, d_v))
+    for s, (beg, end) in enumerate(bounds):
+        for h in range(H):
+            S = np.zeros((d_k, d_v)) if S0 is None else np.array(S0[s, h], dtype=np.float64)
+            for t0 in range(beg, end, C):
+                t1 = min(t0 + C, end)
+                q, k, w, u, gg = Qf[t0:t1, h], Kf[t0:t1, h], Wf[t0:t1, h], Uf[t0:t1, h], gf[t0:t1, h]
+                D = np.tril(np.exp(gg[:, None] - gg[None, :]))
+                ut = u - w @ S
+                O[t0:t1, h] = scale * (np.exp(gg)[:, None] * (q @ S) + ((q @ k.T) * D) @ ut)
+                S = np.exp(gg[-1]) * S + (np.exp(gg[-1] - gg)[:, None] * k).T @ ut
+            S_all[s, h] = S
+    return O.reshape(B, T, H, d_v), S_all
 
 
 def threads(n_threads: int = 0) -> int:

@@ -202,3 +202,69 @@ int tri_inv_oracle_threads(int n_threads) {
   return 1;
 #endif
 }
+
+/*
+ * The gated delta-rule layer as its token-by-token linear recurrence (Sec. 1's recurrent form with the
+ * delta-rule update and the decay gate of the GDN row of Table 1; the chunkwise path with (I+N)^{-1},
+ * W and U is a re-formulation of exactly this).  Per sequence and head, with the state S [d_k][d_v]
+ * starting at S0 (zero when NULL), for every token t in order:
+ *
+ *     a_t   = g_t - g_{t-1}  (g_{t-1} = 0 at the first row of a chunk: g is the within-chunk cumulative sum)
+ *     S    <- exp(a_t) * S                                   decay
+ *     S    <- S + beta_t * k_t (v_t - S^T k_t)^T             delta-rule write
+ *     o_t   = scale * S^T q_t                                read
+ *
+ * Q, K [B,T,H,d_k], V [B,T,H,d_v] in one storage type; beta, g [B,T,H] fp32; S0, S_out
+ * [n_sequences,H,d_k,d_v] double (both nullable); O [B,T,H,d_v] double.  HOST pointers.
+ * OpenMP over (sequence, head); every sum in double in index order.
+ */
+int tri_inv_oracle_gdn_recurrence(const void* Q, const void* K, const void* V, int kv_dtype,
+                                  const float* beta, const float* g, const double* S0,
+                                  double* O, double* S_out, double scale,
+                                  int B, int T, int H, int d_k, int d_v, int C,
+                                  const int32_t* cu_seqlens, int n_seqs, int n_threads) {
+  if (!Q || !K || !V || !beta || !g || !O || B < 1 || T < 0 || H < 1 || d_k < 1 || d_v < 1 || C < 1) return 1;
+  if (cu_seqlens && (B != 1 || n_seqs < 0 || cu_seqlens[0] != 0 || cu_seqlens[n_seqs] != T)) return 1;
+  int nseq = cu_seqlens ? n_seqs : B;
+#ifdef _OPENMP
+  if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+  int64_t total = (int64_t)nseq * H;
+#pragma omp parallel
+  {
+    double* S = (double*)malloc(sizeof(double) * (size_t)d_k * d_v);
+    double* r = (double*)malloc(sizeof(double) * (size_t)d_v);
+#pragma omp for schedule(dynamic, 1)
+    for (int64_t w = 0; w < total; ++w) {
+      int s = (int)(w / H), h = (int)(w % H);
+      int64_t beg = cu_seqlens ? cu_seqlens[s] : (int64_t)s * T;
+      int64_t end = cu_seqlens ? cu_seqlens[s + 1] : (int64_t)(s + 1) * T;
+      for (int i = 0; i < d_k * d_v; ++i) S[i] = S0 ? S0[((size_t)s * H + h) * d_k * d_v + i] : 0.0;
+      for (int64_t t = beg; t < end; ++t) {
+        size_t th = (size_t)t * H + h;
+        int first_of_chunk = ((t - beg) % C) == 0;
+        double a = (double)g[th] - (first_of_chunk ? 0.0 : (double)g[th - H]);
+        double alpha = exp(a), b = (double)beta[th];
+        for (int i = 0; i < d_k * d_v; ++i) S[i] *= alpha;
+        for (int j = 0; j < d_v; ++j) {
+          double acc = 0.0;
+          for (int i = 0; i < d_k; ++i) acc += widen(K, kv_dtype, th * d_k + i) * S[i * d_v + j];
+          r[j] = widen(V, kv_dtype, th * d_v + j) - acc;
+        }
+        for (int i = 0; i < d_k; ++i) {
+          double ki = b * widen(K, kv_dtype, th * d_k + i);
+          for (int j = 0; j < d_v; ++j) S[i * d_v + j] += ki * r[j];
+        }
+        for (int j = 0; j < d_v; ++j) {
+          double acc = 0.0;
+          for (int i = 0; i < d_k; ++i) acc += widen(Q, kv_dtype, th * d_k + i) * S[i * d_v + j];
+          O[th * d_v + j] = scale * acc;
+        }
+      }
+      if (S_out) for (int i = 0; i < d_k * d_v; ++i) S_out[((size_t)s * H + h) * d_k * d_v + i] = S[i];
+    }
+    free(S);
+    free(r);
+  }
+  return 0;
+}

@@ -153,6 +153,22 @@ def per_channel_gate(inp: Inputs, seed: int) -> np.ndarray:
     return np.ascontiguousarray(G.reshape(inp.B, inp.T, inp.H, inp.d_k))
 
 
+def queries(inp: Inputs, seed: int):
+    """Queries for the layer's read step: Q ~ N(0,1) rows L2-normalised (as the keys are), in the storage
+    type of K.  [B,T,H,d_k]."""
+    rng = np.random.default_rng(seed)
+    Q = rng.standard_normal((inp.B, inp.T, inp.H, inp.d_k), dtype=np.float32)
+    Q /= np.sqrt((Q ** 2).sum(axis=-1, keepdims=True, dtype=np.float32))
+    return _store(Q, inp.kv_dtype)
+
+
+def initial_state(inp: Inputs, seed: int) -> np.ndarray:
+    """A carried-in recurrent state S0 [n_sequences,H,d_k,d_v] fp32 ~ N(0,1)/sqrt(d_k) (decode-after-prefill case)."""
+    rng = np.random.default_rng(seed)
+    n = inp.B if inp.cu_seqlens is None else len(inp.cu_seqlens) - 1
+    return (rng.standard_normal((n, inp.H, inp.d_k, inp.d_v), dtype=np.float32) / np.float32(np.sqrt(inp.d_k)))
+
+
 def ragged_lengths(n_seqs: int, max_len: int, rng) -> np.ndarray:
     lens = rng.integers(1, max_len + 1, size=n_seqs)
     return np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)

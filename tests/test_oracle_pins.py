@@ -393,3 +393,87 @@ def test_per_channel_decay_reduces_to_the_scalar_gate_and_to_deltanet():
     off = np.random.default_rng(6).standard_normal((2, 3, 2, 16)).repeat(64, axis=1)[:, :150]
     N3 = oracle.build_A_kda(x.K, Gp + off, x.beta, 64, return_N=True)[1]
     assert np.abs(N3 - N2).max() < 1e-12
+
+
+# ---------------------------------------------------------------- the layer's recurrence and its chunk form
+
+def test_recurrence_hand_worked_scalar_state():
+    # d_k = d_v = 1.  Token 1: k=1, v=2, beta=1/2, no decay: S = 1.  Token 2: decay 1/2 (g_2 - g_1 = -ln 2),
+    # k=2, v=3, beta=1/8: decayed S = 1/2, v - k S = 2, S = 1/2 + (1/8)(2)(2) = 1; read with q=4, scale 1/2: o = 2.
+    K = np.array([1.0, 2.0]).reshape(1, 2, 1, 1)
+    V = np.array([2.0, 3.0]).reshape(1, 2, 1, 1)
+    Q = np.array([1.0, 4.0]).reshape(1, 2, 1, 1)
+    beta = np.array([0.5, 0.125], np.float32).reshape(1, 2, 1)
+    g = np.array([0.0, -np.log(2.0)], np.float32).reshape(1, 2, 1)
+    O, S = oracle.gdn_recurrence(Q, K, V, beta, g, C=64, scale=0.5)
+    assert abs(O[0, 0, 0, 0] - 0.5) < 1e-12 and abs(O[0, 1, 0, 0] - 2.0) < 1e-7 and abs(S[0, 0, 0, 0] - 1.0) < 1e-7
+    # (a write-then-decay order would give S = (1 + (1/8)(2)(3 - 2)) / 2 = 5/8 instead)
+    # the same tokens as two chunks of one token, g = 0: the cumulative sum restarts, token 2 sees no decay:
+    # v - k S = 1, S = 1 + (1/8)(2)(1) = 5/4, o = (1/2)(4)(5/4) = 5/2
+    g0 = np.zeros((1, 2, 1), np.float32)
+    O2, S2 = oracle.gdn_recurrence(Q, K, V, beta, g0, C=1, scale=0.5)
+    assert abs(S2[0, 0, 0, 0] - 1.25) < 1e-12 and abs(O2[0, 1, 0, 0] - 2.5) < 1e-12
+    # g = (-ln 2, -ln 2) as two chunks of one token: token 2's own value is its decay (not the difference, 0)
+    gr = np.full((1, 2, 1), -np.log(2.0), np.float32)
+    _, S3 = oracle.gdn_recurrence(Q, K, V, beta, gr, C=1)
+    assert abs(S3[0, 0, 0, 0] - 1.0) < 1e-7
+    _, S4 = oracle.gdn_recurrence(Q, K, V, beta, gr, C=2)      # one chunk: difference 0, no decay
+    assert abs(S4[0, 0, 0, 0] - 1.25) < 1e-7
+
+
+def test_recurrence_writes_are_exact_reads_and_orthonormal_keys_give_linear_attention():
+    rng = np.random.default_rng(7)
+    d, T = 8, 8
+    Kq, _ = np.linalg.qr(rng.standard_normal((d, d)))          # orthonormal rows
+    K = Kq.reshape(1, T, 1, d)
+    V = rng.standard_normal((1, T, 1, 5))
+    ones, zeros = np.ones((1, T, 1), np.float32), np.zeros((1, T, 1), np.float32)
+    # beta = 1, no decay, unit keys: right after writing (k_t, v_t) the memory returns v_t for the query k_t
+    O, S = oracle.gdn_recurrence(K, K, V, ones, zeros, C=4)
+    assert np.abs(O - V).max() < 1e-12
+    # with mutually orthogonal keys nothing is ever overwritten: S = sum_t k_t v_t^T and the output is the
+    # causal linear attention (Q K^T * M) V of Sec. 1
+    Q = rng.standard_normal((1, T, 1, d))
+    O, S = oracle.gdn_recurrence(Q, K, V, ones, zeros, C=4, scale=0.7)
+    assert np.abs(S[0, 0] - K[0, :, 0].T @ V[0, :, 0]).max() < 1e-12
+    M = np.tril(np.ones((T, T)))
+    assert np.abs(O[0, :, 0] - 0.7 * ((Q[0, :, 0] @ K[0, :, 0].T) * M) @ V[0, :, 0]).max() < 1e-12
+    # a general (non-orthogonal) unit key still reads back its own value right after the write
+    Kn = rng.standard_normal((1, T, 1, d)); Kn /= np.linalg.norm(Kn, axis=-1, keepdims=True)
+    O, _ = oracle.gdn_recurrence(Kn, Kn, V, ones, zeros, C=4)
+    assert np.abs(O - V).max() < 1e-12
+
+
+def test_recurrence_without_writes_only_decays_the_carried_state():
+    x = wl.make("s", 1, 150, 2, 16, 16, 64, wl.F32, seed=41)
+    Q = wl.queries(x, seed=42)
+    S0 = wl.initial_state(x, seed=43)
+    O, S = oracle.gdn_recurrence(Q, x.K, x.V, np.zeros_like(x.beta), x.g, 64, scale=2.0, S0=S0)
+    g = x.g.astype(np.float64)[0]                                # [T,H]; total log-decay up to token t:
+    tot = g.copy()
+    tot[64:128] += g[63]
+    tot[128:] += g[63] + g[127]
+    for h in range(2):
+        want = 2.0 * np.exp(tot[:, h])[:, None] * (Q[0, :, h].astype(np.float64) @ S0[0, h].astype(np.float64))
+        assert np.abs(O[0, :, h] - want).max() < 1e-12
+        assert np.abs(S[0, h] - np.exp(tot[-1, h]) * S0[0, h]).max() < 1e-12
+
+
+def test_chunk_form_with_the_inverse_equals_the_recurrence():
+    # the re-formulation the whole path rests on: U~ = U - W S with W = A diag(beta gamma) K, U = A diag(beta) V
+    cu = np.array([0, 70, 71, 230], np.int32)
+    for cu_seqlens, B, T in ((None, 2, 150), (cu, 1, 230)):
+        x = wl.make("c", B, T, 2, 16, 24, 64, wl.F32, seed=44, cu_seqlens=cu_seqlens)
+        Q = wl.queries(x, seed=45)
+        S0 = wl.initial_state(x, seed=46)
+        A = oracle.build_A(x.K, x.beta, x.g, 64, cu_seqlens=cu_seqlens)
+        Kg = x.K.astype(np.float64) * np.exp(x.g.astype(np.float64))[..., None]
+        W, _ = oracle.wy(A, Kg, None, x.beta, 64, cu_seqlens=cu_seqlens)
+        _, U = oracle.wy(A, x.K, x.V, x.beta, 64, cu_seqlens=cu_seqlens)
+        O1, S1 = oracle.chunk_scan(Q, x.K, W, U, x.g, 64, scale=0.25, S0=S0, cu_seqlens=cu_seqlens)
+        O2, S2 = oracle.gdn_recurrence(Q, x.K, x.V, x.beta, x.g, 64, scale=0.25, S0=S0, cu_seqlens=cu_seqlens)
+        assert np.abs(O1 - O2).max() < 1e-11 and np.abs(S1 - S2).max() < 1e-11
+        # and the plain (not decay-weighted) W does NOT reproduce it: the decay factor belongs in W
+        Wp, _ = oracle.wy(A, x.K, None, x.beta, 64, cu_seqlens=cu_seqlens)
+        O3, _ = oracle.chunk_scan(Q, x.K, Wp, U, x.g, 64, scale=0.25, S0=S0, cu_seqlens=cu_seqlens)
+        assert np.abs(O3 - O2).max() > 1e-3
