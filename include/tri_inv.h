@@ -91,7 +91,11 @@ enum {
 #define TRI_INV_NS_ITERS(m) (((m) & 0xf) << 12)
   /* flag: run the plain fp32 CUDA-core kernel even where a tensor-core kernel
    * exists (same results up to rounding; for cross-checks and odd shapes). */
-  TRI_INV_FORCE_SIMT = 0x10000
+  TRI_INV_FORCE_SIMT = 0x10000,
+  /* flag, tri_inv_fused / tri_inv_fused_raw only: W = A diag(beta) diag(exp g) K, the decay-weighted factor
+   * that the chunk form of the layer's recurrence subtracts from U (tri_inv_chunk_scan consumes it).  U is
+   * unchanged.  Other entry points answer TRI_INV_ERR_UNSUPPORTED. */
+  TRI_INV_W_DECAY = 0x20000
 };
 
 /* ---- problem descriptor --------------------------------------------------- */

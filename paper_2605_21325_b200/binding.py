@@ -33,6 +33,7 @@ def ns_iters(m: int) -> int:
 
 
 FORCE_SIMT = 0x10000
+W_DECAY = 0x20000
 
 EXPORTS = ("tri_inv_build", "tri_inv_build_kda", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
            "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")

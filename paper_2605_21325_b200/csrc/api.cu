@@ -80,8 +80,12 @@ int check_desc(const tri_inv_desc* d, bool need_dv) {
   return TRI_INV_OK;
 }
 
-int check_method(int method) {
+int check_method(int method, bool w_decay_ok = false) {
   int m = method & TRI_INV_METHOD_MASK;
+  if (method & TRI_INV_W_DECAY) {
+    if (!w_decay_ok) return TRI_INV_ERR_UNSUPPORTED;
+    method &= ~TRI_INV_W_DECAY;
+  }
   if (m != TRI_INV_BLOCK_RECURSIVE && m != TRI_INV_PRODUCT_SERIES && m != TRI_INV_NEWTON_SCHULZ) return TRI_INV_ERR_UNSUPPORTED;
   if (method & ~(TRI_INV_METHOD_MASK | TRI_INV_LEAF_SERIES | TRI_INV_REFINE | TRI_INV_NS_ITERS(15) | TRI_INV_FORCE_SIMT)) return TRI_INV_ERR_UNSUPPORTED;
   if ((method & TRI_INV_LEAF_SERIES) && m != TRI_INV_BLOCK_RECURSIVE) return TRI_INV_ERR_UNSUPPORTED;
@@ -181,11 +185,11 @@ int tri_inv_fused(const void* K, const void* V, const float* beta, const float* 
   if (!K || !V || !beta || !g || !W || !U) return TRI_INV_ERR_INVALID_ARG;
   if (!aligned16(K) || !aligned16(V) || !aligned16(beta) || !aligned16(g) || !aligned16(A) || !aligned16(W) || !aligned16(U))
     return TRI_INV_ERR_INVALID_ARG;
-  if ((rc = check_method(method))) return rc;
+  if ((rc = check_method(method, true))) return rc;
   KParams p{};
   p.K = K; p.V = V; p.beta = beta; p.g = g; p.A = A; p.W = W; p.U = U;
-  p.method = method;
-  p.ops = kDoWY | (A ? kStoreA : 0);
+  p.method = method & ~TRI_INV_W_DECAY;
+  p.ops = kDoWY | (A ? kStoreA : 0) | ((method & TRI_INV_W_DECAY) ? kWDecay : 0);
   return run(p, desc, cuda_stream);
 }
 
@@ -198,12 +202,12 @@ int tri_inv_fused_raw(const void* K_raw, const void* V, const float* beta_logit,
   if (!aligned16(K_raw) || !aligned16(V) || !aligned16(beta_logit) || !aligned16(gate_logit) || !aligned16(A) ||
       !aligned16(W) || !aligned16(U) || !aligned16(beta_out) || !aligned16(g_out))
     return TRI_INV_ERR_INVALID_ARG;
-  if ((rc = check_method(method))) return rc;
+  if ((rc = check_method(method, true))) return rc;
   KParams p{};
   p.K = K_raw; p.V = V; p.beta = beta_logit; p.g = gate_logit; p.A = A; p.W = W; p.U = U;
   p.beta_out = beta_out; p.g_out = g_out;
-  p.method = method;
-  p.ops = kDoWY | kRaw | (A ? kStoreA : 0);
+  p.method = method & ~TRI_INV_W_DECAY;
+  p.ops = kDoWY | kRaw | (A ? kStoreA : 0) | ((method & TRI_INV_W_DECAY) ? kWDecay : 0);
   return run(p, desc, cuda_stream);
 }
 

@@ -14,7 +14,8 @@ enum : int {
   kDoWY = 2,    // compute W (and U when V != nullptr)
   kLoadA = 4,   // skip build + inversion, read A from A_in (tri_inv_wy)
   kKda = 16,    // per-channel decay: KParams::V holds G [B,T,H,d_k] fp32 (build only)
-  kRaw = 8,     // K is un-normalised, beta and g are logits: normalise, sigmoid, log-sigmoid + chunk cumsum in the kernel
+  kRaw = 8,
+  kWDecay = 32,  // W = A diag(beta) diag(exp g) K: the decay-weighted factor the chunk-state recurrence consumes     // K is un-normalised, beta and g are logits: normalise, sigmoid, log-sigmoid + chunk cumsum in the kernel
 };
 
 // One entry per chunk of tokens in ragged mode.

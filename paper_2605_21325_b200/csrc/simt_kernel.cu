@@ -365,7 +365,7 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
           for (int e = tid; e < C * kSlice; e += kThreads) {
             int j = e / kSlice, cc = e - j * kSlice;
             float v = 0.f;
-            if (j < rows && c0 + cc < d) v = sb[j] * (which ? 1.f : sr[j]) * load_kv(src, p.kv_dtype, ((size_t)(tok0 + j) * p.H + h) * d + c0 + cc);
+            if (j < rows && c0 + cc < d) v = sb[j] * (which ? 1.f : sr[j] * ((p.ops & kWDecay) ? expf(sg[j]) : 1.f)) * load_kv(src, p.kv_dtype, ((size_t)(tok0 + j) * p.H + h) * d + c0 + cc);
             Ks[j * kSliceLd + cc] = v;
           }
           __syncthreads();

@@ -128,7 +128,12 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
   const bool do_wy = !BO && (p.ops & kDoWY) != 0;
   const bool need_v = do_wy && p.V != nullptr;
   const bool load_a = (p.ops & kLoadA) != 0;
-  constexpr bool raw = RAW;  // the front end (sigmoid, log-sigmoid + chunk cumsum, key normalisation) is compiled in or out
+  // RAW compiles in the code that rewrites the K tile in shared memory before the WY step and the per-row
+  // factors of the gate.  Two run-time uses: the front end (sigmoid, log-sigmoid + chunk cumsum, key
+  // normalisation: kRaw) and the decay-weighted W (rows of K times exp(g_i): kWDecay).
+  constexpr bool raw = RAW;
+  const bool front = RAW && (p.ops & kRaw) != 0;
+  const bool wdecay = RAW && (p.ops & kWDecay) != 0;
   const int total = p.n_chunks * p.H;
 
   // Thread 0 requests the tiles of an item; K and V complete on separate barriers so that the Gram
@@ -216,7 +221,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
 
     // ---- 1. beta, g were fetched during the previous item (sBeta and sG are adjacent: one store each)
     // g is kept multiplied by log2(e) so that the gate can use ex2 directly
-    if (!raw) {
+    if (!raw || !front) {
       sBeta[tid] = bg_next * (tid < C ? 1.f : 1.4426950408889634f);
     } else {
       // raw front end: beta = sigmoid(logit); g = cumulative sum over the chunk of log sigmoid(gate logit)
@@ -297,7 +302,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         const int bx = e / (C * 8), rem = e - bx * (C * 8), r = rem >> 3, c = rem & 7;
         uint4* ptr = reinterpret_cast<uint4*>(smem + cfg::OFF_K + bx * cfg::BOX_BYTES + r * 128 + c * 16);
         uint4 v = *ptr;
-        const float sc = sR[r];
+        const float sc = wdecay ? sR[r] * ex2_approx(sG[r]) : sR[r];
         uint32_t* w = reinterpret_cast<uint32_t*>(&v);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -350,8 +355,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
           if (jb == rb && t == (g >> 1)) {
             const float da = (g & 1) ? sacc[2 * jb][1] : sacc[2 * jb][0];
             const float db = (g & 1) ? sacc[2 * jb + 1][3] : sacc[2 * jb + 1][2];
-            sR[16 * rb + g] = da > 0.f ? rsqrtf(da) : 0.f;
-            sR[16 * rb + g + 8] = db > 0.f ? rsqrtf(db) : 0.f;
+            sR[16 * rb + g] = !front ? 1.f : (da > 0.f ? rsqrtf(da) : 0.f);
+            sR[16 * rb + g + 8] = !front ? 1.f : (db > 0.f ? rsqrtf(db) : 0.f);
           }
         }
         __syncthreads();
@@ -835,7 +840,7 @@ cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handle
   if (p.d_k != 128 || ((p.ops & kDoWY) && p.V && p.d_v != 128)) return cudaSuccess;
   // the stride of the 2-D view (H * d * 2 bytes) is a multiple of 16 because d is a multiple of 8
   *handled = true;
-  const bool raw = (p.ops & kRaw) != 0;
+  const bool raw = (p.ops & (kRaw | kWDecay)) != 0;  // both need the variant that rewrites the K tile
   if (C == 64) {
     if (!raw && !series && !(p.ops & (kDoWY | kLoadA))) return launch_one<64, 128, false, false, true>(p, stream);  // tri_inv_build
     if (raw) return series ? launch_one<64, 128, true, true>(p, stream) : launch_one<64, 128, false, true>(p, stream);

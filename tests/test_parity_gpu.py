@@ -447,3 +447,30 @@ def test_build_kda_with_a_channel_constant_gate_equals_build(bnd):
     A2 = bnd.build(dev["K"], dev["beta"], dev["g"], 64)
     torch.cuda.synchronize()
     assert (A1 - A2).abs().max().item() <= 2e-3
+
+
+# ---------------------------------------------------------------- decay-weighted W (input of the chunk scan)
+
+@pytest.mark.parametrize("C,dtype,d", [(64, wl.BF16, 128), (128, wl.BF16, 128), (64, wl.F32, 64)])
+def test_fused_decay_weighted_w(bnd, C, dtype, d):
+    cu = np.array([0, 2 * C + 9, 3 * C + 9, 3 * C + 10], np.int32)
+    for cu_seqlens, B, T in ((None, 2, 3 * C), (cu, 1, int(cu[-1]))):
+        inp = wl.make("wd", B, T, 2, d, d, C, dtype, seed=70 + C, cu_seqlens=cu_seqlens)
+        A_ref = oracle.build_A(inp.K, inp.beta, inp.g, C, cu_seqlens=cu_seqlens)
+        Kg = bnd.to_numpy_f64(bnd.kv_to_torch(inp.K, "cpu")) * np.exp(inp.g.astype(np.float64))[..., None]
+        W_ref, _ = oracle.wy(A_ref, Kg, None, inp.beta, C, cu_seqlens=cu_seqlens)
+        _, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, C, cu_seqlens=cu_seqlens)
+        dev = bnd.to_device(inp)
+        for m in (bnd.BLOCK_RECURSIVE, bnd.PRODUCT_SERIES):
+            A, W, U = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], C, method=m | bnd.W_DECAY, cu_seqlens=cu_seqlens)
+            torch.cuda.synchronize()
+            assert bnd.last_device_status() == 0
+            assert max_ratio(bnd.to_numpy_f64(W), W_ref) <= TOL_WY[dtype]
+            assert max_ratio(bnd.to_numpy_f64(U), U_ref) <= TOL_WY[dtype]
+
+
+def test_w_decay_is_refused_where_there_is_no_w(bnd):
+    inp = wl.config(1)
+    dev = bnd.to_device(inp)
+    with pytest.raises(bnd.TriInvError):
+        bnd.build(dev["K"], dev["beta"], dev["g"], inp.C, method=bnd.BLOCK_RECURSIVE | bnd.W_DECAY)
