@@ -154,6 +154,27 @@ int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A
                       const tri_inv_desc* desc, int method, void* cuda_stream);
 
 /*
+ * Chunk scan: the consumer of W and U -- the chunk form of the layer's recurrence (the re-formulation Sec. 1
+ * refers to, in which (I+N)^{-1} appears through W and U).  Per sequence and head, chunk after chunk, with the
+ * state S [d_k x d_v] entering the chunk (S0, or zero) and gamma_i = exp(g_i):
+ *     U~ = U - W S
+ *     O  = scale * (diag(gamma) Q S + ((Q K^T) * D) U~),     D_ij = gamma_i / gamma_j for j <= i, else 0
+ *     S <- gamma_last S + (diag(gamma_last / gamma) K)^T U~
+ * W must be the decay-weighted factor (TRI_INV_W_DECAY of the fused calls), U the plain one.  With exact W and U
+ * this equals the token-by-token recurrence  S <- exp(a_t) S;  S <- S + beta_t k_t (v_t - S^T k_t)^T;
+ * o_t = scale S^T q_t.
+ *   Q, K, W [B,T,H,d_k], U [B,T,H,d_v]: device, bf16, 16-byte aligned;  g [B,T,H] fp32 device;
+ *   S0, S_out [n_sequences,H,d_k,d_v] fp32 device, each may be NULL (zero initial state / final state not wanted);
+ *   O [B,T,H,d_v] bf16 device: rows of real tokens are written.
+ * Dense and ragged chunking as in tri_inv_build (desc->cu_seqlens on the HOST).  Supported: bf16,
+ * d_k = d_v = 128, C = 64; anything else answers TRI_INV_ERR_UNSUPPORTED.  Launch is asynchronous on
+ * cuda_stream; nothing is allocated except, in ragged mode, n_sequences + 1 ints from the library's
+ * stream-ordered pool.  A device-side wait that expires raises TRI_INV_ERR_DEVICE_TIMEOUT in the status word.
+ */
+int tri_inv_chunk_scan(const void* Q, const void* K, const void* W, const void* U, const float* g, const float* S0,
+                       void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream);
+
+/*
  * Fused call with the layer's front end folded in: the kernel takes what the projections produce and
  * does the three producers that otherwise run as separate passes over memory before the inversion
  * (the gating recipe of a Gated-DeltaNet layer; in the paper these are among the kernels its fused

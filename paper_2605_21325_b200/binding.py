@@ -35,7 +35,7 @@ def ns_iters(m: int) -> int:
 FORCE_SIMT = 0x10000
 W_DECAY = 0x20000
 
-EXPORTS = ("tri_inv_build", "tri_inv_build_kda", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
+EXPORTS = ("tri_inv_build", "tri_inv_build_kda", "tri_inv_chunk_scan", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
            "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
 
 
@@ -69,6 +69,8 @@ def load():
         lib.tri_inv_fused.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_build_kda.argtypes = [vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_build_kda.restype = i32
+        lib.tri_inv_chunk_scan.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, dp, vp]
+        lib.tri_inv_chunk_scan.restype = i32
         lib.tri_inv_fused_raw.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_fused_raw.restype = i32
         lib.tri_inv_fused_packed_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
@@ -159,6 +161,27 @@ def build_kda(K, G, beta, C, method=BLOCK_RECURSIVE, cu_seqlens=None, out=None, 
     if rc != OK:
         raise TriInvError("tri_inv_build_kda", rc)
     return A
+
+
+def chunk_scan(Q, K, W, U, g, C, scale=1.0, S0=None, cu_seqlens=None, out=None, want_state=True, stream=None):
+    """O, S_final of the chunk form of the layer's recurrence from the decay-weighted W and U (tri_inv_chunk_scan)."""
+    B, T, H, d_k = K.shape
+    d_v = U.shape[3]
+    desc, keep = make_desc(B, T, H, d_k, d_v, C, _dtype_code(K), cu_seqlens)
+    n_seqs = B if cu_seqlens is None else len(cu_seqlens) - 1
+    O = torch.empty((B, T, H, d_v), dtype=U.dtype, device=K.device) if out is None else out
+    S = torch.empty((n_seqs, H, d_k, d_v), dtype=torch.float32, device=K.device) if want_state else None
+    rc = load().tri_inv_chunk_scan(_p(Q), _p(K), _p(W), _p(U), _p(g), _p(S0), _p(O), _p(S), float(scale),
+                                   ctypes.byref(desc), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_chunk_scan", rc)
+    return O, S
+
+
+def gdn_forward(Q, K, V, beta, g, C, scale=1.0, S0=None, method=BLOCK_RECURSIVE, cu_seqlens=None, stream=None):
+    """The whole layer in two launches: fused build + inversion + WY with the decay-weighted W, then the chunk scan."""
+    _, W, U = fused(K, V, beta, g, C, method=method | W_DECAY, cu_seqlens=cu_seqlens, want_A=False, stream=stream)
+    return chunk_scan(Q, K, W, U, g, C, scale=scale, S0=S0, cu_seqlens=cu_seqlens, stream=stream)
 
 
 def wy(A, K, V, beta, cu_seqlens=None, out=None, stream=None):

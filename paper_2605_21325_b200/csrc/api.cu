@@ -225,6 +225,41 @@ int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A
   return run(p, desc, cuda_stream);
 }
 
+int tri_inv_chunk_scan(const void* Q, const void* K, const void* W, const void* U, const float* g, const float* S0,
+                       void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream) {
+  int rc = check_desc(desc, true);
+  if (rc) return rc;
+  if (!Q || !K || !W || !U || !g || !O) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(W) || !aligned16(U) || !aligned16(g) || !aligned16(O) || !aligned16(S0) ||
+      !aligned16(S_out))
+    return TRI_INV_ERR_INVALID_ARG;
+  if (desc->kv_dtype != TRI_INV_BF16 || desc->d_k != 128 || desc->d_v != 128 || desc->C != 64) return TRI_INV_ERR_UNSUPPORTED;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  ScanParams p{};
+  p.U = U; p.g = g; p.S0 = S0; p.O = O; p.S_out = S_out; p.scale = scale;
+  p.H = desc->H; p.T = desc->T;
+  p.n_seqs = desc->cu_seqlens ? desc->n_seqs : desc->B;
+  cudaError_t err;
+  p.status = status_word_for_current_device(&err);
+  if (!p.status) return TRI_INV_ERR_CUDA;
+  const long long tokens = desc->cu_seqlens ? (long long)desc->T : (long long)desc->T * desc->B;
+  if (p.n_seqs == 0 || (tokens == 0 && !S_out)) return TRI_INV_OK;
+  int* dev_off = nullptr;
+  if (desc->cu_seqlens) {
+    cudaMemPool_t pool = table_pool_for_current_device();
+    if (!pool || cudaMallocFromPoolAsync((void**)&dev_off, (size_t)(p.n_seqs + 1) * sizeof(int), pool, stream) != cudaSuccess) return TRI_INV_ERR_CUDA;
+    if (launch_seq_offsets(dev_off, desc, stream) != cudaSuccess) {
+      cudaFreeAsync(dev_off, stream);
+      return TRI_INV_ERR_CUDA;
+    }
+    p.seq_off = dev_off;
+  }
+  err = launch_chunk_scan(p, Q, K, W, tokens > 0 ? tokens : 1, stream);
+  if (err == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (dev_off) cudaFreeAsync(dev_off, stream);
+  return err == cudaSuccess ? TRI_INV_OK : TRI_INV_ERR_CUDA;
+}
+
 int tri_inv_count_matrices(const tri_inv_desc* desc, int64_t* out) {
   int rc = check_desc(desc, false);
   if (rc) return rc;

@@ -74,6 +74,21 @@ __device__ __forceinline__ float load_kv(const void* base, int dtype, size_t idx
 cudaError_t launch_simt(const KParams& p, int C, cudaStream_t stream);
 // Tensor-core path: returns cudaErrorNotSupported when it has no kernel for the request.
 cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
+// Chunk scan (consumer of W and U): parameters other than the three TMA-staged tensors.
+struct ScanParams {
+  const void* U;        // [tokens,H,128] bf16
+  const float* g;       // [tokens,H]
+  const float* S0;      // [n_seqs,H,128,128] fp32 or null (zero state)
+  void* O;              // [tokens,H,128] bf16
+  float* S_out;         // [n_seqs,H,128,128] fp32 or null
+  const int* seq_off;   // device copy of cu_seqlens (ragged) or null (dense: sequence s = tokens [s T, (s+1) T))
+  int* status;
+  int H, T, n_seqs;
+  float scale;
+};
+cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t stream);
+cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,
+                              cudaStream_t stream);
 // Per-channel decay variant on the tensor cores (bf16 keys, d_k = 128, C = 64, block recursion).
 cudaError_t launch_kda_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
 

@@ -1,0 +1,404 @@
+// Chunk scan: the consumer of W and U.  The chunk form of the layer's recurrence (the re-formulation that
+// Sec. 1 refers to; (I+N)^{-1} enters through W and U), per sequence and head, chunk after chunk, with the
+// state S [d_k x d_v] carried in registers:
+//
+//     U~ = U - W S                                   W = A diag(beta exp g) K (decay-weighted), U = A diag(beta) V
+//     O  = scale * (diag(gamma) Q S + P U~)          gamma_i = exp(g_i),  P_ij = (q_i . k_j) gamma_i / gamma_j  (j <= i)
+//     S <- gamma_last S + K^T diag(gamma_last / gamma) U~
+//
+// Columns of S (the d_v axis) never mix, so a CTA owns one (sequence, head, slice of DVS value columns) and walks
+// the chunks in order; the slices of one head run side by side and share W, Q, K through L2.
+//
+// Per chunk, on the tensor cores (tcgen05.mma kind::f16, fp32 accumulators in tensor memory):
+//   T1 = W S   and  QS = Q S   (B operand: S rounded to bf16, kept K-major in shared memory),
+//   QK = Q K^T,   dS = K^T U~' (A operand: the K tile read MN-major; U~' = decay-scaled U~ in bf16),   PU = P U~.
+// The dependent chain of a chunk is  T1 -> U~ -> dS -> S;  QS, QK, P and PU hang off it.
+// TMA brings the W, Q and K tiles (one buffer each, refilled as soon as their last reader has retired);
+// U and g come through registers one chunk ahead.
+// Every mbarrier wait is bounded; on expiry the CTA raises the status word, frees its tensor memory and returns.
+#include "tc_device.cuh"
+
+namespace tri_inv {
+namespace {
+
+constexpr int C = 64, D = 128, NT = 128;
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <int DVS>
+struct ScanCfg {
+  static constexpr int OFF_W = 0, OFF_Q = 16384, OFF_K = 32768;   // bf16 tiles: 2 boxes of 64 rows x 128 B
+  static constexpr int OFF_S = 49152;                             // S^T bf16 [DVS rows][128 d_k]: 2 boxes of DVS rows x 128 B
+  static constexpr int S_BOX = DVS * 128;
+  static constexpr int OFF_UT = OFF_S + 2 * S_BOX;                // U~^T  bf16 [DVS rows][64 tokens]
+  static constexpr int OFF_UD = OFF_UT + DVS * 128;               // U~'^T bf16 (rows scaled by gamma_last / gamma_i)
+  static constexpr int OFF_P = OFF_UD + DVS * 128;                // P bf16 [64][64]
+  static constexpr int OFF_G = OFF_P + 8192;                      // g * log2(e): two buffers of 64 floats
+  static constexpr int OFF_BAR = OFF_G + 512;                     // 7 mbarriers, tensor-memory slot
+  static constexpr int SMEM = OFF_BAR + 64;
+  static constexpr int TM_QK = 0, TM_T1 = 64, TM_QS = 64 + DVS, TM_PU = 64 + 2 * DVS, TM_DS = 64 + 3 * DVS;
+  static constexpr int TMEM_COLS = (64 + 4 * DVS) <= 256 ? 256 : 512;
+  static constexpr int CTAS_PER_SM = TMEM_COLS == 256 ? 2 : 1;
+  static constexpr int NTL = DVS / 8;                             // accumulator n-tiles per row block
+};
+
+// kind::f16 instruction descriptor with an MN-major A operand (bit 15): A is read as stored [k][m].
+__host__ __device__ constexpr uint32_t umma_idesc_amn(int M, int N) { return umma_idesc(M, N, 0) | (1u << 15); }
+
+__device__ __forceinline__ void tmem_ld_16x32(float (&r)[4][4], uint32_t taddr) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=f"(r[0][0]), "=f"(r[0][1]), "=f"(r[0][2]), "=f"(r[0][3]), "=f"(r[1][0]), "=f"(r[1][1]), "=f"(r[1][2]), "=f"(r[1][3]),
+        "=f"(r[2][0]), "=f"(r[2][1]), "=f"(r[2][2]), "=f"(r[2][3]), "=f"(r[3][0]), "=f"(r[3][1]), "=f"(r[3][2]), "=f"(r[3][3])
+      : "r"(taddr));
+}
+template <int NTL>
+__device__ __forceinline__ void tmem_ld_frag(float (&r)[NTL][4], uint32_t taddr) {
+  if constexpr (NTL == 8) tmem_ld_16x64(r, taddr);
+  else tmem_ld_16x32(r, taddr);
+}
+// 32 lanes x 32 columns: thread = lane, 32 consecutive columns
+__device__ __forceinline__ void tmem_ld_32x32(float* r, uint32_t taddr) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=f"(r[0]), "=f"(r[1]), "=f"(r[2]), "=f"(r[3]), "=f"(r[4]), "=f"(r[5]), "=f"(r[6]), "=f"(r[7]), "=f"(r[8]), "=f"(r[9]), "=f"(r[10]),
+        "=f"(r[11]), "=f"(r[12]), "=f"(r[13]), "=f"(r[14]), "=f"(r[15]), "=f"(r[16]), "=f"(r[17]), "=f"(r[18]), "=f"(r[19]), "=f"(r[20]),
+        "=f"(r[21]), "=f"(r[22]), "=f"(r[23]), "=f"(r[24]), "=f"(r[25]), "=f"(r[26]), "=f"(r[27]), "=f"(r[28]), "=f"(r[29]), "=f"(r[30]),
+        "=f"(r[31])
+      : "r"(taddr));
+}
+
+template <int DVS>
+__global__ void __launch_bounds__(NT, ScanCfg<DVS>::CTAS_PER_SM)
+chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmQ,
+                  const __grid_constant__ CUtensorMap tmK, ScanParams p) {
+  using cfg = ScanCfg<DVS>;
+  constexpr int NTL = cfg::NTL, NS = D / DVS;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  float* sG = reinterpret_cast<float*>(smem + cfg::OFF_G);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 56);
+  const uint32_t sW = smem_u32(smem + cfg::OFF_W), sQ = smem_u32(smem + cfg::OFF_Q), sK = smem_u32(smem + cfg::OFF_K);
+  const uint32_t sS = smem_u32(smem + cfg::OFF_S), sUt = smem_u32(smem + cfg::OFF_UT), sUd = smem_u32(smem + cfg::OFF_UD);
+  const uint32_t sP = smem_u32(smem + cfg::OFF_P);
+  const uint32_t bar_w = smem_u32(smem + cfg::OFF_BAR), bar_q = bar_w + 8, bar_k = bar_w + 16, bar_t1 = bar_w + 24,
+                 bar_o = bar_w + 32, bar_s = bar_w + 40, bar_pu = bar_w + 48;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int gq = lane >> 2, t = lane & 3;
+  const int ra = 16 * warp + gq, rb = ra + 8;   // this thread's two rows of every M = 64 accumulator
+
+  const int slice = blockIdx.x % NS, h = (blockIdx.x / NS) % p.H, s = blockIdx.x / (NS * p.H);
+  const int beg = p.seq_off ? p.seq_off[s] : s * p.T;
+  const int end = p.seq_off ? p.seq_off[s + 1] : (s + 1) * p.T;
+  const int n_chunks = (end - beg + C - 1) / C;
+  const int col0 = slice * DVS;                  // first value column of this CTA
+
+  // state: thread tid owns row tid (a key feature) of S, DVS columns
+  float S[DVS];
+  {
+    const float* s0 = p.S0 ? p.S0 + (((size_t)s * p.H + h) * D + tid) * D + col0 : nullptr;
+#pragma unroll
+    for (int n = 0; n < DVS; n += 4) {
+      float4 v = s0 ? *reinterpret_cast<const float4*>(s0 + n) : make_float4(0.f, 0.f, 0.f, 0.f);
+      S[n] = v.x; S[n + 1] = v.y; S[n + 2] = v.z; S[n + 3] = v.w;
+    }
+  }
+  auto store_state = [&]() {
+    if (!p.S_out) return;
+    float* dst = p.S_out + (((size_t)s * p.H + h) * D + tid) * D + col0;
+#pragma unroll
+    for (int n = 0; n < DVS; n += 4) *reinterpret_cast<float4*>(dst + n) = make_float4(S[n], S[n + 1], S[n + 2], S[n + 3]);
+  };
+  if (n_chunks == 0) { store_state(); return; }
+  const bool misaligned = (sW & 1023u) != 0;     // never expected; the swizzle pattern would not match the copies
+
+  // S^T as the K-major B operand: element (n, k) of a [DVS rows][128] bf16 tile, two boxes of 64 features
+  auto write_state_operand = [&]() {
+    uint8_t* base = smem + cfg::OFF_S + (tid >> 6) * cfg::S_BOX + (tid & 7) * 2;
+    const int kc = (tid & 63) >> 3;
+#pragma unroll
+    for (int n = 0; n < DVS; ++n)
+      *reinterpret_cast<__nv_bfloat16*>(base + n * 128 + ((kc ^ (n & 7)) << 4)) = __float2bfloat16_rn(S[n]);
+  };
+  auto issue_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int tok0) {
+    mbar_expect_tx(bar, 16384u);
+    tma_load_2d(dst, tm, bar, h * D, tok0);
+    tma_load_2d(dst + 8192, tm, bar, h * D + 64, tok0);
+  };
+  const __nv_bfloat16* Ug = reinterpret_cast<const __nv_bfloat16*>(p.U);
+  auto fetch_u = [&](uint32_t (&u)[NTL][2], int tok0, int rows) {
+#pragma unroll
+    for (int nt = 0; nt < NTL; ++nt) {
+      const int c = col0 + 8 * nt + 2 * t;
+      u[nt][0] = ra < rows ? *reinterpret_cast<const uint32_t*>(Ug + ((size_t)(tok0 + ra) * p.H + h) * D + c) : 0u;
+      u[nt][1] = rb < rows ? *reinterpret_cast<const uint32_t*>(Ug + ((size_t)(tok0 + rb) * p.H + h) * D + c) : 0u;
+    }
+  };
+  // rows past the sequence end take the last real row's g, so that every exponent stays a difference of real values
+  auto fetch_g = [&](int tok0, int rows) -> float {
+    const int i = tid < rows ? tid : rows - 1;
+    return tid < C ? p.g[(size_t)(tok0 + i) * p.H + h] * kLog2e : 0.f;
+  };
+
+  uint32_t u_next[NTL][2];
+  float g_next;
+  {
+    const int rows0 = end - beg < C ? end - beg : C;
+    if (tid == 0) {
+      prefetch_tmap(&tmW); prefetch_tmap(&tmQ); prefetch_tmap(&tmK);
+      for (int b = 0; b < 7; ++b) mbar_init(bar_w + 8 * b, 1);
+      fence_mbar_init();
+      if (!misaligned) {
+        issue_tile(sW, &tmW, bar_w, beg);
+        issue_tile(sQ, &tmQ, bar_q, beg);
+        issue_tile(sK, &tmK, bar_k, beg);
+      }
+    }
+    fetch_u(u_next, beg, rows0);
+    g_next = fetch_g(beg, rows0);
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(cfg::TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  write_state_operand();
+  if (tid < C) sG[tid] = g_next;
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem_rows = tmem + ((uint32_t)(32 * warp) << 16);
+
+  constexpr uint32_t idesc_n = umma_idesc(C, DVS, 0), idesc_qk = umma_idesc(C, C, 0), idesc_ds = umma_idesc_amn(D, DVS);
+  auto mma_k128 = [&](uint32_t d_tmem, uint32_t a_base, uint32_t b_base, uint32_t b_box, uint32_t idesc) {
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+      const uint64_t da = umma_desc(a_base + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024);
+      const uint64_t db = umma_desc(b_base + (ks >> 2) * b_box + (ks & 3) * 32, 16, 1024);
+      umma_bf16(d_tmem, da, db, idesc, ks > 0);
+    }
+  };
+
+  uint32_t ph = 0;
+  bool failed = misaligned;
+  for (int c = 0; c < n_chunks && !misaligned; ++c) {
+    const int tok0 = beg + c * C;
+    const int rows = end - tok0 < C ? end - tok0 : C;
+    const bool has_next = c + 1 < n_chunks;
+    const int nx_tok0 = tok0 + C, nx_rows = end - nx_tok0 < C ? end - nx_tok0 : C;
+    const float* gb = sG + (c & 1) * C;
+
+    // ---- A. products that need only S and the tiles
+    if (tid == 0) {
+      if (!mbar_wait_bounded(bar_w, ph)) {
+        atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);   // the other threads time out on bar_t1
+      } else {
+        tc_fence_after();
+        mma_k128(tmem + cfg::TM_T1, sW, sS, cfg::S_BOX, idesc_n);
+        umma_commit(bar_t1);
+        if (!mbar_wait_bounded(bar_q, ph) || !mbar_wait_bounded(bar_k, ph)) {
+          atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+        } else {
+          tc_fence_after();
+          mma_k128(tmem + cfg::TM_QS, sQ, sS, cfg::S_BOX, idesc_n);
+          mma_k128(tmem + cfg::TM_QK, sQ, sK, 8192, idesc_qk);
+          umma_commit(bar_o);
+        }
+      }
+    }
+    uint32_t u_cur[NTL][2];
+#pragma unroll
+    for (int nt = 0; nt < NTL; ++nt) { u_cur[nt][0] = u_next[nt][0]; u_cur[nt][1] = u_next[nt][1]; }
+    if (has_next) {
+      fetch_u(u_next, nx_tok0, nx_rows);
+      g_next = fetch_g(nx_tok0, nx_rows);
+    }
+    const float g_a = gb[ra], g_b = gb[rb], g_last = gb[rows - 1];
+
+    // ---- B. U~ = U - W S  ->  bf16 operands U~^T and (decay-scaled) U~'^T
+    if (!mbar_wait_bounded(bar_t1, ph)) { failed = true; break; }
+    tc_fence_after();
+    if (tid == 32 && has_next) issue_tile(sW, &tmW, bar_w, nx_tok0);   // W's only reader has retired
+    {
+      float t1[NTL][4];
+      tmem_ld_frag<NTL>(t1, tmem_rows + cfg::TM_T1);
+      tmem_wait_ld();
+      const float da = ex2_approx(g_last - g_a), db = ex2_approx(g_last - g_b);
+      const int ca = ra >> 3, cb = rb >> 3;
+#pragma unroll
+      for (int nt = 0; nt < NTL; ++nt) {
+        const float2 ua = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u_cur[nt][0]));
+        const float2 ub = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u_cur[nt][1]));
+        const float v0 = ra < rows ? ua.x - t1[nt][0] : 0.f, v1 = ra < rows ? ua.y - t1[nt][1] : 0.f;
+        const float v2 = rb < rows ? ub.x - t1[nt][2] : 0.f, v3 = rb < rows ? ub.y - t1[nt][3] : 0.f;
+        const int n0 = 8 * nt + 2 * t, n1 = n0 + 1;
+        // element (n, token) of a [DVS rows][64 tokens] bf16 tile, 128-byte rows, 16-byte pieces swizzled by the row
+        const uint32_t o0a = n0 * 128 + ((ca ^ (n0 & 7)) << 4) + (ra & 7) * 2, o1a = n1 * 128 + ((ca ^ (n1 & 7)) << 4) + (ra & 7) * 2;
+        const uint32_t o0b = n0 * 128 + ((cb ^ (n0 & 7)) << 4) + (rb & 7) * 2, o1b = n1 * 128 + ((cb ^ (n1 & 7)) << 4) + (rb & 7) * 2;
+        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o0a) = __float2bfloat16_rn(v0);
+        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o1a) = __float2bfloat16_rn(v1);
+        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o0b) = __float2bfloat16_rn(v2);
+        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o1b) = __float2bfloat16_rn(v3);
+        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o0a) = __float2bfloat16_rn(v0 * da);
+        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o1a) = __float2bfloat16_rn(v1 * da);
+        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o0b) = __float2bfloat16_rn(v2 * db);
+        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o1b) = __float2bfloat16_rn(v3 * db);
+      }
+    }
+    // ---- P = (Q K^T) * decay, lower triangle with its diagonal; QS kept in registers for the output
+    if (!mbar_wait_bounded(bar_o, ph)) { failed = true; break; }
+    tc_fence_after();
+    if (tid == 64 && has_next) issue_tile(sQ, &tmQ, bar_q, nx_tok0);   // Q's readers have retired
+    float qs[NTL][4];
+    {
+      float qk[8][4];
+      tmem_ld_16x64(qk, tmem_rows + cfg::TM_QK);
+      tmem_ld_frag<NTL>(qs, tmem_rows + cfg::TM_QS);
+      tmem_wait_ld();
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        const int j = 8 * nt + 2 * t;
+        const float2 gj = *reinterpret_cast<const float2*>(gb + j);
+        const float p0 = j <= ra ? qk[nt][0] * ex2_approx(g_a - gj.x) : 0.f, p1 = j + 1 <= ra ? qk[nt][1] * ex2_approx(g_a - gj.y) : 0.f;
+        const float p2 = j <= rb ? qk[nt][2] * ex2_approx(g_b - gj.x) : 0.f, p3 = j + 1 <= rb ? qk[nt][3] * ex2_approx(g_b - gj.y) : 0.f;
+        *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + ra * 128 + ((nt ^ (ra & 7)) << 4) + 4 * t) = pack_bf16(p0, p1);
+        *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + rb * 128 + ((nt ^ (rb & 7)) << 4) + 4 * t) = pack_bf16(p2, p3);
+      }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- C. dS = K^T U~'  and  PU = P U~
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < C / 16; ++ks) {
+        const uint64_t da = umma_desc(sK + ks * 2048, 8192, 1024);   // K tile read MN-major: 16 tokens per step
+        const uint64_t db = umma_desc(sUd + ks * 32, 16, 1024);
+        umma_bf16(tmem + cfg::TM_DS, da, db, idesc_ds, ks > 0);
+      }
+      umma_commit(bar_s);
+#pragma unroll
+      for (int ks = 0; ks < C / 16; ++ks) {
+        const uint64_t da = umma_desc(sP + ks * 32, 16, 1024);
+        const uint64_t db = umma_desc(sUt + ks * 32, 16, 1024);
+        umma_bf16(tmem + cfg::TM_PU, da, db, idesc_n, ks > 0);
+      }
+      umma_commit(bar_pu);
+    }
+    if (tid < C && has_next) sG[((c + 1) & 1) * C + tid] = g_next;
+
+    // ---- D. state update (thread = row of S) and the bf16 operand for the next chunk
+    if (!mbar_wait_bounded(bar_s, ph)) { failed = true; break; }
+    tc_fence_after();
+    if (tid == 96 && has_next) issue_tile(sK, &tmK, bar_k, nx_tok0);   // K's readers have retired
+    {
+      const float gl = ex2_approx(g_last);
+#pragma unroll
+      for (int n0 = 0; n0 < DVS; n0 += 32) {
+        float ds[32];
+        tmem_ld_32x32(ds, tmem_rows + cfg::TM_DS + n0);
+        tmem_wait_ld();
+#pragma unroll
+        for (int n = 0; n < 32; ++n) S[n0 + n] = fmaf(gl, S[n0 + n], ds[n]);
+      }
+      if (has_next) write_state_operand();
+    }
+    // ---- E. O = scale * (gamma_i QS + PU)
+    if (!mbar_wait_bounded(bar_pu, ph)) { failed = true; break; }
+    tc_fence_after();
+    {
+      float pu[NTL][4];
+      tmem_ld_frag<NTL>(pu, tmem_rows + cfg::TM_PU);
+      tmem_wait_ld();
+      const float sa = p.scale * ex2_approx(g_a), sb = p.scale * ex2_approx(g_b);
+      __nv_bfloat16* Og = reinterpret_cast<__nv_bfloat16*>(p.O);
+#pragma unroll
+      for (int nt = 0; nt < NTL; ++nt) {
+        const int cc = col0 + 8 * nt + 2 * t;
+        if (ra < rows)
+          *reinterpret_cast<uint32_t*>(Og + ((size_t)(tok0 + ra) * p.H + h) * D + cc) =
+              pack_bf16(fmaf(sa, qs[nt][0], p.scale * pu[nt][0]), fmaf(sa, qs[nt][1], p.scale * pu[nt][1]));
+        if (rb < rows)
+          *reinterpret_cast<uint32_t*>(Og + ((size_t)(tok0 + rb) * p.H + h) * D + cc) =
+              pack_bf16(fmaf(sb, qs[nt][2], p.scale * pu[nt][2]), fmaf(sb, qs[nt][3], p.scale * pu[nt][3]));
+      }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    ph ^= 1;
+  }
+  if (failed) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+  else store_state();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(cfg::TMEM_COLS) : "memory");
+}
+
+constexpr int kSeqsPerLaunch = 960;
+struct OffsetBatch {
+  int32_t cu[kSeqsPerLaunch + 1];
+  int32_t n, first;
+};
+__global__ void __launch_bounds__(256) seq_offsets_kernel(int* out, const __grid_constant__ OffsetBatch b) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i <= b.n; i += gridDim.x * blockDim.x) out[b.first + i] = b.cu[i];
+}
+
+template <int DVS>
+cudaError_t launch_scan_one(const ScanParams& p, const CUtensorMap& tmW, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                            cudaStream_t stream) {
+  using cfg = ScanCfg<DVS>;
+  static std::mutex mu;
+  static bool ready[64] = {false};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ready[dev]) {
+      if ((e = cudaFuncSetAttribute(chunk_scan_kernel<DVS>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(chunk_scan_kernel<DVS>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
+      ready[dev] = true;
+    }
+  }
+  const long long grid = (long long)p.n_seqs * p.H * (D / DVS);
+  if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
+  chunk_scan_kernel<DVS><<<(int)grid, NT, cfg::SMEM, stream>>>(tmW, tmQ, tmK, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// The device copy of cu_seqlens (n_seqs + 1 ints), written from kernel parameters: no host-to-device copy.
+cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t stream) {
+  for (int s0 = 0; s0 <= d->n_seqs; s0 += kSeqsPerLaunch) {
+    OffsetBatch b;
+    b.first = s0;
+    b.n = d->n_seqs - s0 < kSeqsPerLaunch ? d->n_seqs - s0 : kSeqsPerLaunch;
+    for (int q = 0; q <= b.n; ++q) b.cu[q] = d->cu_seqlens[s0 + q];
+    seq_offsets_kernel<<<(b.n + 256) / 256, 256, 0, stream>>>(dev_out, b);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (s0 + kSeqsPerLaunch >= d->n_seqs) break;
+  }
+  return cudaSuccess;
+}
+
+// bf16 Q, K, W, U with d_k = d_v = 128 and C = 64.  32 value columns per CTA (two CTAs per SM) unless the batch
+// alone fills the GPU twice over, in which case 64 columns per CTA halve the re-reads of W, Q and K through L2.
+cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,
+                              cudaStream_t stream) {
+  CUtensorMap tmW, tmQ, tmK;
+  if (!make_tmap(&tmW, W, tokens, p.H, D, C, 2) || !make_tmap(&tmQ, Q, tokens, p.H, D, C, 2) || !make_tmap(&tmK, K, tokens, p.H, D, C, 2))
+    return cudaErrorUnknown;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if ((long long)p.n_seqs * p.H * 2 >= 2LL * sms) return launch_scan_one<64>(p, tmW, tmQ, tmK, stream);
+  return launch_scan_one<32>(p, tmW, tmQ, tmK, stream);
+}
+
+}  // namespace tri_inv

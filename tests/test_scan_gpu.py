@@ -1,0 +1,110 @@
+"""GPU parity of the chunk scan (consumer of W and U) and of the two-launch layer forward.
+
+Tolerances (bf16 operands, fp32 accumulation; derived in the design notes):
+  chunk scan alone, given the oracle's W and U rounded to bf16:
+      max|O_gpu - O_ref| / max|O_ref| <= 1e-2,   max|S_gpu - S_ref| / max|S_ref| <= 1e-2
+  whole layer (fused kernel with decay-weighted W, then scan) against the token-by-token recurrence: <= 2e-2.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_21325_b200 import workloads as wl
+from parity_util import max_ratio
+
+pytestmark = pytest.mark.gpu
+
+TOL_SCAN, TOL_LAYER = 1e-2, 2e-2
+
+
+@pytest.fixture(scope="module")
+def bnd():
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2605_21325_b200 import binding
+    torch.cuda.set_device(0)
+    return binding
+
+
+def to_bf16_bits(x64):
+    return wl._store(x64.astype(np.float32), wl.BF16)
+
+
+def exact_wu(inp, cu_seqlens):
+    """The oracle's decay-weighted W and U, rounded once to bf16 storage."""
+    A = oracle.build_A(inp.K, inp.beta, inp.g, inp.C, cu_seqlens=cu_seqlens)
+    Kd = oracle._widen(inp.K) * np.exp(inp.g.astype(np.float64))[..., None]
+    W, _ = oracle.wy(A, Kd, None, inp.beta, inp.C, cu_seqlens=cu_seqlens)
+    _, U = oracle.wy(A, inp.K, inp.V, inp.beta, inp.C, cu_seqlens=cu_seqlens)
+    return to_bf16_bits(W), to_bf16_bits(U)
+
+
+CASES = [
+    ("dense", 2, 5 * 64, 3, None, False),
+    ("dense_partial_s0", 1, 3 * 64 + 17, 2, None, True),
+    ("ragged_s0", 1, 0, 2, np.array([0, 64, 65, 65, 300, 531], np.int32), True),
+    ("many_heads_wide_slices", 5, 2 * 64, 64, None, True),   # 320 (sequence, head) pairs: the 64-column variant
+]
+
+
+@pytest.mark.parametrize("name,B,T,H,cu,with_s0", CASES, ids=[c[0] for c in CASES])
+def test_chunk_scan_matches_its_definition(bnd, name, B, T, H, cu, with_s0):
+    if cu is not None:
+        T = int(cu[-1])
+    inp = wl.make(name, B, T, H, 128, 128, 64, wl.BF16, seed=300 + H, cu_seqlens=cu)
+    Q = wl.queries(inp, seed=301)
+    S0 = wl.initial_state(inp, seed=302) if with_s0 else None
+    Wb, Ub = exact_wu(inp, cu)
+    scale = 128 ** -0.5
+    O_ref, S_ref = oracle.chunk_scan(Q, inp.K, Wb, Ub, inp.g, 64, scale=scale, S0=S0, cu_seqlens=cu)
+    dev = bnd.to_device(inp)
+    Qd, Wd, Ud = (bnd.kv_to_torch(x) for x in (Q, Wb, Ub))
+    S0d = None if S0 is None else torch.from_numpy(S0).cuda()
+    O = torch.full((B, T, H, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    O, S = bnd.chunk_scan(Qd, dev["K"], Wd, Ud, dev["g"], 64, scale=scale, S0=S0d, cu_seqlens=cu, out=O)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    o, s = bnd.to_numpy_f64(O), bnd.to_numpy_f64(S)
+    assert not np.isnan(o).any(), "a row of O was not written"
+    assert max_ratio(o, O_ref) <= TOL_SCAN
+    assert max_ratio(s, S_ref) <= TOL_SCAN
+    # the same inputs through the recurrence itself: the scan is the layer
+    O_rec, S_rec = oracle.gdn_recurrence(Q, inp.K, inp.V, inp.beta, inp.g, 64, scale=scale, S0=S0, cu_seqlens=cu)
+    assert max_ratio(o, O_rec) <= TOL_LAYER and max_ratio(s, S_rec) <= TOL_LAYER
+
+
+def test_layer_forward_two_launches_against_the_recurrence(bnd):
+    cu = np.array([0, 200, 264, 777], np.int32)
+    for cu_seqlens, B, T in ((None, 2, 6 * 64), (cu, 1, 777)):
+        inp = wl.make("layer", B, T, 4, 128, 128, 64, wl.BF16, seed=310, cu_seqlens=cu_seqlens)
+        Q = wl.queries(inp, seed=311)
+        S0 = wl.initial_state(inp, seed=312)
+        O_ref, S_ref = oracle.gdn_recurrence(Q, inp.K, inp.V, inp.beta, inp.g, 64, scale=0.125, S0=S0, cu_seqlens=cu_seqlens)
+        dev = bnd.to_device(inp)
+        O, S = bnd.gdn_forward(bnd.kv_to_torch(Q), dev["K"], dev["V"], dev["beta"], dev["g"], 64, scale=0.125,
+                               S0=torch.from_numpy(S0).cuda(), cu_seqlens=cu_seqlens)
+        torch.cuda.synchronize()
+        assert bnd.last_device_status() == 0
+        assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= TOL_LAYER
+        assert max_ratio(bnd.to_numpy_f64(S), S_ref) <= TOL_LAYER
+
+
+def test_chunk_scan_edge_cases(bnd):
+    # an empty sequence keeps its initial state; unsupported shapes are refused, not approximated
+    cu = np.array([0, 0, 70], np.int32)
+    inp = wl.make("edge", 1, 70, 1, 128, 128, 64, wl.BF16, seed=320, cu_seqlens=cu)
+    Q = wl.queries(inp, seed=321)
+    S0 = wl.initial_state(inp, seed=322)
+    Wb, Ub = exact_wu(inp, cu)
+    dev = bnd.to_device(inp)
+    O, S = bnd.chunk_scan(bnd.kv_to_torch(Q), dev["K"], bnd.kv_to_torch(Wb), bnd.kv_to_torch(Ub), dev["g"], 64,
+                          S0=torch.from_numpy(S0).cuda(), cu_seqlens=cu)
+    torch.cuda.synchronize()
+    assert np.array_equal(S[0].cpu().numpy(), S0[0])
+    _, S_ref = oracle.chunk_scan(Q, inp.K, Wb, Ub, inp.g, 64, S0=S0, cu_seqlens=cu)
+    assert max_ratio(bnd.to_numpy_f64(S), S_ref) <= TOL_SCAN
+    small = wl.make("small", 1, 64, 1, 64, 64, 64, wl.BF16, seed=323)
+    d = bnd.to_device(small)
+    with pytest.raises(bnd.TriInvError):
+        bnd.chunk_scan(d["K"], d["K"], d["K"], d["V"], d["g"], 64)
