@@ -44,6 +44,11 @@ def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True, call="fused"):
     build: K, beta, g read; A written.  wy: the strict lower triangle of A, K, V, beta read; W, U written."""
     if call == "build":
         return C * d_k * elt + 2 * C * 4 + C * C * 4
+    if call == "scan":  # Q, K, W, U, g read; O written
+        return 3 * C * d_k * elt + C * d_v * elt + C * 4 + C * d_v * elt
+    if call == "layer":  # fused kernel (K, V, beta, g in; W, U out, A not stored) + scan
+        return (C * d_k * elt + C * d_v * elt + 2 * C * 4 + C * d_k * elt + C * d_v * elt) + \
+               (3 * C * d_k * elt + C * d_v * elt + C * 4 + C * d_v * elt)
     if call == "kda":  # K, G (fp32 per channel) and beta read; A written
         return C * d_k * elt + C * d_k * 4 + C * 4 + C * C * 4
     if call == "wy":
@@ -194,7 +199,7 @@ def main():
     ap.add_argument("--method", default="block_recursive", choices=["block_recursive", "mixed_recursion", "product_series"])
     ap.add_argument("--paper-T", type=int, default=0,
                     help="instead of --config: the paper's timing shape B=32, H=4, d=128 at this sequence length (1024..16384)")
-    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw", "kda"],
+    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw", "kda", "scan", "layer"],
                     help="entry point timed: the fused path (default, the metric), tri_inv_build alone, tri_inv_wy alone, or "
                          "tri_inv_fused_raw (front end folded in; same shapes, un-normalised keys and logits as inputs)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -245,6 +250,12 @@ def main():
     A = torch.empty((inp.B, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda")
     W, U = torch.empty_like(K), torch.empty_like(V)
     G = torch.from_numpy(wl.per_channel_gate(inp, seed=3000 + args.config)).cuda() if args.call == "kda" else None
+    Q = O = None
+    if args.call in ("scan", "layer"):  # the consumer of W and U: queries, outputs, zero initial state
+        Q_host = wl.queries(inp, seed=4000 + args.config)
+        Q = binding.kv_to_torch(Q_host)
+        O = torch.empty_like(V)
+        q_scale = float(inp.d_k) ** -0.5
     flush = None if args.no_flush else torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
     flush_rd = None if args.no_flush else torch.zeros(64 * 1024 * 1024, dtype=torch.float32, device="cuda")
     stream = torch.cuda.current_stream()
@@ -263,11 +274,18 @@ def main():
             binding.fused_raw(K, V, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U, None, None), stream=stream)
         elif args.call == "build":
             binding.build(K, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
+        elif args.call == "scan":
+            binding.chunk_scan(Q, K, W, U, g, inp.C, scale=q_scale, cu_seqlens=inp.cu_seqlens, out=O, want_state=False, stream=stream)
+        elif args.call == "layer":
+            binding.fused(K, V, beta, g, inp.C, method=method | binding.W_DECAY, cu_seqlens=inp.cu_seqlens, out=(None, W, U), stream=stream)
+            binding.chunk_scan(Q, K, W, U, g, inp.C, scale=q_scale, cu_seqlens=inp.cu_seqlens, out=O, want_state=False, stream=stream)
         elif args.call == "kda":
             binding.build_kda(K, G, beta, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
         else:
             binding.wy(A, K, V, beta, cu_seqlens=inp.cu_seqlens, out=(W, U), stream=stream)
 
+    if args.call == "scan":  # the scan reads stored W (decay-weighted) and U: produce them once, outside the timed region
+        binding.fused(K, V, beta, g, inp.C, method=method | binding.W_DECAY, cu_seqlens=inp.cu_seqlens, out=(None, W, U), stream=stream)
     if args.call == "wy":  # tri_inv_wy reads a stored A: produce it once, outside the timed region
         binding.build(K, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
 
@@ -371,7 +389,13 @@ def main():
             A_k = oracle.build_A_kda(inp.K[:, :Ts] if Ts else inp.K, Gs[:, :Ts] if Ts else Gs, inp.beta[:, :Ts] if Ts else inp.beta,
                                      inp.C, cu_seqlens=None if Ts else inp.cu_seqlens)
             err["A_max_ratio"] = float(np.abs(a - A_k).max() / np.abs(A_k).max())
-        if args.call not in ("build", "kda"):
+        if args.call in ("scan", "layer"):
+            sl = slice(0, Ts) if Ts else slice(None)
+            O_ref, _ = oracle.gdn_recurrence(Q_host[:, sl], inp.K[:, sl], inp.V[:, sl], inp.beta[:, sl], inp.g[:, sl], inp.C,
+                                             scale=q_scale, cu_seqlens=None if Ts else inp.cu_seqlens)
+            err = {"sample": err["sample"], "reference": "token-by-token recurrence",
+                   "O_max_ratio": float(np.abs(binding.to_numpy_f64(O[:, sl]) - O_ref).max() / np.abs(O_ref).max())}
+        elif args.call not in ("build", "kda"):
             err["W_max_ratio"] = float(np.abs(w - W_ref).max() / np.abs(W_ref).max())
             err["U_max_ratio"] = float(np.abs(u - U_ref).max() / np.abs(U_ref).max())
 
@@ -384,7 +408,7 @@ def main():
         traffic = NCU_TRAFFIC_BYTES_PER_MATRIX.get((args.config, args.method)) if args.call == "fused" else None
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": None if traffic is None else traffic * n_mat, "peak_source": "of " + peak_kind,
-                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "kda": "per-channel-decay build+invert", "wy": "WY apply"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
+                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "kda": "per-channel-decay build+invert", "wy": "WY apply", "scan": "chunk scan (state recurrence + output)", "layer": "fused build+invert+WY, then chunk scan (2 launches)"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
                     "algorithmic_bytes_per_launch": alg_bytes * n_mat}
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
@@ -394,7 +418,7 @@ def main():
                "dtype": "bf16" if inp.kv_dtype == wl.BF16 else "f32", "data": "synthetic",
                "config": {"workload": inp.name, "B": inp.B, "T": inp.T, "H": inp.H, "d_k": inp.d_k, "d_v": inp.d_v, "C": inp.C,
                           "chunk_matrices_per_gpu": n_mat, "method": args.method, "call": args.call,
-                          "outputs": {"fused": "A fp32 + W,U", "raw": "A fp32 + W,U", "build": "A fp32", "kda": "A fp32", "wy": "W,U"}[args.call],
+                          "outputs": {"fused": "A fp32 + W,U", "raw": "A fp32 + W,U", "build": "A fp32", "kda": "A fp32", "wy": "W,U", "scan": "O", "layer": "O"}[args.call],
                           "l2": "flushed before every timed step (256 MiB write, then a 256 MiB read so no dirty lines remain)" if flush is not None else "not flushed",
                           "parallelism": "independent replicas, no collective" if world > 1 else "single GPU"},
                "gb_per_s": achieved, "roofline": roofline, "cpu_baseline": cpu,

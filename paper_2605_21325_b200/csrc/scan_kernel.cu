@@ -21,6 +21,21 @@
 namespace tri_inv {
 namespace {
 
+#ifdef TRI_INV_PHASE_CLOCKS
+#define PHASE_BEGIN() long long ph_t = clock64()
+#define PHASE(k)                                                                  \
+  do {                                                                            \
+    long long now = clock64();                                                    \
+    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(p.status + 8 + 12 * (threadIdx.x >> 5) + (k), (int)(now - ph_t)); \
+    ph_t = now;                                                                   \
+  } while (0)
+#define SUBPHASE(k) do { long long now = clock64(); atomicAdd(p.status + 64 + (k), (int)(now - sub_t)); sub_t = now; } while (0)
+#else
+#define PHASE_BEGIN() do {} while (0)
+#define PHASE(k) do {} while (0)
+#define SUBPHASE(k) do {} while (0)
+#endif
+
 constexpr int C = 64, D = 128, NT = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -33,8 +48,8 @@ struct ScanCfg {
   static constexpr int OFF_UD = OFF_UT + DVS * 128;               // U~'^T bf16 (rows scaled by gamma_last / gamma_i)
   static constexpr int OFF_P = OFF_UD + DVS * 128;                // P bf16 [64][64]
   static constexpr int OFF_G = OFF_P + 8192;                      // g * log2(e): two buffers of 64 floats
-  static constexpr int OFF_BAR = OFF_G + 512;                     // 7 mbarriers, tensor-memory slot
-  static constexpr int SMEM = OFF_BAR + 64;
+  static constexpr int OFF_BAR = OFF_G + 512;                     // 10 mbarriers, tensor-memory slot
+  static constexpr int SMEM = OFF_BAR + 96;
   static constexpr int TM_QK = 0, TM_T1 = 64, TM_QS = 64 + DVS, TM_PU = 64 + 2 * DVS, TM_DS = 64 + 3 * DVS;
   static constexpr int TMEM_COLS = (64 + 4 * DVS) <= 256 ? 256 : 512;
   static constexpr int CTAS_PER_SM = TMEM_COLS == 256 ? 2 : 1;
@@ -68,23 +83,32 @@ __device__ __forceinline__ void tmem_ld_32x32(float* r, uint32_t taddr) {
       : "r"(taddr));
 }
 
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 template <int DVS>
-__global__ void __launch_bounds__(NT, ScanCfg<DVS>::CTAS_PER_SM)
+__global__ void __launch_bounds__(NT + 32, ScanCfg<DVS>::CTAS_PER_SM)
 chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmQ,
                   const __grid_constant__ CUtensorMap tmK, ScanParams p) {
   using cfg = ScanCfg<DVS>;
   constexpr int NTL = cfg::NTL, NS = D / DVS;
   extern __shared__ __align__(1024) uint8_t smem[];
   float* sG = reinterpret_cast<float*>(smem + cfg::OFF_G);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 56);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 88);
   const uint32_t sW = smem_u32(smem + cfg::OFF_W), sQ = smem_u32(smem + cfg::OFF_Q), sK = smem_u32(smem + cfg::OFF_K);
   const uint32_t sS = smem_u32(smem + cfg::OFF_S), sUt = smem_u32(smem + cfg::OFF_UT), sUd = smem_u32(smem + cfg::OFF_UD);
   const uint32_t sP = smem_u32(smem + cfg::OFF_P);
+  // copies (TMA):            bar_w, bar_q, bar_k
+  // products done (commit):  bar_t1 (W S), bar_o (Q S, Q K^T), bar_s (K^T U~'), bar_pu (P U~)
+  // operands written (128 arrivals of the compute threads): bar_sr (S^T), bar_ut (U~^T, U~'^T), bar_p (P)
   const uint32_t bar_w = smem_u32(smem + cfg::OFF_BAR), bar_q = bar_w + 8, bar_k = bar_w + 16, bar_t1 = bar_w + 24,
-                 bar_o = bar_w + 32, bar_s = bar_w + 40, bar_pu = bar_w + 48;
+                 bar_o = bar_w + 32, bar_s = bar_w + 40, bar_pu = bar_w + 48, bar_sr = bar_w + 56, bar_ut = bar_w + 64,
+                 bar_p = bar_w + 72;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool control = warp == 4;               // warp 4: one thread issues every product; warps 0..3 compute
   const int gq = lane >> 2, t = lane & 3;
-  const int ra = 16 * warp + gq, rb = ra + 8;   // this thread's two rows of every M = 64 accumulator
+  const int ra = 16 * (warp & 3) + gq, rb = ra + 8;   // this thread's two rows of every M = 64 accumulator
 
   const int slice = blockIdx.x % NS, h = (blockIdx.x / NS) % p.H, s = blockIdx.x / (NS * p.H);
   const int beg = p.seq_off ? p.seq_off[s] : s * p.T;
@@ -92,9 +116,9 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   const int n_chunks = (end - beg + C - 1) / C;
   const int col0 = slice * DVS;                  // first value column of this CTA
 
-  // state: thread tid owns row tid (a key feature) of S, DVS columns
+  // state: compute thread tid owns row tid (a key feature) of S, DVS columns
   float S[DVS];
-  {
+  if (!control) {
     const float* s0 = p.S0 ? p.S0 + (((size_t)s * p.H + h) * D + tid) * D + col0 : nullptr;
 #pragma unroll
     for (int n = 0; n < DVS; n += 4) {
@@ -103,7 +127,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     }
   }
   auto store_state = [&]() {
-    if (!p.S_out) return;
+    if (!p.S_out || control) return;
     float* dst = p.S_out + (((size_t)s * p.H + h) * D + tid) * D + col0;
 #pragma unroll
     for (int n = 0; n < DVS; n += 4) *reinterpret_cast<float4*>(dst + n) = make_float4(S[n], S[n + 1], S[n + 2], S[n + 3]);
@@ -140,12 +164,13 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   };
 
   uint32_t u_next[NTL][2];
-  float g_next;
+  float g_next = 0.f;
   {
     const int rows0 = end - beg < C ? end - beg : C;
-    if (tid == 0) {
+    if (tid == NT) {
       prefetch_tmap(&tmW); prefetch_tmap(&tmQ); prefetch_tmap(&tmK);
       for (int b = 0; b < 7; ++b) mbar_init(bar_w + 8 * b, 1);
+      for (int b = 7; b < 10; ++b) mbar_init(bar_w + 8 * b, NT);
       fence_mbar_init();
       if (!misaligned) {
         issue_tile(sW, &tmW, bar_w, beg);
@@ -153,183 +178,206 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         issue_tile(sK, &tmK, bar_k, beg);
       }
     }
-    fetch_u(u_next, beg, rows0);
-    g_next = fetch_g(beg, rows0);
+    if (!control) {
+      fetch_u(u_next, beg, rows0);
+      g_next = fetch_g(beg, rows0);
+    }
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(cfg::TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  write_state_operand();
-  if (tid < C) sG[tid] = g_next;
+  if (!control) {
+    write_state_operand();
+    if (tid < C) sG[tid] = g_next;
+  }
   fence_proxy_async();
   tc_fence_before();
-  __syncthreads();
+  __syncthreads();   // barriers initialised, tensor memory allocated, first operand of S and first g in place
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_rows = tmem + ((uint32_t)(32 * warp) << 16);
-
-  constexpr uint32_t idesc_n = umma_idesc(C, DVS, 0), idesc_qk = umma_idesc(C, C, 0), idesc_ds = umma_idesc_amn(D, DVS);
-  auto mma_k128 = [&](uint32_t d_tmem, uint32_t a_base, uint32_t b_base, uint32_t b_box, uint32_t idesc) {
-#pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks) {
-      const uint64_t da = umma_desc(a_base + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024);
-      const uint64_t db = umma_desc(b_base + (ks >> 2) * b_box + (ks & 3) * 32, 16, 1024);
-      umma_bf16(d_tmem, da, db, idesc, ks > 0);
-    }
-  };
-
-  uint32_t ph = 0;
+  const uint32_t tmem_rows = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
   bool failed = misaligned;
-  for (int c = 0; c < n_chunks && !misaligned; ++c) {
-    const int tok0 = beg + c * C;
-    const int rows = end - tok0 < C ? end - tok0 : C;
-    const bool has_next = c + 1 < n_chunks;
-    const int nx_tok0 = tok0 + C, nx_rows = end - nx_tok0 < C ? end - nx_tok0 : C;
-    const float* gb = sG + (c & 1) * C;
 
-    // ---- A. products that need only S and the tiles
-    if (tid == 0) {
-      if (!mbar_wait_bounded(bar_w, ph)) {
-        atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);   // the other threads time out on bar_t1
-      } else {
+  if (control) {
+    // ---------------------------------------------------------------- control thread: every tcgen05.mma of the CTA
+    if (lane == 0 && !misaligned) {
+      constexpr uint32_t idesc_n = umma_idesc(C, DVS, 0), idesc_qk = umma_idesc(C, C, 0), idesc_ds = umma_idesc_amn(D, DVS);
+      // descriptors differ from these bases only in the address field (bits 0..13, units of 16 bytes)
+      const uint64_t dW = umma_desc(sW, 16, 1024), dQ = umma_desc(sQ, 16, 1024), dK = umma_desc(sK, 16, 1024),
+                     dS = umma_desc(sS, 16, 1024), dKt = umma_desc(sK, 8192, 1024), dUd = umma_desc(sUd, 16, 1024),
+                     dP = umma_desc(sP, 16, 1024), dUt = umma_desc(sUt, 16, 1024);
+      auto mma_k128 = [&](uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t b_box, uint32_t idesc) {
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          umma_bf16(d_tmem, a + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), b + (((ks >> 2) * b_box + (ks & 3) * 32) >> 4), idesc, ks > 0);
+      };
+      uint32_t ph = 0;
+      for (int c = 0; c < n_chunks; ++c) {
+        // T1 = W S: the head of the chunk's dependent chain, issued first
+        if (!mbar_wait_bounded(bar_sr, ph) || !mbar_wait_bounded(bar_w, ph)) { failed = true; break; }
         tc_fence_after();
-        mma_k128(tmem + cfg::TM_T1, sW, sS, cfg::S_BOX, idesc_n);
+        mma_k128(tmem + cfg::TM_T1, dW, dS, cfg::S_BOX, idesc_n);
         umma_commit(bar_t1);
-        if (!mbar_wait_bounded(bar_q, ph) || !mbar_wait_bounded(bar_k, ph)) {
-          atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
-        } else {
-          tc_fence_after();
-          mma_k128(tmem + cfg::TM_QS, sQ, sS, cfg::S_BOX, idesc_n);
-          mma_k128(tmem + cfg::TM_QK, sQ, sK, 8192, idesc_qk);
-          umma_commit(bar_o);
-        }
+        if (!mbar_wait_bounded(bar_q, ph) || !mbar_wait_bounded(bar_k, ph)) { failed = true; break; }
+        tc_fence_after();
+        mma_k128(tmem + cfg::TM_QK, dQ, dK, 8192, idesc_qk);
+        mma_k128(tmem + cfg::TM_QS, dQ, dS, cfg::S_BOX, idesc_n);
+        umma_commit(bar_o);
+        // dS = K^T U~' as soon as the compute threads have written U~'
+        if (!mbar_wait_bounded(bar_ut, ph)) { failed = true; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < C / 16; ++ks)   // K tile read MN-major: 16 tokens (2048 bytes) per step
+          umma_bf16(tmem + cfg::TM_DS, dKt + ((ks * 2048) >> 4), dUd + ((ks * 32) >> 4), idesc_ds, ks > 0);
+        umma_commit(bar_s);
+        if (!mbar_wait_bounded(bar_p, ph)) { failed = true; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < C / 16; ++ks)
+          umma_bf16(tmem + cfg::TM_PU, dP + ((ks * 32) >> 4), dUt + ((ks * 32) >> 4), idesc_n, ks > 0);
+        umma_commit(bar_pu);
+        ph ^= 1;
       }
     }
-    uint32_t u_cur[NTL][2];
-#pragma unroll
-    for (int nt = 0; nt < NTL; ++nt) { u_cur[nt][0] = u_next[nt][0]; u_cur[nt][1] = u_next[nt][1]; }
-    if (has_next) {
-      fetch_u(u_next, nx_tok0, nx_rows);
-      g_next = fetch_g(nx_tok0, nx_rows);
-    }
-    const float g_a = gb[ra], g_b = gb[rb], g_last = gb[rows - 1];
-
-    // ---- B. U~ = U - W S  ->  bf16 operands U~^T and (decay-scaled) U~'^T
-    if (!mbar_wait_bounded(bar_t1, ph)) { failed = true; break; }
-    tc_fence_after();
-    if (tid == 32 && has_next) issue_tile(sW, &tmW, bar_w, nx_tok0);   // W's only reader has retired
-    {
-      float t1[NTL][4];
-      tmem_ld_frag<NTL>(t1, tmem_rows + cfg::TM_T1);
-      tmem_wait_ld();
-      const float da = ex2_approx(g_last - g_a), db = ex2_approx(g_last - g_b);
-      const int ca = ra >> 3, cb = rb >> 3;
-#pragma unroll
-      for (int nt = 0; nt < NTL; ++nt) {
-        const float2 ua = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u_cur[nt][0]));
-        const float2 ub = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u_cur[nt][1]));
-        const float v0 = ra < rows ? ua.x - t1[nt][0] : 0.f, v1 = ra < rows ? ua.y - t1[nt][1] : 0.f;
-        const float v2 = rb < rows ? ub.x - t1[nt][2] : 0.f, v3 = rb < rows ? ub.y - t1[nt][3] : 0.f;
-        const int n0 = 8 * nt + 2 * t, n1 = n0 + 1;
-        // element (n, token) of a [DVS rows][64 tokens] bf16 tile, 128-byte rows, 16-byte pieces swizzled by the row
-        const uint32_t o0a = n0 * 128 + ((ca ^ (n0 & 7)) << 4) + (ra & 7) * 2, o1a = n1 * 128 + ((ca ^ (n1 & 7)) << 4) + (ra & 7) * 2;
-        const uint32_t o0b = n0 * 128 + ((cb ^ (n0 & 7)) << 4) + (rb & 7) * 2, o1b = n1 * 128 + ((cb ^ (n1 & 7)) << 4) + (rb & 7) * 2;
-        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o0a) = __float2bfloat16_rn(v0);
-        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o1a) = __float2bfloat16_rn(v1);
-        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o0b) = __float2bfloat16_rn(v2);
-        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o1b) = __float2bfloat16_rn(v3);
-        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o0a) = __float2bfloat16_rn(v0 * da);
-        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o1a) = __float2bfloat16_rn(v1 * da);
-        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o0b) = __float2bfloat16_rn(v2 * db);
-        *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o1b) = __float2bfloat16_rn(v3 * db);
-      }
-    }
-    // ---- P = (Q K^T) * decay, lower triangle with its diagonal; QS kept in registers for the output
-    if (!mbar_wait_bounded(bar_o, ph)) { failed = true; break; }
-    tc_fence_after();
-    if (tid == 64 && has_next) issue_tile(sQ, &tmQ, bar_q, nx_tok0);   // Q's readers have retired
-    float qs[NTL][4];
-    {
-      float qk[8][4];
-      tmem_ld_16x64(qk, tmem_rows + cfg::TM_QK);
-      tmem_ld_frag<NTL>(qs, tmem_rows + cfg::TM_QS);
-      tmem_wait_ld();
-#pragma unroll
-      for (int nt = 0; nt < 8; ++nt) {
-        const int j = 8 * nt + 2 * t;
-        const float2 gj = *reinterpret_cast<const float2*>(gb + j);
-        const float p0 = j <= ra ? qk[nt][0] * ex2_approx(g_a - gj.x) : 0.f, p1 = j + 1 <= ra ? qk[nt][1] * ex2_approx(g_a - gj.y) : 0.f;
-        const float p2 = j <= rb ? qk[nt][2] * ex2_approx(g_b - gj.x) : 0.f, p3 = j + 1 <= rb ? qk[nt][3] * ex2_approx(g_b - gj.y) : 0.f;
-        *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + ra * 128 + ((nt ^ (ra & 7)) << 4) + 4 * t) = pack_bf16(p0, p1);
-        *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + rb * 128 + ((nt ^ (rb & 7)) << 4) + 4 * t) = pack_bf16(p2, p3);
-      }
-    }
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-
-    // ---- C. dS = K^T U~'  and  PU = P U~
-    if (tid == 0) {
+  } else {
+    // ---------------------------------------------------------------- compute warps
+    mbar_arrive(bar_sr);   // the first S^T operand (written before the CTA barrier above)
+    uint32_t ph = 0;
+    float qs[NTL][4];      // Q S of the chunk whose output is still to be written
+    float o_sa = 0.f, o_sb = 0.f;
+    int o_tok0 = 0, o_rows = 0;
+    // O = scale * (gamma_i QS + PU) of the previous chunk: written while the next chunk's first product runs
+    auto write_output = [&](uint32_t parity) -> bool {
+      if (!mbar_wait_bounded(bar_pu, parity)) return false;
       tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < C / 16; ++ks) {
-        const uint64_t da = umma_desc(sK + ks * 2048, 8192, 1024);   // K tile read MN-major: 16 tokens per step
-        const uint64_t db = umma_desc(sUd + ks * 32, 16, 1024);
-        umma_bf16(tmem + cfg::TM_DS, da, db, idesc_ds, ks > 0);
-      }
-      umma_commit(bar_s);
-#pragma unroll
-      for (int ks = 0; ks < C / 16; ++ks) {
-        const uint64_t da = umma_desc(sP + ks * 32, 16, 1024);
-        const uint64_t db = umma_desc(sUt + ks * 32, 16, 1024);
-        umma_bf16(tmem + cfg::TM_PU, da, db, idesc_n, ks > 0);
-      }
-      umma_commit(bar_pu);
-    }
-    if (tid < C && has_next) sG[((c + 1) & 1) * C + tid] = g_next;
-
-    // ---- D. state update (thread = row of S) and the bf16 operand for the next chunk
-    if (!mbar_wait_bounded(bar_s, ph)) { failed = true; break; }
-    tc_fence_after();
-    if (tid == 96 && has_next) issue_tile(sK, &tmK, bar_k, nx_tok0);   // K's readers have retired
-    {
-      const float gl = ex2_approx(g_last);
-#pragma unroll
-      for (int n0 = 0; n0 < DVS; n0 += 32) {
-        float ds[32];
-        tmem_ld_32x32(ds, tmem_rows + cfg::TM_DS + n0);
-        tmem_wait_ld();
-#pragma unroll
-        for (int n = 0; n < 32; ++n) S[n0 + n] = fmaf(gl, S[n0 + n], ds[n]);
-      }
-      if (has_next) write_state_operand();
-    }
-    // ---- E. O = scale * (gamma_i QS + PU)
-    if (!mbar_wait_bounded(bar_pu, ph)) { failed = true; break; }
-    tc_fence_after();
-    {
       float pu[NTL][4];
       tmem_ld_frag<NTL>(pu, tmem_rows + cfg::TM_PU);
       tmem_wait_ld();
-      const float sa = p.scale * ex2_approx(g_a), sb = p.scale * ex2_approx(g_b);
       __nv_bfloat16* Og = reinterpret_cast<__nv_bfloat16*>(p.O);
 #pragma unroll
       for (int nt = 0; nt < NTL; ++nt) {
         const int cc = col0 + 8 * nt + 2 * t;
-        if (ra < rows)
-          *reinterpret_cast<uint32_t*>(Og + ((size_t)(tok0 + ra) * p.H + h) * D + cc) =
-              pack_bf16(fmaf(sa, qs[nt][0], p.scale * pu[nt][0]), fmaf(sa, qs[nt][1], p.scale * pu[nt][1]));
-        if (rb < rows)
-          *reinterpret_cast<uint32_t*>(Og + ((size_t)(tok0 + rb) * p.H + h) * D + cc) =
-              pack_bf16(fmaf(sb, qs[nt][2], p.scale * pu[nt][2]), fmaf(sb, qs[nt][3], p.scale * pu[nt][3]));
+        if (ra < o_rows)
+          *reinterpret_cast<uint32_t*>(Og + ((size_t)(o_tok0 + ra) * p.H + h) * D + cc) =
+              pack_bf16(fmaf(o_sa, qs[nt][0], p.scale * pu[nt][0]), fmaf(o_sa, qs[nt][1], p.scale * pu[nt][1]));
+        if (rb < o_rows)
+          *reinterpret_cast<uint32_t*>(Og + ((size_t)(o_tok0 + rb) * p.H + h) * D + cc) =
+              pack_bf16(fmaf(o_sb, qs[nt][2], p.scale * pu[nt][2]), fmaf(o_sb, qs[nt][3], p.scale * pu[nt][3]));
       }
+      tc_fence_before();
+      return true;
+    };
+    for (int c = 0; c < n_chunks && !misaligned; ++c) {
+      const int tok0 = beg + c * C;
+      const int rows = end - tok0 < C ? end - tok0 : C;
+      const bool has_next = c + 1 < n_chunks;
+      const int nx_tok0 = tok0 + C, nx_rows = end - nx_tok0 < C ? end - nx_tok0 : C;
+      const float* gb = sG + (c & 1) * C;
+      PHASE_BEGIN();
+      uint32_t u_cur[NTL][2];
+#pragma unroll
+      for (int nt = 0; nt < NTL; ++nt) { u_cur[nt][0] = u_next[nt][0]; u_cur[nt][1] = u_next[nt][1]; }
+      if (has_next) {
+        fetch_u(u_next, nx_tok0, nx_rows);
+        g_next = fetch_g(nx_tok0, nx_rows);
+      }
+      if (c > 0 && !write_output(ph ^ 1)) { failed = true; break; }
+      PHASE(0);
+
+      // ---- U~ = U - W S  ->  bf16 operands U~^T and (decay-scaled) U~'^T
+      if (!mbar_wait_bounded(bar_t1, ph)) { failed = true; break; }
+      tc_fence_after();
+      PHASE(1);
+      // (this chunk's g was written by other threads during the last chunk: read only after the wait above,
+      // which follows every compute thread's arrival on bar_sr)
+      const float g_a = gb[ra], g_b = gb[rb], g_last = gb[rows - 1];
+      if (tid == 32 && has_next) issue_tile(sW, &tmW, bar_w, nx_tok0);   // W's only reader has retired
+      {
+        float t1[NTL][4];
+        tmem_ld_frag<NTL>(t1, tmem_rows + cfg::TM_T1);
+        tmem_wait_ld();
+        const float da = ex2_approx(g_last - g_a), db = ex2_approx(g_last - g_b);
+        const int ca = ra >> 3, cb = rb >> 3;
+#pragma unroll
+        for (int nt = 0; nt < NTL; ++nt) {
+          const float2 ua = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u_cur[nt][0]));
+          const float2 ub = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u_cur[nt][1]));
+          const float v0 = ra < rows ? ua.x - t1[nt][0] : 0.f, v1 = ra < rows ? ua.y - t1[nt][1] : 0.f;
+          const float v2 = rb < rows ? ub.x - t1[nt][2] : 0.f, v3 = rb < rows ? ub.y - t1[nt][3] : 0.f;
+          const int n0 = 8 * nt + 2 * t, n1 = n0 + 1;
+          // element (n, token) of a [DVS rows][64 tokens] bf16 tile, 128-byte rows, 16-byte pieces swizzled by the row
+          const uint32_t o0a = n0 * 128 + ((ca ^ (n0 & 7)) << 4) + (ra & 7) * 2, o1a = n1 * 128 + ((ca ^ (n1 & 7)) << 4) + (ra & 7) * 2;
+          const uint32_t o0b = n0 * 128 + ((cb ^ (n0 & 7)) << 4) + (rb & 7) * 2, o1b = n1 * 128 + ((cb ^ (n1 & 7)) << 4) + (rb & 7) * 2;
+          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o0a) = __float2bfloat16_rn(v0 * da);
+          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o1a) = __float2bfloat16_rn(v1 * da);
+          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o0b) = __float2bfloat16_rn(v2 * db);
+          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o1b) = __float2bfloat16_rn(v3 * db);
+          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o0a) = __float2bfloat16_rn(v0);
+          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o1a) = __float2bfloat16_rn(v1);
+          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o0b) = __float2bfloat16_rn(v2);
+          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o1b) = __float2bfloat16_rn(v3);
+        }
+      }
+      fence_proxy_async();
+      tc_fence_before();
+      mbar_arrive(bar_ut);
+      PHASE(2);
+
+      // ---- P = (Q K^T) * decay, lower triangle with its diagonal (while K^T U~' runs); QS kept for the output
+      if (!mbar_wait_bounded(bar_o, ph)) { failed = true; break; }
+      tc_fence_after();
+      PHASE(3);
+      if (tid == 64 && has_next) issue_tile(sQ, &tmQ, bar_q, nx_tok0);   // Q's readers have retired
+      {
+        float qk[8][4];
+        tmem_ld_16x64(qk, tmem_rows + cfg::TM_QK);
+        tmem_ld_frag<NTL>(qs, tmem_rows + cfg::TM_QS);
+        tmem_wait_ld();
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+          const int j = 8 * nt + 2 * t;
+          const float2 gj = *reinterpret_cast<const float2*>(gb + j);
+          const float p0 = j <= ra ? qk[nt][0] * ex2_approx(g_a - gj.x) : 0.f, p1 = j + 1 <= ra ? qk[nt][1] * ex2_approx(g_a - gj.y) : 0.f;
+          const float p2 = j <= rb ? qk[nt][2] * ex2_approx(g_b - gj.x) : 0.f, p3 = j + 1 <= rb ? qk[nt][3] * ex2_approx(g_b - gj.y) : 0.f;
+          *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + ra * 128 + ((nt ^ (ra & 7)) << 4) + 4 * t) = pack_bf16(p0, p1);
+          *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + rb * 128 + ((nt ^ (rb & 7)) << 4) + 4 * t) = pack_bf16(p2, p3);
+        }
+      }
+      fence_proxy_async();
+      tc_fence_before();
+      mbar_arrive(bar_p);
+      o_sa = p.scale * ex2_approx(g_a); o_sb = p.scale * ex2_approx(g_b);
+      o_tok0 = tok0; o_rows = rows;
+      if (tid < C && has_next) sG[((c + 1) & 1) * C + tid] = g_next;
+      PHASE(4);
+
+      // ---- state update (thread = row of S) and the bf16 operand for the next chunk
+      if (!mbar_wait_bounded(bar_s, ph)) { failed = true; break; }
+      tc_fence_after();
+      PHASE(5);
+      if (tid == 96 && has_next) issue_tile(sK, &tmK, bar_k, nx_tok0);   // K's readers (Q K^T, K^T U~') have retired
+      {
+        const float gl = ex2_approx(g_last);
+#pragma unroll
+        for (int n0 = 0; n0 < DVS; n0 += 32) {
+          float ds[32];
+          tmem_ld_32x32(ds, tmem_rows + cfg::TM_DS + n0);
+          tmem_wait_ld();
+#pragma unroll
+          for (int n = 0; n < 32; ++n) S[n0 + n] = fmaf(gl, S[n0 + n], ds[n]);
+        }
+        if (has_next) {
+          write_state_operand();   // its readers (W S, Q S of this chunk) retired before bar_s
+          fence_proxy_async();
+          tc_fence_before();
+          mbar_arrive(bar_sr);
+        }
+      }
+      PHASE(6);
+      ph ^= 1;
     }
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    ph ^= 1;
+    if (!failed && !misaligned && !write_output(ph ^ 1)) failed = true;
   }
   if (failed) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
   else store_state();
@@ -367,7 +415,7 @@ cudaError_t launch_scan_one(const ScanParams& p, const CUtensorMap& tmW, const C
   }
   const long long grid = (long long)p.n_seqs * p.H * (D / DVS);
   if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
-  chunk_scan_kernel<DVS><<<(int)grid, NT, cfg::SMEM, stream>>>(tmW, tmQ, tmK, p);
+  chunk_scan_kernel<DVS><<<(int)grid, NT + 32, cfg::SMEM, stream>>>(tmW, tmQ, tmK, p);
   return cudaGetLastError();
 }
 
