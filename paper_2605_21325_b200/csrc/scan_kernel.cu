@@ -47,8 +47,8 @@ struct ScanCfg {
   static constexpr int OFF_UT = OFF_S + 2 * S_BOX;                // U~^T  bf16 [DVS rows][64 tokens]
   static constexpr int OFF_UD = OFF_UT + DVS * 128;               // U~'^T bf16 (rows scaled by gamma_last / gamma_i)
   static constexpr int OFF_P = OFF_UD + DVS * 128;                // P bf16 [64][64]
-  static constexpr int OFF_G = OFF_P + 8192;                      // g * log2(e): two buffers of 64 floats
-  static constexpr int OFF_BAR = OFF_G + 512;                     // 10 mbarriers, tensor-memory slot
+  static constexpr int OFF_G = OFF_P + 8192;                      // g * log2(e): two buffers of 64 floats, then two of column factors
+  static constexpr int OFF_BAR = OFF_G + 1024;                     // 10 mbarriers, tensor-memory slot
   static constexpr int SMEM = OFF_BAR + 96;
   static constexpr int TM_QK = 0, TM_T1 = 64, TM_QS = 64 + DVS, TM_PU = 64 + 2 * DVS, TM_DS = 64 + 3 * DVS;
   static constexpr int TMEM_COLS = (64 + 4 * DVS) <= 256 ? 256 : 512;
@@ -95,6 +95,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   constexpr int NTL = cfg::NTL, NS = D / DVS;
   extern __shared__ __align__(1024) uint8_t smem[];
   float* sG = reinterpret_cast<float*>(smem + cfg::OFF_G);
+  float* sCf = sG + 2 * C;   // 2^(g_ref(j) - g_j), g_ref(j) = g of the first token of j's block of eight
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 88);
   const uint32_t sW = smem_u32(smem + cfg::OFF_W), sQ = smem_u32(smem + cfg::OFF_Q), sK = smem_u32(smem + cfg::OFF_K);
   const uint32_t sS = smem_u32(smem + cfg::OFF_S), sUt = smem_u32(smem + cfg::OFF_UT), sUd = smem_u32(smem + cfg::OFF_UD);
@@ -160,9 +161,18 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   // rows past the sequence end take the last real row's g, so that every exponent stays a difference of real values
   auto fetch_g = [&](int tok0, int rows) -> float {
     const int i = tid < rows ? tid : rows - 1;
-    return tid < C ? p.g[(size_t)(tok0 + i) * p.H + h] * kLog2e : 0.f;
+    return tid < C ? p.g[(size_t)(tok0 + i) * p.H + h] : 0.f;   // raw: scaled where it is stored, not where it is loaded
   };
 
+  // g * log2(e) of a chunk and its column factors: the decay 2^(g_i - g_j) of P is formed as
+  // 2^(g_i - g_ref) * 2^(g_ref - g_j) with g_ref the first token of j's block of eight -- one exponential per
+  // (row, block) instead of one per element; the second factor spans at most seven tokens of decay
+  auto store_g = [&](int buf, float g_raw) {
+    const float gl2 = g_raw * kLog2e;
+    const float gref = __shfl_sync(0xffffffffu, gl2, lane & ~7);
+    sG[buf * C + tid] = gl2;
+    sCf[buf * C + tid] = ex2_approx(gref - gl2);
+  };
   uint32_t u_next[NTL][2];
   float g_next = 0.f;
   {
@@ -189,7 +199,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   }
   if (!control) {
     write_state_operand();
-    if (tid < C) sG[tid] = g_next;
+    if (tid < C) store_g(0, g_next);
   }
   fence_proxy_async();
   tc_fence_before();
@@ -334,14 +344,22 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         tmem_ld_16x64(qk, tmem_rows + cfg::TM_QK);
         tmem_ld_frag<NTL>(qs, tmem_rows + cfg::TM_QS);
         tmem_wait_ld();
+        const float* cf = sCf + (c & 1) * C;
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
           const int j = 8 * nt + 2 * t;
-          const float2 gj = *reinterpret_cast<const float2*>(gb + j);
-          const float p0 = j <= ra ? qk[nt][0] * ex2_approx(g_a - gj.x) : 0.f, p1 = j + 1 <= ra ? qk[nt][1] * ex2_approx(g_a - gj.y) : 0.f;
-          const float p2 = j <= rb ? qk[nt][2] * ex2_approx(g_b - gj.x) : 0.f, p3 = j + 1 <= rb ? qk[nt][3] * ex2_approx(g_b - gj.y) : 0.f;
-          *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + ra * 128 + ((nt ^ (ra & 7)) << 4) + 4 * t) = pack_bf16(p0, p1);
-          *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + rb * 128 + ((nt ^ (rb & 7)) << 4) + 4 * t) = pack_bf16(p2, p3);
+          uint32_t wa = 0u, wb = 0u;
+          if (8 * nt <= rb) {   // blocks right of both rows' diagonals are all zero
+            const float gref = gb[8 * nt];
+            const float2 cj = *reinterpret_cast<const float2*>(cf + j);
+            const float ea = ex2_approx(fminf(g_a - gref, 0.f)), eb = ex2_approx(g_b - gref);
+            const float p0 = j <= ra ? qk[nt][0] * ea * cj.x : 0.f, p1 = j + 1 <= ra ? qk[nt][1] * ea * cj.y : 0.f;
+            const float p2 = j <= rb ? qk[nt][2] * eb * cj.x : 0.f, p3 = j + 1 <= rb ? qk[nt][3] * eb * cj.y : 0.f;
+            wa = pack_bf16(p0, p1);
+            wb = pack_bf16(p2, p3);
+          }
+          *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + ra * 128 + ((nt ^ (ra & 7)) << 4) + 4 * t) = wa;
+          *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + rb * 128 + ((nt ^ (rb & 7)) << 4) + 4 * t) = wb;
         }
       }
       fence_proxy_async();
@@ -349,7 +367,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       mbar_arrive(bar_p);
       o_sa = p.scale * ex2_approx(g_a); o_sb = p.scale * ex2_approx(g_b);
       o_tok0 = tok0; o_rows = rows;
-      if (tid < C && has_next) sG[((c + 1) & 1) * C + tid] = g_next;
+      if (tid < C && has_next) store_g((c + 1) & 1, g_next);
       PHASE(4);
 
       // ---- state update (thread = row of S) and the bf16 operand for the next chunk
