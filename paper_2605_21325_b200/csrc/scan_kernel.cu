@@ -7,14 +7,20 @@
 //     S <- gamma_last S + K^T diag(gamma_last / gamma) U~
 //
 // Columns of S (the d_v axis) never mix, so a CTA owns one (sequence, head, slice of DVS value columns) and walks
-// the chunks in order; the slices of one head run side by side and share W, Q, K through L2.
+// the chunks in order.
 //
-// Per chunk, on the tensor cores (tcgen05.mma kind::f16, fp32 accumulators in tensor memory):
-//   T1 = W S   and  QS = Q S   (B operand: S rounded to bf16, kept K-major in shared memory),
-//   QK = Q K^T,   dS = K^T U~' (A operand: the K tile read MN-major; U~' = decay-scaled U~ in bf16),   PU = P U~.
-// The dependent chain of a chunk is  T1 -> U~ -> dS -> S;  QS, QK, P and PU hang off it.
-// TMA brings the W, Q and K tiles (one buffer each, refilled as soon as their last reader has retired);
-// U and g come through registers one chunk ahead.
+// The tensor pipe spends a near-constant time per tcgen05.mma at these sizes, so the chunk is cut into as few,
+// as large products as the data flow allows -- three per chunk, 16 instructions in all:
+//   P1 [128 x (DVS+64)] = [W ; Q] . [S | K^T]     rows 0..63: W S (and W K^T, unused); rows 64..127: Q S | Q K^T
+//   P3 [128 x DVS]      = K^T . U~'               U~' = decay-scaled U~ (bf16); the K tile is read MN-major
+//   PU [128 x DVS]      = [any ; P] . U~          rows 64..127 = P U~, on the lanes that also hold Q S
+// The dependent chain of a chunk is  P1 -> U~ -> P3 -> S.  Warp 8 holds the one thread that issues every product;
+// warps 0..7 compute.  Warp w works on tensor-memory lanes 32 (w & 3) .. +31 and on half (w >> 2) of the value
+// columns; lanes 0..63 carry W S, so warps of quadrants 0 and 1 form U~ ("chain warps"), those of quadrants 2
+// and 3 form P and the output ("output warps"); all eight update their part of S.  Hand-offs are mbarriers:
+// commits from the products, counted arrivals from the compute threads after their operand writes.
+// TMA brings W, Q and K (K twice: once beside S^T as the B operand of P1, once as the A operand of P3, so that
+// each copy is refilled as early as its own reader allows); U and g come through registers one chunk ahead.
 // Every mbarrier wait is bounded; on expiry the CTA raises the status word, frees its tensor memory and returns.
 #include "tc_device.cuh"
 
@@ -29,35 +35,39 @@ namespace {
     if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(p.status + 8 + 12 * (threadIdx.x >> 5) + (k), (int)(now - ph_t)); \
     ph_t = now;                                                                   \
   } while (0)
-#define SUBPHASE(k) do { long long now = clock64(); atomicAdd(p.status + 64 + (k), (int)(now - sub_t)); sub_t = now; } while (0)
+#define SUB_BEGIN() long long sub_t = clock64()
+#define SUBPHASE(k) do { long long now = clock64(); if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(p.status + 120 + (k), (int)(now - sub_t)); sub_t = now; } while (0)
 #else
 #define PHASE_BEGIN() do {} while (0)
 #define PHASE(k) do {} while (0)
+#define SUB_BEGIN() do {} while (0)
 #define SUBPHASE(k) do {} while (0)
 #endif
 
-constexpr int C = 64, D = 128, NT = 128;
+constexpr int C = 64, D = 128, NT = 256;   // NT compute threads (8 warps) + one control warp
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int DVS>
 struct ScanCfg {
-  static constexpr int OFF_W = 0, OFF_Q = 16384, OFF_K = 32768;   // bf16 tiles: 2 boxes of 64 rows x 128 B
-  static constexpr int OFF_S = 49152;                             // S^T bf16 [DVS rows][128 d_k]: 2 boxes of DVS rows x 128 B
-  static constexpr int S_BOX = DVS * 128;
-  static constexpr int OFF_UT = OFF_S + 2 * S_BOX;                // U~^T  bf16 [DVS rows][64 tokens]
-  static constexpr int OFF_UD = OFF_UT + DVS * 128;               // U~'^T bf16 (rows scaled by gamma_last / gamma_i)
-  static constexpr int OFF_P = OFF_UD + DVS * 128;                // P bf16 [64][64]
-  static constexpr int OFF_G = OFF_P + 8192;                      // g * log2(e): two buffers of 64 floats, then two of column factors
-  static constexpr int OFF_BAR = OFF_G + 1024;                     // 10 mbarriers, tensor-memory slot
+  static constexpr int CW = DVS / 2;                     // value columns per compute warp
+  static constexpr int NTW = CW / 8;                     // accumulator n-tiles per compute warp
+  static constexpr int N1 = DVS + 64;                    // columns of P1
+  // A operand of P1: [W ; Q], two boxes (64 features each) of 128 rows x 128 B
+  static constexpr int OFF_A = 0, A_BOX = 16384;
+  // B operand of P1: [S^T ; K], two boxes of (DVS + 64) rows x 128 B
+  static constexpr int OFF_B = 32768, B_BOX = N1 * 128;
+  static constexpr int OFF_KA = OFF_B + 2 * B_BOX;       // K tile for P3 (MN-major A); its second box doubles as the
+  static constexpr int OFF_P = OFF_KA + 16384;           // unused upper half of PU's A operand, P being the lower half
+  static constexpr int OFF_UT = OFF_P + 8192;            // U~  bf16 [64 tokens][DVS], boxes of 64 columns (MN-major B)
+  static constexpr int U_BYTES = (DVS / 64) * 8192;
+  static constexpr int OFF_UD = OFF_UT + U_BYTES;        // U~' bf16, same layout
+  static constexpr int OFF_G = OFF_UD + U_BYTES;         // g * log2(e): 2 x 64 floats; column factors: 2 x 64 floats
+  static constexpr int OFF_BAR = OFF_G + 1024;           // 9 mbarriers, tensor-memory slot
   static constexpr int SMEM = OFF_BAR + 96;
-  static constexpr int TM_QK = 0, TM_T1 = 64, TM_QS = 64 + DVS, TM_PU = 64 + 2 * DVS, TM_DS = 64 + 3 * DVS;
-  static constexpr int TMEM_COLS = (64 + 4 * DVS) <= 256 ? 256 : 512;
-  static constexpr int CTAS_PER_SM = TMEM_COLS == 256 ? 2 : 1;
-  static constexpr int NTL = DVS / 8;                             // accumulator n-tiles per row block
+  static constexpr int TM_P1 = 0, TM_DS = N1, TM_PU = N1 + DVS;
+  static constexpr int TMEM_COLS = (N1 + 2 * DVS) <= 256 ? 256 : 512;
+  static constexpr int CTAS_PER_SM = 1;   // registers: 9 warps at the kernel's natural register count fill an SM once
 };
-
-// kind::f16 instruction descriptor with an MN-major A operand (bit 15): A is read as stored [k][m].
-__host__ __device__ constexpr uint32_t umma_idesc_amn(int M, int N) { return umma_idesc(M, N, 0) | (1u << 15); }
 
 __device__ __forceinline__ void tmem_ld_16x32(float (&r)[4][4], uint32_t taddr) {
   asm volatile(
@@ -71,20 +81,36 @@ __device__ __forceinline__ void tmem_ld_frag(float (&r)[NTL][4], uint32_t taddr)
   if constexpr (NTL == 8) tmem_ld_16x64(r, taddr);
   else tmem_ld_16x32(r, taddr);
 }
-// 32 lanes x 32 columns: thread = lane, 32 consecutive columns
-__device__ __forceinline__ void tmem_ld_32x32(float* r, uint32_t taddr) {
+__device__ __forceinline__ void tmem_st_16x32(const float (&r)[4][4], uint32_t taddr) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=f"(r[0]), "=f"(r[1]), "=f"(r[2]), "=f"(r[3]), "=f"(r[4]), "=f"(r[5]), "=f"(r[6]), "=f"(r[7]), "=f"(r[8]), "=f"(r[9]), "=f"(r[10]),
-        "=f"(r[11]), "=f"(r[12]), "=f"(r[13]), "=f"(r[14]), "=f"(r[15]), "=f"(r[16]), "=f"(r[17]), "=f"(r[18]), "=f"(r[19]), "=f"(r[20]),
-        "=f"(r[21]), "=f"(r[22]), "=f"(r[23]), "=f"(r[24]), "=f"(r[25]), "=f"(r[26]), "=f"(r[27]), "=f"(r[28]), "=f"(r[29]), "=f"(r[30]),
-        "=f"(r[31])
-      : "r"(taddr));
+      "tcgen05.st.sync.aligned.16x256b.x4.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+      ::"f"(r[0][0]), "f"(r[0][1]), "f"(r[0][2]), "f"(r[0][3]), "f"(r[1][0]), "f"(r[1][1]), "f"(r[1][2]), "f"(r[1][3]),
+        "f"(r[2][0]), "f"(r[2][1]), "f"(r[2][2]), "f"(r[2][3]), "f"(r[3][0]), "f"(r[3][1]), "f"(r[3][2]), "f"(r[3][3]),
+        "r"(taddr)
+      : "memory");
 }
-
+template <int NTL>
+__device__ __forceinline__ void tmem_st_frag(const float (&r)[NTL][4], uint32_t taddr) {
+#pragma unroll
+  for (int b = 0; b < NTL; b += 4) {
+    const float q[4][4] = {{r[b][0], r[b][1], r[b][2], r[b][3]}, {r[b + 1][0], r[b + 1][1], r[b + 1][2], r[b + 1][3]},
+                           {r[b + 2][0], r[b + 2][1], r[b + 2][2], r[b + 2][3]}, {r[b + 3][0], r[b + 3][1], r[b + 3][2], r[b + 3][3]}};
+    tmem_st_16x32(q, taddr + 8 * b);
+  }
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void stmatrix_x4(uint32_t addr, uint32_t m0, uint32_t m1, uint32_t m2, uint32_t m3) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
+}
+__device__ __forceinline__ void stmatrix_x4_trans(uint32_t addr, uint32_t m0, uint32_t m1, uint32_t m2, uint32_t m3) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
+}
+// kind::f16 instruction descriptor, fp32 accumulate, bf16 operands; a_mn / b_mn: operand stored MN-major
+__host__ __device__ constexpr uint32_t umma_idesc_ab(int M, int N, int a_mn, int b_mn) {
+  return umma_idesc(M, N, b_mn) | ((uint32_t)a_mn << 15);
 }
 
 template <int DVS>
@@ -92,78 +118,116 @@ __global__ void __launch_bounds__(NT + 32, ScanCfg<DVS>::CTAS_PER_SM)
 chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmQ,
                   const __grid_constant__ CUtensorMap tmK, ScanParams p) {
   using cfg = ScanCfg<DVS>;
-  constexpr int NTL = cfg::NTL, NS = D / DVS;
+  constexpr int NTW = cfg::NTW, CW = cfg::CW, NS = D / DVS;
   extern __shared__ __align__(1024) uint8_t smem[];
   float* sG = reinterpret_cast<float*>(smem + cfg::OFF_G);
   float* sCf = sG + 2 * C;   // 2^(g_ref(j) - g_j), g_ref(j) = g of the first token of j's block of eight
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 88);
-  const uint32_t sW = smem_u32(smem + cfg::OFF_W), sQ = smem_u32(smem + cfg::OFF_Q), sK = smem_u32(smem + cfg::OFF_K);
-  const uint32_t sS = smem_u32(smem + cfg::OFF_S), sUt = smem_u32(smem + cfg::OFF_UT), sUd = smem_u32(smem + cfg::OFF_UD);
-  const uint32_t sP = smem_u32(smem + cfg::OFF_P);
-  // copies (TMA):            bar_w, bar_q, bar_k
-  // products done (commit):  bar_t1 (W S), bar_o (Q S, Q K^T), bar_s (K^T U~'), bar_pu (P U~)
-  // operands written (128 arrivals of the compute threads): bar_sr (S^T), bar_ut (U~^T, U~'^T), bar_p (P)
-  const uint32_t bar_w = smem_u32(smem + cfg::OFF_BAR), bar_q = bar_w + 8, bar_k = bar_w + 16, bar_t1 = bar_w + 24,
-                 bar_o = bar_w + 32, bar_s = bar_w + 40, bar_pu = bar_w + 48, bar_sr = bar_w + 56, bar_ut = bar_w + 64,
-                 bar_p = bar_w + 72;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 80);
+  const uint32_t sA = smem_u32(smem + cfg::OFF_A), sB = smem_u32(smem + cfg::OFF_B), sKa = smem_u32(smem + cfg::OFF_KA);
+  const uint32_t sP = smem_u32(smem + cfg::OFF_P), sUt = smem_u32(smem + cfg::OFF_UT), sUd = smem_u32(smem + cfg::OFF_UD);
+  // copies (TMA):            bar_a (W and Q), bar_kb (K beside S^T), bar_ka (K for P3)
+  // products done (commit):  bar_t1 (P1), bar_s (P3), bar_pu (PU)
+  // operands written:        bar_sr (S^T, all NT compute threads), bar_ut (U~ and U~', chain warps), bar_p (P, output warps)
+  const uint32_t bar_a = smem_u32(smem + cfg::OFF_BAR), bar_kb = bar_a + 8, bar_ka = bar_a + 16, bar_t1 = bar_a + 24,
+                 bar_s = bar_a + 32, bar_pu = bar_a + 40, bar_sr = bar_a + 48, bar_ut = bar_a + 56, bar_p = bar_a + 64;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bool control = warp == 4;               // warp 4: one thread issues every product; warps 0..3 compute
+  const bool control = warp == 8;
+  const int quad = warp & 3, half = (warp >> 2) & 1;
+  const bool chain = quad < 2;                   // lanes 0..63 of P1 hold W S
   const int gq = lane >> 2, t = lane & 3;
-  const int ra = 16 * (warp & 3) + gq, rb = ra + 8;   // this thread's two rows of every M = 64 accumulator
+  const int tok_w = 32 * (quad & 1);             // first token row of this warp in P1 and PU (either role)
+  const int krow_w = 32 * quad;                  // first row of S of this warp
+  const int cw0 = half * CW;                     // first value column of this warp inside the CTA's slice
 
   const int slice = blockIdx.x % NS, h = (blockIdx.x / NS) % p.H, s = blockIdx.x / (NS * p.H);
   const int beg = p.seq_off ? p.seq_off[s] : s * p.T;
   const int end = p.seq_off ? p.seq_off[s + 1] : (s + 1) * p.T;
   const int n_chunks = (end - beg + C - 1) / C;
-  const int col0 = slice * DVS;                  // first value column of this CTA
+  const int col0 = slice * DVS + cw0;            // this warp's first column in the value dimension
 
-  // state: compute thread tid owns row tid (a key feature) of S, DVS columns
-  float S[DVS];
+  // State in accumulator-fragment layout: lane group lg (rows krow_w + 16 lg + gq and + 8), n-tile nt
+  // (columns cw0 + 8 nt + 2 t and + 1):  S[lg][nt][0..3] = (row, col), (row, col+1), (row+8, col), (row+8, col+1).
+  float S[2][NTW][4];
   if (!control) {
-    const float* s0 = p.S0 ? p.S0 + (((size_t)s * p.H + h) * D + tid) * D + col0 : nullptr;
 #pragma unroll
-    for (int n = 0; n < DVS; n += 4) {
-      float4 v = s0 ? *reinterpret_cast<const float4*>(s0 + n) : make_float4(0.f, 0.f, 0.f, 0.f);
-      S[n] = v.x; S[n + 1] = v.y; S[n + 2] = v.z; S[n + 3] = v.w;
-    }
+    for (int lg = 0; lg < 2; ++lg)
+#pragma unroll
+      for (int nt = 0; nt < NTW; ++nt) {
+        const int k = krow_w + 16 * lg + gq, n = col0 + 8 * nt + 2 * t;
+        float2 a = make_float2(0.f, 0.f), b = a;
+        if (p.S0) {
+          const float* s0 = p.S0 + ((size_t)s * p.H + h) * D * D;
+          a = *reinterpret_cast<const float2*>(s0 + (size_t)k * D + n);
+          b = *reinterpret_cast<const float2*>(s0 + (size_t)(k + 8) * D + n);
+        }
+        S[lg][nt][0] = a.x; S[lg][nt][1] = a.y; S[lg][nt][2] = b.x; S[lg][nt][3] = b.y;
+      }
   }
   auto store_state = [&]() {
     if (!p.S_out || control) return;
-    float* dst = p.S_out + (((size_t)s * p.H + h) * D + tid) * D + col0;
+    float* dst = p.S_out + ((size_t)s * p.H + h) * D * D;
 #pragma unroll
-    for (int n = 0; n < DVS; n += 4) *reinterpret_cast<float4*>(dst + n) = make_float4(S[n], S[n + 1], S[n + 2], S[n + 3]);
+    for (int lg = 0; lg < 2; ++lg)
+#pragma unroll
+      for (int nt = 0; nt < NTW; ++nt) {
+        const int k = krow_w + 16 * lg + gq, n = col0 + 8 * nt + 2 * t;
+        *reinterpret_cast<float2*>(dst + (size_t)k * D + n) = make_float2(S[lg][nt][0], S[lg][nt][1]);
+        *reinterpret_cast<float2*>(dst + (size_t)(k + 8) * D + n) = make_float2(S[lg][nt][2], S[lg][nt][3]);
+      }
   };
   if (n_chunks == 0) { store_state(); return; }
-  const bool misaligned = (sW & 1023u) != 0;     // never expected; the swizzle pattern would not match the copies
+  const bool misaligned = (sA & 1023u) != 0;     // never expected; the swizzle pattern would not match the copies
 
-  // S^T as the K-major B operand: element (n, k) of a [DVS rows][128] bf16 tile, two boxes of 64 features
+  // S^T as rows 0..DVS-1 of the K-major B operand of P1: row n = value column, 16-byte pieces of eight key features.
+  // stmatrix.trans turns the fragments (rows = features, column pairs) into exactly those pieces.
   auto write_state_operand = [&]() {
-    uint8_t* base = smem + cfg::OFF_S + (tid >> 6) * cfg::S_BOX + (tid & 7) * 2;
-    const int kc = (tid & 63) >> 3;
+    const int mi = lane >> 3, r = lane & 7;      // this lane addresses row r of matrix mi of each x4 store
 #pragma unroll
-    for (int n = 0; n < DVS; ++n)
-      *reinterpret_cast<__nv_bfloat16*>(base + n * 128 + ((kc ^ (n & 7)) << 4)) = __float2bfloat16_rn(S[n]);
+    for (int lg = 0; lg < 2; ++lg)
+#pragma unroll
+      for (int nt = 0; nt < NTW; nt += 2) {
+        // matrices: (features +0..7, tile nt), (features +8..15, tile nt), (+0..7, nt+1), (+8..15, nt+1)
+        const int k0 = krow_w + 16 * lg + 8 * (mi & 1);          // first feature of this lane's matrix
+        const int n = cw0 + 8 * (nt + (mi >> 1)) + r;            // row of the operand
+        const uint32_t addr = sB + (k0 >> 6) * cfg::B_BOX + n * 128 + ((((k0 & 63) >> 3) ^ (n & 7)) << 4);
+        stmatrix_x4_trans(addr, pack_bf16(S[lg][nt][0], S[lg][nt][1]), pack_bf16(S[lg][nt][2], S[lg][nt][3]),
+                          pack_bf16(S[lg][nt + 1][0], S[lg][nt + 1][1]), pack_bf16(S[lg][nt + 1][2], S[lg][nt + 1][3]));
+      }
   };
-  auto issue_tile = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int tok0) {
-    mbar_expect_tx(bar, 16384u);
-    tma_load_2d(dst, tm, bar, h * D, tok0);
-    tma_load_2d(dst + 8192, tm, bar, h * D + 64, tok0);
+  auto issue_wq = [&](int tok0) {
+    mbar_expect_tx(bar_a, 32768u);
+    tma_load_2d(sA, &tmW, bar_a, h * D, tok0);
+    tma_load_2d(sA + 8192, &tmQ, bar_a, h * D, tok0);
+    tma_load_2d(sA + cfg::A_BOX, &tmW, bar_a, h * D + 64, tok0);
+    tma_load_2d(sA + cfg::A_BOX + 8192, &tmQ, bar_a, h * D + 64, tok0);
   };
+  auto issue_kb = [&](int tok0) {
+    mbar_expect_tx(bar_kb, 16384u);
+    tma_load_2d(sB + DVS * 128, &tmK, bar_kb, h * D, tok0);
+    tma_load_2d(sB + cfg::B_BOX + DVS * 128, &tmK, bar_kb, h * D + 64, tok0);
+  };
+  auto issue_ka = [&](int tok0) {
+    mbar_expect_tx(bar_ka, 16384u);
+    tma_load_2d(sKa, &tmK, bar_ka, h * D, tok0);
+    tma_load_2d(sKa + 8192, &tmK, bar_ka, h * D + 64, tok0);
+  };
+  // U of the chain warps in fragment layout: u[lg][nt][0] = row tok_w + 16 lg + gq, [1] = that row + 8 (bf16 pairs)
   const __nv_bfloat16* Ug = reinterpret_cast<const __nv_bfloat16*>(p.U);
-  auto fetch_u = [&](uint32_t (&u)[NTL][2], int tok0, int rows) {
+  auto fetch_u = [&](uint32_t (&u)[2][NTW][2], int tok0, int rows) {
 #pragma unroll
-    for (int nt = 0; nt < NTL; ++nt) {
-      const int c = col0 + 8 * nt + 2 * t;
-      u[nt][0] = ra < rows ? *reinterpret_cast<const uint32_t*>(Ug + ((size_t)(tok0 + ra) * p.H + h) * D + c) : 0u;
-      u[nt][1] = rb < rows ? *reinterpret_cast<const uint32_t*>(Ug + ((size_t)(tok0 + rb) * p.H + h) * D + c) : 0u;
-    }
+    for (int lg = 0; lg < 2; ++lg)
+#pragma unroll
+      for (int nt = 0; nt < NTW; ++nt) {
+        const int i = tok_w + 16 * lg + gq, cidx = col0 + 8 * nt + 2 * t;
+        u[lg][nt][0] = i < rows ? *reinterpret_cast<const uint32_t*>(Ug + ((size_t)(tok0 + i) * p.H + h) * D + cidx) : 0u;
+        u[lg][nt][1] = i + 8 < rows ? *reinterpret_cast<const uint32_t*>(Ug + ((size_t)(tok0 + i + 8) * p.H + h) * D + cidx) : 0u;
+      }
   };
   // rows past the sequence end take the last real row's g, so that every exponent stays a difference of real values
   auto fetch_g = [&](int tok0, int rows) -> float {
     const int i = tid < rows ? tid : rows - 1;
     return tid < C ? p.g[(size_t)(tok0 + i) * p.H + h] : 0.f;   // raw: scaled where it is stored, not where it is loaded
   };
-
   // g * log2(e) of a chunk and its column factors: the decay 2^(g_i - g_j) of P is formed as
   // 2^(g_i - g_ref) * 2^(g_ref - g_j) with g_ref the first token of j's block of eight -- one exponential per
   // (row, block) instead of one per element; the second factor spans at most seven tokens of decay
@@ -173,25 +237,26 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     sG[buf * C + tid] = gl2;
     sCf[buf * C + tid] = ex2_approx(gref - gl2);
   };
-  uint32_t u_next[NTL][2];
+
+  uint32_t xr[2][NTW][2];   // chain warps: the next chunk's U (bf16 pairs)
   float g_next = 0.f;
   {
     const int rows0 = end - beg < C ? end - beg : C;
     if (tid == NT) {
       prefetch_tmap(&tmW); prefetch_tmap(&tmQ); prefetch_tmap(&tmK);
-      for (int b = 0; b < 7; ++b) mbar_init(bar_w + 8 * b, 1);
-      for (int b = 7; b < 10; ++b) mbar_init(bar_w + 8 * b, NT);
+      for (int b = 0; b < 6; ++b) mbar_init(bar_a + 8 * b, 1);
+      mbar_init(bar_sr, NT);
+      mbar_init(bar_ut, NT / 2);
+      mbar_init(bar_p, NT / 2);
       fence_mbar_init();
       if (!misaligned) {
-        issue_tile(sW, &tmW, bar_w, beg);
-        issue_tile(sQ, &tmQ, bar_q, beg);
-        issue_tile(sK, &tmK, bar_k, beg);
+        issue_wq(beg);
+        issue_kb(beg);
+        issue_ka(beg);
       }
     }
-    if (!control) {
-      fetch_u(u_next, beg, rows0);
-      g_next = fetch_g(beg, rows0);
-    }
+    if (!control && chain) fetch_u(xr, beg, rows0);
+    if (!control) g_next = fetch_g(beg, rows0);
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(cfg::TMEM_COLS) : "memory");
@@ -206,47 +271,56 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   __syncthreads();   // barriers initialised, tensor memory allocated, first operand of S and first g in place
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_rows = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
+  const uint32_t tmem_w = tmem + ((uint32_t)(32 * quad) << 16);   // this warp's lanes, column 0
   bool failed = misaligned;
 
   if (control) {
     // ---------------------------------------------------------------- control thread: every tcgen05.mma of the CTA
     if (lane == 0 && !misaligned) {
-      constexpr uint32_t idesc_n = umma_idesc(C, DVS, 0), idesc_qk = umma_idesc(C, C, 0), idesc_ds = umma_idesc_amn(D, DVS);
+      constexpr uint32_t idesc_p1 = umma_idesc_ab(128, cfg::N1, 0, 0);   // [W;Q] K-major, [S^T;K] K-major
+      constexpr uint32_t idesc_p3 = umma_idesc_ab(128, DVS, 1, 1);       // K tile MN-major, U~' MN-major
+      constexpr uint32_t idesc_pu = umma_idesc_ab(128, DVS, 0, 1);       // [any;P] K-major, U~ MN-major
       // descriptors differ from these bases only in the address field (bits 0..13, units of 16 bytes)
-      const uint64_t dW = umma_desc(sW, 16, 1024), dQ = umma_desc(sQ, 16, 1024), dK = umma_desc(sK, 16, 1024),
-                     dS = umma_desc(sS, 16, 1024), dKt = umma_desc(sK, 8192, 1024), dUd = umma_desc(sUd, 16, 1024),
-                     dP = umma_desc(sP, 16, 1024), dUt = umma_desc(sUt, 16, 1024);
-      auto mma_k128 = [&](uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t b_box, uint32_t idesc) {
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks)
-          umma_bf16(d_tmem, a + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), b + (((ks >> 2) * b_box + (ks & 3) * 32) >> 4), idesc, ks > 0);
-      };
+      const uint64_t dA = umma_desc(sA, 16, 1024), dB = umma_desc(sB, 16, 1024), dKa = umma_desc(sKa, 8192, 1024),
+                     dUd = umma_desc(sUd, 8192, 1024), dUt = umma_desc(sUt, 8192, 1024),
+                     dPa = umma_desc(sKa + 8192, 16, 1024);              // 128 rows: second K box, then P
       uint32_t ph = 0;
       for (int c = 0; c < n_chunks; ++c) {
-        // T1 = W S: the head of the chunk's dependent chain, issued first
-        if (!mbar_wait_bounded(bar_sr, ph) || !mbar_wait_bounded(bar_w, ph)) { failed = true; break; }
-        tc_fence_after();
-        mma_k128(tmem + cfg::TM_T1, dW, dS, cfg::S_BOX, idesc_n);
-        umma_commit(bar_t1);
-        if (!mbar_wait_bounded(bar_q, ph) || !mbar_wait_bounded(bar_k, ph)) { failed = true; break; }
-        tc_fence_after();
-        mma_k128(tmem + cfg::TM_QK, dQ, dK, 8192, idesc_qk);
-        mma_k128(tmem + cfg::TM_QS, dQ, dS, cfg::S_BOX, idesc_n);
-        umma_commit(bar_o);
-        // dS = K^T U~' as soon as the compute threads have written U~'
-        if (!mbar_wait_bounded(bar_ut, ph)) { failed = true; break; }
+#ifdef TRI_INV_PHASE_CLOCKS
+        long long ct = clock64();
+#define CSUB(k) do { long long now = clock64(); if (blockIdx.x == 0) atomicAdd(p.status + 110 + (k), (int)(now - ct)); ct = now; } while (0)
+#else
+#define CSUB(k) do {} while (0)
+#endif
+        if (!mbar_wait_bounded(bar_sr, ph)) { failed = true; break; }
+        CSUB(0);
+        if (!mbar_wait_bounded(bar_a, ph) || !mbar_wait_bounded(bar_kb, ph)) { failed = true; break; }
+        CSUB(1);
         tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < C / 16; ++ks)   // K tile read MN-major: 16 tokens (2048 bytes) per step
-          umma_bf16(tmem + cfg::TM_DS, dKt + ((ks * 2048) >> 4), dUd + ((ks * 32) >> 4), idesc_ds, ks > 0);
+        for (int ks = 0; ks < D / 16; ++ks)
+          umma_bf16(tmem + cfg::TM_P1, dA + (((ks >> 2) * cfg::A_BOX + (ks & 3) * 32) >> 4),
+                    dB + (((ks >> 2) * cfg::B_BOX + (ks & 3) * 32) >> 4), idesc_p1, ks > 0);
+        umma_commit(bar_t1);
+        CSUB(2);
+        if (!mbar_wait_bounded(bar_ut, ph)) { failed = true; break; }
+        CSUB(3);
+        if (!mbar_wait_bounded(bar_ka, ph)) { failed = true; break; }
+        CSUB(4);
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < C / 16; ++ks)   // 16 tokens (2048 bytes of either operand) per step
+          umma_bf16(tmem + cfg::TM_DS, dKa + ((ks * 2048) >> 4), dUd + ((ks * 2048) >> 4), idesc_p3, ks > 0);
         umma_commit(bar_s);
+        CSUB(5);
         if (!mbar_wait_bounded(bar_p, ph)) { failed = true; break; }
+        CSUB(6);
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < C / 16; ++ks)
-          umma_bf16(tmem + cfg::TM_PU, dP + ((ks * 32) >> 4), dUt + ((ks * 32) >> 4), idesc_n, ks > 0);
+          umma_bf16(tmem + cfg::TM_PU, dPa + ((ks * 32) >> 4), dUt + ((ks * 2048) >> 4), idesc_pu, 1u);   // on top of gamma_i Q S
         umma_commit(bar_pu);
+        CSUB(7);
         ph ^= 1;
       }
     }
@@ -254,26 +328,29 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     // ---------------------------------------------------------------- compute warps
     mbar_arrive(bar_sr);   // the first S^T operand (written before the CTA barrier above)
     uint32_t ph = 0;
-    float qs[NTL][4];      // Q S of the chunk whose output is still to be written
-    float o_sa = 0.f, o_sb = 0.f;
     int o_tok0 = 0, o_rows = 0;
-    // O = scale * (gamma_i QS + PU) of the previous chunk: written while the next chunk's first product runs
+    // O = scale * (gamma_i QS + P U~) of the previous chunk (the PU accumulator starts from gamma_i QS): written
+    // while the next chunk's first product runs
     auto write_output = [&](uint32_t parity) -> bool {
       if (!mbar_wait_bounded(bar_pu, parity)) return false;
       tc_fence_after();
-      float pu[NTL][4];
-      tmem_ld_frag<NTL>(pu, tmem_rows + cfg::TM_PU);
-      tmem_wait_ld();
       __nv_bfloat16* Og = reinterpret_cast<__nv_bfloat16*>(p.O);
 #pragma unroll
-      for (int nt = 0; nt < NTL; ++nt) {
-        const int cc = col0 + 8 * nt + 2 * t;
-        if (ra < o_rows)
-          *reinterpret_cast<uint32_t*>(Og + ((size_t)(o_tok0 + ra) * p.H + h) * D + cc) =
-              pack_bf16(fmaf(o_sa, qs[nt][0], p.scale * pu[nt][0]), fmaf(o_sa, qs[nt][1], p.scale * pu[nt][1]));
-        if (rb < o_rows)
-          *reinterpret_cast<uint32_t*>(Og + ((size_t)(o_tok0 + rb) * p.H + h) * D + cc) =
-              pack_bf16(fmaf(o_sb, qs[nt][2], p.scale * pu[nt][2]), fmaf(o_sb, qs[nt][3], p.scale * pu[nt][3]));
+      for (int lg = 0; lg < 2; ++lg) {
+        float pu[NTW][4];
+        tmem_ld_frag<NTW>(pu, tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_PU + cw0);
+        tmem_wait_ld();
+        const int i = tok_w + 16 * lg + gq;
+#pragma unroll
+        for (int nt = 0; nt < NTW; ++nt) {
+          const int cc = col0 + 8 * nt + 2 * t;
+          if (i < o_rows)
+            *reinterpret_cast<uint32_t*>(Og + ((size_t)(o_tok0 + i) * p.H + h) * D + cc) =
+                pack_bf16(p.scale * pu[nt][0], p.scale * pu[nt][1]);
+          if (i + 8 < o_rows)
+            *reinterpret_cast<uint32_t*>(Og + ((size_t)(o_tok0 + i + 8) * p.H + h) * D + cc) =
+                pack_bf16(p.scale * pu[nt][2], p.scale * pu[nt][3]);
+        }
       }
       tc_fence_before();
       return true;
@@ -285,117 +362,147 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       const int nx_tok0 = tok0 + C, nx_rows = end - nx_tok0 < C ? end - nx_tok0 : C;
       const float* gb = sG + (c & 1) * C;
       PHASE_BEGIN();
-      uint32_t u_cur[NTL][2];
+      if (has_next) g_next = fetch_g(nx_tok0, nx_rows);
+      if (chain && has_next && t == 0) {
+        // next chunk's U rows of this thread into L2 now; the loads into registers follow when this chunk's U is used up
 #pragma unroll
-      for (int nt = 0; nt < NTL; ++nt) { u_cur[nt][0] = u_next[nt][0]; u_cur[nt][1] = u_next[nt][1]; }
-      if (has_next) {
-        fetch_u(u_next, nx_tok0, nx_rows);
-        g_next = fetch_g(nx_tok0, nx_rows);
+        for (int rr = 0; rr < 4; ++rr) {
+          const int i = tok_w + 8 * rr + gq;
+          if (i < nx_rows) asm volatile("prefetch.global.L2 [%0];" ::"l"(Ug + ((size_t)(nx_tok0 + i) * p.H + h) * D + col0));
+        }
       }
-      if (c > 0 && !write_output(ph ^ 1)) { failed = true; break; }
+      if (!chain && c > 0) {
+        if (!write_output(ph ^ 1)) { failed = true; break; }
+        if (tid == 64) issue_ka(tok0);   // PU of the last chunk, the last reader of that buffer, has retired
+      }
       PHASE(0);
 
-      // ---- U~ = U - W S  ->  bf16 operands U~^T and (decay-scaled) U~'^T
       if (!mbar_wait_bounded(bar_t1, ph)) { failed = true; break; }
       tc_fence_after();
       PHASE(1);
+      if (has_next && tid == 32) issue_wq(nx_tok0);    // P1, the only reader of W, Q and of the K beside S^T, has retired
+      if (has_next && tid == 96) issue_kb(nx_tok0);
       // (this chunk's g was written by other threads during the last chunk: read only after the wait above,
       // which follows every compute thread's arrival on bar_sr)
-      const float g_a = gb[ra], g_b = gb[rb], g_last = gb[rows - 1];
-      if (tid == 32 && has_next) issue_tile(sW, &tmW, bar_w, nx_tok0);   // W's only reader has retired
-      {
-        float t1[NTL][4];
-        tmem_ld_frag<NTL>(t1, tmem_rows + cfg::TM_T1);
-        tmem_wait_ld();
-        const float da = ex2_approx(g_last - g_a), db = ex2_approx(g_last - g_b);
-        const int ca = ra >> 3, cb = rb >> 3;
+      const float g_last = gb[rows - 1];
+      if (chain) {
+        // ---- U~ = U - W S  ->  bf16 operands U~ and (decay-scaled) U~', [token rows][value columns]
+        const int mi = lane >> 3, r = lane & 7;
+        SUB_BEGIN();
 #pragma unroll
-        for (int nt = 0; nt < NTL; ++nt) {
-          const float2 ua = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u_cur[nt][0]));
-          const float2 ub = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u_cur[nt][1]));
-          const float v0 = ra < rows ? ua.x - t1[nt][0] : 0.f, v1 = ra < rows ? ua.y - t1[nt][1] : 0.f;
-          const float v2 = rb < rows ? ub.x - t1[nt][2] : 0.f, v3 = rb < rows ? ub.y - t1[nt][3] : 0.f;
-          const int n0 = 8 * nt + 2 * t, n1 = n0 + 1;
-          // element (n, token) of a [DVS rows][64 tokens] bf16 tile, 128-byte rows, 16-byte pieces swizzled by the row
-          const uint32_t o0a = n0 * 128 + ((ca ^ (n0 & 7)) << 4) + (ra & 7) * 2, o1a = n1 * 128 + ((ca ^ (n1 & 7)) << 4) + (ra & 7) * 2;
-          const uint32_t o0b = n0 * 128 + ((cb ^ (n0 & 7)) << 4) + (rb & 7) * 2, o1b = n1 * 128 + ((cb ^ (n1 & 7)) << 4) + (rb & 7) * 2;
-          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o0a) = __float2bfloat16_rn(v0 * da);
-          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o1a) = __float2bfloat16_rn(v1 * da);
-          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o0b) = __float2bfloat16_rn(v2 * db);
-          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UD + o1b) = __float2bfloat16_rn(v3 * db);
-          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o0a) = __float2bfloat16_rn(v0);
-          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o1a) = __float2bfloat16_rn(v1);
-          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o0b) = __float2bfloat16_rn(v2);
-          *reinterpret_cast<__nv_bfloat16*>(smem + cfg::OFF_UT + o1b) = __float2bfloat16_rn(v3);
+        for (int lg = 0; lg < 2; ++lg) {
+          float t1[NTW][4];
+          tmem_ld_frag<NTW>(t1, tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_P1 + cw0);
+          tmem_wait_ld();
+          SUBPHASE(2 * lg);
+          const int i = tok_w + 16 * lg + gq;
+          const float da = ex2_approx(g_last - gb[i]), db = ex2_approx(g_last - gb[i + 8]);
+          const bool va = i < rows, vb = i + 8 < rows;
+          // the x4 store: matrices (tokens +0..7, tile nt), (tokens +8..15, tile nt), (+0..7, nt+1), (+8..15, nt+1)
+          const int tok = tok_w + 16 * lg + 8 * (mi & 1) + r;
+#pragma unroll
+          for (int nt = 0; nt < NTW; nt += 2) {
+            float v[2][4];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              const uint32_t wa = xr[lg][nt + q][0], wb = xr[lg][nt + q][1];   // bf16 pairs: low half = first column
+              const float2 ua = make_float2(__uint_as_float(wa << 16), __uint_as_float(wa & 0xffff0000u));
+              const float2 ub = make_float2(__uint_as_float(wb << 16), __uint_as_float(wb & 0xffff0000u));
+              v[q][0] = va ? ua.x - t1[nt + q][0] : 0.f; v[q][1] = va ? ua.y - t1[nt + q][1] : 0.f;
+              v[q][2] = vb ? ub.x - t1[nt + q][2] : 0.f; v[q][3] = vb ? ub.y - t1[nt + q][3] : 0.f;
+            }
+            const int n = cw0 + 8 * (nt + (mi >> 1));   // first column of this lane's matrix
+            const uint32_t off = (n >> 6) * 8192 + tok * 128 + ((((n & 63) >> 3) ^ (tok & 7)) << 4);
+            stmatrix_x4(sUt + off, pack_bf16(v[0][0], v[0][1]), pack_bf16(v[0][2], v[0][3]), pack_bf16(v[1][0], v[1][1]), pack_bf16(v[1][2], v[1][3]));
+            stmatrix_x4(sUd + off, pack_bf16(v[0][0] * da, v[0][1] * da), pack_bf16(v[0][2] * db, v[0][3] * db),
+                        pack_bf16(v[1][0] * da, v[1][1] * da), pack_bf16(v[1][2] * db, v[1][3] * db));
+          }
+          SUBPHASE(2 * lg + 1);
         }
-      }
-      fence_proxy_async();
-      tc_fence_before();
-      mbar_arrive(bar_ut);
-      PHASE(2);
-
-      // ---- P = (Q K^T) * decay, lower triangle with its diagonal (while K^T U~' runs); QS kept for the output
-      if (!mbar_wait_bounded(bar_o, ph)) { failed = true; break; }
-      tc_fence_after();
-      PHASE(3);
-      if (tid == 64 && has_next) issue_tile(sQ, &tmQ, bar_q, nx_tok0);   // Q's readers have retired
-      {
-        float qk[8][4];
-        tmem_ld_16x64(qk, tmem_rows + cfg::TM_QK);
-        tmem_ld_frag<NTL>(qs, tmem_rows + cfg::TM_QS);
-        tmem_wait_ld();
+        fence_proxy_async();
+        SUBPHASE(4);
+        tc_fence_before();
+        mbar_arrive(bar_ut);
+        SUBPHASE(5);
+        if (tid < C && has_next) store_g((c + 1) & 1, g_next);   // before new loads are issued: waiting for g must not wait for them
+        if (has_next) fetch_u(xr, nx_tok0, nx_rows);   // consumed one chunk from now
+        SUBPHASE(6);
+      } else {
+        // ---- P = (Q K^T) * decay, lower triangle with its diagonal; Q S kept for the output
         const float* cf = sCf + (c & 1) * C;
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-          const int j = 8 * nt + 2 * t;
-          uint32_t wa = 0u, wb = 0u;
-          if (8 * nt <= rb) {   // blocks right of both rows' diagonals are all zero
-            const float gref = gb[8 * nt];
-            const float2 cj = *reinterpret_cast<const float2*>(cf + j);
-            const float ea = ex2_approx(fminf(g_a - gref, 0.f)), eb = ex2_approx(g_b - gref);
-            const float p0 = j <= ra ? qk[nt][0] * ea * cj.x : 0.f, p1 = j + 1 <= ra ? qk[nt][1] * ea * cj.y : 0.f;
-            const float p2 = j <= rb ? qk[nt][2] * eb * cj.x : 0.f, p3 = j + 1 <= rb ? qk[nt][3] * eb * cj.y : 0.f;
-            wa = pack_bf16(p0, p1);
-            wb = pack_bf16(p2, p3);
+        for (int lg = 0; lg < 2; ++lg) {
+          float qk[4][4];   // this warp's half of the columns (tokens j): four blocks of eight
+          float qsf[NTW][4];
+          const uint32_t trow = tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_P1;
+          tmem_ld_16x32(qk, trow + DVS + 32 * half);
+          tmem_ld_frag<NTW>(qsf, trow + cw0);
+          tmem_wait_ld();
+          const int ia = tok_w + 16 * lg + gq, ib = ia + 8;
+          const float g_a = gb[ia], g_b = gb[ib];
+          {
+            // gamma_i Q S becomes the starting value of the PU accumulator (same lanes, same columns)
+            const float ya = ex2_approx(g_a), yb = ex2_approx(g_b);
+#pragma unroll
+            for (int nt = 0; nt < NTW; ++nt) { qsf[nt][0] *= ya; qsf[nt][1] *= ya; qsf[nt][2] *= yb; qsf[nt][3] *= yb; }
+            tmem_st_frag<NTW>(qsf, tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_PU + cw0);
           }
-          *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + ra * 128 + ((nt ^ (ra & 7)) << 4) + 4 * t) = wa;
-          *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + rb * 128 + ((nt ^ (rb & 7)) << 4) + 4 * t) = wb;
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int nt = 4 * half + q4;
+            const int j = 8 * nt + 2 * t;
+            uint32_t wa = 0u, wb = 0u;
+            if (8 * nt <= ib) {   // blocks right of both rows' diagonals are all zero
+              const float gref = gb[8 * nt];
+              const float2 cj = *reinterpret_cast<const float2*>(cf + j);
+              const float ea = ex2_approx(fminf(g_a - gref, 0.f)), eb = ex2_approx(g_b - gref);
+              const float p0 = j <= ia ? qk[q4][0] * ea * cj.x : 0.f, p1 = j + 1 <= ia ? qk[q4][1] * ea * cj.y : 0.f;
+              const float p2 = j <= ib ? qk[q4][2] * eb * cj.x : 0.f, p3 = j + 1 <= ib ? qk[q4][3] * eb * cj.y : 0.f;
+              wa = pack_bf16(p0, p1);
+              wb = pack_bf16(p2, p3);
+            }
+            *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + ia * 128 + ((nt ^ (ia & 7)) << 4) + 4 * t) = wa;
+            *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + ib * 128 + ((nt ^ (ib & 7)) << 4) + 4 * t) = wb;
+          }
         }
+        tmem_wait_st();
+        fence_proxy_async();
+        tc_fence_before();
+        mbar_arrive(bar_p);
+        o_tok0 = tok0; o_rows = rows;
       }
-      fence_proxy_async();
-      tc_fence_before();
-      mbar_arrive(bar_p);
-      o_sa = p.scale * ex2_approx(g_a); o_sb = p.scale * ex2_approx(g_b);
-      o_tok0 = tok0; o_rows = rows;
-      if (tid < C && has_next) store_g((c + 1) & 1, g_next);
-      PHASE(4);
+#ifdef TRI_INV_PHASE_CLOCKS
+      if (chain) { long long now = clock64(); if (blockIdx.x == 0 && tid == 0) atomicAdd(p.status + 127, (int)(now - ph_t)); }
+#endif
+      PHASE(2);
 
-      // ---- state update (thread = row of S) and the bf16 operand for the next chunk
+      // ---- state update and the bf16 operand for the next chunk
       if (!mbar_wait_bounded(bar_s, ph)) { failed = true; break; }
       tc_fence_after();
-      PHASE(5);
-      if (tid == 96 && has_next) issue_tile(sK, &tmK, bar_k, nx_tok0);   // K's readers (Q K^T, K^T U~') have retired
+      PHASE(3);
       {
         const float gl = ex2_approx(g_last);
 #pragma unroll
-        for (int n0 = 0; n0 < DVS; n0 += 32) {
-          float ds[32];
-          tmem_ld_32x32(ds, tmem_rows + cfg::TM_DS + n0);
+        for (int lg = 0; lg < 2; ++lg) {
+          float ds[NTW][4];
+          tmem_ld_frag<NTW>(ds, tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_DS + cw0);
           tmem_wait_ld();
 #pragma unroll
-          for (int n = 0; n < 32; ++n) S[n0 + n] = fmaf(gl, S[n0 + n], ds[n]);
+          for (int nt = 0; nt < NTW; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) S[lg][nt][e] = fmaf(gl, S[lg][nt][e], ds[nt][e]);
         }
         if (has_next) {
-          write_state_operand();   // its readers (W S, Q S of this chunk) retired before bar_s
+          write_state_operand();   // its reader (P1 of this chunk) retired before bar_t1
           fence_proxy_async();
           tc_fence_before();
           mbar_arrive(bar_sr);
         }
       }
-      PHASE(6);
+      PHASE(4);
       ph ^= 1;
     }
-    if (!failed && !misaligned && !write_output(ph ^ 1)) failed = true;
+    if (!chain && !failed && !misaligned && !write_output(ph ^ 1)) failed = true;
   }
   if (failed) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
   else store_state();
@@ -454,8 +561,8 @@ cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t
   return cudaSuccess;
 }
 
-// bf16 Q, K, W, U with d_k = d_v = 128 and C = 64.  32 value columns per CTA (two CTAs per SM) unless the batch
-// alone fills the GPU twice over, in which case 64 columns per CTA halve the re-reads of W, Q and K through L2.
+// bf16 Q, K, W, U with d_k = d_v = 128 and C = 64.  64 value columns per CTA (two CTAs per head) unless the batch
+// alone fills the GPU twice over, in which case one CTA per head does the same work in fewer, larger products.
 cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,
                               cudaStream_t stream) {
   CUtensorMap tmW, tmQ, tmK;
@@ -463,8 +570,8 @@ cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K,
     return cudaErrorUnknown;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if ((long long)p.n_seqs * p.H * 2 >= 2LL * sms) return launch_scan_one<64>(p, tmW, tmQ, tmK, stream);
-  return launch_scan_one<32>(p, tmW, tmQ, tmK, stream);
+  if ((long long)p.n_seqs * p.H >= 2LL * sms) return launch_scan_one<128>(p, tmW, tmQ, tmK, stream);
+  return launch_scan_one<64>(p, tmW, tmQ, tmK, stream);
 }
 
 }  // namespace tri_inv
