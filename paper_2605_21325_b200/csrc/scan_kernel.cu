@@ -35,13 +35,9 @@ namespace {
     if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(p.status + 8 + 12 * (threadIdx.x >> 5) + (k), (int)(now - ph_t)); \
     ph_t = now;                                                                   \
   } while (0)
-#define SUB_BEGIN() long long sub_t = clock64()
-#define SUBPHASE(k) do { long long now = clock64(); if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(p.status + 120 + (k), (int)(now - sub_t)); sub_t = now; } while (0)
 #else
 #define PHASE_BEGIN() do {} while (0)
 #define PHASE(k) do {} while (0)
-#define SUB_BEGIN() do {} while (0)
-#define SUBPHASE(k) do {} while (0)
 #endif
 
 constexpr int C = 64, D = 128, NT = 256;   // NT compute threads (8 warps) + one control warp
@@ -286,41 +282,26 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                      dPa = umma_desc(sKa + 8192, 16, 1024);              // 128 rows: second K box, then P
       uint32_t ph = 0;
       for (int c = 0; c < n_chunks; ++c) {
-#ifdef TRI_INV_PHASE_CLOCKS
-        long long ct = clock64();
-#define CSUB(k) do { long long now = clock64(); if (blockIdx.x == 0) atomicAdd(p.status + 110 + (k), (int)(now - ct)); ct = now; } while (0)
-#else
-#define CSUB(k) do {} while (0)
-#endif
-        if (!mbar_wait_bounded(bar_sr, ph)) { failed = true; break; }
-        CSUB(0);
-        if (!mbar_wait_bounded(bar_a, ph) || !mbar_wait_bounded(bar_kb, ph)) { failed = true; break; }
-        CSUB(1);
+        // the copies land long before the compute threads are done: check them first, S last
+        if (!mbar_wait_bounded(bar_a, ph) || !mbar_wait_bounded(bar_kb, ph) || !mbar_wait_bounded(bar_sr, ph)) { failed = true; break; }
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
           umma_bf16(tmem + cfg::TM_P1, dA + (((ks >> 2) * cfg::A_BOX + (ks & 3) * 32) >> 4),
                     dB + (((ks >> 2) * cfg::B_BOX + (ks & 3) * 32) >> 4), idesc_p1, ks > 0);
         umma_commit(bar_t1);
-        CSUB(2);
-        if (!mbar_wait_bounded(bar_ut, ph)) { failed = true; break; }
-        CSUB(3);
-        if (!mbar_wait_bounded(bar_ka, ph)) { failed = true; break; }
-        CSUB(4);
+        if (!mbar_wait_bounded(bar_ka, ph) || !mbar_wait_bounded(bar_ut, ph)) { failed = true; break; }
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < C / 16; ++ks)   // 16 tokens (2048 bytes of either operand) per step
           umma_bf16(tmem + cfg::TM_DS, dKa + ((ks * 2048) >> 4), dUd + ((ks * 2048) >> 4), idesc_p3, ks > 0);
         umma_commit(bar_s);
-        CSUB(5);
         if (!mbar_wait_bounded(bar_p, ph)) { failed = true; break; }
-        CSUB(6);
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < C / 16; ++ks)
           umma_bf16(tmem + cfg::TM_PU, dPa + ((ks * 32) >> 4), dUt + ((ks * 2048) >> 4), idesc_pu, 1u);   // on top of gamma_i Q S
         umma_commit(bar_pu);
-        CSUB(7);
         ph ^= 1;
       }
     }
@@ -388,13 +369,11 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       if (chain) {
         // ---- U~ = U - W S  ->  bf16 operands U~ and (decay-scaled) U~', [token rows][value columns]
         const int mi = lane >> 3, r = lane & 7;
-        SUB_BEGIN();
 #pragma unroll
         for (int lg = 0; lg < 2; ++lg) {
           float t1[NTW][4];
           tmem_ld_frag<NTW>(t1, tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_P1 + cw0);
           tmem_wait_ld();
-          SUBPHASE(2 * lg);
           const int i = tok_w + 16 * lg + gq;
           const float da = ex2_approx(g_last - gb[i]), db = ex2_approx(g_last - gb[i + 8]);
           const bool va = i < rows, vb = i + 8 < rows;
@@ -417,16 +396,12 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             stmatrix_x4(sUd + off, pack_bf16(v[0][0] * da, v[0][1] * da), pack_bf16(v[0][2] * db, v[0][3] * db),
                         pack_bf16(v[1][0] * da, v[1][1] * da), pack_bf16(v[1][2] * db, v[1][3] * db));
           }
-          SUBPHASE(2 * lg + 1);
         }
         fence_proxy_async();
-        SUBPHASE(4);
         tc_fence_before();
         mbar_arrive(bar_ut);
-        SUBPHASE(5);
         if (tid < C && has_next) store_g((c + 1) & 1, g_next);   // before new loads are issued: waiting for g must not wait for them
         if (has_next) fetch_u(xr, nx_tok0, nx_rows);   // consumed one chunk from now
-        SUBPHASE(6);
       } else {
         // ---- P = (Q K^T) * decay, lower triangle with its diagonal; Q S kept for the output
         const float* cf = sCf + (c & 1) * C;
@@ -471,9 +446,6 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         mbar_arrive(bar_p);
         o_tok0 = tok0; o_rows = rows;
       }
-#ifdef TRI_INV_PHASE_CLOCKS
-      if (chain) { long long now = clock64(); if (blockIdx.x == 0 && tid == 0) atomicAdd(p.status + 127, (int)(now - ph_t)); }
-#endif
       PHASE(2);
 
       // ---- state update and the bf16 operand for the next chunk
