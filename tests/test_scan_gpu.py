@@ -108,3 +108,55 @@ def test_chunk_scan_edge_cases(bnd):
     d = bnd.to_device(small)
     with pytest.raises(bnd.TriInvError):
         bnd.chunk_scan(d["K"], d["K"], d["K"], d["V"], d["g"], 64)
+
+
+# ---------------------------------------------------------------- full sizes, in the launch configuration bench.py times
+
+def test_layer_full_size_config2_sampled_and_restart(bnd):
+    inp = wl.config(2)
+    Q = wl.queries(inp, seed=4002)
+    dev = bnd.to_device(inp)
+    Qd = bnd.kv_to_torch(Q)
+    scale = 128 ** -0.5
+    O, S = bnd.gdn_forward(Qd, dev["K"], dev["V"], dev["beta"], dev["g"], 64, scale=scale)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    assert not bool(torch.isnan(O.float()).any())
+    # (a) the first 8 chunks of every sequence and head against the token-by-token recurrence
+    Ts = 512
+    O_ref, _ = oracle.gdn_recurrence(Q[:, :Ts], inp.K[:, :Ts], inp.V[:, :Ts], inp.beta[:, :Ts], inp.g[:, :Ts], 64, scale=scale)
+    assert max_ratio(bnd.to_numpy_f64(O[:, :Ts]), O_ref) <= TOL_LAYER
+    # (b) at any size: stopping after half the chunks and resuming from the returned state reproduces the
+    # second half of the outputs and the final state bit for bit (same arithmetic, same order)
+    half = inp.T // 2
+    first = [x[:, :half].contiguous() for x in (Qd, dev["K"], dev["V"], dev["beta"], dev["g"])]
+    second = [x[:, half:].contiguous() for x in (Qd, dev["K"], dev["V"], dev["beta"], dev["g"])]
+    O1, S1 = bnd.gdn_forward(*first, 64, scale=scale)
+    O2, S2 = bnd.gdn_forward(*second, 64, scale=scale, S0=S1)
+    torch.cuda.synchronize()
+    assert torch.equal(O1, O[:, :half]) and torch.equal(O2, O[:, half:]) and torch.equal(S2, S)
+    # (c) the last chunk of one sequence and head from the carried state, in fp64: one step of the chunk form
+    t0 = inp.T - 64
+    Wd, Ud = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], 64, method=bnd.W_DECAY, want_A=False)[1:]
+    _, S_prev = bnd.chunk_scan(Qd[:, :t0].contiguous(), dev["K"][:, :t0].contiguous(), Wd[:, :t0].contiguous(),
+                               Ud[:, :t0].contiguous(), dev["g"][:, :t0].contiguous(), 64, scale=scale)
+    torch.cuda.synchronize()
+    sl = slice(t0, inp.T)
+    O_last, S_last = oracle.chunk_scan(Q[:, sl], inp.K[:, sl], wl._store(Wd[:, sl].float().cpu().numpy(), wl.BF16),
+                                       wl._store(Ud[:, sl].float().cpu().numpy(), wl.BF16), inp.g[:, sl], 64, scale=scale,
+                                       S0=S_prev.cpu().numpy())
+    assert max_ratio(bnd.to_numpy_f64(O[:, sl]), O_last) <= TOL_SCAN
+    assert max_ratio(bnd.to_numpy_f64(S), S_last) <= TOL_SCAN
+
+
+def test_layer_full_size_config5_ragged(bnd):
+    inp = wl.config(5)
+    Q = wl.queries(inp, seed=4005)
+    dev = bnd.to_device(inp)
+    O, S = bnd.gdn_forward(bnd.kv_to_torch(Q), dev["K"], dev["V"], dev["beta"], dev["g"], 64, scale=128 ** -0.5,
+                           cu_seqlens=inp.cu_seqlens)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    O_ref, S_ref = oracle.gdn_recurrence(Q, inp.K, inp.V, inp.beta, inp.g, 64, scale=128 ** -0.5, cu_seqlens=inp.cu_seqlens)
+    assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= TOL_LAYER
+    assert max_ratio(bnd.to_numpy_f64(S), S_ref) <= TOL_LAYER
