@@ -163,11 +163,12 @@ int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A
  * W must be the decay-weighted factor (TRI_INV_W_DECAY of the fused calls), U the plain one.  With exact W and U
  * this equals the token-by-token recurrence  S <- exp(a_t) S;  S <- S + beta_t k_t (v_t - S^T k_t)^T;
  * o_t = scale S^T q_t.
- *   Q, K, W [B,T,H,d_k], U [B,T,H,d_v]: device, bf16, 16-byte aligned;  g [B,T,H] fp32 device;
+ *   Q, K, W [B,T,H,d_k], U [B,T,H,d_v]: device, desc->kv_dtype, 16-byte aligned;  g [B,T,H] fp32 device;
  *   S0, S_out [n_sequences,H,d_k,d_v] fp32 device, each may be NULL (zero initial state / final state not wanted);
- *   O [B,T,H,d_v] bf16 device: rows of real tokens are written.
- * Dense and ragged chunking as in tri_inv_build (desc->cu_seqlens on the HOST).  Supported: bf16,
- * d_k = d_v = 128, C = 64; anything else answers TRI_INV_ERR_UNSUPPORTED.  Launch is asynchronous on
+ *   O [B,T,H,d_v] device, desc->kv_dtype: rows of real tokens are written.
+ * Dense and ragged chunking as in tri_inv_build (desc->cu_seqlens on the HOST).  bf16 with d_k = d_v = 128 and
+ * C = 64 runs on the tensor cores; every other shape and fp32 storage run on the CUDA cores in fp32 (d_k <= 256,
+ * else TRI_INV_ERR_UNSUPPORTED).  Launch is asynchronous on
  * cuda_stream; nothing is allocated except, in ragged mode, n_sequences + 1 ints from the library's
  * stream-ordered pool.  A device-side wait that expires raises TRI_INV_ERR_DEVICE_TIMEOUT in the status word.
  */

@@ -233,7 +233,8 @@ int tri_inv_chunk_scan(const void* Q, const void* K, const void* W, const void* 
   if (!aligned16(Q) || !aligned16(K) || !aligned16(W) || !aligned16(U) || !aligned16(g) || !aligned16(O) || !aligned16(S0) ||
       !aligned16(S_out))
     return TRI_INV_ERR_INVALID_ARG;
-  if (desc->kv_dtype != TRI_INV_BF16 || desc->d_k != 128 || desc->d_v != 128 || desc->C != 64) return TRI_INV_ERR_UNSUPPORTED;
+  const bool tc = desc->kv_dtype == TRI_INV_BF16 && desc->d_k == 128 && desc->d_v == 128 && desc->C == 64;
+  if (!tc && desc->d_k > 256) return TRI_INV_ERR_UNSUPPORTED;   // the CUDA-core kernel keeps a d_k x 32 slice of S in shared memory
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   ScanParams p{};
   p.U = U; p.g = g; p.S0 = S0; p.O = O; p.S_out = S_out; p.scale = scale;
@@ -254,7 +255,8 @@ int tri_inv_chunk_scan(const void* Q, const void* K, const void* W, const void* 
     }
     p.seq_off = dev_off;
   }
-  err = launch_chunk_scan(p, Q, K, W, tokens > 0 ? tokens : 1, stream);
+  err = tc ? launch_chunk_scan(p, Q, K, W, tokens > 0 ? tokens : 1, stream)
+           : launch_chunk_scan_simt(p, Q, K, W, desc->d_k, desc->d_v, desc->C, desc->kv_dtype, stream);
   if (err == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);
   if (dev_off) cudaFreeAsync(dev_off, stream);
   return err == cudaSuccess ? TRI_INV_OK : TRI_INV_ERR_CUDA;

@@ -76,11 +76,11 @@ cudaError_t launch_simt(const KParams& p, int C, cudaStream_t stream);
 cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
 // Chunk scan (consumer of W and U): parameters other than the three TMA-staged tensors.
 struct ScanParams {
-  const void* U;        // [tokens,H,128] bf16
+  const void* U;        // [tokens,H,d_v]
   const float* g;       // [tokens,H]
-  const float* S0;      // [n_seqs,H,128,128] fp32 or null (zero state)
-  void* O;              // [tokens,H,128] bf16
-  float* S_out;         // [n_seqs,H,128,128] fp32 or null
+  const float* S0;      // [n_seqs,H,d_k,d_v] fp32 or null (zero state)
+  void* O;              // [tokens,H,d_v], storage type of U
+  float* S_out;         // [n_seqs,H,d_k,d_v] fp32 or null
   const int* seq_off;   // device copy of cu_seqlens (ragged) or null (dense: sequence s = tokens [s T, (s+1) T))
   int* status;
   int H, T, n_seqs;
@@ -89,6 +89,9 @@ struct ScanParams {
 cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t stream);
 cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,
                               cudaStream_t stream);
+// The same scan on the CUDA cores, for every other shape and storage type (fp32 arithmetic).
+cudaError_t launch_chunk_scan_simt(const ScanParams& p, const void* Q, const void* K, const void* W, int d_k, int d_v, int C,
+                                   int kv_dtype, cudaStream_t stream);
 // Per-channel decay variant on the tensor cores (bf16 keys, d_k = 128, C = 64, block recursion).
 cudaError_t launch_kda_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
 

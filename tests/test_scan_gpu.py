@@ -104,10 +104,48 @@ def test_chunk_scan_edge_cases(bnd):
     assert np.array_equal(S[0].cpu().numpy(), S0[0])
     _, S_ref = oracle.chunk_scan(Q, inp.K, Wb, Ub, inp.g, 64, S0=S0, cu_seqlens=cu)
     assert max_ratio(bnd.to_numpy_f64(S), S_ref) <= TOL_SCAN
-    small = wl.make("small", 1, 64, 1, 64, 64, 64, wl.BF16, seed=323)
-    d = bnd.to_device(small)
-    with pytest.raises(bnd.TriInvError):
-        bnd.chunk_scan(d["K"], d["K"], d["K"], d["V"], d["g"], 64)
+
+
+SIMT_CASES = [
+    ("cfg1_shape_fp32", 1, 256, 2, 64, 64, 64, wl.F32, None),
+    ("fp32_c128_partial", 2, 300, 2, 32, 96, 128, wl.F32, None),
+    ("fp32_c16_ragged", 1, 0, 3, 16, 40, 16, wl.F32, np.array([0, 5, 5, 37, 100], np.int32)),
+    ("bf16_d64_c32", 2, 100, 2, 64, 64, 32, wl.BF16, None),
+]
+
+
+@pytest.mark.parametrize("name,B,T,H,d_k,d_v,C,dtype,cu", SIMT_CASES, ids=[c[0] for c in SIMT_CASES])
+def test_chunk_scan_cuda_core_kernel_other_shapes(bnd, name, B, T, H, d_k, d_v, C, dtype, cu):
+    """fp32 storage and shapes outside the tensor-core kernel: fp32 arithmetic throughout, so the scan is held to
+    1e-5 of max|O| against its fp64 definition (bf16 storage: the output's own rounding, 2^-8)."""
+    if cu is not None:
+        T = int(cu[-1])
+    inp = wl.make(name, B, T, H, d_k, d_v, C, dtype, seed=330 + C, cu_seqlens=cu)
+    Q = wl.queries(inp, seed=331)
+    S0 = wl.initial_state(inp, seed=332)
+    A = oracle.build_A(inp.K, inp.beta, inp.g, C, cu_seqlens=cu)
+    Kg = oracle._widen(inp.K) * np.exp(inp.g.astype(np.float64))[..., None]
+    W64, _ = oracle.wy(A, Kg, None, inp.beta, C, cu_seqlens=cu)
+    _, U64 = oracle.wy(A, inp.K, inp.V, inp.beta, C, cu_seqlens=cu)
+    Ws, Us = wl._store(W64.astype(np.float32), dtype), wl._store(U64.astype(np.float32), dtype)
+    O_ref, S_ref = oracle.chunk_scan(Q, inp.K, Ws, Us, inp.g, C, scale=0.5, S0=S0, cu_seqlens=cu)
+    dev = bnd.to_device(inp)
+    O = torch.full((B, T, H, d_v), float("nan"), dtype=dev["V"].dtype, device="cuda")
+    O, S = bnd.chunk_scan(bnd.kv_to_torch(Q), dev["K"], bnd.kv_to_torch(Ws), bnd.kv_to_torch(Us), dev["g"], C, scale=0.5,
+                          S0=torch.from_numpy(S0).cuda(), cu_seqlens=cu, out=O)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    o = bnd.to_numpy_f64(O)
+    assert not np.isnan(o).any()
+    tol = 1e-5 if dtype == wl.F32 else 2.0 ** -8
+    assert max_ratio(o, O_ref) <= tol
+    assert max_ratio(bnd.to_numpy_f64(S), S_ref) <= 1e-5
+    if dtype == wl.F32:   # and the whole layer in fp32 through the CUDA-core kernels against the recurrence
+        O2, S2 = bnd.gdn_forward(bnd.kv_to_torch(Q), dev["K"], dev["V"], dev["beta"], dev["g"], C, scale=0.5,
+                                 S0=torch.from_numpy(S0).cuda(), cu_seqlens=cu)
+        torch.cuda.synchronize()
+        O_rec, S_rec = oracle.gdn_recurrence(Q, inp.K, inp.V, inp.beta, inp.g, C, scale=0.5, S0=S0, cu_seqlens=cu)
+        assert max_ratio(bnd.to_numpy_f64(O2), O_rec) <= 1e-5 and max_ratio(bnd.to_numpy_f64(S2), S_rec) <= 1e-5
 
 
 # ---------------------------------------------------------------- full sizes, in the launch configuration bench.py times
