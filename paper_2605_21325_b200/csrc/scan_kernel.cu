@@ -533,16 +533,13 @@ cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t
   return cudaSuccess;
 }
 
-// bf16 Q, K, W, U with d_k = d_v = 128 and C = 64.  64 value columns per CTA (two CTAs per head) unless the batch
-// alone fills the GPU twice over, in which case one CTA per head does the same work in fewer, larger products.
+// bf16 Q, K, W, U with d_k = d_v = 128 and C = 64: two CTAs per (sequence, head), 64 value columns each.  (One CTA
+// per head with 128 columns was measured too: the same time per unit of work, at a register count that spills.)
 cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,
                               cudaStream_t stream) {
   CUtensorMap tmW, tmQ, tmK;
   if (!make_tmap(&tmW, W, tokens, p.H, D, C, 2) || !make_tmap(&tmQ, Q, tokens, p.H, D, C, 2) || !make_tmap(&tmK, K, tokens, p.H, D, C, 2))
     return cudaErrorUnknown;
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if ((long long)p.n_seqs * p.H >= 2LL * sms) return launch_scan_one<128>(p, tmW, tmQ, tmK, stream);
   return launch_scan_one<64>(p, tmW, tmQ, tmK, stream);
 }
 

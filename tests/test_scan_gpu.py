@@ -44,7 +44,7 @@ CASES = [
     ("dense", 2, 5 * 64, 3, None, False),
     ("dense_partial_s0", 1, 3 * 64 + 17, 2, None, True),
     ("ragged_s0", 1, 0, 2, np.array([0, 64, 65, 65, 300, 531], np.int32), True),
-    ("many_heads_wide_slices", 5, 2 * 64, 64, None, True),   # 320 (sequence, head) pairs: the 64-column variant
+    ("many_heads", 5, 2 * 64, 64, None, True),   # 640 CTAs: several per SM in turn
 ]
 
 
