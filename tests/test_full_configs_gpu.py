@@ -130,3 +130,32 @@ def test_adversarial_keys_report(bnd):
             report[(inp.name, name)] = max_ratio(A.cpu().numpy(), A_ref)
         assert report[(inp.name, "block_recursive")] <= 2e-3, report
     print("adversarial keys, max ratio per method:", report)
+
+
+def test_per_channel_decay_full_size_config2_shape(bnd):
+    """tri_inv_build_kda on the shape of config 2 (4096 matrices, the launch bench.py --call kda times): structure on
+    every element, values on sampled chunks against the fp64 oracle, and -- at any size -- a gate that is the same
+    on every channel must reproduce tri_inv_build's matrices within the rounding of the two bf16 operand copies."""
+    inp = wl.config(2)
+    G = wl.per_channel_gate(inp, seed=3002)
+    dev = bnd.to_device(inp)
+    Gd = torch.from_numpy(G).cuda()
+    A = torch.full((inp.B, inp.T, inp.H, inp.C), float("nan"), dtype=torch.float32, device="cuda")
+    bnd.build_kda(dev["K"], Gd, dev["beta"], inp.C, out=A)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    device_structure_check(A, inp)
+    worst_a = worst_r = 0.0
+    for t0, t1 in sample_ranges(inp):
+        A_ref, N_ref = oracle.build_A_kda(inp.K[:, t0:t1], G[:, t0:t1], inp.beta[:, t0:t1], inp.C, return_N=True)
+        a = A[:, t0:t1].cpu().numpy()
+        worst_a = max(worst_a, max_ratio(a, A_ref))
+        sub = wl.Inputs("s", inp.B, t1 - t0, inp.H, inp.d_k, inp.d_v, inp.C, inp.kv_dtype, inp.K[:, t0:t1], inp.V[:, t0:t1],
+                        inp.beta[:, t0:t1], inp.g[:, t0:t1], None, {})
+        worst_r = max(worst_r, max_residual(a, N_ref, sub))
+    assert worst_a <= TOL_A[wl.BF16] and worst_r <= TOL_RES[wl.BF16], (worst_a, worst_r)
+    Gc = dev["g"].unsqueeze(-1).expand(-1, -1, -1, inp.d_k).contiguous()
+    A_same = bnd.build_kda(dev["K"], Gc, dev["beta"], inp.C)
+    A_scalar = bnd.build(dev["K"], dev["beta"], dev["g"], inp.C)
+    torch.cuda.synchronize()
+    assert float((A_same - A_scalar).abs().max()) <= 2e-3 * float(A_scalar.abs().max())
