@@ -432,18 +432,25 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         for (int s = 0; s <= R; ++s) {
           if (tid == 0) {
             tc_fence_after();
-            if (s < R) {
+            // Y = N^p with p = 2^s is zero within p of the diagonal: Y[i][k] needs k <= i - p, Y[k][j] needs
+            // k >= j + p.  Steps of eight k whose operands are structurally zero are not issued.
+            const int pw = 1 << s;
+            if (s < R) {   // Y.Y: k in [p, C-1-p]
+              const int k_lo = pw >> 3, k_hi = (C - 1 - pw) >> 3;
 #pragma unroll
               for (int ks = 0; ks < C / 8; ++ks) {
+                if (ks < k_lo || ks > k_hi) continue;
                 const uint32_t koff = (ks >> 2) * (C * 128) + (ks & 3) * 32;
-                umma_tf32(tmem, umma_desc(sYb + koff, 16, 1024), umma_desc(sYtb + koff, 16, 1024), idesc_s, ks > 0);
+                umma_tf32(tmem, umma_desc(sYb + koff, 16, 1024), umma_desc(sYtb + koff, 16, 1024), idesc_s, ks > k_lo);
               }
             }
-            if (s >= 1) {
+            if (s >= 1) {  // X.Y: k in [p, C-1]
+              const int k_lo = pw >> 3;
 #pragma unroll
               for (int ks = 0; ks < C / 8; ++ks) {
+                if (ks < k_lo) continue;
                 const uint32_t koff = (ks >> 2) * (C * 128) + (ks & 3) * 32;
-                umma_tf32(tmem + C, umma_desc(sXb + koff, 16, 1024), umma_desc(sYtb + koff, 16, 1024), idesc_s, ks > 0);
+                umma_tf32(tmem + C, umma_desc(sXb + koff, 16, 1024), umma_desc(sYtb + koff, 16, 1024), idesc_s, ks > k_lo);
               }
             }
             umma_commit(bar_mma);
