@@ -163,14 +163,15 @@ def build_kda(K, G, beta, C, method=BLOCK_RECURSIVE, cu_seqlens=None, out=None, 
     return A
 
 
-def chunk_scan(Q, K, W, U, g, C, scale=1.0, S0=None, cu_seqlens=None, out=None, want_state=True, stream=None):
+def chunk_scan(Q, K, W, U, g, C, scale=1.0, S0=None, cu_seqlens=None, out=None, want_state=True, state_out=None, stream=None):
     """O, S_final of the chunk form of the layer's recurrence from the decay-weighted W and U (tri_inv_chunk_scan)."""
     B, T, H, d_k = K.shape
     d_v = U.shape[3]
     desc, keep = make_desc(B, T, H, d_k, d_v, C, _dtype_code(K), cu_seqlens)
     n_seqs = B if cu_seqlens is None else len(cu_seqlens) - 1
     O = torch.empty((B, T, H, d_v), dtype=U.dtype, device=K.device) if out is None else out
-    S = torch.empty((n_seqs, H, d_k, d_v), dtype=torch.float32, device=K.device) if want_state else None
+    S = state_out if state_out is not None else (
+        torch.empty((n_seqs, H, d_k, d_v), dtype=torch.float32, device=K.device) if want_state else None)
     rc = load().tri_inv_chunk_scan(_p(Q), _p(K), _p(W), _p(U), _p(g), _p(S0), _p(O), _p(S), float(scale),
                                    ctypes.byref(desc), _stream(stream))
     if rc != OK:

@@ -199,3 +199,43 @@ def test_layer_full_size_config5_ragged(bnd):
     O_ref, S_ref = oracle.gdn_recurrence(Q, inp.K, inp.V, inp.beta, inp.g, 64, scale=128 ** -0.5, cu_seqlens=inp.cu_seqlens)
     assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= TOL_LAYER
     assert max_ratio(bnd.to_numpy_f64(S), S_ref) <= TOL_LAYER
+
+
+def test_layer_forward_captured_in_a_cuda_graph(bnd):
+    """Dense calls allocate nothing after their first use on a device: the two launches of the layer forward can be
+    captured once and replayed on new inputs written into the same buffers."""
+    inp = wl.make("graph", 2, 4 * 64, 4, 128, 128, 64, wl.BF16, seed=340)
+    Q = wl.queries(inp, seed=341)
+    dev = bnd.to_device(inp)
+    Qd = bnd.kv_to_torch(Q)
+    W, U, O = torch.empty_like(dev["K"]), torch.empty_like(dev["V"]), torch.empty_like(dev["V"])
+    S = torch.empty((2, 4, 128, 128), dtype=torch.float32, device="cuda")
+
+    def forward():
+        bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], 64, method=bnd.W_DECAY, out=(None, W, U))
+        bnd.chunk_scan(Qd, dev["K"], W, U, dev["g"], 64, scale=0.125, out=O, state_out=S)
+
+    forward()                       # first use: per-device set-up happens outside the capture
+    torch.cuda.synchronize()
+    O_eager, S_eager = O.clone(), S.clone()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            forward()
+    torch.cuda.synchronize()
+    O.zero_(); S.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    assert torch.equal(O, O_eager) and torch.equal(S, S_eager)
+    # new inputs in the same buffers: the replay computes the new result
+    inp2 = wl.make("graph2", 2, 4 * 64, 4, 128, 128, 64, wl.BF16, seed=342)
+    dev2 = bnd.to_device(inp2)
+    for k in ("K", "V", "beta", "g"):
+        dev[k].copy_(dev2[k])
+    graph.replay()
+    torch.cuda.synchronize()
+    O_ref, S_ref = oracle.gdn_recurrence(Q, inp2.K, inp2.V, inp2.beta, inp2.g, 64, scale=0.125)
+    assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= TOL_LAYER and max_ratio(bnd.to_numpy_f64(S), S_ref) <= TOL_LAYER
