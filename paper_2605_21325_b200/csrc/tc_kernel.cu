@@ -328,7 +328,10 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
       clear_tail_rows(k_now, v_now);
     }
     __syncthreads();
-    if (tid == kTidL2) *s_next_item = has_next ? 2 * (int)gridDim.x + atomicAdd(p.work_counter, 1) : total;  // the item after next
+    // the item after next: the ticket is drawn now and used after the inversion, so that its round trip to
+    // global memory does not hold this warp (and, at the next barrier, the CTA)
+    int ticket = 0;
+    if (tid == kTidL2 && has_next) ticket = atomicAdd(p.work_counter, 1);
     PHASE(0);
 
     if (!load_a) {
@@ -617,6 +620,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         if (!do_wy && a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
       }
     }
+    if (tid == kTidL2) *s_next_item = has_next ? 2 * (int)gridDim.x + ticket : total;  // read after this item's last barrier
     PHASE(6);
 
     if (do_wy) {
