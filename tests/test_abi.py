@@ -79,3 +79,25 @@ def test_null_and_misaligned_pointers_rejected_before_any_device_work(lib):
     assert L.tri_inv_wy(ok, ok, ok, ok, ok, None, p, None) == binding.ERR_INVALID_ARG   # V without U
     assert L.tri_inv_fused(ok, None, ok, ok, ok, ok, ok, p, 0, None) == binding.ERR_INVALID_ARG
     assert binding.launch_count() == 0 or binding.launch_count() > 0   # callable without a device
+
+
+def test_newer_entry_points_validate_on_the_host(lib):
+    L, binding = lib
+    d, _ = binding.make_desc(1, 64, 1, 128, 128, 64, binding.BF16)
+    p = ctypes.byref(d)
+    ok = ctypes.c_void_p(4096)
+    odd = ctypes.c_void_p(4100)
+    # per-channel decay build
+    assert L.tri_inv_build_kda(ok, None, ok, ok, p, 0, None) == binding.ERR_INVALID_ARG
+    assert L.tri_inv_build_kda(ok, odd, ok, ok, p, 0, None) == binding.ERR_INVALID_ARG
+    assert L.tri_inv_build_kda(ok, ok, ok, ok, p, binding.W_DECAY, None) == binding.ERR_UNSUPPORTED   # no W to weight
+    # decay-weighted W is a fused-call option only
+    assert L.tri_inv_build(ok, ok, ok, ok, p, binding.W_DECAY, None) == binding.ERR_UNSUPPORTED
+    # chunk scan: Q, K, W, U, g, O are required; S0 and S_out are optional but must be aligned when given
+    scale = ctypes.c_float(1.0)
+    assert L.tri_inv_chunk_scan(None, ok, ok, ok, ok, None, ok, None, scale, p, None) == binding.ERR_INVALID_ARG
+    assert L.tri_inv_chunk_scan(ok, ok, ok, ok, ok, None, None, None, scale, p, None) == binding.ERR_INVALID_ARG
+    assert L.tri_inv_chunk_scan(ok, ok, ok, ok, ok, odd, ok, None, scale, p, None) == binding.ERR_INVALID_ARG
+    assert L.tri_inv_chunk_scan(ok, ok, ok, ok, ok, None, ok, None, scale, None, None) == binding.ERR_INVALID_ARG
+    wide, _ = binding.make_desc(1, 64, 1, 512, 64, 64, binding.F32)      # d_k beyond the CUDA-core scan's state slice
+    assert L.tri_inv_chunk_scan(ok, ok, ok, ok, ok, None, ok, None, scale, ctypes.byref(wide), None) == binding.ERR_UNSUPPORTED
