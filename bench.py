@@ -200,8 +200,10 @@ def main():
     ap.add_argument("--paper-T", type=int, default=0,
                     help="instead of --config: the paper's timing shape B=32, H=4, d=128 at this sequence length (1024..16384)")
     ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw", "kda", "scan", "layer"],
-                    help="entry point timed: the fused path (default, the metric), tri_inv_build alone, tri_inv_wy alone, or "
-                         "tri_inv_fused_raw (front end folded in; same shapes, un-normalised keys and logits as inputs)")
+                    help="entry point timed: the fused path (default, the metric), tri_inv_build alone, tri_inv_wy alone, "
+                         "tri_inv_fused_raw (front end folded in; same shapes, un-normalised keys and logits as inputs), "
+                         "tri_inv_build_kda (per-channel decay), tri_inv_chunk_scan alone (W and U produced outside the timed "
+                         "region), or the layer forward (fused call with decay-weighted W, then the scan)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-flush", action="store_true", help="skip the L2 flush between steps (profiling runs)")
