@@ -333,6 +333,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     int ticket = 0;
     if (tid == kTidL2 && has_next) ticket = atomicAdd(p.work_counter, 1);
     PHASE(0);
+    // build only: nothing later in the item hides this load, so it is issued now (the element is in L2 already)
+    if (BO && has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);
 
     if (!load_a) {
       // ---- 2. Gram S = K K^T on the tensor core: one thread issues D/16 MMAs of C x C x 16 into TMEM
@@ -737,7 +739,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
       }
     } else {
       // build only: the fp32 matrix has been read by everyone after this barrier
-      if (has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);
+      if (!BO && has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);
       tc_fence_before();
       __syncthreads();
       ph_k ^= 1;
