@@ -259,12 +259,12 @@ def fused_packed_static(K, V, beta, g, C, cu_seqlens, method=BLOCK_RECURSIVE, ou
 class HostPipeline:
     """tri_inv_fused for callers whose tensors live in pinned host memory.
 
-    The batch is cut into slices (whole sequences when B >= n_slices, else whole chunks of one sequence) and
+    The batch is cut into slices (whole sequences when B >= n_slices, else runs of whole chunks of one sequence) and
     each slice goes host -> device, through the fused kernel, and device -> host on its own stream, so the
     upload of one slice overlaps the kernel of the previous one and the download of the one before.  Device
     buffers are allocated once here; ``run`` allocates nothing.  Dense mode only (packed batches: one slice)."""
 
-    def __init__(self, B, T, H, d_k, d_v, C, dtype=torch.bfloat16, n_slices=4, n_streams=3, cu_seqlens=None, device="cuda"):
+    def __init__(self, B, T, H, d_k, d_v, C, dtype=torch.bfloat16, n_slices=8, n_streams=3, cu_seqlens=None, device="cuda"):
         self.shape = (B, T, H, d_k, d_v, C)
         self.cu_seqlens = cu_seqlens
         self.K = torch.empty((B, T, H, d_k), dtype=dtype, device=device)
@@ -273,21 +273,22 @@ class HostPipeline:
         self.g = torch.empty((B, T, H), dtype=torch.float32, device=device)
         self.A = torch.empty((B, T, H, C), dtype=torch.float32, device=device)
         self.W, self.U = torch.empty_like(self.K), torch.empty_like(self.V)
-        if cu_seqlens is not None:
-            self.slices = [(0, slice(None))]                      # axis, range
+        # a slice is (sequence range, token range): whole sequences, or a run of whole chunks of one sequence --
+        # either way a contiguous block of every tensor
+        if cu_seqlens is not None or B * (T // C) < 2:
+            self.slices = [(slice(None), slice(None))]
         elif B >= n_slices:
             step = -(-B // n_slices)
-            self.slices = [(0, slice(b, min(b + step, B))) for b in range(0, B, step)]
-        elif B == 1 and T >= n_slices * C:
-            step = -(-(T // C) // n_slices) * C
-            self.slices = [(1, slice(t, min(t + step, T))) for t in range(0, T, step)]
+            self.slices = [(slice(b, min(b + step, B)), slice(None)) for b in range(0, B, step)]
         else:
-            self.slices = [(0, slice(None))]
+            per_seq = max(1, min(n_slices // B, T // C))
+            step = -(-(T // C) // per_seq) * C
+            self.slices = [(slice(b, b + 1), slice(t, min(t + step, T))) for b in range(B) for t in range(0, T, step)]
         self.streams = [torch.cuda.Stream(device=device) for _ in range(min(n_streams, len(self.slices)))]
 
     @staticmethod
-    def _cut(t, axis, rng):
-        return t[rng] if axis == 0 else t[:, rng]
+    def _cut(t, brng, trng):
+        return t[brng, trng]
 
     def run(self, hK, hV, hbeta, hg, hA, hW, hU, method=BLOCK_RECURSIVE):
         """All arguments are pinned host tensors of the full batch; hA may be None.  Returns after enqueueing;
@@ -296,11 +297,11 @@ class HostPipeline:
         cur = torch.cuda.current_stream()
         start = torch.cuda.Event()
         start.record(cur)
-        for n, (axis, rng) in enumerate(self.slices):
+        for n, (brng, trng) in enumerate(self.slices):
             st = self.streams[n % len(self.streams)]
             st.wait_event(start)
             with torch.cuda.stream(st):
-                cut = lambda t: self._cut(t, axis, rng)
+                cut = lambda t: self._cut(t, brng, trng)
                 for dst, src in ((self.K, hK), (self.V, hV), (self.beta, hbeta), (self.g, hg)):
                     cut(dst).copy_(cut(src), non_blocking=True)
                 fused(cut(self.K), cut(self.V), cut(self.beta), cut(self.g), C, method=method, cu_seqlens=self.cu_seqlens,
