@@ -610,6 +610,17 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         if (a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
         if (do_wy) put_ap(i, j, v);
       }
+    } else if constexpr (BO) {
+      // Build only: A leaves straight from shared memory, one 256-byte bulk copy per row (no trip through
+      // registers and the load/store pipe, which is what bounds this variant).  The matrix is complete in
+      // shared memory: +0.0 above the diagonal, 1.0f on it.  Rows past the sequence end are not copied.
+      fence_proxy_async();   // the merges' stores become visible to the copy engine
+      __syncthreads();
+      if ((p.ops & kStoreA) && p.A && tid < rows) {
+        float* dst = p.A + ((size_t)(tok0 + tid) * p.H + h) * C;
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(sX + tid * LD)), "r"(C * 4) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
     } else {
 #pragma unroll
       for (int m = 0; m < NV; ++m) {
@@ -740,6 +751,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     } else {
       // build only: the fp32 matrix has been read by everyone after this barrier
       if (!BO && has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);
+      if (BO && tid < C) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // the copies have read their rows
       tc_fence_before();
       __syncthreads();
       ph_k ^= 1;
