@@ -475,3 +475,41 @@ def test_w_decay_is_refused_where_there_is_no_w(bnd):
     dev = bnd.to_device(inp)
     with pytest.raises(bnd.TriInvError):
         bnd.build(dev["K"], dev["beta"], dev["g"], inp.C, method=bnd.BLOCK_RECURSIVE | bnd.W_DECAY)
+
+
+# ---------------------------------------------------------------- re-entrancy
+def test_concurrent_calls_from_two_host_threads_on_two_streams(bnd):
+    """The library is re-entrant: launches that overlap on different streams, issued by different host threads,
+    neither share a work counter nor disturb each other's results (bit-exact against the serial runs)."""
+    import threading
+    cases = []
+    for seed, cu in ((501, None), (502, np.array([0, 300, 301, 900], np.int32))):
+        B, T = (2, 8 * 64) if cu is None else (1, int(cu[-1]))
+        inp = wl.make("mt", B, T, 8, 128, 128, 64, wl.BF16, seed=seed, cu_seqlens=cu)
+        dev = bnd.to_device(inp)
+        ref = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], 64, cu_seqlens=cu)
+        cases.append((inp, dev, cu, ref))
+    torch.cuda.synchronize()
+    errors = []
+
+    def worker(k):
+        try:
+            inp, dev, cu, ref = cases[k]
+            st = torch.cuda.Stream()
+            with torch.cuda.stream(st):
+                for _ in range(25):
+                    A, W, U = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], 64, cu_seqlens=cu, stream=st)
+            st.synchronize()
+            if not (torch.equal(A, ref[0]) and torch.equal(W, ref[1]) and torch.equal(U, ref[2])):
+                errors.append("thread %d: results differ from the serial run" % k)
+        except Exception as e:  # noqa: BLE001
+            errors.append(repr(e))
+
+    threads = [threading.Thread(target=worker, args=(k,)) for k in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    assert bnd.last_device_status() == 0
