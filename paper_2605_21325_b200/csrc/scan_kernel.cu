@@ -65,13 +65,6 @@ struct ScanCfg {
   static constexpr int CTAS_PER_SM = 1;   // registers: 9 warps at the kernel's natural register count fill an SM once
 };
 
-__device__ __forceinline__ void tmem_ld_16x32(float (&r)[4][4], uint32_t taddr) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=f"(r[0][0]), "=f"(r[0][1]), "=f"(r[0][2]), "=f"(r[0][3]), "=f"(r[1][0]), "=f"(r[1][1]), "=f"(r[1][2]), "=f"(r[1][3]),
-        "=f"(r[2][0]), "=f"(r[2][1]), "=f"(r[2][2]), "=f"(r[2][3]), "=f"(r[3][0]), "=f"(r[3][1]), "=f"(r[3][2]), "=f"(r[3][3])
-      : "r"(taddr));
-}
 template <int NTL>
 __device__ __forceinline__ void tmem_ld_frag(float (&r)[NTL][4], uint32_t taddr) {
   if constexpr (NTL == 8) tmem_ld_16x64(r, taddr);

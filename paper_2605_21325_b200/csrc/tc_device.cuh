@@ -300,6 +300,14 @@ __device__ __forceinline__ void tmem_ld_16x64(float (&r)[8][4], uint32_t taddr) 
         "=f"(r[6][0]), "=f"(r[6][1]), "=f"(r[6][2]), "=f"(r[6][3]), "=f"(r[7][0]), "=f"(r[7][1]), "=f"(r[7][2]), "=f"(r[7][3])
       : "r"(taddr));
 }
+// 16 lanes x 32 columns -> 4 n-tiles of accumulator fragments.
+__device__ __forceinline__ void tmem_ld_16x32(float (&r)[4][4], uint32_t taddr) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=f"(r[0][0]), "=f"(r[0][1]), "=f"(r[0][2]), "=f"(r[0][3]), "=f"(r[1][0]), "=f"(r[1][1]), "=f"(r[1][2]), "=f"(r[1][3]),
+        "=f"(r[2][0]), "=f"(r[2][1]), "=f"(r[2][2]), "=f"(r[2][3]), "=f"(r[3][0]), "=f"(r[3][1]), "=f"(r[3][2]), "=f"(r[3][3])
+      : "r"(taddr));
+}
 // 16 lanes x 128 columns -> 16 n-tiles of accumulator fragments.
 __device__ __forceinline__ void tmem_ld_16x128(float (&r)[16][4], uint32_t taddr) {
   asm volatile(

@@ -581,7 +581,100 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
       merge_level<C, 16>(sX, warp, lane);
       PHASE(4);
       merge_level<C, 32>(sX, warp, lane);
-      if constexpr (C == 128) merge_level<C, 64>(sX, warp, lane);
+      if constexpr (C == 128 && cfg::ALIAS) {
+        // Top level at C = 128, X21 = -A22 . N21 . A11 with 64 x 64 blocks, as two tcgen05.mma (kind::tf32) products
+        // instead of about 650 warp-level MMAs per matrix on the legacy pipe, which two resident CTAs share.
+        // Operands (fp32 rounded to TF32, K-major, 128-byte swizzle, two blocks of 32 columns) live in the A' space,
+        // idle until the inversion is done: first N21 and A11^T, then A22 and T^T; accumulators in tensor memory.
+        auto canon64 = [](int r, int c) -> uint32_t {
+          return (uint32_t)((c >> 5) * 8192 + r * 128 + (((((c & 31) >> 2) ^ (r & 7)) << 4) | ((c & 3) * 4)));
+        };
+        uint8_t* opa = smem + cfg::OFF_AP;
+        uint8_t* opb = opa + 16384;
+        constexpr uint32_t idesc_m = umma_idesc_tf32(64, 64, 0);
+        auto copy_block = [&](uint8_t* dst, int r0, int c0) {   // 64 x 64 block of the matrix, row-major -> operand layout
+#pragma unroll
+          for (int m = 0; m < 4; ++m) {
+            const int e = tid + m * cfg::NT, i = e >> 4, k4 = (e & 15) * 4;
+            const float4 v = *reinterpret_cast<const float4*>(sX + (r0 + i) * LD + c0 + k4);
+            uint4 w;
+            w.x = to_tf32(v.x); w.y = to_tf32(v.y); w.z = to_tf32(v.z); w.w = to_tf32(v.w);
+            *reinterpret_cast<uint4*>(dst + canon64(i, k4)) = w;
+          }
+        };
+        auto issue_merge = [&](uint32_t d_col) {
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t koff = (ks >> 2) * 8192 + (ks & 3) * 32;
+            umma_tf32(tmem + d_col, umma_desc(sAp + koff, 16, 1024), umma_desc(sAp + 16384 + koff, 16, 1024), idesc_m, ks > 0);
+          }
+          umma_commit(bar_mma);
+        };
+        const int mq = warp & 3, mh = warp >> 2;           // tensor-memory quadrant (16 rows of an M = 64 result) and column half
+        const uint32_t tm_m = tmem + ((uint32_t)(32 * mq) << 16) + 32 * mh;
+        // product 1: T = N21 . A11  (A = N21 as stored; B = A11^T: element (n, k) = A11[k][n])
+        copy_block(opa, 64, 0);
+        {
+          const int nn = lane & 7, kk = lane >> 3;         // an 8 (n) x 4 (k) patch per warp and step: conflict-free stores
+          float av[16];
+#pragma unroll
+          for (int m = 0; m < 16; ++m) {
+            const int patch = warp * 16 + m;
+            av[m] = sX[(4 * (patch >> 3) + kk) * LD + 8 * (patch & 7) + nn];
+          }
+#pragma unroll
+          for (int m = 0; m < 16; ++m) {
+            const int patch = warp * 16 + m, n = 8 * (patch & 7) + nn, k = 4 * (patch >> 3) + kk;
+            *reinterpret_cast<uint32_t*>(opb + canon64(n, k)) = to_tf32(av[m]);
+          }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) { tc_fence_after(); issue_merge(0); }
+        if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+        ph_mma ^= 1;
+        tc_fence_after();
+        // product 2: X21 = -(A22 . T)  (A = A22; B = T^T: element (n, k) = T[k][n], from this thread's fragments)
+        {
+          float tf[4][4];
+          tmem_ld_16x32(tf, tm_m);
+          tmem_wait_ld();
+          copy_block(opa, 64, 64);
+          const int ka = 16 * mq + g, kb = ka + 8;
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt) {
+            const int n = 32 * mh + 8 * nt + 2 * t;
+            *reinterpret_cast<uint32_t*>(opb + canon64(n, ka)) = to_tf32(tf[nt][0]);
+            *reinterpret_cast<uint32_t*>(opb + canon64(n + 1, ka)) = to_tf32(tf[nt][1]);
+            *reinterpret_cast<uint32_t*>(opb + canon64(n, kb)) = to_tf32(tf[nt][2]);
+            *reinterpret_cast<uint32_t*>(opb + canon64(n + 1, kb)) = to_tf32(tf[nt][3]);
+          }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) { tc_fence_after(); issue_merge(64); }
+        if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+        ph_mma ^= 1;
+        tc_fence_after();
+        {
+          float xf[4][4];
+          tmem_ld_16x32(xf, tm_m + 64);
+          tmem_wait_ld();
+          const int ia = 64 + 16 * mq + g, ib = ia + 8;
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt) {
+            const int c = 32 * mh + 8 * nt + 2 * t;
+            *reinterpret_cast<float2*>(sX + ia * LD + c) = make_float2(-xf[nt][0], -xf[nt][1]);
+            *reinterpret_cast<float2*>(sX + ib * LD + c) = make_float2(-xf[nt][2], -xf[nt][3]);
+          }
+        }
+        tc_fence_before();
+        __syncthreads();
+      } else if constexpr (C == 128) {
+        merge_level<C, 64>(sX, warp, lane);
+      }
       PHASE(5);
       }
     }
