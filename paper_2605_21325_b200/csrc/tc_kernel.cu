@@ -694,7 +694,11 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     };
     float4 xv[cfg::ALIAS ? 1 : NV];
     if constexpr (cfg::ALIAS) {
-      // A' has a region of its own: one pass reads the matrix, stores A and writes A'
+      // A' has a region of its own: one pass reads the matrix (8 rows per step), stores A and writes A'.  K and V come
+      // back into the matrix's space box by box as the pass frees it: a 16 KB box covers 31 rows of the matrix, so
+      // K's boxes are requested after rows 0..31 and 0..63, V's first after rows 0..95 and its second after the pass.
+      static_assert(C != 128 || (cfg::NT == 256 && LD * 4 * 32 >= cfg::BOX_BYTES && LD * 4 * 31 <= cfg::BOX_BYTES),
+                    "the box-by-box reload assumes 8 rows per step and 31 to 32 matrix rows per box");
 #pragma unroll
       for (int m = 0; m < NV; ++m) {
         const int e = tid + m * cfg::NT;
@@ -702,6 +706,19 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         const float4 v = *reinterpret_cast<const float4*>(sX + i * LD + j);
         if (a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
         if (do_wy) put_ap(i, j, v);
+        if (C == 128 && do_wy && (m == 3 || m == 7 || m == 11)) {
+          fence_proxy_async();
+          __syncthreads();   // rows 0 .. 8 m + 7 have been read by everyone
+          if (m == 3 && tid == kTidK) {
+            mbar_expect_tx(bar_k, (uint32_t)cfg::TILE_BYTES);
+            tma_load_2d(sK, &tmK, bar_k, h * D, tok0);
+          }
+          if (m == 7 && tid == kTidK) tma_load_2d(sK + cfg::BOX_BYTES, &tmK, bar_k, h * D + 64, tok0);
+          if (m == 11 && tid == kTidV && need_v) {
+            mbar_expect_tx(bar_v, (uint32_t)cfg::TILE_BYTES);
+            tma_load_2d(sV, &tmV, bar_v, h * D, tok0);
+          }
+        }
       }
     } else if constexpr (BO) {
       // Build only: A leaves straight from shared memory, one 256-byte bulk copy per row (no trip through
@@ -733,9 +750,13 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
       if constexpr (cfg::ALIAS) {
         fence_proxy_async();
         tc_fence_before();
-        __syncthreads();  // the fp32 matrix has been read by everyone: K and V may land in its space
-        if (tid == kTidK) issue_k(tok0, h);
-        if (tid == kTidV && need_v) issue_v(tok0, h);
+        __syncthreads();  // the fp32 matrix has been read by everyone: the last box may land in its space
+        if (C == 128) {
+          if (tid == kTidV && need_v) tma_load_2d(sV + cfg::BOX_BYTES, &tmV, bar_v, h * D + 64, tok0);
+        } else {
+          if (tid == kTidK) issue_k(tok0, h);
+          if (tid == kTidV && need_v) issue_v(tok0, h);
+        }
         if (!load_a) ph_k ^= 1;  // second K copy of this item
         if (!finish_reload()) { failed = true; break; }
       } else {
