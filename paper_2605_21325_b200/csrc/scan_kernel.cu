@@ -423,7 +423,8 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             if (8 * nt <= ib) {   // blocks right of both rows' diagonals are all zero
               const float gref = gb[8 * nt];
               const float2 cj = *reinterpret_cast<const float2*>(cf + j);
-              const float ea = ex2_approx(fminf(g_a - gref, 0.f)), eb = ex2_approx(g_b - gref);
+              // (row a may lie above this block altogether: its entries are masked, the exponent is not formed)
+              const float ea = ex2_approx(8 * nt <= ia ? g_a - gref : 0.f), eb = ex2_approx(g_b - gref);
               const float p0 = j <= ia ? qk[q4][0] * ea * cj.x : 0.f, p1 = j + 1 <= ia ? qk[q4][1] * ea * cj.y : 0.f;
               const float p2 = j <= ib ? qk[q4][2] * eb * cj.x : 0.f, p3 = j + 1 <= ib ? qk[q4][3] * eb * cj.y : 0.f;
               wa = pack_bf16(p0, p1);

@@ -239,3 +239,28 @@ def test_layer_forward_captured_in_a_cuda_graph(bnd):
     torch.cuda.synchronize()
     O_ref, S_ref = oracle.gdn_recurrence(Q, inp2.K, inp2.V, inp2.beta, inp2.g, 64, scale=0.125)
     assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= TOL_LAYER and max_ratio(bnd.to_numpy_f64(S), S_ref) <= TOL_LAYER
+
+
+def test_chunk_scan_with_a_gate_that_is_not_monotone(bnd):
+    """g is taken as given: nothing in the scan assumes that it decreases along the chunk."""
+    inp = wl.make("anyg", 2, 3 * 64 + 5, 2, 128, 128, 64, wl.BF16, seed=350)
+    rng = np.random.default_rng(351)
+    g = (0.5 * rng.standard_normal(inp.g.shape)).astype(np.float32)          # rises and falls, |differences| of a few units
+    Q = wl.queries(inp, seed=352)
+    A = oracle.build_A(inp.K, inp.beta, g, 64)
+    Kg = oracle._widen(inp.K) * np.exp(g.astype(np.float64))[..., None]
+    W64, _ = oracle.wy(A, Kg, None, inp.beta, 64)
+    _, U64 = oracle.wy(A, inp.K, inp.V, inp.beta, 64)
+    Wb, Ub = to_bf16_bits(W64), to_bf16_bits(U64)
+    O_ref, S_ref = oracle.chunk_scan(Q, inp.K, Wb, Ub, g, 64, scale=0.3)
+    dev = bnd.to_device(inp)
+    O, S = bnd.chunk_scan(bnd.kv_to_torch(Q), dev["K"], bnd.kv_to_torch(Wb), bnd.kv_to_torch(Ub), torch.from_numpy(g).cuda(), 64, scale=0.3)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= TOL_SCAN and max_ratio(bnd.to_numpy_f64(S), S_ref) <= TOL_SCAN
+    # and the fused call with the same gate feeds it consistently (decay-weighted W from the kernel)
+    gd = torch.from_numpy(g).cuda()
+    O2, S2 = bnd.gdn_forward(bnd.kv_to_torch(Q), dev["K"], dev["V"], dev["beta"], gd, 64, scale=0.3)
+    torch.cuda.synchronize()
+    O_rec, S_rec = oracle.gdn_recurrence(Q, inp.K, inp.V, inp.beta, g, 64, scale=0.3)
+    assert max_ratio(bnd.to_numpy_f64(O2), O_rec) <= TOL_LAYER and max_ratio(bnd.to_numpy_f64(S2), S_rec) <= TOL_LAYER
