@@ -168,7 +168,9 @@ int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A
  *   O [B,T,H,d_v] device, desc->kv_dtype: rows of real tokens are written.
  * Dense and ragged chunking as in tri_inv_build (desc->cu_seqlens on the HOST).  bf16 with d_k = d_v = 128 and
  * C = 64 runs on the tensor cores; every other shape and fp32 storage run on the CUDA cores in fp32 (d_k <= 256,
- * else TRI_INV_ERR_UNSUPPORTED).  Launch is asynchronous on
+ * else TRI_INV_ERR_UNSUPPORTED).  g is used as given (it need not decrease); the tensor-core path forms exp(g_i - g_j)
+ * as a product of two factors around the first token of j's block of eight, so g may vary by at most about 88
+ * inside eight consecutive tokens of a chunk.  Launch is asynchronous on
  * cuda_stream; nothing is allocated except, in ragged mode, n_sequences + 1 ints from the library's
  * stream-ordered pool.  A device-side wait that expires raises TRI_INV_ERR_DEVICE_TIMEOUT in the status word.
  */
