@@ -513,3 +513,38 @@ def test_concurrent_calls_from_two_host_threads_on_two_streams(bnd):
     torch.cuda.synchronize()
     assert not errors, errors
     assert bnd.last_device_status() == 0
+
+
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_layouts_fused_all_methods(bnd, seed):
+    """Seeded random batch layouts (dense and packed, ragged ends, empty sequences), both chunk sizes, every scheme:
+    within tolerance of the oracle and bit-identical from run to run."""
+    rng = np.random.default_rng(seed)
+    for it in range(10):
+        C = int(rng.choice([64, 128]))
+        H = int(rng.integers(1, 7))
+        if rng.random() < 0.5:
+            n = int(rng.integers(1, 6))
+            lens = rng.integers(0, 5 * C, size=n)
+            lens[rng.integers(0, n)] += 1
+            cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+            B, T = 1, int(cu[-1])
+        else:
+            cu, B, T = None, int(rng.integers(1, 4)), int(rng.integers(1, 6 * C))
+        inp = wl.make("rand", B, T, H, 128, 128, C, wl.BF16, seed=int(rng.integers(1 << 30)), cu_seqlens=cu)
+        dev = bnd.to_device(inp)
+        A_ref, N_ref = oracle.build_A(inp.K, inp.beta, inp.g, C, cu_seqlens=cu, return_N=True)
+        W_ref, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, C, cu_seqlens=cu)
+        for m in (bnd.BLOCK_RECURSIVE, bnd.BLOCK_RECURSIVE | bnd.LEAF_SERIES, bnd.PRODUCT_SERIES):
+            runs = []
+            for _ in range(2):
+                A = nan_like((B, T, H, C), torch.float32)
+                W, U = nan_like(dev["K"].shape, dev["K"].dtype), nan_like(dev["V"].shape, dev["V"].dtype)
+                bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], C, method=m, cu_seqlens=cu, out=(A, W, U))
+                torch.cuda.synchronize()
+                runs.append((A, W, U))
+            assert bnd.last_device_status() == 0
+            assert all(torch.equal(x, y) for x, y in zip(runs[0], runs[1]))
+            check_A(runs[0][0], inp, A_ref, N_ref)
+            assert max_ratio(bnd.to_numpy_f64(runs[0][1]), W_ref) <= TOL_WY[wl.BF16]
+            assert max_ratio(bnd.to_numpy_f64(runs[0][2]), U_ref) <= TOL_WY[wl.BF16]

@@ -264,3 +264,38 @@ def test_chunk_scan_with_a_gate_that_is_not_monotone(bnd):
     torch.cuda.synchronize()
     O_rec, S_rec = oracle.gdn_recurrence(Q, inp.K, inp.V, inp.beta, g, 64, scale=0.3)
     assert max_ratio(bnd.to_numpy_f64(O2), O_rec) <= TOL_LAYER and max_ratio(bnd.to_numpy_f64(S2), S_rec) <= TOL_LAYER
+
+
+def random_layout(rng, C, max_chunks):
+    """A dense or packed layout with ragged ends, empty sequences included."""
+    if rng.random() < 0.5:
+        n = int(rng.integers(1, 6))
+        lens = rng.integers(0, max_chunks * C, size=n)
+        lens[rng.integers(0, n)] += 1
+        cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        return 1, int(cu[-1]), cu
+    return int(rng.integers(1, 4)), int(rng.integers(1, max_chunks * C)), None
+
+
+@pytest.mark.parametrize("seed", [11, 12])
+def test_random_layouts_layer_forward(bnd, seed):
+    """Seeded random batch layouts through both launches: within tolerance of the recurrence and bit-identical
+    from run to run (a race between the kernel's warps would show up as a difference)."""
+    rng = np.random.default_rng(seed)
+    for it in range(12):
+        H = int(rng.integers(1, 9))
+        B, T, cu = random_layout(rng, 64, 7)
+        inp = wl.make("rand", B, T, H, 128, 128, 64, wl.BF16, seed=int(rng.integers(1 << 30)), cu_seqlens=cu)
+        Q = wl.queries(inp, seed=it)
+        S0 = wl.initial_state(inp, seed=it + 1000) if rng.random() < 0.7 else None
+        dev = bnd.to_device(inp)
+        O_ref, S_ref = oracle.gdn_recurrence(Q, inp.K, inp.V, inp.beta, inp.g, 64, scale=0.2, S0=S0, cu_seqlens=cu)
+        runs = []
+        for _ in range(2):
+            O, S = bnd.gdn_forward(bnd.kv_to_torch(Q), dev["K"], dev["V"], dev["beta"], dev["g"], 64, scale=0.2,
+                                   S0=None if S0 is None else torch.from_numpy(S0).cuda(), cu_seqlens=cu)
+            torch.cuda.synchronize()
+            runs.append((O.clone(), S.clone()))
+        assert bnd.last_device_status() == 0
+        assert torch.equal(runs[0][0], runs[1][0]) and torch.equal(runs[0][1], runs[1][1])
+        assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= TOL_LAYER and max_ratio(bnd.to_numpy_f64(S), S_ref) <= TOL_LAYER, (it, B, T, H, cu)
