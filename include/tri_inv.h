@@ -24,6 +24,15 @@
  * every function returns a TRI_INV_* status.  There is no CPU fallback: on a
  * machine without a usable GPU the compute calls return TRI_INV_ERR_CUDA.
  *
+ * Shared state and its limits.  (1) One status word per device, shared by all streams and all
+ * entry points: tri_inv_last_device_status() reports that SOME kernel since the last read gave up
+ * on a wait, not which.  (2) The tensor-core kernels spread their work with a counter pair in
+ * device memory; 64 pairs exist per device and a pair serves one launch at a time (an event behind
+ * the launch tells the host when it is free again).  A launch that finds no free pair -- more than
+ * 64 launches of this library in flight on the device -- and every launch made while its stream is
+ * being captured into a CUDA graph use a fixed work distribution instead: same results, slightly
+ * less even load.  Neither case is an error.
+ *
  * Tensor layouts (contiguous, row-major, flat token index t in [0, B*T)):
  *   K     [B, T, H, d_k]   kv_dtype (fp32, or bf16 as 16-bit patterns)
  *   V     [B, T, H, d_v]   kv_dtype
@@ -114,8 +123,8 @@ typedef struct tri_inv_desc {
 } tri_inv_desc;
 
 /*
- * A = (I + N)^{-1} for every chunk (spec call `tri_inv_build(K, beta, g, C, method) -> A`;
- * N as in Eq. 3 / Table 1, inversion per Sec. 3).
+ * A = (I + N)^{-1} for every chunk: the matrix of Eq. 3 with the phi of Table 1's DeltaNet / GDN rows,
+ * inverted by one of the direct schemes of Sec. 3 (`method`).
  *   K, beta, g : inputs (device).   A : output (device), rows of real tokens only.
  * Errors: INVALID_ARG for null/misaligned pointers or an inconsistent descriptor,
  * UNSUPPORTED for an unknown method, CUDA if the launch fails.
@@ -125,8 +134,7 @@ int tri_inv_build(const void* K, const float* beta, const float* g, float* A,
 
 /*
  * W = A diag(beta) K and U = A diag(beta) V from a given A
- * (spec call `tri_inv_wy(A, K, V, beta) -> W, U`; the WY/UT transform
- * the inverse exists for, Sec. 1).  A is read as stored by tri_inv_build;
+ * (the WY/UT transform that the inverse exists for, Sec. 1).  A is read as stored by tri_inv_build;
  * only its strict lower triangle is used (the diagonal is taken as 1, the upper
  * triangle as 0).  V and U may both be NULL to compute W only.
  */
@@ -221,6 +229,22 @@ int tri_inv_fused_raw(const void* K_raw, const void* V, const float* beta_logit,
 int tri_inv_fused_packed_static(const void* K, const void* V, const float* beta, const float* g,
                                 float* A, void* W, void* U,
                                 const tri_inv_desc* desc, int method, void* cuda_stream);
+
+/*
+ * Self-test of the give-up path of the device-side waits (no step of the paper's method).  Runs tri_inv_fused
+ * (block recursion; bf16, d_k = d_v = 128, C = 64 or 128 only) with every wait limited to wait_limit_ns
+ * nanoseconds instead of two seconds, and with the first thread block leaving out the Gram product of its first
+ * chunk matrix, so that its wait for that product runs out.  Nothing faults, traps or spins without a limit: the
+ * block raises the status word, finishes that one matrix on undefined data (its rows of A, W, U are then
+ * undefined), waits -- again bounded -- for what it still has in flight, frees its tensor memory and returns
+ * without taking further work (with more matrices than resident thread blocks, its second matrix stays
+ * unwritten too); the other blocks do the rest of the batch as usual.  The call synchronises the stream and sets *counters_idle to 1 if
+ * the kernel left every work-distribution counter of the device at zero.  Afterwards
+ * tri_inv_last_device_status() reads TRI_INV_ERR_DEVICE_TIMEOUT (once), and the library is usable as before.
+ */
+int tri_inv_selftest_wait_timeout(const void* K, const void* V, const float* beta, const float* g,
+                                  float* A, void* W, void* U, const tri_inv_desc* desc,
+                                  uint64_t wait_limit_ns, int* counters_idle, void* cuda_stream);
 
 /*
  * Number of chunk matrices (chunks x heads) the descriptor describes.

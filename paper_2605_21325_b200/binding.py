@@ -36,7 +36,7 @@ FORCE_SIMT = 0x10000
 W_DECAY = 0x20000
 
 EXPORTS = ("tri_inv_build", "tri_inv_build_kda", "tri_inv_chunk_scan", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
-           "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
+           "tri_inv_selftest_wait_timeout", "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
 
 
 class Desc(ctypes.Structure):
@@ -75,6 +75,8 @@ def load():
         lib.tri_inv_fused_raw.restype = i32
         lib.tri_inv_fused_packed_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_fused_packed_static.restype = i32
+        lib.tri_inv_selftest_wait_timeout.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, ctypes.c_uint64, ctypes.POINTER(ctypes.c_int), vp]
+        lib.tri_inv_selftest_wait_timeout.restype = i32
         lib.tri_inv_count_matrices.argtypes = [dp, ctypes.POINTER(ctypes.c_int64)]
         lib.tri_inv_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
         for f in ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_count_matrices", "tri_inv_last_device_status"):
@@ -254,6 +256,20 @@ def fused_packed_static(K, V, beta, g, C, cu_seqlens, method=BLOCK_RECURSIVE, ou
     if rc != OK:
         raise TriInvError("tri_inv_fused_packed_static", rc)
     return A, W, U
+
+
+def selftest_wait_timeout(K, V, beta, g, C, wait_limit_ns, out, stream=None):
+    """tri_inv_selftest_wait_timeout: the fused call with short wait limits and one product left out, so that
+    one thread block's wait gives up.  ``out`` = (A, W, U).  Returns True when the work counters are back at zero."""
+    B, T, H, d_k = K.shape
+    desc, keep = make_desc(B, T, H, d_k, V.shape[-1], C, _dtype_code(K), None)
+    A, W, U = out
+    idle = ctypes.c_int(0)
+    rc = load().tri_inv_selftest_wait_timeout(_p(K), _p(V), _p(beta), _p(g), _p(A), _p(W), _p(U), ctypes.byref(desc),
+                                              ctypes.c_uint64(int(wait_limit_ns)), ctypes.byref(idle), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_selftest_wait_timeout", rc)
+    return bool(idle.value)
 
 
 class HostPipeline:

@@ -262,6 +262,31 @@ int tri_inv_chunk_scan(const void* Q, const void* K, const void* W, const void* 
   return err == cudaSuccess ? TRI_INV_OK : TRI_INV_ERR_CUDA;
 }
 
+int tri_inv_selftest_wait_timeout(const void* K, const void* V, const float* beta, const float* g,
+                                  float* A, void* W, void* U, const tri_inv_desc* desc,
+                                  uint64_t wait_limit_ns, int* counters_idle, void* cuda_stream) {
+  int rc = check_desc(desc, true);
+  if (rc) return rc;
+  if (!K || !V || !beta || !g || !A || !W || !U || !counters_idle || wait_limit_ns == 0) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(beta) || !aligned16(g) || !aligned16(A) || !aligned16(W) || !aligned16(U))
+    return TRI_INV_ERR_INVALID_ARG;
+  // only the tensor-core kernel has the stall hook
+  if (desc->kv_dtype != TRI_INV_BF16 || desc->d_k != 128 || desc->d_v != 128 || (desc->C != 64 && desc->C != 128))
+    return TRI_INV_ERR_UNSUPPORTED;
+  KParams p{};
+  p.K = K; p.V = V; p.beta = beta; p.g = g; p.A = A; p.W = W; p.U = U;
+  p.method = TRI_INV_BLOCK_RECURSIVE;
+  p.ops = kDoWY | kStoreA | kTestStall;
+  p.wait_limit_ns = wait_limit_ns;
+  rc = run(p, desc, cuda_stream);
+  if (rc) return rc;
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return TRI_INV_ERR_CUDA;
+  bool idle = false;
+  if (work_counters_idle(&idle) != cudaSuccess) return TRI_INV_ERR_CUDA;
+  *counters_idle = idle ? 1 : 0;
+  return TRI_INV_OK;
+}
+
 int tri_inv_count_matrices(const tri_inv_desc* desc, int64_t* out) {
   int rc = check_desc(desc, false);
   if (rc) return rc;
@@ -293,18 +318,6 @@ int tri_inv_last_device_status(int* out) {
   *out = v;
   return TRI_INV_OK;
 }
-
-#ifdef TRI_INV_PHASE_CLOCKS
-// Development builds only: copies the 128 status/counter words to the host and clears them.
-int tri_inv_debug_counters(int* out) {
-  cudaError_t err;
-  int* word = status_word_for_current_device(&err);
-  if (!word) return TRI_INV_ERR_CUDA;
-  if (cudaMemcpy(out, word, 128 * sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return TRI_INV_ERR_CUDA;
-  if (cudaMemset(word, 0, 128 * sizeof(int)) != cudaSuccess) return TRI_INV_ERR_CUDA;
-  return TRI_INV_OK;
-}
-#endif
 
 int64_t tri_inv_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 

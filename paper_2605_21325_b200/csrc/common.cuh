@@ -13,9 +13,11 @@ enum : int {
   kStoreA = 1,  // write A to global memory
   kDoWY = 2,    // compute W (and U when V != nullptr)
   kLoadA = 4,   // skip build + inversion, read A from A_in (tri_inv_wy)
+  kRaw = 8,     // K is un-normalised, beta and g are logits: normalise, sigmoid, log-sigmoid + chunk cumsum in the kernel
   kKda = 16,    // per-channel decay: KParams::V holds G [B,T,H,d_k] fp32 (build only)
-  kRaw = 8,
-  kWDecay = 32,  // W = A diag(beta) diag(exp g) K: the decay-weighted factor the chunk-state recurrence consumes     // K is un-normalised, beta and g are logits: normalise, sigmoid, log-sigmoid + chunk cumsum in the kernel
+  kFixedStride = 64,  // tensor-core kernel: take no work-counter pair (and create no event for one); items by a fixed stride
+  kTestStall = 128,   // self-test: CTA 0 leaves out the first Gram product so that its bounded wait runs out
+  kWDecay = 32, // W = A diag(beta) diag(exp g) K: the decay-weighted factor the chunk-state recurrence consumes
 };
 
 // One entry per chunk of tokens in ragged mode.
@@ -43,7 +45,8 @@ struct KParams {
   int32_t n_chunks;             // token chunks (all sequences); matrices = n_chunks * H
   int32_t kv_dtype;
   int32_t method;               // TRI_INV_* method with flags
-  int32_t ops;                  // kStoreA | kDoWY | kLoadA
+  int32_t ops;                  // kStoreA | kDoWY | kLoadA | ...
+  unsigned long long wait_limit_ns;  // per bounded device-side wait; 0 = the default of two seconds
 };
 
 // Flat work item -> (first token, real rows, head).  Consecutive items walk the heads of
@@ -98,6 +101,9 @@ cudaError_t launch_kda_tc(const KParams& p, int C, cudaStream_t stream, bool* ha
 // Fills dev_tab (one entry per chunk of tokens, in sequence order) from the host offsets in d->cu_seqlens
 // with small kernels on the stream; no copy and no synchronisation.
 cudaError_t launch_chunk_table(ChunkEntry* dev_tab, const tri_inv_desc* d, cudaStream_t stream);
+
+// True when every work-counter pair of the tensor-core kernel on the current device is back at zero.
+cudaError_t work_counters_idle(bool* idle);
 
 // Adds one to the library's launch counter (tri_inv_launch_count).
 void count_launch();

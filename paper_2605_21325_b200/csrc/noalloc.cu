@@ -59,6 +59,7 @@ extern "C" int tri_inv_fused_packed_static(const void* K, const void* V, const f
   if (method & ~(TRI_INV_METHOD_MASK | TRI_INV_LEAF_SERIES | TRI_INV_FORCE_SIMT)) return TRI_INV_ERR_UNSUPPORTED;
   if ((method & TRI_INV_LEAF_SERIES) && m != TRI_INV_BLOCK_RECURSIVE) return TRI_INV_ERR_UNSUPPORTED;
 
+  if (n_matrices > 0x7fffffffLL) return TRI_INV_ERR_INVALID_ARG;  // the kernels index work items in 32 bits
   const int64_t n_chunks = n_matrices / desc->H;
   if (n_chunks > TRI_INV_STATIC_MAX_CHUNKS) return TRI_INV_ERR_TOO_LARGE;
   if (n_chunks == 0) return TRI_INV_OK;
@@ -71,7 +72,7 @@ extern "C" int tri_inv_fused_packed_static(const void* K, const void* V, const f
   KParams p{};
   p.K = K; p.V = V; p.beta = beta; p.g = g; p.A = A; p.W = W; p.U = U;
   p.method = method;
-  p.ops = kDoWY | (A ? kStoreA : 0);
+  p.ops = kDoWY | (A ? kStoreA : 0) | kFixedStride;  // no counter pair: handing one out may create an event on first use
   p.H = desc->H; p.d_k = desc->d_k; p.d_v = desc->d_v; p.T = desc->T;
   p.kv_dtype = desc->kv_dtype;
   p.n_chunks = static_cast<int32_t>(n_chunks);

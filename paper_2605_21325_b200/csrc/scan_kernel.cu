@@ -27,19 +27,6 @@
 namespace tri_inv {
 namespace {
 
-#ifdef TRI_INV_PHASE_CLOCKS
-#define PHASE_BEGIN() long long ph_t = clock64()
-#define PHASE(k)                                                                  \
-  do {                                                                            \
-    long long now = clock64();                                                    \
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(p.status + 8 + 12 * (threadIdx.x >> 5) + (k), (int)(now - ph_t)); \
-    ph_t = now;                                                                   \
-  } while (0)
-#else
-#define PHASE_BEGIN() do {} while (0)
-#define PHASE(k) do {} while (0)
-#endif
-
 constexpr int C = 64, D = 128, NT = 256;   // NT compute threads (8 warps) + one control warp
 constexpr float kLog2e = 1.4426950408889634f;
 

@@ -9,6 +9,14 @@
 
 #include "common.cuh"
 
+#ifdef TRI_INV_PHASE_CLOCKS
+#include "dev_phase_clocks.cuh"
+#else
+#define CTA_MARK(k) do {} while (0)
+#define PHASE_BEGIN() do {} while (0)
+#define PHASE(k) do {} while (0)
+#endif
+
 namespace tri_inv {
 namespace {
 
@@ -32,25 +40,53 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after about two seconds of wall time (the global timer is read every 64 polls,
-// each poll itself blocks for a hardware-defined time slice) or after kSpinLimit polls, whichever comes
-// first, so a lost copy or product cannot hang the GPU.
+// Bounded wait: gives up after limit_ns of wall time (the global timer is read every 64 polls, each poll
+// itself blocks for a hardware-defined time slice) or after kSpinLimit polls, whichever comes first, so a
+// lost copy or product cannot hang the GPU.  The default limit is two seconds.
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
-  unsigned long long t0;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  const unsigned long long t0 = global_timer_ns();
   for (uint32_t i = 1; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63u) == 0) {
-      unsigned long long t1;
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-      if (t1 - t0 > kWaitLimitNs) return false;
-    }
+    if ((i & 63u) == 0 && global_timer_ns() - t0 > limit_ns) return false;
   }
   return false;
 }
+
+// Give-up protocol of a CTA whose threads wait on the same mbarriers (the tensor-core kernels).  A thread
+// whose wait runs out raises the device status word and three flags in shared memory -- flags[2] "some wait
+// of this CTA has given up" and flags[slot], slot = parity of the CTA's current item -- and then carries on
+// as if the wait had succeeded: it finishes the item on whatever data is there (all indices come from the
+// item number, never from data) with every later wait returning at once.  The CTA leaves its item loop at
+// one place only, after a CTA-wide barrier at the top of the next item, where every thread reads the flag
+// of the PREVIOUS item: all of them see the same value, so the exit is uniform and no thread is left at a
+// barrier or using tensor memory while another frees it.
+struct WaitCtl {
+  volatile int* flags;           // shared memory, 3 ints, zeroed in the prologue
+  int* status;                   // device status word
+  unsigned long long limit_ns;   // per wait
+  __device__ __forceinline__ bool gave_up() const { return flags[2] != 0; }
+  __device__ __forceinline__ bool wait(int slot, uint32_t bar, uint32_t parity) const {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (flags[2]) return false;
+    const unsigned long long t0 = global_timer_ns();
+    for (uint32_t i = 1; i < kSpinLimit; ++i) {
+      if (mbar_try_wait(bar, parity)) return true;
+      if ((i & 63u) == 0 && (flags[2] || global_timer_ns() - t0 > limit_ns)) break;
+    }
+    flags[slot & 1] = 1;
+    flags[2] = 1;
+    atomicMax(status, TRI_INV_ERR_DEVICE_TIMEOUT);
+    return false;
+  }
+};
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
@@ -89,7 +125,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Optional per-phase cycle counters (development builds only: -DTRI_INV_PHASE_CLOCKS).
 template <int C>
 __device__ __forceinline__ uint32_t tile_off(int r, int f) {
   int box = f >> 6, c = (f & 63) >> 3;

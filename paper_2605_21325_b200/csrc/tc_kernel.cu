@@ -25,28 +25,11 @@
 
 #include <mutex>
 
+#define TRI_INV_DEV_DEFINE_EXPORTS  // only read by the development header, which the default build never includes
 #include "tc_device.cuh"
 
 namespace tri_inv {
 namespace {
-
-#ifdef TRI_INV_PHASE_CLOCKS
-__device__ unsigned long long g_cta_times[4096 * 4];
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-__device__ __forceinline__ unsigned smid() { unsigned r; asm volatile("mov.u32 %0, %%smid;" : "=r"(r)); return r; }
-#define CTA_MARK(k) do { if (threadIdx.x == 0 && blockIdx.x < 4096) g_cta_times[blockIdx.x * 4 + (k)] = (k) == 3 ? smid() : gtime(); } while (0)
-#define PHASE_BEGIN() long long ph_t = clock64()
-#define PHASE(k)                                                                  \
-  do {                                                                            \
-    long long now = clock64();                                                    \
-    if (blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(p.status + 8 + 12 * (threadIdx.x >> 5) + (k), (int)(now - ph_t)); \
-    ph_t = now;                                                                   \
-  } while (0)
-#else
-#define CTA_MARK(k) do {} while (0)
-#define PHASE_BEGIN() do {} while (0)
-#define PHASE(k) do {} while (0)
-#endif
 
 // ------------------------------------------------------------------------------------------ layout
 template <int C, int D, bool SER, bool BO = false>
@@ -81,10 +64,11 @@ struct Cfg {
   static constexpr int OFF_BAR = OFF_G + C * 4;
   static constexpr int LEAF_LD = 20;             // per-warp 16 x 16 fp32 scratch of the series leaf
   static constexpr int LEAF_BYTES = NW * 16 * LEAF_LD * 4;
-  // three mbarriers, the TMEM base-address slot, the next-item slot, then the leaf scratch (inside A' with ALIAS)
-  static constexpr int OFF_LEAF = ALIAS ? OFF_AP : (BO ? OFF_K : OFF_BAR + 32);  // BO: in the K tile, dead after the Gram product
+  // 64 bytes of control words: three mbarriers, the TMEM base-address slot, the next-item slot, the exit
+  // mbarrier and the three give-up flags; then the leaf scratch (inside A' with ALIAS)
+  static constexpr int OFF_LEAF = ALIAS ? OFF_AP : (BO ? OFF_K : OFF_BAR + 64);  // BO: in the K tile, dead after the Gram product
   // raw front end: 1 / |k_i| per row, and the per-warp totals of the log-decay scan
-  static constexpr int OFF_R = (ALIAS || BO) ? OFF_BAR + 32 : OFF_LEAF + LEAF_BYTES;
+  static constexpr int OFF_R = (ALIAS || BO) ? OFF_BAR + 64 : OFF_LEAF + LEAF_BYTES;
   static constexpr int END_PLAIN = OFF_R + C * 4 + 32;
   // product-series variant at C = 128: X needs a buffer of its own (at C = 64 it fits where the V tile was)
   static constexpr int OFF_XS = (END_PLAIN + 1023) / 1024 * 1024;
@@ -116,6 +100,9 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
   const uint32_t bar_k = smem_u32(smem + cfg::OFF_BAR);  // K tile landed
   const uint32_t bar_mma = bar_k + 8;                    // a batch of MMAs completed
   const uint32_t bar_v = bar_k + 16;                     // V tile landed
+  const uint32_t bar_exit = bar_k + 32;                  // give-up path only: every product issued so far has retired
+  const WaitCtl wc{reinterpret_cast<volatile int*>(smem + cfg::OFF_BAR + 40), p.status,
+                   p.wait_limit_ns ? p.wait_limit_ns : kWaitLimitNs};
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -143,13 +130,18 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
   // K and V complete on separate barriers: the Gram product starts on K alone, and each buffer is
   // refilled as soon as its last reader is done.
   constexpr int kTidL2 = 32, kTidK = 64, kTidV = 96;
+  uint32_t n_issue_k = 0, n_issue_v = 0;  // copies requested by this thread (the K and the V thread): the exit path waits for the last one
   auto issue_k = [&](int tok0, int h) {
+    if (wc.gave_up()) return;
+    ++n_issue_k;
     fence_proxy_async();
     mbar_expect_tx(bar_k, (uint32_t)cfg::TILE_BYTES);
 #pragma unroll
     for (int bx = 0; bx < cfg::NBOX; ++bx) tma_load_2d(sK + bx * cfg::BOX_BYTES, &tmK, bar_k, h * D + 64 * bx, tok0);
   };
   auto issue_v = [&](int tok0, int h) {
+    if (wc.gave_up()) return;
+    ++n_issue_v;
     fence_proxy_async();
     mbar_expect_tx(bar_v, (uint32_t)cfg::TILE_BYTES);
 #pragma unroll
@@ -169,13 +161,17 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     int tok0 = 0, rows = 0, h = 0;
     const bool any = (int)blockIdx.x < total && !misaligned;
     if (any) locate(p, C, blockIdx.x, tok0, rows, h);
+    // the give-up flags are zeroed by the two threads that read them here (the copy requests check flags[2]) before
+    // they do; nobody can raise one before the barrier that ends the prologue
     if (tid == kTidK) {
+      wc.flags[0] = 0; wc.flags[1] = 0; wc.flags[2] = 0;
       prefetch_tmap(&tmK);
       mbar_init(bar_k, 1);
       fence_mbar_init();
       if (any && !(cfg::ALIAS && load_a)) issue_k(tok0, h);  // with ALIAS, tri_inv_wy fills the matrix first and fetches K later
     }
     if (tid == kTidV) {
+      wc.flags[2] = 0;
       if (need_v) prefetch_tmap(&tmV);
       mbar_init(bar_v, 1);
       fence_mbar_init();
@@ -183,6 +179,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     }
     if (tid == 0) {
       mbar_init(bar_mma, 1);
+      mbar_init(bar_exit, 1);
       fence_mbar_init();
     }
     if (any) bg_next = fetch_bg(tok0, rows, h);
@@ -197,7 +194,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
   const uint32_t tmem = *tmem_slot;
   const uint32_t tmem_rows = tmem + (lane_base << 16);
   uint32_t ph_k = 0, ph_v = 0, ph_mma = 0;  // parities of the next completion to wait for on each barrier
-  bool failed = misaligned;
+  int n_item = 0;  // items this CTA has started: its parity selects the give-up flag of the current item
 
   // Gram S = K K^T: D/16 MMAs of C x C x 16 into the first C columns of tensor memory (thread 0)
   auto issue_gram = [&]() {
@@ -212,11 +209,14 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
   bool gram_early = false;  // thread 0: the Gram product of the coming item was already issued at the end of the last one
   // Work distribution: the first two items of a CTA are fixed (blockIdx, blockIdx + grid), every
   // later one comes from a device counter, fetched one item ahead of its use so that prefetches
-  // know their target.  SMs that run faster simply take more items.
+  // know their target.  SMs that run faster simply take more items.  A launch without a counter
+  // pair (p.work_counter == nullptr) walks its items with the fixed stride gridDim.x.
   int item = blockIdx.x, nx_item = blockIdx.x + gridDim.x;
   while (item < total && !misaligned) {
     int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
+    const int slot = n_item & 1;
+    ++n_item;
     PHASE_BEGIN();
 
     // ---- 1. beta, g were fetched during the previous item (sBeta and sG are adjacent: one store each)
@@ -313,25 +313,29 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
       }
     };
     // after K (and V) were requested again for the WY step: padding rows cleared, keys normalised
-    auto finish_reload = [&]() -> bool {
+    auto finish_reload = [&]() {
       if (rows < C || raw) {
-        if (!mbar_wait_bounded(bar_k, ph_k) || (need_v && rows < C && !mbar_wait_bounded(bar_v, ph_v))) return false;
+        wc.wait(slot, bar_k, ph_k);
+        if (need_v && rows < C) wc.wait(slot, bar_v, ph_v);
         if (rows < C) clear_tail_rows(true, need_v);
         if (raw) { rescale_k_tile(); fence_proxy_async(); }
         __syncthreads();
       }
-      return true;
     };
     if (rows < C) {
       const bool v_now = need_v && !cfg::RELOAD, k_now = !(cfg::ALIAS && load_a);
-      if ((k_now && !mbar_wait_bounded(bar_k, ph_k)) || (v_now && !mbar_wait_bounded(bar_v, ph_v))) { failed = true; break; }
+      if (k_now) wc.wait(slot, bar_k, ph_k);
+      if (v_now) wc.wait(slot, bar_v, ph_v);
       clear_tail_rows(k_now, v_now);
     }
     __syncthreads();
+    // The one exit on a wait that gave up: the flag of the previous item, read by every thread behind this barrier
+    // (a thread that is already further on can only be writing the current item's flag).
+    if (wc.flags[slot ^ 1]) break;
     // the item after next: the ticket is drawn now and used after the inversion, so that its round trip to
     // global memory does not hold this warp (and, at the next barrier, the CTA)
     int ticket = 0;
-    if (tid == kTidL2 && has_next) ticket = atomicAdd(p.work_counter, 1);
+    if (tid == kTidL2 && has_next && p.work_counter) ticket = atomicAdd(p.work_counter, 1);
     PHASE(0);
     // build only: nothing later in the item hides this load, so it is issued now (the element is in L2 already)
     if (BO && has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);
@@ -339,15 +343,15 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     if (!load_a) {
       // ---- 2. Gram S = K K^T on the tensor core: one thread issues D/16 MMAs of C x C x 16 into TMEM
       if (tid == 0 && !gram_early) {
-        if (!mbar_wait_bounded(bar_k, ph_k)) {
-          atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);  // the other threads time out on bar_mma
-        } else {
+        // self-test (kTestStall): CTA 0 leaves out the Gram product of its first item, so the wait below runs out
+        const bool stall = (p.ops & kTestStall) && blockIdx.x == 0 && n_item == 1;
+        if (wc.wait(slot, bar_k, ph_k) && !stall) {
           tc_fence_after();
           issue_gram();
         }
       }
       gram_early = false;
-      if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+      wc.wait(slot, bar_mma, ph_mma);
       ph_mma ^= 1;
       tc_fence_after();
       if (!BO && tid == kTidK && !do_wy && !cfg::RELOAD && has_next) issue_k(nx_tok0, nx_h);  // K's last reader was the Gram product
@@ -432,7 +436,6 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         tc_fence_before();
         __syncthreads();
         constexpr uint32_t idesc_s = umma_idesc_tf32(C, C, 0);
-        bool dead = false;
 #pragma unroll 1
         for (int s = 0; s <= R; ++s) {
           if (tid == 0) {
@@ -460,7 +463,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
             }
             umma_commit(bar_mma);
           }
-          if (!mbar_wait_bounded(bar_mma, ph_mma)) { dead = true; break; }
+          wc.wait(slot, bar_mma, ph_mma);
           ph_mma ^= 1;
           tc_fence_after();
           if (s < R) {  // Y <- Y.Y, written over the old Y and Y^T (their readers, the MMAs, have completed)
@@ -492,7 +495,6 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
             __syncthreads();
           }
         }
-        if (dead) { failed = true; break; }
         // the result goes to the fp32 matrix used by the store and WY steps; the structure of a unit lower
         // triangular matrix is written as constants
 #pragma unroll
@@ -513,7 +515,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
           if (tid == kTidK) issue_k(tok0, h);
           if (tid == kTidV && need_v) issue_v(tok0, h);
           ph_k ^= 1;
-          if (!finish_reload()) { failed = true; break; }
+          finish_reload();
         }
       } else {
       // ---- 3. gate + mask on this warp's rows, N -> shared memory
@@ -632,7 +634,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         tc_fence_before();
         __syncthreads();
         if (tid == 0) { tc_fence_after(); issue_merge(0); }
-        if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+        wc.wait(slot, bar_mma, ph_mma);
         ph_mma ^= 1;
         tc_fence_after();
         // product 2: X21 = -(A22 . T)  (A = A22; B = T^T: element (n, k) = T[k][n], from this thread's fragments)
@@ -655,7 +657,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         tc_fence_before();
         __syncthreads();
         if (tid == 0) { tc_fence_after(); issue_merge(64); }
-        if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+        wc.wait(slot, bar_mma, ph_mma);
         ph_mma ^= 1;
         tc_fence_after();
         {
@@ -710,11 +712,13 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
           fence_proxy_async();
           __syncthreads();   // rows 0 .. 8 m + 7 have been read by everyone
           if (m == 3 && tid == kTidK) {
+            ++n_issue_k;
             mbar_expect_tx(bar_k, (uint32_t)cfg::TILE_BYTES);
             tma_load_2d(sK, &tmK, bar_k, h * D, tok0);
           }
           if (m == 7 && tid == kTidK) tma_load_2d(sK + cfg::BOX_BYTES, &tmK, bar_k, h * D + 64, tok0);
           if (m == 11 && tid == kTidV && need_v) {
+            ++n_issue_v;
             mbar_expect_tx(bar_v, (uint32_t)cfg::TILE_BYTES);
             tma_load_2d(sV, &tmV, bar_v, h * D, tok0);
           }
@@ -743,7 +747,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         if (!do_wy && a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
       }
     }
-    if (tid == kTidL2) *s_next_item = has_next ? 2 * (int)gridDim.x + ticket : total;  // read after this item's last barrier
+    // the item after next (read after this item's last barrier): by ticket, or by a fixed stride without a counter pair
+    if (tid == kTidL2) *s_next_item = !has_next ? total : (p.work_counter ? 2 * (int)gridDim.x + ticket : nx_item + (int)gridDim.x);
     PHASE(6);
 
     if (do_wy) {
@@ -758,7 +763,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
           if (tid == kTidV && need_v) issue_v(tok0, h);
         }
         if (!load_a) ph_k ^= 1;  // second K copy of this item
-        if (!finish_reload()) { failed = true; break; }
+        finish_reload();
       } else {
         tc_fence_before();
         __syncthreads();  // every read of the fp32 matrix (and of S in TMEM) is done: its space becomes A'
@@ -788,10 +793,9 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         umma_commit(bar_mma);
       };
       if (tid == 0) {
-        bool ok = mbar_wait_bounded(bar_k, ph_k);
-        if (C == 128 && need_v) ok = ok && mbar_wait_bounded(bar_v, ph_v);
-        if (!ok) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
-        else { tc_fence_after(); issue_wy(sK); }
+        bool ok = wc.wait(slot, bar_k, ph_k);
+        if (C == 128 && need_v) ok = wc.wait(slot, bar_v, ph_v) && ok;
+        if (ok) { tc_fence_after(); issue_wy(sK); }
       }
       // A goes to global memory while the W product runs (its registers are free again before W returns)
       if (!cfg::ALIAS && a_dst) {
@@ -801,7 +805,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
           if (i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = xv[m];
         }
       }
-      if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+      wc.wait(slot, bar_mma, ph_mma);
       ph_mma ^= 1;
       tc_fence_after();
       PHASE(8);
@@ -819,14 +823,13 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         tc_fence_before();
         __syncthreads();  // every warp holds its rows of W in registers: U may overwrite the columns
         if (tid == 0) {
-          if (!mbar_wait_bounded(bar_v, ph_v)) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
-          else { tc_fence_after(); issue_wy(sV); }
+          if (wc.wait(slot, bar_v, ph_v)) { tc_fence_after(); issue_wy(sV); }
         }
         if (tid == kTidK && has_next) issue_k(nx_tok0, nx_h);  // K's last reader (the W product) is done
         store_frag_piece_bf16(f0, stage, lane, w_row0, row_stride, rows - row0);
         store_frag_piece_bf16(f1, stage, lane, w_row0 + 64, row_stride, rows - row0);
         PHASE(9);
-        if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+        wc.wait(slot, bar_mma, ph_mma);
         ph_mma ^= 1;
         tc_fence_after();
         PHASE(10);
@@ -883,44 +886,92 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     nx_item = *s_next_item;  // written early in this item, several barriers ago
   }
   CTA_MARK(2);
-  if (tid == 0 && atomicAdd(p.work_counter + 1, 1) == (int)gridDim.x - 1) {
+  if (tid == 0 && p.work_counter && atomicAdd(p.work_counter + 1, 1) == (int)gridDim.x - 1) {
     // last CTA out: leave both counters at zero for the next launch that uses this slot
     p.work_counter[0] = 0;
     p.work_counter[1] = 0;
     __threadfence();
   }
-  if (failed) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+  if (misaligned) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+  __syncthreads();  // every thread has left the item loop
+  if (wc.gave_up()) {
+    // A wait gave up.  Before shared and tensor memory go back to the SM, give what this CTA still has in flight a
+    // (bounded) chance to finish: the last copy each tile thread requested, and every product issued so far.
+    if (tid == kTidK && n_issue_k) mbar_wait_bounded(bar_k, (n_issue_k - 1) & 1, wc.limit_ns);
+    if (tid == kTidV && n_issue_v) mbar_wait_bounded(bar_v, (n_issue_v - 1) & 1, wc.limit_ns);
+    if (tid == 0) {
+      umma_commit(bar_exit);
+      mbar_wait_bounded(bar_exit, 0, wc.limit_ns);
+    }
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------ host side
-// Work counters: 64 pairs per device, handed out round-robin so that launches that overlap on
-// different streams do not share one.  Each pair is returned to zero by the kernel that used it.
-__device__ int g_work_counters[64 * 2];
+// Work counters: a launch draws its later items from a {next item, finished CTAs} pair in a static device
+// array.  A pair belongs to ONE launch at a time: the host records an event behind every launch that uses a
+// pair and hands the pair out again only once that event has completed.  A launch that finds no free pair
+// (more than kCounterSlots launches in flight) and every launch made during stream capture (a captured
+// launch is replayed later, when the host can no longer vouch for the pair) gets no pair at all and walks
+// its items with a fixed stride instead -- same results, slightly worse balance.
+constexpr int kCounterSlots = 64;
+__device__ int g_work_counters[kCounterSlots * 2];
 
-int* next_work_counter() {
-  static std::mutex mu;
-  static int* base[64] = {nullptr};
-  static unsigned turn = 0;
+struct CounterRing {
+  int* base = nullptr;
+  cudaEvent_t done[kCounterSlots] = {};
+  unsigned char state[kCounterSlots] = {};  // 0 = never used, 1 = handed out and not yet recorded, 2 = event recorded
+  unsigned turn = 0;
+};
+std::mutex g_ring_mu;
+CounterRing g_rings[64];
+
+// Returns the slot index, or -1 for "no pair: use the fixed stride".
+int acquire_work_counter(cudaStream_t stream, int** pair) {
+  *pair = nullptr;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return -1;
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  std::lock_guard<std::mutex> lock(mu);
-  if (!base[dev]) {
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+  std::lock_guard<std::mutex> lock(g_ring_mu);
+  CounterRing& r = g_rings[dev];
+  if (!r.base) {
     void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_work_counters) != cudaSuccess) return nullptr;
-    base[dev] = static_cast<int*>(ptr);
+    if (cudaGetSymbolAddress(&ptr, g_work_counters) != cudaSuccess) return -1;
+    r.base = static_cast<int*>(ptr);
   }
-  return base[dev] + 2 * (turn++ % 64);
+  for (int tries = 0; tries < 4; ++tries) {
+    const int s = (int)(r.turn++ % kCounterSlots);
+    if (r.state[s] == 1) continue;
+    if (r.state[s] == 2 && cudaEventQuery(r.done[s]) != cudaSuccess) {
+      (void)cudaGetLastError();  // cudaErrorNotReady is not an error of this call
+      continue;
+    }
+    if (!r.done[s] && cudaEventCreateWithFlags(&r.done[s], cudaEventDisableTiming) != cudaSuccess) return -1;
+    r.state[s] = 1;
+    *pair = r.base + 2 * s;
+    return s;
+  }
+  return -1;
+}
+
+// After the launch that uses slot s has been enqueued (or has failed to).
+void release_work_counter(int s, cudaStream_t stream, bool launched) {
+  if (s < 0) return;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return;
+  std::lock_guard<std::mutex> lock(g_ring_mu);
+  CounterRing& r = g_rings[dev];
+  if (launched && cudaEventRecord(r.done[s], stream) == cudaSuccess) r.state[s] = 2;
+  else r.state[s] = launched ? 1 : 0;  // a launched kernel whose event could not be recorded keeps its pair for good
 }
 
 template <int C, int D, bool SER, bool RAW, bool BO = false>
 cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   using cfg = Cfg<C, D, SER, BO>;
   KParams p = p_in;
-  p.work_counter = next_work_counter();
-  if (!p.work_counter) return cudaErrorUnknown;
   // Per-device set-up (function attributes are per device) and grid size, done once per device under a lock.
   static std::mutex mu;
   static int ctas_per_sm_of[64] = {0}, n_sm_of[64] = {0};
@@ -960,17 +1011,24 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   long long total = (long long)p.n_chunks * p.H;
   long long cap = (long long)n_sm * ctas_per_sm;
   int grid = (int)(total < cap ? total : cap);
+  const int slot = (p.ops & kFixedStride) ? -1 : acquire_work_counter(stream, &p.work_counter);
   tc_kernel<C, D, SER, RAW, BO><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
-  return cudaGetLastError();
+  e = cudaGetLastError();
+  release_work_counter(slot, stream, e == cudaSuccess);
+  return e;
 }
 
 }  // namespace
 
-#ifdef TRI_INV_PHASE_CLOCKS
-extern "C" int tri_inv_debug_cta_times(unsigned long long* out, int n) {
-  return cudaMemcpyFromSymbol(out, g_cta_times, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : 3;
+// Self-test support: true when every work-counter pair of the current device reads zero (call after a synchronise).
+cudaError_t work_counters_idle(bool* idle) {
+  int host[kCounterSlots * 2];
+  cudaError_t e = cudaMemcpyFromSymbol(host, g_work_counters, sizeof host);
+  if (e != cudaSuccess) return e;
+  *idle = true;
+  for (int v : host) if (v != 0) *idle = false;
+  return cudaSuccess;
 }
-#endif
 
 cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled) {
   *handled = false;

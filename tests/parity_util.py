@@ -25,7 +25,7 @@ def structure_errors(A_gpu_f32: np.ndarray, inp):
 
 
 def max_ratio(x_gpu: np.ndarray, x_ref: np.ndarray) -> float:
-    """max |x_gpu - x_ref| / max |x_ref| over the whole tensor (the spec ratio)."""
+    """max |x_gpu - x_ref| / max |x_ref| over the whole tensor (the forward error the tolerances are stated in)."""
     den = float(np.abs(x_ref).max())
     if den == 0.0:
         return float(np.abs(x_gpu).max())

@@ -1,0 +1,87 @@
+"""Failure handling and shared state of the tensor-core kernels, on the GPU, without faulting or hanging it.
+
+* A bounded device-side wait that runs out: the kernel must return, raise the status word once, leave the work
+  counters at zero, and the next ordinary call must be bit-exact.  The wait is made to run out by leaving out the
+  product it waits for (tri_inv_selftest_wait_timeout) with a limit of microseconds; every wait stays bounded.
+* Work-counter pairs are private to a launch: a captured graph replayed on one stream while more plain launches
+  than there are pairs run on another stream must give every row right (compared with the fp64 oracle).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_21325_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bnd():
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2605_21325_b200 import binding
+    torch.cuda.set_device(0)
+    return binding
+
+
+def nan_outs(dev, inp):
+    return (torch.full((inp.B, inp.T, inp.H, inp.C), float("nan"), dtype=torch.float32, device="cuda"),
+            torch.full_like(dev["K"], float("nan")), torch.full_like(dev["V"], float("nan")))
+
+
+@pytest.mark.parametrize("C", [64, 128])
+def test_bounded_wait_gives_up_and_the_library_recovers(bnd, C):
+    inp = wl.make("timeout", 2, 16 * C, 8, 128, 128, C, wl.BF16, seed=611)      # 256 matrices
+    dev = bnd.to_device(inp)
+    ref = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], C)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    out = nan_outs(dev, inp)
+    idle = bnd.selftest_wait_timeout(dev["K"], dev["V"], dev["beta"], dev["g"], C, wait_limit_ns=20_000, out=out)
+    assert idle, "a work-counter pair was left non-zero"
+    assert bnd.last_device_status() == bnd.ERR_DEVICE_TIMEOUT     # raised ...
+    assert bnd.last_device_status() == 0                          # ... and cleared by the read
+    # every matrix but the one whose product was left out (thread block 0's first: chunk 0, head 0) is right
+    for r, o in zip(ref, out):
+        r2, o2 = r.clone(), o.clone()
+        r2[0, :C, 0] = 0
+        o2[0, :C, 0] = 0
+        assert torch.equal(r2, o2)
+    # the next ordinary call on the same stream is bit-exact
+    again = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], C, out=nan_outs(dev, inp))
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    for r, o in zip(ref, again):
+        assert torch.equal(r, o)
+
+
+def test_graph_replays_overlapping_many_plain_launches(bnd):
+    a = wl.make("graph_side", 2, 16 * 64, 16, 128, 128, 64, wl.BF16, seed=621)    # 512 matrices: several items per CTA
+    b = wl.make("plain_side", 2, 16 * 64, 16, 128, 128, 64, wl.BF16, seed=622)
+    da, db = bnd.to_device(a), bnd.to_device(b)
+    oa, ob = nan_outs(da, a), nan_outs(db, b)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    bnd.fused(da["K"], da["V"], da["beta"], da["g"], 64, out=oa, stream=s1)      # per-device set-up outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s1):
+        with torch.cuda.graph(graph, stream=s1):
+            bnd.fused(da["K"], da["V"], da["beta"], da["g"], 64, out=oa, stream=s1)
+    for t in oa:
+        t.fill_(float("nan"))
+    torch.cuda.synchronize()
+    for rep in range(8):
+        with torch.cuda.stream(s1):
+            graph.replay()
+        for _ in range(20):                                                       # 160 plain launches in all, unsynchronised
+            bnd.fused(db["K"], db["V"], db["beta"], db["g"], 64, out=ob, stream=s2)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    for inp, out in ((a, oa), (b, ob)):
+        A_ref = oracle.build_A(inp.K, inp.beta, inp.g, inp.C)
+        W_ref, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, inp.C)
+        for o, r, tol in zip(out, (A_ref, W_ref, U_ref), (2e-3, 1e-2, 1e-2)):
+            x = bnd.to_numpy_f64(o)
+            assert not np.isnan(x).any(), "a row was not written: two launches shared a work counter"
+            assert np.abs(x - r).max() <= tol * np.abs(r).max()

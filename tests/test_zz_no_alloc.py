@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2605_21325_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -45,6 +46,32 @@ def test_static_entry_matches_allocating_entry_twice_in_a_row(bnd):
             # same kernel, same inputs: identical; the parity tolerances are the formal bar
             assert (r32 - o32).abs().max().item() <= 2e-3 * r32.abs().max().item()
             assert torch.equal(r, o)
+        # and against the fp64 oracle, with the tolerances of the parity tests (A 2e-3, W and U 1e-2)
+        A_ref = oracle.build_A(inp.K, inp.beta, inp.g, inp.C, cu_seqlens=inp.cu_seqlens)
+        W_ref, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, inp.C, cu_seqlens=inp.cu_seqlens)
+        for o, r, tol in zip(got, (A_ref, W_ref, U_ref), (2e-3, 1e-2, 1e-2)):
+            assert np.abs(bnd.to_numpy_f64(o) - r).max() <= tol * np.abs(r).max()
+
+
+def test_static_entry_allocates_no_device_memory(bnd):
+    """The property the entry point exists for: across a call (after the first one on the device) the free
+    device memory the driver reports does not move, and torch's allocator is not touched either."""
+    inp = packed_case(5, 303)
+    dev = bnd.to_device(inp)
+    out = (torch.empty((1, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda"), torch.empty_like(dev["K"]),
+           torch.empty_like(dev["V"]))
+    bnd.fused_packed_static(dev["K"], dev["V"], dev["beta"], dev["g"], inp.C, inp.cu_seqlens, out=out)   # first call: set-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    reserved0, allocs0 = torch.cuda.memory_reserved(), torch.cuda.memory_stats().get("allocation.all.allocated", 0)
+    for _ in range(3):
+        bnd.fused_packed_static(dev["K"], dev["V"], dev["beta"], dev["g"], inp.C, inp.cu_seqlens, out=out)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert torch.cuda.memory_reserved() == reserved0
+    assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == allocs0
+    assert bnd.last_device_status() == 0
 
 
 def test_static_entry_rejects_what_it_cannot_hold(bnd):
