@@ -27,11 +27,12 @@
  * Shared state and its limits.  (1) One status word per device, shared by all streams and all
  * entry points: tri_inv_last_device_status() reports that SOME kernel since the last read gave up
  * on a wait, not which.  (2) The tensor-core kernels spread their work with a counter pair in
- * device memory; 64 pairs exist per device and a pair serves one launch at a time (an event behind
- * the launch tells the host when it is free again).  A launch that finds no free pair -- more than
- * 64 launches of this library in flight on the device -- and every launch made while its stream is
- * being captured into a CUDA graph use a fixed work distribution instead: same results, slightly
- * less even load.  Neither case is an error.
+ * device memory that must serve one launch at a time.  Launches into one stream run one after the
+ * other, so every stream gets a pair of its own; 64 pairs exist per device.  Launches on a 65th and
+ * further streams, and every launch made while its stream is being captured into a CUDA graph, use a
+ * fixed work distribution instead: same results, slightly less even load.  Neither case is an error.
+ * (Programmatic dependent launch, which lets kernels of one stream overlap, must not be enabled on
+ * this library's launches.)
  *
  * Tensor layouts (contiguous, row-major, flat token index t in [0, B*T)):
  *   K     [B, T, H, d_k]   kv_dtype (fp32, or bf16 as 16-bit patterns)

@@ -17,7 +17,8 @@ import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libtri_inv.so")
+# TRI_INV_LIB selects another build of the same library (the bounds-checking debug build, a development build)
+LIB_PATH = os.environ.get("TRI_INV_LIB") or os.path.join(_PKG, "libtri_inv.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_TOO_LARGE = 0, 1, 2, 3, 4, 5
 STATIC_MAX_CHUNKS = 16384
@@ -75,8 +76,9 @@ def load():
         lib.tri_inv_fused_raw.restype = i32
         lib.tri_inv_fused_packed_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_fused_packed_static.restype = i32
-        lib.tri_inv_selftest_wait_timeout.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, ctypes.c_uint64, ctypes.POINTER(ctypes.c_int), vp]
-        lib.tri_inv_selftest_wait_timeout.restype = i32
+        if hasattr(lib, "tri_inv_selftest_wait_timeout"):
+            lib.tri_inv_selftest_wait_timeout.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, ctypes.c_uint64, ctypes.POINTER(ctypes.c_int), vp]
+            lib.tri_inv_selftest_wait_timeout.restype = i32
         lib.tri_inv_count_matrices.argtypes = [dp, ctypes.POINTER(ctypes.c_int64)]
         lib.tri_inv_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
         for f in ("tri_inv_build", "tri_inv_wy", "tri_inv_fused", "tri_inv_count_matrices", "tri_inv_last_device_status"):

@@ -21,6 +21,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 LIB = os.path.join(PKG, "libtri_inv.so")
 LIB_DEBUG = os.path.join(PKG, "libtri_inv_debug.so")
+LIB_DEV = os.path.join(PKG, "libtri_inv_dev.so")   # development build with phase clocks (-DTRI_INV_PHASE_CLOCKS)
 
 
 def sources():
@@ -42,18 +43,20 @@ def stale(lib: str = LIB) -> bool:
     return _newer(sources() + headers(), lib)
 
 
-def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
-    lib = LIB_DEBUG if debug else LIB
+def build(force: bool = False, verbose: bool = False, debug: bool = False, dev: bool = False) -> str:
+    lib = LIB_DEV if dev else (LIB_DEBUG if debug else LIB)
     if not force and not stale(lib):
         return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    objdir = os.path.join(PKG, "build", "debug" if debug else "release")
+    objdir = os.path.join(PKG, "build", "dev" if dev else ("debug" if debug else "release"))
     os.makedirs(objdir, exist_ok=True)
     flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
              "-I", os.path.join(ROOT, "include"), "-I", os.path.join(PKG, "csrc")]
     flags += os.environ.get("TRI_INV_NVCC_FLAGS", "").split()
     if debug:
         flags.append("-DTRI_INV_DEBUG")
+    if dev:
+        flags.append("-DTRI_INV_PHASE_CLOCKS")
     if verbose:
         flags += ["-Xptxas", "-v"]
     hdrs = headers()
@@ -79,4 +82,4 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv, dev="--dev" in sys.argv))

@@ -100,6 +100,7 @@ int run(KParams p, const tri_inv_desc* d, void* stream_v) {
   p.H = d->H; p.d_k = d->d_k; p.d_v = d->d_v; p.T = d->T;
   p.kv_dtype = d->kv_dtype;
   p.chunk_tab = nullptr;
+  if (!p.wait_limit_ns) p.wait_limit_ns = 2000000000ull;
   cudaError_t err;
   p.status = status_word_for_current_device(&err);
   if (!p.status) return TRI_INV_ERR_CUDA;

@@ -46,7 +46,7 @@ struct KParams {
   int32_t kv_dtype;
   int32_t method;               // TRI_INV_* method with flags
   int32_t ops;                  // kStoreA | kDoWY | kLoadA | ...
-  unsigned long long wait_limit_ns;  // per bounded device-side wait; 0 = the default of two seconds
+  unsigned long long wait_limit_ns;  // per bounded device-side wait (run() fills in the default of two seconds)
 };
 
 // Flat work item -> (first token, real rows, head).  Consecutive items walk the heads of

@@ -78,6 +78,7 @@ extern "C" int tri_inv_fused_packed_static(const void* K, const void* V, const f
   p.n_chunks = static_cast<int32_t>(n_chunks);
   p.chunks_per_seq = 0;
   p.chunk_tab = dev_tab;
+  p.wait_limit_ns = 2000000000ull;
   p.status = status_word_for_current_device(&err);
   if (!p.status) return TRI_INV_ERR_CUDA;
 

@@ -60,33 +60,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
   return false;
 }
 
-// Give-up protocol of a CTA whose threads wait on the same mbarriers (the tensor-core kernels).  A thread
-// whose wait runs out raises the device status word and three flags in shared memory -- flags[2] "some wait
-// of this CTA has given up" and flags[slot], slot = parity of the CTA's current item -- and then carries on
-// as if the wait had succeeded: it finishes the item on whatever data is there (all indices come from the
-// item number, never from data) with every later wait returning at once.  The CTA leaves its item loop at
-// one place only, after a CTA-wide barrier at the top of the next item, where every thread reads the flag
-// of the PREVIOUS item: all of them see the same value, so the exit is uniform and no thread is left at a
-// barrier or using tensor memory while another frees it.
-struct WaitCtl {
-  volatile int* flags;           // shared memory, 3 ints, zeroed in the prologue
-  int* status;                   // device status word
-  unsigned long long limit_ns;   // per wait
-  __device__ __forceinline__ bool gave_up() const { return flags[2] != 0; }
-  __device__ __forceinline__ bool wait(int slot, uint32_t bar, uint32_t parity) const {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (flags[2]) return false;
-    const unsigned long long t0 = global_timer_ns();
-    for (uint32_t i = 1; i < kSpinLimit; ++i) {
-      if (mbar_try_wait(bar, parity)) return true;
-      if ((i & 63u) == 0 && (flags[2] || global_timer_ns() - t0 > limit_ns)) break;
-    }
-    flags[slot & 1] = 1;
-    flags[2] = 1;
-    atomicMax(status, TRI_INV_ERR_DEVICE_TIMEOUT);
-    return false;
-  }
-};
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 

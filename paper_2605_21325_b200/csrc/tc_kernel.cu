@@ -81,7 +81,7 @@ struct Cfg {
 // Byte offset of the 16-byte chunk holding features [f, f+8) of row r inside a swizzled tile.
 template <int C, int D, bool SER, bool RAW, bool BO>
 __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK,
-                                                                             const __grid_constant__ CUtensorMap tmV, KParams p) {
+                                                                             const __grid_constant__ CUtensorMap tmV, const __grid_constant__ KParams p) {
   using cfg = Cfg<C, D, SER, BO>;
   static_assert(D == 128, "tiles are two 64-feature boxes wide");
   constexpr int LD = cfg::LD;
@@ -101,8 +101,18 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
   const uint32_t bar_mma = bar_k + 8;                    // a batch of MMAs completed
   const uint32_t bar_v = bar_k + 16;                     // V tile landed
   const uint32_t bar_exit = bar_k + 32;                  // give-up path only: every product issued so far has retired
-  const WaitCtl wc{reinterpret_cast<volatile int*>(smem + cfg::OFF_BAR + 40), p.status,
-                   p.wait_limit_ns ? p.wait_limit_ns : kWaitLimitNs};
+  // Give-up protocol.  A thread whose bounded wait runs out remembers it ("bad"), skips its later waits, and
+  // carries on with the item on whatever data is there (all indices come from the item number, never from
+  // data).  It raises the CTA's flag in shared memory just before the barrier at the top of the next item;
+  // behind that barrier every thread reads the flag and the whole CTA leaves the loop together, so no thread is
+  // left at a barrier or using tensor memory while another frees it.
+  volatile int* const s_gave_up = reinterpret_cast<volatile int*>(smem + cfg::OFF_BAR + 40);
+  bool bad = false;
+  auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
+    if (bad) return false;
+    bad = !mbar_wait_bounded(bar, parity, p.wait_limit_ns);
+    return !bad;
+  };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -130,18 +140,18 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
   // K and V complete on separate barriers: the Gram product starts on K alone, and each buffer is
   // refilled as soon as its last reader is done.
   constexpr int kTidL2 = 32, kTidK = 64, kTidV = 96;
-  uint32_t n_issue_k = 0, n_issue_v = 0;  // copies requested by this thread (the K and the V thread): the exit path waits for the last one
+  uint32_t n_issue = 0;  // copies requested by this thread (the K thread: K tiles, the V thread: V tiles): the exit path waits for the last one
   auto issue_k = [&](int tok0, int h) {
-    if (wc.gave_up()) return;
-    ++n_issue_k;
+    if (bad) return;
+    ++n_issue;
     fence_proxy_async();
     mbar_expect_tx(bar_k, (uint32_t)cfg::TILE_BYTES);
 #pragma unroll
     for (int bx = 0; bx < cfg::NBOX; ++bx) tma_load_2d(sK + bx * cfg::BOX_BYTES, &tmK, bar_k, h * D + 64 * bx, tok0);
   };
   auto issue_v = [&](int tok0, int h) {
-    if (wc.gave_up()) return;
-    ++n_issue_v;
+    if (bad) return;
+    ++n_issue;
     fence_proxy_async();
     mbar_expect_tx(bar_v, (uint32_t)cfg::TILE_BYTES);
 #pragma unroll
@@ -161,17 +171,15 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     int tok0 = 0, rows = 0, h = 0;
     const bool any = (int)blockIdx.x < total && !misaligned;
     if (any) locate(p, C, blockIdx.x, tok0, rows, h);
-    // the give-up flags are zeroed by the two threads that read them here (the copy requests check flags[2]) before
-    // they do; nobody can raise one before the barrier that ends the prologue
+    // the give-up flag is zeroed here; nobody can raise it before the barrier that ends the prologue
     if (tid == kTidK) {
-      wc.flags[0] = 0; wc.flags[1] = 0; wc.flags[2] = 0;
+      *s_gave_up = 0;
       prefetch_tmap(&tmK);
       mbar_init(bar_k, 1);
       fence_mbar_init();
       if (any && !(cfg::ALIAS && load_a)) issue_k(tok0, h);  // with ALIAS, tri_inv_wy fills the matrix first and fetches K later
     }
     if (tid == kTidV) {
-      wc.flags[2] = 0;
       if (need_v) prefetch_tmap(&tmV);
       mbar_init(bar_v, 1);
       fence_mbar_init();
@@ -194,7 +202,6 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
   const uint32_t tmem = *tmem_slot;
   const uint32_t tmem_rows = tmem + (lane_base << 16);
   uint32_t ph_k = 0, ph_v = 0, ph_mma = 0;  // parities of the next completion to wait for on each barrier
-  int n_item = 0;  // items this CTA has started: its parity selects the give-up flag of the current item
 
   // Gram S = K K^T: D/16 MMAs of C x C x 16 into the first C columns of tensor memory (thread 0)
   auto issue_gram = [&]() {
@@ -215,8 +222,6 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
   while (item < total && !misaligned) {
     int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
-    const int slot = n_item & 1;
-    ++n_item;
     PHASE_BEGIN();
 
     // ---- 1. beta, g were fetched during the previous item (sBeta and sG are adjacent: one store each)
@@ -315,8 +320,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     // after K (and V) were requested again for the WY step: padding rows cleared, keys normalised
     auto finish_reload = [&]() {
       if (rows < C || raw) {
-        wc.wait(slot, bar_k, ph_k);
-        if (need_v && rows < C) wc.wait(slot, bar_v, ph_v);
+        wait(bar_k, ph_k);
+        if (need_v && rows < C) wait(bar_v, ph_v);
         if (rows < C) clear_tail_rows(true, need_v);
         if (raw) { rescale_k_tile(); fence_proxy_async(); }
         __syncthreads();
@@ -324,14 +329,15 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     };
     if (rows < C) {
       const bool v_now = need_v && !cfg::RELOAD, k_now = !(cfg::ALIAS && load_a);
-      if (k_now) wc.wait(slot, bar_k, ph_k);
-      if (v_now) wc.wait(slot, bar_v, ph_v);
+      if (k_now) wait(bar_k, ph_k);
+      if (v_now) wait(bar_v, ph_v);
       clear_tail_rows(k_now, v_now);
     }
+    if (bad) *s_gave_up = 1;
     __syncthreads();
-    // The one exit on a wait that gave up: the flag of the previous item, read by every thread behind this barrier
-    // (a thread that is already further on can only be writing the current item's flag).
-    if (wc.flags[slot ^ 1]) break;
+    // The one exit on a wait that gave up: every thread reads the flag behind this barrier (a thread can raise it
+    // again only before the next item's barrier, which it reaches after everyone has read it here).
+    if (*s_gave_up) break;
     // the item after next: the ticket is drawn now and used after the inversion, so that its round trip to
     // global memory does not hold this warp (and, at the next barrier, the CTA)
     int ticket = 0;
@@ -344,14 +350,14 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
       // ---- 2. Gram S = K K^T on the tensor core: one thread issues D/16 MMAs of C x C x 16 into TMEM
       if (tid == 0 && !gram_early) {
         // self-test (kTestStall): CTA 0 leaves out the Gram product of its first item, so the wait below runs out
-        const bool stall = (p.ops & kTestStall) && blockIdx.x == 0 && n_item == 1;
-        if (wc.wait(slot, bar_k, ph_k) && !stall) {
+        const bool stall = (p.ops & kTestStall) && item == 0;
+        if (wait(bar_k, ph_k) && !stall) {
           tc_fence_after();
           issue_gram();
         }
       }
       gram_early = false;
-      wc.wait(slot, bar_mma, ph_mma);
+      wait(bar_mma, ph_mma);
       ph_mma ^= 1;
       tc_fence_after();
       if (!BO && tid == kTidK && !do_wy && !cfg::RELOAD && has_next) issue_k(nx_tok0, nx_h);  // K's last reader was the Gram product
@@ -463,7 +469,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
             }
             umma_commit(bar_mma);
           }
-          wc.wait(slot, bar_mma, ph_mma);
+          wait(bar_mma, ph_mma);
           ph_mma ^= 1;
           tc_fence_after();
           if (s < R) {  // Y <- Y.Y, written over the old Y and Y^T (their readers, the MMAs, have completed)
@@ -634,7 +640,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         tc_fence_before();
         __syncthreads();
         if (tid == 0) { tc_fence_after(); issue_merge(0); }
-        wc.wait(slot, bar_mma, ph_mma);
+        wait(bar_mma, ph_mma);
         ph_mma ^= 1;
         tc_fence_after();
         // product 2: X21 = -(A22 . T)  (A = A22; B = T^T: element (n, k) = T[k][n], from this thread's fragments)
@@ -657,7 +663,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         tc_fence_before();
         __syncthreads();
         if (tid == 0) { tc_fence_after(); issue_merge(64); }
-        wc.wait(slot, bar_mma, ph_mma);
+        wait(bar_mma, ph_mma);
         ph_mma ^= 1;
         tc_fence_after();
         {
@@ -712,13 +718,13 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
           fence_proxy_async();
           __syncthreads();   // rows 0 .. 8 m + 7 have been read by everyone
           if (m == 3 && tid == kTidK) {
-            ++n_issue_k;
+            ++n_issue;
             mbar_expect_tx(bar_k, (uint32_t)cfg::TILE_BYTES);
             tma_load_2d(sK, &tmK, bar_k, h * D, tok0);
           }
           if (m == 7 && tid == kTidK) tma_load_2d(sK + cfg::BOX_BYTES, &tmK, bar_k, h * D + 64, tok0);
           if (m == 11 && tid == kTidV && need_v) {
-            ++n_issue_v;
+            ++n_issue;
             mbar_expect_tx(bar_v, (uint32_t)cfg::TILE_BYTES);
             tma_load_2d(sV, &tmV, bar_v, h * D, tok0);
           }
@@ -793,8 +799,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         umma_commit(bar_mma);
       };
       if (tid == 0) {
-        bool ok = wc.wait(slot, bar_k, ph_k);
-        if (C == 128 && need_v) ok = wc.wait(slot, bar_v, ph_v) && ok;
+        bool ok = wait(bar_k, ph_k);
+        if (C == 128 && need_v) ok = wait(bar_v, ph_v) && ok;
         if (ok) { tc_fence_after(); issue_wy(sK); }
       }
       // A goes to global memory while the W product runs (its registers are free again before W returns)
@@ -805,7 +811,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
           if (i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = xv[m];
         }
       }
-      wc.wait(slot, bar_mma, ph_mma);
+      wait(bar_mma, ph_mma);
       ph_mma ^= 1;
       tc_fence_after();
       PHASE(8);
@@ -823,13 +829,13 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         tc_fence_before();
         __syncthreads();  // every warp holds its rows of W in registers: U may overwrite the columns
         if (tid == 0) {
-          if (wc.wait(slot, bar_v, ph_v)) { tc_fence_after(); issue_wy(sV); }
+          if (wait(bar_v, ph_v)) { tc_fence_after(); issue_wy(sV); }
         }
         if (tid == kTidK && has_next) issue_k(nx_tok0, nx_h);  // K's last reader (the W product) is done
         store_frag_piece_bf16(f0, stage, lane, w_row0, row_stride, rows - row0);
         store_frag_piece_bf16(f1, stage, lane, w_row0 + 64, row_stride, rows - row0);
         PHASE(9);
-        wc.wait(slot, bar_mma, ph_mma);
+        wait(bar_mma, ph_mma);
         ph_mma ^= 1;
         tc_fence_after();
         PHASE(10);
@@ -892,16 +898,17 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
     p.work_counter[1] = 0;
     __threadfence();
   }
-  if (misaligned) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+  if (bad) *s_gave_up = 1;
+  if (bad || misaligned) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
   __syncthreads();  // every thread has left the item loop
-  if (wc.gave_up()) {
+  if (*s_gave_up) {
     // A wait gave up.  Before shared and tensor memory go back to the SM, give what this CTA still has in flight a
     // (bounded) chance to finish: the last copy each tile thread requested, and every product issued so far.
-    if (tid == kTidK && n_issue_k) mbar_wait_bounded(bar_k, (n_issue_k - 1) & 1, wc.limit_ns);
-    if (tid == kTidV && n_issue_v) mbar_wait_bounded(bar_v, (n_issue_v - 1) & 1, wc.limit_ns);
+    if (tid == kTidK && n_issue) mbar_wait_bounded(bar_k, (n_issue - 1) & 1, p.wait_limit_ns);
+    if (tid == kTidV && n_issue) mbar_wait_bounded(bar_v, (n_issue - 1) & 1, p.wait_limit_ns);
     if (tid == 0) {
       umma_commit(bar_exit);
-      mbar_wait_bounded(bar_exit, 0, wc.limit_ns);
+      mbar_wait_bounded(bar_exit, 0, p.wait_limit_ns);
     }
   }
   tc_fence_before();
@@ -911,61 +918,43 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
 
 // ------------------------------------------------------------------------------------------ host side
 // Work counters: a launch draws its later items from a {next item, finished CTAs} pair in a static device
-// array.  A pair belongs to ONE launch at a time: the host records an event behind every launch that uses a
-// pair and hands the pair out again only once that event has completed.  A launch that finds no free pair
-// (more than kCounterSlots launches in flight) and every launch made during stream capture (a captured
-// launch is replayed later, when the host can no longer vouch for the pair) gets no pair at all and walks
-// its items with a fixed stride instead -- same results, slightly worse balance.
+// array, which the last CTA out returns to zero.  A pair must serve ONE launch at a time.  Kernels launched
+// into the same stream run one after the other, so each stream gets a pair of its own (by the stream's unique
+// id) and nothing has to be tracked: no event, no flag, no synchronisation.  There are kCounterSlots pairs per
+// device; launches on further streams, and every launch made during stream capture (a captured launch is
+// replayed later on whatever stream the graph is launched into), get no pair at all and walk their items with
+// a fixed stride instead: same results, slightly less even load.
 constexpr int kCounterSlots = 64;
 __device__ int g_work_counters[kCounterSlots * 2];
 
-struct CounterRing {
+struct CounterTable {
   int* base = nullptr;
-  cudaEvent_t done[kCounterSlots] = {};
-  unsigned char state[kCounterSlots] = {};  // 0 = never used, 1 = handed out and not yet recorded, 2 = event recorded
-  unsigned turn = 0;
+  unsigned long long stream_id[kCounterSlots] = {};
+  int used = 0;
 };
-std::mutex g_ring_mu;
-CounterRing g_rings[64];
+std::mutex g_table_mu;
+CounterTable g_tables[64];
 
-// Returns the slot index, or -1 for "no pair: use the fixed stride".
-int acquire_work_counter(cudaStream_t stream, int** pair) {
-  *pair = nullptr;
+// The pair of this stream, or nullptr for "no pair: use the fixed stride".
+int* work_counter_for(cudaStream_t stream) {
   cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-  if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return -1;
+  if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return nullptr;
+  unsigned long long id = 0;
+  if (cudaStreamGetId(stream, &id) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
-  std::lock_guard<std::mutex> lock(g_ring_mu);
-  CounterRing& r = g_rings[dev];
-  if (!r.base) {
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_table_mu);
+  CounterTable& t = g_tables[dev];
+  if (!t.base) {
     void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_work_counters) != cudaSuccess) return -1;
-    r.base = static_cast<int*>(ptr);
+    if (cudaGetSymbolAddress(&ptr, g_work_counters) != cudaSuccess) return nullptr;
+    t.base = static_cast<int*>(ptr);
   }
-  for (int tries = 0; tries < 4; ++tries) {
-    const int s = (int)(r.turn++ % kCounterSlots);
-    if (r.state[s] == 1) continue;
-    if (r.state[s] == 2 && cudaEventQuery(r.done[s]) != cudaSuccess) {
-      (void)cudaGetLastError();  // cudaErrorNotReady is not an error of this call
-      continue;
-    }
-    if (!r.done[s] && cudaEventCreateWithFlags(&r.done[s], cudaEventDisableTiming) != cudaSuccess) return -1;
-    r.state[s] = 1;
-    *pair = r.base + 2 * s;
-    return s;
-  }
-  return -1;
-}
-
-// After the launch that uses slot s has been enqueued (or has failed to).
-void release_work_counter(int s, cudaStream_t stream, bool launched) {
-  if (s < 0) return;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return;
-  std::lock_guard<std::mutex> lock(g_ring_mu);
-  CounterRing& r = g_rings[dev];
-  if (launched && cudaEventRecord(r.done[s], stream) == cudaSuccess) r.state[s] = 2;
-  else r.state[s] = launched ? 1 : 0;  // a launched kernel whose event could not be recorded keeps its pair for good
+  for (int s = 0; s < t.used; ++s)
+    if (t.stream_id[s] == id) return t.base + 2 * s;
+  if (t.used == kCounterSlots) return nullptr;
+  t.stream_id[t.used] = id;
+  return t.base + 2 * t.used++;
 }
 
 template <int C, int D, bool SER, bool RAW, bool BO = false>
@@ -1011,11 +1000,9 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   long long total = (long long)p.n_chunks * p.H;
   long long cap = (long long)n_sm * ctas_per_sm;
   int grid = (int)(total < cap ? total : cap);
-  const int slot = (p.ops & kFixedStride) ? -1 : acquire_work_counter(stream, &p.work_counter);
+  p.work_counter = (p.ops & kFixedStride) ? nullptr : work_counter_for(stream);
   tc_kernel<C, D, SER, RAW, BO><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
-  e = cudaGetLastError();
-  release_work_counter(slot, stream, e == cudaSuccess);
-  return e;
+  return cudaGetLastError();
 }
 
 }  // namespace
