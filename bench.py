@@ -199,7 +199,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
-    ap.add_argument("--method", default="block_recursive", choices=["block_recursive", "mixed_recursion", "product_series"])
+    ap.add_argument("--method", default="block_recursive", choices=["block_recursive", "mixed_recursion", "product_series", "block_recursive_refined", "product_series_f16"])
     ap.add_argument("--paper-T", type=int, default=0,
                     help="instead of --config: the paper's timing shape B=32, H=4, d=128 at this sequence length (1024..16384)")
     ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw", "kda", "scan", "layer"],
@@ -241,7 +241,8 @@ def main():
     from paper_2605_21325_b200 import binding
 
     method = {"block_recursive": binding.BLOCK_RECURSIVE, "mixed_recursion": binding.BLOCK_RECURSIVE | binding.LEAF_SERIES,
-              "product_series": binding.PRODUCT_SERIES}[args.method]
+              "product_series": binding.PRODUCT_SERIES, "block_recursive_refined": binding.BLOCK_RECURSIVE | binding.REFINE,
+              "product_series_f16": binding.PRODUCT_SERIES | binding.OPERANDS_F16}[args.method]
     if args.simt:
         method |= binding.FORCE_SIMT
 

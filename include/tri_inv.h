@@ -94,9 +94,16 @@ enum {
    * instead of substitution -- the mixed recursion of Alg. 2 (r = 0). */
   TRI_INV_LEAF_SERIES = 0x100,
   /* flag: one step of iterative refinement after the inversion (Alg. 6 / Sec. 3.6):
-   * R <- I - A (I + N), A <- A + R A.  Block recursion and Newton-Schulz only; runs on the
-   * fp32 CUDA-core kernel (TF32 products could not resolve the residual). */
+   * R <- I - A (I + N), A <- A + R A.  Block recursion and Newton-Schulz only.  After the block recursion on the
+   * tensor-core kernel the residual is formed from TF32 hi/lo splits of both factors (three products, fp32
+   * accumulation) and the correction R A in one TF32 product; Newton-Schulz and fp32 inputs use the CUDA cores. */
   TRI_INV_REFINE = 0x200,
+  /* flag, product series on the tensor-core kernel only (bf16 keys, d = 128, C = 64 or 128): the series' matrix
+   * products take fp16 operands instead of TF32 ones -- the half-precision format Sec. 4.1 prefers to bf16; same
+   * 11-bit significand as TF32, fp32 accumulation, but a range of 6e-8 .. 65504: powers of N that leave it overflow,
+   * which the unstable series (Sec. 3.2) can produce on badly conditioned chunks.  Half the operand bytes and one
+   * stored copy of Y for both operand roles: the fast form of the series.  Elsewhere TRI_INV_ERR_UNSUPPORTED. */
+  TRI_INV_OPERANDS_F16 = 0x400,
   /* Newton-Schulz iteration count, 1..15, in bits 12..15 (0 = default) */
 #define TRI_INV_NS_ITERS(m) (((m) & 0xf) << 12)
   /* flag: run the plain fp32 CUDA-core kernel even where a tensor-core kernel

@@ -26,6 +26,7 @@ F32, BF16 = 0, 1
 BLOCK_RECURSIVE, PRODUCT_SERIES, NEWTON_SCHULZ = 0, 1, 2
 LEAF_SERIES = 0x100
 REFINE = 0x200
+OPERANDS_F16 = 0x400
 
 
 def ns_iters(m: int) -> int:

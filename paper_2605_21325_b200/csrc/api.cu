@@ -87,7 +87,8 @@ int check_method(int method, bool w_decay_ok = false) {
     method &= ~TRI_INV_W_DECAY;
   }
   if (m != TRI_INV_BLOCK_RECURSIVE && m != TRI_INV_PRODUCT_SERIES && m != TRI_INV_NEWTON_SCHULZ) return TRI_INV_ERR_UNSUPPORTED;
-  if (method & ~(TRI_INV_METHOD_MASK | TRI_INV_LEAF_SERIES | TRI_INV_REFINE | TRI_INV_NS_ITERS(15) | TRI_INV_FORCE_SIMT)) return TRI_INV_ERR_UNSUPPORTED;
+  if (method & ~(TRI_INV_METHOD_MASK | TRI_INV_LEAF_SERIES | TRI_INV_REFINE | TRI_INV_NS_ITERS(15) | TRI_INV_FORCE_SIMT | TRI_INV_OPERANDS_F16)) return TRI_INV_ERR_UNSUPPORTED;
+  if ((method & TRI_INV_OPERANDS_F16) && (m != TRI_INV_PRODUCT_SERIES || (method & TRI_INV_FORCE_SIMT))) return TRI_INV_ERR_UNSUPPORTED;
   if ((method & TRI_INV_LEAF_SERIES) && m != TRI_INV_BLOCK_RECURSIVE) return TRI_INV_ERR_UNSUPPORTED;
   if ((method & TRI_INV_REFINE) && m == TRI_INV_PRODUCT_SERIES) return TRI_INV_ERR_UNSUPPORTED;
   if ((method & TRI_INV_NS_ITERS(15)) && m != TRI_INV_NEWTON_SCHULZ) return TRI_INV_ERR_UNSUPPORTED;
@@ -132,9 +133,14 @@ int run(KParams p, const tri_inv_desc* d, void* stream_v) {
   if ((long long)p.n_chunks * d->H > 0x7fffffffLL) return TRI_INV_ERR_INVALID_ARG;  // kernels index work items in 32 bits
   bool handled = false;
   err = cudaSuccess;
-  // Newton-Schulz and the refinement step exist on the fp32 CUDA-core kernel only
-  const bool simt_only = (p.method & (TRI_INV_FORCE_SIMT | TRI_INV_REFINE)) || (p.method & TRI_INV_METHOD_MASK) == TRI_INV_NEWTON_SCHULZ;
+  // Newton-Schulz exists on the fp32 CUDA-core kernel only; so does refinement with the per-channel decay
+  const bool simt_only = (p.method & TRI_INV_FORCE_SIMT) || (p.method & TRI_INV_METHOD_MASK) == TRI_INV_NEWTON_SCHULZ ||
+                         ((p.ops & kKda) && (p.method & TRI_INV_REFINE));
   if (!simt_only) err = (p.ops & kKda) ? launch_kda_tc(p, d->C, stream, &handled) : launch_tc(p, d->C, stream, &handled);
+  if (err == cudaSuccess && !handled && (p.method & TRI_INV_OPERANDS_F16)) {   // only the tensor-core kernel has fp16 operands
+    if (dev_tab) cudaFreeAsync(dev_tab, stream);
+    return TRI_INV_ERR_UNSUPPORTED;
+  }
   if (err == cudaSuccess && !handled) err = launch_simt(p, d->C, stream);
   if (err == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);
   if (dev_tab) cudaFreeAsync(dev_tab, stream);

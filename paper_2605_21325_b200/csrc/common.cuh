@@ -77,6 +77,16 @@ __device__ __forceinline__ float load_kv(const void* base, int dtype, size_t idx
 cudaError_t launch_simt(const KParams& p, int C, cudaStream_t stream);
 // Tensor-core path: returns cudaErrorNotSupported when it has no kernel for the request.
 cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
+// Instantiations of the tensor-core kernel, one group per tc_inst_*.cu file; raw = the variant that rewrites the K tile.
+cudaError_t launch_tc_c64_br(const KParams& p, cudaStream_t stream, bool raw);
+cudaError_t launch_tc_c64_series(const KParams& p, cudaStream_t stream, bool raw);
+cudaError_t launch_tc_c64_build(const KParams& p, cudaStream_t stream);
+cudaError_t launch_tc_c128_br(const KParams& p, cudaStream_t stream, bool raw);
+cudaError_t launch_tc_c128_series(const KParams& p, cudaStream_t stream, bool raw);
+cudaError_t launch_tc_refine(const KParams& p, int C, cudaStream_t stream, bool raw);
+cudaError_t launch_tc_series_f16(const KParams& p, int C, cudaStream_t stream, bool raw);
+// The work-counter pair of a stream (tc_launch.cu), or nullptr: the kernel then walks its items with a fixed stride.
+int* work_counter_for(cudaStream_t stream);
 // Chunk scan (consumer of W and U): parameters other than the three TMA-staged tensors.
 struct ScanParams {
   const void* U;        // [tokens,H,d_v]

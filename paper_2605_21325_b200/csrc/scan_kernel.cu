@@ -57,14 +57,6 @@ __device__ __forceinline__ void tmem_ld_frag(float (&r)[NTL][4], uint32_t taddr)
   if constexpr (NTL == 8) tmem_ld_16x64(r, taddr);
   else tmem_ld_16x32(r, taddr);
 }
-__device__ __forceinline__ void tmem_st_16x32(const float (&r)[4][4], uint32_t taddr) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.16x256b.x4.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
-      ::"f"(r[0][0]), "f"(r[0][1]), "f"(r[0][2]), "f"(r[0][3]), "f"(r[1][0]), "f"(r[1][1]), "f"(r[1][2]), "f"(r[1][3]),
-        "f"(r[2][0]), "f"(r[2][1]), "f"(r[2][2]), "f"(r[2][3]), "f"(r[3][0]), "f"(r[3][1]), "f"(r[3][2]), "f"(r[3][3]),
-        "r"(taddr)
-      : "memory");
-}
 template <int NTL>
 __device__ __forceinline__ void tmem_st_frag(const float (&r)[NTL][4], uint32_t taddr) {
 #pragma unroll
@@ -74,12 +66,8 @@ __device__ __forceinline__ void tmem_st_frag(const float (&r)[NTL][4], uint32_t 
     tmem_st_16x32(q, taddr + 8 * b);
   }
 }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void stmatrix_x4(uint32_t addr, uint32_t m0, uint32_t m1, uint32_t m2, uint32_t m3) {
-  asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
 }
 __device__ __forceinline__ void stmatrix_x4_trans(uint32_t addr, uint32_t m0, uint32_t m1, uint32_t m2, uint32_t m3) {
   asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");

@@ -93,6 +93,11 @@ __device__ __forceinline__ float ex2_approx(float x) {  // 2^x, relative error a
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {   // round-to-nearest-even, lo in the low half
+  uint32_t r;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -229,6 +234,141 @@ __device__ __forceinline__ void merge_level(float* sX, int warp, int lane) {
   __syncthreads();
 }
 
+// One step of iterative refinement (Alg. 6 / Sec. 3.6) for the matrix I + N on the warp-level tensor cores:
+//     R = I - X (I + N) = (I - X) - X N,        X <- X + R X.
+// sX holds X (fp32, unit lower triangular, complete), sN holds N (fp32, strictly lower triangular, zeros
+// elsewhere); both C x C with row length C + 4.  On return sX holds the refined X; sN is overwritten (by R).
+// The residual needs more than one TF32 pass (a single pass has the very error the step is to remove), so
+// X N is formed from the TF32 splits X = Xh + Xl, N = Nh + Nl as Xh Nh + Xl Nh + Xh Nl with fp32 accumulation
+// (the dropped Xl Nl is 2^-22 relative); R is then about as small as the inverse's error, and R X needs one
+// pass only.  8-column tiles of the lower triangle are dealt out to the C / 16 warps by column (warp w takes
+// columns w and C/8 - 1 - w), so the triangular work is shared about evenly; only the k-steps where both operands can be non-zero
+// are issued (X and R lower triangular: k <= i; N strictly lower, X lower: k >= j).
+template <int C>
+__device__ __forceinline__ void refine_step(float* sX, float* sN, int warp, int lane) {
+  constexpr int LD = C + 4, NT8 = C / 8;
+  constexpr int CPW = 2;                   // tile columns per warp: column w and column NT8 - 1 - w (long and short k ranges paired)
+  constexpr int MAXT = (C / 16) * CPW;     // tiles a warp can own: row blocks x its columns
+  const int g = lane >> 2, t = lane & 3;
+  float acc[MAXT][4];
+  auto split = [](float x, uint32_t& hi, uint32_t& lo) {
+    hi = to_tf32(x);
+    lo = to_tf32(x - __uint_as_float(hi));
+  };
+  // ---- R tiles of this warp
+#pragma unroll
+  for (int rb = 0; rb < C / 16; ++rb) {
+#pragma unroll
+    for (int c = 0; c < CPW; ++c) {
+      const int slot = rb * (CPW) + c;
+      acc[slot][0] = acc[slot][1] = acc[slot][2] = acc[slot][3] = 0.f;
+    }
+#pragma unroll
+    for (int q = 0; q < 2 * rb + 2; ++q) {     // k-step of eight: columns 8q .. 8q+7 of X, rows of N
+      bool any = false;
+#pragma unroll
+      for (int c = 0; c < CPW; ++c) any = any || ((c == 0 ? warp : NT8 - 1 - warp) <= q);
+      if (!any) continue;                      // warp-uniform: none of this warp's columns reaches this k-step
+      const float* ap = sX + (16 * rb + g) * LD + 8 * q + t;
+      uint32_t ah[4], al[4];
+      split(ap[0], ah[0], al[0]);
+      split(ap[8 * LD], ah[1], al[1]);
+      split(ap[4], ah[2], al[2]);
+      split(ap[8 * LD + 4], ah[3], al[3]);
+#pragma unroll
+      for (int c = 0; c < CPW; ++c) {
+        const int nt = (c == 0 ? warp : NT8 - 1 - warp);
+        if (nt <= q && nt < 2 * rb + 2) {
+          const float* bp = sN + (8 * q + t) * LD + 8 * nt + g;
+          uint32_t bh0, bl0, bh1, bl1;
+          split(bp[0], bh0, bl0);
+          split(bp[4 * LD], bh1, bl1);
+          float (&d)[4] = acc[rb * (CPW) + c];
+          mma_tf32(d, ah[0], ah[1], ah[2], ah[3], bh0, bh1);
+          mma_tf32(d, al[0], al[1], al[2], al[3], bh0, bh1);
+          mma_tf32(d, ah[0], ah[1], ah[2], ah[3], bl0, bl1);
+        }
+      }
+    }
+  }
+  __syncthreads();   // every warp has read all it needs of N: its space takes R
+#pragma unroll
+  for (int rb = 0; rb < C / 16; ++rb) {
+#pragma unroll
+    for (int c = 0; c < CPW; ++c) {
+      const int nt = (c == 0 ? warp : NT8 - 1 - warp);
+      if (nt < 2 * rb + 2) {
+        const float (&d)[4] = acc[rb * (CPW) + c];
+        const int ra = 16 * rb + g, col = 8 * nt + 2 * t;
+        const float2 xa = *reinterpret_cast<const float2*>(sX + ra * LD + col);
+        const float2 xb = *reinterpret_cast<const float2*>(sX + (ra + 8) * LD + col);
+        // R = I - X - X N, rounded to TF32 once (it is only ever an MMA operand)
+        float2 r0, r1;
+        r0.x = __uint_as_float(to_tf32((col == ra ? 1.f : 0.f) - xa.x - d[0]));
+        r0.y = __uint_as_float(to_tf32((col + 1 == ra ? 1.f : 0.f) - xa.y - d[1]));
+        r1.x = __uint_as_float(to_tf32((col == ra + 8 ? 1.f : 0.f) - xb.x - d[2]));
+        r1.y = __uint_as_float(to_tf32((col + 1 == ra + 8 ? 1.f : 0.f) - xb.y - d[3]));
+        *reinterpret_cast<float2*>(sN + ra * LD + col) = r0;
+        *reinterpret_cast<float2*>(sN + (ra + 8) * LD + col) = r1;
+      }
+    }
+  }
+  __syncthreads();
+  // ---- X + R X on the same tiles (R from shared memory, already TF32; X rounded on the fly)
+#pragma unroll
+  for (int rb = 0; rb < C / 16; ++rb) {
+#pragma unroll
+    for (int c = 0; c < CPW; ++c) {
+      const int nt = (c == 0 ? warp : NT8 - 1 - warp);
+      const int ra = 16 * rb + g, col = 8 * nt + 2 * t;
+      float (&d)[4] = acc[rb * (CPW) + c];
+      if (nt < 2 * rb + 2) {
+        const float2 xa = *reinterpret_cast<const float2*>(sX + ra * LD + col);
+        const float2 xb = *reinterpret_cast<const float2*>(sX + (ra + 8) * LD + col);
+        d[0] = xa.x; d[1] = xa.y; d[2] = xb.x; d[3] = xb.y;
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 2 * rb + 2; ++q) {
+      bool any = false;
+#pragma unroll
+      for (int c = 0; c < CPW; ++c) any = any || ((c == 0 ? warp : NT8 - 1 - warp) <= q);
+      if (!any) continue;
+      const float* ap = sN + (16 * rb + g) * LD + 8 * q + t;
+      const uint32_t a0 = __float_as_uint(ap[0]), a1 = __float_as_uint(ap[8 * LD]), a2 = __float_as_uint(ap[4]),
+                     a3 = __float_as_uint(ap[8 * LD + 4]);
+#pragma unroll
+      for (int c = 0; c < CPW; ++c) {
+        const int nt = (c == 0 ? warp : NT8 - 1 - warp);
+        if (nt <= q && nt < 2 * rb + 2) {
+          const float* bp = sX + (8 * q + t) * LD + 8 * nt + g;
+          mma_tf32(acc[rb * (CPW) + c], a0, a1, a2, a3, to_tf32(bp[0]), to_tf32(bp[4 * LD]));
+        }
+      }
+    }
+  }
+  __syncthreads();   // every warp has read the old X
+#pragma unroll
+  for (int rb = 0; rb < C / 16; ++rb) {
+#pragma unroll
+    for (int c = 0; c < CPW; ++c) {
+      const int nt = (c == 0 ? warp : NT8 - 1 - warp);
+      if (nt < 2 * rb + 2) {
+        const float (&d)[4] = acc[rb * (CPW) + c];
+        const int ra = 16 * rb + g, col = 8 * nt + 2 * t;
+        float2 va, vb;   // the structure of a unit lower triangular matrix is written as constants
+        va.x = (col < ra) ? d[0] : (col == ra ? 1.f : 0.f);
+        va.y = (col + 1 < ra) ? d[1] : (col + 1 == ra ? 1.f : 0.f);
+        vb.x = (col < ra + 8) ? d[2] : (col == ra + 8 ? 1.f : 0.f);
+        vb.y = (col + 1 < ra + 8) ? d[3] : (col + 1 == ra + 8 ? 1.f : 0.f);
+        *reinterpret_cast<float2*>(sX + ra * LD + col) = va;
+        *reinterpret_cast<float2*>(sX + (ra + 8) * LD + col) = vb;
+      }
+    }
+  }
+  __syncthreads();
+}
+
 // 16x16 leaf by forward substitution (Sec. 3.1): lane j owns column j of the inverse; rows of N are read as
 // broadcast float4; the block is overwritten by its inverse (zeros above the diagonal, ones on it).
 template <int LD>
@@ -278,6 +418,10 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
+}
+// The same with fp16 x fp16 operands (format code 0 for both): only the instruction descriptor differs.
+__host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N, int b_mn) {
+  return (1u << 4) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 // kind::tf32: fp32 data in shared memory read as TF32, fp32 accumulate, K = 8 per instruction.
 __host__ __device__ constexpr uint32_t umma_idesc_tf32(int M, int N, int b_mn) {
@@ -331,6 +475,20 @@ __device__ __forceinline__ void tmem_ld_16x128(float (&r)[16][4], uint32_t taddr
         "=f"(r[12][0]), "=f"(r[12][1]), "=f"(r[12][2]), "=f"(r[12][3]), "=f"(r[13][0]), "=f"(r[13][1]), "=f"(r[13][2]), "=f"(r[13][3]),
         "=f"(r[14][0]), "=f"(r[14][1]), "=f"(r[14][2]), "=f"(r[14][3]), "=f"(r[15][0]), "=f"(r[15][1]), "=f"(r[15][2]), "=f"(r[15][3])
       : "r"(taddr));
+}
+
+// Accumulator fragments back into tensor memory (16 lanes x 32 columns), and the wait that makes them visible.
+__device__ __forceinline__ void tmem_st_16x32(const float (&r)[4][4], uint32_t taddr) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.16x256b.x4.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+      ::"f"(r[0][0]), "f"(r[0][1]), "f"(r[0][2]), "f"(r[0][3]), "f"(r[1][0]), "f"(r[1][1]), "f"(r[1][2]), "f"(r[1][3]),
+        "f"(r[2][0]), "f"(r[2][1]), "f"(r[2][2]), "f"(r[2][3]), "f"(r[3][0]), "f"(r[3][1]), "f"(r[3][2]), "f"(r[3][3]),
+        "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void stmatrix_x4(uint32_t addr, uint32_t m0, uint32_t m1, uint32_t m2, uint32_t m3) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
 }
 
 // Epilogue of one 16-row x 64-column piece of W or U: accumulator fragments from tensor memory ->

@@ -21,18 +21,18 @@
 //      staging tile with stmatrix and leave as 16-byte stores covering 128 contiguous bytes per row.
 // Every mbarrier wait is bounded; on expiry the kernel raises the status word, frees its tensor
 // memory and returns.
+#pragma once
 #include <cuda.h>
 
 #include <mutex>
 
-#define TRI_INV_DEV_DEFINE_EXPORTS  // only read by the development header, which the default build never includes
 #include "tc_device.cuh"
 
 namespace tri_inv {
 namespace {
 
 // ------------------------------------------------------------------------------------------ layout
-template <int C, int D, bool SER, bool BO = false>
+template <int C, int D, bool SER, bool BO = false, bool REF = false, bool H16 = false>
 struct Cfg {
   // BO: build-only specialisation (tri_inv_build at C = 64): no V tile, no WY operand or staging, 64 TMEM
   // columns, so six CTAs fit on an SM instead of four.
@@ -46,12 +46,20 @@ struct Cfg {
   // Block recursion at C = 128: the K / V tiles share the space of the fp32 N/X matrix (K is only needed
   // for the Gram product before N is written, and both tiles are fetched again, from L2, for the WY step),
   // which brings the CTA under half an SM's shared memory: two CTAs per SM instead of one.
-  static constexpr bool ALIAS = (C == 128) && !SER;
-  static constexpr bool RELOAD = SER || ALIAS;    // K (and V) are requested after the inversion
+  // REF (one step of iterative refinement after the recursion): N is kept, in fp32, where the K and V tiles are
+  // (the Gram product is done with K by then), so both tiles are fetched again afterwards as in the series variant.
+  static_assert(!REF || (!SER && !BO), "refinement follows the block recursion of the full kernel");
+  // H16 (product series with fp16 operands): Y and X are half the size and one copy of Y serves as both operands, so
+  // they fit in the space of the fp32 matrix and the series needs none of the tiles' space: the layout is the
+  // block recursion's (tiles kept at C = 64, aliased with the matrix at C = 128), not the fp32 series'.
+  static_assert(!H16 || SER, "fp16 operands are a variant of the product series");
+  static constexpr bool ALIAS = (C == 128) && (!SER || H16) && !REF;
+  static constexpr bool RELOAD = (SER && !H16) || ALIAS || REF;    // K (and V) are requested after the inversion
   static constexpr int OFF_K = 0;
   static constexpr int OFF_V = TILE_BYTES;
   static constexpr int X_BYTES = C * LD * 4;
-  static constexpr int OFF_X = ALIAS ? 0 : (BO ? TILE_BYTES : 2 * TILE_BYTES);
+  static constexpr int TILES_BYTES = (REF && X_BYTES > 2 * TILE_BYTES) ? (X_BYTES + 1023) / 1024 * 1024 : 2 * TILE_BYTES;  // REF: room for N
+  static constexpr int OFF_X = ALIAS ? 0 : (BO ? TILE_BYTES : TILES_BYTES);
   // A' (bf16, C x C) and the per-warp 2 KiB output staging tiles: inside the N/X matrix's space once it has
   // been read (A' first, staging behind it), or, with ALIAS, in a region of their own where the staging
   // reuses A' after the WY products have completed.
@@ -72,22 +80,24 @@ struct Cfg {
   static constexpr int END_PLAIN = OFF_R + C * 4 + 32;
   // product-series variant at C = 128: X needs a buffer of its own (at C = 64 it fits where the V tile was)
   static constexpr int OFF_XS = (END_PLAIN + 1023) / 1024 * 1024;
-  static constexpr int BYTES = (SER && C == 128) ? OFF_XS + C * C * 4 : END_PLAIN;
+  static constexpr int BYTES = (SER && !H16 && C == 128) ? OFF_XS + C * C * 4 : END_PLAIN;
+  static_assert(!H16 || 2 * C * C * 2 <= X_BYTES, "the two fp16 operands live in the fp32 matrix's space");
   static constexpr int SMEM = BYTES;
   static constexpr int CTAS_PER_SM = (C == 64) ? (BO ? 6 : 4) : (ALIAS ? 2 : 1);
   static constexpr int TMEM_COLS = (C == 64) ? (BO ? 64 : 128) : 256;
 };
 
 // Byte offset of the 16-byte chunk holding features [f, f+8) of row r inside a swizzled tile.
-template <int C, int D, bool SER, bool RAW, bool BO>
-__global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK,
+template <int C, int D, bool SER, bool RAW, bool BO, bool REF, bool H16>
+__global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SER, BO, REF, H16>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                              const __grid_constant__ CUtensorMap tmV, const __grid_constant__ KParams p) {
-  using cfg = Cfg<C, D, SER, BO>;
+  using cfg = Cfg<C, D, SER, BO, REF, H16>;
   static_assert(D == 128, "tiles are two 64-feature boxes wide");
   constexpr int LD = cfg::LD;
   constexpr int TMEM_COLS = cfg::TMEM_COLS;
   extern __shared__ __align__(1024) uint8_t smem[];  // swizzled tiles need a 1024-byte aligned base
   float* sX = reinterpret_cast<float*>(smem + cfg::OFF_X);
+  float* sN = reinterpret_cast<float*>(smem + cfg::OFF_K);          // REF only: N kept for the refinement step, where the tiles were
   float* sBeta = reinterpret_cast<float*>(smem + cfg::OFF_BETA);
   float* sG = reinterpret_cast<float*>(smem + cfg::OFF_G);
   float* sR = reinterpret_cast<float*>(smem + cfg::OFF_R);          // raw front end: 1 / |k_i|
@@ -377,7 +387,150 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         __syncthreads();
       };
 
-      if constexpr (SER) {
+      if constexpr (SER && H16) {
+        // ---- 3''. product series (Alg. 5) with fp16 operands (the paper's preferred half-precision format, Sec. 4.1).
+        // Y (= N at first) and the operand copy of X are fp16 K-major swizzled tiles (64 columns per 128-byte row)
+        // in the space of the fp32 matrix; one stored copy of Y is the A operand (K-major) of Y.Y and the B operand
+        // (MN-major, which 16-bit types allow) of both products.  X itself lives in tensor memory in fp32: it is
+        // put there once (I - N) and every round accumulates X.Y on top of it, so only its fp16 copy is rewritten.
+        // Operands are written with stmatrix straight from the accumulator-fragment registers.
+        constexpr int R = (C == 64) ? 5 : 6;  // log2(C) - 1 rounds
+        const uint32_t sYh = smem_u32(smem + cfg::OFF_X), sXh = sYh + C * C * 2;
+        const int ra = 16 * rb + g, rbw = ra + 8;
+        // 16 rows x 16 columns (n-tiles nt, nt + 1) of this warp's rows -> fp16 -> one stmatrix into an operand tile
+        auto put16 = [&](uint32_t tile, int nt, const float (&lo)[4], const float (&hi)[4]) {
+          const int mi = lane >> 3, r = 16 * rb + (lane & 7) + 8 * (mi & 1);
+          const int chunk = (nt & 7) + (mi >> 1);
+          const uint32_t addr = tile + (nt >> 3) * cfg::BOX_BYTES + r * 128 + ((chunk ^ (r & 7)) << 4);
+          stmatrix_x4(addr, pack_f16(lo[0], lo[1]), pack_f16(lo[2], lo[3]), pack_f16(hi[0], hi[1]), pack_f16(hi[2], hi[3]));
+        };
+        {
+          const float beta_a = sBeta[ra], beta_b = sBeta[rbw], g_a = sG[ra], g_b = sG[rbw];
+          float sacc[C / 8][4];
+          if constexpr (C == 64) tmem_ld_16x64(sacc, tmem_rows); else tmem_ld_16x128(sacc, tmem_rows);
+          tmem_wait_ld();
+          float ba = beta_a, bb = beta_b;
+          if (raw) {
+            publish_inv_norms(sacc);
+            ba *= sR[ra];
+            bb *= sR[rbw];
+          }
+#pragma unroll
+          for (int nt = 0; nt < C / 8; ++nt) {
+            const int c = 8 * nt + 2 * t;
+            float n4[4] = {0.f, 0.f, 0.f, 0.f};
+            if (nt / 2 <= rb) {  // tiles on or below the diagonal of this row block
+              const float2 gc = *reinterpret_cast<const float2*>(sG + c);
+              const float2 rc = raw ? *reinterpret_cast<const float2*>(sR + c) : make_float2(1.f, 1.f);
+              n4[0] = (c < ra) ? ba * rc.x * sacc[nt][0] * ex2_approx(g_a - gc.x) : 0.f;
+              n4[1] = (c + 1 < ra) ? ba * rc.y * sacc[nt][1] * ex2_approx(g_a - gc.y) : 0.f;
+              n4[2] = (c < rbw) ? bb * rc.x * sacc[nt][2] * ex2_approx(g_b - gc.x) : 0.f;
+              n4[3] = (c + 1 < rbw) ? bb * rc.y * sacc[nt][3] * ex2_approx(g_b - gc.y) : 0.f;
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sacc[nt][e] = n4[e];     // N replaces S in the registers
+          }
+          // the Gram product has completed (the K tile, where the operands go at C = 128, has no reader left)
+#pragma unroll
+          for (int nt = 0; nt < C / 8; nt += 2) put16(sYh, nt, sacc[nt], sacc[nt + 1]);
+#pragma unroll
+          for (int nt = 0; nt < C / 8; ++nt) {
+            const int c = 8 * nt + 2 * t;
+            sacc[nt][0] = (c == ra ? 1.f : 0.f) - sacc[nt][0];
+            sacc[nt][1] = (c + 1 == ra ? 1.f : 0.f) - sacc[nt][1];
+            sacc[nt][2] = (c == rbw ? 1.f : 0.f) - sacc[nt][2];
+            sacc[nt][3] = (c + 1 == rbw ? 1.f : 0.f) - sacc[nt][3];
+          }
+#pragma unroll
+          for (int nt = 0; nt < C / 8; nt += 2) put16(sXh, nt, sacc[nt], sacc[nt + 1]);
+          // X = I - N into tensor memory (columns C .. 2C - 1), where the rounds accumulate on it
+#pragma unroll
+          for (int b4 = 0; b4 < C / 8; b4 += 4) {
+            const float q4[4][4] = {{sacc[b4][0], sacc[b4][1], sacc[b4][2], sacc[b4][3]},
+                                    {sacc[b4 + 1][0], sacc[b4 + 1][1], sacc[b4 + 1][2], sacc[b4 + 1][3]},
+                                    {sacc[b4 + 2][0], sacc[b4 + 2][1], sacc[b4 + 2][2], sacc[b4 + 2][3]},
+                                    {sacc[b4 + 3][0], sacc[b4 + 3][1], sacc[b4 + 3][2], sacc[b4 + 3][3]}};
+            tmem_st_16x32(q4, tmem_rows + C + 8 * b4);
+          }
+          tmem_wait_st();
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        constexpr uint32_t idesc_h = umma_idesc_f16(C, C, 1);
+#pragma unroll 1
+        for (int s = 0; s <= R; ++s) {
+          if (tid == 0 && !bad) {
+            tc_fence_after();
+            // Y = N^p with p = 2^s is zero within p of the diagonal: steps of sixteen k whose operands are structurally
+            // zero are not issued (Y.Y: k in [p, C-1-p]; X.Y: k in [p, C-1]).
+            const int pw = 1 << s;
+            auto da = [&](uint32_t tile, int ks) { return umma_desc(tile + (ks >> 2) * cfg::BOX_BYTES + (ks & 3) * 32, 16, 1024); };
+            auto db = [&](int ks) { return umma_desc(sYh + ks * 2048, cfg::BOX_BYTES, 1024); };
+            if (s < R) {
+              const int k_lo = pw >> 4, k_hi = (C - 1 - pw) >> 4;
+#pragma unroll
+              for (int ks = 0; ks < C / 16; ++ks) {
+                if (ks < k_lo || ks > k_hi) continue;
+                umma_bf16(tmem, da(sYh, ks), db(ks), idesc_h, ks > k_lo);
+              }
+            }
+            if (s >= 1) {
+              const int k_lo = pw >> 4;
+#pragma unroll
+              for (int ks = 0; ks < C / 16; ++ks) {
+                if (ks < k_lo) continue;
+                umma_bf16(tmem + C, da(sXh, ks), db(ks), idesc_h, 1u);   // on top of X
+              }
+            }
+            umma_commit(bar_mma);
+          }
+          wait(bar_mma, ph_mma);
+          ph_mma ^= 1;
+          tc_fence_after();
+          if (s < R) {
+            // new operands, 32 columns at a time: Y <- Y.Y (its readers, the MMAs, have completed), X's fp16 copy
+#pragma unroll
+            for (int b4 = 0; b4 < C / 8; b4 += 4) {
+              float f[4][4];
+              tmem_ld_16x32(f, tmem_rows + 8 * b4);
+              tmem_wait_ld();
+              put16(sYh, b4, f[0], f[1]);
+              put16(sYh, b4 + 2, f[2], f[3]);
+              if (s >= 1) {
+                tmem_ld_16x32(f, tmem_rows + C + 8 * b4);
+                tmem_wait_ld();
+                put16(sXh, b4, f[0], f[1]);
+                put16(sXh, b4 + 2, f[2], f[3]);
+              }
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            __syncthreads();
+          }
+        }
+        // the result leaves tensor memory for the fp32 matrix used by the store and WY steps (over the operands, whose
+        // readers have completed); the structure of a unit lower triangular matrix is written as constants
+#pragma unroll
+        for (int b4 = 0; b4 < C / 8; b4 += 4) {
+          float f[4][4];
+          tmem_ld_16x32(f, tmem_rows + C + 8 * b4);
+          tmem_wait_ld();
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const int c = 8 * (b4 + q4) + 2 * t;
+            float2 va, vb;
+            va.x = (c < ra) ? f[q4][0] : (c == ra ? 1.f : 0.f);
+            va.y = (c + 1 < ra) ? f[q4][1] : (c + 1 == ra ? 1.f : 0.f);
+            vb.x = (c < rbw) ? f[q4][2] : (c == rbw ? 1.f : 0.f);
+            vb.y = (c + 1 < rbw) ? f[q4][3] : (c + 1 == rbw ? 1.f : 0.f);
+            *reinterpret_cast<float2*>(sX + ra * LD + c) = va;
+            *reinterpret_cast<float2*>(sX + rbw * LD + c) = vb;
+          }
+        }
+        tc_fence_before();
+        __syncthreads();
+      } else if constexpr (SER) {
         // ---- 3'. product series (Alg. 5) on the tensor core.  Y (= N at first) and X (= I - N at first)
         // are kept in shared memory as fp32 K-major swizzled operands (32 floats per 128-byte row, blocks of
         // 32 columns); one stored copy of Y serves as the A operand (K-major) and as the B operand
@@ -546,6 +699,10 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
               const int c = 16 * jb + 8 * nt + 2 * t;
               *reinterpret_cast<float2*>(sX + ra * LD + c) = make_float2(0.f, 0.f);
               *reinterpret_cast<float2*>(sX + rbw * LD + c) = make_float2(0.f, 0.f);
+              if constexpr (REF) {
+                *reinterpret_cast<float2*>(sN + ra * LD + c) = make_float2(0.f, 0.f);
+                *reinterpret_cast<float2*>(sN + rbw * LD + c) = make_float2(0.f, 0.f);
+              }
             }
           } else {
 #pragma unroll
@@ -567,6 +724,10 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
               }
               *reinterpret_cast<float2*>(sX + ra * LD + c) = va;
               *reinterpret_cast<float2*>(sX + rbw * LD + c) = vb;
+              if constexpr (REF) {   // the Gram product, the K tile's only reader so far, has completed
+                *reinterpret_cast<float2*>(sN + ra * LD + c) = va;
+                *reinterpret_cast<float2*>(sN + rbw * LD + c) = vb;
+              }
             }
           }
         }
@@ -684,6 +845,16 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
         merge_level<C, 64>(sX, warp, lane);
       }
       PHASE(5);
+      if constexpr (REF) {
+        // ---- 5b. one step of iterative refinement (Alg. 6): X <- X + (I - X (I + N)) X, then K and V come back
+        refine_step<C>(sX, sN, warp, lane);
+        if (do_wy) {
+          if (tid == kTidK) issue_k(tok0, h);
+          if (tid == kTidV && need_v) issue_v(tok0, h);
+          ph_k ^= 1;
+          finish_reload();
+        }
+      }
       }
     }
 
@@ -917,49 +1088,9 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO>::NT, Cfg<C, D, SER, BO>::CT
 }
 
 // ------------------------------------------------------------------------------------------ host side
-// Work counters: a launch draws its later items from a {next item, finished CTAs} pair in a static device
-// array, which the last CTA out returns to zero.  A pair must serve ONE launch at a time.  Kernels launched
-// into the same stream run one after the other, so each stream gets a pair of its own (by the stream's unique
-// id) and nothing has to be tracked: no event, no flag, no synchronisation.  There are kCounterSlots pairs per
-// device; launches on further streams, and every launch made during stream capture (a captured launch is
-// replayed later on whatever stream the graph is launched into), get no pair at all and walk their items with
-// a fixed stride instead: same results, slightly less even load.
-constexpr int kCounterSlots = 64;
-__device__ int g_work_counters[kCounterSlots * 2];
-
-struct CounterTable {
-  int* base = nullptr;
-  unsigned long long stream_id[kCounterSlots] = {};
-  int used = 0;
-};
-std::mutex g_table_mu;
-CounterTable g_tables[64];
-
-// The pair of this stream, or nullptr for "no pair: use the fixed stride".
-int* work_counter_for(cudaStream_t stream) {
-  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-  if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) return nullptr;
-  unsigned long long id = 0;
-  if (cudaStreamGetId(stream, &id) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  std::lock_guard<std::mutex> lock(g_table_mu);
-  CounterTable& t = g_tables[dev];
-  if (!t.base) {
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_work_counters) != cudaSuccess) return nullptr;
-    t.base = static_cast<int*>(ptr);
-  }
-  for (int s = 0; s < t.used; ++s)
-    if (t.stream_id[s] == id) return t.base + 2 * s;
-  if (t.used == kCounterSlots) return nullptr;
-  t.stream_id[t.used] = id;
-  return t.base + 2 * t.used++;
-}
-
-template <int C, int D, bool SER, bool RAW, bool BO = false>
+template <int C, int D, bool SER, bool RAW, bool BO = false, bool REF = false, bool H16 = false>
 cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
-  using cfg = Cfg<C, D, SER, BO>;
+  using cfg = Cfg<C, D, SER, BO, REF, H16>;
   KParams p = p_in;
   // Per-device set-up (function attributes are per device) and grid size, done once per device under a lock.
   static std::mutex mu;
@@ -972,9 +1103,9 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   {
     std::lock_guard<std::mutex> lock(mu);
     if (!ctas_per_sm_of[dev]) {
-      e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
+      e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO, REF, H16>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
       if (e != cudaSuccess) return e;
-      e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+      e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO, REF, H16>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
       if (e != cudaSuccess) return e;
       int sms = 0, smem_per_sm = 0;
       if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
@@ -1000,42 +1131,10 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   long long total = (long long)p.n_chunks * p.H;
   long long cap = (long long)n_sm * ctas_per_sm;
   int grid = (int)(total < cap ? total : cap);
-  p.work_counter = (p.ops & kFixedStride) ? nullptr : work_counter_for(stream);
-  tc_kernel<C, D, SER, RAW, BO><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
+  p.work_counter = (p.ops & kFixedStride) ? nullptr : work_counter_for(stream);  // tc_launch.cu
+  tc_kernel<C, D, SER, RAW, BO, REF, H16><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
   return cudaGetLastError();
 }
 
 }  // namespace
-
-// Self-test support: true when every work-counter pair of the current device reads zero (call after a synchronise).
-cudaError_t work_counters_idle(bool* idle) {
-  int host[kCounterSlots * 2];
-  cudaError_t e = cudaMemcpyFromSymbol(host, g_work_counters, sizeof host);
-  if (e != cudaSuccess) return e;
-  *idle = true;
-  for (int v : host) if (v != 0) *idle = false;
-  return cudaSuccess;
-}
-
-cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handled) {
-  *handled = false;
-  if (p.kv_dtype != TRI_INV_BF16) return cudaSuccess;
-  const bool series = (p.method & TRI_INV_METHOD_MASK) == TRI_INV_PRODUCT_SERIES;
-  if (p.d_k != 128 || ((p.ops & kDoWY) && p.V && p.d_v != 128)) return cudaSuccess;
-  // the stride of the 2-D view (H * d * 2 bytes) is a multiple of 16 because d is a multiple of 8
-  *handled = true;
-  const bool raw = (p.ops & (kRaw | kWDecay)) != 0;  // both need the variant that rewrites the K tile
-  if (C == 64) {
-    if (!raw && !series && !(p.ops & (kDoWY | kLoadA))) return launch_one<64, 128, false, false, true>(p, stream);  // tri_inv_build
-    if (raw) return series ? launch_one<64, 128, true, true>(p, stream) : launch_one<64, 128, false, true>(p, stream);
-    return series ? launch_one<64, 128, true, false>(p, stream) : launch_one<64, 128, false, false>(p, stream);
-  }
-  if (C == 128) {
-    if (raw) return series ? launch_one<128, 128, true, true>(p, stream) : launch_one<128, 128, false, true>(p, stream);
-    return series ? launch_one<128, 128, true, false>(p, stream) : launch_one<128, 128, false, false>(p, stream);
-  }
-  *handled = false;
-  return cudaSuccess;
-}
-
 }  // namespace tri_inv

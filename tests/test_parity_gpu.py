@@ -321,12 +321,84 @@ def test_newton_schulz_and_refinement(bnd, cfg, shrink):
     check_A(A, inp, A_ref, N_ref, tol=1e-5, tol_res=5e-5)
 
 
+@pytest.mark.parametrize("C", [64, 128])
+def test_refinement_step_on_the_tensor_cores(bnd, C):
+    """Alg. 6 after the block recursion, bf16 keys (tensor-core kernel): one step brings the forward error from
+    the TF32 level of the merges (about 1e-4) down to a few 1e-6 or better -- Sec. 4.1's remark that one step gives
+    the mixed recursion its lost digits back.  Dense and packed (short chunks), fused, build-only and raw calls."""
+    rng = np.random.default_rng(77 + C)
+    cu = wl.ragged_lengths(5, 5 * C, rng)
+    cases = [wl.make("ref_dense", 2, 6 * C, 4, 128, 128, C, wl.BF16, seed=910 + C),
+             wl.make("ref_packed", 1, int(cu[-1]), 3, 128, 128, C, wl.BF16, seed=920 + C, cu_seqlens=cu, rng=rng)]
+    for inp in cases:
+        A_ref, N_ref, W_ref, U_ref = oracle_all(inp)
+        A0, _, _ = run_fused(bnd, inp, bnd.BLOCK_RECURSIVE)
+        e_plain = max_ratio(A0.cpu().numpy(), A_ref)
+        for m in (bnd.BLOCK_RECURSIVE | bnd.REFINE, bnd.BLOCK_RECURSIVE | bnd.LEAF_SERIES | bnd.REFINE):
+            A, W, U = run_fused(bnd, inp, m)
+            e_ref, _ = check_A(A, inp, A_ref, N_ref, tol=2e-5, tol_res=5e-5)
+            check_WU(W, U, inp, W_ref, U_ref, bnd)
+            assert e_ref < 0.2 * e_plain, (e_plain, e_ref)
+        dev = bnd.to_device(inp)
+        A = bnd.build(dev["K"], dev["beta"], dev["g"], C, method=bnd.BLOCK_RECURSIVE | bnd.REFINE, cu_seqlens=inp.cu_seqlens,
+                      out=nan_like((inp.B, inp.T, inp.H, C), torch.float32))
+        torch.cuda.synchronize()
+        assert bnd.last_device_status() == 0
+        check_A(A, inp, A_ref, N_ref, tol=2e-5, tol_res=5e-5)
+    # the raw front end with the refinement step
+    raw = wl.make_raw("ref_raw", 2, 4 * C, 2, 128, C, wl.BF16, seed=930 + C)
+    Kh, bh, gh = oracle.raw_front_end(raw.K, raw.beta, raw.g, C)
+    A_ref = oracle.build_A(Kh, bh, gh, C)
+    dev = bnd.to_device(raw)
+    A, W, U, _, _ = bnd.fused_raw(dev["K"], dev["V"], dev["beta"], dev["g"], C, method=bnd.BLOCK_RECURSIVE | bnd.REFINE)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    assert max_ratio(A.cpu().numpy(), A_ref) <= 2e-5
+
+
+@pytest.mark.parametrize("C", [64, 128])
+def test_product_series_with_fp16_operands(bnd, C):
+    """Alg. 5 with fp16 operands (TRI_INV_OPERANDS_F16; Sec. 4.1 ranks fp16 above bf16): same tolerances as the TF32
+    series on the configurations' value distributions; dense, packed with short chunks, build-only and raw calls."""
+    rng = np.random.default_rng(177 + C)
+    cu = wl.ragged_lengths(6, 4 * C, rng)
+    m = bnd.PRODUCT_SERIES | bnd.OPERANDS_F16
+    for inp in (wl.make("h16_dense", 2, 5 * C, 4, 128, 128, C, wl.BF16, seed=940 + C),
+                wl.make("h16_packed", 1, int(cu[-1]), 3, 128, 128, C, wl.BF16, seed=950 + C, cu_seqlens=cu, rng=rng)):
+        A_ref, N_ref, W_ref, U_ref = oracle_all(inp)
+        A, W, U = run_fused(bnd, inp, m)
+        check_A(A, inp, A_ref, N_ref)
+        check_WU(W, U, inp, W_ref, U_ref, bnd)
+        dev = bnd.to_device(inp)
+        A = bnd.build(dev["K"], dev["beta"], dev["g"], C, method=m, cu_seqlens=inp.cu_seqlens, out=nan_like((inp.B, inp.T, inp.H, C), torch.float32))
+        torch.cuda.synchronize()
+        assert bnd.last_device_status() == 0
+        check_A(A, inp, A_ref, N_ref)
+    raw = wl.make_raw("h16_raw", 2, 4 * C, 2, 128, C, wl.BF16, seed=960 + C)
+    Kh, bh, gh = oracle.raw_front_end(raw.K, raw.beta, raw.g, C)
+    A_ref = oracle.build_A(Kh, bh, gh, C)
+    dev = bnd.to_device(raw)
+    A, W, U, _, _ = bnd.fused_raw(dev["K"], dev["V"], dev["beta"], dev["g"], C, method=m)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    assert max_ratio(A.cpu().numpy(), A_ref) <= 2e-3
+    # (the first-difference example of Sec. 3.2 is no case for this variant: its powers of N are binomials up to
+    # about 2^C / sqrt(C), far outside fp16's range -- the overflow the header warns of)
+    # fp32 storage has no fp16-operand kernel: a clear refusal, no launch
+    f32 = wl.config(1)
+    d32 = bnd.to_device(f32)
+    with pytest.raises(bnd.TriInvError) as e:
+        bnd.build(d32["K"], d32["beta"], d32["g"], 64, method=m)
+    assert e.value.status == bnd.ERR_UNSUPPORTED
+
+
 def test_method_flag_combinations_rejected(bnd):
     import ctypes
     d = torch.zeros(64, device="cuda")
     desc, _ = bnd.make_desc(1, 64, 1, 128, 128, 64, bnd.BF16)
     L = bnd.load()
-    for bad in (bnd.PRODUCT_SERIES | bnd.REFINE, bnd.BLOCK_RECURSIVE | bnd.ns_iters(4), bnd.NEWTON_SCHULZ | bnd.LEAF_SERIES, 3):
+    for bad in (bnd.PRODUCT_SERIES | bnd.REFINE, bnd.BLOCK_RECURSIVE | bnd.ns_iters(4), bnd.NEWTON_SCHULZ | bnd.LEAF_SERIES, 3,
+                bnd.BLOCK_RECURSIVE | bnd.OPERANDS_F16, bnd.PRODUCT_SERIES | bnd.OPERANDS_F16 | bnd.FORCE_SIMT):
         rc = L.tri_inv_build(bnd._p(d), bnd._p(d), bnd._p(d), bnd._p(d), ctypes.byref(desc), bad, None)
         assert rc == bnd.ERR_UNSUPPORTED, bad
 
