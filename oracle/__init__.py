@@ -56,6 +56,11 @@ def _load():
         vp, i32 = ctypes.c_void_p, ctypes.c_int
         lib.tri_inv_oracle_build.restype = i32
         lib.tri_inv_oracle_build.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, i32]
+        lib.tri_inv_oracle_build_ex.restype = i32
+        lib.tri_inv_oracle_build_ex.argtypes = [vp, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, i32, i32]
+        lib.tri_inv_oracle_recurrence_ex.restype = i32
+        lib.tri_inv_oracle_recurrence_ex.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, vp, ctypes.c_double,
+                                                     i32, i32, i32, i32, i32, i32, vp, i32, i32]
         lib.tri_inv_oracle_wy.restype = i32
         lib.tri_inv_oracle_wy.argtypes = [vp, vp, vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, i32, i32]
         lib.tri_inv_oracle_gdn_recurrence.restype = i32
@@ -118,7 +123,7 @@ def raw_front_end(K_raw, beta_logit, gate_logit, C, cu_seqlens=None):
     return K_hat, beta, g.reshape(B, T, H)
 
 
-def build_A_kda(K, G, beta, C, cu_seqlens=None, return_N=False):
+def build_A_kda_numpy(K, G, beta, C, cu_seqlens=None, return_N=False):
     """Per-channel decay (the KDA row of Table 1): phi = (K * Gamma)(K / Gamma)^T with Gamma = exp(G),
     G [B,T,H,d] the cumulative per-channel log-decay inside each chunk, and beta scaling rows:
         N_ij = beta_i * sum_c K_ic K_jc exp(G_ic - G_jc)   (i > j),      A = (I + N)^{-1}.
@@ -148,6 +153,61 @@ def build_A_kda(K, G, beta, C, cu_seqlens=None, return_N=False):
                     N[t0:t0 + r, h, :r] = n
     A = A.reshape(B, T, H, C)
     return (A, N.reshape(B, T, H, C)) if return_N else A
+
+
+def build_A_kda(K, G, beta, C, cu_seqlens=None, return_N=False, n_threads=0):
+    """Per-channel decay (the KDA row of Table 1) by the C oracle: N_ij = beta_i sum_c K_ic K_jc exp(G_ic - G_jc) by
+    plain loops, forward substitution for A.  ``build_A_kda_numpy`` is the same definition written with numpy and
+    LAPACK's triangular solve; a pin holds the two against each other."""
+    return _build_ex(K, beta, None, np.ascontiguousarray(G, dtype=np.float32), 0, C, cu_seqlens, n_threads, return_N)
+
+
+def build_A_shifted(K, beta, g, C, cu_seqlens=None, return_N=False, n_threads=0):
+    """The Comba row of Table 1, K K^T * A^{i-1/j}: N_ij = beta_i (k_i . k_j) exp(g_{i-1} - g_j) -- row i decays
+    from token j up to the token BEFORE i.  A = (I + N)^{-1} by forward substitution (C oracle)."""
+    return _build_ex(K, beta, np.ascontiguousarray(g, dtype=np.float32), None, 1, C, cu_seqlens, n_threads, return_N)
+
+
+def _build_ex(K, beta, g, G, gate_shift, C, cu_seqlens, n_threads, return_N):
+    K, dt = _kv(K)
+    B, T, H, d_k = K.shape
+    beta = np.ascontiguousarray(beta, dtype=np.float32)
+    assert beta.shape == (B, T, H) and (g is None or g.shape == (B, T, H)) and (G is None or G.shape == (B, T, H, d_k))
+    A = np.zeros((B, T, H, C), dtype=np.float64)
+    N = np.zeros((B, T, H, C), dtype=np.float64) if return_N else None
+    cu = None if cu_seqlens is None else np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    rc = _load().tri_inv_oracle_build_ex(_ptr(K), dt, _ptr(beta), _ptr(g), _ptr(G), int(gate_shift), _ptr(A), _ptr(N),
+                                         B, T, H, d_k, C, _ptr(cu), 0 if cu is None else len(cu) - 1, int(n_threads))
+    if rc != 0:
+        raise ValueError("tri_inv_oracle_build_ex: invalid arguments")
+    return (A, N) if return_N else A
+
+
+def recurrence_ex(Q, K, V, beta, g, C, G=None, read_before_decay=False, scale=1.0, S0=None, cu_seqlens=None, n_threads=0):
+    """Token-by-token recurrence for the other decay forms of Table 1 (C oracle, fp64): ``G`` [B,T,H,d_k] gives one
+    decay per key feature (KDA row; ``g`` unused); ``read_before_decay`` makes the write's correction read the state
+    before the token's decay (Comba row).  Returns (O, S_final) like ``gdn_recurrence``."""
+    Q, dq = _kv(Q)
+    K, dk = _kv(K)
+    V, dv = _kv(V)
+    if not (dq == dk == dv):
+        Q, K, V, dk = _widen(Q), _widen(K), _widen(V), F64
+    B, T, H, d_k = K.shape
+    d_v = V.shape[3]
+    beta = np.ascontiguousarray(beta, dtype=np.float32)
+    g = None if g is None else np.ascontiguousarray(g, dtype=np.float32)
+    G = None if G is None else np.ascontiguousarray(G, dtype=np.float32)
+    cu = None if cu_seqlens is None else np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    n_seqs = B if cu is None else len(cu) - 1
+    S0 = None if S0 is None else np.ascontiguousarray(S0, dtype=np.float64)
+    O = np.zeros((B, T, H, d_v))
+    S = np.zeros((n_seqs, H, d_k, d_v))
+    rc = _load().tri_inv_oracle_recurrence_ex(_ptr(Q), _ptr(K), _ptr(V), dk, _ptr(beta), _ptr(g), _ptr(G),
+                                              1 if read_before_decay else 0, _ptr(S0), _ptr(O), _ptr(S), float(scale),
+                                              B, T, H, d_k, d_v, C, _ptr(cu), 0 if cu is None else n_seqs, int(n_threads))
+    if rc != 0:
+        raise ValueError("tri_inv_oracle_recurrence_ex: invalid arguments")
+    return O, S
 
 
 def gdn_recurrence(Q, K, V, beta, g, C, scale=1.0, S0=None, cu_seqlens=None, n_threads=0):
@@ -204,6 +264,55 @@ def chunk_scan(Q, K, W, U, g, C, scale=1.0, S0=None, cu_seqlens=None):
                 S = np.exp(gg[-1]) * S + (np.exp(gg[-1] - gg)[:, None] * k).T @ ut
             S_all[s, h] = S
     return O.reshape(B, T, H, d_v), S_all
+
+
+def chunk_scan_kda(Q, K, W, U, G, C, scale=1.0, S0=None, cu_seqlens=None):
+    """The chunk scan with one decay per key feature (KDA row of Table 1), in fp64, chunk by chunk.  With
+    Gamma_i = exp(G_i) (a vector over the key features) and the state S entering the chunk:
+        U~ = U - W S,     P_ij = sum_c Q_ic K_jc exp(G_ic - G_jc)  (j <= i, else 0),
+        O  = scale * ((Q * Gamma) S + P U~),     S <- diag(Gamma_last) S + (K * exp(G_last - G))^T U~.
+    W is the decay-weighted factor A diag(beta) (K * Gamma), U = A diag(beta) V, A from ``build_A_kda``; with those
+    exact this is ``recurrence_ex(G=...)`` re-bracketed (pinned).  Returns (O, S_final)."""
+    Qd, Kd, Wd, Ud = _widen(np.asarray(Q)), _widen(np.asarray(K)), _widen(np.asarray(W)), _widen(np.asarray(U))
+    Gd = np.asarray(G, dtype=np.float64)
+    B, T, H, d_k = Kd.shape
+    d_v = Ud.shape[3]
+    bounds = [(b * T, (b + 1) * T) for b in range(B)] if cu_seqlens is None else \
+             [(int(cu_seqlens[i]), int(cu_seqlens[i + 1])) for i in range(len(cu_seqlens) - 1)]
+    Qf, Kf, Wf, Uf, Gf = (x.reshape((B * T,) + x.shape[2:]) for x in (Qd, Kd, Wd, Ud, Gd))
+    O = np.zeros((B * T, H, d_v))
+    S_all = np.zeros((len(bounds), H, d_k, d_v))
+    for s, (beg, end) in enumerate(bounds):
+        for h in range(H):
+            S = np.zeros((d_k, d_v)) if S0 is None else np.array(S0[s, h], dtype=np.float64)
+            for t0 in range(beg, end, C):
+                t1 = min(t0 + C, end)
+                q, k, w, u, gg = Qf[t0:t1, h], Kf[t0:t1, h], Wf[t0:t1, h], Uf[t0:t1, h], Gf[t0:t1, h]
+                r = t1 - t0
+                P = np.zeros((r, r))
+                for i in range(r):
+                    for j in range(i + 1):
+                        P[i, j] = np.sum(q[i] * k[j] * np.exp(gg[i] - gg[j]))
+                ut = u - w @ S
+                O[t0:t1, h] = scale * ((q * np.exp(gg)) @ S + P @ ut)
+                S = np.exp(gg[-1])[:, None] * S + (k * np.exp(gg[-1][None, :] - gg)).T @ ut
+            S_all[s, h] = S
+    return O.reshape(B, T, H, d_v), S_all
+
+
+def shifted_gate(g, C, cu_seqlens=None):
+    """g_{i-1} for every token (0 at the first token of each chunk): the row factor of the Comba row's decay matrix."""
+    g = np.asarray(g, dtype=np.float64)
+    B, T, H = g.shape
+    gf = g.reshape(B * T, H)
+    out = np.zeros_like(gf)
+    bounds = [(b * T, (b + 1) * T) for b in range(B)] if cu_seqlens is None else \
+             [(int(cu_seqlens[i]), int(cu_seqlens[i + 1])) for i in range(len(cu_seqlens) - 1)]
+    for beg, end in bounds:
+        for t in range(beg, end):
+            if (t - beg) % C:
+                out[t] = gf[t - 1]
+    return out.reshape(B, T, H)
 
 
 def threads(n_threads: int = 0) -> int:

@@ -79,11 +79,33 @@ static int64_t list_chunks(int B, int T, int C, const int32_t* cu, int n_seqs, c
  * A = (I+N)^{-1} for every chunk; N_out (nullable) receives N itself.
  * All pointers are HOST pointers.  Returns 0, or 1 on invalid arguments.
  */
+int tri_inv_oracle_build_ex(const void* K, int kv_dtype, const float* beta, const float* g, const float* G, int gate_shift,
+                            double* A, double* N_out,
+                            int B, int T, int H, int d_k, int C,
+                            const int32_t* cu_seqlens, int n_seqs, int n_threads);
+
 int tri_inv_oracle_build(const void* K, int kv_dtype, const float* beta, const float* g,
                          double* A, double* N_out,
                          int B, int T, int H, int d_k, int C,
                          const int32_t* cu_seqlens, int n_seqs, int n_threads) {
-  if (!K || !beta || !g || !A || B < 1 || T < 0 || H < 1 || d_k < 1 || C < 1) return 1;
+  return tri_inv_oracle_build_ex(K, kv_dtype, beta, g, NULL, 0, A, N_out, B, T, H, d_k, C, cu_seqlens, n_seqs, n_threads);
+}
+
+/*
+ * The same with the other decay matrices of Table 1:
+ *   G != NULL (g ignored):  per-channel decay, the KDA row,   N_ij = beta_i sum_c K_ic K_jc exp(G_ic - G_jc);
+ *                           G [B,T,H,d_k] fp32 is the cumulative per-channel log-decay inside each chunk;
+ *   gate_shift != 0:        the Comba row's decay A^{i-1/j},  N_ij = beta_i (k_i . k_j) exp(g_{i-1} - g_j)
+ *                           (row i takes the cumulative log-decay of the token before it; the first row of a chunk
+ *                           has no entry below the diagonal, so no g_{-1} is ever needed).
+ * The exponent is always taken of the difference.
+ */
+int tri_inv_oracle_build_ex(const void* K, int kv_dtype, const float* beta, const float* g, const float* G, int gate_shift,
+                            double* A, double* N_out,
+                            int B, int T, int H, int d_k, int C,
+                            const int32_t* cu_seqlens, int n_seqs, int n_threads) {
+  if (!K || !beta || (!g && !G) || !A || B < 1 || T < 0 || H < 1 || d_k < 1 || C < 1) return 1;
+  if (G && gate_shift) return 1;
   if (cu_seqlens && (B != 1 || n_seqs < 0 || cu_seqlens[0] != 0 || cu_seqlens[n_seqs] != T)) return 1;
   chunk_t* ch = NULL;
   int64_t n_chunks = list_chunks(B, T, C, cu_seqlens, n_seqs, &ch);
@@ -110,9 +132,17 @@ int tri_inv_oracle_build(const void* K, int kv_dtype, const float* beta, const f
         for (int j = 0; j < i; ++j) {
           size_t bj = (size_t)(t0 + j) * H + h;
           double s = 0.0;
-          for (int k = 0; k < d_k; ++k)
-            s += widen(K, kv_dtype, bi * d_k + k) * widen(K, kv_dtype, bj * d_k + k);
-          N[i * C + j] = (double)beta[bi] * s * exp((double)g[bi] - (double)g[bj]);
+          if (G) {
+            for (int k = 0; k < d_k; ++k)
+              s += widen(K, kv_dtype, bi * d_k + k) * widen(K, kv_dtype, bj * d_k + k) *
+                   exp((double)G[bi * d_k + k] - (double)G[bj * d_k + k]);
+            N[i * C + j] = (double)beta[bi] * s;
+          } else {
+            for (int k = 0; k < d_k; ++k)
+              s += widen(K, kv_dtype, bi * d_k + k) * widen(K, kv_dtype, bj * d_k + k);
+            double g_row = gate_shift ? (double)g[bi - (size_t)H] : (double)g[bi];   /* i >= 1 here: the token before is in the chunk */
+            N[i * C + j] = (double)beta[bi] * s * exp(g_row - (double)g[bj]);
+          }
         }
       }
       /* forward substitution on (I+N) X = I, one column at a time */
@@ -218,12 +248,36 @@ int tri_inv_oracle_threads(int n_threads) {
  * [n_sequences,H,d_k,d_v] double (both nullable); O [B,T,H,d_v] double.  HOST pointers.
  * OpenMP over (sequence, head); every sum in double in index order.
  */
+int tri_inv_oracle_recurrence_ex(const void* Q, const void* K, const void* V, int kv_dtype,
+                                 const float* beta, const float* g, const float* G, int read_before_decay, const double* S0,
+                                 double* O, double* S_out, double scale,
+                                 int B, int T, int H, int d_k, int d_v, int C,
+                                 const int32_t* cu_seqlens, int n_seqs, int n_threads);
+
 int tri_inv_oracle_gdn_recurrence(const void* Q, const void* K, const void* V, int kv_dtype,
                                   const float* beta, const float* g, const double* S0,
                                   double* O, double* S_out, double scale,
                                   int B, int T, int H, int d_k, int d_v, int C,
                                   const int32_t* cu_seqlens, int n_seqs, int n_threads) {
-  if (!Q || !K || !V || !beta || !g || !O || B < 1 || T < 0 || H < 1 || d_k < 1 || d_v < 1 || C < 1) return 1;
+  return tri_inv_oracle_recurrence_ex(Q, K, V, kv_dtype, beta, g, NULL, 0, S0, O, S_out, scale, B, T, H, d_k, d_v, C,
+                                      cu_seqlens, n_seqs, n_threads);
+}
+
+/*
+ * The same recurrence for the other two decay forms of Table 1.
+ *   G != NULL (g ignored): one decay per key feature (KDA row): a_{t,c} = G_{t,c} - G_{t-1,c}, row c of S is
+ *                          multiplied by exp(a_{t,c}); everything else as above.
+ *   read_before_decay:     the write's correction reads the state BEFORE this token's decay (Comba row, whose decay
+ *                          matrix therefore runs from j to i-1):
+ *                              r = v_t - S^T k_t;   S <- exp(a_t) S;   S <- S + beta_t k_t r^T;   o_t = scale S^T q_t.
+ */
+int tri_inv_oracle_recurrence_ex(const void* Q, const void* K, const void* V, int kv_dtype,
+                                 const float* beta, const float* g, const float* G, int read_before_decay, const double* S0,
+                                 double* O, double* S_out, double scale,
+                                 int B, int T, int H, int d_k, int d_v, int C,
+                                 const int32_t* cu_seqlens, int n_seqs, int n_threads) {
+  if (!Q || !K || !V || !beta || (!g && !G) || !O || B < 1 || T < 0 || H < 1 || d_k < 1 || d_v < 1 || C < 1) return 1;
+  if (G && read_before_decay) return 1;
   if (cu_seqlens && (B != 1 || n_seqs < 0 || cu_seqlens[0] != 0 || cu_seqlens[n_seqs] != T)) return 1;
   int nseq = cu_seqlens ? n_seqs : B;
 #ifdef _OPENMP
@@ -243,13 +297,31 @@ int tri_inv_oracle_gdn_recurrence(const void* Q, const void* K, const void* V, i
       for (int64_t t = beg; t < end; ++t) {
         size_t th = (size_t)t * H + h;
         int first_of_chunk = ((t - beg) % C) == 0;
-        double a = (double)g[th] - (first_of_chunk ? 0.0 : (double)g[th - H]);
-        double alpha = exp(a), b = (double)beta[th];
-        for (int i = 0; i < d_k * d_v; ++i) S[i] *= alpha;
-        for (int j = 0; j < d_v; ++j) {
-          double acc = 0.0;
-          for (int i = 0; i < d_k; ++i) acc += widen(K, kv_dtype, th * d_k + i) * S[i * d_v + j];
-          r[j] = widen(V, kv_dtype, th * d_v + j) - acc;
+        double b = (double)beta[th];
+        if (read_before_decay) {   /* the correction term sees the state as the previous token left it */
+          for (int j = 0; j < d_v; ++j) {
+            double acc = 0.0;
+            for (int i = 0; i < d_k; ++i) acc += widen(K, kv_dtype, th * d_k + i) * S[i * d_v + j];
+            r[j] = widen(V, kv_dtype, th * d_v + j) - acc;
+          }
+        }
+        if (G) {
+          for (int i = 0; i < d_k; ++i) {
+            double a = (double)G[th * d_k + i] - (first_of_chunk ? 0.0 : (double)G[(th - H) * d_k + i]);
+            double alpha = exp(a);
+            for (int j = 0; j < d_v; ++j) S[i * d_v + j] *= alpha;
+          }
+        } else {
+          double a = (double)g[th] - (first_of_chunk ? 0.0 : (double)g[th - H]);
+          double alpha = exp(a);
+          for (int i = 0; i < d_k * d_v; ++i) S[i] *= alpha;
+        }
+        if (!read_before_decay) {
+          for (int j = 0; j < d_v; ++j) {
+            double acc = 0.0;
+            for (int i = 0; i < d_k; ++i) acc += widen(K, kv_dtype, th * d_k + i) * S[i * d_v + j];
+            r[j] = widen(V, kv_dtype, th * d_v + j) - acc;
+          }
         }
         for (int i = 0; i < d_k; ++i) {
           double ki = b * widen(K, kv_dtype, th * d_k + i);

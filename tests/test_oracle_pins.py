@@ -365,24 +365,26 @@ def test_raw_front_end_hand_values_and_generator_recipe():
 # ---------------------------------------------------------------- per-channel decay (KDA row of Table 1)
 
 def test_per_channel_decay_reduces_to_the_scalar_gate_and_to_deltanet():
+    # (the numpy + LAPACK statement, which takes G in fp64; the C statement, which reads G in fp32 as the library does, is
+    # held against it in test_per_channel_chunk_form_equals_its_recurrence)
     x = wl.make("kda", 2, 150, 2, 16, 16, 64, wl.BF16, seed=33)
     # Gamma = 1: plain DeltaNet matrix (g = 0)
-    A0 = oracle.build_A_kda(x.K, np.zeros((2, 150, 2, 16)), x.beta, 64)
+    A0 = oracle.build_A_kda_numpy(x.K, np.zeros((2, 150, 2, 16)), x.beta, 64)
     assert np.abs(A0 - oracle.build_A(x.K, x.beta, np.zeros_like(x.g), 64)).max() < 1e-13
     # the same log-decay on every channel: the GDN scalar gate exp(g_i - g_j)
     G = np.repeat(x.g[..., None].astype(np.float64), 16, axis=-1)
-    A1, N1 = oracle.build_A_kda(x.K, G, x.beta, 64, return_N=True)
+    A1, N1 = oracle.build_A_kda_numpy(x.K, G, x.beta, 64, return_N=True)
     A_ref, N_ref = oracle.build_A(x.K, x.beta, x.g, 64, return_N=True)
     assert np.abs(N1 - N_ref).max() < 1e-14 and np.abs(A1 - A_ref).max() < 1e-13
     # a hand value: k_0 = (1, 2), k_1 = (3, 1), G_0 = (0, 0), G_1 = (-ln 2, -ln 4), beta_1 = 2:
     # N_10 = 2 * (3 * 1 / 2 + 1 * 2 / 4) = 4
     K = np.array([[1.0, 2.0], [3.0, 1.0]], np.float32).reshape(1, 2, 1, 2)
     Gh = np.array([[0.0, 0.0], [-np.log(2.0), -np.log(4.0)]]).reshape(1, 2, 1, 2)
-    A, N = oracle.build_A_kda(K, Gh, np.array([1.0, 2.0]).reshape(1, 2, 1), 2, return_N=True)
+    A, N = oracle.build_A_kda_numpy(K, Gh, np.array([1.0, 2.0]).reshape(1, 2, 1), 2, return_N=True)
     assert abs(N[0, 1, 0, 0] - 4.0) < 1e-14 and abs(A[0, 1, 0, 0] + 4.0) < 1e-14
     # defining identities with a genuinely per-channel gate, ragged chunks included
     Gp = wl.per_channel_gate(x, seed=5)
-    A2, N2 = oracle.build_A_kda(x.K, Gp, x.beta, 64, return_N=True)
+    A2, N2 = oracle.build_A_kda_numpy(x.K, Gp, x.beta, 64, return_N=True)
     for b in range(2):
         for t0, r in ((0, 64), (64, 64), (128, 22)):
             n, a = N2[b, t0:t0 + r, 1, :r], A2[b, t0:t0 + r, 1, :r]
@@ -391,7 +393,7 @@ def test_per_channel_decay_reduces_to_the_scalar_gate_and_to_deltanet():
     assert np.abs(A2 - A_ref).max() > 1e-3      # and it is a different matrix from the scalar-gate one
     # only differences inside a chunk enter: a per-(chunk, head, channel) offset of G changes nothing
     off = np.random.default_rng(6).standard_normal((2, 3, 2, 16)).repeat(64, axis=1)[:, :150]
-    N3 = oracle.build_A_kda(x.K, Gp + off, x.beta, 64, return_N=True)[1]
+    N3 = oracle.build_A_kda_numpy(x.K, Gp + off, x.beta, 64, return_N=True)[1]
     assert np.abs(N3 - N2).max() < 1e-12
 
 
@@ -477,3 +479,87 @@ def test_chunk_form_with_the_inverse_equals_the_recurrence():
         Wp, _ = oracle.wy(A, x.K, None, x.beta, 64, cu_seqlens=cu_seqlens)
         O3, _ = oracle.chunk_scan(Q, x.K, Wp, U, x.g, 64, scale=0.25, S0=S0, cu_seqlens=cu_seqlens)
         assert np.abs(O3 - O2).max() > 1e-3
+
+
+# ---------------------------------------------------------------- the other decay forms of Table 1 (Comba, KDA rows)
+
+def test_shifted_gate_hand_values_and_reductions():
+    """Comba row, K K^T * A^{i-1/j}: N_ij = beta_i (k_i . k_j) exp(g_{i-1} - g_j).  Hand values on three tokens with
+    integer keys; without decay it is the DeltaNet matrix; and it is NOT the GDN matrix when g decreases."""
+    K = np.zeros((1, 3, 1, 2), np.float32)
+    K[0, :, 0] = [[1, 0], [2, 1], [1, 3]]
+    beta = np.array([0.5, 0.25, 2.0], np.float32).reshape(1, 3, 1)
+    g = np.log(np.array([0.5, 0.25, 0.125])).astype(np.float32).reshape(1, 3, 1)
+    A, N = oracle.build_A_shifted(K, beta, g, 4, return_N=True)
+    n = N[0, :, 0, :3]
+    # N_10 = 0.25 * 2 * exp(g0 - g0) = 0.5;  N_20 = 2 * 1 * exp(g1 - g0) = 2 * 0.5;  N_21 = 2 * 5 * exp(g1 - g1) = 10
+    assert np.allclose(n, [[0, 0, 0], [0.5, 0, 0], [1.0, 10.0, 0]], atol=1e-7)
+    a = A[0, :, 0, :3]
+    assert np.allclose(a, [[1, 0, 0], [-0.5, 1, 0], [-1.0 + 10 * 0.5, -10.0, 1]], atol=1e-6)
+    x = wl.make("s", 1, 128, 2, 16, 16, 64, wl.F32, seed=71)
+    zero = np.zeros_like(x.g)
+    assert np.array_equal(oracle.build_A_shifted(x.K, x.beta, zero, 64), oracle.build_A(x.K, x.beta, zero, 64))
+    assert np.abs(oracle.build_A_shifted(x.K, x.beta, x.g, 64) - oracle.build_A(x.K, x.beta, x.g, 64)).max() > 1e-3
+    # the shifted matrix is the plain one with row i rescaled by exp(g_{i-1} - g_i): N_shift = diag(exp(-a)) N
+    _, Ns = oracle.build_A_shifted(x.K, x.beta, x.g, 64, return_N=True)
+    _, Np = oracle.build_A(x.K, x.beta, x.g, 64, return_N=True)
+    a_tok = x.g.astype(np.float64) - oracle.shifted_gate(x.g, 64)
+    assert np.abs(Ns - Np * np.exp(-a_tok)[..., None]).max() < 1e-12
+
+
+def test_comba_chunk_form_equals_its_recurrence():
+    """S_t = (alpha_t I - beta_t k_t k_t^T) S_{t-1} + beta_t k_t v_t^T token by token against the chunk form built from the
+    shifted-gate inverse: U~ = U - W S with W = A diag(beta exp(g_{i-1})) K, then the same output and state formulas
+    as the GDN row.  A hand-worked scalar case separates it from the GDN recurrence."""
+    # scalar state, one token: S0 = 1, alpha = 1/2, beta = 1/2, k = 1, v = 3:  S1 = (1/2 - 1/2) * 1 + 1/2 * 3 = 3/2
+    one = np.ones((1, 1, 1, 1), np.float32)
+    O, S = oracle.recurrence_ex(one, one, 3 * one, np.full((1, 1, 1), 0.5, np.float32), np.log(np.full((1, 1, 1), 0.5, np.float32)),
+                                64, read_before_decay=True, S0=np.ones((1, 1, 1, 1)))
+    assert abs(S[0, 0, 0, 0] - 1.5) < 1e-8 and abs(O[0, 0, 0, 0] - 1.5) < 1e-8     # g = ln(1/2) is carried in fp32
+    # (the GDN form gives alpha S0 + beta (v - alpha S0) = 1/2 + 1/2 (3 - 1/2) = 7/4)
+    _, Sg = oracle.gdn_recurrence(one, one, 3 * one, np.full((1, 1, 1), 0.5, np.float32), np.log(np.full((1, 1, 1), 0.5, np.float32)),
+                                  64, S0=np.ones((1, 1, 1, 1)))
+    assert abs(Sg[0, 0, 0, 0] - 1.75) < 1e-8
+    cu = np.array([0, 70, 71, 230], np.int32)
+    for cu_seqlens, B, T in ((None, 2, 150), (cu, 1, 230)):
+        x = wl.make("c", B, T, 2, 16, 24, 64, wl.F32, seed=81, cu_seqlens=cu_seqlens)
+        Q = wl.queries(x, seed=82)
+        S0 = wl.initial_state(x, seed=83)
+        A = oracle.build_A_shifted(x.K, x.beta, x.g, 64, cu_seqlens=cu_seqlens)
+        gs = oracle.shifted_gate(x.g, 64, cu_seqlens=cu_seqlens)
+        W, _ = oracle.wy(A, x.K.astype(np.float64) * np.exp(gs)[..., None], None, x.beta, 64, cu_seqlens=cu_seqlens)
+        _, U = oracle.wy(A, x.K, x.V, x.beta, 64, cu_seqlens=cu_seqlens)
+        O1, S1 = oracle.chunk_scan(Q, x.K, W, U, x.g, 64, scale=0.5, S0=S0, cu_seqlens=cu_seqlens)
+        O2, S2 = oracle.recurrence_ex(Q, x.K, x.V, x.beta, x.g, 64, read_before_decay=True, scale=0.5, S0=S0, cu_seqlens=cu_seqlens)
+        assert np.abs(O1 - O2).max() < 1e-11 and np.abs(S1 - S2).max() < 1e-11
+        # the unshifted inverse does not reproduce it
+        Ag = oracle.build_A(x.K, x.beta, x.g, 64, cu_seqlens=cu_seqlens)
+        _, Ug = oracle.wy(Ag, x.K, x.V, x.beta, 64, cu_seqlens=cu_seqlens)
+        O3, _ = oracle.chunk_scan(Q, x.K, W, Ug, x.g, 64, scale=0.5, S0=S0, cu_seqlens=cu_seqlens)
+        assert np.abs(O3 - O2).max() > 1e-3
+
+
+def test_per_channel_chunk_form_equals_its_recurrence():
+    """KDA row: one decay per key feature.  The C oracle's N equals the numpy + LAPACK statement of the same formula; the
+    chunk form built from it (W = A diag(beta) (K * Gamma), U = A diag(beta) V, then ``chunk_scan_kda``) equals the
+    token-by-token recurrence; and with the same decay on every feature both reduce to the scalar-gate layer."""
+    cu = np.array([0, 70, 71, 200], np.int32)
+    for cu_seqlens, B, T in ((None, 2, 130), (cu, 1, 200)):
+        x = wl.make("k", B, T, 2, 16, 24, 64, wl.F32, seed=91, cu_seqlens=cu_seqlens)
+        G = wl.per_channel_gate(x, seed=92)
+        Q = wl.queries(x, seed=93)
+        S0 = wl.initial_state(x, seed=94)
+        A, N = oracle.build_A_kda(x.K, G, x.beta, 64, cu_seqlens=cu_seqlens, return_N=True)
+        A2, N2 = oracle.build_A_kda_numpy(x.K, G, x.beta, 64, cu_seqlens=cu_seqlens, return_N=True)
+        assert np.abs(N - N2).max() < 1e-14 and np.abs(A - A2).max() < 1e-12
+        Kg = x.K.astype(np.float64) * np.exp(G.astype(np.float64))
+        W, _ = oracle.wy(A, Kg, None, x.beta, 64, cu_seqlens=cu_seqlens)
+        _, U = oracle.wy(A, x.K, x.V, x.beta, 64, cu_seqlens=cu_seqlens)
+        O1, S1 = oracle.chunk_scan_kda(Q, x.K, W, U, G, 64, scale=0.5, S0=S0, cu_seqlens=cu_seqlens)
+        O2, S2 = oracle.recurrence_ex(Q, x.K, x.V, x.beta, None, 64, G=G, scale=0.5, S0=S0, cu_seqlens=cu_seqlens)
+        assert np.abs(O1 - O2).max() < 1e-10 and np.abs(S1 - S2).max() < 1e-10
+        # same decay on every feature: the scalar-gate layer
+        Gs = np.repeat(x.g[..., None], x.d_k, axis=3)
+        O3, S3 = oracle.recurrence_ex(Q, x.K, x.V, x.beta, None, 64, G=Gs, scale=0.5, S0=S0, cu_seqlens=cu_seqlens)
+        O4, S4 = oracle.gdn_recurrence(Q, x.K, x.V, x.beta, x.g, 64, scale=0.5, S0=S0, cu_seqlens=cu_seqlens)
+        assert np.abs(O3 - O4).max() < 1e-12 and np.abs(S3 - S4).max() < 1e-12
