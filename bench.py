@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 METRIC = "chunk matrices inverted/sec (C=64, d=128, bf16) + % of roofline; max err vs fp64 oracle"
 UNIT = "chunk-matrices/s"
 FALLBACK_HBM_GBS = 6650.0
-OUTPUTS = {"fused": "A fp32 + W,U", "raw": "A fp32 + W,U", "build": "A fp32", "kda": "A fp32", "wy": "W,U", "scan": "O", "layer": "O"}
+OUTPUTS = {"fused": "A fp32 + W,U", "raw": "A fp32 + W,U", "build": "A fp32", "kda": "A fp32", "kda_fused": "A fp32 + W,U", "wy": "W,U", "scan": "O", "layer": "O"}
 
 # DRAM bytes per chunk matrix moved by the fused kernel (dram__bytes_read.sum + dram__bytes_write.sum
 # of one ncu capture divided by the matrices of that launch); see profiles/.  None = not captured yet.
@@ -52,6 +52,8 @@ def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True, call="fused"):
                (3 * C * d_k * elt + C * d_v * elt + C * 4 + C * d_v * elt)
     if call == "kda":  # K, G (fp32 per channel) and beta read; A written
         return C * d_k * elt + C * d_k * 4 + C * 4 + C * C * 4
+    if call == "kda_fused":  # what a one-kernel version would move: K, G, V, beta read once; A, W, U written once
+        return C * d_k * elt + C * d_k * 4 + C * d_v * elt + C * 4 + C * C * 4 + C * d_k * elt + C * d_v * elt
     if call == "wy":
         return C * (C - 1) // 2 * 4 + C * d_k * elt + C * d_v * elt + C * 4 + C * d_k * elt + C * d_v * elt
     b = C * d_k * elt + C * d_v * elt + 2 * C * 4 + C * d_k * elt + C * d_v * elt
@@ -202,7 +204,7 @@ def main():
     ap.add_argument("--method", default="block_recursive", choices=["block_recursive", "mixed_recursion", "product_series", "block_recursive_refined", "product_series_f16"])
     ap.add_argument("--paper-T", type=int, default=0,
                     help="instead of --config: the paper's timing shape B=32, H=4, d=128 at this sequence length (1024..16384)")
-    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw", "kda", "scan", "layer"],
+    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw", "kda", "kda_fused", "scan", "layer"],
                     help="entry point timed: the fused path (default, the metric), tri_inv_build alone, tri_inv_wy alone, "
                          "tri_inv_fused_raw (front end folded in; same shapes, un-normalised keys and logits as inputs), "
                          "tri_inv_build_kda (per-channel decay), tri_inv_chunk_scan alone (W and U produced outside the timed "
@@ -255,7 +257,7 @@ def main():
     K, V, beta, g = dev["K"], dev["V"], dev["beta"], dev["g"]
     A = torch.empty((inp.B, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda")
     W, U = torch.empty_like(K), torch.empty_like(V)
-    G = torch.from_numpy(wl.per_channel_gate(inp, seed=3000 + args.config)).cuda() if args.call == "kda" else None
+    G = torch.from_numpy(wl.per_channel_gate(inp, seed=3000 + args.config)).cuda() if args.call in ("kda", "kda_fused") else None
     Q = O = None
     if args.call in ("scan", "layer"):  # the consumer of W and U: queries, outputs, zero initial state
         Q_host = wl.queries(inp, seed=4000 + args.config)
@@ -285,6 +287,8 @@ def main():
         elif args.call == "layer":
             binding.fused(K, V, beta, g, inp.C, method=method | binding.W_DECAY, cu_seqlens=inp.cu_seqlens, out=(None, W, U), stream=stream)
             binding.chunk_scan(Q, K, W, U, g, inp.C, scale=q_scale, cu_seqlens=inp.cu_seqlens, out=O, want_state=False, stream=stream)
+        elif args.call == "kda_fused":
+            binding.fused_kda(K, V, G, beta, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U), stream=stream)
         elif args.call == "kda":
             binding.build_kda(K, G, beta, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
         else:
@@ -382,7 +386,7 @@ def main():
             num[key] = max(num.get(key, 0.0), float(np.abs(x - ref).max()))
             den[key] = max(den.get(key, 0.0), float(np.abs(ref).max()))
 
-        Gs = G.cpu().numpy() if args.call == "kda" else None
+        Gs = G.cpu().numpy() if args.call in ("kda", "kda_fused") else None
         if args.call in ("scan", "layer"):
             O_ref, _ = oracle.gdn_recurrence(Q_host, inp.K, inp.V, inp.beta, inp.g, inp.C, scale=q_scale, cu_seqlens=cu)
             acc("O", binding.to_numpy_f64(O), O_ref)
@@ -391,18 +395,20 @@ def main():
                 Ko, bo, go = inp.K[:, sl], inp.beta[:, sl], inp.g[:, sl]
                 if args.call == "raw":
                     Ko, bo, go = oracle.raw_front_end(Ko, bo, go, inp.C, cu_seqlens=cu)
-                if args.call == "kda":   # the per-channel oracle is a Python loop: a bounded sample of whole chunks
-                    sl = slice(sl.start or 0, (sl.start or 0) + 2 * inp.C) if cu is None else sl
+                if args.call in ("kda", "kda_fused"):
                     A_ref = oracle.build_A_kda(inp.K[:, sl], Gs[:, sl], inp.beta[:, sl], inp.C, cu_seqlens=cu)
+                    Ko = wl.bf16_bits_to_f32(Ko).astype(np.float64) * np.exp(Gs[:, sl].astype(np.float64)) if Ko.dtype == np.uint16 \
+                        else Ko.astype(np.float64) * np.exp(Gs[:, sl].astype(np.float64))   # W = A diag(beta) (K * Gamma)
                 else:
                     A_ref = oracle.build_A(Ko, bo, go, inp.C, cu_seqlens=cu)
                 if args.call != "wy":
                     acc("A", binding.to_numpy_f64(A[:, sl]), A_ref)
                 if args.call not in ("build", "kda"):
-                    W_ref, U_ref = oracle.wy(A_ref, Ko, inp.V[:, sl], bo, inp.C, cu_seqlens=cu)
+                    W_ref, _ = oracle.wy(A_ref, Ko, None, bo, inp.C, cu_seqlens=cu)
+                    _, U_ref = oracle.wy(A_ref, inp.K[:, sl], inp.V[:, sl], bo, inp.C, cu_seqlens=cu)
                     acc("W", binding.to_numpy_f64(W[:, sl]), W_ref)
                     acc("U", binding.to_numpy_f64(U[:, sl]), U_ref)
-        err = {"sample": "first %d tokens of every %d" % (2 * inp.C, slab) if (args.call == "kda" and cu is None) else "all tokens"}
+        err = {"sample": "all tokens"}
         if args.call in ("scan", "layer"):
             err["reference"] = "token-by-token recurrence"
         for key in num:
@@ -417,7 +423,7 @@ def main():
         traffic = NCU_TRAFFIC_BYTES_PER_MATRIX.get((args.config, args.method)) if args.call == "fused" else None
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": None if traffic is None else traffic * n_mat, "peak_source": "of " + peak_kind,
-                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "kda": "per-channel-decay build+invert", "wy": "WY apply", "scan": "chunk scan (state recurrence + output)", "layer": "fused build+invert+WY, then chunk scan (2 launches)"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
+                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "kda": "per-channel-decay build+invert", "kda_fused": "per-channel-decay build+invert, key scaling, WY (3 launches)", "wy": "WY apply", "scan": "chunk scan (state recurrence + output)", "layer": "fused build+invert+WY, then chunk scan (2 launches)"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
                     "algorithmic_bytes_per_launch": alg_bytes * n_mat}
         cpu = None
         if world == 1 and not args.no_cpu_baseline:

@@ -104,6 +104,13 @@ enum {
    * which the unstable series (Sec. 3.2) can produce on badly conditioned chunks.  Half the operand bytes and one
    * stored copy of Y for both operand roles: the fast form of the series.  Elsewhere TRI_INV_ERR_UNSUPPORTED. */
   TRI_INV_OPERANDS_F16 = 0x400,
+  /* flag, tri_inv_build / tri_inv_fused / tri_inv_fused_raw: the decay matrix of Table 1's Comba row, A^{i-1/j}:
+   *     N_ij = beta_i (k_i . k_j) exp(g_{i-1} - g_j)      (i > j)
+   * -- row i decays from token j up to the token BEFORE i, which is what the recurrence
+   * S_t = (alpha_t I - beta_t k_t k_t^T) S_{t-1} + beta_t k_t v_t^T gives (its correction term reads the state before
+   * this token's decay).  With TRI_INV_W_DECAY, row i of W is weighted by exp(g_{i-1}) (1 for the first row of a
+   * chunk); tri_inv_chunk_scan then consumes W and U unchanged.  Other entry points: TRI_INV_ERR_UNSUPPORTED. */
+  TRI_INV_GATE_SHIFTED = 0x800,
   /* Newton-Schulz iteration count, 1..15, in bits 12..15 (0 = default) */
 #define TRI_INV_NS_ITERS(m) (((m) & 0xf) << 12)
   /* flag: run the plain fp32 CUDA-core kernel even where a tensor-core kernel
@@ -168,6 +175,30 @@ int tri_inv_fused(const void* K, const void* V, const float* beta, const float* 
  */
 int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A,
                       const tri_inv_desc* desc, int method, void* cuda_stream);
+
+/*
+ * Per-channel decay through the WY step (KDA row of Table 1, with the decay-weighted factor the layer's chunk form needs):
+ *     A = (I + N)^{-1},  N as for tri_inv_build_kda;     W = A diag(beta) (K * Gamma),  Gamma = exp(G);     U = A diag(beta) V
+ * (the recurrence S_t = (I - beta_t k_t k_t^T) diag(alpha_t) S_{t-1} + beta_t k_t v_t^T re-bracketed per chunk gives
+ * (I + N) U~ = diag(beta) V - diag(beta) (K * Gamma) S, i.e. U~ = U - W S; tri_inv_chunk_scan_kda consumes W and U).
+ *   K, V, W, U [B,T,H,d] kv_dtype;  G [B,T,H,d_k] fp32;  beta [B,T,H] fp32;  A [B,T,H,C] fp32 -- all required (A is also the
+ *   hand-over between the launches).  W may not alias K.
+ * bf16 with d_k = d_v = 128, C = 64 and the block recursion runs on the tensor cores as three launches on the stream
+ * (tri_inv_build_kda's kernel; K * Gamma written into the W buffer; tri_inv_wy's kernel on it); everything else is one launch
+ * of the CUDA-core kernel.  TRI_INV_GATE_SHIFTED and TRI_INV_W_DECAY do not apply (W is always the decay-weighted one).
+ */
+int tri_inv_fused_kda(const void* K, const void* V, const float* G, const float* beta,
+                      float* A, void* W, void* U, const tri_inv_desc* desc, int method, void* cuda_stream);
+
+/*
+ * The chunk scan with one decay per key feature (KDA row): as tri_inv_chunk_scan with g replaced by G [B,T,H,d_k] fp32,
+ *     U~ = U - W S,     P_ij = sum_c Q_ic K_jc exp(G_ic - G_jc)  (j <= i),
+ *     O  = scale * ((Q * Gamma) S + P U~),     S <- diag(Gamma_last) S + (K * exp(G_last - G))^T U~,
+ * W and U from tri_inv_fused_kda.  Runs on the CUDA cores in fp32 for every shape (d_k <= 256); the exponent is taken of
+ * each difference, so G is not restricted.
+ */
+int tri_inv_chunk_scan_kda(const void* Q, const void* K, const void* W, const void* U, const float* G, const float* S0,
+                           void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream);
 
 /*
  * Chunk scan: the consumer of W and U -- the chunk form of the layer's recurrence (the re-formulation Sec. 1

@@ -27,6 +27,7 @@ BLOCK_RECURSIVE, PRODUCT_SERIES, NEWTON_SCHULZ = 0, 1, 2
 LEAF_SERIES = 0x100
 REFINE = 0x200
 OPERANDS_F16 = 0x400
+GATE_SHIFTED = 0x800
 
 
 def ns_iters(m: int) -> int:
@@ -37,7 +38,7 @@ def ns_iters(m: int) -> int:
 FORCE_SIMT = 0x10000
 W_DECAY = 0x20000
 
-EXPORTS = ("tri_inv_build", "tri_inv_build_kda", "tri_inv_chunk_scan", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
+EXPORTS = ("tri_inv_build", "tri_inv_build_kda", "tri_inv_fused_kda", "tri_inv_chunk_scan_kda", "tri_inv_chunk_scan", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
            "tri_inv_selftest_wait_timeout", "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
 
 
@@ -73,6 +74,11 @@ def load():
         lib.tri_inv_build_kda.restype = i32
         lib.tri_inv_chunk_scan.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, dp, vp]
         lib.tri_inv_chunk_scan.restype = i32
+        if hasattr(lib, "tri_inv_fused_kda"):
+            lib.tri_inv_chunk_scan_kda.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, dp, vp]
+            lib.tri_inv_chunk_scan_kda.restype = i32
+            lib.tri_inv_fused_kda.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
+            lib.tri_inv_fused_kda.restype = i32
         lib.tri_inv_fused_raw.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_fused_raw.restype = i32
         lib.tri_inv_fused_packed_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
@@ -181,6 +187,35 @@ def chunk_scan(Q, K, W, U, g, C, scale=1.0, S0=None, cu_seqlens=None, out=None, 
                                    ctypes.byref(desc), _stream(stream))
     if rc != OK:
         raise TriInvError("tri_inv_chunk_scan", rc)
+    return O, S
+
+
+def fused_kda(K, V, G, beta, C, method=BLOCK_RECURSIVE, cu_seqlens=None, out=None, stream=None):
+    """Per-channel decay through the WY step -> (A, W, U) with W = A diag(beta) (K * exp G), U = A diag(beta) V."""
+    B, T, H, d_k = K.shape
+    d_v = V.shape[-1]
+    desc, keep = make_desc(B, T, H, d_k, d_v, C, _dtype_code(K), cu_seqlens)
+    if out is None:
+        out = (torch.zeros((B, T, H, C), dtype=torch.float32, device=K.device), torch.zeros_like(K), torch.zeros_like(V))
+    A, W, U = out
+    rc = load().tri_inv_fused_kda(_p(K), _p(V), _p(G), _p(beta), _p(A), _p(W), _p(U), ctypes.byref(desc), int(method), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_fused_kda", rc)
+    return A, W, U
+
+
+def chunk_scan_kda(Q, K, W, U, G, C, scale=1.0, S0=None, cu_seqlens=None, out=None, want_state=True, stream=None):
+    """tri_inv_chunk_scan_kda: the chunk scan with one decay per key feature -> (O, S_final or None)."""
+    B, T, H, d_k = K.shape
+    d_v = U.shape[3]
+    desc, keep = make_desc(B, T, H, d_k, d_v, C, _dtype_code(K), cu_seqlens)
+    n_seqs = B if cu_seqlens is None else len(cu_seqlens) - 1
+    O = torch.empty((B, T, H, d_v), dtype=U.dtype, device=K.device) if out is None else out
+    S = torch.empty((n_seqs, H, d_k, d_v), dtype=torch.float32, device=K.device) if want_state else None
+    rc = load().tri_inv_chunk_scan_kda(_p(Q), _p(K), _p(W), _p(U), _p(G), _p(S0), _p(O), _p(S), float(scale),
+                                       ctypes.byref(desc), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_chunk_scan_kda", rc)
     return O, S
 
 

@@ -80,8 +80,12 @@ int check_desc(const tri_inv_desc* d, bool need_dv) {
   return TRI_INV_OK;
 }
 
-int check_method(int method, bool w_decay_ok = false) {
+int check_method(int method, bool w_decay_ok = false, bool shift_ok = true) {
   int m = method & TRI_INV_METHOD_MASK;
+  if (method & TRI_INV_GATE_SHIFTED) {
+    if (!shift_ok) return TRI_INV_ERR_UNSUPPORTED;
+    method &= ~TRI_INV_GATE_SHIFTED;
+  }
   if (method & TRI_INV_W_DECAY) {
     if (!w_decay_ok) return TRI_INV_ERR_UNSUPPORTED;
     method &= ~TRI_INV_W_DECAY;
@@ -224,27 +228,32 @@ int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A
   if (rc) return rc;
   if (!K || !G || !beta || !A) return TRI_INV_ERR_INVALID_ARG;
   if (!aligned16(K) || !aligned16(G) || !aligned16(beta) || !aligned16(A)) return TRI_INV_ERR_INVALID_ARG;
-  if ((rc = check_method(method))) return rc;
+  if ((rc = check_method(method, false, false))) return rc;
   KParams p{};
-  p.K = K; p.V = G; p.beta = beta; p.g = nullptr; p.A = A;
+  p.K = K; p.G = G; p.beta = beta; p.g = nullptr; p.A = A;
   p.method = method;
   p.ops = kStoreA | kKda;
   return run(p, desc, cuda_stream);
 }
 
-int tri_inv_chunk_scan(const void* Q, const void* K, const void* W, const void* U, const float* g, const float* S0,
-                       void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+// Shared body of the two chunk-scan entry points: exactly one of g (scalar gate) and G (per-channel gate) is given.
+int chunk_scan_any(const void* Q, const void* K, const void* W, const void* U, const float* g, const float* G, const float* S0,
+                   void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream) {
   int rc = check_desc(desc, true);
   if (rc) return rc;
-  if (!Q || !K || !W || !U || !g || !O) return TRI_INV_ERR_INVALID_ARG;
-  if (!aligned16(Q) || !aligned16(K) || !aligned16(W) || !aligned16(U) || !aligned16(g) || !aligned16(O) || !aligned16(S0) ||
-      !aligned16(S_out))
+  if (!Q || !K || !W || !U || (!g && !G) || !O) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(W) || !aligned16(U) || !aligned16(g) || !aligned16(G) || !aligned16(O) ||
+      !aligned16(S0) || !aligned16(S_out))
     return TRI_INV_ERR_INVALID_ARG;
-  const bool tc = desc->kv_dtype == TRI_INV_BF16 && desc->d_k == 128 && desc->d_v == 128 && desc->C == 64;
+  // the per-channel gate exists on the CUDA-core kernel only
+  const bool tc = !G && desc->kv_dtype == TRI_INV_BF16 && desc->d_k == 128 && desc->d_v == 128 && desc->C == 64;
   if (!tc && desc->d_k > 256) return TRI_INV_ERR_UNSUPPORTED;   // the CUDA-core kernel keeps a d_k x 32 slice of S in shared memory
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   ScanParams p{};
-  p.U = U; p.g = g; p.S0 = S0; p.O = O; p.S_out = S_out; p.scale = scale;
+  p.U = U; p.g = g; p.G = G; p.S0 = S0; p.O = O; p.S_out = S_out; p.scale = scale;
   p.H = desc->H; p.T = desc->T;
   p.n_seqs = desc->cu_seqlens ? desc->n_seqs : desc->B;
   cudaError_t err;
@@ -267,6 +276,49 @@ int tri_inv_chunk_scan(const void* Q, const void* K, const void* W, const void* 
   if (err == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);
   if (dev_off) cudaFreeAsync(dev_off, stream);
   return err == cudaSuccess ? TRI_INV_OK : TRI_INV_ERR_CUDA;
+}
+}  // namespace
+
+extern "C" {
+
+int tri_inv_chunk_scan(const void* Q, const void* K, const void* W, const void* U, const float* g, const float* S0,
+                       void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream) {
+  if (!g) return TRI_INV_ERR_INVALID_ARG;
+  return chunk_scan_any(Q, K, W, U, g, nullptr, S0, O, S_out, scale, desc, cuda_stream);
+}
+
+int tri_inv_chunk_scan_kda(const void* Q, const void* K, const void* W, const void* U, const float* G, const float* S0,
+                           void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream) {
+  if (!G) return TRI_INV_ERR_INVALID_ARG;
+  return chunk_scan_any(Q, K, W, U, nullptr, G, S0, O, S_out, scale, desc, cuda_stream);
+}
+
+int tri_inv_fused_kda(const void* K, const void* V, const float* G, const float* beta,
+                      float* A, void* W, void* U, const tri_inv_desc* desc, int method, void* cuda_stream) {
+  int rc = check_desc(desc, true);
+  if (rc) return rc;
+  if (!K || !V || !G || !beta || !A || !W || !U) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(G) || !aligned16(beta) || !aligned16(A) || !aligned16(W) || !aligned16(U))
+    return TRI_INV_ERR_INVALID_ARG;
+  if ((rc = check_method(method, false, false))) return rc;
+  const bool tc = !(method & (TRI_INV_FORCE_SIMT | TRI_INV_REFINE)) && (method & TRI_INV_METHOD_MASK) == TRI_INV_BLOCK_RECURSIVE &&
+                  desc->kv_dtype == TRI_INV_BF16 && desc->d_k == 128 && desc->d_v == 128 && desc->C == 64;
+  if (tc) {
+    // Tensor-core route, three launches on the stream: A by the per-channel build kernel; K' = K * exp(G) into the W
+    // buffer; W = A diag(beta) K' and U = A diag(beta) V by the WY kernel, which reads each K' tile whole into shared
+    // memory before it writes the same rows of W.
+    if ((rc = tri_inv_build_kda(K, G, beta, A, desc, method, cuda_stream))) return rc;
+    const long long tokens = desc->cu_seqlens ? (long long)desc->T : (long long)desc->T * desc->B;
+    if (launch_kda_scale_keys(K, G, W, tokens * desc->H * desc->d_k, desc->kv_dtype, (cudaStream_t)cuda_stream) != cudaSuccess)
+      return TRI_INV_ERR_CUDA;
+    count_launch();
+    return tri_inv_wy(A, W, V, beta, W, U, desc, cuda_stream);
+  }
+  KParams p{};
+  p.K = K; p.V = V; p.G = G; p.beta = beta; p.g = nullptr; p.A = A; p.W = W; p.U = U;
+  p.method = method | TRI_INV_FORCE_SIMT;
+  p.ops = kStoreA | kDoWY | kKda;
+  return run(p, desc, cuda_stream);
 }
 
 int tri_inv_selftest_wait_timeout(const void* K, const void* V, const float* beta, const float* g,

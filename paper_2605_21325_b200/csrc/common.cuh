@@ -14,7 +14,7 @@ enum : int {
   kDoWY = 2,    // compute W (and U when V != nullptr)
   kLoadA = 4,   // skip build + inversion, read A from A_in (tri_inv_wy)
   kRaw = 8,     // K is un-normalised, beta and g are logits: normalise, sigmoid, log-sigmoid + chunk cumsum in the kernel
-  kKda = 16,    // per-channel decay: KParams::V holds G [B,T,H,d_k] fp32 (build only)
+  kKda = 16,    // per-channel decay (KParams::G); with kDoWY, W = A diag(beta) (K * exp G)
   kFixedStride = 64,  // tensor-core kernel: take no work-counter pair (and create no event for one); items by a fixed stride
   kTestStall = 128,   // self-test: CTA 0 leaves out the first Gram product so that its bounded wait runs out
   kWDecay = 32, // W = A diag(beta) diag(exp g) K: the decay-weighted factor the chunk-state recurrence consumes
@@ -32,6 +32,7 @@ struct KParams {
   const float* beta;
   const float* g;
   const float* A_in;
+  const float* G;               // per-channel decay (kKda): cumulative log-decay [B,T,H,d_k] fp32
   float* A;
   void* W;
   void* U;
@@ -91,6 +92,7 @@ int* work_counter_for(cudaStream_t stream);
 struct ScanParams {
   const void* U;        // [tokens,H,d_v]
   const float* g;       // [tokens,H]
+  const float* G;       // [tokens,H,d_k] per-channel cumulative log-decay (KDA row) or null; CUDA-core kernel only
   const float* S0;      // [n_seqs,H,d_k,d_v] fp32 or null (zero state)
   void* O;              // [tokens,H,d_v], storage type of U
   float* S_out;         // [n_seqs,H,d_k,d_v] fp32 or null
@@ -107,6 +109,9 @@ cudaError_t launch_chunk_scan_simt(const ScanParams& p, const void* Q, const voi
                                    int kv_dtype, cudaStream_t stream);
 // Per-channel decay variant on the tensor cores (bf16 keys, d_k = 128, C = 64, block recursion).
 cudaError_t launch_kda_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
+
+// out = K * exp(G) element by element in the storage type of K (per-channel fused call; kda_ops.cu).
+cudaError_t launch_kda_scale_keys(const void* K, const float* G, void* out, long long n, int kv_dtype, cudaStream_t stream);
 
 // Fills dev_tab (one entry per chunk of tokens, in sequence order) from the host offsets in d->cu_seqlens
 // with small kernels on the stream; no copy and no synchronisation.

@@ -243,7 +243,7 @@ cudaError_t launch_kda_tc(const KParams& p, int Cc, cudaStream_t stream, bool* h
   long long tokens = p.chunk_tab ? (long long)p.T : (long long)p.T * (p.n_chunks / p.chunks_per_seq);
   CUtensorMap tmK, tmG;
   if (!make_tmap(&tmK, p.K, tokens, p.H, D, C, 2)) return cudaErrorUnknown;
-  if (!make_tmap(&tmG, p.V, tokens, p.H, D, C, 4)) return cudaErrorUnknown;
+  if (!make_tmap(&tmG, p.G, tokens, p.H, D, C, 4)) return cudaErrorUnknown;
   long long total = (long long)p.n_chunks * p.H, cap = (long long)n_sm * ctas;
   int grid = (int)(total < cap ? total : cap);
   kda_build_kernel<<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);

@@ -108,11 +108,12 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
   float* sg = sb + C;
   float* sr = sg + C;  // raw front end: 1 / |k_i|
   const bool raw = (p.ops & kRaw) != 0;
-  const bool kda = (p.ops & kKda) != 0;  // per-channel decay: G in p.V, each Gram term weighted by exp(G_ic - G_jc)
+  const bool kda = (p.ops & kKda) != 0;  // per-channel decay: each Gram term weighted by exp(G_ic - G_jc); W rows weighted by exp(G_j) per feature
   const int tid = threadIdx.x;
   const int total = p.n_chunks * p.H;
   constexpr int kAcc = (C * C + kThreads - 1) / kThreads;
   const int method = p.method & TRI_INV_METHOD_MASK;
+  const int gshift = (p.method & TRI_INV_GATE_SHIFTED) ? 1 : 0;  // Comba row: row i decays from the token before it
 
   for (int item = blockIdx.x; item < total; item += gridDim.x) {
     int tok0, rows, h;
@@ -165,7 +166,7 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
           Ks[i * kSliceLd + kk] = v;
           if (kda) {  // the scratch matrix is free during the Gram phase: it holds the slice of G
             float gv = 0.f;
-            if (i < rows && ks + kk < p.d_k) gv = ((const float*)p.V)[((size_t)(tok0 + i) * p.H + h) * p.d_k + ks + kk];
+            if (i < rows && ks + kk < p.d_k) gv = p.G[((size_t)(tok0 + i) * p.H + h) * p.d_k + ks + kk];
             Zm[i * kSliceLd + kk] = gv;
           }
         }
@@ -205,7 +206,7 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
       for (int m = 0; m < kAcc; ++m) {
         int e = tid + m * kThreads;
         int i = e / C, j = e - i * C;
-        if (e < C * C && j < i && i < rows) Nm[i * LD + j] = sb[i] * (acc[m] * sr[i] * sr[j]) * expf(sg[i] - sg[j]);
+        if (e < C * C && j < i && i < rows) Nm[i * LD + j] = sb[i] * (acc[m] * sr[i] * sr[j]) * expf(sg[i - gshift] - sg[j]);  // i > j >= 0, so i - 1 is in the chunk
       }
       __syncthreads();
 
@@ -365,7 +366,11 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
           for (int e = tid; e < C * kSlice; e += kThreads) {
             int j = e / kSlice, cc = e - j * kSlice;
             float v = 0.f;
-            if (j < rows && c0 + cc < d) v = sb[j] * (which ? 1.f : sr[j] * ((p.ops & kWDecay) ? expf(sg[j]) : 1.f)) * load_kv(src, p.kv_dtype, ((size_t)(tok0 + j) * p.H + h) * d + c0 + cc);
+            if (j < rows && c0 + cc < d) {
+              const size_t idx = ((size_t)(tok0 + j) * p.H + h) * d + c0 + cc;
+              v = sb[j] * (which ? 1.f : sr[j] * ((p.ops & kWDecay) ? ((gshift && j == 0) ? 1.f : expf(sg[j - gshift])) : 1.f)) * load_kv(src, p.kv_dtype, idx);
+              if (kda && !which) v *= expf(p.G[idx]);   // W = A diag(beta) (K * Gamma): the decay-weighted factor of the per-channel form
+            }
             Ks[j * kSliceLd + cc] = v;
           }
           __syncthreads();

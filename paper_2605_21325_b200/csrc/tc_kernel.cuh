@@ -141,6 +141,9 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
   constexpr bool raw = RAW;
   const bool front = RAW && (p.ops & kRaw) != 0;
   const bool wdecay = RAW && (p.ops & kWDecay) != 0;
+  // Comba row of Table 1 (decay matrix A^{i-1/j}): row i of N, and row i of the decay-weighted W, take the cumulative
+  // log-decay of the token before it (the first row of a chunk has nothing below the diagonal and weight 1)
+  const int gshift = (p.method & TRI_INV_GATE_SHIFTED) ? 1 : 0;
   const int total = p.n_chunks * p.H;
 
   // Thread 0 requests the tiles of an item; K and V complete on separate barriers so that the Gram
@@ -317,7 +320,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         const int bx = e / (C * 8), rem = e - bx * (C * 8), r = rem >> 3, c = rem & 7;
         uint4* ptr = reinterpret_cast<uint4*>(smem + cfg::OFF_K + bx * cfg::BOX_BYTES + r * 128 + c * 16);
         uint4 v = *ptr;
-        const float sc = wdecay ? sR[r] * ex2_approx(sG[r]) : sR[r];
+        const float sc = wdecay ? sR[r] * ((gshift && r == 0) ? 1.f : ex2_approx(sG[r - gshift])) : sR[r];
         uint32_t* w = reinterpret_cast<uint32_t*>(&v);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -405,7 +408,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
           stmatrix_x4(addr, pack_f16(lo[0], lo[1]), pack_f16(lo[2], lo[3]), pack_f16(hi[0], hi[1]), pack_f16(hi[2], hi[3]));
         };
         {
-          const float beta_a = sBeta[ra], beta_b = sBeta[rbw], g_a = sG[ra], g_b = sG[rbw];
+          const float beta_a = sBeta[ra], beta_b = sBeta[rbw], g_a = sG[ra - (gshift && ra > 0)], g_b = sG[rbw - gshift];
           float sacc[C / 8][4];
           if constexpr (C == 64) tmem_ld_16x64(sacc, tmem_rows); else tmem_ld_16x128(sacc, tmem_rows);
           tmem_wait_ld();
@@ -549,7 +552,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
           return (uint32_t)((c >> 5) * (C * 128) + r * 128 + (((((c & 31) >> 2) ^ (r & 7)) << 4) | ((c & 3) * 4)));
         };
         const int ra = 16 * rb + g, rbw = ra + 8;
-        const float beta_a = sBeta[ra], beta_b = sBeta[rbw], g_a = sG[ra], g_b = sG[rbw];
+        const float beta_a = sBeta[ra], beta_b = sBeta[rbw], g_a = sG[ra - (gshift && ra > 0)], g_b = sG[rbw - gshift];
         float xr[C / 8][4];  // this warp's 16 rows of X, accumulator-fragment layout, kept across rounds
         // rows ra, rbw of Y (pairs of columns) and the same values into Y^T (column ra / rbw of rows c, c+1)
         auto put_y = [&](int c, float2 ya, float2 yw) {
@@ -679,7 +682,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       } else {
       // ---- 3. gate + mask on this warp's rows, N -> shared memory
       const int ra = 16 * rb + g, rbw = ra + 8;
-      const float beta_a = sBeta[ra], beta_b = sBeta[rbw], g_a = sG[ra], g_b = sG[rbw];
+      const float beta_a = sBeta[ra], beta_b = sBeta[rbw], g_a = sG[ra - (gshift && ra > 0)], g_b = sG[rbw - gshift];
       {
         float sacc[C / 8][4];   // this warp's 16 rows of S, all C columns, in one tensor-memory load
         if constexpr (C == 64) tmem_ld_16x64(sacc, tmem_rows); else tmem_ld_16x128(sacc, tmem_rows);

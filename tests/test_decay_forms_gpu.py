@@ -1,0 +1,125 @@
+"""GPU parity for the other decay forms of Table 1: the Comba row (decay matrix from j to i-1, TRI_INV_GATE_SHIFTED) and the
+KDA row through the whole layer (per-channel decay: tri_inv_fused_kda, tri_inv_chunk_scan_kda), against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_21325_b200 import workloads as wl
+from parity_util import max_ratio, max_residual, structure_errors
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bnd():
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2605_21325_b200 import binding
+    torch.cuda.set_device(0)
+    return binding
+
+
+def cases(C, dtype, d):
+    rng = np.random.default_rng(500 + C + d)
+    cu = wl.ragged_lengths(5, 4 * C, rng)
+    return [wl.make("dense", 2, 5 * C, 3, d, d, C, dtype, seed=1200 + C + d),
+            wl.make("packed", 1, int(cu[-1]), 2, d, d, C, dtype, seed=1300 + C + d, cu_seqlens=cu, rng=rng)]
+
+
+@pytest.mark.parametrize("C,dtype,d", [(64, wl.BF16, 128), (128, wl.BF16, 128), (64, wl.F32, 64), (32, wl.BF16, 64)])
+def test_shifted_gate_build_and_wy(bnd, C, dtype, d):
+    """N_ij = beta_i (k_i . k_j) exp(g_{i-1} - g_j): A for every scheme, and the decay-weighted W (row i weighted by
+    exp(g_{i-1})) and U, on the tensor-core kernel (bf16, d = 128) and the CUDA-core kernel (other shapes, fp32)."""
+    tol_a, tol_r, tol_w = (2e-3, 5e-3, 1e-2) if dtype == wl.BF16 else (1e-5, 5e-5, 1e-5)
+    for inp in cases(C, dtype, d):
+        cu = inp.cu_seqlens
+        A_ref, N_ref = oracle.build_A_shifted(inp.K, inp.beta, inp.g, C, cu_seqlens=cu, return_N=True)
+        gs = oracle.shifted_gate(inp.g, C, cu_seqlens=cu)
+        Kd = inp.kv_as_f32("K").astype(np.float64)
+        W_ref, _ = oracle.wy(A_ref, Kd * np.exp(gs)[..., None], None, inp.beta, C, cu_seqlens=cu)
+        _, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, C, cu_seqlens=cu)
+        dev = bnd.to_device(inp)
+        for m in (bnd.BLOCK_RECURSIVE, bnd.BLOCK_RECURSIVE | bnd.LEAF_SERIES, bnd.PRODUCT_SERIES):
+            A, W, U = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], C, method=m | bnd.GATE_SHIFTED | bnd.W_DECAY, cu_seqlens=cu)
+            torch.cuda.synchronize()
+            assert bnd.last_device_status() == 0
+            a = A.cpu().numpy()
+            assert structure_errors(a, inp) == (0, 0)
+            assert max_ratio(a, A_ref) <= tol_a and max_residual(a, N_ref, inp) <= tol_r
+            assert max_ratio(bnd.to_numpy_f64(W), W_ref) <= tol_w and max_ratio(bnd.to_numpy_f64(U), U_ref) <= tol_w
+        A = bnd.build(dev["K"], dev["beta"], dev["g"], C, method=bnd.GATE_SHIFTED, cu_seqlens=cu)
+        torch.cuda.synchronize()
+        assert max_ratio(A.cpu().numpy(), A_ref) <= tol_a
+        # the flag matters: without it the matrix differs visibly
+        A0 = bnd.build(dev["K"], dev["beta"], dev["g"], C, cu_seqlens=cu)
+        torch.cuda.synchronize()
+        assert max_ratio(A0.cpu().numpy(), A_ref) > 10 * tol_a
+
+
+def test_comba_layer_two_launches_against_its_recurrence(bnd):
+    """Fused call with the shifted gate and the decay-weighted W, then the unchanged chunk scan, against
+    S_t = (alpha_t I - beta_t k_t k_t^T) S_{t-1} + beta_t k_t v_t^T token by token."""
+    for inp in cases(64, wl.BF16, 128):
+        cu = inp.cu_seqlens
+        Q = wl.queries(inp, seed=77)
+        S0 = wl.initial_state(inp, seed=78)
+        dev = bnd.to_device(inp)
+        _, W, U = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], 64, method=bnd.GATE_SHIFTED | bnd.W_DECAY, cu_seqlens=cu, want_A=False)
+        O, S = bnd.chunk_scan(bnd.kv_to_torch(Q), dev["K"], W, U, dev["g"], 64, scale=0.5, S0=torch.from_numpy(S0).cuda(), cu_seqlens=cu)
+        torch.cuda.synchronize()
+        assert bnd.last_device_status() == 0
+        O_ref, S_ref = oracle.recurrence_ex(Q, inp.K, inp.V, inp.beta, inp.g, 64, read_before_decay=True, scale=0.5, S0=S0, cu_seqlens=cu)
+        assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= 2e-2 and max_ratio(bnd.to_numpy_f64(S), S_ref) <= 2e-2
+
+
+@pytest.mark.parametrize("C,dtype,d", [(64, wl.BF16, 128), (64, wl.F32, 64), (32, wl.BF16, 64), (128, wl.BF16, 128)])
+def test_per_channel_decay_through_wy_and_scan(bnd, C, dtype, d):
+    """tri_inv_fused_kda (tensor-core route at bf16 / d = 128 / C = 64, CUDA cores elsewhere) against the oracle's A, W, U;
+    then tri_inv_chunk_scan_kda on them against the token-by-token recurrence with one decay per key feature."""
+    tol_a, tol_r, tol_w, tol_o = (2e-3, 5e-3, 1e-2, 2e-2) if dtype == wl.BF16 else (1e-5, 5e-5, 1e-5, 1e-4)
+    for inp in cases(C, dtype, d):
+        cu = inp.cu_seqlens
+        G = wl.per_channel_gate(inp, seed=61)
+        A_ref, N_ref = oracle.build_A_kda(inp.K, G, inp.beta, C, cu_seqlens=cu, return_N=True)
+        Kd = inp.kv_as_f32("K").astype(np.float64)
+        W_ref, _ = oracle.wy(A_ref, Kd * np.exp(G.astype(np.float64)), None, inp.beta, C, cu_seqlens=cu)
+        _, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, C, cu_seqlens=cu)
+        dev = bnd.to_device(inp)
+        Gd = torch.from_numpy(G).cuda()
+        nan = lambda t: torch.full_like(t, float("nan"))
+        out = (torch.full((inp.B, inp.T, inp.H, C), float("nan"), dtype=torch.float32, device="cuda"), nan(dev["K"]), nan(dev["V"]))
+        A, W, U = bnd.fused_kda(dev["K"], dev["V"], Gd, dev["beta"], C, cu_seqlens=cu, out=out)
+        torch.cuda.synchronize()
+        assert bnd.last_device_status() == 0
+        a = A.cpu().numpy()
+        assert not np.isnan(a).any() and structure_errors(a, inp) == (0, 0)
+        assert max_ratio(a, A_ref) <= tol_a and max_residual(a, N_ref, inp) <= tol_r
+        w, u = bnd.to_numpy_f64(W), bnd.to_numpy_f64(U)
+        assert not np.isnan(w).any() and not np.isnan(u).any()
+        assert max_ratio(w, W_ref) <= tol_w and max_ratio(u, U_ref) <= tol_w
+        Q = wl.queries(inp, seed=62)
+        S0 = wl.initial_state(inp, seed=63)
+        O, S = bnd.chunk_scan_kda(bnd.kv_to_torch(Q), dev["K"], W, U, Gd, C, scale=0.5, S0=torch.from_numpy(S0).cuda(), cu_seqlens=cu)
+        torch.cuda.synchronize()
+        assert bnd.last_device_status() == 0
+        O_ref, S_ref = oracle.recurrence_ex(Q, inp.K, inp.V, inp.beta, None, C, G=G, scale=0.5, S0=S0, cu_seqlens=cu)
+        assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= tol_o and max_ratio(bnd.to_numpy_f64(S), S_ref) <= tol_o
+        # the scan alone, fed the oracle's own W and U (rounded to the storage type), against its definition
+        if dtype == wl.F32:
+            Wt, Ut = torch.from_numpy(W_ref.astype(np.float32)).cuda(), torch.from_numpy(U_ref.astype(np.float32)).cuda()
+            O2, S2 = bnd.chunk_scan_kda(bnd.kv_to_torch(Q), dev["K"], Wt, Ut, Gd, C, scale=0.5, S0=torch.from_numpy(S0).cuda(), cu_seqlens=cu)
+            O3, S3 = oracle.chunk_scan_kda(Q, inp.K, W_ref.astype(np.float32), U_ref.astype(np.float32), G, C, scale=0.5, S0=S0, cu_seqlens=cu)
+            torch.cuda.synchronize()
+            assert max_ratio(bnd.to_numpy_f64(O2), O3) <= 1e-5 and max_ratio(bnd.to_numpy_f64(S2), S3) <= 1e-5
+
+
+def test_flags_the_per_channel_calls_refuse(bnd):
+    import ctypes
+    d = torch.zeros(64, device="cuda")
+    desc, _ = bnd.make_desc(1, 64, 1, 128, 128, 64, bnd.BF16)
+    L = bnd.load()
+    p = bnd._p(d)
+    assert L.tri_inv_build_kda(p, p, p, p, ctypes.byref(desc), bnd.GATE_SHIFTED, None) == bnd.ERR_UNSUPPORTED
+    assert L.tri_inv_fused_kda(p, p, p, p, p, p, p, ctypes.byref(desc), bnd.W_DECAY, None) == bnd.ERR_UNSUPPORTED
+    assert L.tri_inv_fused_kda(p, p, p, p, None, p, p, ctypes.byref(desc), 0, None) == bnd.ERR_INVALID_ARG

@@ -172,27 +172,26 @@ def test_adversarial_keys_report(bnd):
 
 
 def test_per_channel_decay_full_size_config2_shape(bnd):
-    """tri_inv_build_kda on the shape of config 2 (4096 matrices, the launch bench.py --call kda times): structure on
-    every element, values on sampled chunks against the fp64 oracle, and -- at any size -- a gate that is the same
-    on every channel must reproduce tri_inv_build's matrices within the rounding of the two bf16 operand copies."""
+    """tri_inv_fused_kda on the shape of config 2 (4096 matrices, the launches bench.py --call kda_fused times): structure on
+    every element, EVERY matrix's A, W and U against the fp64 oracle, and -- at any size -- a gate that is the same on every
+    channel must reproduce tri_inv_build's matrices within the rounding of the two bf16 operand copies."""
     inp = wl.config(2)
     G = wl.per_channel_gate(inp, seed=3002)
     dev = bnd.to_device(inp)
     Gd = torch.from_numpy(G).cuda()
     A = torch.full((inp.B, inp.T, inp.H, inp.C), float("nan"), dtype=torch.float32, device="cuda")
-    bnd.build_kda(dev["K"], Gd, dev["beta"], inp.C, out=A)
+    W, U = torch.full_like(dev["K"], float("nan")), torch.full_like(dev["V"], float("nan"))
+    bnd.fused_kda(dev["K"], dev["V"], Gd, dev["beta"], inp.C, out=(A, W, U))
     torch.cuda.synchronize()
     assert bnd.last_device_status() == 0
     device_structure_check(A, inp)
-    worst_a = worst_r = 0.0
-    for t0, t1 in sample_ranges(inp):
-        A_ref, N_ref = oracle.build_A_kda(inp.K[:, t0:t1], G[:, t0:t1], inp.beta[:, t0:t1], inp.C, return_N=True)
-        a = A[:, t0:t1].cpu().numpy()
-        worst_a = max(worst_a, max_ratio(a, A_ref))
-        sub = wl.Inputs("s", inp.B, t1 - t0, inp.H, inp.d_k, inp.d_v, inp.C, inp.kv_dtype, inp.K[:, t0:t1], inp.V[:, t0:t1],
-                        inp.beta[:, t0:t1], inp.g[:, t0:t1], None, {})
-        worst_r = max(worst_r, max_residual(a, N_ref, sub))
-    assert worst_a <= TOL_A[wl.BF16] and worst_r <= TOL_RES[wl.BF16], (worst_a, worst_r)
+    A_ref, N_ref = oracle.build_A_kda(inp.K, G, inp.beta, inp.C, return_N=True)
+    a = A.cpu().numpy()
+    assert max_ratio(a, A_ref) <= TOL_A[wl.BF16] and max_residual(a, N_ref, inp) <= TOL_RES[wl.BF16]
+    Kg = wl.bf16_bits_to_f32(inp.K).astype(np.float64) * np.exp(G.astype(np.float64))
+    W_ref, _ = oracle.wy(A_ref, Kg, None, inp.beta, inp.C)
+    _, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, inp.C)
+    assert max_ratio(bnd.to_numpy_f64(W), W_ref) <= 1e-2 and max_ratio(bnd.to_numpy_f64(U), U_ref) <= 1e-2
     Gc = dev["g"].unsqueeze(-1).expand(-1, -1, -1, inp.d_k).contiguous()
     A_same = bnd.build_kda(dev["K"], Gc, dev["beta"], inp.C)
     A_scalar = bnd.build(dev["K"], dev["beta"], dev["g"], inp.C)
