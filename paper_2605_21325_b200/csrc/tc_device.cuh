@@ -74,6 +74,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
 __device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* tm, int x, int y) {
   asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(x), "r"(y) : "memory");
 }
+// Tile from shared memory to global memory through the copy engine (bulk async-group completion).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// every bulk store this thread has committed has finished READING its shared-memory source
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tm) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
@@ -492,11 +499,18 @@ __device__ __forceinline__ void stmatrix_x4(uint32_t addr, uint32_t m0, uint32_t
 }
 
 // Epilogue of one 16-row x 64-column piece of W or U: accumulator fragments from tensor memory ->
-// bf16 -> stmatrix into a per-warp, swizzled 2 KiB staging tile -> 16-byte loads -> coalesced
-// 16-byte global stores (8 lanes cover one 128-byte row segment).
+// bf16 -> stmatrix into a per-warp, swizzled 2 KiB staging tile.  A piece with all 16 rows inside its sequence
+// then leaves through the copy engine (one tiled bulk store: tm is a 2-D map of the output with boxes of 64
+// columns x 16 rows in the same 128-byte swizzle, x / y the piece's first column and token), which costs
+// the warp no load/store instructions; lane 0 owns the stores, and waits for the previous one to have read the
+// staging tile before it is rewritten.  The caller waits again (bulk_wait_read, lane 0) before the staging
+// space is used for anything else.  A piece cut short by its sequence's end takes 16-byte loads and
+// coalesced 16-byte global stores of its real rows only (8 lanes cover one 128-byte row segment).
 __device__ __forceinline__ void store_frag_piece_bf16(const float (&f)[8][4], uint32_t stage, int lane, __nv_bfloat16* out_row0,
-                                                      size_t row_stride, int rows_left) {
+                                                      size_t row_stride, int rows_left, const CUtensorMap* tm, int x, int y) {
   const int mi = lane >> 3, r = (lane & 7) + 8 * (mi & 1);
+  if (lane == 0) bulk_wait_read();
+  __syncwarp();
 #pragma unroll
   for (int nt = 0; nt < 8; nt += 2) {
     const uint32_t m0 = pack_bf16(f[nt][0], f[nt][1]), m1 = pack_bf16(f[nt][2], f[nt][3]);
@@ -504,6 +518,15 @@ __device__ __forceinline__ void store_frag_piece_bf16(const float (&f)[8][4], ui
     const int chunk = nt + (mi >> 1);
     const uint32_t addr = stage + r * 128 + ((chunk ^ (r & 7)) << 4);
     asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
+  }
+  if (rows_left >= 16) {
+    fence_proxy_async();   // this lane's staging writes become visible to the copy engine
+    __syncwarp();
+    if (lane == 0) {
+      tma_store_2d(tm, stage, x, y);
+      bulk_commit();
+    }
+    return;
   }
   __syncwarp();
 #pragma unroll
@@ -516,11 +539,11 @@ __device__ __forceinline__ void store_frag_piece_bf16(const float (&f)[8][4], ui
   __syncwarp();
 }
 __device__ __forceinline__ void store_piece_bf16(uint32_t taddr, uint32_t stage, int lane, __nv_bfloat16* out_row0,
-                                                 size_t row_stride, int rows_left) {
+                                                 size_t row_stride, int rows_left, const CUtensorMap* tm, int x, int y) {
   float f[8][4];
   tmem_ld_16x64(f, taddr);
   tmem_wait_ld();
-  store_frag_piece_bf16(f, stage, lane, out_row0, row_stride, rows_left);
+  store_frag_piece_bf16(f, stage, lane, out_row0, row_stride, rows_left, tm, x, y);
 }
 
 // ------------------------------------------------------------------------------------------ host side
@@ -543,7 +566,7 @@ inline EncodeTiledFn encode_fn() {
 
 // 2-D view of a [tokens, H*d] tensor of bf16 (elt = 2) or fp32 (elt = 4); one box = 128 bytes of features
 // (64 bf16 or 32 fp32, swizzled) x C tokens.
-inline bool make_tmap(CUtensorMap* tm, const void* base, long long tokens, int H, int d, int C, int elt = 2) {
+inline bool make_tmap(CUtensorMap* tm, const void* base, long long tokens, int H, int d, int C, int elt = 2) {   // C = tokens per box
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)H * d, (cuuint64_t)tokens};

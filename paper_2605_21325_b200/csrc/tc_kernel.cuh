@@ -89,7 +89,7 @@ struct Cfg {
 
 // Byte offset of the 16-byte chunk holding features [f, f+8) of row r inside a swizzled tile.
 template <int C, int D, bool SER, bool RAW, bool BO, bool REF, bool H16>
-__global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SER, BO, REF, H16>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SER, BO, REF, H16>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                                                                              const __grid_constant__ CUtensorMap tmV, const __grid_constant__ KParams p) {
   using cfg = Cfg<C, D, SER, BO, REF, H16>;
   static_assert(D == 128, "tiles are two 64-feature boxes wide");
@@ -346,6 +346,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       if (v_now) wait(bar_v, ph_v);
       clear_tail_rows(k_now, v_now);
     }
+    if (lane == 0) bulk_wait_read();   // this warp's last W / U stores have read their staging tile, which lies in the matrix's space
     if (bad) *s_gave_up = 1;
     __syncthreads();
     // The one exit on a wait that gave up: every thread reads the flag behind this barrier (a thread can raise it
@@ -1006,8 +1007,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
           if (wait(bar_v, ph_v)) { tc_fence_after(); issue_wy(sV); }
         }
         if (tid == kTidK && has_next) issue_k(nx_tok0, nx_h);  // K's last reader (the W product) is done
-        store_frag_piece_bf16(f0, stage, lane, w_row0, row_stride, rows - row0);
-        store_frag_piece_bf16(f1, stage, lane, w_row0 + 64, row_stride, rows - row0);
+        store_frag_piece_bf16(f0, stage, lane, w_row0, row_stride, rows - row0, &tmW, h * D + 0, tok0 + row0);
+        store_frag_piece_bf16(f1, stage, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
         PHASE(9);
         wait(bar_mma, ph_mma);
         ph_mma ^= 1;
@@ -1027,16 +1028,16 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
           issue_gram();
           gram_early = true;
         }
-        store_frag_piece_bf16(f0, stage, lane, u_row0, row_stride, rows - row0);
-        store_frag_piece_bf16(f1, stage, lane, u_row0 + 64, row_stride, rows - row0);
+        store_frag_piece_bf16(f0, stage, lane, u_row0, row_stride, rows - row0, &tmU, h * D + 0, tok0 + row0);
+        store_frag_piece_bf16(f1, stage, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
       } else {
         // C = 128 (W and U side by side in 256 columns) or W only
         if (cfg::ALIAS && tid == kTidK && has_next && !load_a) issue_k(nx_tok0, nx_h);  // all MMAs on the tiles are done
-        store_piece_bf16(tmem_rows, stage, lane, w_row0, row_stride, rows - row0);
-        store_piece_bf16(tmem_rows + 64, stage, lane, w_row0 + 64, row_stride, rows - row0);
+        store_piece_bf16(tmem_rows, stage, lane, w_row0, row_stride, rows - row0, &tmW, h * D, tok0 + row0);
+        store_piece_bf16(tmem_rows + 64, stage, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
         if (need_v) {
-          store_piece_bf16(tmem_rows + 128, stage, lane, u_row0, row_stride, rows - row0);
-          store_piece_bf16(tmem_rows + 192, stage, lane, u_row0 + 64, row_stride, rows - row0);
+          store_piece_bf16(tmem_rows + 128, stage, lane, u_row0, row_stride, rows - row0, &tmU, h * D, tok0 + row0);
+          store_piece_bf16(tmem_rows + 192, stage, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
         }
         tc_fence_before();
         __syncthreads();
@@ -1072,6 +1073,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
     p.work_counter[1] = 0;
     __threadfence();
   }
+  if (lane == 0) bulk_wait_read();
   if (bad) *s_gave_up = 1;
   if (bad || misaligned) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
   __syncthreads();  // every thread has left the item loop
@@ -1131,11 +1133,15 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   if (!make_tmap(&tmK, p.K, tokens, p.H, D, C)) return cudaErrorUnknown;
   if (p.V) { if (!make_tmap(&tmV, p.V, tokens, p.H, D, C)) return cudaErrorUnknown; }
   else tmV = tmK;
+  // W and U leave in boxes of 64 columns x 16 tokens (one warp's piece)
+  CUtensorMap tmW = tmK, tmU = tmK;
+  if (p.W && !make_tmap(&tmW, p.W, tokens, p.H, D, 16)) return cudaErrorUnknown;
+  if (p.U && !make_tmap(&tmU, p.U, tokens, p.H, D, 16)) return cudaErrorUnknown;
   long long total = (long long)p.n_chunks * p.H;
   long long cap = (long long)n_sm * ctas_per_sm;
   int grid = (int)(total < cap ? total : cap);
   p.work_counter = (p.ops & kFixedStride) ? nullptr : work_counter_for(stream);  // tc_launch.cu
-  tc_kernel<C, D, SER, RAW, BO, REF, H16><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmV, p);
+  tc_kernel<C, D, SER, RAW, BO, REF, H16><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmW, tmU, tmV, p);
   return cudaGetLastError();
 }
 
