@@ -69,7 +69,10 @@ enum {
   TRI_INV_ERR_UNSUPPORTED = 2,   /* a valid request this build has no kernel for */
   TRI_INV_ERR_CUDA = 3,          /* a CUDA runtime call or the launch failed */
   TRI_INV_ERR_DEVICE_TIMEOUT = 4,/* a bounded device-side wait expired (see tri_inv_last_device_status) */
-  TRI_INV_ERR_TOO_LARGE = 5      /* more chunks than the fixed scratch of tri_inv_fused_packed_static holds */
+  TRI_INV_ERR_TOO_LARGE = 5,     /* more chunks than the fixed scratch of tri_inv_fused_packed_static holds */
+  TRI_INV_ERR_DEBUG_CHECK = 6    /* device status word only, bounds-checking build only (-DTRI_INV_DEBUG): a kernel
+                                    found an index outside its buffer or tile, or an mbarrier phase out of step;
+                                    the access concerned was skipped, nothing trapped */
 };
 
 /* ---- storage type of K, V, W, U ------------------------------------------ */
@@ -284,6 +287,16 @@ int tri_inv_fused_packed_static(const void* K, const void* V, const float* beta,
 int tri_inv_selftest_wait_timeout(const void* K, const void* V, const float* beta, const float* g,
                                   float* A, void* W, void* U, const tri_inv_desc* desc,
                                   uint64_t wait_limit_ns, int* counters_idle, void* cuda_stream);
+
+/*
+ * Self-test of the bounds-checking build (no step of the paper's method).  tri_inv_fused (block recursion) with the token
+ * bound that the debug build's checks use understated by one chunk: the buffers are as large as the descriptor says, so
+ * no access is out of range either way.  In the bounds-checking build (libtri_inv_debug.so) the work items of the last
+ * chunk of tokens fail their range check, are reduced to no rows (their rows of A, W, U stay unwritten) and the status
+ * word reads TRI_INV_ERR_DEBUG_CHECK; in the ordinary build the call is tri_inv_fused.
+ */
+int tri_inv_selftest_bounds_check(const void* K, const void* V, const float* beta, const float* g,
+                                  float* A, void* W, void* U, const tri_inv_desc* desc, void* cuda_stream);
 
 /*
  * Number of chunk matrices (chunks x heads) the descriptor describes.

@@ -20,7 +20,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 # TRI_INV_LIB selects another build of the same library (the bounds-checking debug build, a development build)
 LIB_PATH = os.environ.get("TRI_INV_LIB") or os.path.join(_PKG, "libtri_inv.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_TOO_LARGE = 0, 1, 2, 3, 4, 5
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_TOO_LARGE, ERR_DEBUG_CHECK = 0, 1, 2, 3, 4, 5, 6
 STATIC_MAX_CHUNKS = 16384
 F32, BF16 = 0, 1
 BLOCK_RECURSIVE, PRODUCT_SERIES, NEWTON_SCHULZ = 0, 1, 2
@@ -39,7 +39,7 @@ FORCE_SIMT = 0x10000
 W_DECAY = 0x20000
 
 EXPORTS = ("tri_inv_build", "tri_inv_build_kda", "tri_inv_fused_kda", "tri_inv_chunk_scan_kda", "tri_inv_chunk_scan", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
-           "tri_inv_selftest_wait_timeout", "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
+           "tri_inv_selftest_wait_timeout", "tri_inv_selftest_bounds_check", "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
 
 
 class Desc(ctypes.Structure):
@@ -83,6 +83,9 @@ def load():
         lib.tri_inv_fused_raw.restype = i32
         lib.tri_inv_fused_packed_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_fused_packed_static.restype = i32
+        if hasattr(lib, "tri_inv_selftest_bounds_check"):
+            lib.tri_inv_selftest_bounds_check.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, vp]
+            lib.tri_inv_selftest_bounds_check.restype = i32
         if hasattr(lib, "tri_inv_selftest_wait_timeout"):
             lib.tri_inv_selftest_wait_timeout.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, ctypes.c_uint64, ctypes.POINTER(ctypes.c_int), vp]
             lib.tri_inv_selftest_wait_timeout.restype = i32

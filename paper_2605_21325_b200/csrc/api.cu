@@ -106,6 +106,8 @@ int run(KParams p, const tri_inv_desc* d, void* stream_v) {
   p.kv_dtype = d->kv_dtype;
   p.chunk_tab = nullptr;
   if (!p.wait_limit_ns) p.wait_limit_ns = 2000000000ull;
+  p.n_tokens = d->cu_seqlens ? (long long)d->T : (long long)d->T * d->B;
+  if (p.ops & kTestShrink) p.n_tokens -= d->C;
   cudaError_t err;
   p.status = status_word_for_current_device(&err);
   if (!p.status) return TRI_INV_ERR_CUDA;
@@ -346,6 +348,20 @@ int tri_inv_selftest_wait_timeout(const void* K, const void* V, const float* bet
   return TRI_INV_OK;
 }
 
+int tri_inv_selftest_bounds_check(const void* K, const void* V, const float* beta, const float* g,
+                                  float* A, void* W, void* U, const tri_inv_desc* desc, void* cuda_stream) {
+  int rc = check_desc(desc, true);
+  if (rc) return rc;
+  if (!K || !V || !beta || !g || !A || !W || !U) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(beta) || !aligned16(g) || !aligned16(A) || !aligned16(W) || !aligned16(U))
+    return TRI_INV_ERR_INVALID_ARG;
+  KParams p{};
+  p.K = K; p.V = V; p.beta = beta; p.g = g; p.A = A; p.W = W; p.U = U;
+  p.method = TRI_INV_BLOCK_RECURSIVE;
+  p.ops = kDoWY | kStoreA | kTestShrink;
+  return run(p, desc, cuda_stream);
+}
+
 int tri_inv_count_matrices(const tri_inv_desc* desc, int64_t* out) {
   int rc = check_desc(desc, false);
   if (rc) return rc;
@@ -378,6 +394,17 @@ int tri_inv_last_device_status(int* out) {
   return TRI_INV_OK;
 }
 
+#ifdef TRI_INV_DEBUG
+// Bounds-checking build only: source line (in the kernels' files) of the first check that failed since the last call; 0 if none.
+int tri_inv_debug_first_failed_check(int* line) {
+  cudaError_t err;
+  int* word = status_word_for_current_device(&err);
+  if (!word || !line) return TRI_INV_ERR_CUDA;
+  if (cudaMemcpy(line, word + 1, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return TRI_INV_ERR_CUDA;
+  return cudaMemset(word + 1, 0, sizeof(int)) == cudaSuccess ? TRI_INV_OK : TRI_INV_ERR_CUDA;
+}
+#endif
+
 int64_t tri_inv_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 
 const char* tri_inv_status_string(int status) {
@@ -388,6 +415,7 @@ const char* tri_inv_status_string(int status) {
     case TRI_INV_ERR_CUDA: return "CUDA runtime error";
     case TRI_INV_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
     case TRI_INV_ERR_TOO_LARGE: return "more chunks than the static scratch table holds";
+    case TRI_INV_ERR_DEBUG_CHECK: return "a bounds or phase check of the debug build failed";
     default: return "unknown status";
   }
 }

@@ -16,6 +16,7 @@ enum : int {
   kRaw = 8,     // K is un-normalised, beta and g are logits: normalise, sigmoid, log-sigmoid + chunk cumsum in the kernel
   kKda = 16,    // per-channel decay (KParams::G); with kDoWY, W = A diag(beta) (K * exp G)
   kFixedStride = 64,  // tensor-core kernel: take no work-counter pair (and create no event for one); items by a fixed stride
+  kTestShrink = 256,  // self-test: the token bound the debug build checks against is understated by one chunk
   kTestStall = 128,   // self-test: CTA 0 leaves out the first Gram product so that its bounded wait runs out
   kWDecay = 32, // W = A diag(beta) diag(exp g) K: the decay-weighted factor the chunk-state recurrence consumes
 };
@@ -48,7 +49,17 @@ struct KParams {
   int32_t method;               // TRI_INV_* method with flags
   int32_t ops;                  // kStoreA | kDoWY | kLoadA | ...
   unsigned long long wait_limit_ns;  // per bounded device-side wait (run() fills in the default of two seconds)
+  long long n_tokens;           // flat tokens of the tensors (B * T, or T when packed): the bound the debug build checks rows against
 };
+
+// Bounds-checking build (-DTRI_INV_DEBUG, libtri_inv_debug.so): TRI_INV_CHECK(p, cond) raises TRI_INV_ERR_DEBUG_CHECK in
+// the device status word when cond is false and evaluates to cond, so that the guarded access can be skipped; in the
+// ordinary build it is the constant true and costs nothing.  Never a trap or a device assert.
+#ifdef TRI_INV_DEBUG
+#define TRI_INV_CHECK(p, cond) ((cond) ? true : (atomicMax((p).status, (int)TRI_INV_ERR_DEBUG_CHECK), atomicCAS((p).status + 1, 0, __LINE__), false))   // word 1: source line of the first failed check
+#else
+#define TRI_INV_CHECK(p, cond) (true)
+#endif
 
 // Flat work item -> (first token, real rows, head).  Consecutive items walk the heads of
 // one chunk of tokens, so neighbouring CTAs touch neighbouring memory.  Items and tokens are
@@ -57,7 +68,7 @@ __device__ __forceinline__ void locate(const KParams& p, int C, int item, int& t
   const unsigned c = (unsigned)item / (unsigned)p.H;
   h = (int)((unsigned)item - c * (unsigned)p.H);
   if (p.chunk_tab) {
-    ChunkEntry e = p.chunk_tab[c];
+    ChunkEntry e = TRI_INV_CHECK(p, c < (unsigned)p.n_chunks) ? p.chunk_tab[c] : ChunkEntry{0, 0};
     tok0 = e.tok0;
     rows = e.rows;
   } else {

@@ -79,6 +79,7 @@ extern "C" int tri_inv_fused_packed_static(const void* K, const void* V, const f
   p.chunks_per_seq = 0;
   p.chunk_tab = dev_tab;
   p.wait_limit_ns = 2000000000ull;
+  p.n_tokens = desc->T;   // packed mode: T is the total
   p.status = status_word_for_current_device(&err);
   if (!p.status) return TRI_INV_ERR_CUDA;
 

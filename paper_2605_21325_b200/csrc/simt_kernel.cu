@@ -118,6 +118,8 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
   for (int item = blockIdx.x; item < total; item += gridDim.x) {
     int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
+    // bounds-checking build: an item outside the tensors is reduced to no rows (nothing of it is then read or stored)
+    if (!TRI_INV_CHECK(p, rows >= 1 && rows <= C && tok0 >= 0 && (long long)tok0 + rows <= p.n_tokens && h >= 0 && h < p.H)) { tok0 = 0; rows = 0; h = 0; }
     __syncthreads();  // previous item's readers are done with shared memory
     for (int i = tid; i < C; i += kThreads) {
       size_t bi = (size_t)(tok0 + i) * p.H + h;
@@ -347,7 +349,7 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
     if ((p.ops & kStoreA) && p.A) {
       for (int e = tid; e < C * C; e += kThreads) {
         int i = e / C, j = e - i * C;
-        if (i < rows) {
+        if (i < rows && TRI_INV_CHECK(p, (long long)tok0 + i < p.n_tokens)) {
           float v = (j < i) ? Xres[i * LD + j] : (j == i ? 1.f : 0.f);
           p.A[((size_t)(tok0 + i) * p.H + h) * C + j] = v;
         }
@@ -378,7 +380,7 @@ __global__ void __launch_bounds__(kThreads) simt_kernel(KParams p) {
           for (int i = tid / kSlice; i < rows; i += kThreads / kSlice) {
             float s = Ks[i * kSliceLd + cc];  // diagonal term, A_ii = 1
             for (int j = 0; j < i; ++j) s = fmaf(Xres[i * LD + j], Ks[j * kSliceLd + cc], s);
-            if (c0 + cc < d) {
+            if (c0 + cc < d && TRI_INV_CHECK(p, (long long)tok0 + i < p.n_tokens)) {
               size_t o = ((size_t)(tok0 + i) * p.H + h) * d + c0 + cc;
               if (p.kv_dtype == TRI_INV_F32) ((float*)dst)[o] = s;
               else ((__nv_bfloat16*)dst)[o] = __float2bfloat16_rn(s);

@@ -520,6 +520,9 @@ __device__ __forceinline__ void store_frag_piece_bf16(const float (&f)[8][4], ui
     asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
   }
   if (rows_left >= 16) {
+#ifdef TRI_INV_DEBUG
+    if (x < 0 || y < 0 || (x & 7)) return;   // a tiled store must start on a 16-byte boundary and inside the tensor (the caller's item check covers y + 16)
+#endif
     fence_proxy_async();   // this lane's staging writes become visible to the copy engine
     __syncwarp();
     if (lane == 0) {

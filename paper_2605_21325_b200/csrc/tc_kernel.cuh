@@ -118,8 +118,15 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
   // left at a barrier or using tensor memory while another frees it.
   volatile int* const s_gave_up = reinterpret_cast<volatile int*>(smem + cfg::OFF_BAR + 40);
   bool bad = false;
+  uint32_t n_issue = 0;  // copies requested by this thread (the K thread: K tiles, the V thread: V tiles): the exit path waits for the last one
   auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
     if (bad) return false;
+#ifdef TRI_INV_DEBUG
+    // mbarrier bookkeeping, checked by the thread that requests the copies: the phase it waits for must be the one its
+    // most recent request completes
+    if ((bar == bar_k && threadIdx.x == 64) || (bar == bar_v && threadIdx.x == 96))
+      TRI_INV_CHECK(p, n_issue > 0 && ((n_issue - 1) & 1u) == parity);
+#endif
     bad = !mbar_wait_bounded(bar, parity, p.wait_limit_ns);
     return !bad;
   };
@@ -153,10 +160,12 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
   // K and V complete on separate barriers: the Gram product starts on K alone, and each buffer is
   // refilled as soon as its last reader is done.
   constexpr int kTidL2 = 32, kTidK = 64, kTidV = 96;
-  uint32_t n_issue = 0;  // copies requested by this thread (the K thread: K tiles, the V thread: V tiles): the exit path waits for the last one
   auto issue_k = [&](int tok0, int h) {
     if (bad) return;
     ++n_issue;
+#ifdef TRI_INV_DEBUG
+    if (!TRI_INV_CHECK(p, tok0 >= 0 && tok0 < p.n_tokens && h >= 0 && h < p.H)) return;
+#endif
     fence_proxy_async();
     mbar_expect_tx(bar_k, (uint32_t)cfg::TILE_BYTES);
 #pragma unroll
@@ -165,6 +174,9 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
   auto issue_v = [&](int tok0, int h) {
     if (bad) return;
     ++n_issue;
+#ifdef TRI_INV_DEBUG
+    if (!TRI_INV_CHECK(p, tok0 >= 0 && tok0 < p.n_tokens && h >= 0 && h < p.H)) return;
+#endif
     fence_proxy_async();
     mbar_expect_tx(bar_v, (uint32_t)cfg::TILE_BYTES);
 #pragma unroll
@@ -174,7 +186,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
   auto fetch_bg = [&](int tok0, int rows, int h) -> float {
     const int i = tid < C ? tid : tid - C;
     const float* src = tid < C ? p.beta : p.g;
-    return (i < rows && src) ? src[(size_t)(tok0 + i) * p.H + h] : 0.f;
+    return (i < rows && src && TRI_INV_CHECK(p, (long long)tok0 + i < p.n_tokens)) ? src[(size_t)(tok0 + i) * p.H + h] : 0.f;
   };
   // Prologue.  The threads that own the K and V barriers initialise them and request the first
   // item's tiles at once, so that the copies run while tensor memory is being allocated.
@@ -235,6 +247,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
   while (item < total && !misaligned) {
     int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
+    // bounds-checking build: an item outside the tensors is reduced to no rows (nothing of it is then stored)
+    if (!TRI_INV_CHECK(p, rows >= 1 && rows <= C && tok0 >= 0 && (long long)tok0 + rows <= p.n_tokens && h >= 0 && h < p.H)) { tok0 = 0; rows = 0; h = 0; }
     PHASE_BEGIN();
 
     // ---- 1. beta, g were fetched during the previous item (sBeta and sG are adjacent: one store each)
@@ -292,7 +306,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         const int e = tid + m * cfg::NT;
         const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (i < rows && j < i) v = *reinterpret_cast<const float4*>(a_src + (size_t)m * a_step);
+        if (i < rows && j < i && TRI_INV_CHECK(p, (long long)tok0 + i < p.n_tokens)) v = *reinterpret_cast<const float4*>(a_src + (size_t)m * a_step);
         v.x = (j + 0 < i) ? v.x : (j + 0 == i ? 1.f : 0.f);
         v.y = (j + 1 < i) ? v.y : (j + 1 == i ? 1.f : 0.f);
         v.z = (j + 2 < i) ? v.z : (j + 2 == i ? 1.f : 0.f);
@@ -873,7 +887,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       const float4 b = *reinterpret_cast<const float4*>(sBeta + j);
       const uint32_t lo = pack_bf16(v.x * b.x, v.y * b.y), hi = pack_bf16(v.z * b.z, v.w * b.w);
       const uint32_t off = (uint32_t)((j >> 6) * (C * 128) + i * 128 + (((((j & 63) >> 3) ^ (i & 7)) << 4) | ((j & 7) * 2)));
-      asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sAp + off), "r"(lo), "r"(hi) : "memory");
+      if (TRI_INV_CHECK(p, off + 8 <= (uint32_t)(C * C * 2) && i < C && j + 4 <= C))
+        asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sAp + off), "r"(lo), "r"(hi) : "memory");
     };
     float4 xv[cfg::ALIAS ? 1 : NV];
     if constexpr (cfg::ALIAS) {
@@ -887,7 +902,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         const int e = tid + m * cfg::NT;
         const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
         const float4 v = *reinterpret_cast<const float4*>(sX + i * LD + j);
-        if (a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
+        if (a_dst && i < rows && TRI_INV_CHECK(p, (long long)tok0 + i < p.n_tokens && j + 4 <= C)) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
         if (do_wy) put_ap(i, j, v);
         if (C == 128 && do_wy && (m == 3 || m == 7 || m == 11)) {
           fence_proxy_async();
@@ -911,7 +926,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       // shared memory: +0.0 above the diagonal, 1.0f on it.  Rows past the sequence end are not copied.
       fence_proxy_async();   // the merges' stores become visible to the copy engine
       __syncthreads();
-      if ((p.ops & kStoreA) && p.A && tid < rows) {
+      if ((p.ops & kStoreA) && p.A && tid < rows && TRI_INV_CHECK(p, (long long)tok0 + tid < p.n_tokens)) {
         float* dst = p.A + ((size_t)(tok0 + tid) * p.H + h) * C;
         asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(sX + tid * LD)), "r"(C * 4) : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -925,7 +940,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         const float4 v = *reinterpret_cast<const float4*>(sX + i * LD + j);
         xv[m] = v;
         // without a WY product there is nothing to overlap the stores with: issue them right away
-        if (!do_wy && a_dst && i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
+        if (!do_wy && a_dst && i < rows && TRI_INV_CHECK(p, (long long)tok0 + i < p.n_tokens && j + 4 <= C)) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
       }
     }
     // the item after next (read after this item's last barrier): by ticket, or by a fixed stride without a counter pair
@@ -983,7 +998,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
 #pragma unroll
         for (int m = 0; m < NV; ++m) {
           const int i = (tid + m * cfg::NT) / (C / 4);
-          if (i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = xv[m];
+          if (i < rows && TRI_INV_CHECK(p, (long long)tok0 + i < p.n_tokens)) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = xv[m];
         }
       }
       wait(bar_mma, ph_mma);
