@@ -1,10 +1,10 @@
 """numpy fp64 restatements of the paper's inversion algorithms (TEST INFRASTRUCTURE ONLY).
 
 Each function inverts ``I + L`` for one strictly lower triangular ``L`` (n a
-power of two), taking the steps in the paper's order and notation.  They exist
-so the tests can check that the two schemes the CUDA library implements reach,
-in exact arithmetic, the same matrix as forward substitution; they are never
-used by the product.
+power of two) by one of the schemes the paper analyses, written here from the
+identity each scheme rests on.  They exist so the tests can check that the
+schemes the CUDA library implements reach, in exact arithmetic, the same matrix
+as forward substitution; they are never used by the product.
 
 Sign convention: every routine here inverts ``I + L``; Eq. 3's ``I - phi .* L^-``
 is the same thing with ``L := -phi .* L^-``.
@@ -40,16 +40,16 @@ def neumann_series(L: np.ndarray) -> np.ndarray:
 
 
 def mch(L: np.ndarray) -> np.ndarray:
-    """Alg. 5 (repeated squaring).  X <- I - L, Y <- L, then log2(n) - 1 rounds of
-    Y <- Y.Y ; X <- X + X.Y, which sums the series up to power n - 1."""
+    """Repeated squaring of the nilpotent series (Alg. 5 / Sec. 3.2).  With P_k = L^(2^k) the partial sum up to power
+    2^(k+1) - 1 is S_k = (I - L)(I + P_1)(I + P_2) ... (I + P_k); each round squares P and multiplies the sum by the
+    next factor, and log2(n) - 1 rounds reach power n - 1, beyond which every power vanishes."""
     n = L.shape[0]
-    X = np.eye(n) - L
-    Y = L.copy()
-    rounds = max(int(np.log2(n)) - 1, 0)
-    for _ in range(rounds):
-        Y = Y @ Y
-        X = X + X @ Y
-    return X
+    total = np.eye(n) - L
+    power = L.copy()
+    for _ in range(max(int(np.log2(n)) - 1, 0)):
+        power = power @ power
+        total = total @ (np.eye(n) + power)
+    return total
 
 
 def product_form(L: np.ndarray) -> np.ndarray:
@@ -63,27 +63,19 @@ def product_form(L: np.ndarray) -> np.ndarray:
     return X
 
 
-def _diag_blocks(X: np.ndarray, b: int, parity: int) -> np.ndarray:
-    n = X.shape[0]
-    D = np.zeros_like(X)
-    for t in range(n // b):
-        if t % 2 == parity:
-            s = slice(t * b, (t + 1) * b)
-            D[s, s] = X[s, s]
-    return D
-
-
 def mbh(L: np.ndarray, X0: np.ndarray | None = None, b0: int = 1) -> np.ndarray:
-    """Alg. 4 (unrolled Bunch-Hopcroft): for b = b0, 2 b0, ... < n:
-    X <- D_e + D_o - D_o . L . D_e with D_e / D_o the 1st,3rd,.. / 2nd,4th,.. b x b
-    diagonal blocks of X (Lemma C.1 stops at b = n/2; the b = n step is a no-op)."""
+    """Bunch-Hopcroft recursion, bottom up (Alg. 4 / Sec. 3.3).  X0 holds the inverses of the b0 x b0 diagonal blocks
+    of I + L (the identity for b0 = 1).  At block size b every adjacent pair (upper block r, lower block r + b) is
+    joined by the 2x2 block identity for a lower triangular matrix: the pair's off-diagonal block becomes
+    -X_low . L_low,up . X_up; doubling b until one block is left gives the inverse.  Only the blocks the next level
+    reads are formed."""
     n = L.shape[0]
-    X = np.eye(n) if X0 is None else X0.copy()
+    X = np.eye(n) if X0 is None else np.array(X0, dtype=np.float64)
     b = b0
     while b < n:
-        De = _diag_blocks(X, b, 0)
-        Do = _diag_blocks(X, b, 1)
-        X = De + Do - Do @ L @ De
+        for r in range(0, n, 2 * b):
+            up, low = slice(r, r + b), slice(r + b, r + 2 * b)
+            X[low, up] = -(X[low, low] @ L[low, up] @ X[up, up])
         b *= 2
     return X
 
@@ -100,16 +92,13 @@ def mxr(L: np.ndarray, b0: int = 16) -> np.ndarray:
 
 
 def newton_schulz(L: np.ndarray, m: int | None = None, x0_scale: float | None = None) -> np.ndarray:
-    """Alg. 3: A = I + L, X_0 = I / n (the initial guess I / n^{O(1)} of Prop. 3.2 with exponent 1),
-    then m rounds of Y <- A.X, X <- 2X - X.Y.  Default m = 2 log2(n)."""
+    """Newton's iteration for the inverse of M = I + L (Alg. 3 / Sec. 3.5): X <- X (2I - M X), whose residual I - M X
+    squares every round, from X_0 = I / n (the exponent-1 reading of Prop. 3.2's I / n^O(1)).  Default 2 log2(n) rounds."""
     n = L.shape[0]
-    A = np.eye(n) + L
+    M = np.eye(n) + L
     X = np.eye(n) * (1.0 / n if x0_scale is None else x0_scale)
-    if m is None:
-        m = 2 * int(np.log2(n))
-    for _ in range(m):
-        Y = A @ X
-        X = 2 * X - X @ Y
+    for _ in range(2 * int(np.log2(n)) if m is None else m):
+        X = X @ (2.0 * np.eye(n) - M @ X)
     return X
 
 
