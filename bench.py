@@ -347,12 +347,13 @@ def main():
     d2h = sum(x.numel() * x.element_size() for x in (hA, hW, hU))
 
     pipe = None
-    if args.call == "fused":
-        pipe = binding.HostPipeline(inp.B, inp.T, inp.H, inp.d_k, inp.d_v, inp.C, dtype=K.dtype, cu_seqlens=inp.cu_seqlens)
+    if args.call == "fused":   # the C-ABI call that takes host buffers: tri_inv_fused_host with a device workspace of the caller's
+        pipe = torch.empty(binding.fused_host_workspace_bytes(inp.B, inp.T, inp.H, inp.d_k, inp.d_v, inp.C, binding._dtype_code(K),
+                                                              inp.cu_seqlens), dtype=torch.uint8, device="cuda")
 
     def e2e_step():
-        if pipe is not None:  # the public host-to-host call: slices of the batch overlap upload, kernel and download
-            pipe.run(hK, hV, hb, hg, hA, hW, hU, method=method)
+        if pipe is not None:  # slices of the batch overlap upload, kernel and download inside the call
+            binding.fused_host(hK, hV, hb, hg, inp.C, hA, hW, hU, pipe, method=method, cu_seqlens=inp.cu_seqlens, stream=stream)
             return
         K.copy_(hK, non_blocking=True); V.copy_(hV, non_blocking=True)
         beta.copy_(hb, non_blocking=True); g.copy_(hg, non_blocking=True)
@@ -440,7 +441,7 @@ def main():
                           "parallelism": "independent replicas, no collective" if world > 1 else "single GPU"},
                "gb_per_s": achieved, "roofline": roofline, "cpu_baseline": cpu,
                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-                       "api": "binding.HostPipeline.run (pinned host in, pinned host out, %d slices)" % len(pipe.slices) if pipe else "copies + " + args.call},
+                       "api": "tri_inv_fused_host (C ABI: pinned host buffers in and out, device workspace of the caller's)" if pipe is not None else "copies + " + args.call},
                "gpu_launches": launches, "clocks": clocks, "error_vs_oracle": err}
         print(json.dumps(out))
     if world > 1:

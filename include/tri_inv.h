@@ -56,6 +56,7 @@
 #ifndef TRI_INV_H_
 #define TRI_INV_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -178,6 +179,24 @@ int tri_inv_fused(const void* K, const void* V, const float* beta, const float* 
  */
 int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A,
                       const tri_inv_desc* desc, int method, void* cuda_stream);
+
+/*
+ * tri_inv_fused for tensors in HOST memory (no step of the paper's method: the end-to-end form of the fused call).
+ *   K, V, beta, g        HOST inputs, layouts as above; pinned (page-locked) memory makes the copies asynchronous
+ *   A (nullable), W, U   HOST outputs
+ *   workspace            DEVICE memory, 256-byte aligned, at least tri_inv_fused_host_workspace(desc) bytes, the caller's
+ * The batch is cut into up to 16 slices of whole chunks (a dense batch whose T is a multiple of C; anything else goes as
+ * one slice); each slice is copied in, run through tri_inv_fused and copied out on one of three streams the library keeps
+ * per device, so uploads, kernels and downloads overlap.  The work is ordered after what is already in cuda_stream, and
+ * cuda_stream is made to wait for all of it: synchronising cuda_stream (or an event recorded on it) after the call
+ * covers the outputs.  The call itself returns after enqueueing when the host buffers are pinned.  One call at a time per
+ * device: calls from several host threads must be serialised by the caller (they share the three streams).  Results are
+ * those of tri_inv_fused.  Errors as for tri_inv_fused; INVALID_ARG also for a workspace that is too small or misaligned.
+ */
+int tri_inv_fused_host_workspace(const tri_inv_desc* desc, size_t* bytes);
+int tri_inv_fused_host(const void* K, const void* V, const float* beta, const float* g,
+                       float* A, void* W, void* U, void* workspace, size_t workspace_bytes,
+                       const tri_inv_desc* desc, int method, void* cuda_stream);
 
 /*
  * Per-channel decay through the WY step (KDA row of Table 1, with the decay-weighted factor the layer's chunk form needs):

@@ -39,7 +39,7 @@ FORCE_SIMT = 0x10000
 W_DECAY = 0x20000
 
 EXPORTS = ("tri_inv_build", "tri_inv_build_kda", "tri_inv_fused_kda", "tri_inv_chunk_scan_kda", "tri_inv_chunk_scan", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
-           "tri_inv_selftest_wait_timeout", "tri_inv_selftest_bounds_check", "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
+           "tri_inv_fused_host", "tri_inv_fused_host_workspace", "tri_inv_selftest_wait_timeout", "tri_inv_selftest_bounds_check", "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
 
 
 class Desc(ctypes.Structure):
@@ -83,6 +83,11 @@ def load():
         lib.tri_inv_fused_raw.restype = i32
         lib.tri_inv_fused_packed_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, i32, vp]
         lib.tri_inv_fused_packed_static.restype = i32
+        if hasattr(lib, "tri_inv_fused_host"):
+            lib.tri_inv_fused_host_workspace.argtypes = [dp, ctypes.POINTER(ctypes.c_size_t)]
+            lib.tri_inv_fused_host_workspace.restype = i32
+            lib.tri_inv_fused_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, dp, i32, vp]
+            lib.tri_inv_fused_host.restype = i32
         if hasattr(lib, "tri_inv_selftest_bounds_check"):
             lib.tri_inv_selftest_bounds_check.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, vp]
             lib.tri_inv_selftest_bounds_check.restype = i32
@@ -311,6 +316,27 @@ def selftest_wait_timeout(K, V, beta, g, C, wait_limit_ns, out, stream=None):
     if rc != OK:
         raise TriInvError("tri_inv_selftest_wait_timeout", rc)
     return bool(idle.value)
+
+
+def fused_host_workspace_bytes(B, T, H, d_k, d_v, C, kv_dtype, cu_seqlens=None) -> int:
+    desc, keep = make_desc(B, T, H, d_k, d_v, C, kv_dtype, cu_seqlens)
+    n = ctypes.c_size_t(0)
+    rc = load().tri_inv_fused_host_workspace(ctypes.byref(desc), ctypes.byref(n))
+    if rc != OK:
+        raise TriInvError("tri_inv_fused_host_workspace", rc)
+    return int(n.value)
+
+
+def fused_host(hK, hV, hbeta, hg, C, hA, hW, hU, workspace, method=BLOCK_RECURSIVE, cu_seqlens=None, stream=None):
+    """tri_inv_fused_host: every tensor argument is a HOST tensor (pinned for asynchronous copies), ``workspace`` a CUDA
+    uint8 tensor of at least ``fused_host_workspace_bytes`` bytes.  hA may be None.  Enqueues and returns."""
+    B, T, H, d_k = hK.shape
+    desc, keep = make_desc(B, T, H, d_k, hV.shape[-1], C, _dtype_code(hK), cu_seqlens)
+    hp = lambda t: None if t is None else ctypes.c_void_p(t.data_ptr())
+    rc = load().tri_inv_fused_host(hp(hK), hp(hV), hp(hbeta), hp(hg), hp(hA), hp(hW), hp(hU), ctypes.c_void_p(workspace.data_ptr()),
+                                   ctypes.c_size_t(workspace.numel() * workspace.element_size()), ctypes.byref(desc), int(method), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_fused_host", rc)
 
 
 class HostPipeline:
