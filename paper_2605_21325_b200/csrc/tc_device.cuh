@@ -270,7 +270,7 @@ __device__ __forceinline__ void refine_step(float* sX, float* sN, int warp, int 
       const int slot = rb * (CPW) + c;
       acc[slot][0] = acc[slot][1] = acc[slot][2] = acc[slot][3] = 0.f;
     }
-#pragma unroll
+#pragma unroll 1                               // (a run-time loop: unrolled, the step's code would not fit the instruction cache)
     for (int q = 0; q < 2 * rb + 2; ++q) {     // k-step of eight: columns 8q .. 8q+7 of X, rows of N
       bool any = false;
 #pragma unroll
@@ -335,7 +335,7 @@ __device__ __forceinline__ void refine_step(float* sX, float* sN, int warp, int 
         d[0] = xa.x; d[1] = xa.y; d[2] = xb.x; d[3] = xb.y;
       }
     }
-#pragma unroll
+#pragma unroll 1
     for (int q = 0; q < 2 * rb + 2; ++q) {
       bool any = false;
 #pragma unroll

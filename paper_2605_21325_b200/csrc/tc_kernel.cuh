@@ -88,7 +88,10 @@ struct Cfg {
 };
 
 // Byte offset of the 16-byte chunk holding features [f, f+8) of row r inside a swizzled tile.
-template <int C, int D, bool SER, bool RAW, bool BO, bool REF, bool H16>
+// VAR specialises two run-time switches away so that the common case carries less code (the instruction cache is shared
+// by four CTAs in different phases): 0 = fused / build call with substitution leaves, 1 = with series leaves,
+// 2 = tri_inv_wy (A read from memory), 3 = decided at run time.
+template <int C, int D, bool SER, bool RAW, bool BO, bool REF, bool H16, int VAR>
 __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SER, BO, REF, H16>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                                                                              const __grid_constant__ CUtensorMap tmV, const __grid_constant__ KParams p) {
   using cfg = Cfg<C, D, SER, BO, REF, H16>;
@@ -141,7 +144,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
   const uint32_t lane_base = (C == 64) ? 32u * warp : 16u * rb;
   const bool do_wy = !BO && (p.ops & kDoWY) != 0;
   const bool need_v = do_wy && p.V != nullptr;
-  const bool load_a = (p.ops & kLoadA) != 0;
+  const bool load_a = VAR == 3 ? (p.ops & kLoadA) != 0 : VAR == 2;
+  const bool leaf_series_on = VAR == 3 ? (p.method & TRI_INV_LEAF_SERIES) != 0 : VAR == 1;
   // RAW compiles in the code that rewrites the K tile in shared memory before the WY step and the per-row
   // factors of the gate.  Two run-time uses: the front end (sigmoid, log-sigmoid + chunk cumsum, key
   // normalisation: kRaw) and the decay-weighted W (rows of K times exp(g_i): kWDecay).
@@ -754,7 +758,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       PHASE(2);
 
       // ---- 4. leaf: invert this warp's 16x16 diagonal block
-      if (p.method & TRI_INV_LEAF_SERIES) {
+      if (leaf_series_on) {
         leaf_series<LD, cfg::LEAF_LD>(sX + 16 * rb * LD + 16 * rb,
                                       reinterpret_cast<float*>(smem + cfg::OFF_LEAF) + warp * 16 * cfg::LEAF_LD, lane);
       } else {
@@ -1108,7 +1112,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
 }
 
 // ------------------------------------------------------------------------------------------ host side
-template <int C, int D, bool SER, bool RAW, bool BO = false, bool REF = false, bool H16 = false>
+template <int C, int D, bool SER, bool RAW, bool BO = false, bool REF = false, bool H16 = false, int VAR = 3>
 cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   using cfg = Cfg<C, D, SER, BO, REF, H16>;
   KParams p = p_in;
@@ -1123,9 +1127,9 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   {
     std::lock_guard<std::mutex> lock(mu);
     if (!ctas_per_sm_of[dev]) {
-      e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO, REF, H16>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
+      e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO, REF, H16, VAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM);
       if (e != cudaSuccess) return e;
-      e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO, REF, H16>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+      e = cudaFuncSetAttribute(tc_kernel<C, D, SER, RAW, BO, REF, H16, VAR>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
       if (e != cudaSuccess) return e;
       int sms = 0, smem_per_sm = 0;
       if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
@@ -1156,7 +1160,7 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   long long cap = (long long)n_sm * ctas_per_sm;
   int grid = (int)(total < cap ? total : cap);
   p.work_counter = (p.ops & kFixedStride) ? nullptr : work_counter_for(stream);  // tc_launch.cu
-  tc_kernel<C, D, SER, RAW, BO, REF, H16><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmW, tmU, tmV, p);
+  tc_kernel<C, D, SER, RAW, BO, REF, H16, VAR><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmW, tmU, tmV, p);
   return cudaGetLastError();
 }
 
