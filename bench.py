@@ -35,9 +35,15 @@ UNIT = "chunk-matrices/s"
 FALLBACK_HBM_GBS = 6650.0
 OUTPUTS = {"fused": "A fp32 + W,U", "raw": "A fp32 + W,U", "build": "A fp32", "kda": "A fp32", "kda_fused": "A fp32 + W,U", "wy": "W,U", "scan": "O", "layer": "O"}
 
-# DRAM bytes per chunk matrix moved by the fused kernel (dram__bytes_read.sum + dram__bytes_write.sum
-# of one ncu capture divided by the matrices of that launch); see profiles/.  None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_MATRIX = {(2, "block_recursive"): 68890}  # profiles/tc_kernel_c64_cfg2.md
+def ncu_traffic_bytes_per_matrix(call, config, method):
+    """DRAM bytes per chunk matrix (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture divided by the matrices
+    of that launch) from profiles/ncu_traffic.json, which is rewritten whenever the kernel is captured again; None when
+    that call / configuration / method has no capture."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "ncu_traffic.json")) as f:
+            return json.load(f)["%s:cfg%d:%s" % (call, config, method)]["dram_bytes_per_matrix"]
+    except Exception:
+        return None
 
 
 def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True, call="fused"):
@@ -421,7 +427,7 @@ def main():
         kernel_ms = statistics.mean(times_ms)               # one launch per step, timed alone by its event pair
         achieved = alg_bytes * n_mat / (kernel_ms * 1e-3) / 1e9
         peak, peak_kind = measured_peak_gbs()
-        traffic = NCU_TRAFFIC_BYTES_PER_MATRIX.get((args.config, args.method)) if args.call == "fused" else None
+        traffic = None if args.paper_T else ncu_traffic_bytes_per_matrix(args.call, args.config, args.method)
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": None if traffic is None else traffic * n_mat, "peak_source": "of " + peak_kind,
                     "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "kda": "per-channel-decay build+invert", "kda_fused": "per-channel-decay build+invert, key scaling, WY (3 launches)", "wy": "WY apply", "scan": "chunk scan (state recurrence + output)", "layer": "fused build+invert+WY, then chunk scan (2 launches)"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),

@@ -81,6 +81,9 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // every bulk store this thread has committed has finished READING its shared-memory source
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// ... all but the KEEP most recent ones have (two staging tiles used in turn: KEEP = 1)
+template <int KEEP>
+__device__ __forceinline__ void bulk_wait_read_keep() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(KEEP) : "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tm) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
@@ -503,13 +506,14 @@ __device__ __forceinline__ void stmatrix_x4(uint32_t addr, uint32_t m0, uint32_t
 // then leaves through the copy engine (one tiled bulk store: tm is a 2-D map of the output with boxes of 64
 // columns x 16 rows in the same 128-byte swizzle, x / y the piece's first column and token), which costs
 // the warp no load/store instructions; lane 0 owns the stores, and waits for the previous one to have read the
-// staging tile before it is rewritten.  The caller waits again (bulk_wait_read, lane 0) before the staging
+// staging tile before it is rewritten (with two tiles used in turn, KEEP = 1 lets the latest store go on).  The caller waits again (bulk_wait_read, lane 0) before the staging
 // space is used for anything else.  A piece cut short by its sequence's end takes 16-byte loads and
 // coalesced 16-byte global stores of its real rows only (8 lanes cover one 128-byte row segment).
+template <int KEEP = 0>
 __device__ __forceinline__ void store_frag_piece_bf16(const float (&f)[8][4], uint32_t stage, int lane, __nv_bfloat16* out_row0,
                                                       size_t row_stride, int rows_left, const CUtensorMap* tm, int x, int y) {
   const int mi = lane >> 3, r = (lane & 7) + 8 * (mi & 1);
-  if (lane == 0) bulk_wait_read();
+  if (lane == 0) bulk_wait_read_keep<KEEP>();   // KEEP = 1: the store issued just before this one used the other staging tile
   __syncwarp();
 #pragma unroll
   for (int nt = 0; nt < 8; nt += 2) {
@@ -541,12 +545,13 @@ __device__ __forceinline__ void store_frag_piece_bf16(const float (&f)[8][4], ui
   }
   __syncwarp();
 }
+template <int KEEP = 0>
 __device__ __forceinline__ void store_piece_bf16(uint32_t taddr, uint32_t stage, int lane, __nv_bfloat16* out_row0,
                                                  size_t row_stride, int rows_left, const CUtensorMap* tm, int x, int y) {
   float f[8][4];
   tmem_ld_16x64(f, taddr);
   tmem_wait_ld();
-  store_frag_piece_bf16(f, stage, lane, out_row0, row_stride, rows_left, tm, x, y);
+  store_frag_piece_bf16<KEEP>(f, stage, lane, out_row0, row_stride, rows_left, tm, x, y);
 }
 
 // ------------------------------------------------------------------------------------------ host side

@@ -24,6 +24,7 @@
 #pragma once
 #include <cuda.h>
 
+#include <cstdlib>
 #include <mutex>
 
 #include "tc_device.cuh"
@@ -1048,15 +1049,20 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
           gram_early = true;
         }
         store_frag_piece_bf16(f0, stage, lane, u_row0, row_stride, rows - row0, &tmU, h * D + 0, tok0 + row0);
-        store_frag_piece_bf16(f1, stage, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
+        // second staging tile: the A' operand's space, whose last reader (the U product) has completed
+        store_frag_piece_bf16<1>(f1, sAp + warp * 2048, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
       } else {
         // C = 128 (W and U side by side in 256 columns) or W only
         if (cfg::ALIAS && tid == kTidK && has_next && !load_a) issue_k(nx_tok0, nx_h);  // all MMAs on the tiles are done
-        store_piece_bf16(tmem_rows, stage, lane, w_row0, row_stride, rows - row0, &tmW, h * D, tok0 + row0);
-        store_piece_bf16(tmem_rows + 64, stage, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
+        // two staging tiles in turn where there is room for a second one (with ALIAS: the upper half of the A' region;
+        // every product that reads A' has completed)
+        const uint32_t stage2 = cfg::ALIAS ? stage + cfg::NW * 2048 : stage;
+        constexpr int KEEP = cfg::ALIAS ? 1 : 0;
+        store_piece_bf16<0>(tmem_rows, stage, lane, w_row0, row_stride, rows - row0, &tmW, h * D, tok0 + row0);
+        store_piece_bf16<KEEP>(tmem_rows + 64, stage2, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
         if (need_v) {
-          store_piece_bf16(tmem_rows + 128, stage, lane, u_row0, row_stride, rows - row0, &tmU, h * D, tok0 + row0);
-          store_piece_bf16(tmem_rows + 192, stage, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
+          store_piece_bf16<KEEP>(tmem_rows + 128, stage, lane, u_row0, row_stride, rows - row0, &tmU, h * D, tok0 + row0);
+          store_piece_bf16<KEEP>(tmem_rows + 192, stage2, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
         }
         tc_fence_before();
         __syncthreads();
@@ -1159,6 +1165,9 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   long long total = (long long)p.n_chunks * p.H;
   long long cap = (long long)n_sm * ctas_per_sm;
   int grid = (int)(total < cap ? total : cap);
+#ifdef TRI_INV_PHASE_CLOCKS
+  if (const char* gc = getenv("TRI_INV_GRID_CAP")) { int g2 = atoi(gc); if (g2 > 0 && g2 < grid) grid = g2; }
+#endif
   p.work_counter = (p.ops & kFixedStride) ? nullptr : work_counter_for(stream);  // tc_launch.cu
   tc_kernel<C, D, SER, RAW, BO, REF, H16, VAR><<<grid, cfg::NT, cfg::SMEM, stream>>>(tmK, tmW, tmU, tmV, p);
   return cudaGetLastError();
