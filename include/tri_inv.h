@@ -24,6 +24,9 @@
  * every function returns a TRI_INV_* status.  There is no CPU fallback: on a
  * machine without a usable GPU the compute calls return TRI_INV_ERR_CUDA.
  *
+ * TRI_INV_LOG=1 in the environment makes the build / WY / fused calls print one line per kernel launch on stderr
+ * (shape, method, which kernel took it); nothing else in the library writes to a stream.
+ *
  * Shared state and its limits.  (1) One status word per device, shared by all streams and all
  * entry points: tri_inv_last_device_status() reports that SOME kernel since the last read gave up
  * on a wait, not which.  (2) The tensor-core kernels spread their work with a counter pair in

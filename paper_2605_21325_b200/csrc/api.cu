@@ -1,5 +1,7 @@
 // extern "C" boundary: argument validation, chunk table for packed sequences, dispatch.
 #include <atomic>
+#include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -57,6 +59,12 @@ cudaMemPool_t table_pool_for_current_device() {
     pools[dev] = pool;
   }
   return pools[dev];
+}
+
+// TRI_INV_LOG=1 in the environment: one line per kernel launch of the build / WY / fused calls on stderr (host side only).
+bool log_enabled() {
+  static const bool on = [] { const char* v = getenv("TRI_INV_LOG"); return v && *v && *v != '0'; }();
+  return on;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -137,6 +145,10 @@ int run(KParams p, const tri_inv_desc* d, void* stream_v) {
   }
 
   if ((long long)p.n_chunks * d->H > 0x7fffffffLL) return TRI_INV_ERR_INVALID_ARG;  // kernels index work items in 32 bits
+  if (log_enabled())
+    fprintf(stderr, "[tri_inv] launch: B=%d T=%d H=%d d_k=%d d_v=%d C=%d dtype=%s %s, %d chunks x %d heads, method=0x%x ops=0x%x stream=%p\n",
+            d->B, d->T, d->H, d->d_k, d->d_v, d->C, d->kv_dtype == TRI_INV_BF16 ? "bf16" : "f32", d->cu_seqlens ? "packed" : "dense",
+            p.n_chunks, d->H, p.method, p.ops, stream_v);
   bool handled = false;
   err = cudaSuccess;
   // Newton-Schulz exists on the fp32 CUDA-core kernel only; so does refinement with the per-channel decay
@@ -150,6 +162,7 @@ int run(KParams p, const tri_inv_desc* d, void* stream_v) {
   if (err == cudaSuccess && !handled) err = launch_simt(p, d->C, stream);
   if (err == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);
   if (dev_tab) cudaFreeAsync(dev_tab, stream);
+  if (log_enabled()) fprintf(stderr, "[tri_inv]   -> %s kernel, %s\n", handled ? "tensor-core" : "CUDA-core", cudaGetErrorString(err));
   return err == cudaSuccess ? TRI_INV_OK : TRI_INV_ERR_CUDA;
 }
 

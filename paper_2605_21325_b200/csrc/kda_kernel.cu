@@ -81,7 +81,16 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid
   const uint32_t tmem = *tmem_slot;
   const uint32_t tmem_rows = tmem + ((32u * warp) << 16);
   uint32_t ph = 0, ph_mma = 0;   // K and G complete once per item: one parity for both
-  bool failed = misaligned;
+  // Give-up protocol as in the main kernel: a thread whose bounded wait runs out remembers it, skips its later waits and
+  // finishes the item on whatever data is there; it raises the CTA's flag before the item's last barrier, behind which
+  // every thread reads it, so the whole CTA leaves the loop at one place.
+  __shared__ int s_gave_up;
+  bool bad = false;
+  auto wait = [&](uint32_t bar, uint32_t parity) {
+    if (!bad) bad = !mbar_wait_bounded(bar, parity, p.wait_limit_ns);
+  };
+  if (tid == 0) s_gave_up = 0;   // read only behind later barriers
+  bool k_pending = false;        // thread 64: a K tile has been requested that nobody has waited for yet
 
   for (int item = blockIdx.x; item < total && !misaligned; item += gridDim.x) {
     int tok0, rows, h;
@@ -99,7 +108,8 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid
     }
 
     // ---- 2. K+ = K * 2^x over K, K- = K * 2^-x, x = (G - G_ref) log2(e); rows past the chunk's end are zero
-    if (!mbar_wait_bounded(bar_k, ph) || !mbar_wait_bounded(bar_g, ph)) { failed = true; break; }
+    wait(bar_k, ph);
+    wait(bar_g, ph);
     const int rref = rows >> 1;
 #pragma unroll
     for (int m = 0; m < 8; ++m) {
@@ -149,10 +159,11 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid
       }
       umma_commit(bar_mma);
     }
-    if (!mbar_wait_bounded(bar_mma, ph_mma)) { failed = true; break; }
+    wait(bar_mma, ph_mma);
     ph_mma ^= 1;
     tc_fence_after();
-    if (tid == 64 && has_next) issue_k(nx_tok0, nx_h);  // the operands' only reader has completed
+    k_pending = false;
+    if (tid == 64 && has_next && !bad) { issue_k(nx_tok0, nx_h); k_pending = true; }  // the operands' only reader has completed
     if (has_next) beta_next = fetch_beta(nx_tok0, nx_rows, nx_h);
 
     // ---- 4. gate (beta_i, strict-lower mask), N -> shared memory over the G tile (all of G has been consumed)
@@ -197,12 +208,18 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid
         if (i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
       }
     }
+    if (bad) s_gave_up = 1;
     tc_fence_before();
     __syncthreads();   // the fp32 matrix has been read by everyone: the next G tile may land in its space
+    if (s_gave_up) break;   // uniform: every thread reads the flag behind the same barrier
     ph ^= 1;
     if (tid == 96 && has_next) issue_g(nx_tok0, nx_h);
   }
-  if (failed) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+  if (bad || misaligned) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+  if (s_gave_up) {
+    // what may still be in flight: the K tile requested for the next item (the G tile is requested after the exit test)
+    if (tid == 64 && k_pending) mbar_wait_bounded(bar_k, ph ^ 1, p.wait_limit_ns);
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
@@ -210,7 +227,7 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid
 
 }  // namespace
 
-// G rides in KParams::V (an fp32 [B,T,H,d_k] tensor).  Handles bf16 keys with d_k = 128 at C = 64 and the
+// G is KParams::G (an fp32 [B,T,H,d_k] tensor).  Handles bf16 keys with d_k = 128 at C = 64 and the
 // block recursion; anything else is left to the CUDA-core kernel.
 cudaError_t launch_kda_tc(const KParams& p, int Cc, cudaStream_t stream, bool* handled) {
   *handled = false;
