@@ -319,14 +319,14 @@ int tri_inv_fused_kda(const void* K, const void* V, const float* G, const float*
   const bool tc = !(method & (TRI_INV_FORCE_SIMT | TRI_INV_REFINE)) && (method & TRI_INV_METHOD_MASK) == TRI_INV_BLOCK_RECURSIVE &&
                   desc->kv_dtype == TRI_INV_BF16 && desc->d_k == 128 && desc->d_v == 128 && desc->C == 64;
   if (tc) {
-    // Tensor-core route, three launches on the stream: A by the per-channel build kernel; K' = K * exp(G) into the W
-    // buffer; W = A diag(beta) K' and U = A diag(beta) V by the WY kernel, which reads each K' tile whole into shared
-    // memory before it writes the same rows of W.
-    if ((rc = tri_inv_build_kda(K, G, beta, A, desc, method, cuda_stream))) return rc;
-    const long long tokens = desc->cu_seqlens ? (long long)desc->T : (long long)desc->T * desc->B;
-    if (launch_kda_scale_keys(K, G, W, tokens * desc->H * desc->d_k, desc->kv_dtype, (cudaStream_t)cuda_stream) != cudaSuccess)
-      return TRI_INV_ERR_CUDA;
-    count_launch();
+    // Tensor-core route, two launches on the stream: the per-channel build kernel, which also writes K' = K * exp(G) into
+    // the W buffer while it has K and G in shared memory; then W = A diag(beta) K' and U = A diag(beta) V by the WY kernel,
+    // which reads each K' tile whole into shared memory before it writes the same rows of W.
+    KParams p{};
+    p.K = K; p.G = G; p.beta = beta; p.g = nullptr; p.A = A; p.W = W;
+    p.method = method;
+    p.ops = kStoreA | kKda;
+    if ((rc = run(p, desc, cuda_stream))) return rc;
     return tri_inv_wy(A, W, V, beta, W, U, desc, cuda_stream);
   }
   KParams p{};

@@ -121,9 +121,6 @@ cudaError_t launch_chunk_scan_simt(const ScanParams& p, const void* Q, const voi
 // Per-channel decay variant on the tensor cores (bf16 keys, d_k = 128, C = 64, block recursion).
 cudaError_t launch_kda_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
 
-// out = K * exp(G) element by element in the storage type of K (per-channel fused call; kda_ops.cu).
-cudaError_t launch_kda_scale_keys(const void* K, const float* G, void* out, long long n, int kv_dtype, cudaStream_t stream);
-
 // Fills dev_tab (one entry per chunk of tokens, in sequence order) from the host offsets in d->cu_seqlens
 // with small kernels on the stream; no copy and no synchronisation.
 cudaError_t launch_chunk_table(ChunkEntry* dev_tab, const tri_inv_desc* d, cudaStream_t stream);

@@ -31,6 +31,7 @@ constexpr int TMEM_COLS = 64;
 constexpr int CTAS_PER_SM = 3;
 static_assert(OFF_LEAF + NW * 16 * LEAF_LD * 4 <= OFF_BETA, "leaf scratch must fit behind the fp32 matrix");
 
+template <bool KG>   // KG: also write K * exp(G) into p.W (the fused call)
 __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                      const __grid_constant__ CUtensorMap tmG, KParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -134,12 +135,17 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid
         uint32_t* pw = reinterpret_cast<uint32_t*>(&kp);
         uint32_t* mw = reinterpret_cast<uint32_t*>(&km);
 #pragma unroll
+        uint4 kg;                                         // K * exp(G): the key operand of the WY step that follows (fused call)
+        uint32_t* gw = reinterpret_cast<uint32_t*>(&kg);
         for (int q = 0; q < 4; ++q) {
           const float2 kf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kw[q]));
           const float x0 = (gv[2 * q] - gr[2 * q]) * 1.4426950408889634f, x1 = (gv[2 * q + 1] - gr[2 * q + 1]) * 1.4426950408889634f;
           pw[q] = pack_bf16(kf.x * ex2_approx(x0), kf.y * ex2_approx(x1));
           mw[q] = pack_bf16(kf.x * ex2_approx(-x0), kf.y * ex2_approx(-x1));
+          if constexpr (KG) gw[q] = pack_bf16(kf.x * ex2_approx(gv[2 * q] * 1.4426950408889634f), kf.y * ex2_approx(gv[2 * q + 1] * 1.4426950408889634f));
         }
+        // 16 consecutive threads cover the 256 contiguous bytes of one token's keys of this head
+        if constexpr (KG) *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.W) + ((size_t)(tok0 + r) * p.H + h) * D + 8 * cf) = kg;
       }
       asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sK + koff), "r"(kp.x), "r"(kp.y), "r"(kp.z), "r"(kp.w) : "memory");
       asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + koff), "r"(km.x), "r"(km.y), "r"(km.z), "r"(km.w) : "memory");
@@ -244,8 +250,10 @@ cudaError_t launch_kda_tc(const KParams& p, int Cc, cudaStream_t stream, bool* h
   {
     std::lock_guard<std::mutex> lock(mu);
     if (!n_sm_of[dev]) {
-      if ((e = cudaFuncSetAttribute(kda_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) != cudaSuccess) return e;
-      if ((e = cudaFuncSetAttribute(kda_build_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(kda_build_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(kda_build_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(kda_build_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(kda_build_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
       int sms = 0, smem_per_sm = 0;
       if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
       if ((e = cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev)) != cudaSuccess) return e;
@@ -263,7 +271,8 @@ cudaError_t launch_kda_tc(const KParams& p, int Cc, cudaStream_t stream, bool* h
   if (!make_tmap(&tmG, p.G, tokens, p.H, D, C, 4)) return cudaErrorUnknown;
   long long total = (long long)p.n_chunks * p.H, cap = (long long)n_sm * ctas;
   int grid = (int)(total < cap ? total : cap);
-  kda_build_kernel<<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
+  if (p.W) kda_build_kernel<true><<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
+  else kda_build_kernel<false><<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
   return cudaGetLastError();
 }
 
