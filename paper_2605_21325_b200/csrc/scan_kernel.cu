@@ -42,23 +42,27 @@ struct ScanCfg {
   static constexpr int OFF_KA = OFF_B + 2 * B_BOX;       // K tile for P3 (MN-major A); its second box doubles as the
   static constexpr int OFF_P = OFF_KA + 16384;           // unused upper half of PU's A operand, P being the lower half
   static constexpr int OFF_UT = OFF_P + 8192;            // U~  bf16 [64 tokens][DVS], boxes of 64 columns (MN-major B)
-  static constexpr int U_BYTES = (DVS / 64) * 8192;
+  static constexpr int U_BYTES = 8192 * (DVS > 64 ? DVS / 64 : 1);   // a narrower slice fills the first DVS columns of one box
   static constexpr int OFF_UD = OFF_UT + U_BYTES;        // U~' bf16, same layout
   static constexpr int OFF_G = OFF_UD + U_BYTES;         // g * log2(e): 2 x 64 floats; column factors: 2 x 64 floats
   static constexpr int OFF_BAR = OFF_G + 1024;           // 9 mbarriers, tensor-memory slot
   static constexpr int SMEM = OFF_BAR + 96;
   static constexpr int TM_P1 = 0, TM_DS = N1, TM_PU = N1 + DVS;
   static constexpr int TMEM_COLS = (N1 + 2 * DVS) <= 256 ? 256 : 512;
-  static constexpr int CTAS_PER_SM = 1;   // registers: 9 warps at the kernel's natural register count fill an SM once
+  // DVS = 64: 9 warps at the kernel's natural register count fill an SM once.  DVS = 32 halves the state and the
+  // operand registers, and two CTAs (99 KiB of shared memory and 256 tensor-memory columns each) share an SM.
+  static constexpr int CTAS_PER_SM = DVS <= 32 ? 2 : 1;
 };
 
 template <int NTL>
 __device__ __forceinline__ void tmem_ld_frag(float (&r)[NTL][4], uint32_t taddr) {
   if constexpr (NTL == 8) tmem_ld_16x64(r, taddr);
-  else tmem_ld_16x32(r, taddr);
+  else if constexpr (NTL == 4) tmem_ld_16x32(r, taddr);
+  else tmem_ld_16x16(r, taddr);
 }
 template <int NTL>
 __device__ __forceinline__ void tmem_st_frag(const float (&r)[NTL][4], uint32_t taddr) {
+  if constexpr (NTL == 2) { tmem_st_16x16(r, taddr); return; }
 #pragma unroll
   for (int b = 0; b < NTL; b += 4) {
     const float q[4][4] = {{r[b][0], r[b][1], r[b][2], r[b][3]}, {r[b + 1][0], r[b + 1][1], r[b + 1][2], r[b + 1][3]},
@@ -504,11 +508,18 @@ cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t
 
 // bf16 Q, K, W, U with d_k = d_v = 128 and C = 64: two CTAs per (sequence, head), 64 value columns each.  (One CTA
 // per head with 128 columns was measured too: the same time per unit of work, at a register count that spills.)
+// A launch whose (sequence, head) pairs would leave three quarters of the SMs idle takes four CTAs of 32 columns
+// per pair instead, still at most one per SM: the per-chunk chain of a CTA is a little shorter (7 % on one sequence
+// of 32 heads), and every output column is computed by the same operations in the same order either way.  With more
+// pairs than that the narrow slices would share SMs and repeat the Q K^T part of the first product: measured slower.
 cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,
                               cudaStream_t stream) {
   CUtensorMap tmW, tmQ, tmK;
   if (!make_tmap(&tmW, W, tokens, p.H, D, C, 2) || !make_tmap(&tmQ, Q, tokens, p.H, D, C, 2) || !make_tmap(&tmK, K, tokens, p.H, D, C, 2))
     return cudaErrorUnknown;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
+  if ((long long)p.n_seqs * p.H * 4 <= sms) return launch_scan_one<32>(p, tmW, tmQ, tmK, stream);
   return launch_scan_one<64>(p, tmW, tmQ, tmK, stream);
 }
 

@@ -470,6 +470,12 @@ __device__ __forceinline__ void tmem_ld_16x32(float (&r)[4][4], uint32_t taddr) 
         "=f"(r[2][0]), "=f"(r[2][1]), "=f"(r[2][2]), "=f"(r[2][3]), "=f"(r[3][0]), "=f"(r[3][1]), "=f"(r[3][2]), "=f"(r[3][3])
       : "r"(taddr));
 }
+// 16 lanes x 16 columns -> 2 n-tiles of accumulator fragments.
+__device__ __forceinline__ void tmem_ld_16x16(float (&r)[2][4], uint32_t taddr) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=f"(r[0][0]), "=f"(r[0][1]), "=f"(r[0][2]), "=f"(r[0][3]), "=f"(r[1][0]), "=f"(r[1][1]), "=f"(r[1][2]), "=f"(r[1][3])
+               : "r"(taddr));
+}
 // 16 lanes x 128 columns -> 16 n-tiles of accumulator fragments.
 __device__ __forceinline__ void tmem_ld_16x128(float (&r)[16][4], uint32_t taddr) {
   asm volatile(
@@ -495,6 +501,11 @@ __device__ __forceinline__ void tmem_st_16x32(const float (&r)[4][4], uint32_t t
         "f"(r[2][0]), "f"(r[2][1]), "f"(r[2][2]), "f"(r[2][3]), "f"(r[3][0]), "f"(r[3][1]), "f"(r[3][2]), "f"(r[3][3]),
         "r"(taddr)
       : "memory");
+}
+__device__ __forceinline__ void tmem_st_16x16(const float (&r)[2][4], uint32_t taddr) {
+  asm volatile("tcgen05.st.sync.aligned.16x256b.x2.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
+               ::"f"(r[0][0]), "f"(r[0][1]), "f"(r[0][2]), "f"(r[0][3]), "f"(r[1][0]), "f"(r[1][1]), "f"(r[1][2]), "f"(r[1][3]), "r"(taddr)
+               : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void stmatrix_x4(uint32_t addr, uint32_t m0, uint32_t m1, uint32_t m2, uint32_t m3) {

@@ -46,6 +46,9 @@ CASES = [
     ("dense_partial_s0", 1, 3 * 64 + 17, 2, None, True),
     ("ragged_s0", 1, 0, 2, np.array([0, 64, 65, 65, 300, 531], np.int32), True),
     ("many_heads", 5, 2 * 64, 64, None, True),   # 640 CTAs: several per SM in turn
+    # few (sequence, head) pairs run as four CTAs of 32 value columns per pair, more as two of 64: both sides of the switch
+    ("pairs_36", 2, 3 * 64 + 9, 18, None, True),
+    ("pairs_40", 2, 3 * 64 + 9, 20, None, True),
 ]
 
 
