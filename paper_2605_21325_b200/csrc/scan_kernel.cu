@@ -27,6 +27,14 @@
 namespace tri_inv {
 namespace {
 
+// Development build only: the clock of one chunk's steps, per warp, in the device status words (a snapshot that the
+// development tools read back); nothing otherwise.
+#ifdef TRI_INV_PHASE_CLOCKS
+#define TL(k) do { if (blockIdx.x == 0 && c == 20 && lane == 0) p.status[8 + 12 * warp + (k)] = (int)clock64(); } while (0)
+#else
+#define TL(k) do {} while (0)
+#endif
+
 constexpr int C = 64, D = 128, NT = 256;   // NT compute threads (8 warps) + one control warp
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -44,14 +52,15 @@ struct ScanCfg {
   static constexpr int OFF_UT = OFF_P + 8192;            // U~  bf16 [64 tokens][DVS], boxes of 64 columns (MN-major B)
   static constexpr int U_BYTES = 8192 * (DVS > 64 ? DVS / 64 : 1);   // a narrower slice fills the first DVS columns of one box
   static constexpr int OFF_UD = OFF_UT + U_BYTES;        // U~' bf16, same layout
-  static constexpr int OFF_G = OFF_UD + U_BYTES;         // g * log2(e): 2 x 64 floats; column factors: 2 x 64 floats
-  static constexpr int OFF_BAR = OFF_G + 1024;           // 9 mbarriers, tensor-memory slot
+  static constexpr int OFF_U = OFF_UD + U_BYTES;         // U tiles of two chunks in turn: bf16 [64 tokens][64 columns], as copied
+  static constexpr int OFF_G = OFF_U + 2 * 8192;         // g * log2(e): 2 x 64 floats; column factors: 2 x 64 floats
+  static constexpr int OFF_BAR = OFF_G + 1024;           // 11 mbarriers, tensor-memory slot
   static constexpr int SMEM = OFF_BAR + 96;
   static constexpr int TM_P1 = 0, TM_DS = N1, TM_PU = N1 + DVS;
   static constexpr int TMEM_COLS = (N1 + 2 * DVS) <= 256 ? 256 : 512;
-  // DVS = 64: 9 warps at the kernel's natural register count fill an SM once.  DVS = 32 halves the state and the
-  // operand registers, and two CTAs (99 KiB of shared memory and 256 tensor-memory columns each) share an SM.
-  static constexpr int CTAS_PER_SM = DVS <= 32 ? 2 : 1;
+  // 9 warps at the kernel's natural register count fill an SM once (the narrow slice is only launched when its
+  // CTAs get an SM each).
+  static constexpr int CTAS_PER_SM = 1;
 };
 
 template <int NTL>
@@ -62,9 +71,9 @@ __device__ __forceinline__ void tmem_ld_frag(float (&r)[NTL][4], uint32_t taddr)
 }
 template <int NTL>
 __device__ __forceinline__ void tmem_st_frag(const float (&r)[NTL][4], uint32_t taddr) {
-  if constexpr (NTL == 2) { tmem_st_16x16(r, taddr); return; }
+  if constexpr (NTL == 2) tmem_st_16x16(r, taddr);
 #pragma unroll
-  for (int b = 0; b < NTL; b += 4) {
+  for (int b = 0; b + 4 <= NTL; b += 4) {
     const float q[4][4] = {{r[b][0], r[b][1], r[b][2], r[b][3]}, {r[b + 1][0], r[b + 1][1], r[b + 1][2], r[b + 1][3]},
                            {r[b + 2][0], r[b + 2][1], r[b + 2][2], r[b + 2][3]}, {r[b + 3][0], r[b + 3][1], r[b + 3][2], r[b + 3][3]}};
     tmem_st_16x32(q, taddr + 8 * b);
@@ -72,6 +81,16 @@ __device__ __forceinline__ void tmem_st_frag(const float (&r)[NTL][4], uint32_t 
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// One arrival for the whole warp: every lane has made its operand writes visible to the async proxy (the caller's
+// fences) before the lanes meet; lane 0 then arrives for all of them.  Eight arrivals per hand-off instead of 256
+// on one shared-memory word.
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& m0, uint32_t& m1, uint32_t& m2, uint32_t& m3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(m0), "=r"(m1), "=r"(m2), "=r"(m3) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void stmatrix_x4_trans(uint32_t addr, uint32_t m0, uint32_t m1, uint32_t m2, uint32_t m3) {
   asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(m0), "r"(m1), "r"(m2), "r"(m3) : "memory");
@@ -82,9 +101,9 @@ __host__ __device__ constexpr uint32_t umma_idesc_ab(int M, int N, int a_mn, int
 }
 
 template <int DVS>
-__global__ void __launch_bounds__(NT + 32, ScanCfg<DVS>::CTAS_PER_SM)
+__global__ void __launch_bounds__(NT + 64, ScanCfg<DVS>::CTAS_PER_SM)
 chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmQ,
-                  const __grid_constant__ CUtensorMap tmK, ScanParams p) {
+                  const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmU, ScanParams p) {
   using cfg = ScanCfg<DVS>;
   constexpr int NTW = cfg::NTW, CW = cfg::CW, NS = D / DVS;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -93,13 +112,18 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 80);
   const uint32_t sA = smem_u32(smem + cfg::OFF_A), sB = smem_u32(smem + cfg::OFF_B), sKa = smem_u32(smem + cfg::OFF_KA);
   const uint32_t sP = smem_u32(smem + cfg::OFF_P), sUt = smem_u32(smem + cfg::OFF_UT), sUd = smem_u32(smem + cfg::OFF_UD);
-  // copies (TMA):            bar_a (W and Q), bar_kb (K beside S^T), bar_ka (K for P3)
+  const uint32_t sU = smem_u32(smem + cfg::OFF_U);
+  // copies (TMA):            bar_a (W and Q), bar_kb (K beside S^T), bar_ka (K for P3), bar_u0 / bar_u1 (U, chunks in turn)
   // products done (commit):  bar_t1 (P1), bar_s (P3), bar_pu (PU)
-  // operands written:        bar_sr (S^T, all NT compute threads), bar_ut (U~ and U~', chain warps), bar_p (P, output warps)
+  // operands written:        bar_sr (S^T by the compute warps, the next chunk's g by the gate warp), bar_ut (U~ and U~',
+  //                          chain warps), bar_p (P, output warps); one arrival per warp
   const uint32_t bar_a = smem_u32(smem + cfg::OFF_BAR), bar_kb = bar_a + 8, bar_ka = bar_a + 16, bar_t1 = bar_a + 24,
-                 bar_s = bar_a + 32, bar_pu = bar_a + 40, bar_sr = bar_a + 48, bar_ut = bar_a + 56, bar_p = bar_a + 64;
+                 bar_s = bar_a + 32, bar_pu = bar_a + 40, bar_sr = bar_a + 48, bar_ut = bar_a + 56, bar_p = bar_a + 64,
+                 bar_u0 = bar_a + 72, bar_u1 = bar_a + 88;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool control = warp == 8;
+  const bool gate_warp = warp == 9;              // brings g of the chunks to come into shared memory
+  const bool compute = warp < 8;
   const int quad = warp & 3, half = (warp >> 2) & 1;
   const bool chain = quad < 2;                   // lanes 0..63 of P1 hold W S
   const int gq = lane >> 2, t = lane & 3;
@@ -116,7 +140,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   // State in accumulator-fragment layout: lane group lg (rows krow_w + 16 lg + gq and + 8), n-tile nt
   // (columns cw0 + 8 nt + 2 t and + 1):  S[lg][nt][0..3] = (row, col), (row, col+1), (row+8, col), (row+8, col+1).
   float S[2][NTW][4];
-  if (!control) {
+  if (compute) {
 #pragma unroll
     for (int lg = 0; lg < 2; ++lg)
 #pragma unroll
@@ -132,7 +156,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       }
   }
   auto store_state = [&]() {
-    if (!p.S_out || control) return;
+    if (!p.S_out || !compute) return;
     float* dst = p.S_out + ((size_t)s * p.H + h) * D * D;
 #pragma unroll
     for (int lg = 0; lg < 2; ++lg)
@@ -179,61 +203,62 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     tma_load_2d(sKa, &tmK, bar_ka, h * D, tok0);
     tma_load_2d(sKa + 8192, &tmK, bar_ka, h * D + 64, tok0);
   };
-  // U of the chain warps in fragment layout: u[lg][nt][0] = row tok_w + 16 lg + gq, [1] = that row + 8 (bf16 pairs)
-  const __nv_bfloat16* Ug = reinterpret_cast<const __nv_bfloat16*>(p.U);
-  auto fetch_u = [&](uint32_t (&u)[2][NTW][2], int tok0, int rows) {
-#pragma unroll
-    for (int lg = 0; lg < 2; ++lg)
-#pragma unroll
-      for (int nt = 0; nt < NTW; ++nt) {
-        const int i = tok_w + 16 * lg + gq, cidx = col0 + 8 * nt + 2 * t;
-        u[lg][nt][0] = i < rows ? *reinterpret_cast<const uint32_t*>(Ug + ((size_t)(tok0 + i) * p.H + h) * D + cidx) : 0u;
-        u[lg][nt][1] = i + 8 < rows ? *reinterpret_cast<const uint32_t*>(Ug + ((size_t)(tok0 + i + 8) * p.H + h) * D + cidx) : 0u;
-      }
+  // U of chunk c: the 64-column box that holds this CTA's slice, into the buffer of c's parity
+  auto issue_u = [&](int c) {
+    const uint32_t bar = (c & 1) ? bar_u1 : bar_u0;
+    mbar_expect_tx(bar, 8192u);
+    tma_load_2d(sU + (c & 1) * 8192, &tmU, bar, h * D + (slice * DVS) / 64 * 64, beg + c * C);
   };
-  // rows past the sequence end take the last real row's g, so that every exponent stays a difference of real values
-  auto fetch_g = [&](int tok0, int rows) -> float {
-    const int i = tid < rows ? tid : rows - 1;
-    return tid < C ? p.g[(size_t)(tok0 + i) * p.H + h] : 0.f;   // raw: scaled where it is stored, not where it is loaded
+  // g of a chunk, by the gate warp (lane l: tokens l and l + 32).  Rows past the sequence end take the last real
+  // row's g, so that every exponent stays a difference of real values.
+  auto fetch_g = [&](int c, float (&gr)[2]) {
+    const int tok0 = beg + c * C, rows = end - tok0 < C ? end - tok0 : C;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int i = lane + 32 * q < rows ? lane + 32 * q : rows - 1;
+      gr[q] = p.g[(size_t)(tok0 + i) * p.H + h];
+    }
   };
   // g * log2(e) of a chunk and its column factors: the decay 2^(g_i - g_j) of P is formed as
   // 2^(g_i - g_ref) * 2^(g_ref - g_j) with g_ref the first token of j's block of eight -- one exponential per
   // (row, block) instead of one per element; the second factor spans at most seven tokens of decay
-  auto store_g = [&](int buf, float g_raw) {
-    const float gl2 = g_raw * kLog2e;
-    const float gref = __shfl_sync(0xffffffffu, gl2, lane & ~7);
-    sG[buf * C + tid] = gl2;
-    sCf[buf * C + tid] = ex2_approx(gref - gl2);
+  auto store_g = [&](int buf, const float (&gr)[2]) {
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const float gl2 = gr[q] * kLog2e;
+      const float gref = __shfl_sync(0xffffffffu, gl2, lane & ~7);
+      sG[buf * C + lane + 32 * q] = gl2;
+      sCf[buf * C + lane + 32 * q] = ex2_approx(gref - gl2);
+    }
   };
 
-  uint32_t xr[2][NTW][2];   // chain warps: the next chunk's U (bf16 pairs)
-  float g_next = 0.f;
-  {
-    const int rows0 = end - beg < C ? end - beg : C;
-    if (tid == NT) {
-      prefetch_tmap(&tmW); prefetch_tmap(&tmQ); prefetch_tmap(&tmK);
-      for (int b = 0; b < 6; ++b) mbar_init(bar_a + 8 * b, 1);
-      mbar_init(bar_sr, NT);
-      mbar_init(bar_ut, NT / 2);
-      mbar_init(bar_p, NT / 2);
-      fence_mbar_init();
-      if (!misaligned) {
-        issue_wq(beg);
-        issue_kb(beg);
-        issue_ka(beg);
-      }
+  float g_raw[2] = {0.f, 0.f};   // gate warp: g of the chunk it stores next
+  if (tid == NT) {
+    prefetch_tmap(&tmW); prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmU);
+    for (int b = 0; b < 6; ++b) mbar_init(bar_a + 8 * b, 1);
+    mbar_init(bar_u0, 1);
+    mbar_init(bar_u1, 1);
+    mbar_init(bar_sr, NT / 32 + 1);   // one arrival per warp (lane 0, after the warp's lanes have fenced and met); the gate warp too
+    mbar_init(bar_ut, NT / 64);
+    mbar_init(bar_p, NT / 64);
+    fence_mbar_init();
+    if (!misaligned) {
+      issue_wq(beg);
+      issue_kb(beg);
+      issue_ka(beg);
+      issue_u(0);
     }
-    if (!control && chain) fetch_u(xr, beg, rows0);
-    if (!control) g_next = fetch_g(beg, rows0);
+  }
+  if (gate_warp) {
+    fetch_g(0, g_raw);
+    store_g(0, g_raw);
+    if (n_chunks > 1) fetch_g(1, g_raw);
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(cfg::TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (!control) {
-    write_state_operand();
-    if (tid < C) store_g(0, g_next);
-  }
+  if (compute) write_state_operand();
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();   // barriers initialised, tensor memory allocated, first operand of S and first g in place
@@ -257,29 +282,64 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         // the copies land long before the compute threads are done: check them first, S last
         if (!mbar_wait_bounded(bar_a, ph) || !mbar_wait_bounded(bar_kb, ph) || !mbar_wait_bounded(bar_sr, ph)) { failed = true; break; }
         tc_fence_after();
+        TL(0);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
           umma_bf16(tmem + cfg::TM_P1, dA + (((ks >> 2) * cfg::A_BOX + (ks & 3) * 32) >> 4),
                     dB + (((ks >> 2) * cfg::B_BOX + (ks & 3) * 32) >> 4), idesc_p1, ks > 0);
         umma_commit(bar_t1);
+        TL(1);
+        // Refills, from this thread so that no compute warp spends issue slots on them.  Products retire in issue
+        // order: PU of the last chunk (the last reader of the K tile of P3) before P1 of this one, whose commit
+        // frees W, Q and the K beside S^T.  Both waits end long before U~ is ready, the next thing this thread needs.
+        // (U of the next chunk: its buffer was last read for the chunk before this one, which every compute warp left
+        // before its arrival on bar_sr, seen above)
+        if (c + 1 < n_chunks) issue_u(c + 1);
+        if (c > 0) {
+          if (!mbar_wait_bounded(bar_pu, ph ^ 1)) { failed = true; break; }
+          issue_ka(beg + c * C);
+        }
+        if (!mbar_wait_bounded(bar_t1, ph)) { failed = true; break; }
+        TL(2);
+        if (c + 1 < n_chunks) {
+          issue_wq(beg + (c + 1) * C);
+          issue_kb(beg + (c + 1) * C);
+        }
         if (!mbar_wait_bounded(bar_ka, ph) || !mbar_wait_bounded(bar_ut, ph)) { failed = true; break; }
         tc_fence_after();
+        TL(3);
 #pragma unroll
         for (int ks = 0; ks < C / 16; ++ks)   // 16 tokens (2048 bytes of either operand) per step
           umma_bf16(tmem + cfg::TM_DS, dKa + ((ks * 2048) >> 4), dUd + ((ks * 2048) >> 4), idesc_p3, ks > 0);
         umma_commit(bar_s);
+        TL(4);
         if (!mbar_wait_bounded(bar_p, ph)) { failed = true; break; }
         tc_fence_after();
+        TL(5);
 #pragma unroll
         for (int ks = 0; ks < C / 16; ++ks)
           umma_bf16(tmem + cfg::TM_PU, dPa + ((ks * 32) >> 4), dUt + ((ks * 2048) >> 4), idesc_pu, 1u);   // on top of gamma_i Q S
         umma_commit(bar_pu);
+        TL(6);
         ph ^= 1;
       }
     }
+  } else if (gate_warp) {
+    // ---------------------------------------------------------------- gate warp: g of chunk c + 1, during chunk c
+    // Its arrival on bar_sr tells the control thread, and through the first product's commit every reader, that
+    // the chunk's g is in place.  The global loads run a chunk ahead of their use, in a warp that waits for nothing
+    // else: a compute warp with a global load in flight would also wait for it at its next tensor-memory load.
+    warp_arrive(bar_sr, lane);   // g of the first chunk (written before the CTA barrier above)
+    for (int c = 0; c + 1 < n_chunks && !misaligned; ++c) {
+      // the buffer of c + 1 held g of c - 1: every compute warp has left that chunk once the arrivals that end it are in
+      if (c > 0 && !mbar_wait_bounded(bar_sr, (uint32_t)(c & 1))) { failed = true; break; }
+      store_g((c + 1) & 1, g_raw);
+      warp_arrive(bar_sr, lane);
+      if (c + 2 < n_chunks) fetch_g(c + 2, g_raw);
+    }
   } else {
     // ---------------------------------------------------------------- compute warps
-    mbar_arrive(bar_sr);   // the first S^T operand (written before the CTA barrier above)
+    warp_arrive(bar_sr, lane);   // the first S^T operand (written before the CTA barrier above)
     uint32_t ph = 0;
     int o_tok0 = 0, o_rows = 0;
     // O = scale * (gamma_i QS + P U~) of the previous chunk (the PU accumulator starts from gamma_i QS): written
@@ -288,21 +348,22 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       if (!mbar_wait_bounded(bar_pu, parity)) return false;
       tc_fence_after();
       __nv_bfloat16* Og = reinterpret_cast<__nv_bfloat16*>(p.O);
+      float pu[2][NTW][4];
+      tmem_ld_frag<NTW>(pu[0], tmem_w + cfg::TM_PU + cw0);
+      tmem_ld_frag<NTW>(pu[1], tmem_w + (16u << 16) + cfg::TM_PU + cw0);
+      tmem_wait_ld();
 #pragma unroll
       for (int lg = 0; lg < 2; ++lg) {
-        float pu[NTW][4];
-        tmem_ld_frag<NTW>(pu, tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_PU + cw0);
-        tmem_wait_ld();
         const int i = tok_w + 16 * lg + gq;
 #pragma unroll
         for (int nt = 0; nt < NTW; ++nt) {
           const int cc = col0 + 8 * nt + 2 * t;
           if (i < o_rows)
             *reinterpret_cast<uint32_t*>(Og + ((size_t)(o_tok0 + i) * p.H + h) * D + cc) =
-                pack_bf16(p.scale * pu[nt][0], p.scale * pu[nt][1]);
+                pack_bf16(p.scale * pu[lg][nt][0], p.scale * pu[lg][nt][1]);
           if (i + 8 < o_rows)
             *reinterpret_cast<uint32_t*>(Og + ((size_t)(o_tok0 + i + 8) * p.H + h) * D + cc) =
-                pack_bf16(p.scale * pu[nt][2], p.scale * pu[nt][3]);
+                pack_bf16(p.scale * pu[lg][nt][2], p.scale * pu[lg][nt][3]);
         }
       }
       tc_fence_before();
@@ -312,40 +373,35 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       const int tok0 = beg + c * C;
       const int rows = end - tok0 < C ? end - tok0 : C;
       const bool has_next = c + 1 < n_chunks;
-      const int nx_tok0 = tok0 + C, nx_rows = end - nx_tok0 < C ? end - nx_tok0 : C;
       const float* gb = sG + (c & 1) * C;
-      PHASE_BEGIN();
-      if (has_next) g_next = fetch_g(nx_tok0, nx_rows);
-      if (chain && has_next && t == 0) {
-        // next chunk's U rows of this thread into L2 now; the loads into registers follow when this chunk's U is used up
-#pragma unroll
-        for (int rr = 0; rr < 4; ++rr) {
-          const int i = tok_w + 8 * rr + gq;
-          if (i < nx_rows) asm volatile("prefetch.global.L2 [%0];" ::"l"(Ug + ((size_t)(nx_tok0 + i) * p.H + h) * D + col0));
-        }
-      }
+      TL(0);
       if (!chain && c > 0) {
         if (!write_output(ph ^ 1)) { failed = true; break; }
-        if (tid == 64) issue_ka(tok0);   // PU of the last chunk, the last reader of that buffer, has retired
       }
-      PHASE(0);
+      TL(1);
 
       if (!mbar_wait_bounded(bar_t1, ph)) { failed = true; break; }
       tc_fence_after();
-      PHASE(1);
-      if (has_next && tid == 32) issue_wq(nx_tok0);    // P1, the only reader of W, Q and of the K beside S^T, has retired
-      if (has_next && tid == 96) issue_kb(nx_tok0);
-      // (this chunk's g was written by other threads during the last chunk: read only after the wait above,
-      // which follows every compute thread's arrival on bar_sr)
+      TL(2);
+      // (this chunk's g was written by the gate warp during the last chunk: read only after the wait above,
+      // which follows that warp's arrival on bar_sr)
       const float g_last = gb[rows - 1];
       if (chain) {
         // ---- U~ = U - W S  ->  bf16 operands U~ and (decay-scaled) U~', [token rows][value columns]
         const int mi = lane >> 3, r = lane & 7;
+        if (!mbar_wait_bounded((c & 1) ? bar_u1 : bar_u0, (uint32_t)((c >> 1) & 1))) { failed = true; break; }   // landed a chunk ago
+        TL(3);
+        const uint32_t sUc = sU + (c & 1) * 8192;
+        constexpr int ucol0 = DVS < 64 ? 1 : 0;      // a narrow slice: which part of the copied 64-column box is ours
+        const int u_shift = ucol0 * ((slice * DVS) & 63);
+        float ws[2][NTW][4];
+        tmem_ld_frag<NTW>(ws[0], tmem_w + cfg::TM_P1 + cw0);
+        tmem_ld_frag<NTW>(ws[1], tmem_w + (16u << 16) + cfg::TM_P1 + cw0);
+        tmem_wait_ld();
+        TL(4);
 #pragma unroll
         for (int lg = 0; lg < 2; ++lg) {
-          float t1[NTW][4];
-          tmem_ld_frag<NTW>(t1, tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_P1 + cw0);
-          tmem_wait_ld();
+          const float (&t1)[NTW][4] = ws[lg];
           const int i = tok_w + 16 * lg + gq;
           const float da = ex2_approx(g_last - gb[i]), db = ex2_approx(g_last - gb[i + 8]);
           const bool va = i < rows, vb = i + 8 < rows;
@@ -353,98 +409,122 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
           const int tok = tok_w + 16 * lg + 8 * (mi & 1) + r;
 #pragma unroll
           for (int nt = 0; nt < NTW; nt += 2) {
+            const int n = cw0 + 8 * (nt + (mi >> 1));   // first column of this lane's matrix
+            const uint32_t off = (n >> 6) * 8192 + tok * 128 + ((((n & 63) >> 3) ^ (tok & 7)) << 4);
+            // U comes out of its tile the way U~ goes into its own: the same four 8 x 8 matrices per instruction
+            uint32_t xu[2][2];
+            ldmatrix_x4(sUc + tok * 128 + (((((n + u_shift) & 63) >> 3) ^ (tok & 7)) << 4), xu[0][0], xu[0][1], xu[1][0], xu[1][1]);
             float v[2][4];
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
-              const uint32_t wa = xr[lg][nt + q][0], wb = xr[lg][nt + q][1];   // bf16 pairs: low half = first column
+              const uint32_t wa = xu[q][0], wb = xu[q][1];   // bf16 pairs: low half = first column
               const float2 ua = make_float2(__uint_as_float(wa << 16), __uint_as_float(wa & 0xffff0000u));
               const float2 ub = make_float2(__uint_as_float(wb << 16), __uint_as_float(wb & 0xffff0000u));
               v[q][0] = va ? ua.x - t1[nt + q][0] : 0.f; v[q][1] = va ? ua.y - t1[nt + q][1] : 0.f;
               v[q][2] = vb ? ub.x - t1[nt + q][2] : 0.f; v[q][3] = vb ? ub.y - t1[nt + q][3] : 0.f;
             }
-            const int n = cw0 + 8 * (nt + (mi >> 1));   // first column of this lane's matrix
-            const uint32_t off = (n >> 6) * 8192 + tok * 128 + ((((n & 63) >> 3) ^ (tok & 7)) << 4);
             stmatrix_x4(sUt + off, pack_bf16(v[0][0], v[0][1]), pack_bf16(v[0][2], v[0][3]), pack_bf16(v[1][0], v[1][1]), pack_bf16(v[1][2], v[1][3]));
             stmatrix_x4(sUd + off, pack_bf16(v[0][0] * da, v[0][1] * da), pack_bf16(v[0][2] * db, v[0][3] * db),
                         pack_bf16(v[1][0] * da, v[1][1] * da), pack_bf16(v[1][2] * db, v[1][3] * db));
           }
         }
+        TL(5);
         fence_proxy_async();
         tc_fence_before();
-        mbar_arrive(bar_ut);
-        if (tid < C && has_next) store_g((c + 1) & 1, g_next);   // before new loads are issued: waiting for g must not wait for them
-        if (has_next) fetch_u(xr, nx_tok0, nx_rows);   // consumed one chunk from now
+        warp_arrive(bar_ut, lane);
+        TL(6);
       } else {
         // ---- P = (Q K^T) * decay, lower triangle with its diagonal; Q S kept for the output
         const float* cf = sCf + (c & 1) * C;
+        float qk[2][4][4];   // this warp's half of the columns (tokens j): four blocks of eight
+        float qsf[2][NTW][4];
 #pragma unroll
         for (int lg = 0; lg < 2; ++lg) {
-          float qk[4][4];   // this warp's half of the columns (tokens j): four blocks of eight
-          float qsf[NTW][4];
           const uint32_t trow = tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_P1;
-          tmem_ld_16x32(qk, trow + DVS + 32 * half);
-          tmem_ld_frag<NTW>(qsf, trow + cw0);
-          tmem_wait_ld();
+          tmem_ld_16x32(qk[lg], trow + DVS + 32 * half);
+          tmem_ld_frag<NTW>(qsf[lg], trow + cw0);
+        }
+        // what the blocks need from shared memory, while the loads above are in flight
+        float gref[4];
+        float2 cj[4];
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          gref[q4] = gb[8 * (4 * half + q4)];
+          cj[q4] = *reinterpret_cast<const float2*>(cf + 8 * (4 * half + q4) + 2 * t);
+        }
+        tmem_wait_ld();
+        TL(3);
+#pragma unroll
+        for (int lg = 0; lg < 2; ++lg) {
           const int ia = tok_w + 16 * lg + gq, ib = ia + 8;
           const float g_a = gb[ia], g_b = gb[ib];
           {
             // gamma_i Q S becomes the starting value of the PU accumulator (same lanes, same columns)
             const float ya = ex2_approx(g_a), yb = ex2_approx(g_b);
 #pragma unroll
-            for (int nt = 0; nt < NTW; ++nt) { qsf[nt][0] *= ya; qsf[nt][1] *= ya; qsf[nt][2] *= yb; qsf[nt][3] *= yb; }
-            tmem_st_frag<NTW>(qsf, tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_PU + cw0);
+            for (int nt = 0; nt < NTW; ++nt) { qsf[lg][nt][0] *= ya; qsf[lg][nt][1] *= ya; qsf[lg][nt][2] *= yb; qsf[lg][nt][3] *= yb; }
+            tmem_st_frag<NTW>(qsf[lg], tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_PU + cw0);
           }
+          // No branch around a block: entries right of a row's diagonal are masked by selection, and the exponent of
+          // a row that lies above the whole block is not formed (its argument is replaced by zero), so the four
+          // blocks are independent straight-line code that the scheduler can interleave.
+          uint32_t wa[4], wb[4];
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             const int nt = 4 * half + q4;
             const int j = 8 * nt + 2 * t;
-            uint32_t wa = 0u, wb = 0u;
-            if (8 * nt <= ib) {   // blocks right of both rows' diagonals are all zero
-              const float gref = gb[8 * nt];
-              const float2 cj = *reinterpret_cast<const float2*>(cf + j);
-              // (row a may lie above this block altogether: its entries are masked, the exponent is not formed)
-              const float ea = ex2_approx(8 * nt <= ia ? g_a - gref : 0.f), eb = ex2_approx(g_b - gref);
-              const float p0 = j <= ia ? qk[q4][0] * ea * cj.x : 0.f, p1 = j + 1 <= ia ? qk[q4][1] * ea * cj.y : 0.f;
-              const float p2 = j <= ib ? qk[q4][2] * eb * cj.x : 0.f, p3 = j + 1 <= ib ? qk[q4][3] * eb * cj.y : 0.f;
-              wa = pack_bf16(p0, p1);
-              wb = pack_bf16(p2, p3);
-            }
-            *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + ia * 128 + ((nt ^ (ia & 7)) << 4) + 4 * t) = wa;
-            *reinterpret_cast<uint32_t*>(smem + cfg::OFF_P + ib * 128 + ((nt ^ (ib & 7)) << 4) + 4 * t) = wb;
+            const float ea = ex2_approx(8 * nt <= ia ? g_a - gref[q4] : 0.f), eb = ex2_approx(8 * nt <= ib ? g_b - gref[q4] : 0.f);
+            const float p0 = j <= ia ? qk[lg][q4][0] * ea * cj[q4].x : 0.f, p1 = j + 1 <= ia ? qk[lg][q4][1] * ea * cj[q4].y : 0.f;
+            const float p2 = j <= ib ? qk[lg][q4][2] * eb * cj[q4].x : 0.f, p3 = j + 1 <= ib ? qk[lg][q4][3] * eb * cj[q4].y : 0.f;
+            wa[q4] = pack_bf16(p0, p1);
+            wb[q4] = pack_bf16(p2, p3);
           }
+          // into the K-major operand (row i, 16-byte pieces of eight tokens j, swizzled): two x4 stores of the matrices
+          // (rows +0..7, block), (rows +8..15, block), (rows +0..7, block + 1), (rows +8..15, block + 1)
+          {
+            const int mi = lane >> 3, row = tok_w + 16 * lg + 8 * (mi & 1) + (lane & 7);
+#pragma unroll
+            for (int q4 = 0; q4 < 4; q4 += 2) {
+              const int blk = 4 * half + q4 + (mi >> 1);
+              stmatrix_x4(sP + row * 128 + ((blk ^ (row & 7)) << 4), wa[q4], wb[q4], wa[q4 + 1], wb[q4 + 1]);
+            }
+          }
+          if (lg == 0) TL(5);
         }
         tmem_wait_st();
         fence_proxy_async();
         tc_fence_before();
-        mbar_arrive(bar_p);
+        warp_arrive(bar_p, lane);
+        TL(6);
         o_tok0 = tok0; o_rows = rows;
       }
-      PHASE(2);
 
       // ---- state update and the bf16 operand for the next chunk
       if (!mbar_wait_bounded(bar_s, ph)) { failed = true; break; }
       tc_fence_after();
-      PHASE(3);
+      TL(7);
       {
         const float gl = ex2_approx(g_last);
+        float ds[2][NTW][4];
+        tmem_ld_frag<NTW>(ds[0], tmem_w + cfg::TM_DS + cw0);
+        tmem_ld_frag<NTW>(ds[1], tmem_w + (16u << 16) + cfg::TM_DS + cw0);
+        tmem_wait_ld();
 #pragma unroll
-        for (int lg = 0; lg < 2; ++lg) {
-          float ds[NTW][4];
-          tmem_ld_frag<NTW>(ds, tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_DS + cw0);
-          tmem_wait_ld();
+        for (int lg = 0; lg < 2; ++lg)
 #pragma unroll
           for (int nt = 0; nt < NTW; ++nt)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) S[lg][nt][e] = fmaf(gl, S[lg][nt][e], ds[nt][e]);
-        }
+            for (int e = 0; e < 4; ++e) S[lg][nt][e] = fmaf(gl, S[lg][nt][e], ds[lg][nt][e]);
+        TL(8);
         if (has_next) {
           write_state_operand();   // its reader (P1 of this chunk) retired before bar_t1
+          TL(9);
           fence_proxy_async();
           tc_fence_before();
-          mbar_arrive(bar_sr);
+          warp_arrive(bar_sr, lane);
         }
       }
-      PHASE(4);
+      TL(10);
       ph ^= 1;
     }
     if (!chain && !failed && !misaligned && !write_output(ph ^ 1)) failed = true;
@@ -467,7 +547,7 @@ __global__ void __launch_bounds__(256) seq_offsets_kernel(int* out, const __grid
 
 template <int DVS>
 cudaError_t launch_scan_one(const ScanParams& p, const CUtensorMap& tmW, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                            cudaStream_t stream) {
+                            const CUtensorMap& tmU, cudaStream_t stream) {
   using cfg = ScanCfg<DVS>;
   static std::mutex mu;
   static bool ready[64] = {false};
@@ -485,7 +565,7 @@ cudaError_t launch_scan_one(const ScanParams& p, const CUtensorMap& tmW, const C
   }
   const long long grid = (long long)p.n_seqs * p.H * (D / DVS);
   if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
-  chunk_scan_kernel<DVS><<<(int)grid, NT + 32, cfg::SMEM, stream>>>(tmW, tmQ, tmK, p);
+  chunk_scan_kernel<DVS><<<(int)grid, NT + 64, cfg::SMEM, stream>>>(tmW, tmQ, tmK, tmU, p);
   return cudaGetLastError();
 }
 
@@ -514,13 +594,14 @@ cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t
 // pairs than that the narrow slices would share SMs and repeat the Q K^T part of the first product: measured slower.
 cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,
                               cudaStream_t stream) {
-  CUtensorMap tmW, tmQ, tmK;
-  if (!make_tmap(&tmW, W, tokens, p.H, D, C, 2) || !make_tmap(&tmQ, Q, tokens, p.H, D, C, 2) || !make_tmap(&tmK, K, tokens, p.H, D, C, 2))
+  CUtensorMap tmW, tmQ, tmK, tmU;
+  if (!make_tmap(&tmW, W, tokens, p.H, D, C, 2) || !make_tmap(&tmQ, Q, tokens, p.H, D, C, 2) || !make_tmap(&tmK, K, tokens, p.H, D, C, 2) ||
+      !make_tmap(&tmU, p.U, tokens, p.H, D, C, 2))
     return cudaErrorUnknown;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
-  if ((long long)p.n_seqs * p.H * 4 <= sms) return launch_scan_one<32>(p, tmW, tmQ, tmK, stream);
-  return launch_scan_one<64>(p, tmW, tmQ, tmK, stream);
+  if ((long long)p.n_seqs * p.H * 4 <= sms) return launch_scan_one<32>(p, tmW, tmQ, tmK, tmU, stream);
+  return launch_scan_one<64>(p, tmW, tmQ, tmK, tmU, stream);
 }
 
 }  // namespace tri_inv
