@@ -54,8 +54,8 @@ struct ScanCfg {
   static constexpr int OFF_UD = OFF_UT + U_BYTES;        // U~' bf16, same layout
   static constexpr int OFF_U = OFF_UD + U_BYTES;         // U tiles of two chunks in turn: bf16 [64 tokens][64 columns], as copied
   static constexpr int OFF_G = OFF_U + 2 * 8192;         // g * log2(e): 2 x 64 floats; column factors: 2 x 64 floats
-  static constexpr int OFF_BAR = OFF_G + 1024;           // 11 mbarriers, tensor-memory slot
-  static constexpr int SMEM = OFF_BAR + 96;
+  static constexpr int OFF_BAR = OFF_G + 1024;           // 12 mbarriers, tensor-memory slot
+  static constexpr int SMEM = OFF_BAR + 128;
   static constexpr int TM_P1 = 0, TM_DS = N1, TM_PU = N1 + DVS;
   static constexpr int TMEM_COLS = (N1 + 2 * DVS) <= 256 ? 256 : 512;
   // 9 warps at the kernel's natural register count fill an SM once (the narrow slice is only launched when its
@@ -119,7 +119,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   //                          chain warps), bar_p (P, output warps); one arrival per warp
   const uint32_t bar_a = smem_u32(smem + cfg::OFF_BAR), bar_kb = bar_a + 8, bar_ka = bar_a + 16, bar_t1 = bar_a + 24,
                  bar_s = bar_a + 32, bar_pu = bar_a + 40, bar_sr = bar_a + 48, bar_ut = bar_a + 56, bar_p = bar_a + 64,
-                 bar_u0 = bar_a + 72, bar_u1 = bar_a + 88;
+                 bar_u0 = bar_a + 72, bar_u1 = bar_a + 88, bar_ud = bar_a + 96;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool control = warp == 8;
   const bool gate_warp = warp == 9;              // brings g of the chunks to come into shared memory
@@ -239,6 +239,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     mbar_init(bar_u0, 1);
     mbar_init(bar_u1, 1);
     mbar_init(bar_sr, NT / 32 + 1);   // one arrival per warp (lane 0, after the warp's lanes have fenced and met); the gate warp too
+    mbar_init(bar_ud, NT / 64);
     mbar_init(bar_ut, NT / 64);
     mbar_init(bar_p, NT / 64);
     fence_mbar_init();
@@ -305,7 +306,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
           issue_wq(beg + (c + 1) * C);
           issue_kb(beg + (c + 1) * C);
         }
-        if (!mbar_wait_bounded(bar_ka, ph) || !mbar_wait_bounded(bar_ut, ph)) { failed = true; break; }
+        if (!mbar_wait_bounded(bar_ka, ph) || !mbar_wait_bounded(bar_ud, ph)) { failed = true; break; }
         tc_fence_after();
         TL(3);
 #pragma unroll
@@ -313,7 +314,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
           umma_bf16(tmem + cfg::TM_DS, dKa + ((ks * 2048) >> 4), dUd + ((ks * 2048) >> 4), idesc_p3, ks > 0);
         umma_commit(bar_s);
         TL(4);
-        if (!mbar_wait_bounded(bar_p, ph)) { failed = true; break; }
+        if (!mbar_wait_bounded(bar_ut, ph) || !mbar_wait_bounded(bar_p, ph)) { failed = true; break; }
         tc_fence_after();
         TL(5);
 #pragma unroll
@@ -387,50 +388,74 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       // which follows that warp's arrival on bar_sr)
       const float g_last = gb[rows - 1];
       if (chain) {
-        // ---- U~ = U - W S  ->  bf16 operands U~ and (decay-scaled) U~', [token rows][value columns]
+        // ---- U~ = U - W S  ->  bf16 operands [token rows][value columns]: first the decay-scaled U~' that the chain
+        // waits for (its own arrival), then U~ itself for the third product
         const int mi = lane >> 3, r = lane & 7;
         if (!mbar_wait_bounded((c & 1) ? bar_u1 : bar_u0, (uint32_t)((c >> 1) & 1))) { failed = true; break; }   // landed a chunk ago
         TL(3);
         const uint32_t sUc = sU + (c & 1) * 8192;
-        constexpr int ucol0 = DVS < 64 ? 1 : 0;      // a narrow slice: which part of the copied 64-column box is ours
-        const int u_shift = ucol0 * ((slice * DVS) & 63);
-        float ws[2][NTW][4];
-        tmem_ld_frag<NTW>(ws[0], tmem_w + cfg::TM_P1 + cw0);
-        tmem_ld_frag<NTW>(ws[1], tmem_w + (16u << 16) + cfg::TM_P1 + cw0);
-        tmem_wait_ld();
-        TL(4);
+        const int u_shift = DVS < 64 ? ((slice * DVS) & 63) : 0;   // a narrow slice: which part of the copied 64-column box is ours
+        float v[2][NTW][4];
+        tmem_ld_frag<NTW>(v[0], tmem_w + cfg::TM_P1 + cw0);
+        tmem_ld_frag<NTW>(v[1], tmem_w + (16u << 16) + cfg::TM_P1 + cw0);
+        // while those are in flight: U out of its tile the way U~ goes into its own (the same four 8 x 8 matrices per
+        // instruction: (tokens +0..7, tile nt), (tokens +8..15, tile nt), (+0..7, nt+1), (+8..15, nt+1)), and the decays
+        uint32_t xu[2][NTW][2], off[2][NTW / 2];
+        float da[2], db[2];
 #pragma unroll
         for (int lg = 0; lg < 2; ++lg) {
-          const float (&t1)[NTW][4] = ws[lg];
-          const int i = tok_w + 16 * lg + gq;
-          const float da = ex2_approx(g_last - gb[i]), db = ex2_approx(g_last - gb[i + 8]);
-          const bool va = i < rows, vb = i + 8 < rows;
-          // the x4 store: matrices (tokens +0..7, tile nt), (tokens +8..15, tile nt), (+0..7, nt+1), (+8..15, nt+1)
           const int tok = tok_w + 16 * lg + 8 * (mi & 1) + r;
 #pragma unroll
           for (int nt = 0; nt < NTW; nt += 2) {
             const int n = cw0 + 8 * (nt + (mi >> 1));   // first column of this lane's matrix
-            const uint32_t off = (n >> 6) * 8192 + tok * 128 + ((((n & 63) >> 3) ^ (tok & 7)) << 4);
-            // U comes out of its tile the way U~ goes into its own: the same four 8 x 8 matrices per instruction
-            uint32_t xu[2][2];
-            ldmatrix_x4(sUc + tok * 128 + (((((n + u_shift) & 63) >> 3) ^ (tok & 7)) << 4), xu[0][0], xu[0][1], xu[1][0], xu[1][1]);
-            float v[2][4];
+            off[lg][nt / 2] = (n >> 6) * 8192 + tok * 128 + ((((n & 63) >> 3) ^ (tok & 7)) << 4);
+            ldmatrix_x4(sUc + tok * 128 + (((((n + u_shift) & 63) >> 3) ^ (tok & 7)) << 4), xu[lg][nt][0], xu[lg][nt][1], xu[lg][nt + 1][0], xu[lg][nt + 1][1]);
+          }
+          const int i = tok_w + 16 * lg + gq;
+          da[lg] = ex2_approx(g_last - gb[i]);
+          db[lg] = ex2_approx(g_last - gb[i + 8]);
+        }
+        tmem_wait_ld();
+        TL(4);
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              const uint32_t wa = xu[q][0], wb = xu[q][1];   // bf16 pairs: low half = first column
-              const float2 ua = make_float2(__uint_as_float(wa << 16), __uint_as_float(wa & 0xffff0000u));
-              const float2 ub = make_float2(__uint_as_float(wb << 16), __uint_as_float(wb & 0xffff0000u));
-              v[q][0] = va ? ua.x - t1[nt + q][0] : 0.f; v[q][1] = va ? ua.y - t1[nt + q][1] : 0.f;
-              v[q][2] = vb ? ub.x - t1[nt + q][2] : 0.f; v[q][3] = vb ? ub.y - t1[nt + q][3] : 0.f;
+        for (int lg = 0; lg < 2; ++lg)
+#pragma unroll
+          for (int nt = 0; nt < NTW; ++nt) {
+            const uint32_t wa = xu[lg][nt][0], wb = xu[lg][nt][1];   // bf16 pairs: low half = first column
+            v[lg][nt][0] = __uint_as_float(wa << 16) - v[lg][nt][0];
+            v[lg][nt][1] = __uint_as_float(wa & 0xffff0000u) - v[lg][nt][1];
+            v[lg][nt][2] = __uint_as_float(wb << 16) - v[lg][nt][2];
+            v[lg][nt][3] = __uint_as_float(wb & 0xffff0000u) - v[lg][nt][3];
+          }
+        if (rows < C) {   // rows past the sequence end count as zero
+#pragma unroll
+          for (int lg = 0; lg < 2; ++lg) {
+            const int i = tok_w + 16 * lg + gq;
+            const bool va = i < rows, vb = i + 8 < rows;
+#pragma unroll
+            for (int nt = 0; nt < NTW; ++nt) {
+              v[lg][nt][0] = va ? v[lg][nt][0] : 0.f; v[lg][nt][1] = va ? v[lg][nt][1] : 0.f;
+              v[lg][nt][2] = vb ? v[lg][nt][2] : 0.f; v[lg][nt][3] = vb ? v[lg][nt][3] : 0.f;
             }
-            stmatrix_x4(sUt + off, pack_bf16(v[0][0], v[0][1]), pack_bf16(v[0][2], v[0][3]), pack_bf16(v[1][0], v[1][1]), pack_bf16(v[1][2], v[1][3]));
-            stmatrix_x4(sUd + off, pack_bf16(v[0][0] * da, v[0][1] * da), pack_bf16(v[0][2] * db, v[0][3] * db),
-                        pack_bf16(v[1][0] * da, v[1][1] * da), pack_bf16(v[1][2] * db, v[1][3] * db));
           }
         }
-        TL(5);
+#pragma unroll
+        for (int lg = 0; lg < 2; ++lg)
+#pragma unroll
+          for (int nt = 0; nt < NTW; nt += 2)
+            stmatrix_x4(sUd + off[lg][nt / 2], pack_bf16(v[lg][nt][0] * da[lg], v[lg][nt][1] * da[lg]), pack_bf16(v[lg][nt][2] * db[lg], v[lg][nt][3] * db[lg]),
+                        pack_bf16(v[lg][nt + 1][0] * da[lg], v[lg][nt + 1][1] * da[lg]), pack_bf16(v[lg][nt + 1][2] * db[lg], v[lg][nt + 1][3] * db[lg]));
         fence_proxy_async();
         tc_fence_before();
+        warp_arrive(bar_ud, lane);
+        TL(5);
+#pragma unroll
+        for (int lg = 0; lg < 2; ++lg)
+#pragma unroll
+          for (int nt = 0; nt < NTW; nt += 2)
+            stmatrix_x4(sUt + off[lg][nt / 2], pack_bf16(v[lg][nt][0], v[lg][nt][1]), pack_bf16(v[lg][nt][2], v[lg][nt][3]),
+                        pack_bf16(v[lg][nt + 1][0], v[lg][nt + 1][1]), pack_bf16(v[lg][nt + 1][2], v[lg][nt + 1][3]));
+        fence_proxy_async();
         warp_arrive(bar_ut, lane);
         TL(6);
       } else {
