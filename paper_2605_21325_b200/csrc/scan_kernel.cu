@@ -43,12 +43,14 @@ struct ScanCfg {
   static constexpr int CW = DVS / 2;                     // value columns per compute warp
   static constexpr int NTW = CW / 8;                     // accumulator n-tiles per compute warp
   static constexpr int N1 = DVS + 64;                    // columns of P1
+  // Both operands of P1 exist twice, used by the chunks in turn, so that a chunk's copies can start a whole chunk
+  // before its first product (a copy that misses L2 takes most of a chunk's time).
   // A operand of P1: [W ; Q], two boxes (64 features each) of 128 rows x 128 B
-  static constexpr int OFF_A = 0, A_BOX = 16384;
+  static constexpr int OFF_A = 0, A_BOX = 16384, A_TILE = 2 * A_BOX;
   // B operand of P1: [S^T ; K], two boxes of (DVS + 64) rows x 128 B
-  static constexpr int OFF_B = 32768, B_BOX = N1 * 128;
-  static constexpr int OFF_KA = OFF_B + 2 * B_BOX;       // K tile for P3 (MN-major A); its second box doubles as the
-  static constexpr int OFF_P = OFF_KA + 16384;           // unused upper half of PU's A operand, P being the lower half
+  static constexpr int OFF_B = 2 * A_TILE, B_BOX = N1 * 128, B_TILE = 2 * B_BOX;
+  // (the K rows of the B tile are also the MN-major A operand of P3: the tile stays whole until the chunk after next)
+  static constexpr int OFF_P = OFF_B + 2 * B_TILE;       // P, the lower half of PU's A operand; the unused upper half is whatever precedes it
   static constexpr int OFF_UT = OFF_P + 8192;            // U~  bf16 [64 tokens][DVS], boxes of 64 columns (MN-major B)
   static constexpr int U_BYTES = 8192 * (DVS > 64 ? DVS / 64 : 1);   // a narrower slice fills the first DVS columns of one box
   static constexpr int OFF_UD = OFF_UT + U_BYTES;        // U~' bf16, same layout
@@ -110,10 +112,10 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   float* sG = reinterpret_cast<float*>(smem + cfg::OFF_G);
   float* sCf = sG + 2 * C;   // 2^(g_ref(j) - g_j), g_ref(j) = g of the first token of j's block of eight
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 80);
-  const uint32_t sA = smem_u32(smem + cfg::OFF_A), sB = smem_u32(smem + cfg::OFF_B), sKa = smem_u32(smem + cfg::OFF_KA);
+  const uint32_t sA = smem_u32(smem + cfg::OFF_A), sB = smem_u32(smem + cfg::OFF_B);
   const uint32_t sP = smem_u32(smem + cfg::OFF_P), sUt = smem_u32(smem + cfg::OFF_UT), sUd = smem_u32(smem + cfg::OFF_UD);
   const uint32_t sU = smem_u32(smem + cfg::OFF_U);
-  // copies (TMA):            bar_a (W and Q), bar_kb (K beside S^T), bar_ka (K for P3), bar_u0 / bar_u1 (U, chunks in turn)
+  // copies (TMA):            bar_a (W and Q), bar_kb (K beside S^T), bar_u0 / bar_u1 (U, chunks in turn)
   // products done (commit):  bar_t1 (P1), bar_s (P3), bar_pu (PU)
   // operands written:        bar_sr (S^T by the compute warps, the next chunk's g by the gate warp), bar_ut (U~ and U~',
   //                          chain warps), bar_p (P, output warps); one arrival per warp
@@ -172,7 +174,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 
   // S^T as rows 0..DVS-1 of the K-major B operand of P1: row n = value column, 16-byte pieces of eight key features.
   // stmatrix.trans turns the fragments (rows = features, column pairs) into exactly those pieces.
-  auto write_state_operand = [&]() {
+  auto write_state_operand = [&](int buf) {
     const int mi = lane >> 3, r = lane & 7;      // this lane addresses row r of matrix mi of each x4 store
 #pragma unroll
     for (int lg = 0; lg < 2; ++lg)
@@ -181,27 +183,27 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         // matrices: (features +0..7, tile nt), (features +8..15, tile nt), (+0..7, nt+1), (+8..15, nt+1)
         const int k0 = krow_w + 16 * lg + 8 * (mi & 1);          // first feature of this lane's matrix
         const int n = cw0 + 8 * (nt + (mi >> 1)) + r;            // row of the operand
-        const uint32_t addr = sB + (k0 >> 6) * cfg::B_BOX + n * 128 + ((((k0 & 63) >> 3) ^ (n & 7)) << 4);
+        const uint32_t addr = sB + buf * cfg::B_TILE + (k0 >> 6) * cfg::B_BOX + n * 128 + ((((k0 & 63) >> 3) ^ (n & 7)) << 4);
         stmatrix_x4_trans(addr, pack_bf16(S[lg][nt][0], S[lg][nt][1]), pack_bf16(S[lg][nt][2], S[lg][nt][3]),
                           pack_bf16(S[lg][nt + 1][0], S[lg][nt + 1][1]), pack_bf16(S[lg][nt + 1][2], S[lg][nt + 1][3]));
       }
   };
-  auto issue_wq = [&](int tok0) {
+  // W, Q and the K beside S^T of chunk c, into the tiles of c's parity
+  auto issue_wq = [&](int c) {
+    const uint32_t dst = sA + (c & 1) * cfg::A_TILE;
+    const int tok0 = beg + c * C;
     mbar_expect_tx(bar_a, 32768u);
-    tma_load_2d(sA, &tmW, bar_a, h * D, tok0);
-    tma_load_2d(sA + 8192, &tmQ, bar_a, h * D, tok0);
-    tma_load_2d(sA + cfg::A_BOX, &tmW, bar_a, h * D + 64, tok0);
-    tma_load_2d(sA + cfg::A_BOX + 8192, &tmQ, bar_a, h * D + 64, tok0);
+    tma_load_2d(dst, &tmW, bar_a, h * D, tok0);
+    tma_load_2d(dst + 8192, &tmQ, bar_a, h * D, tok0);
+    tma_load_2d(dst + cfg::A_BOX, &tmW, bar_a, h * D + 64, tok0);
+    tma_load_2d(dst + cfg::A_BOX + 8192, &tmQ, bar_a, h * D + 64, tok0);
   };
-  auto issue_kb = [&](int tok0) {
+  auto issue_kb = [&](int c) {
+    const uint32_t dst = sB + (c & 1) * cfg::B_TILE + DVS * 128;
+    const int tok0 = beg + c * C;
     mbar_expect_tx(bar_kb, 16384u);
-    tma_load_2d(sB + DVS * 128, &tmK, bar_kb, h * D, tok0);
-    tma_load_2d(sB + cfg::B_BOX + DVS * 128, &tmK, bar_kb, h * D + 64, tok0);
-  };
-  auto issue_ka = [&](int tok0) {
-    mbar_expect_tx(bar_ka, 16384u);
-    tma_load_2d(sKa, &tmK, bar_ka, h * D, tok0);
-    tma_load_2d(sKa + 8192, &tmK, bar_ka, h * D + 64, tok0);
+    tma_load_2d(dst, &tmK, bar_kb, h * D, tok0);
+    tma_load_2d(dst + cfg::B_BOX, &tmK, bar_kb, h * D + 64, tok0);
   };
   // U of chunk c: the 64-column box that holds this CTA's slice, into the buffer of c's parity
   auto issue_u = [&](int c) {
@@ -244,9 +246,8 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     mbar_init(bar_p, NT / 64);
     fence_mbar_init();
     if (!misaligned) {
-      issue_wq(beg);
-      issue_kb(beg);
-      issue_ka(beg);
+      issue_wq(0);
+      issue_kb(0);
       issue_u(0);
     }
   }
@@ -259,7 +260,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(cfg::TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (compute) write_state_operand();
+  if (compute) write_state_operand(0);
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();   // barriers initialised, tensor memory allocated, first operand of S and first g in place
@@ -275,43 +276,41 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       constexpr uint32_t idesc_p3 = umma_idesc_ab(128, DVS, 1, 1);       // K tile MN-major, U~' MN-major
       constexpr uint32_t idesc_pu = umma_idesc_ab(128, DVS, 0, 1);       // [any;P] K-major, U~ MN-major
       // descriptors differ from these bases only in the address field (bits 0..13, units of 16 bytes)
-      const uint64_t dA = umma_desc(sA, 16, 1024), dB = umma_desc(sB, 16, 1024), dKa = umma_desc(sKa, 8192, 1024),
+      const uint64_t dA = umma_desc(sA, 16, 1024), dB = umma_desc(sB, 16, 1024), dKa = umma_desc(sB + DVS * 128, cfg::B_BOX, 1024),   // the K rows of the B tile, MN-major
                      dUd = umma_desc(sUd, 8192, 1024), dUt = umma_desc(sUt, 8192, 1024),
-                     dPa = umma_desc(sKa + 8192, 16, 1024);              // 128 rows: second K box, then P
+                     dPa = umma_desc(sP - 8192, 16, 1024);               // 128 rows: 64 of whatever lies before P (results unused), then P
       uint32_t ph = 0;
       for (int c = 0; c < n_chunks; ++c) {
         // the copies land long before the compute threads are done: check them first, S last
-        if (!mbar_wait_bounded(bar_a, ph) || !mbar_wait_bounded(bar_kb, ph) || !mbar_wait_bounded(bar_sr, ph)) { failed = true; break; }
+        TL(9);
+        if (!mbar_wait_bounded(bar_a, ph)) { failed = true; break; }
+        TL(7);
+        if (!mbar_wait_bounded(bar_kb, ph)) { failed = true; break; }
+        TL(8);
+        if (!mbar_wait_bounded(bar_sr, ph)) { failed = true; break; }
         tc_fence_after();
         TL(0);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
-          umma_bf16(tmem + cfg::TM_P1, dA + (((ks >> 2) * cfg::A_BOX + (ks & 3) * 32) >> 4),
-                    dB + (((ks >> 2) * cfg::B_BOX + (ks & 3) * 32) >> 4), idesc_p1, ks > 0);
+          umma_bf16(tmem + cfg::TM_P1, dA + (((c & 1) * cfg::A_TILE + (ks >> 2) * cfg::A_BOX + (ks & 3) * 32) >> 4),
+                    dB + (((c & 1) * cfg::B_TILE + (ks >> 2) * cfg::B_BOX + (ks & 3) * 32) >> 4), idesc_p1, ks > 0);
         umma_commit(bar_t1);
         TL(1);
-        // Refills, from this thread so that no compute warp spends issue slots on them.  Products retire in issue
-        // order: PU of the last chunk (the last reader of the K tile of P3) before P1 of this one, whose commit
-        // frees W, Q and the K beside S^T.  Both waits end long before U~ is ready, the next thing this thread needs.
-        // (U of the next chunk: its buffer was last read for the chunk before this one, which every compute warp left
-        // before its arrival on bar_sr, seen above)
-        if (c + 1 < n_chunks) issue_u(c + 1);
-        if (c > 0) {
-          if (!mbar_wait_bounded(bar_pu, ph ^ 1)) { failed = true; break; }
-          issue_ka(beg + c * C);
-        }
-        if (!mbar_wait_bounded(bar_t1, ph)) { failed = true; break; }
-        TL(2);
+        // Copies for the next chunk, from this thread so that no compute warp spends issue slots on them.  They go
+        // into the other tiles, whose last readers (P1 and P3 of the chunk before this one; for U the chain warps, a
+        // chunk ago) were done before the arrivals on bar_sr seen above: nothing to wait for.
         if (c + 1 < n_chunks) {
-          issue_wq(beg + (c + 1) * C);
-          issue_kb(beg + (c + 1) * C);
+          issue_u(c + 1);
+          issue_kb(c + 1);
+          issue_wq(c + 1);
         }
-        if (!mbar_wait_bounded(bar_ka, ph) || !mbar_wait_bounded(bar_ud, ph)) { failed = true; break; }
+        TL(2);
+        if (!mbar_wait_bounded(bar_ud, ph)) { failed = true; break; }
         tc_fence_after();
         TL(3);
 #pragma unroll
         for (int ks = 0; ks < C / 16; ++ks)   // 16 tokens (2048 bytes of either operand) per step
-          umma_bf16(tmem + cfg::TM_DS, dKa + ((ks * 2048) >> 4), dUd + ((ks * 2048) >> 4), idesc_p3, ks > 0);
+          umma_bf16(tmem + cfg::TM_DS, dKa + (((c & 1) * cfg::B_TILE + ks * 2048) >> 4), dUd + ((ks * 2048) >> 4), idesc_p3, ks > 0);
         umma_commit(bar_s);
         TL(4);
         if (!mbar_wait_bounded(bar_ut, ph) || !mbar_wait_bounded(bar_p, ph)) { failed = true; break; }
@@ -542,7 +541,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             for (int e = 0; e < 4; ++e) S[lg][nt][e] = fmaf(gl, S[lg][nt][e], ds[lg][nt][e]);
         TL(8);
         if (has_next) {
-          write_state_operand();   // its reader (P1 of this chunk) retired before bar_t1
+          write_state_operand((c + 1) & 1);   // that tile's last reader was P1 of the chunk before this one
           TL(9);
           fence_proxy_async();
           tc_fence_before();
