@@ -14,13 +14,17 @@
 //   P1 [128 x (DVS+64)] = [W ; Q] . [S | K^T]     rows 0..63: W S (and W K^T, unused); rows 64..127: Q S | Q K^T
 //   P3 [128 x DVS]      = K^T . U~'               U~' = decay-scaled U~ (bf16); the K tile is read MN-major
 //   PU [128 x DVS]      = [any ; P] . U~          rows 64..127 = P U~, on the lanes that also hold Q S
-// The dependent chain of a chunk is  P1 -> U~ -> P3 -> S.  Warp 8 holds the one thread that issues every product;
-// warps 0..7 compute.  Warp w works on tensor-memory lanes 32 (w & 3) .. +31 and on half (w >> 2) of the value
-// columns; lanes 0..63 carry W S, so warps of quadrants 0 and 1 form U~ ("chain warps"), those of quadrants 2
-// and 3 form P and the output ("output warps"); all eight update their part of S.  Hand-offs are mbarriers:
-// commits from the products, counted arrivals from the compute threads after their operand writes.
-// TMA brings W, Q and K (K twice: once beside S^T as the B operand of P1, once as the A operand of P3, so that
-// each copy is refilled as early as its own reader allows); U and g come through registers one chunk ahead.
+// The dependent chain of a chunk is  P1 -> U~' -> P3 -> S.  Warp 8 holds the one thread that issues every product
+// and every tile copy; warp 9 brings g; warps 0..7 compute.  Warp w works on tensor-memory lanes 32 (w & 3) .. +31
+// and on half (w >> 2) of the value columns; lanes 0..63 carry W S, so warps of quadrants 0 and 1 form U~' and U~
+// ("chain warps"), those of quadrants 2 and 3 form P and the output ("output warps"); all eight update their
+// part of S.  Hand-offs are mbarriers: commits from the products, one arrival per warp after its operand writes
+// (U~' first: the second product, on the chain, needs only that; U~, for the third, follows).
+// TMA brings W, Q, K and U.  Both operands of P1 ([W ; Q] and [S^T ; K]) exist twice and are used by the chunks in
+// turn: a chunk's copies are issued a whole chunk before its first product (a copy that misses L2 takes most of a
+// chunk's time), and the K rows of the B tile stay in place to serve as the MN-major A operand of P3.  g is loaded
+// by a warp of its own a chunk ahead, because a compute warp with a global load in flight would also wait for it at
+// its next tensor-memory load.
 // Every mbarrier wait is bounded; on expiry the CTA raises the status word, frees its tensor memory and returns.
 #include "tc_device.cuh"
 
@@ -35,7 +39,7 @@ namespace {
 #define TL(k) do {} while (0)
 #endif
 
-constexpr int C = 64, D = 128, NT = 256;   // NT compute threads (8 warps) + one control warp
+constexpr int C = 64, D = 128, NT = 256;   // NT compute threads (8 warps) + the control warp + the gate warp
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int DVS>

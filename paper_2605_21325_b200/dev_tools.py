@@ -3,8 +3,9 @@
 
     python -m paper_2605_21325_b200.dev_tools phases   [--config 2]     cycles between the kernel's phase marks, per warp of CTA 0
     python -m paper_2605_21325_b200.dev_tools timeline [--config 2]     when each CTA ran its first / last instruction, and on which SM
+    python -m paper_2605_21325_b200.dev_tools scan_chunk [--config 2]   clock of every step of one chunk of the chunk scan, per warp of CTA 0
 
-Both run the fused call of one configuration a few times on cuda:0.  The development build's TRI_INV_GRID_CAP=<n>
+The first two run the fused call of one configuration a few times on cuda:0, the third the chunk scan.  The development build's TRI_INV_GRID_CAP=<n>
 environment variable caps the grid (to vary the resident CTAs per SM).
 """
 from __future__ import annotations
@@ -27,11 +28,13 @@ def main():
     import torch
     from paper_2605_21325_b200 import binding as b, workloads as wl
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["phases", "timeline"])
+    ap.add_argument("what", choices=["phases", "timeline", "scan_chunk"])
     ap.add_argument("--config", type=int, default=2)
     args = ap.parse_args()
     inp = wl.config(args.config)
     d = b.to_device(inp)
+    if args.what == "scan_chunk":
+        return scan_chunk(b, wl, inp, d)
     out = (torch.empty((inp.B, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda"), torch.empty_like(d["K"]), torch.empty_like(d["V"]))
     L = b.load()
     if not hasattr(L, "tri_inv_debug_counters"):
@@ -63,6 +66,39 @@ def main():
     print("first instruction of a CTA, us after the first: min %.1f median %.1f max %.1f" % (start.min(), np.median(start), start.max()))
     print("last instruction of a CTA: min %.1f median %.1f max %.1f" % (end.min(), np.median(end), end.max()))
     print("SMs by number of CTAs they ran:", np.bincount(np.bincount(sm.astype(int))).tolist())
+
+
+SCAN_COMPUTE = ["loop top", "last chunk's O written", "P1 seen", "chain: U tile seen | output: P loads done", "chain: W S loaded",
+                "chain: U~' arrived | output: first 16 rows of P", "chain: U~ arrived | output: P arrived", "P3 seen", "state updated",
+                "S^T stored", "S^T arrived"]
+SCAN_CONTROL = ["state operand seen", "P1 issued", "copies issued", "U~' seen", "P3 issued", "U~ and P seen", "PU issued", "W/Q copy seen",
+                "K copy seen", "loop top"]
+
+
+def scan_chunk(b, wl, inp, d):
+    """The development build stamps clock64 at every step of the 21st chunk of CTA 0 (macro TL in scan_kernel.cu);
+    printed here in cycles from the moment the control thread sees that chunk's state operand."""
+    import numpy as np
+    import torch
+    Q = b.kv_to_torch(wl.queries(inp, seed=1))
+    W = torch.randn_like(d["K"].float()).mul_(0.1).to(torch.bfloat16)
+    U = d["V"].clone()
+    O = torch.empty_like(d["V"])
+    L = b.load()
+    if not hasattr(L, "tri_inv_debug_counters"):
+        raise SystemExit("%s is not a development build" % b.LIB_PATH)
+    words = (ctypes.c_int * 128)()
+    for _ in range(3):
+        L.tri_inv_debug_counters(words)
+        b.chunk_scan(Q, d["K"], W, U, d["g"], inp.C, scale=0.1, cu_seqlens=inp.cu_seqlens, out=O, want_state=False)
+        torch.cuda.synchronize()
+    L.tri_inv_debug_counters(words)
+    w = np.array(words[:], dtype=np.int64)[8:].reshape(10, 12)
+    base = w[8, 0]
+    for i in range(8):
+        role = "chain " if (i & 3) < 2 else "output"
+        print("warp %d (%s): " % (i, role) + ", ".join("%s %d" % (n, w[i, k] - base) for k, n in enumerate(SCAN_COMPUTE) if w[i, k]))
+    print("control thread: " + ", ".join("%s %d" % (n, w[8, k] - base) for k, n in enumerate(SCAN_CONTROL) if w[8, k]))
 
 
 if __name__ == "__main__":
