@@ -317,7 +317,7 @@ int tri_inv_fused_kda(const void* K, const void* V, const float* G, const float*
     return TRI_INV_ERR_INVALID_ARG;
   if ((rc = check_method(method, false, false))) return rc;
   const bool tc = !(method & (TRI_INV_FORCE_SIMT | TRI_INV_REFINE)) && (method & TRI_INV_METHOD_MASK) == TRI_INV_BLOCK_RECURSIVE &&
-                  desc->kv_dtype == TRI_INV_BF16 && desc->d_k == 128 && desc->d_v == 128 && desc->C == 64;
+                  desc->kv_dtype == TRI_INV_BF16 && desc->d_k == 128 && desc->d_v == 128 && (desc->C == 64 || desc->C == 128);
   if (tc) {
     // Tensor-core route, two launches on the stream: the per-channel build kernel, which also writes K' = K * exp(G) into
     // the W buffer while it has K and G in shared memory; then W = A diag(beta) K' and U = A diag(beta) V by the WY kernel,

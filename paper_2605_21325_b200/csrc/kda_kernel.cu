@@ -233,13 +233,14 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid
 
 }  // namespace
 
-// G is KParams::G (an fp32 [B,T,H,d_k] tensor).  Handles bf16 keys with d_k = 128 at C = 64 and the
-// block recursion; anything else is left to the CUDA-core kernel.
+// G is KParams::G (an fp32 [B,T,H,d_k] tensor).  Handles bf16 keys with d_k = 128 at C = 64 (here) and C = 128
+// (kda_kernel_c128.cu) and the block recursion; anything else is left to the CUDA-core kernel.
 cudaError_t launch_kda_tc(const KParams& p, int Cc, cudaStream_t stream, bool* handled) {
   *handled = false;
-  if (p.kv_dtype != TRI_INV_BF16 || p.d_k != 128 || Cc != 64) return cudaSuccess;
+  if (p.kv_dtype != TRI_INV_BF16 || p.d_k != 128 || (Cc != 64 && Cc != 128)) return cudaSuccess;
   if ((p.method & TRI_INV_METHOD_MASK) != TRI_INV_BLOCK_RECURSIVE) return cudaSuccess;
   *handled = true;
+  if (Cc == 128) return launch_kda_tc_c128(p, stream);
   static std::mutex mu;
   static int n_sm_of[64] = {0}, ctas_of[64] = {0};
   int dev = 0;

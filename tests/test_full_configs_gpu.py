@@ -171,12 +171,14 @@ def test_adversarial_keys_report(bnd):
     print("adversarial keys, max ratio per method:", report)
 
 
-def test_per_channel_decay_full_size_config2_shape(bnd):
-    """tri_inv_fused_kda on the shape of config 2 (4096 matrices, the launches bench.py --call kda_fused times): structure on
-    every element, EVERY matrix's A, W and U against the fp64 oracle, and -- at any size -- a gate that is the same on every
-    channel must reproduce tri_inv_build's matrices within the rounding of the two bf16 operand copies."""
-    inp = wl.config(2)
-    G = wl.per_channel_gate(inp, seed=3002)
+@pytest.mark.parametrize("cfg", [2, 4], ids=["config2_C64", "config4_C128"])
+def test_per_channel_decay_full_size(bnd, cfg):
+    """tri_inv_fused_kda on the shapes of config 2 (4096 matrices of 64 tokens) and config 4 (2048 of 128), the launches
+    bench.py --call kda_fused times: structure on every element, EVERY matrix's A, W and U against the fp64 oracle, and -- at
+    any size -- a gate that is the same on every channel must reproduce tri_inv_build's matrices within the rounding of the
+    two bf16 operand copies."""
+    inp = wl.config(cfg)
+    G = wl.per_channel_gate(inp, seed=3000 + cfg)
     dev = bnd.to_device(inp)
     Gd = torch.from_numpy(G).cuda()
     A = torch.full((inp.B, inp.T, inp.H, inp.C), float("nan"), dtype=torch.float32, device="cuda")
