@@ -176,8 +176,10 @@ int tri_inv_fused(const void* K, const void* V, const float* beta, const float* 
  *     N_ij = beta_i * sum_c K_ic K_jc exp(G_ic - G_jc)   (i > j),      A = (I + N)^{-1}
  * G [B,T,H,d_k] fp32 is the cumulative per-channel log-decay inside each chunk (only differences inside a
  * chunk are used).  Same layouts, chunking modes, methods and error codes as tri_inv_build.  On the tensor
- * cores (bf16 keys, d_k = 128, C = 64, block recursion) the two factors are formed around the chunk's middle
- * row, so |G_i - G_mid| log2(e) must stay inside the fp32 exponent range (about 88 in natural-log units);
+ * cores (bf16 keys, d_k = 128, C = 64 or 128, block recursion) the two factors are formed around a reference
+ * row -- the chunk's middle row at C = 64, the middle row of each half at C = 128 -- so |G_i - G_ref| log2(e)
+ * must stay inside the fp32 exponent range (about 88 in natural-log units), and at C = 128 G must not increase
+ * from the first half of a chunk to the middle of the second (a cumulative log-decay never does);
  * other shapes take the exponent of each difference directly.
  */
 int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A,
