@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 METRIC = "chunk matrices inverted/sec (C=64, d=128, bf16) + % of roofline; max err vs fp64 oracle"
 UNIT = "chunk-matrices/s"
 FALLBACK_HBM_GBS = 6650.0
-OUTPUTS = {"fused": "A fp32 + W,U", "raw": "A fp32 + W,U", "build": "A fp32", "kda": "A fp32", "kda_fused": "A fp32 + W,U", "wy": "W,U", "scan": "O", "layer": "O"}
+OUTPUTS = {"fused": "A fp32 + W,U", "raw": "A fp32 + W,U", "build": "A fp32", "kda": "A fp32", "kda_fused": "A fp32 + W,U", "wy": "W,U", "scan": "O", "layer": "O", "kda_scan": "O", "kda_layer": "O"}
 
 def ncu_traffic_bytes_per_matrix(call, config, method):
     """DRAM bytes per chunk matrix (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture divided by the matrices
@@ -53,6 +53,11 @@ def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True, call="fused"):
         return C * d_k * elt + 2 * C * 4 + C * C * 4
     if call == "scan":  # Q, K, W, U, g read; O written
         return 3 * C * d_k * elt + C * d_v * elt + C * 4 + C * d_v * elt
+    if call == "kda_scan":  # what ONE kernel would move: Q, K, W, U and G (fp32 per channel) read; O written (the call is two launches)
+        return 3 * C * d_k * elt + C * d_v * elt + C * d_k * 4 + C * d_v * elt
+    if call == "kda_layer":  # kda_fused without A, plus kda_scan
+        return (C * d_k * elt + C * d_k * 4 + C * d_v * elt + C * 4 + C * d_k * elt + C * d_v * elt) + \
+               (3 * C * d_k * elt + C * d_v * elt + C * d_k * 4 + C * d_v * elt)
     if call == "layer":  # fused kernel (K, V, beta, g in; W, U out, A not stored) + scan
         return (C * d_k * elt + C * d_v * elt + 2 * C * 4 + C * d_k * elt + C * d_v * elt) + \
                (3 * C * d_k * elt + C * d_v * elt + C * 4 + C * d_v * elt)
@@ -210,7 +215,7 @@ def main():
     ap.add_argument("--method", default="block_recursive", choices=["block_recursive", "mixed_recursion", "product_series", "block_recursive_refined", "product_series_f16"])
     ap.add_argument("--paper-T", type=int, default=0,
                     help="instead of --config: the paper's timing shape B=32, H=4, d=128 at this sequence length (1024..16384)")
-    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw", "kda", "kda_fused", "scan", "layer"],
+    ap.add_argument("--call", default="fused", choices=["fused", "build", "wy", "raw", "kda", "kda_fused", "scan", "layer", "kda_scan", "kda_layer"],
                     help="entry point timed: the fused path (default, the metric), tri_inv_build alone, tri_inv_wy alone, "
                          "tri_inv_fused_raw (front end folded in; same shapes, un-normalised keys and logits as inputs), "
                          "tri_inv_build_kda (per-channel decay), tri_inv_chunk_scan alone (W and U produced outside the timed "
@@ -263,9 +268,11 @@ def main():
     K, V, beta, g = dev["K"], dev["V"], dev["beta"], dev["g"]
     A = torch.empty((inp.B, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda")
     W, U = torch.empty_like(K), torch.empty_like(V)
-    G = torch.from_numpy(wl.per_channel_gate(inp, seed=3000 + args.config)).cuda() if args.call in ("kda", "kda_fused") else None
+    KDA_CALLS = ("kda", "kda_fused", "kda_scan", "kda_layer")
+    G = torch.from_numpy(wl.per_channel_gate(inp, seed=3000 + args.config)).cuda() if args.call in KDA_CALLS else None
     Q = O = None
-    if args.call in ("scan", "layer"):  # the consumer of W and U: queries, outputs, zero initial state
+    SCAN_CALLS = ("scan", "layer", "kda_scan", "kda_layer")
+    if args.call in SCAN_CALLS:  # the consumer of W and U: queries, outputs, zero initial state
         Q_host = wl.queries(inp, seed=4000 + args.config)
         Q = binding.kv_to_torch(Q_host)
         O = torch.empty_like(V)
@@ -295,6 +302,11 @@ def main():
             binding.chunk_scan(Q, K, W, U, g, inp.C, scale=q_scale, cu_seqlens=inp.cu_seqlens, out=O, want_state=False, stream=stream)
         elif args.call == "kda_fused":
             binding.fused_kda(K, V, G, beta, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U), stream=stream)
+        elif args.call == "kda_scan":
+            binding.chunk_scan_kda(Q, K, W, U, G, inp.C, scale=q_scale, cu_seqlens=inp.cu_seqlens, out=O, want_state=False, stream=stream)
+        elif args.call == "kda_layer":
+            binding.fused_kda(K, V, G, beta, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U), stream=stream)
+            binding.chunk_scan_kda(Q, K, W, U, G, inp.C, scale=q_scale, cu_seqlens=inp.cu_seqlens, out=O, want_state=False, stream=stream)
         elif args.call == "kda":
             binding.build_kda(K, G, beta, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
         else:
@@ -302,6 +314,8 @@ def main():
 
     if args.call == "scan":  # the scan reads stored W (decay-weighted) and U: produce them once, outside the timed region
         binding.fused(K, V, beta, g, inp.C, method=method | binding.W_DECAY, cu_seqlens=inp.cu_seqlens, out=(None, W, U), stream=stream)
+    if args.call == "kda_scan":
+        binding.fused_kda(K, V, G, beta, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=(A, W, U), stream=stream)
     if args.call == "wy":  # tri_inv_wy reads a stored A: produce it once, outside the timed region
         binding.build(K, beta, g, inp.C, method=method, cu_seqlens=inp.cu_seqlens, out=A, stream=stream)
 
@@ -393,8 +407,11 @@ def main():
             num[key] = max(num.get(key, 0.0), float(np.abs(x - ref).max()))
             den[key] = max(den.get(key, 0.0), float(np.abs(ref).max()))
 
-        Gs = G.cpu().numpy() if args.call in ("kda", "kda_fused") else None
-        if args.call in ("scan", "layer"):
+        Gs = G.cpu().numpy() if args.call in KDA_CALLS else None
+        if args.call in ("kda_scan", "kda_layer"):
+            O_ref, _ = oracle.recurrence_ex(Q_host, inp.K, inp.V, inp.beta, None, inp.C, G=Gs, scale=q_scale, cu_seqlens=cu)
+            acc("O", binding.to_numpy_f64(O), O_ref)
+        elif args.call in ("scan", "layer"):
             O_ref, _ = oracle.gdn_recurrence(Q_host, inp.K, inp.V, inp.beta, inp.g, inp.C, scale=q_scale, cu_seqlens=cu)
             acc("O", binding.to_numpy_f64(O), O_ref)
         else:
@@ -416,7 +433,7 @@ def main():
                     acc("W", binding.to_numpy_f64(W[:, sl]), W_ref)
                     acc("U", binding.to_numpy_f64(U[:, sl]), U_ref)
         err = {"sample": "all tokens"}
-        if args.call in ("scan", "layer"):
+        if args.call in SCAN_CALLS:
             err["reference"] = "token-by-token recurrence"
         for key in num:
             err[key + "_max_ratio"] = num[key] / den[key] if den[key] > 0 else num[key]
@@ -430,7 +447,7 @@ def main():
         traffic = None if args.paper_T else ncu_traffic_bytes_per_matrix(args.call, args.config, args.method)
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": None if traffic is None else traffic * n_mat, "peak_source": "of " + peak_kind,
-                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "kda": "per-channel-decay build+invert", "kda_fused": "per-channel-decay build+invert (+ scaled keys), then WY (2 launches)", "wy": "WY apply", "scan": "chunk scan (state recurrence + output)", "layer": "fused build+invert+WY, then chunk scan (2 launches)"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
+                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "kda": "per-channel-decay build+invert", "kda_fused": "per-channel-decay build+invert (+ scaled keys), then WY (2 launches)", "wy": "WY apply", "scan": "chunk scan (state recurrence + output)", "layer": "fused build+invert+WY, then chunk scan (2 launches)", "kda_scan": "per-channel-decay chunk scan: operand preparation, then the scan (2 launches)", "kda_layer": "per-channel-decay build+invert, WY, operand preparation, chunk scan (4 launches)"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
                     "algorithmic_bytes_per_launch": alg_bytes * n_mat}
         cpu = None
         if world == 1 and not args.no_cpu_baseline:

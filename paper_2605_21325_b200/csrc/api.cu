@@ -1,4 +1,5 @@
 // extern "C" boundary: argument validation, chunk table for packed sequences, dispatch.
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstdlib>
@@ -263,8 +264,8 @@ int chunk_scan_any(const void* Q, const void* K, const void* W, const void* U, c
   if (!aligned16(Q) || !aligned16(K) || !aligned16(W) || !aligned16(U) || !aligned16(g) || !aligned16(G) || !aligned16(O) ||
       !aligned16(S0) || !aligned16(S_out))
     return TRI_INV_ERR_INVALID_ARG;
-  // the per-channel gate exists on the CUDA-core kernel only
-  const bool tc = !G && desc->kv_dtype == TRI_INV_BF16 && desc->d_k == 128 && desc->d_v == 128 && desc->C == 64;
+  // the tensor-core kernel's shape; with a per-channel gate its operands are prepared first (one more launch)
+  const bool tc = desc->kv_dtype == TRI_INV_BF16 && desc->d_k == 128 && desc->d_v == 128 && desc->C == 64;
   if (!tc && desc->d_k > 256) return TRI_INV_ERR_UNSUPPORTED;   // the CUDA-core kernel keeps a d_k x 32 slice of S in shared memory
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   ScanParams p{};
@@ -286,9 +287,39 @@ int chunk_scan_any(const void* Q, const void* K, const void* W, const void* U, c
     }
     p.seq_off = dev_off;
   }
-  err = tc ? launch_chunk_scan(p, Q, K, W, tokens > 0 ? tokens : 1, stream)
-           : launch_chunk_scan_simt(p, Q, K, W, desc->d_k, desc->d_v, desc->C, desc->kv_dtype, stream);
+  void* work = nullptr;
+  if (tc && G && tokens > 0) {
+    // Per-channel gate on the tensor cores: Q+, K-, K^, W- (bf16, the tensors' own shape) and the per-chunk vectors
+    // exp(G_last), exp(G_ref), in stream-ordered scratch memory that is released behind the scan.
+    int max_len = desc->T;
+    if (desc->cu_seqlens) {
+      max_len = 0;
+      for (int q = 0; q < desc->n_seqs; ++q) max_len = std::max(max_len, desc->cu_seqlens[q + 1] - desc->cu_seqlens[q]);
+    }
+    const size_t tensor_bytes = ((size_t)tokens * desc->H * 128 * 2 + 255) & ~(size_t)255;
+    const size_t slots = (size_t)(tokens / 64) + (size_t)p.n_seqs + 1;
+    const size_t vec_bytes = (slots * desc->H * 128 * sizeof(float) + 255) & ~(size_t)255;
+    cudaMemPool_t pool = table_pool_for_current_device();
+    if (!pool || cudaMallocFromPoolAsync(&work, 4 * tensor_bytes + 2 * vec_bytes, pool, stream) != cudaSuccess) {
+      if (dev_off) cudaFreeAsync(dev_off, stream);
+      return TRI_INV_ERR_CUDA;
+    }
+    char* w = reinterpret_cast<char*>(work);
+    void *Qp = w, *Km = w + tensor_bytes, *Kl = w + 2 * tensor_bytes, *Wm = w + 3 * tensor_bytes;
+    float* EL = reinterpret_cast<float*>(w + 4 * tensor_bytes);
+    float* ER = reinterpret_cast<float*>(w + 4 * tensor_bytes + vec_bytes);
+    p.EL = EL; p.ER = ER;
+    err = launch_kda_scan_prep(p, Q, K, W, Qp, Km, Kl, Wm, EL, ER, (max_len + 63) / 64, stream);
+    if (err == cudaSuccess) {
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+      err = launch_chunk_scan(p, Qp, Km, Wm, tokens, stream, Kl);
+    }
+  } else {
+    err = (tc && !G) ? launch_chunk_scan(p, Q, K, W, tokens > 0 ? tokens : 1, stream)
+                     : launch_chunk_scan_simt(p, Q, K, W, desc->d_k, desc->d_v, desc->C, desc->kv_dtype, stream);
+  }
   if (err == cudaSuccess) g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (work) cudaFreeAsync(work, stream);
   if (dev_off) cudaFreeAsync(dev_off, stream);
   return err == cudaSuccess ? TRI_INV_OK : TRI_INV_ERR_CUDA;
 }

@@ -42,7 +42,14 @@ namespace {
 constexpr int C = 64, D = 128, NT = 256;   // NT compute threads (8 warps) + the control warp + the gate warp
 constexpr float kLog2e = 1.4426950408889634f;
 
-template <int DVS>
+// KDA: the per-channel form (one decay per key feature, the KDA row of Table 1).  Its decays are folded into the
+// operands beforehand (kda_scan_prep_kernel, scan_kda_prep.cu): with G_ref the middle row of a chunk and G_last its last,
+//     W- = W exp(-G_ref),  Q+ = Q exp(G - G_ref),  K- = K exp(G_ref - G),  K^ = K exp(G_last - G),
+// P1 = [W- ; Q+] . [(diag(exp G_ref) S) | K-^T] gives W S, (Q exp G) S and the decayed Q K^T at once, P3 = K^^T U~ is
+// the state increment (no second, decay-scaled copy of U~), and S decays by exp(G_last) per row.  The kernel then
+// differs from the scalar-gate one only in where its operands come from and in a few scalings: the S^T operand is
+// scaled per row by exp(G_ref) of the coming chunk, P needs no decay, K^ has a tile of its own.
+template <int DVS, bool KDA = false>
 struct ScanCfg {
   static constexpr int CW = DVS / 2;                     // value columns per compute warp
   static constexpr int NTW = CW / 8;                     // accumulator n-tiles per compute warp
@@ -54,13 +61,15 @@ struct ScanCfg {
   // B operand of P1: [S^T ; K], two boxes of (DVS + 64) rows x 128 B
   static constexpr int OFF_B = 2 * A_TILE, B_BOX = N1 * 128, B_TILE = 2 * B_BOX;
   // (the K rows of the B tile are also the MN-major A operand of P3: the tile stays whole until the chunk after next)
-  static constexpr int OFF_P = OFF_B + 2 * B_TILE;       // P, the lower half of PU's A operand; the unused upper half is whatever precedes it
+  static constexpr int OFF_KA = OFF_B + 2 * B_TILE;      // per-channel form: K^ tiles of two chunks in turn (MN-major A operand of P3)
+  static constexpr int OFF_P = OFF_KA + (KDA ? 2 * 16384 : 0);   // P, the lower half of PU's A operand; the unused upper half is whatever precedes it
   static constexpr int OFF_UT = OFF_P + 8192;            // U~  bf16 [64 tokens][DVS], boxes of 64 columns (MN-major B)
   static constexpr int U_BYTES = 8192 * (DVS > 64 ? DVS / 64 : 1);   // a narrower slice fills the first DVS columns of one box
   static constexpr int OFF_UD = OFF_UT + U_BYTES;        // U~' bf16, same layout
   static constexpr int OFF_U = OFF_UD + U_BYTES;         // U tiles of two chunks in turn: bf16 [64 tokens][64 columns], as copied
   static constexpr int OFF_G = OFF_U + 2 * 8192;         // g * log2(e): 2 x 64 floats; column factors: 2 x 64 floats
-  static constexpr int OFF_BAR = OFF_G + 1024;           // 12 mbarriers, tensor-memory slot
+                                                         // per-channel form: exp(G_last) and exp(G_ref), 128 floats each, of three chunks in turn
+  static constexpr int OFF_BAR = OFF_G + (KDA ? 3072 : 1024);   // 12 mbarriers, tensor-memory slot
   static constexpr int SMEM = OFF_BAR + 128;
   static constexpr int TM_P1 = 0, TM_DS = N1, TM_PU = N1 + DVS;
   static constexpr int TMEM_COLS = (N1 + 2 * DVS) <= 256 ? 256 : 512;
@@ -106,11 +115,12 @@ __host__ __device__ constexpr uint32_t umma_idesc_ab(int M, int N, int a_mn, int
   return umma_idesc(M, N, b_mn) | ((uint32_t)a_mn << 15);
 }
 
-template <int DVS>
-__global__ void __launch_bounds__(NT + 64, ScanCfg<DVS>::CTAS_PER_SM)
+template <int DVS, bool KDA>
+__global__ void __launch_bounds__(NT + 64, ScanCfg<DVS, KDA>::CTAS_PER_SM)
 chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmQ,
-                  const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmU, ScanParams p) {
-  using cfg = ScanCfg<DVS>;
+                  const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmU,
+                  const __grid_constant__ CUtensorMap tmKL, ScanParams p) {
+  using cfg = ScanCfg<DVS, KDA>;
   constexpr int NTW = cfg::NTW, CW = cfg::CW, NS = D / DVS;
   extern __shared__ __align__(1024) uint8_t smem[];
   float* sG = reinterpret_cast<float*>(smem + cfg::OFF_G);
@@ -118,12 +128,14 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 80);
   const uint32_t sA = smem_u32(smem + cfg::OFF_A), sB = smem_u32(smem + cfg::OFF_B);
   const uint32_t sP = smem_u32(smem + cfg::OFF_P), sUt = smem_u32(smem + cfg::OFF_UT), sUd = smem_u32(smem + cfg::OFF_UD);
-  const uint32_t sU = smem_u32(smem + cfg::OFF_U);
+  const uint32_t sU = smem_u32(smem + cfg::OFF_U), sKa = smem_u32(smem + cfg::OFF_KA);
+  float* sEl = sG;                 // per-channel form: exp(G_last) [3][128], then exp(G_ref) [3][128]
+  float* sEr = sG + 3 * D;
   // copies (TMA):            bar_a (W and Q), bar_kb (K beside S^T), bar_u0 / bar_u1 (U, chunks in turn)
   // products done (commit):  bar_t1 (P1), bar_s (P3), bar_pu (PU)
   // operands written:        bar_sr (S^T by the compute warps, the next chunk's g by the gate warp), bar_ut (U~ and U~',
   //                          chain warps), bar_p (P, output warps); one arrival per warp
-  const uint32_t bar_a = smem_u32(smem + cfg::OFF_BAR), bar_kb = bar_a + 8, bar_t1 = bar_a + 24,
+  const uint32_t bar_a = smem_u32(smem + cfg::OFF_BAR), bar_kb = bar_a + 8, bar_ka = bar_a + 16, bar_t1 = bar_a + 24,
                  bar_s = bar_a + 32, bar_pu = bar_a + 40, bar_sr = bar_a + 48, bar_ut = bar_a + 56, bar_p = bar_a + 64,
                  bar_u0 = bar_a + 72, bar_u1 = bar_a + 88, bar_ud = bar_a + 96;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -178,19 +190,23 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 
   // S^T as rows 0..DVS-1 of the K-major B operand of P1: row n = value column, 16-byte pieces of eight key features.
   // stmatrix.trans turns the fragments (rows = features, column pairs) into exactly those pieces.
-  auto write_state_operand = [&](int buf) {
+  // (per-channel form: row k of S times er[k], exp(G_ref) of the chunk that will read the operand)
+  auto write_state_operand = [&](int buf, const float* er) {
     const int mi = lane >> 3, r = lane & 7;      // this lane addresses row r of matrix mi of each x4 store
 #pragma unroll
-    for (int lg = 0; lg < 2; ++lg)
+    for (int lg = 0; lg < 2; ++lg) {
+      float ea = 1.f, eb = 1.f;
+      if constexpr (KDA) { ea = er[krow_w + 16 * lg + gq]; eb = er[krow_w + 16 * lg + gq + 8]; }
 #pragma unroll
       for (int nt = 0; nt < NTW; nt += 2) {
         // matrices: (features +0..7, tile nt), (features +8..15, tile nt), (+0..7, nt+1), (+8..15, nt+1)
         const int k0 = krow_w + 16 * lg + 8 * (mi & 1);          // first feature of this lane's matrix
         const int n = cw0 + 8 * (nt + (mi >> 1)) + r;            // row of the operand
         const uint32_t addr = sB + buf * cfg::B_TILE + (k0 >> 6) * cfg::B_BOX + n * 128 + ((((k0 & 63) >> 3) ^ (n & 7)) << 4);
-        stmatrix_x4_trans(addr, pack_bf16(S[lg][nt][0], S[lg][nt][1]), pack_bf16(S[lg][nt][2], S[lg][nt][3]),
-                          pack_bf16(S[lg][nt + 1][0], S[lg][nt + 1][1]), pack_bf16(S[lg][nt + 1][2], S[lg][nt + 1][3]));
+        stmatrix_x4_trans(addr, pack_bf16(ea * S[lg][nt][0], ea * S[lg][nt][1]), pack_bf16(eb * S[lg][nt][2], eb * S[lg][nt][3]),
+                          pack_bf16(ea * S[lg][nt + 1][0], ea * S[lg][nt + 1][1]), pack_bf16(eb * S[lg][nt + 1][2], eb * S[lg][nt + 1][3]));
       }
+    }
   };
   // W, Q and the K beside S^T of chunk c, into the tiles of c's parity
   auto issue_wq = [&](int c) {
@@ -208,6 +224,12 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     mbar_expect_tx(bar_kb, 16384u);
     tma_load_2d(dst, &tmK, bar_kb, h * D, tok0);
     tma_load_2d(dst + cfg::B_BOX, &tmK, bar_kb, h * D + 64, tok0);
+  };
+  // per-channel form: K^ of chunk c, the MN-major A operand of P3, into the tile of c's parity
+  auto issue_ka = [&](int c) {
+    mbar_expect_tx(bar_ka, 16384u);
+    tma_load_2d(sKa + (c & 1) * 16384, &tmKL, bar_ka, h * D, beg + c * C);
+    tma_load_2d(sKa + (c & 1) * 16384 + 8192, &tmKL, bar_ka, h * D + 64, beg + c * C);
   };
   // U of chunk c: the 64-column box that holds this CTA's slice, into the buffer of c's parity
   auto issue_u = [&](int c) {
@@ -238,6 +260,18 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     }
   };
 
+  // per-channel form: exp(G_last) and exp(G_ref) of a chunk (128 floats each, written by the preparation kernel at the
+  // chunk's slot), by the gate warp: lane l brings features 4 l .. 4 l + 3 of both; three chunks' worth are kept in turn
+  auto fetch_e = [&](int c, float4 (&ev)[2]) {
+    const size_t slot = (size_t)((beg + c * C) / C + s);
+    ev[0] = *reinterpret_cast<const float4*>(p.EL + (slot * p.H + h) * D + 4 * lane);
+    ev[1] = *reinterpret_cast<const float4*>(p.ER + (slot * p.H + h) * D + 4 * lane);
+  };
+  auto store_e = [&](int c, const float4 (&ev)[2]) {
+    *reinterpret_cast<float4*>(sEl + (c % 3) * D + 4 * lane) = ev[0];
+    *reinterpret_cast<float4*>(sEr + (c % 3) * D + 4 * lane) = ev[1];
+  };
+  float4 e_raw[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
   float g_raw[2] = {0.f, 0.f};   // gate warp: g of the chunk it stores next
   if (tid == NT) {
     prefetch_tmap(&tmW); prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmU);
@@ -250,25 +284,41 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     mbar_init(bar_p, NT / 64);
     fence_mbar_init();
     if (!misaligned) {
+      if constexpr (KDA) issue_ka(0);
       issue_wq(0);
       issue_kb(0);
       issue_u(0);
     }
   }
   if (gate_warp) {
-    fetch_g(0, g_raw);
-    store_g(0, g_raw);
-    if (n_chunks > 1) fetch_g(1, g_raw);
+    if constexpr (KDA) {
+      // the vectors of the first two chunks are in place before the loop starts, the third chunk's in registers
+      fetch_e(0, e_raw);
+      store_e(0, e_raw);
+      if (n_chunks > 1) { fetch_e(1, e_raw); store_e(1, e_raw); }
+      if (n_chunks > 2) fetch_e(2, e_raw);
+    } else {
+      fetch_g(0, g_raw);
+      store_g(0, g_raw);
+      if (n_chunks > 1) fetch_g(1, g_raw);
+    }
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(cfg::TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (compute) write_state_operand(0);
+  if (compute && !KDA) write_state_operand(0, nullptr);
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();   // barriers initialised, tensor memory allocated, first operand of S and first g in place
   tc_fence_after();
+  if constexpr (KDA) {
+    // the first operand of S needs exp(G_ref) of the first chunk, which the gate warp has just stored
+    if (compute) {
+      write_state_operand(0, sEr);
+      fence_proxy_async();
+    }
+  }
   const uint32_t tmem = *tmem_slot;
   const uint32_t tmem_w = tmem + ((uint32_t)(32 * quad) << 16);   // this warp's lanes, column 0
   bool failed = misaligned;
@@ -280,7 +330,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       constexpr uint32_t idesc_p3 = umma_idesc_ab(128, DVS, 1, 1);       // K tile MN-major, U~' MN-major
       constexpr uint32_t idesc_pu = umma_idesc_ab(128, DVS, 0, 1);       // [any;P] K-major, U~ MN-major
       // descriptors differ from these bases only in the address field (bits 0..13, units of 16 bytes)
-      const uint64_t dA = umma_desc(sA, 16, 1024), dB = umma_desc(sB, 16, 1024), dKa = umma_desc(sB + DVS * 128, cfg::B_BOX, 1024),   // the K rows of the B tile, MN-major
+      const uint64_t dA = umma_desc(sA, 16, 1024), dB = umma_desc(sB, 16, 1024), dKa = KDA ? umma_desc(sKa, 8192, 1024) : umma_desc(sB + DVS * 128, cfg::B_BOX, 1024),   // MN-major: the K^ tile, or the K rows of the B tile
                      dUd = umma_desc(sUd, 8192, 1024), dUt = umma_desc(sUt, 8192, 1024),
                      dPa = umma_desc(sP - 8192, 16, 1024);               // 128 rows: 64 of whatever lies before P (results unused), then P
       uint32_t ph = 0;
@@ -290,6 +340,8 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         if (!mbar_wait_bounded(bar_a, ph)) { failed = true; break; }
         TL(7);
         if (!mbar_wait_bounded(bar_kb, ph)) { failed = true; break; }
+        // (a barrier's phase has to be over before the copy of the next chunk is announced on it, below)
+        if (KDA && !mbar_wait_bounded(bar_ka, ph)) { failed = true; break; }
         TL(8);
         if (!mbar_wait_bounded(bar_sr, ph)) { failed = true; break; }
         tc_fence_after();
@@ -304,6 +356,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         // into the other tiles, whose last readers (P1 and P3 of the chunk before this one; for U the chain warps, a
         // chunk ago) were done before the arrivals on bar_sr seen above: nothing to wait for.
         if (c + 1 < n_chunks) {
+          if constexpr (KDA) issue_ka(c + 1);
           issue_u(c + 1);
           issue_kb(c + 1);
           issue_wq(c + 1);
@@ -314,7 +367,8 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         TL(3);
 #pragma unroll
         for (int ks = 0; ks < C / 16; ++ks)   // 16 tokens (2048 bytes of either operand) per step
-          umma_bf16(tmem + cfg::TM_DS, dKa + (((c & 1) * cfg::B_TILE + ks * 2048) >> 4), dUd + ((ks * 2048) >> 4), idesc_p3, ks > 0);
+          umma_bf16(tmem + cfg::TM_DS, dKa + (((c & 1) * (KDA ? 16384 : cfg::B_TILE) + ks * 2048) >> 4),
+                    (KDA ? dUt : dUd) + ((ks * 2048) >> 4), idesc_p3, ks > 0);   // per-channel form: U~ itself, the decay is in K^
         umma_commit(bar_s);
         TL(4);
         if (!mbar_wait_bounded(bar_ut, ph) || !mbar_wait_bounded(bar_p, ph)) { failed = true; break; }
@@ -337,9 +391,18 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     for (int c = 0; c + 1 < n_chunks && !misaligned; ++c) {
       // the buffer of c + 1 held g of c - 1: every compute warp has left that chunk once the arrivals that end it are in
       if (c > 0 && !mbar_wait_bounded(bar_sr, (uint32_t)(c & 1))) { failed = true; break; }
-      store_g((c + 1) & 1, g_raw);
-      warp_arrive(bar_sr, lane);
-      if (c + 2 < n_chunks) fetch_g(c + 2, g_raw);
+      if constexpr (KDA) {
+        // The vectors run one chunk further ahead than g: exp(G_ref) of chunk c + 1 is read at the end of chunk c (it
+        // scales the S^T operand), so it has to be in place, and announced by an arrival, a chunk earlier.  Those of
+        // c + 2 go where those of c - 1 were.
+        if (c + 2 < n_chunks) store_e(c + 2, e_raw);
+        warp_arrive(bar_sr, lane);
+        if (c + 3 < n_chunks) fetch_e(c + 3, e_raw);
+      } else {
+        store_g((c + 1) & 1, g_raw);
+        warp_arrive(bar_sr, lane);
+        if (c + 2 < n_chunks) fetch_g(c + 2, g_raw);
+      }
     }
   } else {
     // ---------------------------------------------------------------- compute warps
@@ -389,7 +452,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       TL(2);
       // (this chunk's g was written by the gate warp during the last chunk: read only after the wait above,
       // which follows that warp's arrival on bar_sr)
-      const float g_last = gb[rows - 1];
+      const float g_last = KDA ? 0.f : gb[rows - 1];
       if (chain) {
         // ---- U~ = U - W S  ->  bf16 operands [token rows][value columns]: first the decay-scaled U~' that the chain
         // waits for (its own arrival), then U~ itself for the third product
@@ -415,8 +478,10 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             ldmatrix_x4(sUc + tok * 128 + (((((n + u_shift) & 63) >> 3) ^ (tok & 7)) << 4), xu[lg][nt][0], xu[lg][nt][1], xu[lg][nt + 1][0], xu[lg][nt + 1][1]);
           }
           const int i = tok_w + 16 * lg + gq;
-          da[lg] = ex2_approx(g_last - gb[i]);
-          db[lg] = ex2_approx(g_last - gb[i + 8]);
+          if constexpr (!KDA) {
+            da[lg] = ex2_approx(g_last - gb[i]);
+            db[lg] = ex2_approx(g_last - gb[i + 8]);
+          }
         }
         tmem_wait_ld();
         TL(4);
@@ -442,15 +507,17 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             }
           }
         }
+        if constexpr (!KDA) {
 #pragma unroll
-        for (int lg = 0; lg < 2; ++lg)
+          for (int lg = 0; lg < 2; ++lg)
 #pragma unroll
-          for (int nt = 0; nt < NTW; nt += 2)
-            stmatrix_x4(sUd + off[lg][nt / 2], pack_bf16(v[lg][nt][0] * da[lg], v[lg][nt][1] * da[lg]), pack_bf16(v[lg][nt][2] * db[lg], v[lg][nt][3] * db[lg]),
-                        pack_bf16(v[lg][nt + 1][0] * da[lg], v[lg][nt + 1][1] * da[lg]), pack_bf16(v[lg][nt + 1][2] * db[lg], v[lg][nt + 1][3] * db[lg]));
-        fence_proxy_async();
-        tc_fence_before();
-        warp_arrive(bar_ud, lane);
+            for (int nt = 0; nt < NTW; nt += 2)
+              stmatrix_x4(sUd + off[lg][nt / 2], pack_bf16(v[lg][nt][0] * da[lg], v[lg][nt][1] * da[lg]), pack_bf16(v[lg][nt][2] * db[lg], v[lg][nt][3] * db[lg]),
+                          pack_bf16(v[lg][nt + 1][0] * da[lg], v[lg][nt + 1][1] * da[lg]), pack_bf16(v[lg][nt + 1][2] * db[lg], v[lg][nt + 1][3] * db[lg]));
+          fence_proxy_async();
+          tc_fence_before();
+          warp_arrive(bar_ud, lane);
+        }
         TL(5);
 #pragma unroll
         for (int lg = 0; lg < 2; ++lg)
@@ -459,6 +526,10 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             stmatrix_x4(sUt + off[lg][nt / 2], pack_bf16(v[lg][nt][0], v[lg][nt][1]), pack_bf16(v[lg][nt][2], v[lg][nt][3]),
                         pack_bf16(v[lg][nt + 1][0], v[lg][nt + 1][1]), pack_bf16(v[lg][nt + 1][2], v[lg][nt + 1][3]));
         fence_proxy_async();
+        if constexpr (KDA) {   // U~ itself is the operand of both later products
+          tc_fence_before();
+          warp_arrive(bar_ud, lane);
+        }
         warp_arrive(bar_ut, lane);
         TL(6);
       } else {
@@ -475,22 +546,27 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         // what the blocks need from shared memory, while the loads above are in flight
         float gref[4];
         float2 cj[4];
+        if constexpr (!KDA) {
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          gref[q4] = gb[8 * (4 * half + q4)];
-          cj[q4] = *reinterpret_cast<const float2*>(cf + 8 * (4 * half + q4) + 2 * t);
+          for (int q4 = 0; q4 < 4; ++q4) {
+            gref[q4] = gb[8 * (4 * half + q4)];
+            cj[q4] = *reinterpret_cast<const float2*>(cf + 8 * (4 * half + q4) + 2 * t);
+          }
         }
         tmem_wait_ld();
         TL(3);
 #pragma unroll
         for (int lg = 0; lg < 2; ++lg) {
           const int ia = tok_w + 16 * lg + gq, ib = ia + 8;
-          const float g_a = gb[ia], g_b = gb[ib];
+          const float g_a = KDA ? 0.f : gb[ia], g_b = KDA ? 0.f : gb[ib];
           {
-            // gamma_i Q S becomes the starting value of the PU accumulator (same lanes, same columns)
-            const float ya = ex2_approx(g_a), yb = ex2_approx(g_b);
+            // gamma_i Q S becomes the starting value of the PU accumulator (same lanes, same columns); in the
+            // per-channel form the decay is inside the product already
+            if constexpr (!KDA) {
+              const float ya = ex2_approx(g_a), yb = ex2_approx(g_b);
 #pragma unroll
-            for (int nt = 0; nt < NTW; ++nt) { qsf[lg][nt][0] *= ya; qsf[lg][nt][1] *= ya; qsf[lg][nt][2] *= yb; qsf[lg][nt][3] *= yb; }
+              for (int nt = 0; nt < NTW; ++nt) { qsf[lg][nt][0] *= ya; qsf[lg][nt][1] *= ya; qsf[lg][nt][2] *= yb; qsf[lg][nt][3] *= yb; }
+            }
             tmem_st_frag<NTW>(qsf[lg], tmem_w + ((uint32_t)(16 * lg) << 16) + cfg::TM_PU + cw0);
           }
           // No branch around a block: entries right of a row's diagonal are masked by selection, and the exponent of
@@ -501,9 +577,15 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
           for (int q4 = 0; q4 < 4; ++q4) {
             const int nt = 4 * half + q4;
             const int j = 8 * nt + 2 * t;
-            const float ea = ex2_approx(8 * nt <= ia ? g_a - gref[q4] : 0.f), eb = ex2_approx(8 * nt <= ib ? g_b - gref[q4] : 0.f);
-            const float p0 = j <= ia ? qk[lg][q4][0] * ea * cj[q4].x : 0.f, p1 = j + 1 <= ia ? qk[lg][q4][1] * ea * cj[q4].y : 0.f;
-            const float p2 = j <= ib ? qk[lg][q4][2] * eb * cj[q4].x : 0.f, p3 = j + 1 <= ib ? qk[lg][q4][3] * eb * cj[q4].y : 0.f;
+            float p0, p1, p2, p3;
+            if constexpr (KDA) {   // the product carries its decay: only the mask is left
+              p0 = j <= ia ? qk[lg][q4][0] : 0.f; p1 = j + 1 <= ia ? qk[lg][q4][1] : 0.f;
+              p2 = j <= ib ? qk[lg][q4][2] : 0.f; p3 = j + 1 <= ib ? qk[lg][q4][3] : 0.f;
+            } else {
+              const float ea = ex2_approx(8 * nt <= ia ? g_a - gref[q4] : 0.f), eb = ex2_approx(8 * nt <= ib ? g_b - gref[q4] : 0.f);
+              p0 = j <= ia ? qk[lg][q4][0] * ea * cj[q4].x : 0.f; p1 = j + 1 <= ia ? qk[lg][q4][1] * ea * cj[q4].y : 0.f;
+              p2 = j <= ib ? qk[lg][q4][2] * eb * cj[q4].x : 0.f; p3 = j + 1 <= ib ? qk[lg][q4][3] * eb * cj[q4].y : 0.f;
+            }
             wa[q4] = pack_bf16(p0, p1);
             wb[q4] = pack_bf16(p2, p3);
           }
@@ -533,6 +615,14 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       TL(7);
       {
         const float gl = ex2_approx(g_last);
+        float el[2][2];   // per-channel form: exp(G_last) of this thread's four rows of S
+        if constexpr (KDA) {
+#pragma unroll
+          for (int lg = 0; lg < 2; ++lg) {
+            el[lg][0] = sEl[(c % 3) * D + krow_w + 16 * lg + gq];
+            el[lg][1] = sEl[(c % 3) * D + krow_w + 16 * lg + gq + 8];
+          }
+        }
         float ds[2][NTW][4];
         tmem_ld_frag<NTW>(ds[0], tmem_w + cfg::TM_DS + cw0);
         tmem_ld_frag<NTW>(ds[1], tmem_w + (16u << 16) + cfg::TM_DS + cw0);
@@ -542,10 +632,10 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 #pragma unroll
           for (int nt = 0; nt < NTW; ++nt)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) S[lg][nt][e] = fmaf(gl, S[lg][nt][e], ds[lg][nt][e]);
+            for (int e = 0; e < 4; ++e) S[lg][nt][e] = fmaf(KDA ? el[lg][e >> 1] : gl, S[lg][nt][e], ds[lg][nt][e]);
         TL(8);
         if (has_next) {
-          write_state_operand((c + 1) & 1);   // that tile's last reader was P1 of the chunk before this one
+          write_state_operand((c + 1) & 1, sEr + ((c + 1) % 3) * D);   // that tile's last reader was P1 of the chunk before this one
           TL(9);
           fence_proxy_async();
           tc_fence_before();
@@ -573,10 +663,10 @@ __global__ void __launch_bounds__(256) seq_offsets_kernel(int* out, const __grid
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i <= b.n; i += gridDim.x * blockDim.x) out[b.first + i] = b.cu[i];
 }
 
-template <int DVS>
+template <int DVS, bool KDA>
 cudaError_t launch_scan_one(const ScanParams& p, const CUtensorMap& tmW, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                            const CUtensorMap& tmU, cudaStream_t stream) {
-  using cfg = ScanCfg<DVS>;
+                            const CUtensorMap& tmU, const CUtensorMap& tmKL, cudaStream_t stream) {
+  using cfg = ScanCfg<DVS, KDA>;
   static std::mutex mu;
   static bool ready[64] = {false};
   int dev = 0;
@@ -586,14 +676,14 @@ cudaError_t launch_scan_one(const ScanParams& p, const CUtensorMap& tmW, const C
   {
     std::lock_guard<std::mutex> lock(mu);
     if (!ready[dev]) {
-      if ((e = cudaFuncSetAttribute(chunk_scan_kernel<DVS>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM)) != cudaSuccess) return e;
-      if ((e = cudaFuncSetAttribute(chunk_scan_kernel<DVS>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(chunk_scan_kernel<DVS, KDA>, cudaFuncAttributeMaxDynamicSharedMemorySize, cfg::SMEM)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(chunk_scan_kernel<DVS, KDA>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
       ready[dev] = true;
     }
   }
   const long long grid = (long long)p.n_seqs * p.H * (D / DVS);
   if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
-  chunk_scan_kernel<DVS><<<(int)grid, NT + 64, cfg::SMEM, stream>>>(tmW, tmQ, tmK, tmU, p);
+  chunk_scan_kernel<DVS, KDA><<<(int)grid, NT + 64, cfg::SMEM, stream>>>(tmW, tmQ, tmK, tmU, tmKL, p);
   return cudaGetLastError();
 }
 
@@ -620,16 +710,19 @@ cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t
 // per pair instead, still at most one per SM: the per-chunk chain of a CTA is a little shorter (7 % on one sequence
 // of 32 heads), and every output column is computed by the same operations in the same order either way.  With more
 // pairs than that the narrow slices would share SMs and repeat the Q K^T part of the first product: measured slower.
+// K_last != nullptr selects the per-channel form: Q, K, W are then the prepared operands Q+, K-, W- and K_last is K^
+// (scan_kda_prep.cu), with p.EL / p.ER the per-chunk vectors.
 cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,
-                              cudaStream_t stream) {
-  CUtensorMap tmW, tmQ, tmK, tmU;
+                              cudaStream_t stream, const void* K_last) {
+  CUtensorMap tmW, tmQ, tmK, tmU, tmKL;
   if (!make_tmap(&tmW, W, tokens, p.H, D, C, 2) || !make_tmap(&tmQ, Q, tokens, p.H, D, C, 2) || !make_tmap(&tmK, K, tokens, p.H, D, C, 2) ||
-      !make_tmap(&tmU, p.U, tokens, p.H, D, C, 2))
+      !make_tmap(&tmU, p.U, tokens, p.H, D, C, 2) || !make_tmap(&tmKL, K_last ? K_last : K, tokens, p.H, D, C, 2))
     return cudaErrorUnknown;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
-  if ((long long)p.n_seqs * p.H * 4 <= sms) return launch_scan_one<32>(p, tmW, tmQ, tmK, tmU, stream);
-  return launch_scan_one<64>(p, tmW, tmQ, tmK, tmU, stream);
+  const bool narrow = (long long)p.n_seqs * p.H * 4 <= sms;
+  if (K_last) return narrow ? launch_scan_one<32, true>(p, tmW, tmQ, tmK, tmU, tmKL, stream) : launch_scan_one<64, true>(p, tmW, tmQ, tmK, tmU, tmKL, stream);
+  return narrow ? launch_scan_one<32, false>(p, tmW, tmQ, tmK, tmU, tmKL, stream) : launch_scan_one<64, false>(p, tmW, tmQ, tmK, tmU, tmKL, stream);
 }
 
 }  // namespace tri_inv

@@ -302,6 +302,10 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       }
     }
     if (load_a) {
+      // The staging tiles of the last item's W / U stores lie in the matrix's space, which every thread is about to
+      // write: each warp's stores must have read their tile first (its lane 0 issued them), and everyone must know.
+      if (lane == 0) bulk_wait_read();
+      __syncthreads();
       // tri_inv_wy: the stored A comes in with 16-byte loads; only its strict lower triangle is used
       // (unit diagonal and zero upper triangle are written as constants)
       const size_t a_step = (size_t)(cfg::NT / (C / 4)) * p.H * C;

@@ -171,7 +171,28 @@ def test_adversarial_keys_report(bnd):
     print("adversarial keys, max ratio per method:", report)
 
 
-@pytest.mark.parametrize("cfg", [2, 4], ids=["config2_C64", "config4_C128"])
+@pytest.mark.parametrize("cfg", [2, 3, 5])
+def test_wy_alone_reproduces_the_fused_call_at_full_size(bnd, cfg):
+    """tri_inv_wy on the A that tri_inv_build stored gives, bit for bit, the W and U of the fused call (the same kernel
+    with the matrix loaded instead of built), on every token of the large configurations -- also in place, with the keys
+    in the buffer that receives W (the form tri_inv_fused_kda uses).  The matrix is loaded into the space that the output
+    staging tiles of the item before live in: the stores that read them must be through first."""
+    inp = wl.config(cfg)
+    dev = bnd.to_device(inp)
+    cu = inp.cu_seqlens
+    _, W_ref, U_ref = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], inp.C, cu_seqlens=cu, want_A=False)
+    A = bnd.build(dev["K"], dev["beta"], dev["g"], inp.C, cu_seqlens=cu)
+    for in_place in (False, True):
+        for _ in range(3):
+            W = dev["K"].clone() if in_place else torch.full_like(dev["K"], float("nan"))
+            U = torch.full_like(dev["V"], float("nan"))
+            bnd.wy(A, W if in_place else dev["K"], dev["V"], dev["beta"], cu_seqlens=cu, out=(W, U))
+            torch.cuda.synchronize()
+            assert bnd.last_device_status() == 0
+            assert torch.equal(W.view(torch.int16), W_ref.view(torch.int16)) and torch.equal(U.view(torch.int16), U_ref.view(torch.int16))
+
+
+@pytest.mark.parametrize("cfg", [2, 3, 4], ids=["config2_C64", "config3_C64", "config4_C128"])
 def test_per_channel_decay_full_size(bnd, cfg):
     """tri_inv_fused_kda on the shapes of config 2 (4096 matrices of 64 tokens) and config 4 (2048 of 128), the launches
     bench.py --call kda_fused times: structure on every element, EVERY matrix's A, W and U against the fp64 oracle, and -- at
