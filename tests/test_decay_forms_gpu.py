@@ -123,3 +123,49 @@ def test_flags_the_per_channel_calls_refuse(bnd):
     assert L.tri_inv_build_kda(p, p, p, p, ctypes.byref(desc), bnd.GATE_SHIFTED, None) == bnd.ERR_UNSUPPORTED
     assert L.tri_inv_fused_kda(p, p, p, p, p, p, p, ctypes.byref(desc), bnd.W_DECAY, None) == bnd.ERR_UNSUPPORTED
     assert L.tri_inv_fused_kda(p, p, p, p, None, p, p, ctypes.byref(desc), 0, None) == bnd.ERR_INVALID_ARG
+
+
+def test_per_channel_scan_on_the_tensor_cores_full_size_ragged(bnd):
+    """tri_inv_chunk_scan_kda at bf16 / d = 128 / C = 64 (operand preparation + the tensor-core scan) on the packed, ragged
+    shape of config 5: EVERY token of O and every final state against the token-by-token recurrence with one decay per
+    key feature; the same launch twice gives the same bits; and a sequence resumed from a returned state reproduces the
+    continuous run bit for bit."""
+    inp = wl.config(5)
+    cu = inp.cu_seqlens
+    G = wl.per_channel_gate(inp, seed=3005)
+    Q = wl.queries(inp, seed=64)
+    S0 = wl.initial_state(inp, seed=65)
+    dev = bnd.to_device(inp)
+    Gd, Qd, S0d = torch.from_numpy(G).cuda(), bnd.kv_to_torch(Q), torch.from_numpy(S0).cuda()
+    _, W, U = bnd.fused_kda(dev["K"], dev["V"], Gd, dev["beta"], 64, cu_seqlens=cu)
+    O = torch.full_like(dev["V"], float("nan"))
+    O, S = bnd.chunk_scan_kda(Qd, dev["K"], W, U, Gd, 64, scale=0.25, S0=S0d, cu_seqlens=cu, out=O)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    O_ref, S_ref = oracle.recurrence_ex(Q, inp.K, inp.V, inp.beta, None, 64, G=G, scale=0.25, S0=S0, cu_seqlens=cu)
+    o = bnd.to_numpy_f64(O)
+    assert not np.isnan(o).any(), "a row of O was not written"
+    assert max_ratio(o, O_ref) <= 2e-2 and max_ratio(bnd.to_numpy_f64(S), S_ref) <= 2e-2
+    O2, S2 = bnd.chunk_scan_kda(Qd, dev["K"], W, U, Gd, 64, scale=0.25, S0=S0d, cu_seqlens=cu)
+    torch.cuda.synchronize()
+    assert torch.equal(O2.view(torch.int16), O.view(torch.int16)) and torch.equal(S2, S)
+
+
+def test_per_channel_scan_resumes_bit_for_bit(bnd):
+    """Dense batch cut at a chunk boundary: the second part, started from the first part's returned state, gives the very
+    bits of the uncut run (few (sequence, head) pairs: the 32-column instance; many: the 64-column one)."""
+    for B, H in ((1, 2), (3, 20)):
+        T, cut = 6 * 64 + 23, 4 * 64
+        inp = wl.make("resume", B, T, H, 128, 128, 64, wl.BF16, seed=1400 + H)
+        G = wl.per_channel_gate(inp, seed=66)
+        Q = wl.queries(inp, seed=67)
+        dev = bnd.to_device(inp)
+        Gd, Qd = torch.from_numpy(G).cuda(), bnd.kv_to_torch(Q)
+        _, W, U = bnd.fused_kda(dev["K"], dev["V"], Gd, dev["beta"], 64)
+        O, S = bnd.chunk_scan_kda(Qd, dev["K"], W, U, Gd, 64, scale=0.5)
+        part = lambda t, a, b: t[:, a:b].contiguous()
+        O1, S1 = bnd.chunk_scan_kda(part(Qd, 0, cut), part(dev["K"], 0, cut), part(W, 0, cut), part(U, 0, cut), part(Gd, 0, cut), 64, scale=0.5)
+        O2, S2 = bnd.chunk_scan_kda(part(Qd, cut, T), part(dev["K"], cut, T), part(W, cut, T), part(U, cut, T), part(Gd, cut, T), 64, scale=0.5, S0=S1)
+        torch.cuda.synchronize()
+        assert bnd.last_device_status() == 0
+        assert torch.equal(torch.cat([O1, O2], dim=1).view(torch.int16), O.view(torch.int16)) and torch.equal(S2, S)
