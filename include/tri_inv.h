@@ -221,8 +221,14 @@ int tri_inv_fused_kda(const void* K, const void* V, const float* G, const float*
  * The chunk scan with one decay per key feature (KDA row): as tri_inv_chunk_scan with g replaced by G [B,T,H,d_k] fp32,
  *     U~ = U - W S,     P_ij = sum_c Q_ic K_jc exp(G_ic - G_jc)  (j <= i),
  *     O  = scale * ((Q * Gamma) S + P U~),     S <- diag(Gamma_last) S + (K * exp(G_last - G))^T U~,
- * W and U from tri_inv_fused_kda.  Runs on the CUDA cores in fp32 for every shape (d_k <= 256); the exponent is taken of
- * each difference, so G is not restricted.
+ * W and U from tri_inv_fused_kda.  bf16 with d_k = d_v = 128 and C = 64 runs on the tensor cores, in two launches on the
+ * stream: a pass that folds the decays into the operands around each chunk's middle row G_ref and last row G_last
+ * (Q exp(G - G_ref), K exp(G_ref - G), K exp(G_last - G), W exp(-G_ref): |G_i - G_ref| must stay inside the fp32 exponent
+ * range, about 88 in natural-log units, and G must not increase along a chunk), then the scan kernel of
+ * tri_inv_chunk_scan on them.  The pass writes into stream-ordered scratch memory of four times the size of K (the
+ * driver's memory pool; returned behind the scan); TRI_INV_ERR_CUDA if it cannot be had.  Every other shape and fp32
+ * storage run on the CUDA cores in fp32 (d_k <= 256), where the exponent is taken of each difference and G is not
+ * restricted.
  */
 int tri_inv_chunk_scan_kda(const void* Q, const void* K, const void* W, const void* U, const float* G, const float* S0,
                            void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream);
