@@ -131,11 +131,11 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   const uint32_t sU = smem_u32(smem + cfg::OFF_U), sKa = smem_u32(smem + cfg::OFF_KA);
   float* sEl = sG;                 // per-channel form: exp(G_last) [3][128], then exp(G_ref) [3][128]
   float* sEr = sG + 3 * D;
-  // copies (TMA):            bar_a (W and Q), bar_kb (K beside S^T), bar_u0 / bar_u1 (U, chunks in turn)
+  // copies (TMA):            bar_a (W, Q, the K beside S^T and, per-channel form, K^), bar_u0 / bar_u1 (U, chunks in turn)
   // products done (commit):  bar_t1 (P1), bar_s (P3), bar_pu (PU)
   // operands written:        bar_sr (S^T by the compute warps, the next chunk's g by the gate warp), bar_ut (U~ and U~',
   //                          chain warps), bar_p (P, output warps); one arrival per warp
-  const uint32_t bar_a = smem_u32(smem + cfg::OFF_BAR), bar_kb = bar_a + 8, bar_ka = bar_a + 16, bar_t1 = bar_a + 24,
+  const uint32_t bar_a = smem_u32(smem + cfg::OFF_BAR), bar_t1 = bar_a + 24,
                  bar_s = bar_a + 32, bar_pu = bar_a + 40, bar_sr = bar_a + 48, bar_ut = bar_a + 56, bar_p = bar_a + 64,
                  bar_u0 = bar_a + 72, bar_u1 = bar_a + 88, bar_ud = bar_a + 96;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -212,7 +212,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   auto issue_wq = [&](int c) {
     const uint32_t dst = sA + (c & 1) * cfg::A_TILE;
     const int tok0 = beg + c * C;
-    mbar_expect_tx(bar_a, 32768u);
+    mbar_expect_tx(bar_a, 32768u + 16384u + (KDA ? 16384u : 0u));   // with the K copies below: one barrier, one wait
     tma_load_2d(dst, &tmW, bar_a, h * D, tok0);
     tma_load_2d(dst + 8192, &tmQ, bar_a, h * D, tok0);
     tma_load_2d(dst + cfg::A_BOX, &tmW, bar_a, h * D + 64, tok0);
@@ -221,15 +221,13 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   auto issue_kb = [&](int c) {
     const uint32_t dst = sB + (c & 1) * cfg::B_TILE + DVS * 128;
     const int tok0 = beg + c * C;
-    mbar_expect_tx(bar_kb, 16384u);
-    tma_load_2d(dst, &tmK, bar_kb, h * D, tok0);
-    tma_load_2d(dst + cfg::B_BOX, &tmK, bar_kb, h * D + 64, tok0);
+    tma_load_2d(dst, &tmK, bar_a, h * D, tok0);
+    tma_load_2d(dst + cfg::B_BOX, &tmK, bar_a, h * D + 64, tok0);
   };
   // per-channel form: K^ of chunk c, the MN-major A operand of P3, into the tile of c's parity
   auto issue_ka = [&](int c) {
-    mbar_expect_tx(bar_ka, 16384u);
-    tma_load_2d(sKa + (c & 1) * 16384, &tmKL, bar_ka, h * D, beg + c * C);
-    tma_load_2d(sKa + (c & 1) * 16384 + 8192, &tmKL, bar_ka, h * D + 64, beg + c * C);
+    tma_load_2d(sKa + (c & 1) * 16384, &tmKL, bar_a, h * D, beg + c * C);
+    tma_load_2d(sKa + (c & 1) * 16384 + 8192, &tmKL, bar_a, h * D + 64, beg + c * C);
   };
   // U of chunk c: the 64-column box that holds this CTA's slice, into the buffer of c's parity
   auto issue_u = [&](int c) {
@@ -284,9 +282,9 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     mbar_init(bar_p, NT / 64);
     fence_mbar_init();
     if (!misaligned) {
-      if constexpr (KDA) issue_ka(0);
-      issue_wq(0);
+      issue_wq(0);   // (announces the bytes of all three copies on their common barrier)
       issue_kb(0);
+      if constexpr (KDA) issue_ka(0);
       issue_u(0);
     }
   }
@@ -335,14 +333,12 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                      dPa = umma_desc(sP - 8192, 16, 1024);               // 128 rows: 64 of whatever lies before P (results unused), then P
       uint32_t ph = 0;
       for (int c = 0; c < n_chunks; ++c) {
-        // the copies land long before the compute threads are done: check them first, S last
+        // the copies land long before the compute threads are done: check them first, S last (one barrier for all of
+        // a chunk's copies: every wait costs this thread some 90 cycles, and its phase has to be over anyway before
+        // the copies of the next chunk are announced on it, below)
         TL(9);
         if (!mbar_wait_bounded(bar_a, ph)) { failed = true; break; }
         TL(7);
-        if (!mbar_wait_bounded(bar_kb, ph)) { failed = true; break; }
-        // (a barrier's phase has to be over before the copy of the next chunk is announced on it, below)
-        if (KDA && !mbar_wait_bounded(bar_ka, ph)) { failed = true; break; }
-        TL(8);
         if (!mbar_wait_bounded(bar_sr, ph)) { failed = true; break; }
         tc_fence_after();
         TL(0);
@@ -356,10 +352,10 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         // into the other tiles, whose last readers (P1 and P3 of the chunk before this one; for U the chain warps, a
         // chunk ago) were done before the arrivals on bar_sr seen above: nothing to wait for.
         if (c + 1 < n_chunks) {
+          issue_wq(c + 1);
+          issue_kb(c + 1);
           if constexpr (KDA) issue_ka(c + 1);
           issue_u(c + 1);
-          issue_kb(c + 1);
-          issue_wq(c + 1);
         }
         TL(2);
         if (!mbar_wait_bounded(bar_ud, ph)) { failed = true; break; }

@@ -71,8 +71,8 @@ def main():
 SCAN_COMPUTE = ["loop top", "last chunk's O written", "P1 seen", "chain: U tile seen | output: P loads done", "chain: W S loaded",
                 "chain: U~' arrived | output: first 16 rows of P", "chain: U~ arrived | output: P arrived", "P3 seen", "state updated",
                 "S^T stored", "S^T arrived"]
-SCAN_CONTROL = ["state operand seen", "P1 issued", "copies issued", "U~' seen", "P3 issued", "U~ and P seen", "PU issued", "W/Q copy seen",
-                "K copy seen", "loop top"]
+SCAN_CONTROL = ["state operand seen", "P1 issued", "copies issued", "U~' seen", "P3 issued", "U~ and P seen", "PU issued", "copies seen",
+                "", "loop top"]
 
 
 def scan_chunk(b, wl, inp, d):
