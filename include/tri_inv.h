@@ -319,6 +319,19 @@ int tri_inv_selftest_wait_timeout(const void* K, const void* V, const float* bet
                                   uint64_t wait_limit_ns, int* counters_idle, void* cuda_stream);
 
 /*
+ * The same for the tensor-core chunk scan (bf16, d_k = d_v = 128, C = 64; no step of the paper's method): tri_inv_chunk_scan
+ * (zero initial state, scale 1, final state not returned) with every device-side wait limited to wait_limit_ns nanoseconds
+ * and with the first thread block -- sequence 0, head 0, the first slice of value columns -- leaving out the state-update
+ * product of its second chunk.  The block's waits run out one after the other (each warp gives up at its next wait and
+ * leaves its loop), it raises the status word, frees its tensor memory and returns; what it had written of O stays (its
+ * first chunk), the rest of its columns of sequence 0, head 0 is undefined.  All other blocks finish as usual.  The limit
+ * should leave a tile copy time to land (tens of microseconds are plenty).  The call synchronises the stream; afterwards
+ * tri_inv_last_device_status() reads TRI_INV_ERR_DEVICE_TIMEOUT (once), and the library is usable as before.
+ */
+int tri_inv_selftest_scan_wait_timeout(const void* Q, const void* K, const void* W, const void* U, const float* g, void* O,
+                                       const tri_inv_desc* desc, uint64_t wait_limit_ns, void* cuda_stream);
+
+/*
  * Self-test of the bounds-checking build (no step of the paper's method).  tri_inv_fused (block recursion) with the token
  * bound that the debug build's checks use understated by one chunk: the buffers are as large as the descriptor says, so
  * no access is out of range either way.  In the bounds-checking build (libtri_inv_debug.so) the work items of the last

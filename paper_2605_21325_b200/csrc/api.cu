@@ -257,7 +257,8 @@ int tri_inv_build_kda(const void* K, const float* G, const float* beta, float* A
 namespace {
 // Shared body of the two chunk-scan entry points: exactly one of g (scalar gate) and G (per-channel gate) is given.
 int chunk_scan_any(const void* Q, const void* K, const void* W, const void* U, const float* g, const float* G, const float* S0,
-                   void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream) {
+                   void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream,
+                   unsigned long long wait_limit_ns = 0, int test_stall = 0) {
   int rc = check_desc(desc, true);
   if (rc) return rc;
   if (!Q || !K || !W || !U || (!g && !G) || !O) return TRI_INV_ERR_INVALID_ARG;
@@ -270,6 +271,7 @@ int chunk_scan_any(const void* Q, const void* K, const void* W, const void* U, c
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   ScanParams p{};
   p.U = U; p.g = g; p.G = G; p.S0 = S0; p.O = O; p.S_out = S_out; p.scale = scale;
+  p.wait_limit_ns = wait_limit_ns; p.test_stall = test_stall;
   p.H = desc->H; p.T = desc->T;
   p.n_seqs = desc->cu_seqlens ? desc->n_seqs : desc->B;
   cudaError_t err;
@@ -337,6 +339,18 @@ int tri_inv_chunk_scan_kda(const void* Q, const void* K, const void* W, const vo
                            void* O, float* S_out, float scale, const tri_inv_desc* desc, void* cuda_stream) {
   if (!G) return TRI_INV_ERR_INVALID_ARG;
   return chunk_scan_any(Q, K, W, U, nullptr, G, S0, O, S_out, scale, desc, cuda_stream);
+}
+
+int tri_inv_selftest_scan_wait_timeout(const void* Q, const void* K, const void* W, const void* U, const float* g, void* O,
+                                       const tri_inv_desc* desc, uint64_t wait_limit_ns, void* cuda_stream) {
+  int rc = check_desc(desc, true);
+  if (rc) return rc;
+  if (!g || wait_limit_ns == 0) return TRI_INV_ERR_INVALID_ARG;
+  // only the tensor-core kernel has the stall hook
+  if (desc->kv_dtype != TRI_INV_BF16 || desc->d_k != 128 || desc->d_v != 128 || desc->C != 64) return TRI_INV_ERR_UNSUPPORTED;
+  rc = chunk_scan_any(Q, K, W, U, g, nullptr, nullptr, O, nullptr, 1.f, desc, cuda_stream, wait_limit_ns, 1);
+  if (rc) return rc;
+  return cudaStreamSynchronize((cudaStream_t)cuda_stream) == cudaSuccess ? TRI_INV_OK : TRI_INV_ERR_CUDA;
 }
 
 int tri_inv_fused_kda(const void* K, const void* V, const float* G, const float* beta,

@@ -113,6 +113,8 @@ struct ScanParams {
   int* status;
   int H, T, n_seqs;
   float scale;
+  unsigned long long wait_limit_ns;   // limit of every device-side wait of the tensor-core scan; 0: two seconds
+  int test_stall;                     // self-test: the first CTA leaves out the second product of its second chunk
 };
 cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t stream);
 cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,

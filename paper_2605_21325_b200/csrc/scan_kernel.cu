@@ -138,6 +138,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   const uint32_t bar_a = smem_u32(smem + cfg::OFF_BAR), bar_t1 = bar_a + 24,
                  bar_s = bar_a + 32, bar_pu = bar_a + 40, bar_sr = bar_a + 48, bar_ut = bar_a + 56, bar_p = bar_a + 64,
                  bar_u0 = bar_a + 72, bar_u1 = bar_a + 88, bar_ud = bar_a + 96;
+  const unsigned long long lim = p.wait_limit_ns ? p.wait_limit_ns : kWaitLimitNs;   // every wait of the kernel gives up after this long
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool control = warp == 8;
   const bool gate_warp = warp == 9;              // brings g of the chunks to come into shared memory
@@ -337,9 +338,9 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         // a chunk's copies: every wait costs this thread some 90 cycles, and its phase has to be over anyway before
         // the copies of the next chunk are announced on it, below)
         TL(9);
-        if (!mbar_wait_bounded(bar_a, ph)) { failed = true; break; }
+        if (!mbar_wait_bounded(bar_a, ph, lim)) { failed = true; break; }
         TL(7);
-        if (!mbar_wait_bounded(bar_sr, ph)) { failed = true; break; }
+        if (!mbar_wait_bounded(bar_sr, ph, lim)) { failed = true; break; }
         tc_fence_after();
         TL(0);
 #pragma unroll
@@ -358,16 +359,20 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
           issue_u(c + 1);
         }
         TL(2);
-        if (!mbar_wait_bounded(bar_ud, ph)) { failed = true; break; }
+        if (!mbar_wait_bounded(bar_ud, ph, lim)) { failed = true; break; }
         tc_fence_after();
         TL(3);
+        // self-test (ScanParams::test_stall): the first CTA leaves out this product in its second chunk, so that the
+        // waits for it, and then every other wait of the CTA, run out
+        if (!(p.test_stall && blockIdx.x == 0 && c == 1)) {
 #pragma unroll
-        for (int ks = 0; ks < C / 16; ++ks)   // 16 tokens (2048 bytes of either operand) per step
-          umma_bf16(tmem + cfg::TM_DS, dKa + (((c & 1) * (KDA ? 16384 : cfg::B_TILE) + ks * 2048) >> 4),
-                    (KDA ? dUt : dUd) + ((ks * 2048) >> 4), idesc_p3, ks > 0);   // per-channel form: U~ itself, the decay is in K^
-        umma_commit(bar_s);
+          for (int ks = 0; ks < C / 16; ++ks)   // 16 tokens (2048 bytes of either operand) per step
+            umma_bf16(tmem + cfg::TM_DS, dKa + (((c & 1) * (KDA ? 16384 : cfg::B_TILE) + ks * 2048) >> 4),
+                      (KDA ? dUt : dUd) + ((ks * 2048) >> 4), idesc_p3, ks > 0);   // per-channel form: U~ itself, the decay is in K^
+          umma_commit(bar_s);
+        }
         TL(4);
-        if (!mbar_wait_bounded(bar_ut, ph) || !mbar_wait_bounded(bar_p, ph)) { failed = true; break; }
+        if (!mbar_wait_bounded(bar_ut, ph, lim) || !mbar_wait_bounded(bar_p, ph, lim)) { failed = true; break; }
         tc_fence_after();
         TL(5);
 #pragma unroll
@@ -386,7 +391,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     warp_arrive(bar_sr, lane);   // g of the first chunk (written before the CTA barrier above)
     for (int c = 0; c + 1 < n_chunks && !misaligned; ++c) {
       // the buffer of c + 1 held g of c - 1: every compute warp has left that chunk once the arrivals that end it are in
-      if (c > 0 && !mbar_wait_bounded(bar_sr, (uint32_t)(c & 1))) { failed = true; break; }
+      if (c > 0 && !mbar_wait_bounded(bar_sr, (uint32_t)(c & 1), lim)) { failed = true; break; }
       if constexpr (KDA) {
         // The vectors run one chunk further ahead than g: exp(G_ref) of chunk c + 1 is read at the end of chunk c (it
         // scales the S^T operand), so it has to be in place, and announced by an arrival, a chunk earlier.  Those of
@@ -408,7 +413,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     // O = scale * (gamma_i QS + P U~) of the previous chunk (the PU accumulator starts from gamma_i QS): written
     // while the next chunk's first product runs
     auto write_output = [&](uint32_t parity) -> bool {
-      if (!mbar_wait_bounded(bar_pu, parity)) return false;
+      if (!mbar_wait_bounded(bar_pu, parity, lim)) return false;
       tc_fence_after();
       __nv_bfloat16* Og = reinterpret_cast<__nv_bfloat16*>(p.O);
       float pu[2][NTW][4];
@@ -443,7 +448,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       }
       TL(1);
 
-      if (!mbar_wait_bounded(bar_t1, ph)) { failed = true; break; }
+      if (!mbar_wait_bounded(bar_t1, ph, lim)) { failed = true; break; }
       tc_fence_after();
       TL(2);
       // (this chunk's g was written by the gate warp during the last chunk: read only after the wait above,
@@ -453,7 +458,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         // ---- U~ = U - W S  ->  bf16 operands [token rows][value columns]: first the decay-scaled U~' that the chain
         // waits for (its own arrival), then U~ itself for the third product
         const int mi = lane >> 3, r = lane & 7;
-        if (!mbar_wait_bounded((c & 1) ? bar_u1 : bar_u0, (uint32_t)((c >> 1) & 1))) { failed = true; break; }   // landed a chunk ago
+        if (!mbar_wait_bounded((c & 1) ? bar_u1 : bar_u0, (uint32_t)((c >> 1) & 1), lim)) { failed = true; break; }   // landed a chunk ago
         TL(3);
         const uint32_t sUc = sU + (c & 1) * 8192;
         const int u_shift = DVS < 64 ? ((slice * DVS) & 63) : 0;   // a narrow slice: which part of the copied 64-column box is ours
@@ -606,7 +611,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       }
 
       // ---- state update and the bf16 operand for the next chunk
-      if (!mbar_wait_bounded(bar_s, ph)) { failed = true; break; }
+      if (!mbar_wait_bounded(bar_s, ph, lim)) { failed = true; break; }
       tc_fence_after();
       TL(7);
       {

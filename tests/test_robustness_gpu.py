@@ -85,3 +85,34 @@ def test_graph_replays_overlapping_many_plain_launches(bnd):
             x = bnd.to_numpy_f64(o)
             assert not np.isnan(x).any(), "a row was not written: two launches shared a work counter"
             assert np.abs(x - r).max() <= tol * np.abs(r).max()
+
+
+@pytest.mark.parametrize("B,H", [(1, 2), (4, 16)], ids=["narrow_slices", "wide_slices"])
+def test_scan_waits_that_run_out(bnd, B, H):
+    """The chunk-scan kernel's ten warps wait for one another through barriers only; with one product of the first thread
+    block left out (tri_inv_selftest_scan_wait_timeout, limit 100 us) every one of that block's waits must give up in turn,
+    the kernel must return with the status word raised once, the other blocks' output must be untouched by it, and the
+    next ordinary call must give the bits of the call before."""
+    inp = wl.make("scan_stall", B, 6 * 64, H, 128, 128, 64, wl.BF16, seed=631 + H)
+    dev = bnd.to_device(inp)
+    Q = bnd.kv_to_torch(wl.queries(inp, seed=632))
+    _, W, U = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], 64, method=bnd.W_DECAY, want_A=False)
+    ref, _ = bnd.chunk_scan(Q, dev["K"], W, U, dev["g"], 64, scale=1.0, want_state=False)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    O = torch.full_like(dev["V"], float("nan"))
+    bnd.selftest_scan_wait_timeout(Q, dev["K"], W, U, dev["g"], 64, wait_limit_ns=100_000, out=O)
+    assert bnd.last_device_status() == bnd.ERR_DEVICE_TIMEOUT     # raised ...
+    assert bnd.last_device_status() == 0                          # ... and cleared by the read
+    # the stalled block is (sequence 0, head 0, first slice of value columns: 32 or 64 wide); its first chunk was written
+    # before the product was left out
+    width = 32 if B * H * 4 <= torch.cuda.get_device_properties(0).multi_processor_count else 64
+    r2, o2 = ref.clone(), O.clone()
+    assert torch.equal(o2[0, :64, 0, :width].view(torch.int16), r2[0, :64, 0, :width].view(torch.int16))
+    r2[0, 64:, 0, :width] = 0
+    o2[0, 64:, 0, :width] = 0
+    assert torch.equal(r2.view(torch.int16), o2.view(torch.int16))
+    again, _ = bnd.chunk_scan(Q, dev["K"], W, U, dev["g"], 64, scale=1.0, want_state=False)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    assert torch.equal(again.view(torch.int16), ref.view(torch.int16))
