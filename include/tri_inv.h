@@ -223,9 +223,10 @@ int tri_inv_fused_kda(const void* K, const void* V, const float* G, const float*
  *     O  = scale * ((Q * Gamma) S + P U~),     S <- diag(Gamma_last) S + (K * exp(G_last - G))^T U~,
  * W and U from tri_inv_fused_kda.  bf16 with d_k = d_v = 128 and C = 64 runs on the tensor cores, in two launches on the
  * stream: a pass that folds the decays into the operands around each chunk's middle row G_ref and last row G_last
- * (Q exp(G - G_ref), K exp(G_ref - G), K exp(G_last - G), W exp(-G_ref): |G_i - G_ref| must stay inside the fp32 exponent
- * range, about 88 in natural-log units, and G must not increase along a chunk), then the scan kernel of
- * tri_inv_chunk_scan on them.  The pass writes into stream-ordered scratch memory of four times the size of K (the
+ * (Q exp(G - G_ref), K exp(G_ref - G), W exp(-G_ref), and per chunk the vectors exp(G_last), exp(G_ref),
+ * exp(G_last - G_ref): |G_i - G_ref| must stay inside the fp32 exponent range, about 88 in natural-log units, and G must
+ * not increase along a chunk), then the scan kernel of
+ * tri_inv_chunk_scan on them.  The pass writes into stream-ordered scratch memory of three times the size of K (the
  * driver's memory pool; returned behind the scan); TRI_INV_ERR_CUDA if it cannot be had.  Every other shape and fp32
  * storage run on the CUDA cores in fp32 (d_k <= 256), where the exponent is taken of each difference and G is not
  * restricted.

@@ -291,8 +291,8 @@ int chunk_scan_any(const void* Q, const void* K, const void* W, const void* U, c
   }
   void* work = nullptr;
   if (tc && G && tokens > 0) {
-    // Per-channel gate on the tensor cores: Q+, K-, K^, W- (bf16, the tensors' own shape) and the per-chunk vectors
-    // exp(G_last), exp(G_ref), in stream-ordered scratch memory that is released behind the scan.
+    // Per-channel gate on the tensor cores: Q+, K-, W- (bf16, the tensors' own shape) and the per-chunk vectors
+    // exp(G_last), exp(G_ref), exp(G_last - G_ref), in stream-ordered scratch memory that is released behind the scan.
     int max_len = desc->T;
     if (desc->cu_seqlens) {
       max_len = 0;
@@ -302,19 +302,20 @@ int chunk_scan_any(const void* Q, const void* K, const void* W, const void* U, c
     const size_t slots = (size_t)(tokens / 64) + (size_t)p.n_seqs + 1;
     const size_t vec_bytes = (slots * desc->H * 128 * sizeof(float) + 255) & ~(size_t)255;
     cudaMemPool_t pool = table_pool_for_current_device();
-    if (!pool || cudaMallocFromPoolAsync(&work, 4 * tensor_bytes + 2 * vec_bytes, pool, stream) != cudaSuccess) {
+    if (!pool || cudaMallocFromPoolAsync(&work, 3 * tensor_bytes + 3 * vec_bytes, pool, stream) != cudaSuccess) {
       if (dev_off) cudaFreeAsync(dev_off, stream);
       return TRI_INV_ERR_CUDA;
     }
     char* w = reinterpret_cast<char*>(work);
-    void *Qp = w, *Km = w + tensor_bytes, *Kl = w + 2 * tensor_bytes, *Wm = w + 3 * tensor_bytes;
-    float* EL = reinterpret_cast<float*>(w + 4 * tensor_bytes);
-    float* ER = reinterpret_cast<float*>(w + 4 * tensor_bytes + vec_bytes);
-    p.EL = EL; p.ER = ER;
-    err = launch_kda_scan_prep(p, Q, K, W, Qp, Km, Kl, Wm, EL, ER, (max_len + 63) / 64, stream);
+    void *Qp = w, *Km = w + tensor_bytes, *Wm = w + 2 * tensor_bytes;
+    float* EL = reinterpret_cast<float*>(w + 3 * tensor_bytes);
+    float* ER = reinterpret_cast<float*>(w + 3 * tensor_bytes + vec_bytes);
+    float* EX = reinterpret_cast<float*>(w + 3 * tensor_bytes + 2 * vec_bytes);
+    p.EL = EL; p.ER = ER; p.EX = EX;
+    err = launch_kda_scan_prep(p, Q, K, W, Qp, Km, Wm, EL, ER, EX, (max_len + 63) / 64, stream);
     if (err == cudaSuccess) {
       g_launches.fetch_add(1, std::memory_order_relaxed);
-      err = launch_chunk_scan(p, Qp, Km, Wm, tokens, stream, Kl);
+      err = launch_chunk_scan(p, Qp, Km, Wm, tokens, stream, true);
     }
   } else {
     err = (tc && !G) ? launch_chunk_scan(p, Q, K, W, tokens > 0 ? tokens : 1, stream)

@@ -105,7 +105,8 @@ struct ScanParams {
   const float* g;       // [tokens,H]
   const float* G;       // [tokens,H,d_k] per-channel cumulative log-decay (KDA row) or null; CUDA-core kernel and preparation kernel
   const float* EL;      // per-channel form on the tensor cores: exp(G_last) per chunk slot [slots,H,d_k] ...
-  const float* ER;      // ... and exp(G_ref), both written by the preparation kernel (slot of a chunk: first token / C + sequence index)
+  const float* ER;      // ... exp(G_ref) ...
+  const float* EX;      // ... and exp(G_last - G_ref), all written by the preparation kernel (slot of a chunk: first token / C + sequence index)
   const float* S0;      // [n_seqs,H,d_k,d_v] fp32 or null (zero state)
   void* O;              // [tokens,H,d_v], storage type of U
   float* S_out;         // [n_seqs,H,d_k,d_v] fp32 or null
@@ -118,12 +119,12 @@ struct ScanParams {
 };
 cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t stream);
 cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,
-                              cudaStream_t stream, const void* K_last = nullptr);
+                              cudaStream_t stream, bool kda = false);
 // Per-channel form: the operands of the tensor-core scan from Q, K, W (bf16, [tokens,H,128]) and G, C = 64:
-// Qp = Q exp(G - G_ref), Km = K exp(G_ref - G), Kl = K exp(G_last - G), Wm = W exp(-G_ref) and the per-chunk vectors
-// EL = exp(G_last), ER = exp(G_ref) ([slots,H,128] fp32), G_ref the middle row of each chunk, G_last its last.
-cudaError_t launch_kda_scan_prep(const ScanParams& p, const void* Q, const void* K, const void* W, void* Qp, void* Km, void* Kl,
-                                 void* Wm, float* EL, float* ER, int max_chunks_per_seq, cudaStream_t stream);
+// Qp = Q exp(G - G_ref), Km = K exp(G_ref - G), Wm = W exp(-G_ref) and the per-chunk vectors EL = exp(G_last),
+// ER = exp(G_ref), EX = exp(G_last - G_ref) ([slots,H,128] fp32), G_ref the middle row of each chunk, G_last its last.
+cudaError_t launch_kda_scan_prep(const ScanParams& p, const void* Q, const void* K, const void* W, void* Qp, void* Km, void* Wm,
+                                 float* EL, float* ER, float* EX, int max_chunks_per_seq, cudaStream_t stream);
 // The same scan on the CUDA cores, for every other shape and storage type (fp32 arithmetic).
 cudaError_t launch_chunk_scan_simt(const ScanParams& p, const void* Q, const void* K, const void* W, int d_k, int d_v, int C,
                                    int kv_dtype, cudaStream_t stream);

@@ -3,11 +3,12 @@
 // row and G_last its last row, the chunk form
 //     P_ij = sum_k Q_ik K_jk exp(G_ik - G_jk),   O = (Q exp G) S + P U~,   S <- diag(exp G_last) S + (K exp(G_last - G))^T U~
 // becomes the scalar-gate kernel's three products on
-//     Q+ = Q exp(G - G_ref),   K- = K exp(G_ref - G),   K^ = K exp(G_last - G),   W- = W exp(-G_ref)
-// (each factor within exp(+-|G over 32 tokens|); K^ <= |K|), with the state operand scaled per row by exp(G_ref):
-//     [W- ; Q+] . [diag(exp G_ref) S | K-^T]  =  [W S | . ; (Q exp G) S | Q+ K-^T].
-// One pass over Q, K, W and G writes the four bf16 tensors and, per chunk, exp(G_last) and exp(G_ref); the exponent of
-// each difference is taken once per element instead of once per (i, j, k).
+//     Q+ = Q exp(G - G_ref),   K- = K exp(G_ref - G),   W- = W exp(-G_ref)
+// (each factor within exp(+-|G over 32 tokens|)), with the state operand scaled per row by exp(G_ref),
+//     [W- ; Q+] . [diag(exp G_ref) S | K-^T]  =  [W S | . ; (Q exp G) S | Q+ K-^T],
+// and the state increment taken from K- as well: (K exp(G_last - G))^T U~ = diag(exp(G_last - G_ref)) K-^T U~.
+// One pass over Q, K, W and G writes the three bf16 tensors and, per chunk, exp(G_last), exp(G_ref) and
+// exp(G_last - G_ref); the exponent of each difference is taken once per element instead of once per (i, j, k).
 #include "common.cuh"
 
 namespace tri_inv {
@@ -19,8 +20,8 @@ constexpr float kLog2e = 1.4426950408889634f;
 struct PrepArgs {
   const __nv_bfloat16 *Q, *K, *W;
   const float* G;
-  __nv_bfloat16 *Qp, *Km, *Kl, *Wm;
-  float *EL, *ER;
+  __nv_bfloat16 *Qp, *Km, *Wm;
+  float *EL, *ER, *EX;
   const int* seq_off;
   int H, T, n_seqs;
 };
@@ -59,6 +60,8 @@ __global__ void __launch_bounds__(NT) kda_scan_prep_kernel(PrepArgs a) {
       for (int q = 0; q < 2; ++q) {
         *reinterpret_cast<float4*>(a.EL + slot + 4 * q) = make_float4(ex2f(glast[4 * q]), ex2f(glast[4 * q + 1]), ex2f(glast[4 * q + 2]), ex2f(glast[4 * q + 3]));
         *reinterpret_cast<float4*>(a.ER + slot + 4 * q) = make_float4(ex2f(gref[4 * q]), ex2f(gref[4 * q + 1]), ex2f(gref[4 * q + 2]), ex2f(gref[4 * q + 3]));
+        *reinterpret_cast<float4*>(a.EX + slot + 4 * q) = make_float4(ex2f(glast[4 * q] - gref[4 * q]), ex2f(glast[4 * q + 1] - gref[4 * q + 1]),
+                                                                      ex2f(glast[4 * q + 2] - gref[4 * q + 2]), ex2f(glast[4 * q + 3] - gref[4 * q + 3]));
       }
     }
     float wneg[8];
@@ -80,9 +83,8 @@ __global__ void __launch_bounds__(NT) kda_scan_prep_kernel(PrepArgs a) {
       const uint32_t* qw = reinterpret_cast<const uint32_t*>(&qv);
       const uint32_t* kw = reinterpret_cast<const uint32_t*>(&kv);
       const uint32_t* ww = reinterpret_cast<const uint32_t*>(&wv);
-      uint4 qo, mo, lo, wo;
-      uint32_t *qp = reinterpret_cast<uint32_t*>(&qo), *mp = reinterpret_cast<uint32_t*>(&mo), *lp = reinterpret_cast<uint32_t*>(&lo),
-               *wp = reinterpret_cast<uint32_t*>(&wo);
+      uint4 qo, mo, wo;
+      uint32_t *qp = reinterpret_cast<uint32_t*>(&qo), *mp = reinterpret_cast<uint32_t*>(&mo), *wp = reinterpret_cast<uint32_t*>(&wo);
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const float2 qf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&qw[e]));
@@ -91,12 +93,10 @@ __global__ void __launch_bounds__(NT) kda_scan_prep_kernel(PrepArgs a) {
         const float x0 = g[2 * e] - gref[2 * e], x1 = g[2 * e + 1] - gref[2 * e + 1];
         qp[e] = pack2(qf.x * ex2f(x0), qf.y * ex2f(x1));
         mp[e] = pack2(kf.x * ex2f(-x0), kf.y * ex2f(-x1));
-        lp[e] = pack2(kf.x * ex2f(glast[2 * e] - g[2 * e]), kf.y * ex2f(glast[2 * e + 1] - g[2 * e + 1]));
         wp[e] = pack2(wf.x * wneg[2 * e], wf.y * wneg[2 * e + 1]);
       }
       *reinterpret_cast<uint4*>(a.Qp + idx) = qo;
       *reinterpret_cast<uint4*>(a.Km + idx) = mo;
-      *reinterpret_cast<uint4*>(a.Kl + idx) = lo;
       *reinterpret_cast<uint4*>(a.Wm + idx) = wo;
     }
   }
@@ -104,11 +104,11 @@ __global__ void __launch_bounds__(NT) kda_scan_prep_kernel(PrepArgs a) {
 
 }  // namespace
 
-cudaError_t launch_kda_scan_prep(const ScanParams& p, const void* Q, const void* K, const void* W, void* Qp, void* Km, void* Kl,
-                                 void* Wm, float* EL, float* ER, int max_chunks_per_seq, cudaStream_t stream) {
+cudaError_t launch_kda_scan_prep(const ScanParams& p, const void* Q, const void* K, const void* W, void* Qp, void* Km, void* Wm,
+                                 float* EL, float* ER, float* EX, int max_chunks_per_seq, cudaStream_t stream) {
   PrepArgs a{reinterpret_cast<const __nv_bfloat16*>(Q), reinterpret_cast<const __nv_bfloat16*>(K), reinterpret_cast<const __nv_bfloat16*>(W), p.G,
-             reinterpret_cast<__nv_bfloat16*>(Qp), reinterpret_cast<__nv_bfloat16*>(Km), reinterpret_cast<__nv_bfloat16*>(Kl),
-             reinterpret_cast<__nv_bfloat16*>(Wm), EL, ER, p.seq_off, p.H, p.T, p.n_seqs};
+             reinterpret_cast<__nv_bfloat16*>(Qp), reinterpret_cast<__nv_bfloat16*>(Km), reinterpret_cast<__nv_bfloat16*>(Wm), EL, ER, EX,
+             p.seq_off, p.H, p.T, p.n_seqs};
   const long long gx = (long long)p.n_seqs * p.H;
   if (gx > 0x7fffffffLL) return cudaErrorInvalidValue;
   if (gx == 0 || max_chunks_per_seq <= 0) return cudaSuccess;

@@ -44,11 +44,13 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 // KDA: the per-channel form (one decay per key feature, the KDA row of Table 1).  Its decays are folded into the
 // operands beforehand (kda_scan_prep_kernel, scan_kda_prep.cu): with G_ref the middle row of a chunk and G_last its last,
-//     W- = W exp(-G_ref),  Q+ = Q exp(G - G_ref),  K- = K exp(G_ref - G),  K^ = K exp(G_last - G),
-// P1 = [W- ; Q+] . [(diag(exp G_ref) S) | K-^T] gives W S, (Q exp G) S and the decayed Q K^T at once, P3 = K^^T U~ is
-// the state increment (no second, decay-scaled copy of U~), and S decays by exp(G_last) per row.  The kernel then
-// differs from the scalar-gate one only in where its operands come from and in a few scalings: the S^T operand is
-// scaled per row by exp(G_ref) of the coming chunk, P needs no decay, K^ has a tile of its own.
+//     W- = W exp(-G_ref),  Q+ = Q exp(G - G_ref),  K- = K exp(G_ref - G),
+// P1 = [W- ; Q+] . [(diag(exp G_ref) S) | K-^T] gives W S, (Q exp G) S and the decayed Q K^T at once; P3 = K-^T U~,
+// scaled per row by exp(G_last - G_ref), is the state increment (K exp(G_last - G) = K- exp(G_last - G_ref): no second,
+// decay-scaled copy of U~, and the K rows of the B tile serve as in the scalar form); S decays by exp(G_last) per row.
+// The kernel then differs from the scalar-gate one only in where its operands come from and in a few scalings: the
+// S^T operand is scaled per row by exp(G_ref) of the coming chunk, P needs no decay, the state update has two per-row
+// factors.
 template <int DVS, bool KDA = false>
 struct ScanCfg {
   static constexpr int CW = DVS / 2;                     // value columns per compute warp
@@ -61,15 +63,14 @@ struct ScanCfg {
   // B operand of P1: [S^T ; K], two boxes of (DVS + 64) rows x 128 B
   static constexpr int OFF_B = 2 * A_TILE, B_BOX = N1 * 128, B_TILE = 2 * B_BOX;
   // (the K rows of the B tile are also the MN-major A operand of P3: the tile stays whole until the chunk after next)
-  static constexpr int OFF_KA = OFF_B + 2 * B_TILE;      // per-channel form: K^ tiles of two chunks in turn (MN-major A operand of P3)
-  static constexpr int OFF_P = OFF_KA + (KDA ? 2 * 16384 : 0);   // P, the lower half of PU's A operand; the unused upper half is whatever precedes it
+  static constexpr int OFF_P = OFF_B + 2 * B_TILE;       // P, the lower half of PU's A operand; the unused upper half is whatever precedes it
   static constexpr int OFF_UT = OFF_P + 8192;            // U~  bf16 [64 tokens][DVS], boxes of 64 columns (MN-major B)
   static constexpr int U_BYTES = 8192 * (DVS > 64 ? DVS / 64 : 1);   // a narrower slice fills the first DVS columns of one box
   static constexpr int OFF_UD = OFF_UT + U_BYTES;        // U~' bf16, same layout
   static constexpr int OFF_U = OFF_UD + U_BYTES;         // U tiles of two chunks in turn: bf16 [64 tokens][64 columns], as copied
   static constexpr int OFF_G = OFF_U + 2 * 8192;         // g * log2(e): 2 x 64 floats; column factors: 2 x 64 floats
-                                                         // per-channel form: exp(G_last) and exp(G_ref), 128 floats each, of three chunks in turn
-  static constexpr int OFF_BAR = OFF_G + (KDA ? 3072 : 1024);   // 12 mbarriers, tensor-memory slot
+                                                         // per-channel form: exp(G_last), exp(G_ref), exp(G_last - G_ref), 128 floats each, of three chunks in turn
+  static constexpr int OFF_BAR = OFF_G + (KDA ? 4608 : 1024);   // 12 mbarriers, tensor-memory slot
   static constexpr int SMEM = OFF_BAR + 128;
   static constexpr int TM_P1 = 0, TM_DS = N1, TM_PU = N1 + DVS;
   static constexpr int TMEM_COLS = (N1 + 2 * DVS) <= 256 ? 256 : 512;
@@ -118,8 +119,7 @@ __host__ __device__ constexpr uint32_t umma_idesc_ab(int M, int N, int a_mn, int
 template <int DVS, bool KDA>
 __global__ void __launch_bounds__(NT + 64, ScanCfg<DVS, KDA>::CTAS_PER_SM)
 chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmQ,
-                  const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmU,
-                  const __grid_constant__ CUtensorMap tmKL, ScanParams p) {
+                  const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmU, ScanParams p) {
   using cfg = ScanCfg<DVS, KDA>;
   constexpr int NTW = cfg::NTW, CW = cfg::CW, NS = D / DVS;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -128,9 +128,10 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + cfg::OFF_BAR + 80);
   const uint32_t sA = smem_u32(smem + cfg::OFF_A), sB = smem_u32(smem + cfg::OFF_B);
   const uint32_t sP = smem_u32(smem + cfg::OFF_P), sUt = smem_u32(smem + cfg::OFF_UT), sUd = smem_u32(smem + cfg::OFF_UD);
-  const uint32_t sU = smem_u32(smem + cfg::OFF_U), sKa = smem_u32(smem + cfg::OFF_KA);
-  float* sEl = sG;                 // per-channel form: exp(G_last) [3][128], then exp(G_ref) [3][128]
+  const uint32_t sU = smem_u32(smem + cfg::OFF_U);
+  float* sEl = sG;                 // per-channel form: exp(G_last) [3][128], exp(G_ref) [3][128], exp(G_last - G_ref) [3][128]
   float* sEr = sG + 3 * D;
+  float* sEx = sG + 6 * D;
   // copies (TMA):            bar_a (W, Q, the K beside S^T and, per-channel form, K^), bar_u0 / bar_u1 (U, chunks in turn)
   // products done (commit):  bar_t1 (P1), bar_s (P3), bar_pu (PU)
   // operands written:        bar_sr (S^T by the compute warps, the next chunk's g by the gate warp), bar_ut (U~ and U~',
@@ -213,7 +214,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   auto issue_wq = [&](int c) {
     const uint32_t dst = sA + (c & 1) * cfg::A_TILE;
     const int tok0 = beg + c * C;
-    mbar_expect_tx(bar_a, 32768u + 16384u + (KDA ? 16384u : 0u));   // with the K copies below: one barrier, one wait
+    mbar_expect_tx(bar_a, 32768u + 16384u);   // with the K copy below: one barrier, one wait
     tma_load_2d(dst, &tmW, bar_a, h * D, tok0);
     tma_load_2d(dst + 8192, &tmQ, bar_a, h * D, tok0);
     tma_load_2d(dst + cfg::A_BOX, &tmW, bar_a, h * D + 64, tok0);
@@ -224,11 +225,6 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     const int tok0 = beg + c * C;
     tma_load_2d(dst, &tmK, bar_a, h * D, tok0);
     tma_load_2d(dst + cfg::B_BOX, &tmK, bar_a, h * D + 64, tok0);
-  };
-  // per-channel form: K^ of chunk c, the MN-major A operand of P3, into the tile of c's parity
-  auto issue_ka = [&](int c) {
-    tma_load_2d(sKa + (c & 1) * 16384, &tmKL, bar_a, h * D, beg + c * C);
-    tma_load_2d(sKa + (c & 1) * 16384 + 8192, &tmKL, bar_a, h * D + 64, beg + c * C);
   };
   // U of chunk c: the 64-column box that holds this CTA's slice, into the buffer of c's parity
   auto issue_u = [&](int c) {
@@ -261,16 +257,18 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 
   // per-channel form: exp(G_last) and exp(G_ref) of a chunk (128 floats each, written by the preparation kernel at the
   // chunk's slot), by the gate warp: lane l brings features 4 l .. 4 l + 3 of both; three chunks' worth are kept in turn
-  auto fetch_e = [&](int c, float4 (&ev)[2]) {
+  auto fetch_e = [&](int c, float4 (&ev)[3]) {
     const size_t slot = (size_t)((beg + c * C) / C + s);
     ev[0] = *reinterpret_cast<const float4*>(p.EL + (slot * p.H + h) * D + 4 * lane);
     ev[1] = *reinterpret_cast<const float4*>(p.ER + (slot * p.H + h) * D + 4 * lane);
+    ev[2] = *reinterpret_cast<const float4*>(p.EX + (slot * p.H + h) * D + 4 * lane);
   };
-  auto store_e = [&](int c, const float4 (&ev)[2]) {
+  auto store_e = [&](int c, const float4 (&ev)[3]) {
     *reinterpret_cast<float4*>(sEl + (c % 3) * D + 4 * lane) = ev[0];
     *reinterpret_cast<float4*>(sEr + (c % 3) * D + 4 * lane) = ev[1];
+    *reinterpret_cast<float4*>(sEx + (c % 3) * D + 4 * lane) = ev[2];
   };
-  float4 e_raw[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+  float4 e_raw[3] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
   float g_raw[2] = {0.f, 0.f};   // gate warp: g of the chunk it stores next
   if (tid == NT) {
     prefetch_tmap(&tmW); prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmU);
@@ -285,7 +283,6 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     if (!misaligned) {
       issue_wq(0);   // (announces the bytes of all three copies on their common barrier)
       issue_kb(0);
-      if constexpr (KDA) issue_ka(0);
       issue_u(0);
     }
   }
@@ -329,7 +326,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       constexpr uint32_t idesc_p3 = umma_idesc_ab(128, DVS, 1, 1);       // K tile MN-major, U~' MN-major
       constexpr uint32_t idesc_pu = umma_idesc_ab(128, DVS, 0, 1);       // [any;P] K-major, U~ MN-major
       // descriptors differ from these bases only in the address field (bits 0..13, units of 16 bytes)
-      const uint64_t dA = umma_desc(sA, 16, 1024), dB = umma_desc(sB, 16, 1024), dKa = KDA ? umma_desc(sKa, 8192, 1024) : umma_desc(sB + DVS * 128, cfg::B_BOX, 1024),   // MN-major: the K^ tile, or the K rows of the B tile
+      const uint64_t dA = umma_desc(sA, 16, 1024), dB = umma_desc(sB, 16, 1024), dKa = umma_desc(sB + DVS * 128, cfg::B_BOX, 1024),   // the K rows of the B tile, MN-major
                      dUd = umma_desc(sUd, 8192, 1024), dUt = umma_desc(sUt, 8192, 1024),
                      dPa = umma_desc(sP - 8192, 16, 1024);               // 128 rows: 64 of whatever lies before P (results unused), then P
       uint32_t ph = 0;
@@ -355,7 +352,6 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         if (c + 1 < n_chunks) {
           issue_wq(c + 1);
           issue_kb(c + 1);
-          if constexpr (KDA) issue_ka(c + 1);
           issue_u(c + 1);
         }
         TL(2);
@@ -367,8 +363,8 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         if (!(p.test_stall && blockIdx.x == 0 && c == 1)) {
 #pragma unroll
           for (int ks = 0; ks < C / 16; ++ks)   // 16 tokens (2048 bytes of either operand) per step
-            umma_bf16(tmem + cfg::TM_DS, dKa + (((c & 1) * (KDA ? 16384 : cfg::B_TILE) + ks * 2048) >> 4),
-                      (KDA ? dUt : dUd) + ((ks * 2048) >> 4), idesc_p3, ks > 0);   // per-channel form: U~ itself, the decay is in K^
+            umma_bf16(tmem + cfg::TM_DS, dKa + (((c & 1) * cfg::B_TILE + ks * 2048) >> 4),
+                      (KDA ? dUt : dUd) + ((ks * 2048) >> 4), idesc_p3, ks > 0);   // per-channel form: U~ itself, the decay is in K- and in the update
           umma_commit(bar_s);
         }
         TL(4);
@@ -616,12 +612,14 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       TL(7);
       {
         const float gl = ex2_approx(g_last);
-        float el[2][2];   // per-channel form: exp(G_last) of this thread's four rows of S
+        float el[2][2], ex[2][2];   // per-channel form: exp(G_last) and exp(G_last - G_ref) of this thread's four rows of S
         if constexpr (KDA) {
 #pragma unroll
           for (int lg = 0; lg < 2; ++lg) {
             el[lg][0] = sEl[(c % 3) * D + krow_w + 16 * lg + gq];
             el[lg][1] = sEl[(c % 3) * D + krow_w + 16 * lg + gq + 8];
+            ex[lg][0] = sEx[(c % 3) * D + krow_w + 16 * lg + gq];
+            ex[lg][1] = sEx[(c % 3) * D + krow_w + 16 * lg + gq + 8];
           }
         }
         float ds[2][NTW][4];
@@ -633,7 +631,8 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 #pragma unroll
           for (int nt = 0; nt < NTW; ++nt)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) S[lg][nt][e] = fmaf(KDA ? el[lg][e >> 1] : gl, S[lg][nt][e], ds[lg][nt][e]);
+            for (int e = 0; e < 4; ++e)
+              S[lg][nt][e] = KDA ? fmaf(el[lg][e >> 1], S[lg][nt][e], ex[lg][e >> 1] * ds[lg][nt][e]) : fmaf(gl, S[lg][nt][e], ds[lg][nt][e]);
         TL(8);
         if (has_next) {
           write_state_operand((c + 1) & 1, sEr + ((c + 1) % 3) * D);   // that tile's last reader was P1 of the chunk before this one
@@ -666,7 +665,7 @@ __global__ void __launch_bounds__(256) seq_offsets_kernel(int* out, const __grid
 
 template <int DVS, bool KDA>
 cudaError_t launch_scan_one(const ScanParams& p, const CUtensorMap& tmW, const CUtensorMap& tmQ, const CUtensorMap& tmK,
-                            const CUtensorMap& tmU, const CUtensorMap& tmKL, cudaStream_t stream) {
+                            const CUtensorMap& tmU, cudaStream_t stream) {
   using cfg = ScanCfg<DVS, KDA>;
   static std::mutex mu;
   static bool ready[64] = {false};
@@ -684,7 +683,7 @@ cudaError_t launch_scan_one(const ScanParams& p, const CUtensorMap& tmW, const C
   }
   const long long grid = (long long)p.n_seqs * p.H * (D / DVS);
   if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
-  chunk_scan_kernel<DVS, KDA><<<(int)grid, NT + 64, cfg::SMEM, stream>>>(tmW, tmQ, tmK, tmU, tmKL, p);
+  chunk_scan_kernel<DVS, KDA><<<(int)grid, NT + 64, cfg::SMEM, stream>>>(tmW, tmQ, tmK, tmU, p);
   return cudaGetLastError();
 }
 
@@ -711,19 +710,19 @@ cudaError_t launch_seq_offsets(int* dev_out, const tri_inv_desc* d, cudaStream_t
 // per pair instead, still at most one per SM: the per-chunk chain of a CTA is a little shorter (7 % on one sequence
 // of 32 heads), and every output column is computed by the same operations in the same order either way.  With more
 // pairs than that the narrow slices would share SMs and repeat the Q K^T part of the first product: measured slower.
-// K_last != nullptr selects the per-channel form: Q, K, W are then the prepared operands Q+, K-, W- and K_last is K^
-// (scan_kda_prep.cu), with p.EL / p.ER the per-chunk vectors.
+// kda selects the per-channel form: Q, K, W are then the prepared operands Q+, K-, W- (scan_kda_prep.cu), with p.EL,
+// p.ER, p.EX the per-chunk vectors.
 cudaError_t launch_chunk_scan(const ScanParams& p, const void* Q, const void* K, const void* W, long long tokens,
-                              cudaStream_t stream, const void* K_last) {
-  CUtensorMap tmW, tmQ, tmK, tmU, tmKL;
+                              cudaStream_t stream, bool kda) {
+  CUtensorMap tmW, tmQ, tmK, tmU;
   if (!make_tmap(&tmW, W, tokens, p.H, D, C, 2) || !make_tmap(&tmQ, Q, tokens, p.H, D, C, 2) || !make_tmap(&tmK, K, tokens, p.H, D, C, 2) ||
-      !make_tmap(&tmU, p.U, tokens, p.H, D, C, 2) || !make_tmap(&tmKL, K_last ? K_last : K, tokens, p.H, D, C, 2))
+      !make_tmap(&tmU, p.U, tokens, p.H, D, C, 2))
     return cudaErrorUnknown;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
   const bool narrow = (long long)p.n_seqs * p.H * 4 <= sms;
-  if (K_last) return narrow ? launch_scan_one<32, true>(p, tmW, tmQ, tmK, tmU, tmKL, stream) : launch_scan_one<64, true>(p, tmW, tmQ, tmK, tmU, tmKL, stream);
-  return narrow ? launch_scan_one<32, false>(p, tmW, tmQ, tmK, tmU, tmKL, stream) : launch_scan_one<64, false>(p, tmW, tmQ, tmK, tmU, tmKL, stream);
+  if (kda) return narrow ? launch_scan_one<32, true>(p, tmW, tmQ, tmK, tmU, stream) : launch_scan_one<64, true>(p, tmW, tmQ, tmK, tmU, stream);
+  return narrow ? launch_scan_one<32, false>(p, tmW, tmQ, tmK, tmU, stream) : launch_scan_one<64, false>(p, tmW, tmQ, tmK, tmU, stream);
 }
 
 }  // namespace tri_inv
