@@ -226,8 +226,9 @@ int tri_inv_fused_kda(const void* K, const void* V, const float* G, const float*
  * (Q exp(G - G_ref), K exp(G_ref - G), W exp(-G_ref), and per chunk the vectors exp(G_last), exp(G_ref),
  * exp(G_last - G_ref): |G_i - G_ref| must stay inside the fp32 exponent range, about 88 in natural-log units, and G must
  * not increase along a chunk), then the scan kernel of
- * tri_inv_chunk_scan on them.  The pass writes into stream-ordered scratch memory of three times the size of K (the
- * driver's memory pool; returned behind the scan); TRI_INV_ERR_CUDA if it cannot be had.  Every other shape and fp32
+ * tri_inv_chunk_scan on them.  The pass writes into stream-ordered scratch memory of three times the size of K (from a
+ * memory pool that the library keeps per device: handed back to the pool behind the scan and reused by later calls, so
+ * it stays reserved for the life of the process); TRI_INV_ERR_CUDA if it cannot be had.  Every other shape and fp32
  * storage run on the CUDA cores in fp32 (d_k <= 256), where the exponent is taken of each difference and G is not
  * restricted.
  */

@@ -563,3 +563,44 @@ def test_per_channel_chunk_form_equals_its_recurrence():
         O3, S3 = oracle.recurrence_ex(Q, x.K, x.V, x.beta, None, 64, G=Gs, scale=0.5, S0=S0, cu_seqlens=cu_seqlens)
         O4, S4 = oracle.gdn_recurrence(Q, x.K, x.V, x.beta, x.g, 64, scale=0.5, S0=S0, cu_seqlens=cu_seqlens)
         assert np.abs(O3 - O4).max() < 1e-12 and np.abs(S3 - S4).max() < 1e-12
+
+
+def test_per_channel_chunk_form_on_rescaled_operands():
+    """The form the tensor-core scan runs for the KDA row: with G_ref the middle row of a chunk and G_last its last,
+        [W exp(-G_ref) ; Q exp(G - G_ref)] . [diag(exp G_ref) S | (K exp(G_ref - G))^T]
+    holds W S, (Q exp G) S and the decayed Q K^T, and the state increment is diag(exp(G_last - G_ref)) (K exp(G_ref - G))^T U~.
+    Written out here in fp64 with three plain matrix products per chunk and compared with the oracle's chunk form (which takes
+    the exponent of every difference) on ragged sequences: the two must agree to rounding."""
+    rng = np.random.default_rng(91)
+    C, H, d = 8, 2, 6
+    cu = np.array([0, 5, 5, 21, 38], np.int32)
+    T = int(cu[-1])
+    Q, K, W, U = (rng.standard_normal((1, T, H, d)) for _ in range(4))
+    G = np.zeros((1, T, H, d))
+    for beg, end in zip(cu[:-1], cu[1:]):
+        for t0 in range(beg, end, C):
+            t1 = min(t0 + C, end)
+            G[0, t0:t1] = -np.cumsum(rng.uniform(0.0, 0.6, size=(t1 - t0, H, d)), axis=0)   # cumulative log-decay inside the chunk
+    S0 = rng.standard_normal((len(cu) - 1, H, d, d))
+    O_ref, S_ref = oracle.chunk_scan_kda(Q, K, W, U, G, C, scale=0.7, S0=S0, cu_seqlens=cu)
+    O = np.zeros_like(O_ref)
+    S_out = np.zeros_like(S_ref)
+    for s in range(len(cu) - 1):
+        for h in range(H):
+            S = S0[s, h].copy()
+            for t0 in range(cu[s], cu[s + 1], C):
+                t1 = min(t0 + C, cu[s + 1])
+                r = t1 - t0
+                g = G[0, t0:t1, h]
+                g_ref, g_last = g[r // 2], g[r - 1]
+                Wm = W[0, t0:t1, h] * np.exp(-g_ref)
+                Qp = Q[0, t0:t1, h] * np.exp(g - g_ref)
+                Km = K[0, t0:t1, h] * np.exp(g_ref - g)
+                P1 = np.concatenate([Wm, Qp]) @ np.concatenate([np.exp(g_ref)[:, None] * S, Km.T], axis=1)   # one product
+                Ut = U[0, t0:t1, h] - P1[:r, :d]
+                P = np.tril(P1[r:, d:])
+                O[0, t0:t1, h] = 0.7 * (P1[r:, :d] + P @ Ut)
+                S = np.exp(g_last)[:, None] * S + np.exp(g_last - g_ref)[:, None] * (Km.T @ Ut)
+            S_out[s, h] = S
+    assert np.abs(O - O_ref).max() <= 1e-12 * max(1.0, np.abs(O_ref).max())
+    assert np.abs(S_out - S_ref).max() <= 1e-12 * max(1.0, np.abs(S_ref).max())
