@@ -169,3 +169,46 @@ def test_per_channel_scan_resumes_bit_for_bit(bnd):
         torch.cuda.synchronize()
         assert bnd.last_device_status() == 0
         assert torch.equal(torch.cat([O1, O2], dim=1).view(torch.int16), O.view(torch.int16)) and torch.equal(S2, S)
+
+
+def test_per_channel_layer_captured_in_a_cuda_graph(bnd):
+    """The four launches of the per-channel layer forward (build, WY, operand preparation, scan) and the scan's scratch
+    memory (stream-ordered allocation and release) can be captured once and replayed on new inputs in the same buffers."""
+    inp = wl.make("kda_graph", 2, 4 * 64, 4, 128, 128, 64, wl.BF16, seed=1500)
+    G = wl.per_channel_gate(inp, seed=68)
+    Q = wl.queries(inp, seed=69)
+    dev = bnd.to_device(inp)
+    Gd, Qd = torch.from_numpy(G).cuda(), bnd.kv_to_torch(Q)
+    A = torch.empty((2, 4 * 64, 4, 64), dtype=torch.float32, device="cuda")
+    W, U, O = torch.empty_like(dev["K"]), torch.empty_like(dev["V"]), torch.empty_like(dev["V"])
+
+    def forward():
+        bnd.fused_kda(dev["K"], dev["V"], Gd, dev["beta"], 64, out=(A, W, U))
+        bnd.chunk_scan_kda(Qd, dev["K"], W, U, Gd, 64, scale=0.125, out=O, want_state=False)
+
+    forward()                       # first use: per-device set-up happens outside the capture
+    torch.cuda.synchronize()
+    O_eager = O.clone()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            forward()
+    torch.cuda.synchronize()
+    O.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    assert torch.equal(O.view(torch.int16), O_eager.view(torch.int16))
+    inp2 = wl.make("kda_graph2", 2, 4 * 64, 4, 128, 128, 64, wl.BF16, seed=1501)
+    G2 = wl.per_channel_gate(inp2, seed=70)
+    dev2 = bnd.to_device(inp2)
+    for k in ("K", "V", "beta"):
+        dev[k].copy_(dev2[k])
+    Gd.copy_(torch.from_numpy(G2).cuda())
+    graph.replay()
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    O_ref, _ = oracle.recurrence_ex(Q, inp2.K, inp2.V, inp2.beta, None, 64, G=G2, scale=0.125)
+    assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= 2e-2
