@@ -12,7 +12,8 @@
 // (tokens 0..63 against reference 1 have G_ref1 - G_j <= 0, G being non-increasing along a chunk: no overflow).
 // An M = 64 accumulator puts rows 16 q .. 16 q + 15 on tensor-memory lanes 32 q .. 32 q + 15, so warp w of eight reads
 // the 16 rows it also inverts the diagonal block of.  Gate, 16 x 16 leaves, three merge levels and the store of A follow
-// the scalar-gate kernels; the fp32 matrix reuses the G tile's space.  One CTA of eight warps per SM.
+// the scalar-gate kernels.  Two CTAs of eight warps per SM: G (64 KB per item in fp32) passes through two 16 KB slots,
+// one box of 32 channels at a time, and the fp32 matrix lies over the K- operand and the slots once they are spent.
 // Every mbarrier wait is bounded; on expiry the kernel raises the status word, frees its tensor memory and returns.
 #include "tc_device.cuh"
 
@@ -25,27 +26,28 @@ constexpr int KM_ROWS = 192, KM_BOX = KM_ROWS * 128;   // K- operand: tokens 0..
 constexpr int G_BOX = C * 128;                 // one box of the G tile: 128 rows x 32 channels (fp32)
 constexpr int OFF_K = 0;                       // K tile, then K+                      (32 KB)
 constexpr int OFF_KM = OFF_K + 2 * K_BOX;      // K-                                    (48 KB)
-constexpr int OFF_LEAF = OFF_KM;               // series-leaf scratch: inside K-, dead once the products are through
+constexpr int OFF_G = OFF_KM + 2 * KM_BOX;     // two slots for boxes of G             (2 x 16 KB)
+constexpr int OFF_X = OFF_KM;                  // the fp32 N / X matrix (67,584 B) over K- and the slots, once they are spent
+constexpr int X_BYTES = C * LD * 4;
+constexpr int OFF_LEAF = OFF_X + X_BYTES;      // series-leaf scratch: behind the matrix, in the second slot's space
 constexpr int LEAF_LD = 20;
-constexpr int OFF_G = OFF_KM + 2 * KM_BOX;     // G tile (64 KB); the fp32 N / X matrix over it (67,584 B)
-constexpr int OFF_X = OFF_G;
-constexpr int OFF_BETA = OFF_G + 67 * 1024;
-constexpr int OFF_BAR = OFF_BETA + C * 4;      // bar_k, bar_mma, bar_g, TMEM slot
-constexpr int SMEM_BYTES = OFF_BAR + 32;
+constexpr int OFF_BETA = OFF_G + 2 * G_BOX;
+constexpr int OFF_BAR = OFF_BETA + C * 4;      // bar_k, bar_mma, bar_g0, bar_g1, TMEM slot
+constexpr int SMEM_BYTES = OFF_BAR + 40;
 constexpr int TMEM_COLS = 256;                 // columns 0..63: rows 0..63; columns 64..191: rows 64..127
-static_assert(C * LD * 4 <= 67 * 1024, "the fp32 matrix must fit its space");
-static_assert(NW * 16 * LEAF_LD * 4 <= 2 * KM_BOX, "leaf scratch must fit inside the K- tile");
+static_assert(OFF_LEAF + NW * 16 * LEAF_LD * 4 <= OFF_BETA, "the fp32 matrix and the leaf scratch must fit over K- and the slots");
 static_assert(OFF_G % 1024 == 0 && OFF_KM % 1024 == 0 && KM_BOX % 1024 == 0, "swizzled tiles start on 1 KiB");
+static_assert(2 * (SMEM_BYTES + 1024 + 8) <= 228 * 1024, "two CTAs per SM");
 
 template <bool KG>   // KG: also write K * exp(G) into p.W (the fused call)
-__global__ void __launch_bounds__(NT, 1) kda_build_kernel_c128(const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(NT, 2) kda_build_kernel_c128(const __grid_constant__ CUtensorMap tmK,
                                                                const __grid_constant__ CUtensorMap tmG, KParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
   float* sX = reinterpret_cast<float*>(smem + OFF_X);
   float* sBeta = reinterpret_cast<float*>(smem + OFF_BETA);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 24);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 32);
   const uint32_t sK = smem_u32(smem + OFF_K), sKm = smem_u32(smem + OFF_KM), sG = smem_u32(smem + OFF_G);
-  const uint32_t bar_k = smem_u32(smem + OFF_BAR), bar_mma = bar_k + 8, bar_g = bar_k + 16;
+  const uint32_t bar_k = smem_u32(smem + OFF_BAR), bar_mma = bar_k + 8, bar_g0 = bar_k + 16, bar_g1 = bar_k + 24;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, t = lane & 3;
   const int rb = warp;                         // this warp's 16 rows: half rb >> 2, tensor-memory quadrant rb & 3
@@ -58,11 +60,12 @@ __global__ void __launch_bounds__(NT, 1) kda_build_kernel_c128(const __grid_cons
 #pragma unroll
     for (int bx = 0; bx < 2; ++bx) tma_load_2d(sK + bx * K_BOX, &tmK, bar_k, h * D + 64 * bx, tok0);
   };
-  auto issue_g = [&](int tok0, int h) {
+  // box bx of G (channels 32 bx .. + 31) into slot bx & 1
+  auto issue_g = [&](int tok0, int h, int bx) {
+    const uint32_t bar = (bx & 1) ? bar_g1 : bar_g0;
     fence_proxy_async();
-    mbar_expect_tx(bar_g, 4u * G_BOX);
-#pragma unroll
-    for (int bx = 0; bx < 4; ++bx) tma_load_2d(sG + bx * G_BOX, &tmG, bar_g, h * D + 32 * bx, tok0);
+    mbar_expect_tx(bar, (uint32_t)G_BOX);
+    tma_load_2d(sG + (bx & 1) * G_BOX, &tmG, bar, h * D + 32 * bx, tok0);
   };
   auto fetch_beta = [&](int tok0, int rows, int h) -> float {
     return (tid < C && tid < rows) ? p.beta[(size_t)(tok0 + tid) * p.H + h] : 0.f;
@@ -74,7 +77,10 @@ __global__ void __launch_bounds__(NT, 1) kda_build_kernel_c128(const __grid_cons
     const bool any = (int)blockIdx.x < total && !misaligned;
     if (any) locate(p, C, blockIdx.x, tok0, rows, h);
     if (tid == 64) { prefetch_tmap(&tmK); mbar_init(bar_k, 1); fence_mbar_init(); if (any) issue_k(tok0, h); }
-    if (tid == 96) { prefetch_tmap(&tmG); mbar_init(bar_g, 1); fence_mbar_init(); if (any) issue_g(tok0, h); }
+    if (tid == 96) {
+      prefetch_tmap(&tmG); mbar_init(bar_g0, 1); mbar_init(bar_g1, 1); fence_mbar_init();
+      if (any) { issue_g(tok0, h, 0); issue_g(tok0, h, 1); }
+    }
     if (tid == 0) { mbar_init(bar_mma, 1); fence_mbar_init(); }
     if (any) beta_next = fetch_beta(tok0, rows, h);
   }
@@ -87,16 +93,16 @@ __global__ void __launch_bounds__(NT, 1) kda_build_kernel_c128(const __grid_cons
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tmem_rows = tmem + ((32u * (warp & 3)) << 16);
-  uint32_t ph = 0, ph_mma = 0;   // K and G complete once per item: one parity for both
+  uint32_t ph = 0, ph_mma = 0;   // K completes once per item; each slot of G twice (parities 0, 1 within every item)
   // Give-up protocol as in the other kernels: a thread whose bounded wait runs out remembers it, skips its later waits
   // and finishes the item on whatever data is there; it raises the CTA's flag before the item's last barrier, behind
   // which every thread reads it, so the whole CTA leaves the loop at one place.
-  __shared__ int s_gave_up;
+  int* const gave_up = reinterpret_cast<int*>(smem + OFF_BAR + 36);   // (in the dynamic block: a static one would cost 1 KiB)
   bool bad = false;
   auto wait = [&](uint32_t bar, uint32_t parity) {
     if (!bad) bad = !mbar_wait_bounded(bar, parity, p.wait_limit_ns);
   };
-  if (tid == 0) s_gave_up = 0;   // read only behind later barriers
+  if (tid == 0) *gave_up = 0;   // read only behind later barriers
   bool k_pending = false;        // thread 64: a K tile has been requested that nobody has waited for yet
 
   for (int item = blockIdx.x; item < total && !misaligned; item += gridDim.x) {
@@ -117,13 +123,17 @@ __global__ void __launch_bounds__(NT, 1) kda_build_kernel_c128(const __grid_cons
     // ---- 2. K+ = K * 2^x over K, K- = K * 2^-x, x = (G - G_ref) log2(e), G_ref the middle row of the row's half of
     // the chunk; tokens 0..63 also against the second half's reference.  Rows past the chunk's end are zero.
     wait(bar_k, ph);
-    wait(bar_g, ph);
     const int rows0 = rows < 64 ? rows : 64, rows1 = rows - rows0;
     const int rref0 = rows0 >> 1, rref1 = 64 + (rows1 >> 1);   // (rref1 is used only where rows1 > 0)
-#pragma unroll 2
-    for (int m = 0; m < 8; ++m) {
+    // G comes through two slots, a box of 32 channels at a time: boxes 0 and 1 were requested before the item, boxes
+    // 2 and 3 follow into the slots that boxes 0 and 1 leave (behind a barrier: every thread has read the slot).
+#pragma unroll 1
+    for (int bx = 0; bx < 4; ++bx) {
+    wait((bx & 1) ? bar_g1 : bar_g0, (uint32_t)(bx >> 1));
+#pragma unroll
+    for (int m = 0; m < 2; ++m) {
       const int e = tid + m * NT;
-      const int r = e >> 4, cf = e & 15;                 // row, 16-byte chunk of 8 features
+      const int r = e >> 2, cf = 4 * bx + (e & 3);       // row, 16-byte chunk of 8 features (four per box of G)
       const int hf = r >> 6;
       const uint32_t sw = (uint32_t)((((cf & 7) ^ (r & 7)) << 4));   // (rows r, r + 64 and r + 128 share r & 7)
       const uint32_t koff = (uint32_t)((cf >> 3) * K_BOX + r * 128) + sw;
@@ -133,7 +143,7 @@ __global__ void __launch_bounds__(NT, 1) kda_build_kernel_c128(const __grid_cons
         uint4 kv;
         asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kv.x), "=r"(kv.y), "=r"(kv.z), "=r"(kv.w) : "r"(sK + koff));
         const int q0 = 2 * (cf & 3);                     // first of the two float4 of G for these 8 channels
-        const uint32_t gbox = sG + (cf >> 2) * G_BOX;
+        const uint32_t gbox = sG + (bx & 1) * G_BOX;
         const int rref = hf ? rref1 : rref0;
         const bool cross = !hf && rows1 > 0;             // a token of the first half that the second half's rows see
         float gv[8], gr[8], gx[8];
@@ -171,6 +181,11 @@ __global__ void __launch_bounds__(NT, 1) kda_build_kernel_c128(const __grid_cons
       asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sK + koff), "r"(kp.x), "r"(kp.y), "r"(kp.z), "r"(kp.w) : "memory");
       asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + moff), "r"(km.x), "r"(km.y), "r"(km.z), "r"(km.w) : "memory");
       if (!hf) asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + moff + 64 * 128), "r"(km1.x), "r"(km1.y), "r"(km1.z), "r"(km1.w) : "memory");
+    }
+    if (bx < 2) {
+      __syncthreads();
+      if (tid == 96 && !bad) issue_g(tok0, h, bx + 2);
+    }
     }
     fence_proxy_async();
     tc_fence_before();
@@ -248,15 +263,15 @@ __global__ void __launch_bounds__(NT, 1) kda_build_kernel_c128(const __grid_cons
         if (i < rows) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
       }
     }
-    if (bad) s_gave_up = 1;
+    if (bad) *gave_up = 1;
     tc_fence_before();
     __syncthreads();   // the fp32 matrix has been read by everyone: the next G tile may land in its space
-    if (s_gave_up) break;   // uniform: every thread reads the flag behind the same barrier
+    if (*gave_up) break;   // uniform: every thread reads the flag behind the same barrier
     ph ^= 1;
-    if (tid == 96 && has_next) issue_g(nx_tok0, nx_h);
+    if (tid == 96 && has_next) { issue_g(nx_tok0, nx_h, 0); issue_g(nx_tok0, nx_h, 1); }
   }
   if (bad || misaligned) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
-  if (s_gave_up) {
+  if (*gave_up) {
     // what may still be in flight: the K tile requested for the next item (the G tile is requested after the exit test)
     if (tid == 64 && k_pending) mbar_wait_bounded(bar_k, ph ^ 1, p.wait_limit_ns);
   }
@@ -281,6 +296,8 @@ cudaError_t launch_kda_tc_c128(const KParams& p, cudaStream_t stream) {
     if (!n_sm_of[dev]) {
       if ((e = cudaFuncSetAttribute(kda_build_kernel_c128<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) != cudaSuccess) return e;
       if ((e = cudaFuncSetAttribute(kda_build_kernel_c128<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(kda_build_kernel_c128<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(kda_build_kernel_c128<true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
       int sms = 0;
       if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
       n_sm_of[dev] = sms > 0 ? sms : 1;
@@ -292,7 +309,8 @@ cudaError_t launch_kda_tc_c128(const KParams& p, cudaStream_t stream) {
   if (!make_tmap(&tmK, p.K, tokens, p.H, D, C, 2)) return cudaErrorUnknown;
   if (!make_tmap(&tmG, p.G, tokens, p.H, D, C, 4)) return cudaErrorUnknown;
   long long total = (long long)p.n_chunks * p.H;
-  int grid = (int)(total < n_sm ? total : n_sm);
+  const long long cap = 2LL * n_sm;   // two CTAs per SM
+  int grid = (int)(total < cap ? total : cap);
   if (grid == 0) return cudaSuccess;
   if (p.W) kda_build_kernel_c128<true><<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
   else kda_build_kernel_c128<false><<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
