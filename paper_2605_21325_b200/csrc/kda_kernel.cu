@@ -134,9 +134,9 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid
         const uint32_t* kw = reinterpret_cast<const uint32_t*>(&kv);
         uint32_t* pw = reinterpret_cast<uint32_t*>(&kp);
         uint32_t* mw = reinterpret_cast<uint32_t*>(&km);
-#pragma unroll
         uint4 kg;                                         // K * exp(G): the key operand of the WY step that follows (fused call)
         uint32_t* gw = reinterpret_cast<uint32_t*>(&kg);
+#pragma unroll
         for (int q = 0; q < 4; ++q) {
           const float2 kf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kw[q]));
           const float x0 = (gv[2 * q] - gr[2 * q]) * 1.4426950408889634f, x1 = (gv[2 * q + 1] - gr[2 * q + 1]) * 1.4426950408889634f;
