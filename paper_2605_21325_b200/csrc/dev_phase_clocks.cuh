@@ -23,6 +23,10 @@ __device__ __forceinline__ unsigned dev_smid() { unsigned r; asm volatile("mov.u
     ph_t = now;                                                                   \
   } while (0)
 
+// Chunk scan: the clock of one chunk's steps (the 21st chunk of thread block 0), per warp, as a snapshot in the
+// same status words; `warp`, `lane` and the chunk index `c` are the kernel's own variables at the mark.
+#define TL(k) do { if (blockIdx.x == 0 && c == 20 && lane == 0) p.status[8 + 12 * warp + (k)] = (int)clock64(); } while (0)
+
 #ifdef TRI_INV_DEV_DEFINE_EXPORTS
 // One translation unit (the one that defines TRI_INV_DEV_DEFINE_EXPORTS) carries the read-back calls.
 extern "C" int tri_inv_debug_cta_times(unsigned long long* out, int n) {

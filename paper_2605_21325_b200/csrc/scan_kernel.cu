@@ -31,14 +31,6 @@
 namespace tri_inv {
 namespace {
 
-// Development build only: the clock of one chunk's steps, per warp, in the device status words (a snapshot that the
-// development tools read back); nothing otherwise.
-#ifdef TRI_INV_PHASE_CLOCKS
-#define TL(k) do { if (blockIdx.x == 0 && c == 20 && lane == 0) p.status[8 + 12 * warp + (k)] = (int)clock64(); } while (0)
-#else
-#define TL(k) do {} while (0)
-#endif
-
 constexpr int C = 64, D = 128, NT = 256;   // NT compute threads (8 warps) + the control warp + the gate warp
 constexpr float kLog2e = 1.4426950408889634f;
 

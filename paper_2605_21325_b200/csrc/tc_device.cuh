@@ -15,6 +15,7 @@
 #define CTA_MARK(k) do {} while (0)
 #define PHASE_BEGIN() do {} while (0)
 #define PHASE(k) do {} while (0)
+#define TL(k) do {} while (0)
 #endif
 
 namespace tri_inv {
