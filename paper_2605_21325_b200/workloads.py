@@ -143,11 +143,12 @@ def make_raw(name, B, T, H, d, C, kv_dtype, seed, cu_seqlens=None):
                   {"kind": "raw", "seed": seed})
 
 
-def per_channel_gate(inp: Inputs, seed: int) -> np.ndarray:
+def per_channel_gate(inp: Inputs, seed: int, mean: float = 2.0) -> np.ndarray:
     """Cumulative per-channel log-decay G [B,T,H,d_k] fp32 for the per-channel (KDA-type) variant:
-    log sigmoid(N(2,1)) per token and channel, summed along the tokens of each chunk."""
+    log sigmoid(N(mean,1)) per token and channel, summed along the tokens of each chunk.  mean = 2 is the configurations'
+    gate (about -0.15 per token); a lower mean decays faster (mean = -0.5: about -1 per token)."""
     rng = np.random.default_rng(seed)
-    z = rng.standard_normal((inp.B * inp.T, inp.H * inp.d_k), dtype=np.float32) + np.float32(2.0)
+    z = rng.standard_normal((inp.B * inp.T, inp.H * inp.d_k), dtype=np.float32) + np.float32(mean)
     ls = (-np.log1p(np.exp(-z.astype(np.float64)))).astype(np.float32)
     G = _chunk_cumsum(ls, inp.seq_bounds(), inp.C)
     return np.ascontiguousarray(G.reshape(inp.B, inp.T, inp.H, inp.d_k))

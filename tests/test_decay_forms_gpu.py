@@ -212,3 +212,38 @@ def test_per_channel_layer_captured_in_a_cuda_graph(bnd):
     assert bnd.last_device_status() == 0
     O_ref, _ = oracle.recurrence_ex(Q, inp2.K, inp2.V, inp2.beta, None, 64, G=G2, scale=0.125)
     assert max_ratio(bnd.to_numpy_f64(O), O_ref) <= 2e-2
+
+
+@pytest.mark.parametrize("C", [64, 128])
+def test_per_channel_forms_under_strong_decay(bnd, C):
+    """A gate that falls by about one (natural-log unit) per token and channel: G reaches -60 .. -75 at the end of a chunk of
+    64 and twice that at 128, so that exp(G_i - G_j) spans the whole fp32 range and exp(-G) alone would overflow.  The
+    tensor-core kernels scale rows against a reference row in the middle of the chunk (of each half at C = 128), which keeps
+    every factor within exp(+-|G over 32 tokens|): A, W, U must still match the fp64 oracle, and at C = 64 the scan on the
+    prepared operands must still match the token-by-token recurrence."""
+    inp = wl.make("strong", 2, 3 * C + 11, 3, 128, 128, C, wl.BF16, seed=1600 + C)
+    G = wl.per_channel_gate(inp, seed=71, mean=-0.5)
+    assert G.min() < (-100.0 if C == 128 else -50.0)
+    A_ref, N_ref = oracle.build_A_kda(inp.K, G, inp.beta, C, return_N=True)
+    Kd = inp.kv_as_f32("K").astype(np.float64)
+    W_ref, _ = oracle.wy(A_ref, Kd * np.exp(G.astype(np.float64)), None, inp.beta, C)
+    _, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, C)
+    dev = bnd.to_device(inp)
+    Gd = torch.from_numpy(G).cuda()
+    A, W, U = bnd.fused_kda(dev["K"], dev["V"], Gd, dev["beta"], C)
+    torch.cuda.synchronize()
+    assert bnd.last_device_status() == 0
+    a = A.cpu().numpy()
+    assert np.isfinite(a).all() and structure_errors(a, inp) == (0, 0)
+    assert max_ratio(a, A_ref) <= 2e-3 and max_residual(a, N_ref, inp) <= 5e-3
+    assert max_ratio(bnd.to_numpy_f64(W), W_ref) <= 1e-2 and max_ratio(bnd.to_numpy_f64(U), U_ref) <= 1e-2
+    if C == 64:
+        Q = wl.queries(inp, seed=72)
+        S0 = wl.initial_state(inp, seed=73)
+        O, S = bnd.chunk_scan_kda(bnd.kv_to_torch(Q), dev["K"], W, U, Gd, C, scale=0.5, S0=torch.from_numpy(S0).cuda())
+        torch.cuda.synchronize()
+        assert bnd.last_device_status() == 0
+        O_ref, S_ref = oracle.recurrence_ex(Q, inp.K, inp.V, inp.beta, None, C, G=G, scale=0.5, S0=S0)
+        o, s_ = bnd.to_numpy_f64(O), bnd.to_numpy_f64(S)
+        assert np.isfinite(o).all() and np.isfinite(s_).all()
+        assert max_ratio(o, O_ref) <= 2e-2 and max_ratio(s_, S_ref) <= 2e-2
