@@ -128,7 +128,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   // products done (commit):  bar_t1 (P1), bar_s (P3), bar_pu (PU)
   // operands written:        bar_sr (S^T by the compute warps, the next chunk's g by the gate warp), bar_ut (U~ and U~',
   //                          chain warps), bar_p (P, output warps); one arrival per warp
-  const uint32_t bar_a = smem_u32(smem + cfg::OFF_BAR), bar_t1 = bar_a + 24,
+  const uint32_t bar_a = smem_u32(smem + cfg::OFF_BAR), bar_exit = bar_a + 8, bar_t1 = bar_a + 24,
                  bar_s = bar_a + 32, bar_pu = bar_a + 40, bar_sr = bar_a + 48, bar_ut = bar_a + 56, bar_p = bar_a + 64,
                  bar_u0 = bar_a + 72, bar_u1 = bar_a + 88, bar_ud = bar_a + 96;
   const unsigned long long lim = p.wait_limit_ns ? p.wait_limit_ns : kWaitLimitNs;   // every wait of the kernel gives up after this long
@@ -322,12 +322,14 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                      dUd = umma_desc(sUd, 8192, 1024), dUt = umma_desc(sUt, 8192, 1024),
                      dPa = umma_desc(sP - 8192, 16, 1024);               // 128 rows: 64 of whatever lies before P (results unused), then P
       uint32_t ph = 0;
+      int pending = 0;   // chunk whose copies have been requested and not yet seen to land (-1: none)
       for (int c = 0; c < n_chunks; ++c) {
         // the copies land long before the compute threads are done: check them first, S last (one barrier for all of
         // a chunk's copies: every wait costs this thread some 90 cycles, and its phase has to be over anyway before
         // the copies of the next chunk are announced on it, below)
         TL(9);
         if (!mbar_wait_bounded(bar_a, ph, lim)) { failed = true; break; }
+        pending = -1;
         TL(7);
         if (!mbar_wait_bounded(bar_sr, ph, lim)) { failed = true; break; }
         tc_fence_after();
@@ -345,6 +347,7 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
           issue_wq(c + 1);
           issue_kb(c + 1);
           issue_u(c + 1);
+          pending = c + 1;
         }
         TL(2);
         if (!mbar_wait_bounded(bar_ud, ph, lim)) { failed = true; break; }
@@ -369,6 +372,17 @@ chunk_scan_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         umma_commit(bar_pu);
         TL(6);
         ph ^= 1;
+      }
+      if (failed) {
+        // A wait has run out and this CTA is about to give up its shared and tensor memory: what it may still have in
+        // flight is waited for first, again with a limit -- the copies requested for the coming chunk (U on its own
+        // barrier) and every product issued so far (a commit on a spare barrier).
+        if (pending >= 0) {
+          mbar_wait_bounded(bar_a, (uint32_t)(pending & 1), lim);
+          mbar_wait_bounded((pending & 1) ? bar_u1 : bar_u0, (uint32_t)((pending >> 1) & 1), lim);
+        }
+        umma_commit(bar_exit);
+        mbar_wait_bounded(bar_exit, 0u, lim);
       }
     }
   } else if (gate_warp) {
