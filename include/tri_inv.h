@@ -121,7 +121,9 @@ enum {
   /* Newton-Schulz iteration count, 1..15, in bits 12..15 (0 = default) */
 #define TRI_INV_NS_ITERS(m) (((m) & 0xf) << 12)
   /* flag: run the plain fp32 CUDA-core kernel even where a tensor-core kernel
-   * exists (same results up to rounding; for cross-checks and odd shapes). */
+   * exists (same results up to rounding; for cross-checks and odd shapes).  Tensor-core kernels exist for bf16
+   * storage with d_k = d_v = 128 at C = 64 and 128 (every scheme but Newton-Schulz) and with d_k = d_v = 64 at
+   * C = 64 (block recursion, with or without TRI_INV_LEAF_SERIES, no other flag). */
   TRI_INV_FORCE_SIMT = 0x10000,
   /* flag, tri_inv_fused / tri_inv_fused_raw only: W = A diag(beta) diag(exp g) K, the decay-weighted factor
    * that the chunk form of the layer's recurrence subtracts from U (tri_inv_chunk_scan consumes it).  U is

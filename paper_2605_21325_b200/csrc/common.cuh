@@ -93,6 +93,7 @@ cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handle
 cudaError_t launch_tc_c64_br(const KParams& p, cudaStream_t stream, bool raw);
 cudaError_t launch_tc_c64_series(const KParams& p, cudaStream_t stream, bool raw);
 cudaError_t launch_tc_c64_build(const KParams& p, cudaStream_t stream);
+cudaError_t launch_tc_c64_d64(const KParams& p, cudaStream_t stream);   // head dimension 64
 cudaError_t launch_tc_c128_br(const KParams& p, cudaStream_t stream, bool raw);
 cudaError_t launch_tc_c128_series(const KParams& p, cudaStream_t stream, bool raw);
 cudaError_t launch_tc_refine(const KParams& p, int C, cudaStream_t stream, bool raw);

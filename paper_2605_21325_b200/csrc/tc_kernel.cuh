@@ -96,7 +96,8 @@ template <int C, int D, bool SER, bool RAW, bool BO, bool REF, bool H16, int VAR
 __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SER, BO, REF, H16>::CTAS_PER_SM) tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmU,
                                                                              const __grid_constant__ CUtensorMap tmV, const __grid_constant__ KParams p) {
   using cfg = Cfg<C, D, SER, BO, REF, H16>;
-  static_assert(D == 128, "tiles are two 64-feature boxes wide");
+  static_assert(D == 128 || (D == 64 && C == 64 && !SER && !RAW && !REF && !H16),
+                "tiles are two 64-feature boxes wide; one box only for the plain block recursion at C = 64");
   constexpr int LD = cfg::LD;
   constexpr int TMEM_COLS = cfg::TMEM_COLS;
   extern __shared__ __align__(1024) uint8_t smem[];  // swizzled tiles need a 1024-byte aligned base
@@ -986,7 +987,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       if (has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);  // consumed at the top of the next item
 
       // ---- 7. WY: [W | U] = A' . [K | V] with the staged tiles as the MN-major B operand
-      constexpr int NWU = (C == 64) ? 128 : 256;   // columns per MMA: C = 64 runs W then U through the same 128 columns
+      constexpr int NWU = (C == 64) ? D : 2 * D;   // columns per MMA: C = 64 runs W then U through the same D columns
+      static_assert(D == 128 || (D == 64 && C == 64), "head dimensions: 128, or 64 at C = 64");
       constexpr uint32_t idesc_wy = umma_idesc(C, NWU, 1);
       auto issue_wy = [&](uint32_t b_tile) {
 #pragma unroll
@@ -1023,7 +1025,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       if (C == 64 && need_v) {
         float f0[8][4], f1[8][4];
         tmem_ld_16x64(f0, tmem_rows);
-        tmem_ld_16x64(f1, tmem_rows + 64);
+        if constexpr (D == 128) tmem_ld_16x64(f1, tmem_rows + 64);
         tmem_wait_ld();
         tc_fence_before();
         __syncthreads();  // every warp holds its rows of W in registers: U may overwrite the columns
@@ -1032,14 +1034,14 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         }
         if (tid == kTidK && has_next) issue_k(nx_tok0, nx_h);  // K's last reader (the W product) is done
         store_frag_piece_bf16(f0, stage, lane, w_row0, row_stride, rows - row0, &tmW, h * D + 0, tok0 + row0);
-        store_frag_piece_bf16(f1, stage, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
+        if constexpr (D == 128) store_frag_piece_bf16(f1, stage, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
         PHASE(9);
         wait(bar_mma, ph_mma);
         ph_mma ^= 1;
         tc_fence_after();
         PHASE(10);
         tmem_ld_16x64(f0, tmem_rows);
-        tmem_ld_16x64(f1, tmem_rows + 64);
+        if constexpr (D == 128) tmem_ld_16x64(f1, tmem_rows + 64);
         tmem_wait_ld();
         tc_fence_before();
         __syncthreads();  // all MMAs done and all accumulators read: tiles, A' and tensor memory are free
@@ -1054,7 +1056,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         }
         store_frag_piece_bf16(f0, stage, lane, u_row0, row_stride, rows - row0, &tmU, h * D + 0, tok0 + row0);
         // second staging tile: the A' operand's space, whose last reader (the U product) has completed
-        store_frag_piece_bf16<1>(f1, sAp + warp * 2048, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
+        if constexpr (D == 128) store_frag_piece_bf16<1>(f1, sAp + warp * 2048, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
       } else {
         // C = 128 (W and U side by side in 256 columns) or W only
         if (cfg::ALIAS && tid == kTidK && has_next && !load_a) issue_k(nx_tok0, nx_h);  // all MMAs on the tiles are done
@@ -1063,8 +1065,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         const uint32_t stage2 = cfg::ALIAS ? stage + cfg::NW * 2048 : stage;
         constexpr int KEEP = cfg::ALIAS ? 1 : 0;
         store_piece_bf16<0>(tmem_rows, stage, lane, w_row0, row_stride, rows - row0, &tmW, h * D, tok0 + row0);
-        store_piece_bf16<KEEP>(tmem_rows + 64, stage2, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
-        if (need_v) {
+        if constexpr (D == 128) store_piece_bf16<KEEP>(tmem_rows + 64, stage2, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
+        if (need_v && C == 128) {
           store_piece_bf16<KEEP>(tmem_rows + 128, stage, lane, u_row0, row_stride, rows - row0, &tmU, h * D, tok0 + row0);
           store_piece_bf16<KEEP>(tmem_rows + 192, stage2, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
         }

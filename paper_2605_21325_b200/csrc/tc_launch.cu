@@ -74,11 +74,17 @@ cudaError_t launch_tc(const KParams& p, int C, cudaStream_t stream, bool* handle
   if (p.kv_dtype != TRI_INV_BF16) return cudaSuccess;
   const bool series = (p.method & TRI_INV_METHOD_MASK) == TRI_INV_PRODUCT_SERIES;
   if ((p.method & TRI_INV_METHOD_MASK) == TRI_INV_NEWTON_SCHULZ) return cudaSuccess;   // CUDA-core kernel only
-  if (p.d_k != 128 || ((p.ops & kDoWY) && p.V && p.d_v != 128)) return cudaSuccess;
   if (C != 64 && C != 128) return cudaSuccess;
+  const bool raw = (p.ops & (kRaw | kWDecay)) != 0;  // both need the variant that rewrites the K tile
+  if (p.d_k == 64 && C == 64 && !series && !raw && !(p.method & (TRI_INV_REFINE | TRI_INV_OPERANDS_F16)) &&
+      !((p.ops & kDoWY) && p.V && p.d_v != 64)) {
+    // head dimension 64: block recursion (and series leaves) of the plain calls; everything else stays on the CUDA cores
+    *handled = true;
+    return launch_tc_c64_d64(p, stream);
+  }
+  if (p.d_k != 128 || ((p.ops & kDoWY) && p.V && p.d_v != 128)) return cudaSuccess;
   // the stride of the 2-D view (H * d * 2 bytes) is a multiple of 16 because d is a multiple of 8
   *handled = true;
-  const bool raw = (p.ops & (kRaw | kWDecay)) != 0;  // both need the variant that rewrites the K tile
   if ((p.method & TRI_INV_REFINE) && !(p.ops & kLoadA)) return launch_tc_refine(p, C, stream, raw);
   if ((p.method & TRI_INV_OPERANDS_F16) && series) return launch_tc_series_f16(p, C, stream, raw);
   if (C == 64) {

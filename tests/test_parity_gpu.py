@@ -620,3 +620,40 @@ def test_random_layouts_fused_all_methods(bnd, seed):
             check_A(runs[0][0], inp, A_ref, N_ref)
             assert max_ratio(bnd.to_numpy_f64(runs[0][1]), W_ref) <= TOL_WY[wl.BF16]
             assert max_ratio(bnd.to_numpy_f64(runs[0][2]), U_ref) <= TOL_WY[wl.BF16]
+
+
+def test_head_dimension_64_on_the_tensor_cores(bnd):
+    """bf16 keys and values with d_k = d_v = 64 at C = 64: tri_inv_build, tri_inv_fused (block recursion and series
+    leaves) and tri_inv_wy take the tensor-core kernel's one-box instances.  Dense and packed ragged layouts, every
+    matrix against the fp64 oracle; sentinels show that every row of real tokens is written and no other."""
+    rng = np.random.default_rng(77)
+    cu = wl.ragged_lengths(7, 5 * 64, rng)
+    cases = [wl.make("d64_dense", 3, 6 * 64, 5, 64, 64, 64, wl.BF16, seed=1700),
+             wl.make("d64_packed", 1, int(cu[-1]), 4, 64, 64, 64, wl.BF16, seed=1701, cu_seqlens=cu, rng=rng)]
+    for inp in cases:
+        cuq = inp.cu_seqlens
+        A_ref, N_ref = oracle.build_A(inp.K, inp.beta, inp.g, 64, cu_seqlens=cuq, return_N=True)
+        W_ref, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, 64, cu_seqlens=cuq)
+        dev = bnd.to_device(inp)
+        nan = lambda t: torch.full_like(t, float("nan"))
+        for m in (bnd.BLOCK_RECURSIVE, bnd.BLOCK_RECURSIVE | bnd.LEAF_SERIES):
+            out = (torch.full((inp.B, inp.T, inp.H, 64), float("nan"), dtype=torch.float32, device="cuda"), nan(dev["K"]), nan(dev["V"]))
+            A, W, U = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], 64, method=m, cu_seqlens=cuq, out=out)
+            torch.cuda.synchronize()
+            assert bnd.last_device_status() == 0
+            a = A.cpu().numpy()
+            assert not np.isnan(a).any() and structure_errors(a, inp) == (0, 0)
+            assert max_ratio(a, A_ref) <= TOL_A[wl.BF16] and max_residual(a, N_ref, inp) <= TOL_RES[wl.BF16]
+            w, u = bnd.to_numpy_f64(W), bnd.to_numpy_f64(U)
+            assert not np.isnan(w).any() and not np.isnan(u).any()
+            assert max_ratio(w, W_ref) <= 1e-2 and max_ratio(u, U_ref) <= 1e-2
+        A_only = bnd.build(dev["K"], dev["beta"], dev["g"], 64, cu_seqlens=cuq)
+        W2, U2 = bnd.wy(A_only, dev["K"], dev["V"], dev["beta"], cu_seqlens=cuq)
+        torch.cuda.synchronize()
+        assert bnd.last_device_status() == 0
+        assert max_ratio(A_only.cpu().numpy(), A_ref) <= TOL_A[wl.BF16]
+        assert max_ratio(bnd.to_numpy_f64(W2), W_ref) <= 1e-2 and max_ratio(bnd.to_numpy_f64(U2), U_ref) <= 1e-2
+        # the CUDA-core kernel, which served this shape before, agrees within the two paths' rounding
+        A_simt, W_simt, U_simt = bnd.fused(dev["K"], dev["V"], dev["beta"], dev["g"], 64, method=bnd.FORCE_SIMT, cu_seqlens=cuq)
+        torch.cuda.synchronize()
+        assert float((A_simt - A).abs().max()) <= 4e-3 * float(A_simt.abs().max())
