@@ -364,8 +364,16 @@ int tri_inv_fused_kda(const void* K, const void* V, const float* G, const float*
   if ((rc = check_method(method, false, false))) return rc;
   const bool tc = !(method & (TRI_INV_FORCE_SIMT | TRI_INV_REFINE)) && (method & TRI_INV_METHOD_MASK) == TRI_INV_BLOCK_RECURSIVE &&
                   desc->kv_dtype == TRI_INV_BF16 && desc->d_k == 128 && desc->d_v == 128 && (desc->C == 64 || desc->C == 128);
+  if (tc && desc->C == 64) {
+    // one kernel: build, inversion and both factors (W's columns scaled by exp(G_ref) on the way out)
+    KParams p{};
+    p.K = K; p.V = V; p.G = G; p.beta = beta; p.g = nullptr; p.A = A; p.W = W; p.U = U;
+    p.method = method;
+    p.ops = kStoreA | kDoWY | kKda;
+    return run(p, desc, cuda_stream);
+  }
   if (tc) {
-    // Tensor-core route, two launches on the stream: the per-channel build kernel, which also writes K' = K * exp(G) into
+    // C = 128, two launches on the stream: the per-channel build kernel, which also writes K' = K * exp(G) into
     // the W buffer while it has K and G in shared memory; then W = A diag(beta) K' and U = A diag(beta) V by the WY kernel,
     // which reads each K' tile whole into shared memory before it writes the same rows of W.
     KParams p{};

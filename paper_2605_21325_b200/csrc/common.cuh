@@ -132,6 +132,8 @@ cudaError_t launch_chunk_scan_simt(const ScanParams& p, const void* Q, const voi
 // Per-channel decay variant on the tensor cores (bf16 keys, d_k = 128, C = 64 or 128, block recursion).
 cudaError_t launch_kda_tc(const KParams& p, int C, cudaStream_t stream, bool* handled);
 cudaError_t launch_kda_tc_c128(const KParams& p, cudaStream_t stream);
+// Per-channel decay, build + inversion + W and U in one kernel (bf16, d_k = d_v = 128, C = 64, block recursion).
+cudaError_t launch_kda_fused_tc(const KParams& p, cudaStream_t stream);
 
 // Fills dev_tab (one entry per chunk of tokens, in sequence order) from the host offsets in d->cu_seqlens
 // with small kernels on the stream; no copy and no synchronisation.

@@ -239,6 +239,11 @@ cudaError_t launch_kda_tc(const KParams& p, int Cc, cudaStream_t stream, bool* h
   *handled = false;
   if (p.kv_dtype != TRI_INV_BF16 || p.d_k != 128 || (Cc != 64 && Cc != 128)) return cudaSuccess;
   if ((p.method & TRI_INV_METHOD_MASK) != TRI_INV_BLOCK_RECURSIVE) return cudaSuccess;
+  if (p.ops & kDoWY) {   // build + inversion + WY in one kernel: C = 64 only (tri_inv_fused_kda makes two launches at C = 128)
+    if (Cc != 64 || p.d_v != 128 || !p.V || !p.W || !p.U) return cudaSuccess;
+    *handled = true;
+    return launch_kda_fused_tc(p, stream);
+  }
   *handled = true;
   if (Cc == 128) return launch_kda_tc_c128(p, stream);
   static std::mutex mu;

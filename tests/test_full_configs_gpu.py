@@ -220,3 +220,35 @@ def test_per_channel_decay_full_size(bnd, cfg):
     A_scalar = bnd.build(dev["K"], dev["beta"], dev["g"], inp.C)
     torch.cuda.synchronize()
     assert float((A_same - A_scalar).abs().max()) <= 2e-3 * float(A_scalar.abs().max())
+
+
+def test_per_channel_fused_call_on_the_ragged_configuration_repeats_bit_for_bit(bnd):
+    """tri_inv_fused_kda (one kernel at C = 64) on config 5, whose 160 sequences end inside chunks: EVERY matrix's A, W and U
+    against the fp64 oracle, nothing written past a sequence's end, and three calls into fresh buffers give the same bits
+    (the kernel's staging tiles share their space with the operand tiles of the item before and after)."""
+    inp = wl.config(5)
+    cu = inp.cu_seqlens
+    G = wl.per_channel_gate(inp, seed=3005)
+    dev = bnd.to_device(inp)
+    Gd = torch.from_numpy(G).cuda()
+    outs = []
+    for _ in range(3):
+        A = torch.full((inp.B, inp.T, inp.H, inp.C), float("nan"), dtype=torch.float32, device="cuda")
+        W, U = torch.full_like(dev["K"], float("nan")), torch.full_like(dev["V"], float("nan"))
+        bnd.fused_kda(dev["K"], dev["V"], Gd, dev["beta"], inp.C, cu_seqlens=cu, out=(A, W, U))
+        torch.cuda.synchronize()
+        assert bnd.last_device_status() == 0
+        outs.append((A, W, U))
+    for A, W, U in outs[1:]:
+        assert torch.equal(A.view(torch.int32), outs[0][0].view(torch.int32))
+        assert torch.equal(W.view(torch.int16), outs[0][1].view(torch.int16)) and torch.equal(U.view(torch.int16), outs[0][2].view(torch.int16))
+    A, W, U = outs[0]
+    assert not torch.isnan(A).any() and not torch.isnan(W).any() and not torch.isnan(U).any()
+    A_ref, N_ref = oracle.build_A_kda(inp.K, G, inp.beta, inp.C, cu_seqlens=cu, return_N=True)
+    device_structure_check(A, inp)
+    a = A.cpu().numpy()
+    assert max_ratio(a, A_ref) <= TOL_A[wl.BF16] and max_residual(a, N_ref, inp) <= TOL_RES[wl.BF16]
+    Kg = wl.bf16_bits_to_f32(inp.K).astype(np.float64) * np.exp(G.astype(np.float64))
+    W_ref, _ = oracle.wy(A_ref, Kg, None, inp.beta, inp.C, cu_seqlens=cu)
+    _, U_ref = oracle.wy(A_ref, inp.K, inp.V, inp.beta, inp.C, cu_seqlens=cu)
+    assert max_ratio(bnd.to_numpy_f64(W), W_ref) <= 1e-2 and max_ratio(bnd.to_numpy_f64(U), U_ref) <= 1e-2
