@@ -119,6 +119,7 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
   for (int item = blockIdx.x; item < total && !misaligned; item += gridDim.x) {
     int tok0, rows, h;
     locate(p, C, item, tok0, rows, h);
+    PHASE_BEGIN();
     const int nx_item = item + gridDim.x;
     const bool has_next = nx_item < total;
     int nx_tok0 = 0, nx_rows = 0, nx_h = 0;
@@ -137,47 +138,75 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
     // ---- 2. K+ = K * 2^x over K, K- = K * 2^-x, x = (G - G_ref) log2(e); rows past the chunk's end are zero
     wait(bar_k, ph);
     wait(bar_g, ph);
+    // The item before: its U stores must have read their staging tiles (K-'s and A''s space) before this item writes there;
+    // that wait runs behind the copies' above.  The barrier is also where a CTA that gave up leaves, all threads at once.
+    if (lane == 0) bulk_wait_read();
+    if (bad) *s_gave_up = 1;
+    tc_fence_before();
+    __syncthreads();
+    if (*s_gave_up) break;
+    PHASE(0);
     const int rref = rows >> 1;
+    {
+      // This thread's 8 channels are the same in every pass (NT is a multiple of 16): the reference row is read once.  The
+      // passes are branch-free (rows past the chunk's end are read like the others and replaced by zeros), so that the
+      // loads of one pass are in flight while the exponentials of the pass before are formed.
+      const int cf = tid & 15;                            // 16-byte chunk of 8 features
+      const int q0 = 2 * (cf & 3);                        // first of the two float4 of G for these 8 channels
+      const uint32_t gbox = sG + (cf >> 2) * 8192;
+      float gr[8];
 #pragma unroll
-    for (int m = 0; m < 8; ++m) {
-      const int e = tid + m * NT;
-      const int r = e >> 4, cf = e & 15;                 // row, 16-byte chunk of 8 features
-      const uint32_t koff = (uint32_t)((cf >> 3) * 8192 + r * 128 + (((cf & 7) ^ (r & 7)) << 4));
-      uint4 kp = make_uint4(0, 0, 0, 0), km = kp;
-      if (r < rows) {
-        uint4 kv;
-        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kv.x), "=r"(kv.y), "=r"(kv.z), "=r"(kv.w) : "r"(sK + koff));
-        const int q0 = 2 * (cf & 3);                     // first of the two float4 of G for these 8 channels
-        const uint32_t gbox = sG + (cf >> 2) * 8192;
-        float gv[8], gr[8];
+      for (int hq = 0; hq < 2; ++hq)
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gr[4 * hq]), "=f"(gr[4 * hq + 1]), "=f"(gr[4 * hq + 2]), "=f"(gr[4 * hq + 3])
+                     : "r"(gbox + rref * 128 + (((q0 + hq) ^ (rref & 7)) << 4)));
 #pragma unroll
-        for (int hq = 0; hq < 2; ++hq) {
-          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gv[4 * hq]), "=f"(gv[4 * hq + 1]), "=f"(gv[4 * hq + 2]), "=f"(gv[4 * hq + 3])
-                       : "r"(gbox + r * 128 + (((q0 + hq) ^ (r & 7)) << 4)));
-          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gr[4 * hq]), "=f"(gr[4 * hq + 1]), "=f"(gr[4 * hq + 2]), "=f"(gr[4 * hq + 3])
-                       : "r"(gbox + rref * 128 + (((q0 + hq) ^ (rref & 7)) << 4)));
+      for (int q = 0; q < 8; ++q) gr[q] *= kLog2e;
+      if ((tid >> 4) == 0) {   // exp(G_ref) of the 128 channels, for W's columns
+#pragma unroll
+        for (int q = 0; q < 8; ++q) sER[8 * cf + q] = ex2_approx(gr[q]);
+      }
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        // the loads of four passes first (shared-memory loads and stores keep their program order), then their arithmetic
+        uint4 kv[4];
+        float gv[4][8];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          const int r = (tid >> 4) + 8 * (4 * half + m);
+          const uint32_t koff = (uint32_t)((cf >> 3) * 8192 + r * 128 + (((cf & 7) ^ (r & 7)) << 4));
+          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kv[m].x), "=r"(kv[m].y), "=r"(kv[m].z), "=r"(kv[m].w) : "r"(sK + koff));
+#pragma unroll
+          for (int hq = 0; hq < 2; ++hq)
+            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gv[m][4 * hq]), "=f"(gv[m][4 * hq + 1]), "=f"(gv[m][4 * hq + 2]), "=f"(gv[m][4 * hq + 3])
+                         : "r"(gbox + r * 128 + (((q0 + hq) ^ (r & 7)) << 4)));
         }
-        const uint32_t* kw = reinterpret_cast<const uint32_t*>(&kv);
-        uint32_t* pw = reinterpret_cast<uint32_t*>(&kp);
-        uint32_t* mw = reinterpret_cast<uint32_t*>(&km);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float2 kf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kw[q]));
-          const float x0 = (gv[2 * q] - gr[2 * q]) * kLog2e, x1 = (gv[2 * q + 1] - gr[2 * q + 1]) * kLog2e;
-          pw[q] = pack_bf16(kf.x * ex2_approx(x0), kf.y * ex2_approx(x1));
-          mw[q] = pack_bf16(kf.x * ex2_approx(-x0), kf.y * ex2_approx(-x1));
-        }
-        if (r == rref) {   // the reference row's thread keeps exp(G_ref) of its 8 channels for W's columns
+        for (int m = 0; m < 4; ++m) {
+          const int r = (tid >> 4) + 8 * (4 * half + m);
+          const uint32_t koff = (uint32_t)((cf >> 3) * 8192 + r * 128 + (((cf & 7) ^ (r & 7)) << 4));
+          uint4 kp, km;
+          const uint32_t* kw = reinterpret_cast<const uint32_t*>(&kv[m]);
+          uint32_t* pw = reinterpret_cast<uint32_t*>(&kp);
+          uint32_t* mw = reinterpret_cast<uint32_t*>(&km);
+          const bool live = r < rows;
 #pragma unroll
-          for (int q = 0; q < 8; ++q) sER[8 * cf + q] = ex2_approx(gr[q] * kLog2e);
+          for (int q = 0; q < 4; ++q) {
+            const float2 kf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kw[q]));
+            const float x0 = fmaf(gv[m][2 * q], kLog2e, -gr[2 * q]), x1 = fmaf(gv[m][2 * q + 1], kLog2e, -gr[2 * q + 1]);
+            const uint32_t vp = pack_bf16(kf.x * ex2_approx(x0), kf.y * ex2_approx(x1));
+            const uint32_t vm = pack_bf16(kf.x * ex2_approx(-x0), kf.y * ex2_approx(-x1));
+            pw[q] = live ? vp : 0u;
+            mw[q] = live ? vm : 0u;
+          }
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sK + koff), "r"(kp.x), "r"(kp.y), "r"(kp.z), "r"(kp.w) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + koff), "r"(km.x), "r"(km.y), "r"(km.z), "r"(km.w) : "memory");
         }
       }
-      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sK + koff), "r"(kp.x), "r"(kp.y), "r"(kp.z), "r"(kp.w) : "memory");
-      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + koff), "r"(km.x), "r"(km.y), "r"(km.z), "r"(km.w) : "memory");
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    PHASE(1);
 
     // ---- 3. S = K+ (K-)^T
     if (tid == 0) {
@@ -193,7 +222,8 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
     wait(bar_mma, ph_mma);
     ph_mma ^= 1;
     tc_fence_after();
-    if (tid == kTidV && !bad) issue_v(tok0, h);   // K-'s only reader has completed: V comes into its space
+    if (tid == kTidV && !bad) issue_v(tok0, h);
+    PHASE(2);   // K-'s only reader has completed: V comes into its space
     if (has_next) beta_next = fetch_beta(nx_tok0, nx_rows, nx_h);
 
     // ---- 4. gate (beta_i, strict-lower mask), N -> shared memory over the G tile (all of G has been consumed)
@@ -218,13 +248,16 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
       }
     }
     __syncwarp();
+    PHASE(3);
     if (p.method & TRI_INV_LEAF_SERIES)
       leaf_series<LD, LEAF_LD>(sX + 16 * rb * LD + 16 * rb, reinterpret_cast<float*>(smem + OFF_LEAF) + warp * 16 * LEAF_LD, lane);
     else
       leaf_substitution<LD>(sX + 16 * rb * LD + 16 * rb, lane);
     __syncthreads();
+    PHASE(4);
     merge_level<C, 16>(sX, warp, lane);
     merge_level<C, 32>(sX, warp, lane);
+    PHASE(5);
 
     // ---- 5. one pass over the finished matrix (zeros above the diagonal, ones on it): A to global memory, A' = A diag(beta)
     //         as the bf16 K-major swizzled operand of the two products
@@ -255,6 +288,7 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
     tc_fence_before();
     __syncthreads();       // the fp32 matrix has been read by everyone: the next G tile may land in its space
     if (tid == kTidG && has_next && !bad) issue_g(nx_tok0, nx_h);
+    PHASE(6);
 
     // ---- 6. W = (A' K+) diag(exp G_ref), U = A' V: the tiles are the MN-major B operand, 16 tokens per k-step
     constexpr uint32_t idesc_wy = umma_idesc(C, D, 1);
@@ -268,6 +302,7 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
     wait(bar_mma, ph_mma);
     ph_mma ^= 1;
     tc_fence_after();
+    PHASE(7);
     const int row0 = 16 * rb;
     const size_t row_stride = (size_t)p.H * D;
     __nv_bfloat16* w_row0 = reinterpret_cast<__nv_bfloat16*>(p.W) + ((size_t)(tok0 + row0) * p.H + h) * D;
@@ -278,6 +313,7 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
     tmem_wait_ld();
     tc_fence_before();
     __syncthreads();   // every warp holds its rows of W in registers: U may overwrite the columns, K+ has been read
+    PHASE(8);
     if (tid == 0) {
       if (wait(bar_v, ph)) { tc_fence_after(); issue_wy(sKm); }
     }
@@ -290,9 +326,11 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
     // four staging tiles per warp and item, each used once: nothing to wait for before they are written
     store_frag_piece_bf16<3>(f0, sK + warp * 2048, lane, w_row0, row_stride, rows - row0, &tmW, h * D, tok0 + row0);
     store_frag_piece_bf16<3>(f1, sK + 8192 + warp * 2048, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
+    PHASE(9);
     wait(bar_mma, ph_mma);
     ph_mma ^= 1;
     tc_fence_after();
+    PHASE(10);
     tmem_ld_16x64(f0, tmem_rows);
     tmem_ld_16x64(f1, tmem_rows + 64);
     tmem_wait_ld();
@@ -302,15 +340,13 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
     if (tid == kTidK && has_next && !bad) issue_k(nx_tok0, nx_h);
     store_frag_piece_bf16<3>(f0, sAp + warp * 2048, lane, u_row0, row_stride, rows - row0, &tmU, h * D, tok0 + row0);
     store_frag_piece_bf16<3>(f1, sKm + warp * 2048, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
-    if (lane == 0) bulk_wait_read();   // ... and the U stores theirs, before the next item writes K- and A'
-    if (bad) *s_gave_up = 1;
-    tc_fence_before();
-    __syncthreads();
-    if (*s_gave_up) break;   // uniform: every thread reads the flag behind the same barrier
     ph ^= 1;
+    PHASE(11);
   }
-  if (bad || misaligned) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
   if (lane == 0) bulk_wait_read();
+  if (bad) *s_gave_up = 1;   // a wait of the last item ran out: nobody has looked at the flag since
+  if (bad || misaligned) atomicMax(p.status, TRI_INV_ERR_DEVICE_TIMEOUT);
+  __syncthreads();           // every thread has left the item loop
   if (*s_gave_up) {
     // what may still be in flight: the last copy each tile thread requested, and every product issued so far
     if (tid == kTidK && n_k) mbar_wait_bounded(bar_k, (n_k - 1) & 1, p.wait_limit_ns);

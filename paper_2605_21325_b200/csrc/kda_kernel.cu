@@ -31,7 +31,6 @@ constexpr int TMEM_COLS = 64;
 constexpr int CTAS_PER_SM = 3;
 static_assert(OFF_LEAF + NW * 16 * LEAF_LD * 4 <= OFF_BETA, "leaf scratch must fit behind the fp32 matrix");
 
-template <bool KG>   // KG: also write K * exp(G) into p.W (the fused call)
 __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                      const __grid_constant__ CUtensorMap tmG, KParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -112,43 +111,57 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid
     wait(bar_k, ph);
     wait(bar_g, ph);
     const int rref = rows >> 1;
+    {
+      // This thread's 8 channels are the same in every pass (NT is a multiple of 16): the reference row is read once.  The
+      // passes are branch-free (rows past the chunk's end are read like the others and replaced by zeros), so that the
+      // loads of one pass are in flight while the exponentials of the pass before are formed.
+      const int cf = tid & 15;                            // 16-byte chunk of 8 features
+      const int q0 = 2 * (cf & 3);                        // first of the two float4 of G for these 8 channels
+      const uint32_t gbox = sG + (cf >> 2) * 8192;
+      float gr[8];
 #pragma unroll
-    for (int m = 0; m < 8; ++m) {
-      const int e = tid + m * NT;
-      const int r = e >> 4, cf = e & 15;                 // row, 16-byte chunk of 8 features
-      const uint32_t koff = (uint32_t)((cf >> 3) * 8192 + r * 128 + (((cf & 7) ^ (r & 7)) << 4));
-      uint4 kp = make_uint4(0, 0, 0, 0), km = kp;
-      if (r < rows) {
-        uint4 kv;
-        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kv.x), "=r"(kv.y), "=r"(kv.z), "=r"(kv.w) : "r"(sK + koff));
-        const int q0 = 2 * (cf & 3);                     // first of the two float4 of G for these 8 channels
-        const uint32_t gbox = sG + (cf >> 2) * 8192;
-        float gv[8], gr[8];
+      for (int hq = 0; hq < 2; ++hq)
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gr[4 * hq]), "=f"(gr[4 * hq + 1]), "=f"(gr[4 * hq + 2]), "=f"(gr[4 * hq + 3])
+                     : "r"(gbox + rref * 128 + (((q0 + hq) ^ (rref & 7)) << 4)));
 #pragma unroll
-        for (int hq = 0; hq < 2; ++hq) {
-          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gv[4 * hq]), "=f"(gv[4 * hq + 1]), "=f"(gv[4 * hq + 2]), "=f"(gv[4 * hq + 3])
-                       : "r"(gbox + r * 128 + (((q0 + hq) ^ (r & 7)) << 4)));
-          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gr[4 * hq]), "=f"(gr[4 * hq + 1]), "=f"(gr[4 * hq + 2]), "=f"(gr[4 * hq + 3])
-                       : "r"(gbox + rref * 128 + (((q0 + hq) ^ (rref & 7)) << 4)));
+      for (int q = 0; q < 8; ++q) gr[q] *= 1.4426950408889634f;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        // the loads of four passes first (shared-memory loads and stores keep their program order), then their arithmetic
+        uint4 kv[4];
+        float gv[4][8];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          const int r = (tid >> 4) + 8 * (4 * half + m);
+          const uint32_t koff = (uint32_t)((cf >> 3) * 8192 + r * 128 + (((cf & 7) ^ (r & 7)) << 4));
+          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kv[m].x), "=r"(kv[m].y), "=r"(kv[m].z), "=r"(kv[m].w) : "r"(sK + koff));
+#pragma unroll
+          for (int hq = 0; hq < 2; ++hq)
+            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gv[m][4 * hq]), "=f"(gv[m][4 * hq + 1]), "=f"(gv[m][4 * hq + 2]), "=f"(gv[m][4 * hq + 3])
+                         : "r"(gbox + r * 128 + (((q0 + hq) ^ (r & 7)) << 4)));
         }
-        const uint32_t* kw = reinterpret_cast<const uint32_t*>(&kv);
-        uint32_t* pw = reinterpret_cast<uint32_t*>(&kp);
-        uint32_t* mw = reinterpret_cast<uint32_t*>(&km);
-        uint4 kg;                                         // K * exp(G): the key operand of the WY step that follows (fused call)
-        uint32_t* gw = reinterpret_cast<uint32_t*>(&kg);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float2 kf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kw[q]));
-          const float x0 = (gv[2 * q] - gr[2 * q]) * 1.4426950408889634f, x1 = (gv[2 * q + 1] - gr[2 * q + 1]) * 1.4426950408889634f;
-          pw[q] = pack_bf16(kf.x * ex2_approx(x0), kf.y * ex2_approx(x1));
-          mw[q] = pack_bf16(kf.x * ex2_approx(-x0), kf.y * ex2_approx(-x1));
-          if constexpr (KG) gw[q] = pack_bf16(kf.x * ex2_approx(gv[2 * q] * 1.4426950408889634f), kf.y * ex2_approx(gv[2 * q + 1] * 1.4426950408889634f));
+        for (int m = 0; m < 4; ++m) {
+          const int r = (tid >> 4) + 8 * (4 * half + m);
+          const uint32_t koff = (uint32_t)((cf >> 3) * 8192 + r * 128 + (((cf & 7) ^ (r & 7)) << 4));
+          uint4 kp, km;
+          const uint32_t* kw = reinterpret_cast<const uint32_t*>(&kv[m]);
+          uint32_t* pw = reinterpret_cast<uint32_t*>(&kp);
+          uint32_t* mw = reinterpret_cast<uint32_t*>(&km);
+          const bool live = r < rows;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float2 kf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kw[q]));
+            const float x0 = fmaf(gv[m][2 * q], 1.4426950408889634f, -gr[2 * q]), x1 = fmaf(gv[m][2 * q + 1], 1.4426950408889634f, -gr[2 * q + 1]);
+            const uint32_t vp = pack_bf16(kf.x * ex2_approx(x0), kf.y * ex2_approx(x1));
+            const uint32_t vm = pack_bf16(kf.x * ex2_approx(-x0), kf.y * ex2_approx(-x1));
+            pw[q] = live ? vp : 0u;
+            mw[q] = live ? vm : 0u;
+          }
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sK + koff), "r"(kp.x), "r"(kp.y), "r"(kp.z), "r"(kp.w) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + koff), "r"(km.x), "r"(km.y), "r"(km.z), "r"(km.w) : "memory");
         }
-        // 16 consecutive threads cover the 256 contiguous bytes of one token's keys of this head
-        if constexpr (KG) *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.W) + ((size_t)(tok0 + r) * p.H + h) * D + 8 * cf) = kg;
       }
-      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sK + koff), "r"(kp.x), "r"(kp.y), "r"(kp.z), "r"(kp.w) : "memory");
-      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + koff), "r"(km.x), "r"(km.y), "r"(km.z), "r"(km.w) : "memory");
     }
     fence_proxy_async();
     tc_fence_before();
@@ -246,6 +259,7 @@ cudaError_t launch_kda_tc(const KParams& p, int Cc, cudaStream_t stream, bool* h
   }
   *handled = true;
   if (Cc == 128) return launch_kda_tc_c128(p, stream);
+  if (p.W) return cudaErrorNotSupported;   // K exp(G) as a by-product is the C = 128 kernel's; nothing asks for it here
   static std::mutex mu;
   static int n_sm_of[64] = {0}, ctas_of[64] = {0};
   int dev = 0;
@@ -256,10 +270,8 @@ cudaError_t launch_kda_tc(const KParams& p, int Cc, cudaStream_t stream, bool* h
   {
     std::lock_guard<std::mutex> lock(mu);
     if (!n_sm_of[dev]) {
-      if ((e = cudaFuncSetAttribute(kda_build_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) != cudaSuccess) return e;
-      if ((e = cudaFuncSetAttribute(kda_build_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
-      if ((e = cudaFuncSetAttribute(kda_build_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) != cudaSuccess) return e;
-      if ((e = cudaFuncSetAttribute(kda_build_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(kda_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(kda_build_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
       int sms = 0, smem_per_sm = 0;
       if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
       if ((e = cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev)) != cudaSuccess) return e;
@@ -277,8 +289,7 @@ cudaError_t launch_kda_tc(const KParams& p, int Cc, cudaStream_t stream, bool* h
   if (!make_tmap(&tmG, p.G, tokens, p.H, D, C, 4)) return cudaErrorUnknown;
   long long total = (long long)p.n_chunks * p.H, cap = (long long)n_sm * ctas;
   int grid = (int)(total < cap ? total : cap);
-  if (p.W) kda_build_kernel<true><<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
-  else kda_build_kernel<false><<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
+  kda_build_kernel<<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
   return cudaGetLastError();
 }
 

@@ -130,57 +130,73 @@ __global__ void __launch_bounds__(NT, 2) kda_build_kernel_c128(const __grid_cons
 #pragma unroll 1
     for (int bx = 0; bx < 4; ++bx) {
     wait((bx & 1) ? bar_g1 : bar_g0, (uint32_t)(bx >> 1));
+    {
+      // Branch-free (rows past the chunk's end are read like the others and replaced by zeros) and loads first: the
+      // thread's 8 channels are the same for its two rows (r and r + 64), so the two reference rows are read once per box.
+      constexpr float kL2e = 1.4426950408889634f;
+      const int cf = 4 * bx + (tid & 3);                  // 16-byte chunk of 8 features (four per box of G)
+      const int q0 = 2 * (tid & 3);                       // first of the two float4 of G for these 8 channels
+      const uint32_t gbox = sG + (bx & 1) * G_BOX;
+      float gr0[8], gr1[8];
 #pragma unroll
-    for (int m = 0; m < 2; ++m) {
-      const int e = tid + m * NT;
-      const int r = e >> 2, cf = 4 * bx + (e & 3);       // row, 16-byte chunk of 8 features (four per box of G)
-      const int hf = r >> 6;
-      const uint32_t sw = (uint32_t)((((cf & 7) ^ (r & 7)) << 4));   // (rows r, r + 64 and r + 128 share r & 7)
-      const uint32_t koff = (uint32_t)((cf >> 3) * K_BOX + r * 128) + sw;
-      const uint32_t moff = (uint32_t)((cf >> 3) * KM_BOX + (hf ? r + 64 : r) * 128) + sw;   // K- against the row's own reference
-      uint4 kp = make_uint4(0, 0, 0, 0), km = kp, km1 = kp;
-      if (r < rows) {
-        uint4 kv;
-        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kv.x), "=r"(kv.y), "=r"(kv.z), "=r"(kv.w) : "r"(sK + koff));
-        const int q0 = 2 * (cf & 3);                     // first of the two float4 of G for these 8 channels
-        const uint32_t gbox = sG + (bx & 1) * G_BOX;
-        const int rref = hf ? rref1 : rref0;
-        const bool cross = !hf && rows1 > 0;             // a token of the first half that the second half's rows see
-        float gv[8], gr[8], gx[8];
+      for (int hq = 0; hq < 2; ++hq) {
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gr0[4 * hq]), "=f"(gr0[4 * hq + 1]), "=f"(gr0[4 * hq + 2]), "=f"(gr0[4 * hq + 3])
+                     : "r"(gbox + rref0 * 128 + (((q0 + hq) ^ (rref0 & 7)) << 4)));
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gr1[4 * hq]), "=f"(gr1[4 * hq + 1]), "=f"(gr1[4 * hq + 2]), "=f"(gr1[4 * hq + 3])
+                     : "r"(gbox + rref1 * 128 + (((q0 + hq) ^ (rref1 & 7)) << 4)));
+      }
+      uint4 kv[2];
+      float gv[2][8];
 #pragma unroll
-        for (int hq = 0; hq < 2; ++hq) {
-          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gv[4 * hq]), "=f"(gv[4 * hq + 1]), "=f"(gv[4 * hq + 2]), "=f"(gv[4 * hq + 3])
+      for (int m = 0; m < 2; ++m) {
+        const int r = (tid >> 2) + 64 * m;
+        const uint32_t sw = (uint32_t)((((cf & 7) ^ (r & 7)) << 4));   // (rows r, r + 64 and r + 128 share r & 7)
+        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(kv[m].x), "=r"(kv[m].y), "=r"(kv[m].z), "=r"(kv[m].w)
+                     : "r"(sK + (uint32_t)((cf >> 3) * K_BOX + r * 128) + sw));
+#pragma unroll
+        for (int hq = 0; hq < 2; ++hq)
+          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gv[m][4 * hq]), "=f"(gv[m][4 * hq + 1]), "=f"(gv[m][4 * hq + 2]), "=f"(gv[m][4 * hq + 3])
                        : "r"(gbox + r * 128 + (((q0 + hq) ^ (r & 7)) << 4)));
-          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gr[4 * hq]), "=f"(gr[4 * hq + 1]), "=f"(gr[4 * hq + 2]), "=f"(gr[4 * hq + 3])
-                       : "r"(gbox + rref * 128 + (((q0 + hq) ^ (rref & 7)) << 4)));
-          if (cross)
-            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(gx[4 * hq]), "=f"(gx[4 * hq + 1]), "=f"(gx[4 * hq + 2]), "=f"(gx[4 * hq + 3])
-                         : "r"(gbox + rref1 * 128 + (((q0 + hq) ^ (rref1 & 7)) << 4)));
-        }
-        const uint32_t* kw = reinterpret_cast<const uint32_t*>(&kv);
+      }
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { gr0[q] *= kL2e; gr1[q] *= kL2e; }
+#pragma unroll
+      for (int m = 0; m < 2; ++m) {
+        const int r = (tid >> 2) + 64 * m;                // m is the row's half of the chunk
+        const uint32_t sw = (uint32_t)((((cf & 7) ^ (r & 7)) << 4));
+        const uint32_t koff = (uint32_t)((cf >> 3) * K_BOX + r * 128) + sw;
+        const uint32_t moff = (uint32_t)((cf >> 3) * KM_BOX + (m ? r + 64 : r) * 128) + sw;   // K- against the row's own reference
+        const bool live = r < rows;
+        const bool cross = live && rows1 > 0;             // m = 0: a token of the first half that the second half's rows see
+        uint4 kp, km, km1, kg;                            // kg = K * exp(G): the key operand of the WY step that follows (fused call)
+        const uint32_t* kw = reinterpret_cast<const uint32_t*>(&kv[m]);
         uint32_t* pw = reinterpret_cast<uint32_t*>(&kp);
         uint32_t* mw = reinterpret_cast<uint32_t*>(&km);
         uint32_t* xw = reinterpret_cast<uint32_t*>(&km1);
-        uint4 kg;                                         // K * exp(G): the key operand of the WY step that follows (fused call)
         uint32_t* gw = reinterpret_cast<uint32_t*>(&kg);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const float2 kf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&kw[q]));
-          const float x0 = (gv[2 * q] - gr[2 * q]) * 1.4426950408889634f, x1 = (gv[2 * q + 1] - gr[2 * q + 1]) * 1.4426950408889634f;
-          pw[q] = pack_bf16(kf.x * ex2_approx(x0), kf.y * ex2_approx(x1));
-          mw[q] = pack_bf16(kf.x * ex2_approx(-x0), kf.y * ex2_approx(-x1));
-          if (cross) {
-            const float y0 = (gx[2 * q] - gv[2 * q]) * 1.4426950408889634f, y1 = (gx[2 * q + 1] - gv[2 * q + 1]) * 1.4426950408889634f;
-            xw[q] = pack_bf16(kf.x * ex2_approx(y0), kf.y * ex2_approx(y1));
+          const float ga = gv[m][2 * q] * kL2e, gb = gv[m][2 * q + 1] * kL2e;
+          const float x0 = ga - (m ? gr1[2 * q] : gr0[2 * q]), x1 = gb - (m ? gr1[2 * q + 1] : gr0[2 * q + 1]);
+          const uint32_t vp = pack_bf16(kf.x * ex2_approx(x0), kf.y * ex2_approx(x1));
+          const uint32_t vm = pack_bf16(kf.x * ex2_approx(-x0), kf.y * ex2_approx(-x1));
+          pw[q] = live ? vp : 0u;
+          mw[q] = live ? vm : 0u;
+          if (m == 0) {
+            const uint32_t vx = pack_bf16(kf.x * ex2_approx(gr1[2 * q] - ga), kf.y * ex2_approx(gr1[2 * q + 1] - gb));
+            xw[q] = cross ? vx : 0u;
           }
-          if constexpr (KG) gw[q] = pack_bf16(kf.x * ex2_approx(gv[2 * q] * 1.4426950408889634f), kf.y * ex2_approx(gv[2 * q + 1] * 1.4426950408889634f));
+          if constexpr (KG) gw[q] = pack_bf16(kf.x * ex2_approx(ga), kf.y * ex2_approx(gb));
         }
         // 16 consecutive threads cover the 256 contiguous bytes of one token's keys of this head
-        if constexpr (KG) *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.W) + ((size_t)(tok0 + r) * p.H + h) * D + 8 * cf) = kg;
+        if constexpr (KG) {
+          if (live) *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.W) + ((size_t)(tok0 + r) * p.H + h) * D + 8 * cf) = kg;
+        }
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sK + koff), "r"(kp.x), "r"(kp.y), "r"(kp.z), "r"(kp.w) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + moff), "r"(km.x), "r"(km.y), "r"(km.z), "r"(km.w) : "memory");
+        if (m == 0) asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + moff + 64 * 128), "r"(km1.x), "r"(km1.y), "r"(km1.z), "r"(km1.w) : "memory");
       }
-      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sK + koff), "r"(kp.x), "r"(kp.y), "r"(kp.z), "r"(kp.w) : "memory");
-      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + moff), "r"(km.x), "r"(km.y), "r"(km.z), "r"(km.w) : "memory");
-      if (!hf) asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sKm + moff + 64 * 128), "r"(km1.x), "r"(km1.y), "r"(km1.z), "r"(km1.w) : "memory");
     }
     if (bx < 2) {
       __syncthreads();

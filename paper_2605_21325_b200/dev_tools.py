@@ -28,13 +28,15 @@ def main():
     import torch
     from paper_2605_21325_b200 import binding as b, workloads as wl
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["phases", "timeline", "scan_chunk"])
+    ap.add_argument("what", choices=["phases", "timeline", "scan_chunk", "kda_phases"])
     ap.add_argument("--config", type=int, default=2)
     args = ap.parse_args()
     inp = wl.config(args.config)
     d = b.to_device(inp)
     if args.what == "scan_chunk":
         return scan_chunk(b, wl, inp, d)
+    if args.what == "kda_phases":
+        return kda_phases(b, wl, inp, d)
     out = (torch.empty((inp.B, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda"), torch.empty_like(d["K"]), torch.empty_like(d["V"]))
     L = b.load()
     if not hasattr(L, "tri_inv_debug_counters"):
@@ -73,6 +75,31 @@ SCAN_COMPUTE = ["loop top", "last chunk's O written", "P1 seen", "chain: U tile 
                 "S^T stored", "S^T arrived"]
 SCAN_CONTROL = ["state operand seen", "P1 issued", "copies issued", "U~' seen", "P3 issued", "U~ and P seen", "PU issued", "copies seen",
                 "", "loop top"]
+
+
+KDA_PHASES = ["K, G waited", "K+ K- pass", "Gram wait", "gate", "leaf", "merges", "A, A' pass", "W wait", "W loaded", "W stored",
+              "U wait", "U stored, end"]
+
+
+def kda_phases(b, wl, inp, d):
+    """Cycles per item and warp between the PHASE marks of the one-kernel per-channel call (thread block 0)."""
+    import torch
+    G = torch.from_numpy(wl.per_channel_gate(inp, seed=1)).cuda()
+    out = (torch.empty((inp.B, inp.T, inp.H, inp.C), dtype=torch.float32, device="cuda"), torch.empty_like(d["K"]), torch.empty_like(d["V"]))
+    L = b.load()
+    if not hasattr(L, "tri_inv_debug_counters"):
+        raise SystemExit("%s is not a development build" % b.LIB_PATH)
+    words = (ctypes.c_int * 128)()
+    for _ in range(3):
+        L.tri_inv_debug_counters(words)
+        b.fused_kda(d["K"], d["V"], G, d["beta"], inp.C, cu_seqlens=inp.cu_seqlens, out=out)
+        torch.cuda.synchronize()
+    L.tri_inv_debug_counters(words)
+    grid = min(148 * 3, inp.n_matrices)
+    items = -(-inp.n_matrices // grid)
+    for w in range(4):
+        v = [words[8 + 12 * w + k] / items for k in range(12)]
+        print("warp %d: " % w + ", ".join("%s %.0f" % (n, x) for n, x in zip(KDA_PHASES, v)) + "; total %.0f cycles per item" % sum(v))
 
 
 def scan_chunk(b, wl, inp, d):
