@@ -893,8 +893,10 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
     float* a_dst = ((p.ops & kStoreA) && p.A)
                        ? p.A + ((size_t)(tok0 + tid / (C / 4)) * p.H + h) * C + 4 * (tid % (C / 4)) : nullptr;
     // bf16 pair stores of one float4 of A scaled by beta: K-major, 128-byte swizzle, 64 tokens per row block
+    // (a thread's columns j are the same in every pass: NT is a multiple of C / 4)
+    const float4 beta_j = *reinterpret_cast<const float4*>(sBeta + 4 * (tid % (C / 4)));
     auto put_ap = [&](int i, int j, const float4& v) {
-      const float4 b = *reinterpret_cast<const float4*>(sBeta + j);
+      const float4 b = beta_j;
       const uint32_t lo = pack_bf16(v.x * b.x, v.y * b.y), hi = pack_bf16(v.z * b.z, v.w * b.w);
       const uint32_t off = (uint32_t)((j >> 6) * (C * 128) + i * 128 + (((((j & 63) >> 3) ^ (i & 7)) << 4) | ((j & 7) * 2)));
       if (TRI_INV_CHECK(p, off + 8 <= (uint32_t)(C * C * 2) && i < C && j + 4 <= C))
@@ -907,13 +909,27 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       // K's boxes are requested after rows 0..31 and 0..63, V's first after rows 0..95 and its second after the pass.
       static_assert(C != 128 || (cfg::NT == 256 && LD * 4 * 32 >= cfg::BOX_BYTES && LD * 4 * 31 <= cfg::BOX_BYTES),
                     "the box-by-box reload assumes 8 rows per step and 31 to 32 matrix rows per box");
+      static_assert(NV % 4 == 0, "four passes at a time");
 #pragma unroll
-      for (int m = 0; m < NV; ++m) {
+      for (int m0 = 0; m0 < NV; m0 += 4) {
+        // four passes' loads first: the operand stores below keep their program order with every later shared-memory load
+        float4 v4[4];
+#pragma unroll
+        for (int mm = 0; mm < 4; ++mm) {
+          const int e = tid + (m0 + mm) * cfg::NT;
+          const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
+          v4[mm] = *reinterpret_cast<const float4*>(sX + i * LD + j);
+        }
+#pragma unroll
+        for (int mm = 0; mm < 4; ++mm) {
+        const int m = m0 + mm;
         const int e = tid + m * cfg::NT;
         const int i = e / (C / 4), j = 4 * (e - i * (C / 4));
-        const float4 v = *reinterpret_cast<const float4*>(sX + i * LD + j);
+        const float4 v = v4[mm];
         if (a_dst && i < rows && TRI_INV_CHECK(p, (long long)tok0 + i < p.n_tokens && j + 4 <= C)) *reinterpret_cast<float4*>(a_dst + (size_t)m * a_step) = v;
         if (do_wy) put_ap(i, j, v);
+        }
+        const int m = m0 + 3;
         if (C == 128 && do_wy && (m == 3 || m == 7 || m == 11)) {
           fence_proxy_async();
           __syncthreads();   // rows 0 .. 8 m + 7 have been read by everyone
