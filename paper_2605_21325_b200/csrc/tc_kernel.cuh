@@ -718,6 +718,11 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
           ba *= sR[ra];
           bb *= sR[rbw];
         }
+        // g of every column this lane meets, before the first store to the matrix (a load behind such a store would wait for it:
+        // the compiler cannot tell the two apart)
+        float2 gcs[C / 8];
+#pragma unroll
+        for (int q = 0; q < C / 8; ++q) gcs[q] = *reinterpret_cast<const float2*>(sG + 8 * q + 2 * t);
 #pragma unroll
         for (int jb = 0; jb < cfg::NW; ++jb) {
           if (jb > rb) {
@@ -736,7 +741,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt) {
               const int c = 16 * jb + 8 * nt + 2 * t;
-              const float2 gc = *reinterpret_cast<const float2*>(sG + c);
+              const float2 gc = gcs[2 * jb + nt];
               const float2 rc = raw ? *reinterpret_cast<const float2*>(sR + c) : make_float2(1.f, 1.f);
               const float (&a4)[4] = sacc[2 * jb + nt];
               float2 va, vb;
