@@ -116,6 +116,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
   const uint32_t bar_mma = bar_k + 8;                    // a batch of MMAs completed
   const uint32_t bar_v = bar_k + 16;                     // V tile landed
   const uint32_t bar_exit = bar_k + 32;                  // give-up path only: every product issued so far has retired
+  const uint32_t bar_mma_u = bar_k + 48;                 // C = 128: the U product, committed right behind W (a barrier of its own:
+                                                         // two phases of one barrier must not complete before the first is seen)
   // Give-up protocol.  A thread whose bounded wait runs out remembers it ("bad"), skips its later waits, and
   // carries on with the item on whatever data is there (all indices come from the item number, never from
   // data).  It raises the CTA's flag in shared memory just before the barrier at the top of the next item;
@@ -218,6 +220,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
     }
     if (tid == 0) {
       mbar_init(bar_mma, 1);
+      mbar_init(bar_mma_u, 1);
       mbar_init(bar_exit, 1);
       fence_mbar_init();
     }
@@ -232,7 +235,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tmem_rows = tmem + (lane_base << 16);
-  uint32_t ph_k = 0, ph_v = 0, ph_mma = 0;  // parities of the next completion to wait for on each barrier
+  uint32_t ph_k = 0, ph_v = 0, ph_mma = 0, ph_u = 0;  // parities of the next completion to wait for on each barrier
 
   // Gram S = K K^T: D/16 MMAs of C x C x 16 into the first C columns of tensor memory (thread 0)
   auto issue_gram = [&]() {
@@ -795,12 +798,17 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         uint8_t* opb = opa + 16384;
         constexpr uint32_t idesc_m = umma_idesc_tf32(64, 64, 0);
         auto copy_block = [&](uint8_t* dst, int r0, int c0) {   // 64 x 64 block of the matrix, row-major -> operand layout
+          float4 v[4];   // loads first: a load behind a store to shared memory waits for it
 #pragma unroll
           for (int m = 0; m < 4; ++m) {
             const int e = tid + m * cfg::NT, i = e >> 4, k4 = (e & 15) * 4;
-            const float4 v = *reinterpret_cast<const float4*>(sX + (r0 + i) * LD + c0 + k4);
+            v[m] = *reinterpret_cast<const float4*>(sX + (r0 + i) * LD + c0 + k4);
+          }
+#pragma unroll
+          for (int m = 0; m < 4; ++m) {
+            const int e = tid + m * cfg::NT, i = e >> 4, k4 = (e & 15) * 4;
             uint4 w;
-            w.x = to_tf32(v.x); w.y = to_tf32(v.y); w.z = to_tf32(v.z); w.w = to_tf32(v.w);
+            w.x = to_tf32(v[m].x); w.y = to_tf32(v[m].y); w.z = to_tf32(v[m].z); w.w = to_tf32(v[m].w);
             *reinterpret_cast<uint4*>(dst + canon64(i, k4)) = w;
           }
         };
@@ -815,7 +823,6 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         const int mq = warp & 3, mh = warp >> 2;           // tensor-memory quadrant (16 rows of an M = 64 result) and column half
         const uint32_t tm_m = tmem + ((uint32_t)(32 * mq) << 16) + 32 * mh;
         // product 1: T = N21 . A11  (A = N21 as stored; B = A11^T: element (n, k) = A11[k][n])
-        copy_block(opa, 64, 0);
         {
           const int nn = lane & 7, kk = lane >> 3;         // an 8 (n) x 4 (k) patch per warp and step: conflict-free stores
           float av[16];
@@ -824,6 +831,7 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
             const int patch = warp * 16 + m;
             av[m] = sX[(4 * (patch >> 3) + kk) * LD + 8 * (patch & 7) + nn];
           }
+          copy_block(opa, 64, 0);   // (behind the loads above: its stores would hold them up)
 #pragma unroll
           for (int m = 0; m < 16; ++m) {
             const int patch = warp * 16 + m, n = 8 * (patch & 7) + nn, k = 4 * (patch >> 3) + kk;
@@ -841,8 +849,8 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         {
           float tf[4][4];
           tmem_ld_16x32(tf, tm_m);
+          copy_block(opa, 64, 64);   // while the tensor-memory load is in flight (product 1, the last reader of opa, has completed)
           tmem_wait_ld();
-          copy_block(opa, 64, 64);
           const int ka = 16 * mq + g, kb = ka + 8;
 #pragma unroll
           for (int nt = 0; nt < 4; ++nt) {
@@ -1008,22 +1016,24 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       if (has_next) bg_next = fetch_bg(nx_tok0, nx_rows, nx_h);  // consumed at the top of the next item
 
       // ---- 7. WY: [W | U] = A' . [K | V] with the staged tiles as the MN-major B operand
-      constexpr int NWU = (C == 64) ? D : 2 * D;   // columns per MMA: C = 64 runs W then U through the same D columns
+      // W and U are two products of D columns each: at C = 64 through the same columns (W leaves before U arrives), at C = 128
+      // side by side, U behind a commit of its own so that W is stored while U runs (and V's last box may still be on its way)
       static_assert(D == 128 || (D == 64 && C == 64), "head dimensions: 128, or 64 at C = 64");
-      constexpr uint32_t idesc_wy = umma_idesc(C, NWU, 1);
-      auto issue_wy = [&](uint32_t b_tile) {
+      constexpr uint32_t idesc_wy = umma_idesc(C, D, 1);
+      auto issue_wy = [&](uint32_t b_tile, uint32_t d_col = 0, bool second = false) {
 #pragma unroll
         for (int ks = 0; ks < C / 16; ++ks) {
           const uint64_t da = umma_desc(sAp + (ks >> 2) * (C * 128) + (ks & 3) * 32, 16, 1024);
           const uint64_t db = umma_desc(b_tile + ks * 2048, cfg::BOX_BYTES, 1024);
-          umma_bf16(tmem, da, db, idesc_wy, ks > 0);
+          umma_bf16(tmem + d_col, da, db, idesc_wy, ks > 0);
         }
-        umma_commit(bar_mma);
+        umma_commit(second ? bar_mma_u : bar_mma);
       };
       if (tid == 0) {
-        bool ok = wait(bar_k, ph_k);
-        if (C == 128 && need_v) ok = wait(bar_v, ph_v) && ok;
-        if (ok) { tc_fence_after(); issue_wy(sK); }
+        if (wait(bar_k, ph_k)) { tc_fence_after(); issue_wy(sK); }
+        if (C == 128 && need_v) {
+          if (wait(bar_v, ph_v)) { tc_fence_after(); issue_wy(sV, D, true); }
+        }
       }
       // A goes to global memory while the W product runs (its registers are free again before W returns)
       if (!cfg::ALIAS && a_dst) {
@@ -1079,15 +1089,30 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
         // second staging tile: the A' operand's space, whose last reader (the U product) has completed
         if constexpr (D == 128) store_frag_piece_bf16<1>(f1, sAp + warp * 2048, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
       } else {
-        // C = 128 (W and U side by side in 256 columns) or W only
-        if (cfg::ALIAS && tid == kTidK && has_next && !load_a) issue_k(nx_tok0, nx_h);  // all MMAs on the tiles are done
+        // C = 128 (W and U side by side in 256 columns, U behind its own commit) or W only
+        // With ALIAS the staging tiles lie in the A' region, which the U product is still reading: W is then staged in the
+        // K tile (its last reader, the W product, has completed), and the next K tile is requested once those stores
+        // have read it.
+        constexpr bool kSplit = cfg::ALIAS && C == 128;
+        const bool split = kSplit && need_v;
+        if (cfg::ALIAS && !split && tid == kTidK && has_next && !load_a) issue_k(nx_tok0, nx_h);  // all MMAs on the tiles are done
         // two staging tiles in turn where there is room for a second one (with ALIAS: the upper half of the A' region;
         // every product that reads A' has completed)
         const uint32_t stage2 = cfg::ALIAS ? stage + cfg::NW * 2048 : stage;
         constexpr int KEEP = cfg::ALIAS ? 1 : 0;
-        store_piece_bf16<0>(tmem_rows, stage, lane, w_row0, row_stride, rows - row0, &tmW, h * D, tok0 + row0);
-        if constexpr (D == 128) store_piece_bf16<KEEP>(tmem_rows + 64, stage2, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
+        const uint32_t stage_w = split ? sK + warp * 2048 : stage, stage_w2 = split ? sK + cfg::BOX_BYTES + warp * 2048 : stage2;
+        store_piece_bf16<0>(tmem_rows, stage_w, lane, w_row0, row_stride, rows - row0, &tmW, h * D, tok0 + row0);
+        if constexpr (D == 128) store_piece_bf16<KEEP>(tmem_rows + 64, stage_w2, lane, w_row0 + 64, row_stride, rows - row0, &tmW, h * D + 64, tok0 + row0);
         if (need_v && C == 128) {
+          wait(bar_mma_u, ph_u);   // the U product
+          ph_u ^= 1;
+          tc_fence_after();
+          if (split) {
+            if (lane == 0) bulk_wait_read();   // this warp's W stores have read their tiles in the K tile's space
+            tc_fence_before();
+            __syncthreads();
+            if (tid == kTidK && has_next && !load_a) issue_k(nx_tok0, nx_h);
+          }
           store_piece_bf16<KEEP>(tmem_rows + 128, stage, lane, u_row0, row_stride, rows - row0, &tmU, h * D, tok0 + row0);
           store_piece_bf16<KEEP>(tmem_rows + 192, stage2, lane, u_row0 + 64, row_stride, rows - row0, &tmU, h * D + 64, tok0 + row0);
         }
