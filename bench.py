@@ -63,7 +63,7 @@ def algorithmic_bytes_per_matrix(C, d_k, d_v, elt, want_A=True, call="fused"):
                (3 * C * d_k * elt + C * d_v * elt + C * 4 + C * d_v * elt)
     if call == "kda":  # K, G (fp32 per channel) and beta read; A written
         return C * d_k * elt + C * d_k * 4 + C * 4 + C * C * 4
-    if call == "kda_fused":  # what ONE kernel would move: K, G, V, beta read once; A, W, U written once (the call is two launches)
+    if call == "kda_fused":  # what ONE kernel would move: K, G, V, beta read once; A, W, U written once (one kernel at C = 64, two launches at C = 128)
         return C * d_k * elt + C * d_k * 4 + C * d_v * elt + C * 4 + C * C * 4 + C * d_k * elt + C * d_v * elt
     if call == "wy":
         return C * (C - 1) // 2 * 4 + C * d_k * elt + C * d_v * elt + C * 4 + C * d_k * elt + C * d_v * elt
@@ -447,7 +447,7 @@ def main():
         traffic = None if args.paper_T else ncu_traffic_bytes_per_matrix(args.call, args.config, args.method)
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": None if traffic is None else traffic * n_mat, "peak_source": "of " + peak_kind,
-                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "kda": "per-channel-decay build+invert", "kda_fused": "per-channel-decay build+invert (+ scaled keys), then WY (2 launches)", "wy": "WY apply", "scan": "chunk scan (state recurrence + output)", "layer": "fused build+invert+WY, then chunk scan (2 launches)", "kda_scan": "per-channel-decay chunk scan: operand preparation, then the scan (2 launches)", "kda_layer": "per-channel-decay build+invert, WY, operand preparation, chunk scan (4 launches)"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
+                    "kernel": {"fused": "fused build+invert+WY", "raw": "front end + build+invert+WY", "build": "build+invert", "kda": "per-channel-decay build+invert", "kda_fused": "per-channel-decay build+invert+WY (one kernel)" if inp.C == 64 else "per-channel-decay build+invert (+ scaled keys), then WY (2 launches)", "wy": "WY apply", "scan": "chunk scan (state recurrence + output)", "layer": "fused build+invert+WY, then chunk scan (2 launches)", "kda_scan": "per-channel-decay chunk scan: operand preparation, then the scan (2 launches)", "kda_layer": "per-channel-decay build+invert+WY, operand preparation, chunk scan (3 launches)"}[args.call], "kernel_ms": kernel_ms, "kernel_ms_min": min(times_ms),
                     "algorithmic_bytes_per_launch": alg_bytes * n_mat}
         cpu = None
         if world == 1 and not args.no_cpu_baseline:

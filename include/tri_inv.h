@@ -210,11 +210,15 @@ int tri_inv_fused_host(const void* K, const void* V, const float* beta, const fl
  *     A = (I + N)^{-1},  N as for tri_inv_build_kda;     W = A diag(beta) (K * Gamma),  Gamma = exp(G);     U = A diag(beta) V
  * (the recurrence S_t = (I - beta_t k_t k_t^T) diag(alpha_t) S_{t-1} + beta_t k_t v_t^T re-bracketed per chunk gives
  * (I + N) U~ = diag(beta) V - diag(beta) (K * Gamma) S, i.e. U~ = U - W S; tri_inv_chunk_scan_kda consumes W and U).
- *   K, V, W, U [B,T,H,d] kv_dtype;  G [B,T,H,d_k] fp32;  beta [B,T,H] fp32;  A [B,T,H,C] fp32 -- all required (A is also the
- *   hand-over between the launches).  W may not alias K.
- * bf16 with d_k = d_v = 128, C = 64 and the block recursion runs on the tensor cores as two launches on the stream
- * (tri_inv_build_kda's kernel, which also writes K * Gamma into the W buffer while it holds K and G on chip; then
- * tri_inv_wy's kernel on that buffer, in place); everything else is one launch of the CUDA-core kernel.  TRI_INV_GATE_SHIFTED and TRI_INV_W_DECAY do not apply (W is always the decay-weighted one).
+ *   K, V, W, U [B,T,H,d] kv_dtype;  G [B,T,H,d_k] fp32;  beta [B,T,H] fp32;  A [B,T,H,C] fp32 -- all required (at C = 128
+ *   A is also the hand-over between two launches).  W may not alias K; G as for tri_inv_build_kda (and exp(G_ref) must be
+ *   representable: G is a cumulative log-decay, at most 0).
+ * bf16 with d_k = d_v = 128 and the block recursion runs on the tensor cores: at C = 64 as ONE kernel (build, inversion and
+ * both factors; W is formed as (A diag(beta) (K * exp(G - G_ref))) diag(exp G_ref), G_ref the chunk's middle row, so no
+ * factor leaves exp(+-|G over 32 tokens|)), at C = 128 as two launches on the stream (tri_inv_build_kda's kernel, which
+ * also writes K * Gamma into the W buffer while it holds K and G on chip; then tri_inv_wy's kernel on that buffer, in
+ * place); everything else is one launch of the CUDA-core kernel.  TRI_INV_GATE_SHIFTED and TRI_INV_W_DECAY do not apply
+ * (W is always the decay-weighted one).
  */
 int tri_inv_fused_kda(const void* K, const void* V, const float* G, const float* beta,
                       float* A, void* W, void* U, const tri_inv_desc* desc, int method, void* cuda_stream);

@@ -343,18 +343,32 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
     };
     // raw front end: the K tile in shared memory becomes the normalised keys (row i times 1 / |k_i|, bf16 in place)
     auto rescale_k_tile = [&]() {
-      for (int e = tid; e < C * 8 * cfg::NBOX; e += cfg::NT) {
-        const int bx = e / (C * 8), rem = e - bx * (C * 8), r = rem >> 3, c = rem & 7;
-        uint4* ptr = reinterpret_cast<uint4*>(smem + cfg::OFF_K + bx * cfg::BOX_BYTES + r * 128 + c * 16);
-        uint4 v = *ptr;
-        const float sc = wdecay ? sR[r] * ((gshift && r == 0) ? 1.f : ex2_approx(sG[r - gshift])) : sR[r];
-        uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+      constexpr int PER = C * 8 * cfg::NBOX / cfg::NT;   // 16-byte pieces per thread
+      static_assert(PER % 4 == 0 && PER * cfg::NT == C * 8 * cfg::NBOX, "four pieces at a time");
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float2 f = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[q]));
-          w[q] = pack_bf16(f.x * sc, f.y * sc);
+      for (int m0 = 0; m0 < PER; m0 += 4) {
+        // four pieces' loads first: a load behind a store to the tile would wait for it
+        uint4 v[4];
+        float sc[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          const int e = tid + (m0 + m) * cfg::NT;
+          const int bx = e / (C * 8), rem = e - bx * (C * 8), r = rem >> 3, c = rem & 7;
+          v[m] = *reinterpret_cast<const uint4*>(smem + cfg::OFF_K + bx * cfg::BOX_BYTES + r * 128 + c * 16);
+          sc[m] = wdecay ? sR[r] * ((gshift && r == 0) ? 1.f : ex2_approx(sG[r - gshift])) : sR[r];
         }
-        *ptr = v;
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          const int e = tid + (m0 + m) * cfg::NT;
+          const int bx = e / (C * 8), rem = e - bx * (C * 8), r = rem >> 3, c = rem & 7;
+          uint32_t* w = reinterpret_cast<uint32_t*>(&v[m]);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float2 f = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&w[q]));
+            w[q] = pack_bf16(f.x * sc[m], f.y * sc[m]);
+          }
+          *reinterpret_cast<uint4*>(smem + cfg::OFF_K + bx * cfg::BOX_BYTES + r * 128 + c * 16) = v[m];
+        }
       }
     };
     // after K (and V) were requested again for the WY step: padding rows cleared, keys normalised
