@@ -340,6 +340,21 @@ int tri_inv_selftest_scan_wait_timeout(const void* Q, const void* K, const void*
                                        const tri_inv_desc* desc, uint64_t wait_limit_ns, void* cuda_stream);
 
 /*
+ * The same for the per-channel kernels (bf16, d_k = d_v = 128, C = 64 or 128, block recursion; no step of the paper's
+ * method): tri_inv_fused_kda -- or, with V, W and U all NULL, tri_inv_build_kda -- with every device-side wait limited to
+ * wait_limit_ns nanoseconds and with the first thread block leaving out the Gram product of its first chunk matrix (chunk
+ * 0, head 0).  That block's waits run out, it raises the status word, finishes the one matrix on undefined data (its rows
+ * of A, W, U are then undefined), waits -- bounded -- for the copies it still has in flight, frees its tensor memory and
+ * returns without taking further work: these kernels hand out work with a fixed stride, so with more matrices than
+ * resident thread blocks (three per SM at C = 64, two at C = 128) the block's later matrices stay unwritten as well.  All
+ * other blocks finish as usual.  The call synchronises the stream; afterwards tri_inv_last_device_status() reads
+ * TRI_INV_ERR_DEVICE_TIMEOUT (once), and the library is usable as before.
+ */
+int tri_inv_selftest_kda_wait_timeout(const void* K, const void* V, const float* G, const float* beta,
+                                      float* A, void* W, void* U, const tri_inv_desc* desc,
+                                      uint64_t wait_limit_ns, void* cuda_stream);
+
+/*
  * Self-test of the bounds-checking build (no step of the paper's method).  tri_inv_fused (block recursion) with the token
  * bound that the debug build's checks use understated by one chunk: the buffers are as large as the descriptor says, so
  * no access is out of range either way.  In the bounds-checking build (libtri_inv_debug.so) the work items of the last

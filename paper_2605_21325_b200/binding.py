@@ -39,7 +39,7 @@ FORCE_SIMT = 0x10000
 W_DECAY = 0x20000
 
 EXPORTS = ("tri_inv_build", "tri_inv_build_kda", "tri_inv_fused_kda", "tri_inv_chunk_scan_kda", "tri_inv_chunk_scan", "tri_inv_wy", "tri_inv_fused", "tri_inv_fused_raw", "tri_inv_fused_packed_static", "tri_inv_count_matrices",
-           "tri_inv_fused_host", "tri_inv_fused_host_workspace", "tri_inv_selftest_wait_timeout", "tri_inv_selftest_scan_wait_timeout", "tri_inv_selftest_bounds_check", "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
+           "tri_inv_fused_host", "tri_inv_fused_host_workspace", "tri_inv_selftest_wait_timeout", "tri_inv_selftest_scan_wait_timeout", "tri_inv_selftest_kda_wait_timeout", "tri_inv_selftest_bounds_check", "tri_inv_last_device_status", "tri_inv_launch_count", "tri_inv_status_string")
 
 
 class Desc(ctypes.Structure):
@@ -94,6 +94,9 @@ def load():
         if hasattr(lib, "tri_inv_selftest_scan_wait_timeout"):
             lib.tri_inv_selftest_scan_wait_timeout.argtypes = [vp, vp, vp, vp, vp, vp, dp, ctypes.c_uint64, vp]
             lib.tri_inv_selftest_scan_wait_timeout.restype = i32
+        if hasattr(lib, "tri_inv_selftest_kda_wait_timeout"):
+            lib.tri_inv_selftest_kda_wait_timeout.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, ctypes.c_uint64, vp]
+            lib.tri_inv_selftest_kda_wait_timeout.restype = i32
         if hasattr(lib, "tri_inv_selftest_wait_timeout"):
             lib.tri_inv_selftest_wait_timeout.argtypes = [vp, vp, vp, vp, vp, vp, vp, dp, ctypes.c_uint64, ctypes.POINTER(ctypes.c_int), vp]
             lib.tri_inv_selftest_wait_timeout.restype = i32
@@ -319,6 +322,21 @@ def selftest_wait_timeout(K, V, beta, g, C, wait_limit_ns, out, stream=None):
     if rc != OK:
         raise TriInvError("tri_inv_selftest_wait_timeout", rc)
     return bool(idle.value)
+
+
+def selftest_kda_wait_timeout(K, V, G, beta, C, wait_limit_ns, out, stream=None):
+    """tri_inv_selftest_kda_wait_timeout: the per-channel fused call (``V`` None: the per-channel build) with short wait limits
+    and one product of the first thread block left out.  ``out`` = (A, W, U) or (A, None, None)."""
+    B, T, H, d_k = K.shape
+    desc, keep = make_desc(B, T, H, d_k, d_k if V is None else V.shape[-1], C, _dtype_code(K), None)
+    A, W, U = out
+    none = ctypes.c_void_p(None)
+    rc = load().tri_inv_selftest_kda_wait_timeout(_p(K), none if V is None else _p(V), _p(G), _p(beta), _p(A),
+                                                  none if W is None else _p(W), none if U is None else _p(U), ctypes.byref(desc),
+                                                  ctypes.c_uint64(int(wait_limit_ns)), _stream(stream))
+    if rc != OK:
+        raise TriInvError("tri_inv_selftest_kda_wait_timeout", rc)
+    return out
 
 
 def selftest_scan_wait_timeout(Q, K, W, U, g, C, wait_limit_ns, out, stream=None):

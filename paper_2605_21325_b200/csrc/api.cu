@@ -415,6 +415,37 @@ int tri_inv_selftest_wait_timeout(const void* K, const void* V, const float* bet
   return TRI_INV_OK;
 }
 
+int tri_inv_selftest_kda_wait_timeout(const void* K, const void* V, const float* G, const float* beta,
+                                      float* A, void* W, void* U, const tri_inv_desc* desc,
+                                      uint64_t wait_limit_ns, void* cuda_stream) {
+  int rc = check_desc(desc, true);
+  if (rc) return rc;
+  if (!K || !G || !beta || !A || wait_limit_ns == 0) return TRI_INV_ERR_INVALID_ARG;
+  const bool wy = V || W || U;
+  if (wy && (!V || !W || !U)) return TRI_INV_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(G) || !aligned16(beta) || !aligned16(A) || (wy && (!aligned16(V) || !aligned16(W) || !aligned16(U))))
+    return TRI_INV_ERR_INVALID_ARG;
+  // only the tensor-core kernels have the stall hook
+  if (desc->kv_dtype != TRI_INV_BF16 || desc->d_k != 128 || desc->d_v != 128 || (desc->C != 64 && desc->C != 128))
+    return TRI_INV_ERR_UNSUPPORTED;
+  KParams p{};
+  p.K = K; p.G = G; p.beta = beta; p.g = nullptr; p.A = A;
+  p.method = TRI_INV_BLOCK_RECURSIVE;
+  p.wait_limit_ns = wait_limit_ns;
+  if (wy && desc->C == 64) {          // the one-kernel form
+    p.V = V; p.W = W; p.U = U;
+    p.ops = kStoreA | kDoWY | kKda | kTestStall;
+    rc = run(p, desc, cuda_stream);
+  } else {                            // the build kernel (C = 128 with W, U: its instance that also writes K exp(G), then the WY kernel)
+    p.W = wy ? W : nullptr;
+    p.ops = kStoreA | kKda | kTestStall;
+    rc = run(p, desc, cuda_stream);
+    if (!rc && wy) rc = tri_inv_wy(A, W, V, beta, W, U, desc, cuda_stream);
+  }
+  if (rc) return rc;
+  return cudaStreamSynchronize((cudaStream_t)cuda_stream) == cudaSuccess ? TRI_INV_OK : TRI_INV_ERR_CUDA;
+}
+
 int tri_inv_selftest_bounds_check(const void* K, const void* V, const float* beta, const float* g,
                                   float* A, void* W, void* U, const tri_inv_desc* desc, void* cuda_stream) {
   int rc = check_desc(desc, true);

@@ -116,3 +116,43 @@ def test_scan_waits_that_run_out(bnd, B, H):
     torch.cuda.synchronize()
     assert bnd.last_device_status() == 0
     assert torch.equal(again.view(torch.int16), ref.view(torch.int16))
+
+
+@pytest.mark.parametrize("C,with_wy", [(64, True), (64, False), (128, True)], ids=["C64_one_kernel", "C64_build", "C128_two_launches"])
+def test_per_channel_waits_that_run_out(bnd, C, with_wy):
+    """The per-channel kernels' give-up path (tri_inv_selftest_kda_wait_timeout, limit 50 us): the first thread block leaves out
+    the Gram product of its first matrix, its waits run out, it raises the status word, drains what it has in flight, frees
+    its tensor memory and returns.  256 matrices, fewer than resident thread blocks, so every other matrix must come out
+    bit for bit as in an ordinary call; the status word reads DEVICE_TIMEOUT once; the next ordinary call is exact."""
+    inp = wl.make("kda_timeout", 2, 16 * C, 8, 128, 128, C, wl.BF16, seed=612)
+    dev = bnd.to_device(inp)
+    Gd = torch.from_numpy(wl.per_channel_gate(inp, seed=613)).cuda()
+
+    def call(selftest):
+        A = torch.full((inp.B, inp.T, inp.H, C), float("nan"), dtype=torch.float32, device="cuda")
+        W, U = (torch.full_like(dev["K"], float("nan")), torch.full_like(dev["V"], float("nan"))) if with_wy else (None, None)
+        if selftest:
+            bnd.selftest_kda_wait_timeout(dev["K"], dev["V"] if with_wy else None, Gd, dev["beta"], C, wait_limit_ns=50_000, out=(A, W, U))
+        elif with_wy:
+            bnd.fused_kda(dev["K"], dev["V"], Gd, dev["beta"], C, out=(A, W, U))
+        else:
+            bnd.build_kda(dev["K"], Gd, dev["beta"], C, out=A)
+        torch.cuda.synchronize()
+        return [t for t in (A, W, U) if t is not None]
+
+    ref = call(False)
+    assert bnd.last_device_status() == 0
+    out = call(True)
+    assert bnd.last_device_status() == bnd.ERR_DEVICE_TIMEOUT     # raised ...
+    assert bnd.last_device_status() == 0                          # ... and cleared by the read
+    for r, o in zip(ref, out):
+        r2, o2 = r.clone(), o.clone()
+        r2[0, :C, 0] = 0
+        o2[0, :C, 0] = 0
+        assert torch.equal(r2.view(torch.int32 if r.dtype == torch.float32 else torch.int16),
+                           o2.view(torch.int32 if o.dtype == torch.float32 else torch.int16))
+    again = call(False)
+    assert bnd.last_device_status() == 0
+    for r, o in zip(ref, again):
+        assert torch.equal(r.view(torch.int32 if r.dtype == torch.float32 else torch.int16),
+                           o.view(torch.int32 if o.dtype == torch.float32 else torch.int16))
