@@ -49,6 +49,7 @@ struct KParams {
   int32_t method;               // TRI_INV_* method with flags
   int32_t ops;                  // kStoreA | kDoWY | kLoadA | ...
   unsigned long long wait_limit_ns;  // per bounded device-side wait (run() fills in the default of two seconds)
+  int32_t a_box;                // build-only tensor-core kernel: 1 when the W tensor-map slot carries the 3-D map of A (whole-matrix store)
   long long n_tokens;           // flat tokens of the tensors (B * T, or T when packed): the bound the debug build checks rows against
 };
 

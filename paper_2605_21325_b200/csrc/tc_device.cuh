@@ -79,6 +79,9 @@ __device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* tm, int x,
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm), "r"(src), "r"(x), "r"(y) : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(tm), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // every bulk store this thread has committed has finished READING its shared-memory source
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
@@ -586,6 +589,22 @@ inline EncodeTiledFn encode_fn() {
 
 // 2-D view of a [tokens, H*d] tensor of bf16 (elt = 2) or fp32 (elt = 4); one box = 128 bytes of features
 // (64 bf16 or 32 fp32, swizzled) x C tokens.
+// 3-D view of A [tokens, H, C] fp32 for the store of one whole chunk matrix straight from its padded rows in shared memory:
+// one box = C tokens x one head x LD floats (LD >= C, the row length in shared memory, a multiple of 4), no swizzle.  The
+// box is wider than the tensor's innermost extent; the columns past C fall outside the tensor and are not written.
+inline bool make_tmap_a(CUtensorMap* tm, const float* base, long long tokens, int H, int C, int LD) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)H, (cuuint64_t)tokens};
+  cuuint64_t strides[2] = {(cuuint64_t)C * 4, (cuuint64_t)H * C * 4};
+  cuuint32_t box[3] = {(cuuint32_t)LD, 1, (cuuint32_t)C};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 inline bool make_tmap(CUtensorMap* tm, const void* base, long long tokens, int H, int d, int C, int elt = 2) {   // C = tokens per box
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;

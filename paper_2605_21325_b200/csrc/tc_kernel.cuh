@@ -979,7 +979,14 @@ __global__ void __launch_bounds__(Cfg<C, D, SER, BO, REF, H16>::NT, Cfg<C, D, SE
       // shared memory: +0.0 above the diagonal, 1.0f on it.  Rows past the sequence end are not copied.
       fence_proxy_async();   // the merges' stores become visible to the copy engine
       __syncthreads();
-      if ((p.ops & kStoreA) && p.A && tid < rows && TRI_INV_CHECK(p, (long long)tok0 + tid < p.n_tokens)) {
+      if ((p.ops & kStoreA) && p.A && rows == C && p.a_box) {
+        // a whole chunk: ONE tiled bulk store of C tokens x LD floats (tmW is the 3-D map of A here; the LD - C padding
+        // columns fall outside the tensor's innermost extent and are dropped) instead of C row copies
+        if (tid == 0 && TRI_INV_CHECK(p, (long long)tok0 + C <= p.n_tokens)) {
+          tma_store_3d(&tmW, smem_u32(sX), 0, h, tok0);
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+      } else if ((p.ops & kStoreA) && p.A && tid < rows && TRI_INV_CHECK(p, (long long)tok0 + tid < p.n_tokens)) {
         float* dst = p.A + ((size_t)(tok0 + tid) * p.H + h) * C;
         asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(sX + tid * LD)), "r"(C * 4) : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -1226,7 +1233,12 @@ cudaError_t launch_one(const KParams& p_in, cudaStream_t stream) {
   else tmV = tmK;
   // W and U leave in boxes of 64 columns x 16 tokens (one warp's piece)
   CUtensorMap tmW = tmK, tmU = tmK;
-  if (p.W && !make_tmap(&tmW, p.W, tokens, p.H, D, 16)) return cudaErrorUnknown;
+  if constexpr (BO) {
+    // build only: the W slot carries the map of A for the whole-matrix store (if the driver refuses the map, rows go one by one)
+    p.a_box = (p.A && (p.ops & kStoreA) && make_tmap_a(&tmW, p.A, tokens, p.H, C, C + 4)) ? 1 : 0;
+    if (!p.a_box) tmW = tmK;
+  }
+  if (!BO && p.W && !make_tmap(&tmW, p.W, tokens, p.H, D, 16)) return cudaErrorUnknown;
   if (p.U && !make_tmap(&tmU, p.U, tokens, p.H, D, 16)) return cudaErrorUnknown;
   long long total = (long long)p.n_chunks * p.H;
   long long cap = (long long)n_sm * ctas_per_sm;
