@@ -42,7 +42,8 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
                                                                      const __grid_constant__ CUtensorMap tmG,
                                                                      const __grid_constant__ CUtensorMap tmV,
                                                                      const __grid_constant__ CUtensorMap tmW,
-                                                                     const __grid_constant__ CUtensorMap tmU, KParams p) {
+                                                                     const __grid_constant__ CUtensorMap tmU,
+                                                                     const __grid_constant__ CUtensorMap tmA, KParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
   float* sX = reinterpret_cast<float*>(smem + OFF_X);
   float* sBeta = reinterpret_cast<float*>(smem + OFF_BETA);
@@ -262,9 +263,21 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
 
     // ---- 5. one pass over the finished matrix (zeros above the diagonal, ones on it): A to global memory, A' = A diag(beta)
     //         as the bf16 K-major swizzled operand of the two products
+    // A whole chunk's A leaves as ONE tiled bulk store straight from the matrix (3-D map of A, box of 64 tokens x LD floats:
+    // the padding columns fall outside the tensor and are dropped); the thread that requests the next G tile issues it and
+    // waits, before that request, until the copy engine has read the matrix.
+    const bool a_tma = p.A && rows == C && p.a_box;
+    if (a_tma) {
+      fence_proxy_async();   // the merges' stores become visible to the copy engine
+      __syncthreads();
+      if (tid == kTidG) {
+        tma_store_3d(&tmA, smem_u32(sX), 0, h, tok0);
+        bulk_commit();
+      }
+    }
     {
       const size_t a_step = (size_t)(NT / (C / 4)) * p.H * C;
-      float* a_dst = p.A ? p.A + ((size_t)(tok0 + tid / (C / 4)) * p.H + h) * C + 4 * (tid % (C / 4)) : nullptr;
+      float* a_dst = (p.A && !a_tma) ? p.A + ((size_t)(tok0 + tid / (C / 4)) * p.H + h) * C + 4 * (tid % (C / 4)) : nullptr;
 #pragma unroll
       for (int m = 0; m < C / 8; ++m) {
         const int e = tid + m * NT;
@@ -288,7 +301,10 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_fused_kernel(const __grid
     fence_proxy_async();   // generic-proxy writes of A' (and V's cleared rows) become visible to the tensor core's reads
     tc_fence_before();
     __syncthreads();       // the fp32 matrix has been read by everyone: the next G tile may land in its space
-    if (tid == kTidG && has_next && !bad) issue_g(nx_tok0, nx_h);
+    if (tid == kTidG) {
+      if (a_tma) bulk_wait_read();
+      if (has_next && !bad) issue_g(nx_tok0, nx_h);
+    }
     PHASE(6);
 
     // ---- 6. W = (A' K+) diag(exp G_ref), U = A' V: the tiles are the MN-major B operand, 16 tokens per k-step
@@ -392,15 +408,18 @@ cudaError_t launch_kda_fused_tc(const KParams& p, cudaStream_t stream) {
     ctas = ctas_of[dev];
   }
   const long long tokens = p.chunk_tab ? (long long)p.T : (long long)p.T * (p.n_chunks / p.chunks_per_seq);
-  CUtensorMap tmK, tmG, tmV, tmW, tmU;
+  CUtensorMap tmK, tmG, tmV, tmW, tmU, tmA;
   if (!make_tmap(&tmK, p.K, tokens, p.H, D, C, 2)) return cudaErrorUnknown;
   if (!make_tmap(&tmG, p.G, tokens, p.H, D, C, 4)) return cudaErrorUnknown;
   if (!make_tmap(&tmV, p.V, tokens, p.H, D, C, 2)) return cudaErrorUnknown;
   if (!make_tmap(&tmW, p.W, tokens, p.H, D, 16, 2)) return cudaErrorUnknown;
   if (!make_tmap(&tmU, p.U, tokens, p.H, D, 16, 2)) return cudaErrorUnknown;
+  KParams q = p;
+  q.a_box = (p.A && make_tmap_a(&tmA, p.A, tokens, p.H, C, LD)) ? 1 : 0;   // refused: A leaves through ordinary stores
+  if (!q.a_box) tmA = tmK;
   const long long total = (long long)p.n_chunks * p.H, cap = (long long)n_sm * ctas;
   const int grid = (int)(total < cap ? total : cap);
-  kda_fused_kernel<<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, tmV, tmW, tmU, p);
+  kda_fused_kernel<<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, tmV, tmW, tmU, tmA, q);
   return cudaGetLastError();
 }
 

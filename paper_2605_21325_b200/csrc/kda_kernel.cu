@@ -32,7 +32,8 @@ constexpr int CTAS_PER_SM = 3;
 static_assert(OFF_LEAF + NW * 16 * LEAF_LD * 4 <= OFF_BETA, "leaf scratch must fit behind the fp32 matrix");
 
 __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid_constant__ CUtensorMap tmK,
-                                                                     const __grid_constant__ CUtensorMap tmG, KParams p) {
+                                                                     const __grid_constant__ CUtensorMap tmG,
+                                                                 const __grid_constant__ CUtensorMap tmA, KParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
   float* sX = reinterpret_cast<float*>(smem + OFF_X);
   float* sBeta = reinterpret_cast<float*>(smem + OFF_BETA);
@@ -217,7 +218,18 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) kda_build_kernel(const __grid
     merge_level<C, 32>(sX, warp, lane);
 
     // ---- 5. store A (the matrix in shared memory is complete: zeros above the diagonal, ones on it)
-    if (p.A) {
+    if (p.A && rows == C && p.a_box) {
+      // a whole chunk: ONE tiled bulk store of 64 tokens x LD floats straight from the matrix (3-D map of A; the padding
+      // columns fall outside the tensor and are dropped).  The thread that requests the next G tile issues it and waits
+      // until the copy engine has read the matrix, whose space that tile lands in.
+      fence_proxy_async();   // the merges' stores become visible to the copy engine
+      __syncthreads();
+      if (tid == 96) {
+        tma_store_3d(&tmA, smem_u32(sX), 0, h, tok0);
+        bulk_commit();
+        bulk_wait_read();
+      }
+    } else if (p.A) {
       const size_t a_step = (size_t)(NT / (C / 4)) * p.H * C;
       float* a_dst = p.A + ((size_t)(tok0 + tid / (C / 4)) * p.H + h) * C + 4 * (tid % (C / 4));
 #pragma unroll
@@ -285,12 +297,15 @@ cudaError_t launch_kda_tc(const KParams& p, int Cc, cudaStream_t stream, bool* h
     ctas = ctas_of[dev];
   }
   long long tokens = p.chunk_tab ? (long long)p.T : (long long)p.T * (p.n_chunks / p.chunks_per_seq);
-  CUtensorMap tmK, tmG;
+  CUtensorMap tmK, tmG, tmA;
   if (!make_tmap(&tmK, p.K, tokens, p.H, D, C, 2)) return cudaErrorUnknown;
   if (!make_tmap(&tmG, p.G, tokens, p.H, D, C, 4)) return cudaErrorUnknown;
+  KParams q = p;
+  q.a_box = (p.A && make_tmap_a(&tmA, p.A, tokens, p.H, C, LD)) ? 1 : 0;   // refused: A leaves through ordinary stores
+  if (!q.a_box) tmA = tmK;
   long long total = (long long)p.n_chunks * p.H, cap = (long long)n_sm * ctas;
   int grid = (int)(total < cap ? total : cap);
-  kda_build_kernel<<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
+  kda_build_kernel<<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, tmA, q);
   return cudaGetLastError();
 }
 

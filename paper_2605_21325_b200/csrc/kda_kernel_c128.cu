@@ -41,7 +41,8 @@ static_assert(2 * (SMEM_BYTES + 1024 + 8) <= 228 * 1024, "two CTAs per SM");
 
 template <bool KG>   // KG: also write K * exp(G) into p.W (the fused call)
 __global__ void __launch_bounds__(NT, 2) kda_build_kernel_c128(const __grid_constant__ CUtensorMap tmK,
-                                                               const __grid_constant__ CUtensorMap tmG, KParams p) {
+                                                               const __grid_constant__ CUtensorMap tmG,
+                                                               const __grid_constant__ CUtensorMap tmA, KParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
   float* sX = reinterpret_cast<float*>(smem + OFF_X);
   float* sBeta = reinterpret_cast<float*>(smem + OFF_BETA);
@@ -269,7 +270,18 @@ __global__ void __launch_bounds__(NT, 2) kda_build_kernel_c128(const __grid_cons
     merge_level<C, 64>(sX, warp, lane);
 
     // ---- 5. store A (the matrix in shared memory is complete: zeros above the diagonal, ones on it)
-    if (p.A) {
+    if (p.A && rows == C && p.a_box) {
+      // a whole chunk: ONE tiled bulk store of 128 tokens x LD floats straight from the matrix (3-D map of A; the padding
+      // columns fall outside the tensor and are dropped).  The thread that requests the next G boxes issues it and waits
+      // until the copy engine has read the matrix, whose space those boxes land in.
+      fence_proxy_async();   // the merges' stores become visible to the copy engine
+      __syncthreads();
+      if (tid == 96) {
+        tma_store_3d(&tmA, smem_u32(sX), 0, h, tok0);
+        bulk_commit();
+        bulk_wait_read();
+      }
+    } else if (p.A) {
       const size_t a_step = (size_t)(NT / (C / 4)) * p.H * C;
       float* a_dst = p.A + ((size_t)(tok0 + tid / (C / 4)) * p.H + h) * C + 4 * (tid % (C / 4));
 #pragma unroll 4
@@ -322,15 +334,18 @@ cudaError_t launch_kda_tc_c128(const KParams& p, cudaStream_t stream) {
     n_sm = n_sm_of[dev];
   }
   long long tokens = p.chunk_tab ? (long long)p.T : (long long)p.T * (p.n_chunks / p.chunks_per_seq);
-  CUtensorMap tmK, tmG;
+  CUtensorMap tmK, tmG, tmA;
   if (!make_tmap(&tmK, p.K, tokens, p.H, D, C, 2)) return cudaErrorUnknown;
   if (!make_tmap(&tmG, p.G, tokens, p.H, D, C, 4)) return cudaErrorUnknown;
+  KParams q = p;
+  q.a_box = (p.A && make_tmap_a(&tmA, p.A, tokens, p.H, C, LD)) ? 1 : 0;   // refused: A leaves through ordinary stores
+  if (!q.a_box) tmA = tmK;
   long long total = (long long)p.n_chunks * p.H;
   const long long cap = 2LL * n_sm;   // two CTAs per SM
   int grid = (int)(total < cap ? total : cap);
   if (grid == 0) return cudaSuccess;
-  if (p.W) kda_build_kernel_c128<true><<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
-  else kda_build_kernel_c128<false><<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, p);
+  if (p.W) kda_build_kernel_c128<true><<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, tmA, q);
+  else kda_build_kernel_c128<false><<<grid, NT, SMEM_BYTES, stream>>>(tmK, tmG, tmA, q);
   return cudaGetLastError();
 }
 
