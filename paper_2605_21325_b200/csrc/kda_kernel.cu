@@ -8,8 +8,11 @@
 //      K- = K * exp(G_ref - G), with G_ref the row in the middle of the chunk, so that each factor stays
 //      within exp(+-|G_0 - G_mid|); their product carries exp(G_i - G_j) per channel.
 //   3. S = K+ (K-)^T as tcgen05.mma (kind::f16, fp32 accumulator in tensor memory).
-//   4. Gate (beta_i, strict-lower mask), block recursion from 16x16 leaves and the store of A exactly as in
-//      the scalar-gate kernel; the fp32 matrix reuses the G tile's space.
+//   4. Gate (beta_i, strict-lower mask) and block recursion from 16x16 leaves exactly as in the scalar-gate
+//      kernel; the fp32 matrix reuses the G tile's space.  A whole chunk's A leaves as one tiled bulk store
+//      straight from that matrix (a 3-D map of A whose box is as wide as the padded rows in shared memory:
+//      the padding columns fall outside the tensor and are dropped); a chunk cut short by its sequence's end
+//      takes 16-byte stores.
 // Every mbarrier wait is bounded; on expiry the kernel raises the status word, frees its tensor memory
 // and returns.
 #include "tc_device.cuh"

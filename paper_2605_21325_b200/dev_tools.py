@@ -28,10 +28,12 @@ def main():
     import torch
     from paper_2605_21325_b200 import binding as b, workloads as wl
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["phases", "build_phases", "timeline", "scan_chunk", "kda_phases"])
+    ap.add_argument("what", choices=["phases", "build_phases", "raw_phases", "timeline", "scan_chunk", "kda_phases"])
     ap.add_argument("--config", type=int, default=2)
     args = ap.parse_args()
     inp = wl.config(args.config)
+    if args.what == "raw_phases":   # the same shape with the inputs the projections hand over (un-normalised keys, logits)
+        inp = wl.make_raw(inp.name + "_raw", inp.B, inp.T, inp.H, inp.d_k, inp.C, inp.kv_dtype, 2000 + args.config, inp.cu_seqlens)
     d = b.to_device(inp)
     if args.what == "scan_chunk":
         return scan_chunk(b, wl, inp, d)
@@ -47,7 +49,9 @@ def main():
         flush.fill_(1)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        if args.what == "build_phases":
+        if args.what == "raw_phases":
+            b.fused_raw(d["K"], d["V"], d["beta"], d["g"], inp.C, cu_seqlens=inp.cu_seqlens, out=(out[0], out[1], out[2], None, None))
+        elif args.what == "build_phases":
             b.build(d["K"], d["beta"], d["g"], inp.C, cu_seqlens=inp.cu_seqlens, out=out[0])
         else:
             b.fused(d["K"], d["V"], d["beta"], d["g"], inp.C, cu_seqlens=inp.cu_seqlens, out=out)
@@ -56,7 +60,7 @@ def main():
         L.tri_inv_debug_counters(words)          # read and clear: the last launch's counters stay in `words`
     resident = 148 * ((6 if args.what == "build_phases" else 4) if inp.C == 64 else 2)
     grid = min(int(os.environ.get("TRI_INV_GRID_CAP", resident)), resident, inp.n_matrices)
-    if args.what in ("phases", "build_phases"):
+    if args.what in ("phases", "build_phases", "raw_phases"):
         items = -(-inp.n_matrices // grid)      # items of CTA 0, about
         for w in range(inp.C // 16):
             v = [words[8 + 12 * w + k] / items for k in range(12)]
